@@ -1,0 +1,402 @@
+/*
+ * firp_oracle.c -- TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, single-purpose CPU statement of what one FIRP draft+verify
+ * decoder step computes, written from the paper (arXiv 2410.20488) so that the
+ * CUDA path can be compared against it.  Nothing in the product may call it:
+ * only tests, the smoke check and the benchmark's CPU-baseline leg do.  It
+ * shares no code with the CUDA path.
+ *
+ * Precision: activations, KV cache and logits are stored as fp32; every
+ * reduction (dot products, RMS, softmax, weighted sums) is accumulated in
+ * fp64; weights are bf16 bit patterns widened exactly to fp32.  There is no
+ * blocking, fusion or reordering: each function is the formula written out.
+ *
+ * What is computed, with the passage each part follows:
+ *   - Llama-style decoder block (the paper builds on the HuggingFace Llama
+ *     architecture, Section 4 "Setup"): RMSNorm, q/k/v projections, rotary
+ *     embedding in the rotate-half pairing (c, c + dh/2), softmax attention,
+ *     output projection, SwiGLU MLP, residual adds, final RMSNorm, untied
+ *     lm-head.
+ *   - Tree attention (Section 3.4 "Tree attention"): the flattened tree keeps
+ *     each token's positional index n + depth, and a row attends to the
+ *     committed prefix plus its own ancestors and itself.
+ *   - Pseudo hidden states (Section 3.2, Section 3.3 Eq. 3): at the input of
+ *     layer l, k rows h~_i = W_i h[anchor] + b_i are appended.  Pseudo row i
+ *     stands for position pos[anchor] + i; it sees the prefix, the anchor's
+ *     ancestors and the anchor, the earlier pseudo rows ("No masked" setting
+ *     of Section 4.3) and itself (Section 3.3, paragraph after Eq. 3).
+ *   - Greedy verification (Section 3.4, Section 4 "greedy sampling"): walk
+ *     from the root, following the child whose token equals the argmax of the
+ *     current row; the walk's nodes are the accepted path, the last argmax is
+ *     the bonus token.
+ *   - Next tree (Section 3.4): node v at depth j of a static template takes
+ *     the rank[v]-th best token of pseudo row j.
+ *   - KV compaction: the cache rows of the accepted path move to slots
+ *     n .. n+a, and n grows by a+1.
+ *
+ * Readings where the paper is silent: W is stored [out][in] (h~[o] = sum_c
+ * W[o][c] h[c] + b[o]); the map is applied to the raw residual stream; ties in
+ * argmax/top-B go to the lowest token id, duplicate sibling tokens to the
+ * lowest node index; tree rows never see pseudo rows.
+ *
+ * Pins: tests/test_oracle_pins.py checks this file against an independent
+ * library implementation of the Llama decoder (autoregressive greedy decoding
+ * for T=1,k=0; per-path causal forwards for tree rows; a causal forward with
+ * rows replaced at layer l for the pseudo chain), closed forms for Eq. 3, and
+ * the losslessness invariant of Eq. 1.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+typedef struct {
+  int32_t L, d, H, Hkv, dh, F, V;
+  int32_t max_ctx;   /* cache slots per sequence (committed + one step's rows) */
+  int32_t n_maps;    /* predictor maps available (k <= n_maps) */
+  int32_t n_seq;     /* independent sequences, each with its own cache */
+  float eps, theta;
+} oracle_cfg;
+
+typedef struct {
+  const uint16_t *embed;    /* [V][d] */
+  const uint16_t *lm_head;  /* [V][d] */
+  const uint16_t *g_final;  /* [d] */
+  const uint16_t *pred_w;   /* [n_maps][d][d], [out][in] */
+  const uint16_t *pred_b;   /* [n_maps][d] or NULL */
+  const uint16_t *const *wq, *const *wk, *const *wv;  /* per layer: [H*dh][d], [Hkv*dh][d] x2 */
+  const uint16_t *const *wo;                          /* [d][H*dh] */
+  const uint16_t *const *wgate, *const *wup;          /* [F][d] */
+  const uint16_t *const *wdown;                       /* [d][F] */
+  const uint16_t *const *g_attn, *const *g_mlp;       /* [d] */
+} oracle_weights;
+
+typedef struct {
+  oracle_cfg cfg;
+  oracle_weights w;
+  int32_t *n;      /* committed length per sequence */
+  float **kc;      /* per sequence: [L][max_ctx][Hkv*dh] */
+  float **vc;
+} oracle_t;
+
+static inline float bf16f(uint16_t b) {
+  union { uint32_t u; float f; } v; v.u = (uint32_t)b << 16; return v.f;
+}
+
+void *oracle_create(const oracle_cfg *cfg) {
+  oracle_t *o = (oracle_t *)calloc(1, sizeof(oracle_t));
+  o->cfg = *cfg;
+  o->n = (int32_t *)calloc(cfg->n_seq, sizeof(int32_t));
+  o->kc = (float **)calloc(cfg->n_seq, sizeof(float *));
+  o->vc = (float **)calloc(cfg->n_seq, sizeof(float *));
+  size_t per = (size_t)cfg->L * cfg->max_ctx * cfg->Hkv * cfg->dh;
+  for (int s = 0; s < cfg->n_seq; ++s) {
+    o->kc[s] = (float *)calloc(per, sizeof(float));
+    o->vc[s] = (float *)calloc(per, sizeof(float));
+    if (!o->kc[s] || !o->vc[s]) return NULL;
+  }
+  return o;
+}
+
+void oracle_destroy(void *h) {
+  oracle_t *o = (oracle_t *)h;
+  if (!o) return;
+  for (int s = 0; s < o->cfg.n_seq; ++s) { free(o->kc[s]); free(o->vc[s]); }
+  free(o->kc); free(o->vc); free(o->n); free(o);
+}
+
+void oracle_set_weights(void *h, const oracle_weights *w) { ((oracle_t *)h)->w = *w; }
+int32_t oracle_context_len(void *h, int32_t seq) { return ((oracle_t *)h)->n[seq]; }
+/* Rewind the committed length (rows >= n become scratch again); n = 0 empties the cache. */
+void oracle_set_context_len(void *h, int32_t seq, int32_t n) { ((oracle_t *)h)->n[seq] = n; }
+
+/* y[m][o] = sum_c W[o][c] * x[m][c]   (W bf16 [n_out][n_in]; x rows ldx apart; y rows ldy apart) */
+static void linear(const uint16_t *W, const float *x, int ldx, float *y, int ldy, int M, int n_in, int n_out) {
+#pragma omp parallel
+  {
+    float *wrow = (float *)malloc(sizeof(float) * n_in);
+#pragma omp for schedule(static)
+    for (int o = 0; o < n_out; ++o) {
+      for (int c = 0; c < n_in; ++c) wrow[c] = bf16f(W[(size_t)o * n_in + c]);
+      for (int m = 0; m < M; ++m) {
+        const float *xr = x + (size_t)m * ldx;
+        double acc = 0.0;
+#pragma omp simd reduction(+ : acc)
+        for (int c = 0; c < n_in; ++c) acc += (double)wrow[c] * (double)xr[c];
+        y[(size_t)m * ldy + o] = (float)acc;
+      }
+    }
+    free(wrow);
+  }
+}
+
+/* x[m][c] = h[m][c] / sqrt(mean_c h[m][c]^2 + eps) * g[c] */
+static void rmsnorm(const float *h, const uint16_t *g, float eps, float *x, int M, int d) {
+  for (int m = 0; m < M; ++m) {
+    double ss = 0.0;
+    for (int c = 0; c < d; ++c) ss += (double)h[(size_t)m * d + c] * (double)h[(size_t)m * d + c];
+    double r = 1.0 / sqrt(ss / d + (double)eps);
+    for (int c = 0; c < d; ++c) x[(size_t)m * d + c] = (float)((double)h[(size_t)m * d + c] * r * (double)bf16f(g[c]));
+  }
+}
+
+/* Rotary embedding at position p on one head vector, rotate-half pairing (c, c+dh/2). */
+static void rope(float *x, int dh, int p, double theta) {
+  int half = dh / 2;
+  for (int c = 0; c < half; ++c) {
+    double inv_freq = pow(theta, -2.0 * c / dh);
+    double ang = (double)p * inv_freq, cs = cos(ang), sn = sin(ang);
+    double a = x[c], b = x[c + half];
+    x[c] = (float)(a * cs - b * sn);
+    x[c + half] = (float)(b * cs + a * sn);
+  }
+}
+
+/*
+ * Tree bookkeeping (Section 3.4 "Tree attention"; Section 3.3 for pseudo rows).
+ * Rows 0..T-1 are tree nodes, rows T..T+k-1 the pseudo chain hanging off `anchor`.
+ * depth[v], mask[v][u] = 1 iff u is v or an ancestor of v, rank[v] = ordinal of v
+ * among its parent's children in index order (tree rows only; rank[0] = 0).
+ * Returns 0, or -1 for a malformed tree.
+ */
+int32_t oracle_tree_prep(const int32_t *parents, int32_t T, int32_t k, int32_t anchor,
+                         int32_t *ext_parent, int32_t *depth, uint8_t *mask, int32_t *rank) {
+  int M = T + k;
+  if (T < 1 || parents[0] != -1 || anchor < 0 || anchor >= T) return -1;
+  for (int v = 1; v < T; ++v) if (parents[v] < 0 || parents[v] >= v) return -1;
+  for (int v = 0; v < T; ++v) ext_parent[v] = parents[v];
+  for (int i = 1; i <= k; ++i) ext_parent[T + i - 1] = (i == 1) ? anchor : T + i - 2;
+  memset(mask, 0, (size_t)M * M);
+  for (int v = 0; v < M; ++v) {
+    depth[v] = (ext_parent[v] < 0) ? 0 : depth[ext_parent[v]] + 1;
+    for (int u = v; u >= 0; u = ext_parent[u]) mask[(size_t)v * M + u] = 1;
+  }
+  if (rank) {
+    for (int v = 0; v < T; ++v) {
+      int r = 0;
+      for (int u = 1; u < v; ++u) if (parents[u] == parents[v]) ++r;
+      rank[v] = (v == 0) ? 0 : r;
+    }
+  }
+  return 0;
+}
+
+/*
+ * One forward pass over the T tree rows (+ k pseudo rows from layer l on) of
+ * sequence `seq`, on top of its committed cache of n positions.  Cache slots
+ * n..n+T+k-1 receive the rows' keys/values (scratch until oracle_commit).
+ *
+ * logits      [(T+k)][V] fp32 out; rows < logit_row0 are skipped (left untouched)
+ * h_at_l      optional [(T+k)][d]: residual stream entering layer l, after insertion
+ * Returns 0, -1 malformed tree, -2 capacity.
+ */
+int32_t oracle_forward(void *hnd, int32_t seq, const int32_t *tokens, const int32_t *parents,
+                       int32_t T, int32_t k, int32_t l, int32_t anchor, int32_t logit_row0,
+                       float *logits, int32_t *depth_out, uint8_t *mask_out, float *h_at_l) {
+  oracle_t *o = (oracle_t *)hnd;
+  const oracle_cfg *c = &o->cfg;
+  const oracle_weights *w = &o->w;
+  const int d = c->d, H = c->H, Hkv = c->Hkv, dh = c->dh, F = c->F, V = c->V;
+  const int nq = H * dh, nkv = Hkv * dh, M = T + k, n = o->n[seq];
+  if (k < 0 || k > c->n_maps || (k > 0 && (l < 0 || l >= c->L))) return -1;
+  if (n + M > c->max_ctx) return -2;
+
+  int32_t *ext_parent = (int32_t *)malloc(sizeof(int32_t) * M);
+  int32_t *depth = (int32_t *)malloc(sizeof(int32_t) * M);
+  uint8_t *mask = (uint8_t *)malloc((size_t)M * M);
+  if (oracle_tree_prep(parents, T, k, anchor, ext_parent, depth, mask, NULL) != 0) {
+    free(ext_parent); free(depth); free(mask); return -1;
+  }
+
+  float *h = (float *)calloc((size_t)M * d, sizeof(float));
+  float *x = (float *)calloc((size_t)M * d, sizeof(float));
+  float *q = (float *)calloc((size_t)M * nq, sizeof(float));
+  float *att = (float *)calloc((size_t)M * nq, sizeof(float));
+  float *delta = (float *)calloc((size_t)M * d, sizeof(float));
+  float *gate = (float *)calloc((size_t)M * F, sizeof(float));
+  float *up = (float *)calloc((size_t)M * F, sizeof(float));
+  double *p = (double *)malloc(sizeof(double) * (n + M));
+
+  /* token embeddings of the tree rows */
+  for (int v = 0; v < T; ++v)
+    for (int cc = 0; cc < d; ++cc) h[(size_t)v * d + cc] = bf16f(w->embed[(size_t)tokens[v] * d + cc]);
+
+  int rows = T;  /* rows alive: T before layer l, T+k from layer l on */
+  for (int j = 0; j < c->L; ++j) {
+    if (k > 0 && j == l) {
+      /* Eq. 3: h~_i = W_i h[anchor] + b_i, appended as rows T..T+k-1 */
+      for (int i = 0; i < k; ++i) {
+        float *dst = h + (size_t)(T + i) * d;
+        linear(w->pred_w + (size_t)i * d * d, h + (size_t)anchor * d, d, dst, d, 1, d, d);
+        if (w->pred_b) for (int cc = 0; cc < d; ++cc) dst[cc] += bf16f(w->pred_b[(size_t)i * d + cc]);
+      }
+      rows = M;
+    }
+    if (h_at_l && j == l) memcpy(h_at_l, h, sizeof(float) * (size_t)M * d);
+
+    float *kc = o->kc[seq] + (size_t)j * c->max_ctx * nkv;
+    float *vc = o->vc[seq] + (size_t)j * c->max_ctx * nkv;
+
+    /* attention block */
+    rmsnorm(h, w->g_attn[j], c->eps, x, rows, d);
+    linear(w->wq[j], x, d, q, nq, rows, d, nq);
+    linear(w->wk[j], x, d, kc + (size_t)n * nkv, nkv, rows, d, nkv);
+    linear(w->wv[j], x, d, vc + (size_t)n * nkv, nkv, rows, d, nkv);
+    for (int v = 0; v < rows; ++v) {
+      int pos = n + depth[v];
+      for (int hd = 0; hd < H; ++hd) rope(q + (size_t)v * nq + hd * dh, dh, pos, c->theta);
+      for (int hd = 0; hd < Hkv; ++hd) rope(kc + (size_t)(n + v) * nkv + hd * dh, dh, pos, c->theta);
+    }
+    for (int v = 0; v < rows; ++v) {
+      for (int hd = 0; hd < H; ++hd) {
+        const int kvh = hd / (H / Hkv);
+        const float *qv = q + (size_t)v * nq + hd * dh;
+        /* scores over the committed prefix and the visible new rows */
+        double mx = -INFINITY;
+        for (int u = 0; u < n + rows; ++u) {
+          int visible = (u < n) || mask[(size_t)v * M + (u - n)];
+          if (!visible) { p[u] = -INFINITY; continue; }
+          const float *ku = kc + (size_t)u * nkv + kvh * dh;
+          double s = 0.0;
+          for (int cc = 0; cc < dh; ++cc) s += (double)qv[cc] * (double)ku[cc];
+          p[u] = s / sqrt((double)dh);
+          if (p[u] > mx) mx = p[u];
+        }
+        double sum = 0.0;
+        for (int u = 0; u < n + rows; ++u) { p[u] = (p[u] == -INFINITY) ? 0.0 : exp(p[u] - mx); sum += p[u]; }
+        for (int cc = 0; cc < dh; ++cc) {
+          double acc = 0.0;
+          for (int u = 0; u < n + rows; ++u) acc += p[u] * (double)vc[(size_t)u * nkv + kvh * dh + cc];
+          att[(size_t)v * nq + hd * dh + cc] = (float)(acc / sum);
+        }
+      }
+    }
+    linear(w->wo[j], att, nq, delta, d, rows, nq, d);
+    for (size_t i = 0; i < (size_t)rows * d; ++i) h[i] += delta[i];
+
+    /* SwiGLU MLP block */
+    rmsnorm(h, w->g_mlp[j], c->eps, x, rows, d);
+    linear(w->wgate[j], x, d, gate, F, rows, d, F);
+    linear(w->wup[j], x, d, up, F, rows, d, F);
+    for (size_t i = 0; i < (size_t)rows * F; ++i) {
+      double g = gate[i];
+      gate[i] = (float)(g / (1.0 + exp(-g)) * (double)up[i]);
+    }
+    linear(w->wdown[j], gate, F, delta, d, rows, F, d);
+    for (size_t i = 0; i < (size_t)rows * d; ++i) h[i] += delta[i];
+  }
+
+  /* final norm + original lm-head on every row (Section 3.2) */
+  rmsnorm(h, w->g_final, c->eps, x, M, d);
+  if (logit_row0 < 0) logit_row0 = 0;
+  if (logits && logit_row0 < M)
+    linear(w->lm_head, x + (size_t)logit_row0 * d, d, logits + (size_t)logit_row0 * V, V, M - logit_row0, d, V);
+
+  if (depth_out) memcpy(depth_out, depth, sizeof(int32_t) * M);
+  if (mask_out) memcpy(mask_out, mask, (size_t)M * M);
+  free(ext_parent); free(depth); free(mask);
+  free(h); free(x); free(q); free(att); free(delta); free(gate); free(up); free(p);
+  return 0;
+}
+
+/* argmax with ties to the lowest index */
+static int32_t argmax_row(const float *row, int V) {
+  int32_t best = 0;
+  for (int t = 1; t < V; ++t) if (row[t] > row[best]) best = t;
+  return best;
+}
+
+/*
+ * Greedy verification (Section 3.4): best[v] = argmax logits[v] for tree rows;
+ * path[0] = 0; from cur, move to the lowest-index child whose token equals
+ * best[cur]; stop when there is none.  accepted = tokens of path[1..a] followed
+ * by the bonus token best[path[a]].  Returns a+1 (tokens emitted).
+ */
+int32_t oracle_verify(const float *logits, const int32_t *tokens, const int32_t *parents, int32_t T, int32_t V,
+                      int32_t *best, int32_t *path, int32_t *accepted) {
+  for (int v = 0; v < T; ++v) best[v] = argmax_row(logits + (size_t)v * V, V);
+  int cur = 0, a = 0;
+  path[0] = 0;
+  for (;;) {
+    int next = -1;
+    for (int ch = cur + 1; ch < T; ++ch)
+      if (parents[ch] == cur && tokens[ch] == best[cur]) { next = ch; break; }
+    if (next < 0) break;
+    accepted[a] = tokens[next];
+    path[++a] = next;
+    cur = next;
+  }
+  accepted[a] = best[cur];
+  return a + 1;
+}
+
+/*
+ * Top-B of each pseudo row, ordered by (value descending, id ascending), and the
+ * next tree on a static template (Section 3.4): next[0] = bonus; a node at depth
+ * j >= 1 with sibling rank r takes topb[j-1][r].  Returns 0, or -1 if the
+ * template needs a depth beyond k or a rank beyond B.
+ */
+int32_t oracle_next_tree(const float *logits, int32_t T, int32_t k, int32_t V, int32_t B, int32_t bonus,
+                         const int32_t *next_parents, int32_t T_next,
+                         int32_t *topb_ids, float *topb_vals, int32_t *next_tokens) {
+  for (int i = 0; i < k; ++i) {
+    const float *row = logits + (size_t)(T + i) * V;
+    for (int b = 0; b < B; ++b) {
+      int32_t pick = -1;
+      for (int t = 0; t < V; ++t) {
+        int taken = 0;
+        for (int e = 0; e < b; ++e) if (topb_ids[i * B + e] == t) taken = 1;
+        if (taken) continue;
+        if (pick < 0 || row[t] > row[pick]) pick = t;
+      }
+      topb_ids[i * B + b] = pick;
+      topb_vals[i * B + b] = row[pick];
+    }
+  }
+  int32_t *depth = (int32_t *)malloc(sizeof(int32_t) * T_next);
+  int rc = 0;
+  next_tokens[0] = bonus;
+  depth[0] = 0;
+  for (int v = 1; v < T_next; ++v) {
+    depth[v] = depth[next_parents[v]] + 1;
+    int r = 0;
+    for (int u = 1; u < v; ++u) if (next_parents[u] == next_parents[v]) ++r;
+    if (depth[v] > k || r >= B) { rc = -1; break; }
+    next_tokens[v] = topb_ids[(depth[v] - 1) * B + r];
+  }
+  free(depth);
+  return rc;
+}
+
+/*
+ * Commit: cache rows of path[j] (row index within the last step) move to slot
+ * n + j in every layer; n += len.  path is strictly increasing with path[j] >= j.
+ */
+int32_t oracle_commit(void *hnd, int32_t seq, const int32_t *path, int32_t len) {
+  oracle_t *o = (oracle_t *)hnd;
+  const oracle_cfg *c = &o->cfg;
+  const int nkv = c->Hkv * c->dh, n = o->n[seq];
+  if (n + len > c->max_ctx) return -2;
+  for (int j = 0; j < len; ++j) if (path[j] < j || (j > 0 && path[j] <= path[j - 1])) return -1;
+  for (int lay = 0; lay < c->L; ++lay) {
+    float *kc = o->kc[seq] + (size_t)lay * c->max_ctx * nkv;
+    float *vc = o->vc[seq] + (size_t)lay * c->max_ctx * nkv;
+    for (int j = 0; j < len; ++j) {
+      if (path[j] == j) continue;
+      memmove(kc + (size_t)(n + j) * nkv, kc + (size_t)(n + path[j]) * nkv, sizeof(float) * nkv);
+      memmove(vc + (size_t)(n + j) * nkv, vc + (size_t)(n + path[j]) * nkv, sizeof(float) * nkv);
+    }
+  }
+  o->n[seq] = n + len;
+  return 0;
+}
+
+/* Read one committed/scratch cache row (tests of the compaction). which: 0 = K, 1 = V. */
+void oracle_read_cache(void *hnd, int32_t seq, int32_t layer, int32_t which, int32_t slot, float *out) {
+  oracle_t *o = (oracle_t *)hnd;
+  const oracle_cfg *c = &o->cfg;
+  const int nkv = c->Hkv * c->dh;
+  const float *base = (which ? o->vc[seq] : o->kc[seq]) + ((size_t)layer * c->max_ctx + slot) * nkv;
+  memcpy(out, base, sizeof(float) * nkv);
+}

@@ -1,0 +1,95 @@
+"""An independent library implementation of the Llama decoder (HuggingFace
+transformers, CPU, float64) loaded with the same bf16 weights.  The paper's own
+implementation is built on this architecture (Section 4 "Setup"), so the oracle's
+special cases must reduce to it.  Used only to pin the oracle."""
+import numpy as np
+import torch
+
+import synth_inputs as si
+
+
+def build_hf_llama(shape, weights):
+    from transformers import LlamaConfig, LlamaForCausalLM
+    s = shape
+    cfg = LlamaConfig(hidden_size=s.d, intermediate_size=s.F, num_hidden_layers=s.L, num_attention_heads=s.H,
+                      num_key_value_heads=s.Hkv, vocab_size=s.V, rms_norm_eps=s.eps, rope_theta=s.theta,
+                      tie_word_embeddings=False, head_dim=s.dh, max_position_embeddings=4096,
+                      attention_bias=False, mlp_bias=False)
+    cfg._attn_implementation = "eager"
+    model = LlamaForCausalLM(cfg).double().eval()
+
+    def f(bits):
+        return torch.from_numpy(si.bf16_bits_to_f32(np.ascontiguousarray(bits)).astype(np.float64))
+
+    sd = {"model.embed_tokens.weight": f(weights["embed"]), "lm_head.weight": f(weights["lm_head"]),
+          "model.norm.weight": f(weights["g_final"])}
+    for i, lw in enumerate(weights["layers"]):
+        p = "model.layers.%d." % i
+        sd[p + "self_attn.q_proj.weight"] = f(lw["wqkv"][: s.n_q])
+        sd[p + "self_attn.k_proj.weight"] = f(lw["wqkv"][s.n_q: s.n_q + s.n_kv])
+        sd[p + "self_attn.v_proj.weight"] = f(lw["wqkv"][s.n_q + s.n_kv:])
+        sd[p + "self_attn.o_proj.weight"] = f(lw["wo"])
+        sd[p + "mlp.gate_proj.weight"] = f(lw["wgu"][: s.F])
+        sd[p + "mlp.up_proj.weight"] = f(lw["wgu"][s.F:])
+        sd[p + "mlp.down_proj.weight"] = f(lw["wd"])
+        sd[p + "input_layernorm.weight"] = f(lw["g_attn"])
+        sd[p + "post_attention_layernorm.weight"] = f(lw["g_mlp"])
+    model.load_state_dict(sd, strict=True)
+    return model
+
+
+def hf_logits(model, token_ids):
+    """Plain causal forward, no cache: logits [len, V] as float64 numpy."""
+    with torch.no_grad():
+        ids = torch.as_tensor(np.asarray(token_ids, dtype=np.int64))[None]
+        return model(ids, use_cache=False).logits[0].numpy()
+
+
+def hf_greedy(model, prompt_ids, count):
+    """Cache-free greedy decoding by full recompute."""
+    ids = [int(t) for t in prompt_ids]
+    out = []
+    for _ in range(count):
+        t = int(np.argmax(hf_logits(model, ids)[-1]))
+        out.append(t)
+        ids.append(t)
+    return out
+
+
+def hf_kv(model, token_ids):
+    """Post-rotary keys and values of a from-scratch forward: lists per layer of [len, Hkv*dh]."""
+    with torch.no_grad():
+        ids = torch.as_tensor(np.asarray(token_ids, dtype=np.int64))[None]
+        out = model(ids, use_cache=True)
+    pkv = out.past_key_values
+    ks, vs = [], []
+    for layer in range(model.config.num_hidden_layers):
+        try:
+            k, v = pkv.layers[layer].keys, pkv.layers[layer].values
+        except AttributeError:
+            k, v = pkv[layer][0], pkv[layer][1]
+        ks.append(k[0].transpose(0, 1).reshape(k.shape[2], -1).numpy())
+        vs.append(v[0].transpose(0, 1).reshape(v.shape[2], -1).numpy())
+    return ks, vs
+
+
+def hf_logits_with_replaced_rows(model, token_ids, layer, first_row, maps_w, maps_b, anchor_row):
+    """Causal forward in which, at the input of decoder layer `layer`, rows
+    first_row.. are replaced by W_i h[anchor_row] + b_i (i = 0..len(maps_w)-1)."""
+    def hook(module, args, kwargs):
+        hs = args[0] if args else kwargs["hidden_states"]
+        hs = hs.clone()
+        src = hs[0, anchor_row]
+        for i, W in enumerate(maps_w):
+            hs[0, first_row + i] = torch.from_numpy(W) @ src + torch.from_numpy(maps_b[i])
+        if args:
+            return (hs,) + tuple(args[1:]), kwargs
+        kwargs = dict(kwargs)
+        kwargs["hidden_states"] = hs
+        return args, kwargs
+
+    handle = model.model.layers[layer].register_forward_pre_hook(hook, with_kwargs=True)
+    try:
+        return hf_logits(model, token_ids)
+    finally:
+        handle.remove()

@@ -1,0 +1,309 @@
+"""Pins for the CPU oracle: it is checked against things other than itself.
+
+  P1  T=1, k=0 stepping == cache-free greedy decoding by an independent library decoder
+  P2  every tree row's logits == a plain causal forward over prefix + root->row path
+  P3  Eq. 3 closed forms (W = I, W = 0, permutation W, non-zero bias)
+  P4  losslessness (Eq. 1): emitted tokens == the autoregressive greedy stream
+  P5  tree rows do not depend on k or on the predictor maps
+  P6  committed cache == keys/values of a from-scratch forward over the committed tokens
+  P7  forced-accept mode accepts the full depth every step
+  P8  the pseudo chain == a causal forward whose rows are replaced at layer l
+  P9  predictor size k*d^2 equals the draft-module sizes printed in the paper's Table 1
+plus hand-worked cases for the mask, the acceptance walk, the tie rules and the next tree.
+"""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+import synth_inputs as si
+from hf_reference import (build_hf_llama, hf_greedy, hf_kv, hf_logits, hf_logits_with_replaced_rows)
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+@pytest.fixture(scope="module")
+def hf(c1, c1_weights):
+    return build_hf_llama(c1, c1_weights)
+
+
+def fresh(c1, weights, max_ctx=256, n_seq=1):
+    return oracle.Oracle(c1, weights, max_ctx=max_ctx, n_seq=n_seq)
+
+
+def path_to(parents, v):
+    p = []
+    while v >= 0:
+        p.append(v)
+        v = int(parents[v])
+    return p[::-1]
+
+
+# ---------------------------------------------------------------- P1
+def test_p1_t1_k0_is_autoregressive_greedy(c1, c1_weights, hf):
+    prompt = si.prompt(c1)
+    want = hf_greedy(hf, prompt, 12)
+    o = fresh(c1, c1_weights)
+    r = o.prefill(prompt, 0, 0, None)
+    got, tok, ids = [r["root"]], r["root"], list(prompt)
+    one = np.array([-1], np.int32)
+    for _ in range(11):
+        out = o.step([tok], one, 0, 0)
+        ids.append(tok)
+        ref = hf_logits(hf, ids)[-1]
+        assert np.abs(out["logits"][0] - ref).max() < 1e-5
+        assert out["n_accepted"] == 1 and out["path"].tolist() == [0]
+        o.commit([0])
+        tok = int(out["accepted"][0])
+        got.append(tok)
+    assert got == want
+
+
+# ---------------------------------------------------------------- P2
+@pytest.mark.parametrize("case", range(4))
+def test_p2_tree_rows_equal_per_path_causal_forward(c1, c1_weights, hf, case):
+    prompt = si.prompt(c1, length=20 + 3 * case)
+    T = (8, 13, 16, 5)[case]
+    parents = si.tree_template(8) if case == 0 else si.random_tree(7, T, 3, case)
+    tokens = si.random_tokens(c1, T, case)
+    o = fresh(c1, c1_weights)
+    o.prefill(prompt, 0, 0, None)
+    out = o.forward(tokens, parents, 3, 1)
+    for v in range(T):
+        ids = list(prompt) + [int(tokens[u]) for u in path_to(parents, v)]
+        ref = hf_logits(hf, ids)[-1]
+        assert np.abs(out["logits"][v] - ref).max() < 1e-5, v
+        assert out["depth"][v] == len(path_to(parents, v)) - 1
+
+
+def test_mask_is_ancestor_closure_bruteforce():
+    for case in range(6):
+        T, k = 5 + 4 * case, case % 4
+        parents = si.random_tree(11, T, 6, case)
+        anchor = case % T
+        tp = oracle.tree_prep(parents, k, anchor)
+        ext = list(parents) + [anchor if i == 0 else T + i - 1 for i in range(k)]
+        for v in range(T + k):
+            anc = set(path_to(ext, v))
+            assert set(np.nonzero(tp["mask"][v])[0].tolist()) == anc
+            assert tp["depth"][v] == len(anc) - 1
+        # tree rows never see pseudo rows
+        assert not tp["mask"][:T, T:].any()
+        for v in range(1, T):
+            sib = [u for u in range(1, T) if parents[u] == parents[v]]
+            assert tp["rank"][v] == sib.index(v)
+
+
+def test_mask_worked_example():
+    # the 8-node 2-2-1 template: root->1->2->3, root->4->6, 1->5->7; pseudo chain off the root
+    tp = oracle.tree_prep(si.tree_template(8), 3, 0)
+    with open(os.path.join(GOLDEN, "mask_t8_k3.txt")) as f:
+        rows = [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+    want = np.array([[int(c) for c in r] for r in rows], np.uint8)
+    assert (tp["mask"] == want).all()
+    assert tp["depth"].tolist() == [0, 1, 2, 3, 1, 2, 2, 3, 1, 2, 3]
+
+
+def test_malformed_trees_rejected():
+    for bad in ([0, 0], [-1, 1], [-1, 2, 0], [-1, -1]):
+        with pytest.raises(ValueError):
+            oracle.tree_prep(np.array(bad, np.int32), 0, 0)
+
+
+# ---------------------------------------------------------------- P3
+def with_maps(weights, pred_w_f32, pred_b_f32):
+    import torch
+    w = dict(weights)
+    to_bits = lambda a: torch.from_numpy(np.ascontiguousarray(a, np.float32)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    w["pred_w"], w["pred_b"] = to_bits(pred_w_f32), to_bits(pred_b_f32)
+    return w
+
+
+def test_p3_eq3_closed_forms(c1, c1_weights):
+    d, k = c1.d, 3
+    prompt = si.prompt(c1)
+    tokens, parents = si.random_tokens(c1, 8, 5), si.tree_template(8)
+    perm = np.roll(np.arange(d), 5)
+    Wp = np.zeros((d, d), np.float32); Wp[np.arange(d), perm] = 1.0          # h~[o] = h[perm[o]]
+    W = np.stack([np.eye(d, dtype=np.float32), np.zeros((d, d), np.float32), 2.0 * Wp])
+    b = np.zeros((k, d), np.float32); b[1] = np.linspace(-1, 1, d); b[2] = 0.5
+    w = with_maps(c1_weights, W, b)
+    b_rounded = si.bf16_bits_to_f32(w["pred_b"])
+    for anchor in (0, 4):
+        o = fresh(c1, w)
+        o.prefill(prompt, 0, 0, None)
+        out = o.forward(tokens, parents, k, 1, anchor=anchor, want_h_at_l=True)
+        h = out["h_at_l"]
+        assert np.array_equal(h[8], h[anchor])                                 # W = I, b = 0
+        assert np.array_equal(h[9], b_rounded[1])                              # W = 0
+        assert np.allclose(h[10], 2.0 * h[anchor][perm] + b_rounded[2], rtol=0, atol=1e-6)   # permutation
+        assert out["depth"][8:].tolist() == [out["depth"][anchor] + i for i in (1, 2, 3)]
+
+
+def test_p3_eq3_orientation_out_in(c1, c1_weights):
+    # a single non-zero entry W[o=3][c=7] = 1.5 must move coordinate 7 into coordinate 3
+    d = c1.d
+    W = np.zeros((3, d, d), np.float32); W[0, 3, 7] = 1.5
+    w = with_maps(c1_weights, W, np.zeros((3, d), np.float32))
+    o = fresh(c1, w)
+    o.prefill(si.prompt(c1), 0, 0, None)
+    h = o.forward([5], [-1], 3, 1, want_h_at_l=True)["h_at_l"]
+    want = np.zeros(d, np.float32); want[3] = np.float32(1.5) * h[0, 7]
+    assert np.allclose(h[1], want, rtol=0, atol=1e-7) and h[0, 7] != 0
+
+
+# ---------------------------------------------------------------- P8
+@pytest.mark.parametrize("l", [0, 1])
+def test_p8_pseudo_chain_is_causal_forward_with_replaced_rows(c1, c1_weights, hf, l):
+    k = 3
+    prompt = si.prompt(c1, length=17)
+    Wf = si.bf16_bits_to_f32(c1_weights["pred_w"]).astype(np.float64)
+    bf = np.zeros((k, c1.d))
+    o = fresh(c1, c1_weights)
+    # plain picture of Section 3.2: chain over the prompt, anchor = last prompt token
+    chain = si.chain_template(prompt.size)
+    out = o.forward(prompt, chain, k, l, anchor=prompt.size - 1)
+    ids = list(prompt) + [0] * k            # filler ids: their rows are replaced at layer l
+    ref = hf_logits_with_replaced_rows(hf, ids, l, prompt.size, list(Wf), list(bf), prompt.size - 1)
+    assert np.abs(out["logits"][prompt.size:] - ref[prompt.size:]).max() < 1e-5
+    assert np.abs(out["logits"][: prompt.size] - ref[: prompt.size]).max() < 1e-5
+    # chain off the root of a tree step (anchor 0) on top of a committed prefix
+    o.commit(np.arange(prompt.size))
+    tokens, parents = si.random_tokens(c1, 8, 9), si.tree_template(8)
+    out = o.forward(tokens, parents, k, l, anchor=0)
+    ids = list(prompt) + [int(tokens[0])] + [0] * k
+    ref = hf_logits_with_replaced_rows(hf, ids, l, prompt.size + 1, list(Wf), list(bf), prompt.size)
+    assert np.abs(out["logits"][8:] - ref[prompt.size + 1:]).max() < 1e-5
+
+
+# ---------------------------------------------------------------- P5
+def test_p5_tree_rows_independent_of_k_and_maps(c1, c1_weights):
+    prompt, tokens, parents = si.prompt(c1), si.random_tokens(c1, 8, 2), si.tree_template(8)
+    o = fresh(c1, c1_weights)
+    o.prefill(prompt, 0, 0, None)
+    a = o.forward(tokens, parents, 0, 0)["logits"]
+    b = o.forward(tokens, parents, 3, 1)["logits"]
+    w2 = with_maps(c1_weights, np.random.default_rng(0).normal(size=(3, c1.d, c1.d)).astype(np.float32),
+                   np.ones((3, c1.d), np.float32))
+    o2 = fresh(c1, w2)
+    o2.prefill(prompt, 0, 0, None)
+    c = o2.forward(tokens, parents, 3, 0)["logits"]
+    assert np.array_equal(a, b[:8]) and np.array_equal(a, c[:8])
+    assert not np.array_equal(b[8:], c[8:])
+
+
+# ---------------------------------------------------------------- P4, P6, P7
+def run_free(o, c1, prompt, steps, forced, hf_stream=None):
+    """Free-running decode with the oracle's own trees; returns emitted tokens and per-step a."""
+    parents = si.tree_template(c1.T)
+    tp = oracle.tree_prep(parents)
+    D = int(tp["depth"].max())
+    principal = [0]
+    for _ in range(D):
+        principal.append(min(u for u in range(c1.T) if parents[u] == principal[-1]))
+    r = o.prefill(prompt, c1.k, c1.l, parents)
+    tokens, emitted, accs = r["next_tokens"].copy(), [r["root"]], []
+    for _ in range(steps):
+        if forced:
+            g = o.ar_greedy(int(tokens[0]), D)
+            for j in range(1, D + 1):
+                v = principal[j]
+                sibs = [u for u in range(c1.T) if parents[u] == parents[v] and u != v and tokens[u] == g[j - 1]]
+                for u in sibs:
+                    tokens[u] = tokens[v]
+                tokens[v] = g[j - 1]
+        out = o.step(tokens, parents, c1.k, c1.l)
+        o.commit(out["path"])
+        emitted += out["accepted"].tolist()
+        accs.append(out["n_accepted"] - 1)
+        tokens = out["next_tokens"].copy()
+    return emitted, accs, D
+
+
+def test_p4_lossless_and_p6_cache_and_p7_forced(c1, c1_weights, hf):
+    prompt = si.prompt(c1)
+    want = hf_greedy(hf, prompt, 70)
+    for forced in (False, True):
+        o = fresh(c1, c1_weights)
+        emitted, accs, D = run_free(o, c1, prompt, 16, forced)
+        assert emitted == want[: len(emitted)]                       # P4 (Eq. 1)
+        if forced:
+            assert accs == [D] * 16 and len(emitted) == 1 + 16 * (D + 1)   # P7
+        # P6: committed cache == from-scratch keys/values over the committed tokens
+        n = o.context_len()
+        committed = list(prompt) + emitted[: n - prompt.size]
+        assert len(committed) == n
+        ks, vs = hf_kv(hf, committed)
+        for layer in range(c1.L):
+            for slot in (0, prompt.size - 1, prompt.size, n - 2, n - 1):
+                assert np.abs(o.read_cache(0, layer, 0, slot) - ks[layer][slot]).max() < 1e-5
+                assert np.abs(o.read_cache(0, layer, 1, slot) - vs[layer][slot]).max() < 1e-5
+
+
+def test_p4_lossless_with_arbitrary_trees(c1, c1_weights, hf):
+    # any tree contents give the same stream: random tokens, random shapes
+    prompt = si.prompt(c1, length=11)
+    want = hf_greedy(hf, prompt, 14)
+    o = fresh(c1, c1_weights)
+    r = o.prefill(prompt, 3, 1, si.tree_template(8))
+    emitted, root = [r["root"]], r["root"]
+    for step in range(6):
+        T = 4 + step
+        parents = si.random_tree(3, T, 3, step)
+        tokens = si.random_tokens(c1, T, 50 + step)
+        tokens[0] = root
+        if step % 2 == 0:            # plant the true next token on a child of the root
+            tokens[1] = want[len(emitted)]
+        out = o.step(tokens, parents, 3, 1)
+        o.commit(out["path"])
+        emitted += out["accepted"].tolist()
+        root = int(out["accepted"][-1])
+    assert emitted == want[: len(emitted)]
+    assert len(emitted) > 7                                       # the planted tokens were accepted
+
+
+# ---------------------------------------------------------------- hand-worked verification / next tree
+def test_verify_walk_and_ties_hand_example(c1, c1_weights):
+    o = fresh(c1, c1_weights)
+    V = c1.V
+    parents = np.array([-1, 0, 0, 1, 1, 2], np.int32)
+    tokens = np.array([9, 5, 5, 7, 3, 7], np.int32)     # duplicate sibling token 5 on nodes 1 and 2
+    lg = np.zeros((6, V), np.float32)
+    lg[0, 5] = 1.0; lg[0, 900] = 1.0                     # tie 5 vs 900 -> lowest id 5
+    lg[1, 3] = 2.0; lg[1, 7] = 1.5                       # node 1 wants 3 -> child 4
+    lg[4, 11] = 4.0                                      # bonus 11
+    lg[2, 7] = 9.0                                       # never reached: node 1 (lower index) wins the duplicate
+    r = o.verify(lg, tokens, parents)
+    assert r["best"].tolist()[:2] == [5, 3] and r["best"][4] == 11
+    assert r["path"].tolist() == [0, 1, 4] and r["accepted"].tolist() == [5, 3, 11] and r["n_accepted"] == 3
+    lg[0, 900] = 1.5                                     # now the root wants 900: nothing accepted
+    r = o.verify(lg, tokens, parents)
+    assert r["path"].tolist() == [0] and r["accepted"].tolist() == [900]
+
+
+def test_next_tree_hand_example(c1, c1_weights):
+    o = fresh(c1, c1_weights)
+    V, T, k = c1.V, 2, 3
+    lg = np.zeros((T + k, V), np.float32)
+    lg[2, [10, 20, 30]] = [3.0, 2.0, 2.0]                # depth-1 list: 10, 20, 30 (tie -> lower id first)
+    lg[3, [40, 41]] = [1.0, 5.0]                          # depth-2 list: 41, 40
+    lg[4, 77] = 1.0                                       # depth-3 list: 77, then zeros by ascending id: 0, 1, ...
+    parents = si.tree_template(8)                         # depths 0 1 2 3 1 2 2 3, ranks 0 0 0 0 1 1 0 0
+    r = o.next_tree(lg, T, k, bonus=99, next_parents=parents)
+    assert r["topb_ids"][0, :3].tolist() == [10, 20, 30] and r["topb_ids"][1, :2].tolist() == [41, 40]
+    assert r["topb_ids"][2, :3].tolist() == [77, 0, 1]
+    assert r["topb_ids"][0, 3:].tolist() == [0, 1, 2, 3, 4]
+    assert r["next_tokens"].tolist() == [99, 10, 41, 77, 20, 40, 41, 77]
+    with pytest.raises(ValueError):                       # a template deeper than k cannot be filled
+        o.next_tree(lg, T, 2, 99, parents)
+
+
+# ---------------------------------------------------------------- P9
+def test_p9_predictor_size_matches_paper_table1():
+    with open(os.path.join(GOLDEN, "paper_table1_draft_module_params.txt")) as f:
+        rows = [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+    for name, d, k, billions in rows:
+        n_params = int(k) * int(d) ** 2
+        assert round(n_params / 1e9, 2) == float(billions), name
+    assert 3 * si.CONFIGS["c2"].d ** 2 == 50331648 and 3 * si.CONFIGS["c3"].d ** 2 == 78643200
