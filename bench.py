@@ -1,0 +1,358 @@
+#!/usr/bin/env python
+"""Benchmark of the FIRP draft+verify step on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+
+One "step" = one pass of the whole hot path: firp_step (tree prep, embedding, all decoder layers
+with the pseudo hidden states inserted at layer l, lm-head, top-B, acceptance walk, next tree)
+followed by firp_kv_commit, on the Llama-2-7B-shaped synthetic workload (T = 32, k = 3, l = 16,
+512 committed tokens, random bf16 weights from the seeded generator).  Prints ONE JSON line.
+
+N > 1 runs N independent replicas (the step does not shard; there is no collective): every rank
+steps its own sequence on its own GPU, the job's value is the sum of the units over the maximum
+of the device times.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "verify+draft step: accepted tokens/s (step latency in ms_per_step), Llama-2-7B shape; HBM GB/s vs peak"
+UNIT = "tokens/s"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", help="c1 | c2 | c3 | c4:T:n (sweep point on the c2 weights)")
+    ap.add_argument("--layers", type=int, default=0, help="debug only: truncate the decoder (marks the line invalid)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--profile-kernels", action="store_true", default=True)
+    return ap.parse_args()
+
+
+def pick_shape(name: str, layers: int):
+    import synth_inputs as si
+    if name.startswith("c4:"):
+        _, T, n = name.split(":")
+        shape = si.c4_point(int(T), int(n))
+    else:
+        shape = si.CONFIGS[name]
+    if layers:
+        shape = si.scaled(shape, L=layers, l=min(shape.l, layers - 1), name=shape.name + "-L%d" % layers)
+    return shape
+
+
+def algorithmic_bytes(shape, n_ctx: float) -> dict:
+    """Bytes one step must move: every weight once, the KV cache read once per layer, the new
+    rows' KV written once, the embedding rows (logits stay on the device and are not exported)."""
+    s = shape
+    M_lo, M_hi = s.T, s.T + s.k
+    weights = s.weight_bytes()
+    kv_row = 2 * 2 * s.n_kv                       # K and V, bf16
+    kv_read = kv_write = 0
+    for j in range(s.L):
+        M = M_hi if (s.k > 0 and j >= s.l) else M_lo
+        kv_read += kv_row * (n_ctx + M)
+        kv_write += kv_row * M
+    return dict(weights=weights, kv_read=kv_read, kv_write=kv_write, embed=2 * s.T * s.d,
+                total=weights + kv_read + kv_write + 2 * s.T * s.d)
+
+
+def gemm_class_bytes(shape) -> dict:
+    """Algorithmic bytes of each weight-streaming kernel class per launch (weights only)."""
+    s = shape
+    return dict(gemm_qkv=2 * s.n_qkv * s.d, gemm_o=2 * s.d * s.n_q, gemm_gate_up=2 * 2 * s.F * s.d,
+                gemm_down=2 * s.d * s.F, gemm_lm_head=2 * s.V * s.d, pseudo_proj=2 * s.k * s.d * s.d)
+
+
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.mktemp(suffix=".csv")
+        self.f = open(self.path, "w")
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.FIELDS,
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self) -> dict:
+        if self.p is not None:
+            self.p.terminate()
+            try:
+                self.p.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.p.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        try:
+            for ln in open(self.path):
+                c = [x.strip() for x in ln.split(",")]
+                if len(c) < 9:
+                    continue
+                try:
+                    sm.append(float(c[1])); mx.append(float(c[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except OSError:
+            pass
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def time_oracle(shape, weights, steps: int, warmup: int, n_ctx: int = 32):
+    """The CPU oracle, as it stands, on a bounded sample: `steps` full draft+verify steps (all layers,
+    T + k rows) on top of a short prefilled context."""
+    import oracle
+    import synth_inputs as si
+    parents = si.tree_template(shape.T)
+    orc = oracle.Oracle(shape, weights, max_ctx=n_ctx + (steps + warmup + 1) * (shape.k + 1) + shape.T + shape.k + 8)
+    r = orc.prefill(si.prompt(shape, length=n_ctx), shape.k, shape.l, parents)
+    tokens = r["next_tokens"]
+    emitted, t_total = 0, 0.0
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        out = orc.step(tokens, parents, shape.k, shape.l)
+        orc.commit(out["path"])
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            t_total += dt
+            emitted += int(out["n_accepted"])
+        tokens = out["next_tokens"]
+    return emitted / t_total, t_total / steps * 1e3
+
+
+def load_weights(shape, local_rank: int, world: int):
+    """Rank-local generation of the seeded weights (every rank needs the same tensors)."""
+    import synth_inputs as si
+    if world > 1:
+        os.environ.setdefault("OMP_NUM_THREADS", str(max(1, host_cores() // world)))
+    return si.all_weights(shape)
+
+
+def run_reference(args, shape):
+    """The reference arm of this tier is the CPU oracle, timed on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import synth_inputs as si
+    weights = si.all_weights(shape)
+    steps, warmup = max(1, min(args.steps, 3)), min(args.warmup, 1)
+    tps, ms = time_oracle(shape, weights, steps, warmup)
+    sample = "%d oracle steps (+%d warm-up) of T=%d,k=%d,l=%d over all %d layers on a 32-token context" % (
+        steps, warmup, shape.T, shape.k, shape.l, shape.L)
+    line = dict(metric=METRIC, value=tps, unit=UNIT, n_gpus=args.gpus, steps=steps, warmup=warmup, ms_per_step=ms,
+                higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32 storage, f64 accumulation",
+                data="synthetic", impl="reference",
+                config=dict(workload=shape.name, T=shape.T, k=shape.k, l=shape.l, context=32),
+                cpu_baseline=dict(value=tps, unit=UNIT, cores=host_cores(), kind="oracle", sample=sample),
+                e2e=dict(value=tps, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+def main():
+    args = parse()
+    shape = pick_shape(args.workload, args.layers)
+    if args.impl == "reference":
+        return run_reference(args, shape)
+
+    import torch
+    import torch.distributed as dist
+    import synth_inputs as si
+    from paper_2410_20488_b200 import FirpEngine, build as firp_build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the FIRP step has no CPU fallback")
+    if rank == 0:
+        firp_build.build()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+
+    K, W = args.steps, max(args.warmup, 3)
+    weights = load_weights(shape, local_rank, world)
+    parents = si.tree_template(shape.T)
+    depth_max = {1: 0}.get(shape.T, 3)
+    S = max(shape.k, 1) + 1
+    total_steps = 2 * (K + W) + 16
+    max_ctx = shape.prompt_len + total_steps * S + shape.T + shape.k + 64
+    eng = FirpEngine(shape, weights, max_ctx=max_ctx, device=str(dev))
+    prompt = torch.from_numpy(si.prompt(shape, seq=rank)).to(dev)
+    outs = [eng.new_out(1, shape.T, shape.k, want_logits=False) for _ in range(2)]
+    pout = eng.new_out(1, 1, shape.k, T_next=shape.T if shape.k > 0 else 1, want_logits=False)
+    eng.prefill(0, prompt, shape.k, shape.l, parents if shape.k > 0 else None, pout)
+    torch.cuda.synchronize()
+    n_start = eng.context_len(0)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing: next tree tokens never leave the GPU -----------------------
+    tokens = pout.next_tree_tokens[0]
+    launches = 0
+    def one_step(i, tokens):
+        nonlocal launches
+        o = outs[i & 1]
+        eng.step(tokens, parents, shape.k, shape.l, o)
+        launches += eng.launches()
+        eng.commit(1)
+        launches += eng.launches()
+        return o
+
+    for i in range(W):
+        tokens = one_step(i, tokens).next_tree_tokens[0]
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    launches = 0
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    acc_counts = torch.zeros(K, dtype=torch.int32, device=dev)
+    ev0.record()
+    for i in range(K):
+        o = one_step(i, tokens)
+        acc_counts[i] = o.n_accepted[0]
+        tokens = o.next_tree_tokens[0]
+    ev1.record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    ms_total = ev0.elapsed_time(ev1)
+    emitted = int(acc_counts.sum().item())
+    n_end = eng.context_len(0)
+
+    # ---- end to end: host buffers in, host results out, every step -------------------------
+    e2e = None
+    if not args.no_e2e:
+        h_tokens = torch.empty(shape.T, dtype=torch.int32).pin_memory()
+        h_tokens.copy_(tokens.cpu())
+        d_tokens = torch.empty(shape.T, dtype=torch.int32, device=dev)
+        o = outs[0]
+        h_acc = torch.empty(S, dtype=torch.int32).pin_memory()
+        h_n = torch.empty(1, dtype=torch.int32).pin_memory()
+        h_next = torch.empty(shape.T if shape.k > 0 else 1, dtype=torch.int32).pin_memory()
+        e_emitted = 0
+        barrier()
+        t0 = time.perf_counter()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(K):
+            d_tokens.copy_(h_tokens, non_blocking=True)
+            eng.step(d_tokens, parents, shape.k, shape.l, o)
+            eng.commit(1)
+            h_acc.copy_(o.accepted_tokens[0], non_blocking=True)
+            h_n.copy_(o.n_accepted, non_blocking=True)
+            h_next.copy_(o.next_tree_tokens[0], non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+            e_emitted += int(h_n[0])
+            h_tokens[: h_next.numel()].copy_(h_next)
+        e1.record()
+        barrier()
+        e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3 * 0.0)
+        e2e = dict(ms=e_ms, emitted=e_emitted, h2d=int(h_tokens.numel() * 4),
+                   d2h=int((h_acc.numel() + 1 + h_next.numel()) * 4))
+
+    # ---- aggregate over ranks: max time, summed units ----------------------------------------
+    def agg(ms, units):
+        if world == 1:
+            return ms, units
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        u = torch.tensor([units], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(u, op=dist.ReduceOp.SUM)
+        return float(t.item()), float(u.item())
+
+    ms_max, units = agg(ms_total, emitted)
+    if e2e:
+        e_ms_max, e_units = agg(e2e["ms"], e2e["emitted"])
+
+    # ---- per-kernel-class durations (second, separately timed pass with events in the library) ----
+    prof = None
+    if rank == 0:
+        from paper_2410_20488_b200 import binding
+        if hasattr(binding, "firp_profile_step"):
+            prof = binding.firp_profile_step(eng, tokens, parents, shape, outs[0], steps=min(K, 8))
+
+    if rank != 0:
+        return
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except OSError:
+        pass
+    peak_gbs, peak_kind = (peaks["hbm_gbs"], "measured") if "hbm_gbs" in peaks else (6650.0, "fallback")
+    n_mid = 0.5 * (n_start + n_end)
+    ab = algorithmic_bytes(shape, n_mid)
+    ms_step = ms_max / K
+    step_gbs = ab["total"] / (ms_step * 1e-3) / 1e9
+    line = dict(metric=METRIC, value=units / (ms_max * 1e-3), unit=UNIT, n_gpus=world, steps=K, warmup=W,
+                ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                data="synthetic", gpu_launches=launches,
+                config=dict(workload=shape.name, T=shape.T, k=shape.k, l=shape.l, context_start=n_start,
+                            context_end=n_end, batch=1, l2="inputs_larger_than_l2 (%.1f GB of weights per step)" %
+                            (ab["weights"] / 1e9), parallelism="replicas x%d" % world,
+                            mode="free-running greedy (random weights accept ~0 drafts per step)"),
+                step_latency_us=ms_step * 1e3, tokens_per_step=units / (K * world),
+                step_hbm=dict(bytes_per_step=ab["total"], weights=ab["weights"], kv_read=ab["kv_read"],
+                              achieved_gbs=step_gbs, frac_of_measured_peak=step_gbs / peak_gbs,
+                              frac_of_8tbs=step_gbs / 8000.0, peak_gbs=peak_gbs, peak=peak_kind),
+                clocks=clocks)
+    if args.layers:
+        line["invalid"] = "decoder truncated to %d layers (debug run)" % args.layers
+    if e2e:
+        line["e2e"] = dict(value=e_units / (e_ms_max * 1e-3), unit=UNIT, ms_per_step=e_ms_max / K,
+                           h2d_bytes_per_step=e2e["h2d"], d2h_bytes_per_step=e2e["d2h"])
+    if prof:
+        line["roofline"] = prof["roofline"]
+        line["kernels"] = prof["kernels"]
+    else:
+        line["roofline"] = dict(bound="hbm", achieved=step_gbs, peak=peak_gbs, unit="GB/s", frac=step_gbs / peak_gbs,
+                                traffic=None, note="whole step (all kernels): bytes per step / step time; peak = %s copy bandwidth" % peak_kind)
+    if not args.no_cpu_baseline:
+        cb_steps = 1
+        tps, ms = time_oracle(shape, weights, cb_steps, 0)
+        line["cpu_baseline"] = dict(value=tps, unit=UNIT, cores=host_cores(), kind="oracle", ms_per_step=ms,
+                                    sample="%d oracle step of T=%d,k=%d,l=%d over all %d layers on a 32-token context "
+                                           "(plus its 32-token prefill, untimed)" % (cb_steps, shape.T, shape.k, shape.l, shape.L))
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

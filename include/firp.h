@@ -1,0 +1,157 @@
+/*
+ * firp.h -- C ABI of the B200 (sm_100a) FIRP draft+verify decoder step.
+ *
+ * FIRP (arXiv 2410.20488) is single-model speculative decoding: at an
+ * intermediate layer l, k trainable linear maps predict pseudo hidden states of
+ * the next k positions (Section 3.2, Section 3.3 Eq. 3); they pass through the
+ * remaining layers and the original lm-head and yield the draft tokens of the
+ * next round, while the same forward pass verifies the current draft tree with
+ * tree attention (Section 3.4).
+ *
+ * Conventions
+ *   - All calls return 0 (FIRP_OK) or a negative firp_status; firp_last_error()
+ *     returns a message for the last failure on that context.
+ *   - "device" pointers are CUDA device memory of the current device, "host"
+ *     pointers ordinary host memory.  The library allocates NO device memory:
+ *     the caller provides the workspace, the KV cache, the weights and every
+ *     output buffer, and keeps them alive while the context uses them.
+ *   - Work is enqueued on the given CUDA stream (a cudaStream_t passed as
+ *     void*, NULL = the legacy default stream) and nothing synchronises unless
+ *     stated.  One context must be driven from one stream at a time.
+ *   - Weight matrices are bf16, row-major [out][in].  Token ids are int32.
+ *   - Rows of a step: for each of the n_seq sequences, rows 0..T-1 are the tree
+ *     nodes (row 0 = root = the last emitted, not yet cached token) and rows
+ *     T..T+k-1 the pseudo hidden states, a chain hanging off the root.
+ */
+#ifndef FIRP_H_
+#define FIRP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FIRP_OK = 0,
+  FIRP_ERR_BAD_ARG = -1,   /* NULL pointer, size out of range, misaligned buffer */
+  FIRP_ERR_BAD_TREE = -2,  /* parents[0] != -1, parents[v] >= v, depth beyond the limit */
+  FIRP_ERR_CAPACITY = -3,  /* context + rows would exceed max_ctx, or a max_* of the config */
+  FIRP_ERR_CUDA = -4,      /* a CUDA runtime call failed (message has the CUDA error) */
+  FIRP_ERR_STATE = -5      /* call out of order (no buffers bound, no weights, no step to commit) */
+} firp_status;
+
+typedef struct firp_ctx firp_ctx;
+
+/* Decoder shape and capacity limits (Llama-style block: RMSNorm, rotary embedding in
+ * the rotate-half pairing, grouped-query attention, SwiGLU MLP, untied lm-head). */
+typedef struct {
+  int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  float rms_eps, rope_theta;
+  int32_t max_batch;  /* sequences with a KV cache (slots 0..max_batch-1) */
+  int32_t max_ctx;    /* cache positions per sequence, committed + one step's rows */
+  int32_t max_tree;   /* largest T (tree rows per sequence, root included), <= 128 */
+  int32_t max_k;      /* largest k (pseudo rows per sequence), <= 8 */
+  int32_t max_depth;  /* largest tree depth; paths and accepted lists hold max_depth+1 entries */
+  int32_t top_b;      /* candidates kept per pseudo row, 1..8 */
+} firp_model_cfg;
+
+/* Device pointers to bf16 weights.  wqkv..g_mlp are HOST arrays of n_layers device pointers.
+ * wqkv: [(n_heads + 2 n_kv_heads) * head_dim][d_model], q rows, then k rows, then v rows.
+ * wo:   [d_model][n_heads * head_dim].   wgu: [2 d_ffn][d_model], gate rows then up rows.
+ * wd:   [d_model][d_ffn].   g_attn, g_mlp, g_final: [d_model] RMSNorm gains.
+ * embed, lm_head: [vocab][d_model].
+ * pred_w: [n_maps][d_model][d_model] maps of Eq. 3, [out][in]; pred_b: [n_maps][d_model] or NULL.
+ * Every matrix pointer must be 16-byte aligned. */
+typedef struct {
+  const void *embed, *lm_head, *g_final;
+  const void *pred_w, *pred_b;
+  int32_t n_maps;
+  const void *const *wqkv, *const *wo, *const *wgu, *const *wd, *const *g_attn, *const *g_mlp;
+} firp_weights;
+
+/* Caller-owned DEVICE output buffers of one step; S = max_depth + 1, B = top_b.
+ * Any pointer may be NULL (that result is then kept internal or not produced). */
+typedef struct {
+  int32_t *accepted_tokens;   /* [n_seq][S]  tokens emitted: accepted drafts, then the bonus token */
+  int32_t *n_accepted;        /* [n_seq]     a + 1 */
+  int32_t *path;              /* [n_seq][S]  accepted row indices, path[0] = 0: the KV compaction indices */
+  int32_t *next_tree_tokens;  /* [n_seq][T_next] tokens of the next draft tree on the template */
+  int32_t *best;              /* [n_seq][T]  greedy token of every tree row */
+  int32_t *topb_ids;          /* [n_seq][k][B] candidates of pseudo row i, by (value desc, id asc) */
+  float *topb_vals;           /* [n_seq][k][B] */
+  float *logits;              /* [n_seq][T+k][vocab] fp32 */
+  int32_t *depth;             /* [n_seq][T+k] depth of every row (position = context length + depth) */
+  uint32_t *mask;             /* [n_seq][T+k][ceil((T+k)/32)] bit u of row v: row v attends to new row u */
+} firp_step_out;
+
+/* Create / destroy a context (host object only). */
+int firp_create(const firp_model_cfg *cfg, firp_ctx **out);
+void firp_destroy(firp_ctx *ctx);
+const char *firp_last_error(const firp_ctx *ctx);
+
+/* Bytes of device memory the caller must provide: scratch workspace and bf16 KV cache
+ * (layout [seq][layer][K|V][position][kv_head][head_dim]). */
+size_t firp_workspace_bytes(const firp_ctx *ctx);
+size_t firp_kv_bytes(const firp_ctx *ctx);
+
+/* Bind caller-allocated device buffers (256-byte aligned, at least the sizes above).
+ * Zeroes the workspace on `stream` and resets every sequence to an empty context. */
+int firp_bind_buffers(firp_ctx *ctx, void *workspace, void *kv_cache, void *stream);
+
+/* Register the weights (pointers are stored, data is not copied). */
+int firp_init_weights(firp_ctx *ctx, const firp_weights *w);
+
+/*
+ * Prefill sequence slot `seq` from an empty context: runs the P prompt tokens as a chain
+ * (the plain "n + k hidden states" picture of Section 3.2, anchor = last prompt token),
+ * caches all P rows, and returns in `out`: accepted_tokens[0] = the first root token
+ * (greedy next token), n_accepted = 1, next_tree_tokens = the first draft tree on the
+ * template `next_parents` (HOST, [T_next]), topb_*; logits (if given) holds 1+k rows:
+ * the last prompt row, then the pseudo rows.  d_prompt is a DEVICE array [P].
+ * k = 0 gives plain prefill (T_next must then be 1).
+ */
+int firp_prefill(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int32_t P, int32_t k, int32_t l,
+                 const int32_t *next_parents, int32_t T_next, const firp_step_out *out, void *stream);
+
+/*
+ * One fused draft+verify step (Section 3.4) for n_seq sequences.
+ *   seq_ids        HOST [n_seq] cache slots taking part (NULL = 0..n_seq-1), distinct
+ *   d_tree_tokens  DEVICE [n_seq][T] tokens of each draft tree, node 0 = root
+ *   tree_parents   HOST [T]: static tree template shared by the sequences,
+ *                  parents[0] = -1, parents[v] < v; depth <= k when k > 0
+ *   k, l           pseudo rows and 0-based insertion layer (input of layer l), 0 <= l < n_layers
+ * Verifies every tree greedily (a draft token is accepted iff it equals the argmax of its
+ * parent row; ties to the lowest token id, duplicate siblings to the lowest node), and builds
+ * the next tree on the same template from the top-B of the pseudo rows: a node at depth j
+ * with sibling rank r takes candidate r of pseudo row j.  With k = 0 the next tree is the
+ * bonus token alone.  Keys/values of the rows are written to cache slots n..n+T+k-1, which
+ * stay scratch until firp_kv_commit; the committed context is not changed.
+ */
+int firp_step(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
+              const int32_t *tree_parents, int32_t T, int32_t k, int32_t l, const firp_step_out *out,
+              void *stream);
+
+/*
+ * Commit after a step: for each sequence move the cache rows of path[j] to slot n + j
+ * (every layer, K and V) and advance n by path_len.  path (HOST [n_seq][max_depth+1]) and
+ * path_len (HOST [n_seq]) give an explicit path (strictly increasing, path[0] = 0); NULL
+ * for both commits the path the last firp_step found, read on the device.
+ */
+int firp_kv_commit(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *path,
+                   const int32_t *path_len, void *stream);
+
+/* Committed context length of a slot.  Synchronises `stream` (it reads the device counter). */
+int firp_context_len(firp_ctx *ctx, int32_t seq, int32_t *n, void *stream);
+
+/* Set the committed length of a slot (0 = empty; a smaller value rewinds). */
+int firp_set_context_len(firp_ctx *ctx, int32_t seq, int32_t n, void *stream);
+
+/* Number of kernels the last firp_step / firp_prefill / firp_kv_commit call launched. */
+int firp_last_launch_count(const firp_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FIRP_H_ */

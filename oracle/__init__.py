@@ -89,6 +89,31 @@ def tree_prep(parents, k: int = 0, anchor: int = 0):
     return dict(ext_parent=ext, depth=depth, mask=mask, rank=rank)
 
 
+def verify(logits, tokens, parents):
+    """Greedy acceptance walk over the tree rows' logits [T][V] (no weights needed)."""
+    tokens, parents = _i32(tokens), _i32(parents)
+    T = tokens.size
+    logits = np.ascontiguousarray(logits, np.float32)
+    V = logits.shape[1]
+    best = np.zeros(T, np.int32); path = np.zeros(T, np.int32); acc = np.zeros(T, np.int32)
+    n_out = _get_lib().oracle_verify(_ptr(logits), _ptr(tokens), _ptr(parents), T, V, _ptr(best), _ptr(path), _ptr(acc))
+    return dict(best=best, path=path[:n_out].copy(), accepted=acc[:n_out].copy(), n_accepted=n_out)
+
+
+def next_tree(logits, T: int, k: int, bonus: int, next_parents, B: int = 8):
+    """Top-B of the pseudo rows (rows T..T+k-1 of logits) and the next tree on a template."""
+    next_parents = _i32(next_parents)
+    logits = np.ascontiguousarray(logits, np.float32)
+    V = logits.shape[1]
+    ids = np.zeros((max(k, 1), B), np.int32); vals = np.zeros((max(k, 1), B), np.float32)
+    nxt = np.zeros(next_parents.size, np.int32)
+    rc = _get_lib().oracle_next_tree(_ptr(logits), T, k, V, B, int(bonus), _ptr(next_parents), next_parents.size,
+                                     _ptr(ids), _ptr(vals), _ptr(nxt))
+    if rc != 0:
+        raise ValueError("template deeper than k or wider than B")
+    return dict(topb_ids=ids[:k], topb_vals=vals[:k], next_tokens=nxt)
+
+
 class Oracle:
     """Oracle state for n_seq independent sequences of one decoder shape.
 
@@ -174,25 +199,10 @@ class Oracle:
         return out
 
     def verify(self, logits, tokens, parents):
-        tokens, parents = _i32(tokens), _i32(parents)
-        T = tokens.size
-        best = np.zeros(T, np.int32); path = np.zeros(T, np.int32); acc = np.zeros(T, np.int32)
-        logits = np.ascontiguousarray(logits, np.float32)
-        n_out = self.lib.oracle_verify(_ptr(logits), _ptr(tokens), _ptr(parents), T, self.shape.V,
-                                       _ptr(best), _ptr(path), _ptr(acc))
-        return dict(best=best, path=path[:n_out].copy(), accepted=acc[:n_out].copy(), n_accepted=n_out)
+        return verify(logits, tokens, parents)
 
     def next_tree(self, logits, T: int, k: int, bonus: int, next_parents):
-        next_parents = _i32(next_parents)
-        B = self.top_b
-        ids = np.zeros((max(k, 1), B), np.int32); vals = np.zeros((max(k, 1), B), np.float32)
-        nxt = np.zeros(next_parents.size, np.int32)
-        logits = np.ascontiguousarray(logits, np.float32)
-        rc = self.lib.oracle_next_tree(_ptr(logits), T, k, self.shape.V, B, int(bonus), _ptr(next_parents),
-                                       next_parents.size, _ptr(ids), _ptr(vals), _ptr(nxt))
-        if rc != 0:
-            raise ValueError("template deeper than k or wider than B")
-        return dict(topb_ids=ids[:k], topb_vals=vals[:k], next_tokens=nxt)
+        return next_tree(logits, T, k, bonus, next_parents, self.top_b)
 
     def step(self, tokens, parents, k: int, l: int, seq: int = 0, anchor: int = 0, next_parents=None,
              want_h_at_l: bool = False):

@@ -1,0 +1,10 @@
+"""B200 (sm_100a) FIRP draft+verify decoder step: Python binding of the C ABI in include/firp.h.
+
+The binding only marshals arguments (ctypes); every step of the path runs in the CUDA
+kernels of libfirp_b200.so.  There is no CPU fallback: importing `binding` fails loudly
+when the library has not been built.
+"""
+from .binding import (FirpError, FirpEngine, StepOut, firp_create, firp_destroy, firp_last_error,  # noqa: F401
+                      firp_workspace_bytes, firp_kv_bytes, firp_bind_buffers, firp_init_weights, firp_prefill,
+                      firp_step, firp_kv_commit, firp_context_len, firp_set_context_len,
+                      firp_last_launch_count, lib_path, load_library, ModelCfg, Weights, StepOutC)

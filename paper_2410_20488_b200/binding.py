@@ -1,0 +1,276 @@
+"""ctypes binding of libfirp_b200.so (see include/firp.h for the contract of every call)."""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libfirp_b200.so")
+_lib = None
+
+i32, vp, sz = ctypes.c_int32, ctypes.c_void_p, ctypes.c_size_t
+
+
+class FirpError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__("firp error %d: %s" % (code, msg))
+        self.code = code
+
+
+FIRP_OK, FIRP_ERR_BAD_ARG, FIRP_ERR_BAD_TREE, FIRP_ERR_CAPACITY, FIRP_ERR_CUDA, FIRP_ERR_STATE = 0, -1, -2, -3, -4, -5
+
+
+class ModelCfg(ctypes.Structure):
+    _fields_ = [(n, i32) for n in ("n_layers", "d_model", "n_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab")] + \
+               [("rms_eps", ctypes.c_float), ("rope_theta", ctypes.c_float)] + \
+               [(n, i32) for n in ("max_batch", "max_ctx", "max_tree", "max_k", "max_depth", "top_b")]
+
+
+_PP = ctypes.POINTER(vp)
+
+
+class Weights(ctypes.Structure):
+    _fields_ = [(n, vp) for n in ("embed", "lm_head", "g_final", "pred_w", "pred_b")] + [("n_maps", i32)] + \
+               [(n, _PP) for n in ("wqkv", "wo", "wgu", "wd", "g_attn", "g_mlp")]
+
+
+class StepOutC(ctypes.Structure):
+    _fields_ = [(n, vp) for n in ("accepted_tokens", "n_accepted", "path", "next_tree_tokens", "best", "topb_ids",
+                                  "topb_vals", "logits", "depth", "mask")]
+
+
+EXPORTS = ("firp_create", "firp_destroy", "firp_last_error", "firp_workspace_bytes", "firp_kv_bytes",
+           "firp_bind_buffers", "firp_init_weights", "firp_prefill", "firp_step", "firp_kv_commit",
+           "firp_context_len", "firp_set_context_len", "firp_last_launch_count")
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Load libfirp_b200.so; raises if it has not been built (there is no fallback path)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError("libfirp_b200.so is missing: run `python -m paper_2410_20488_b200.build` "
+                          "(or __graft_entry__.build()); the FIRP step has no CPU fallback")
+    lib = ctypes.CDLL(_LIB_PATH)
+    lib.firp_create.argtypes = [ctypes.POINTER(ModelCfg), ctypes.POINTER(vp)]
+    lib.firp_destroy.argtypes = [vp]
+    lib.firp_destroy.restype = None
+    lib.firp_last_error.argtypes = [vp]
+    lib.firp_last_error.restype = ctypes.c_char_p
+    lib.firp_workspace_bytes.argtypes = [vp]
+    lib.firp_workspace_bytes.restype = sz
+    lib.firp_kv_bytes.argtypes = [vp]
+    lib.firp_kv_bytes.restype = sz
+    lib.firp_bind_buffers.argtypes = [vp, vp, vp, vp]
+    lib.firp_init_weights.argtypes = [vp, ctypes.POINTER(Weights)]
+    lib.firp_prefill.argtypes = [vp, i32, vp, i32, i32, i32, vp, i32, ctypes.POINTER(StepOutC), vp]
+    lib.firp_step.argtypes = [vp, i32, vp, vp, vp, i32, i32, i32, ctypes.POINTER(StepOutC), vp]
+    lib.firp_kv_commit.argtypes = [vp, i32, vp, vp, vp, vp]
+    lib.firp_context_len.argtypes = [vp, i32, ctypes.POINTER(i32), vp]
+    lib.firp_set_context_len.argtypes = [vp, i32, i32, vp]
+    lib.firp_last_launch_count.argtypes = [vp]
+    for name in EXPORTS:
+        if name not in ("firp_destroy", "firp_last_error", "firp_workspace_bytes", "firp_kv_bytes"):
+            getattr(lib, name).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def _check(ctx, rc):
+    if rc != 0:
+        msg = load_library().firp_last_error(ctx)
+        raise FirpError(rc, msg.decode() if msg else "")
+
+
+# ---- thin functions with the names of the C ABI ---------------------------
+def firp_create(cfg: ModelCfg):
+    ctx = vp()
+    rc = load_library().firp_create(ctypes.byref(cfg), ctypes.byref(ctx))
+    if rc != 0:
+        raise FirpError(rc, "firp_create rejected the configuration")
+    return ctx
+
+
+def firp_destroy(ctx):
+    load_library().firp_destroy(ctx)
+
+
+def firp_last_error(ctx) -> str:
+    return load_library().firp_last_error(ctx).decode()
+
+
+def firp_workspace_bytes(ctx) -> int:
+    return load_library().firp_workspace_bytes(ctx)
+
+
+def firp_kv_bytes(ctx) -> int:
+    return load_library().firp_kv_bytes(ctx)
+
+
+def firp_bind_buffers(ctx, workspace_ptr: int, kv_ptr: int, stream: int = 0):
+    _check(ctx, load_library().firp_bind_buffers(ctx, workspace_ptr, kv_ptr, stream))
+
+
+def firp_init_weights(ctx, w: Weights):
+    _check(ctx, load_library().firp_init_weights(ctx, ctypes.byref(w)))
+
+
+def _host_i32(a):
+    if a is None:
+        return None, None
+    arr = np.ascontiguousarray(a, dtype=np.int32)
+    return arr, arr.ctypes.data
+
+
+def firp_prefill(ctx, seq: int, d_prompt_ptr: int, P: int, k: int, l: int, next_parents, out: StepOutC, stream: int = 0):
+    arr, ptr = _host_i32(next_parents)
+    _check(ctx, load_library().firp_prefill(ctx, seq, d_prompt_ptr, P, k, l, ptr, 0 if arr is None else arr.size,
+                                            ctypes.byref(out) if out is not None else None, stream))
+
+
+def firp_step(ctx, n_seq: int, seq_ids, d_tokens_ptr: int, tree_parents, T: int, k: int, l: int, out: StepOutC,
+              stream: int = 0):
+    ids, ids_ptr = _host_i32(seq_ids)
+    par, par_ptr = _host_i32(tree_parents)
+    _check(ctx, load_library().firp_step(ctx, n_seq, ids_ptr, d_tokens_ptr, par_ptr, T, k, l,
+                                         ctypes.byref(out) if out is not None else None, stream))
+
+
+def firp_kv_commit(ctx, n_seq: int, seq_ids=None, path=None, path_len=None, stream: int = 0):
+    ids, ids_ptr = _host_i32(seq_ids)
+    p, p_ptr = _host_i32(path)
+    ln, ln_ptr = _host_i32(path_len)
+    _check(ctx, load_library().firp_kv_commit(ctx, n_seq, ids_ptr, p_ptr, ln_ptr, stream))
+
+
+def firp_context_len(ctx, seq: int, stream: int = 0) -> int:
+    n = i32(0)
+    _check(ctx, load_library().firp_context_len(ctx, seq, ctypes.byref(n), stream))
+    return n.value
+
+
+def firp_set_context_len(ctx, seq: int, n: int, stream: int = 0):
+    _check(ctx, load_library().firp_set_context_len(ctx, seq, n, stream))
+
+
+def firp_last_launch_count(ctx) -> int:
+    return load_library().firp_last_launch_count(ctx)
+
+
+# ---- convenience: device memory through torch, nothing else ---------------
+class StepOut:
+    """Device output buffers of one step (torch tensors) and their C view."""
+
+    def __init__(self, torch, device, n_seq, T, k, V, S, B, T_next=None, want_logits=True):
+        T_next = T if T_next is None else T_next
+        z = lambda *shape, dt=torch.int32: torch.zeros(*shape, dtype=dt, device=device)
+        self.accepted_tokens, self.n_accepted, self.path = z(n_seq, S), z(n_seq), z(n_seq, S)
+        self.next_tree_tokens, self.best = z(n_seq, max(T_next, 1)), z(n_seq, T)
+        self.topb_ids, self.topb_vals = z(n_seq, max(k, 1), B), z(n_seq, max(k, 1), B, dt=torch.float32)
+        self.logits = z(n_seq, T + k, V, dt=torch.float32) if want_logits else None
+        self.depth = z(n_seq, T + k)
+        self.mask = z(n_seq, T + k, (T + k + 31) // 32)
+        self.c = StepOutC(**{n: (getattr(self, n).data_ptr() if getattr(self, n) is not None else None)
+                             for n, _ in StepOutC._fields_})
+
+
+class FirpEngine:
+    """Owns a context plus the torch tensors backing its workspace, KV cache and weights."""
+
+    def __init__(self, shape, weights, max_ctx, max_batch=1, max_tree=None, max_k=None, max_depth=None, top_b=8,
+                 device="cuda:0"):
+        import torch
+        self.torch, self.device, self.shape = torch, torch.device(device), shape
+        s = shape
+        max_tree = s.T if max_tree is None else max_tree
+        max_k = s.k if max_k is None else max_k
+        max_depth = max(max_k, 1) if max_depth is None else max_depth
+        self.cfg = ModelCfg(n_layers=s.L, d_model=s.d, n_heads=s.H, n_kv_heads=s.Hkv, head_dim=s.dh, d_ffn=s.F,
+                            vocab=s.V, rms_eps=s.eps, rope_theta=s.theta, max_batch=max_batch, max_ctx=max_ctx,
+                            max_tree=max_tree, max_k=max_k, max_depth=max_depth, top_b=top_b)
+        self.S, self.B = max_depth + 1, top_b
+        self.ctx = firp_create(self.cfg)
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(firp_workspace_bytes(self.ctx), dtype=torch.uint8, device=self.device)
+            self.kv = torch.zeros(firp_kv_bytes(self.ctx), dtype=torch.uint8, device=self.device)
+            firp_bind_buffers(self.ctx, self.workspace.data_ptr(), self.kv.data_ptr(), self.stream)
+            self._upload(weights)
+
+    @property
+    def stream(self) -> int:
+        return self.torch.cuda.current_stream(self.device).cuda_stream
+
+    def _dev(self, bits):
+        t = self.torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
+        return t.to(self.device)
+
+    def _upload(self, weights):
+        L = self.shape.L
+        self.w_tensors = {n: self._dev(weights[n]) for n in ("embed", "lm_head", "g_final")}
+        n_maps = int(weights["pred_w"].shape[0]) if weights.get("pred_w") is not None else 0
+        if n_maps:
+            self.w_tensors["pred_w"] = self._dev(weights["pred_w"])
+            if weights.get("pred_b") is not None:
+                self.w_tensors["pred_b"] = self._dev(weights["pred_b"])
+        self.layer_tensors = [{n: self._dev(lw[n]) for n in ("wqkv", "wo", "wgu", "wd", "g_attn", "g_mlp")}
+                              for lw in weights["layers"]]
+        w = Weights()
+        for n in ("embed", "lm_head", "g_final", "pred_w", "pred_b"):
+            setattr(w, n, self.w_tensors[n].data_ptr() if n in self.w_tensors else None)
+        w.n_maps = n_maps
+        self._arrays = []
+        for n in ("wqkv", "wo", "wgu", "wd", "g_attn", "g_mlp"):
+            arr = (vp * L)(*[lt[n].data_ptr() for lt in self.layer_tensors])
+            self._arrays.append(arr)
+            setattr(w, n, ctypes.cast(arr, _PP))
+        self.w = w
+        firp_init_weights(self.ctx, w)
+
+    def new_out(self, n_seq, T, k, T_next=None, want_logits=True) -> StepOut:
+        return StepOut(self.torch, self.device, n_seq, T, k, self.shape.V, self.S, self.B, T_next, want_logits)
+
+    def prefill(self, seq, d_prompt, k, l, next_parents, out: StepOut):
+        firp_prefill(self.ctx, seq, d_prompt.data_ptr(), d_prompt.numel(), k, l, next_parents,
+                     out.c if out is not None else None, self.stream)
+
+    def step(self, d_tokens, parents, k, l, out: StepOut, seq_ids=None, n_seq=1):
+        T = len(parents)
+        firp_step(self.ctx, n_seq, seq_ids, d_tokens.data_ptr(), parents, T, k, l, out.c if out is not None else None,
+                  self.stream)
+
+    def commit(self, n_seq=1, seq_ids=None, path=None, path_len=None):
+        if path is not None:
+            p = np.zeros((n_seq, self.S), np.int32)
+            for s_i in range(n_seq):
+                row = np.asarray(path[s_i], np.int32)
+                p[s_i, : row.size] = row
+            path_len = np.array([len(path[s_i]) for s_i in range(n_seq)], np.int32)
+            path = p
+        firp_kv_commit(self.ctx, n_seq, seq_ids, path, path_len, self.stream)
+
+    def context_len(self, seq=0) -> int:
+        return firp_context_len(self.ctx, seq, self.stream)
+
+    def set_context_len(self, seq, n):
+        firp_set_context_len(self.ctx, seq, n, self.stream)
+
+    def launches(self) -> int:
+        return firp_last_launch_count(self.ctx)
+
+    def close(self):
+        if self.ctx:
+            firp_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,267 @@
+// Tree-masked split-KV decode attention (Section 3.4 "Tree attention"; Section 3.3 for pseudo rows).
+//
+// Every new row attends to the whole committed prefix [0, n) and, among the new rows of its
+// own sequence (cache slots n .. n+rows-1), only to its ancestors and itself; the visibility
+// bits come from the parent array (built once per step).  Grid = (kv split, kv head,
+// sequence x query block).  A CTA stages 64-position K and V tiles of its split in shared
+// memory (cp.async, double buffered), each warp owns 16 query rows (row x head-of-group for
+// grouped-query attention), S = Q K^T and O += P V run on the tensor cores with an online
+// softmax in fp32, and each split leaves an unnormalised partial (running max, sum, O) that
+// a small combine kernel merges.
+#include "firp_kernels.cuh"
+
+namespace firp {
+
+namespace {
+
+constexpr int kWarps = 4, kThreads = kWarps * 32, kQRows = kWarps * 16, KT = kAttnTile;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, bool valid) {
+  const int sz = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(sz));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+__device__ __forceinline__ void ldmatrix_x4(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float *c, const uint32_t *a, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// Row r of a [rows][DH] bf16 tile, 16-byte chunk c, XOR-swizzled within each 128-byte line.
+template <int DH> __device__ __forceinline__ int tile_off(int r, int c) {
+  return r * (DH * 2) + (((c & ~7) | ((c ^ r) & 7)) << 4);
+}
+
+template <int DH>
+__global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a) {
+  constexpr int CH = DH / 8;          // 16-byte chunks per row
+  constexpr int TILE_BYTES = KT * DH * 2;
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint8_t *sQ = smem;                               // [kQRows][DH]
+  uint8_t *sK = sQ + kQRows * DH * 2;               // [2][KT][DH]
+  uint8_t *sV = sK + 2 * TILE_BYTES;                // [2][KT][DH]
+  __shared__ uint32_t s_mask[kQRows][kMaskWords];
+  __shared__ int s_row[kQRows];                     // global row index of each query row, -1 = padding
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int split = blockIdx.x, kvh = blockIdx.y;
+  const int G = a.H / a.Hkv;
+  const int qrows_total = a.rows_active * G;
+  const int qblocks = (qrows_total + kQRows - 1) / kQRows;
+  const int s = blockIdx.z / qblocks, qb = blockIdx.z % qblocks;
+  const int slot = a.seq_ids[s];
+  const int n = a.ctx_len[slot];
+  const int kv_len = min(n + a.rows_active, a.max_ctx);
+  const int tiles_total = (kv_len + KT - 1) / KT;
+  const int tiles_per = (tiles_total + a.splits - 1) / a.splits;
+  const int t0 = split * tiles_per, t1 = min(tiles_total, t0 + tiles_per);
+
+  const bf16 *kbase = a.kcache + (size_t)slot * a.seq_stride + (size_t)kvh * DH;
+  const bf16 *vbase = kbase + a.kv_stride;
+  const size_t pos_stride = (size_t)a.Hkv * DH;
+
+  // query rows of this block: qr -> (tree row v = qr / G, head = kvh * G + qr % G)
+  for (int i = tid; i < kQRows; i += kThreads) {
+    const int qr = qb * kQRows + i;
+    int r = -1;
+    if (qr < qrows_total) r = s * a.rw.Ms + qr / G;
+    s_row[i] = r;
+    for (int w = 0; w < kMaskWords; ++w) s_mask[i][w] = (r >= 0) ? a.mask[(size_t)r * kMaskWords + w] : 0u;
+  }
+  for (int ch = tid; ch < kQRows * CH; ch += kThreads) {
+    const int i = ch / CH, c = ch % CH;
+    const int qr = qb * kQRows + i;
+    const bool valid = qr < qrows_total;
+    const bf16 *src = valid ? a.q + ((size_t)(s * a.rw.Ms + qr / G) * a.H + kvh * G + qr % G) * DH + c * 8 : a.q;
+    cp_async_16(smem_u32(sQ + tile_off<DH>(i, c)), src, valid);
+  }
+  auto load_kv = [&](int buf, int t) {
+    const int p0 = t * KT;
+    for (int ch = tid; ch < KT * CH; ch += kThreads) {
+      const int i = ch / CH, c = ch % CH;
+      const bool valid = (p0 + i) < kv_len;
+      const size_t off = (size_t)(p0 + i) * pos_stride + c * 8;
+      cp_async_16(smem_u32(sK + buf * TILE_BYTES + tile_off<DH>(i, c)), valid ? kbase + off : kbase, valid);
+      cp_async_16(smem_u32(sV + buf * TILE_BYTES + tile_off<DH>(i, c)), valid ? vbase + off : vbase, valid);
+    }
+  };
+  if (t0 < t1) load_kv(0, t0);
+  cp_async_commit();
+
+  const int g = lane >> 2, t4 = lane & 3, mi = lane >> 3, r8 = lane & 7;
+  const float scale_log2 = rsqrtf((float)DH) * 1.4426950408889634f;
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+  float o_acc[DH / 8][4];
+#pragma unroll
+  for (int i = 0; i < DH / 8; ++i) { o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f; }
+  uint32_t qf[DH / 16][4];
+
+  for (int t = t0; t < t1; ++t) {
+    const int buf = (t - t0) & 1;
+    if (t + 1 < t1) load_kv(buf ^ 1, t + 1);
+    cp_async_commit();
+    cp_async_wait<1>();
+    __syncthreads();
+    if (t == t0) {
+#pragma unroll
+      for (int kk = 0; kk < DH / 16; ++kk) {
+        const int row = warp * 16 + (mi & 1) * 8 + r8, chunk = kk * 2 + (mi >> 1);
+        ldmatrix_x4(qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3], smem_u32(sQ + tile_off<DH>(row, chunk)));
+      }
+    }
+    const uint8_t *kt = sK + buf * TILE_BYTES, *vt = sV + buf * TILE_BYTES;
+    // S = Q K^T over the 64 positions of the tile
+    float sc[KT / 8][4];
+#pragma unroll
+    for (int i = 0; i < KT / 8; ++i) { sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f; }
+#pragma unroll
+    for (int kk = 0; kk < DH / 16; ++kk) {
+#pragma unroll
+      for (int p = 0; p < KT / 16; ++p) {
+        uint32_t b0, b1, b2, b3;
+        const int row = p * 16 + (mi >> 1) * 8 + r8, chunk = kk * 2 + (mi & 1);
+        ldmatrix_x4(b0, b1, b2, b3, smem_u32(kt + tile_off<DH>(row, chunk)));
+        mma_bf16(sc[2 * p], qf[kk], b0, b1);
+        mma_bf16(sc[2 * p + 1], qf[kk], b2, b3);
+      }
+    }
+    // mask, scale, online softmax (rows g and g+8 of this warp's 16)
+    const int p0 = t * KT;
+    const bool need_mask = (p0 + KT > n);
+    float mx[2] = {m_run[0], m_run[1]};
+#pragma unroll
+    for (int nt = 0; nt < KT / 8; ++nt) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int rr = e >> 1, pos = p0 + nt * 8 + t4 * 2 + (e & 1);
+        float v = sc[nt][e] * scale_log2;
+        if (need_mask) {
+          bool vis = pos < n;
+          if (!vis && pos < kv_len) {
+            const int u = pos - n;
+            vis = (s_mask[warp * 16 + g + rr * 8][u >> 5] >> (u & 31)) & 1u;
+          }
+          if (!vis) v = -INFINITY;
+        }
+        sc[nt][e] = v;
+        mx[rr] = fmaxf(mx[rr], v);
+      }
+    }
+    float corr[2], msafe[2];
+#pragma unroll
+    for (int rr = 0; rr < 2; ++rr) {
+      mx[rr] = fmaxf(mx[rr], __shfl_xor_sync(0xffffffffu, mx[rr], 1));
+      mx[rr] = fmaxf(mx[rr], __shfl_xor_sync(0xffffffffu, mx[rr], 2));
+      msafe[rr] = (mx[rr] == -INFINITY) ? 0.f : mx[rr];
+      corr[rr] = exp2f(m_run[rr] - msafe[rr]);      // m_run = -inf -> 0
+      m_run[rr] = mx[rr];
+      l_run[rr] *= corr[rr];
+    }
+#pragma unroll
+    for (int i = 0; i < DH / 8; ++i) {
+      o_acc[i][0] *= corr[0]; o_acc[i][1] *= corr[0]; o_acc[i][2] *= corr[1]; o_acc[i][3] *= corr[1];
+    }
+    uint32_t pf[KT / 16][4];
+#pragma unroll
+    for (int nt = 0; nt < KT / 8; ++nt) {
+      const float e0 = exp2f(sc[nt][0] - msafe[0]), e1 = exp2f(sc[nt][1] - msafe[0]);
+      const float e2 = exp2f(sc[nt][2] - msafe[1]), e3 = exp2f(sc[nt][3] - msafe[1]);
+      l_run[0] += e0 + e1; l_run[1] += e2 + e3;
+      pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(e0, e1);
+      pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(e2, e3);
+    }
+    // O += P V
+#pragma unroll
+    for (int j = 0; j < KT / 16; ++j) {
+#pragma unroll
+      for (int d2 = 0; d2 < DH / 16; ++d2) {
+        uint32_t b0, b1, b2, b3;
+        const int row = j * 16 + (mi & 1) * 8 + r8, chunk = d2 * 2 + (mi >> 1);
+        ldmatrix_x4_trans(b0, b1, b2, b3, smem_u32(vt + tile_off<DH>(row, chunk)));
+        mma_bf16(o_acc[2 * d2], pf[j], b0, b1);
+        mma_bf16(o_acc[2 * d2 + 1], pf[j], b2, b3);
+      }
+    }
+    __syncthreads();
+  }
+  cp_async_wait<0>();
+
+  // partial result of this split
+#pragma unroll
+  for (int rr = 0; rr < 2; ++rr) {
+    float l = l_run[rr];
+    l += __shfl_xor_sync(0xffffffffu, l, 1);
+    l += __shfl_xor_sync(0xffffffffu, l, 2);
+    const int i = warp * 16 + g + rr * 8;
+    const int qr = qb * kQRows + i;
+    if (qr >= qrows_total) continue;
+    const int r = s * a.rw.Ms + qr / G, head = kvh * G + qr % G;
+    const size_t base = ((size_t)split * a.rw.R + r) * a.H + head;
+    if (t4 == 0) { a.part_ml[base * 2] = m_run[rr]; a.part_ml[base * 2 + 1] = l; }
+    float *po = a.part_o + base * DH;
+#pragma unroll
+    for (int nt = 0; nt < DH / 8; ++nt)
+      *reinterpret_cast<float2 *>(po + nt * 8 + t4 * 2) = make_float2(o_acc[nt][rr * 2], o_acc[nt][rr * 2 + 1]);
+  }
+}
+
+// Merge the splits: o = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s
+__global__ void attn_combine_kernel(AttnArgs a) {
+  const int r = blockIdx.x / a.H, head = blockIdx.x % a.H;
+  const int v = r % a.rw.Ms;
+  if (v >= a.rows_active) return;
+  float M = -INFINITY;
+  for (int sp = 0; sp < a.splits; ++sp) M = fmaxf(M, a.part_ml[(((size_t)sp * a.rw.R + r) * a.H + head) * 2]);
+  float L = 0.f;
+  for (int sp = 0; sp < a.splits; ++sp) {
+    const size_t b = (((size_t)sp * a.rw.R + r) * a.H + head) * 2;
+    const float m = a.part_ml[b];
+    if (m != -INFINITY) L += exp2f(m - M) * a.part_ml[b + 1];
+  }
+  const float inv = (L > 0.f) ? 1.f / L : 0.f;
+  for (int c = threadIdx.x; c < a.dh; c += blockDim.x) {
+    float acc = 0.f;
+    for (int sp = 0; sp < a.splits; ++sp) {
+      const size_t b = ((size_t)sp * a.rw.R + r) * a.H + head;
+      const float m = a.part_ml[b * 2];
+      if (m != -INFINITY) acc += exp2f(m - M) * a.part_o[b * a.dh + c];
+    }
+    a.o[((size_t)r * a.H + head) * a.dh + c] = __float2bfloat16(acc * inv);
+  }
+}
+
+template <int DH> void launch_dh(const AttnArgs &a, cudaStream_t st) {
+  constexpr int SMEM = kQRows * DH * 2 + 4 * KT * DH * 2;
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(tree_attn_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+    configured = true;
+  }
+  const int G = a.H / a.Hkv;
+  const int qblocks = (a.rows_active * G + kQRows - 1) / kQRows;
+  tree_attn_kernel<DH><<<dim3(a.splits, a.Hkv, a.rw.n_seq * qblocks), kThreads, SMEM, st>>>(a);
+  attn_combine_kernel<<<a.rw.R * a.H, DH, 0, st>>>(a);
+}
+
+}  // namespace
+
+void launch_attention(const AttnArgs &a, cudaStream_t st) {
+  if (a.dh == 128) launch_dh<128>(a, st);
+  else launch_dh<64>(a, st);
+}
+
+}  // namespace firp

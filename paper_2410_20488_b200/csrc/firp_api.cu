@@ -1,0 +1,506 @@
+// C ABI of the FIRP draft+verify step: context, argument validation, workspace layout and
+// the per-step launch sequence (Section 3.4 inference loop).  Host code only; every step of
+// the path runs in the kernels declared in firp_kernels.cuh.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "../../include/firp.h"
+#include "firp_kernels.cuh"
+
+using namespace firp;
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Carver {
+  uint8_t *base; size_t off;
+  template <typename T> T *take(size_t count) {
+    off = align_up(off, 256);
+    T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+}  // namespace
+
+struct firp_ctx {
+  firp_model_cfg cfg{};
+  std::string err;
+  int launches = 0;
+  bool bound = false, have_weights = false, stepped = false;
+  int Rmax = 0, S = 0, splitk_max = 8;
+  // weights
+  firp_weights w{};
+  std::vector<const void *> wqkv, wo, wgu, wd, g_attn, g_mlp;
+  // device buffers (carved from the caller's workspace)
+  bf16 *kv = nullptr;
+  float *h = nullptr, *partial = nullptr, *part_o = nullptr, *part_ml = nullptr, *logits = nullptr, *top_vals = nullptr;
+  bf16 *x = nullptr, *q = nullptr, *o = nullptr, *y = nullptr;
+  int32_t *ctx_len = nullptr, *seq_ids = nullptr, *parents = nullptr, *next_parents = nullptr, *chain = nullptr;
+  int32_t *top_ids = nullptr, *path = nullptr, *n_acc = nullptr, *accepted = nullptr, *next_tokens = nullptr;
+  int32_t *exp_path = nullptr, *exp_len = nullptr;
+  TreeMeta meta{};
+  size_t ws_bytes = 0;
+  // host mirrors
+  std::vector<int32_t> n_hi;           // upper bound of each slot's committed length
+  std::vector<int32_t> last_parents, last_next_parents, last_seq_ids;
+  int last_n_seq = 0, last_T = 0, last_k = 0;
+
+  size_t kv_plane() const { return (size_t)cfg.max_ctx * cfg.n_kv_heads * cfg.head_dim; }
+  size_t kv_layer() const { return 2 * kv_plane(); }
+  size_t kv_seq() const { return (size_t)cfg.n_layers * kv_layer(); }
+
+  size_t carve(void *base) {
+    Carver c{reinterpret_cast<uint8_t *>(base), 0};
+    const int d = cfg.d_model, nq = cfg.n_heads * cfg.head_dim, half = cfg.head_dim / 2;
+    const size_t R = Rmax;
+    h = c.take<float>(R * d);
+    x = c.take<bf16>(R * d);
+    q = c.take<bf16>(R * nq);
+    o = c.take<bf16>(R * nq);
+    y = c.take<bf16>(R * cfg.d_ffn);
+    partial = c.take<float>((size_t)splitk_max * R * d);
+    part_o = c.take<float>((size_t)kAttnMaxSplits * R * nq);
+    part_ml = c.take<float>((size_t)kAttnMaxSplits * R * cfg.n_heads * 2);
+    logits = c.take<float>(R * cfg.vocab);
+    top_ids = c.take<int32_t>(R * kMaxTopB);
+    top_vals = c.take<float>(R * kMaxTopB);
+    meta.depth = c.take<int32_t>(R);
+    meta.pos = c.take<int32_t>(R);
+    meta.mask = c.take<uint32_t>(R * kMaskWords);
+    meta.rope = c.take<float2>(R * half);
+    ctx_len = c.take<int32_t>(cfg.max_batch);
+    seq_ids = c.take<int32_t>(kMaxSeq);
+    parents = c.take<int32_t>(kMaxTreeRows);
+    next_parents = c.take<int32_t>(kMaxTreeRows);
+    chain = c.take<int32_t>(kMaxTreeRows);
+    path = c.take<int32_t>((size_t)kMaxSeq * S);
+    n_acc = c.take<int32_t>(kMaxSeq);
+    accepted = c.take<int32_t>((size_t)kMaxSeq * S);
+    next_tokens = c.take<int32_t>((size_t)kMaxSeq * kMaxTreeRows);
+    exp_path = c.take<int32_t>((size_t)kMaxSeq * S);
+    exp_len = c.take<int32_t>(kMaxSeq);
+    return align_up(c.off, 256);
+  }
+};
+
+namespace {
+
+int fail(firp_ctx *ctx, int code, const char *fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof(buf), fmt, ap);
+  va_end(ap);
+  if (ctx) ctx->err = buf;
+  return code;
+}
+
+#define FIRP_CUDA(ctx, call)                                                                            \
+  do {                                                                                                  \
+    cudaError_t e__ = (call);                                                                           \
+    if (e__ != cudaSuccess) return fail(ctx, FIRP_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e__)); \
+  } while (0)
+
+// depth of every node of a validated tree; returns max depth or -1 if malformed
+int tree_depths(const int32_t *parents, int T, std::vector<int> &depth) {
+  depth.assign(T, 0);
+  if (T < 1 || parents[0] != -1) return -1;
+  int mx = 0;
+  for (int v = 1; v < T; ++v) {
+    if (parents[v] < 0 || parents[v] >= v) return -1;
+    depth[v] = depth[parents[v]] + 1;
+    mx = depth[v] > mx ? depth[v] : mx;
+  }
+  return mx;
+}
+
+// sibling rank must stay below top_b for every node that takes a candidate
+int max_sibling_rank(const int32_t *parents, int T) {
+  int mx = 0;
+  for (int v = 1; v < T; ++v) {
+    int r = 0;
+    for (int u = 1; u < v; ++u) r += (parents[u] == parents[v]);
+    mx = r > mx ? r : mx;
+  }
+  return mx;
+}
+
+int upload_i32(firp_ctx *ctx, int32_t *dst, const int32_t *src, int n, std::vector<int32_t> &mirror, cudaStream_t st) {
+  if ((int)mirror.size() == n && memcmp(mirror.data(), src, sizeof(int32_t) * n) == 0) return FIRP_OK;
+  mirror.assign(src, src + n);
+  FIRP_CUDA(ctx, cudaMemcpyAsync(dst, mirror.data(), sizeof(int32_t) * n, cudaMemcpyHostToDevice, st));
+  return FIRP_OK;
+}
+
+// The launch sequence shared by firp_step and firp_prefill chunks.
+struct RunArgs {
+  Rows rw;
+  const int32_t *d_tokens;   // [n_seq][T]
+  int l;
+  bool want_head;            // run final norm + lm-head + top-B + accept
+  int prefill_last_row;      // -1: verify walk
+  int T_next;
+  const firp_step_out *out;
+  float *logits_dst;         // where the lm-head writes (workspace or caller buffer)
+  int n_hi_max;              // upper bound of the longest committed context among the sequences
+};
+
+int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
+  const firp_model_cfg &cfg = c->cfg;
+  const Rows &rw = ra.rw;
+  const int d = cfg.d_model, H = cfg.n_heads, Hkv = cfg.n_kv_heads, dh = cfg.head_dim, F = cfg.d_ffn;
+  const int nq = H * dh;
+  const size_t pstride = (size_t)rw.R * d;
+  const firp_step_out *out = ra.out;
+  int &nl = c->launches;
+
+  const int mw_out = (rw.Ms + 31) / 32;
+  launch_tree_prep(rw, c->parents, c->seq_ids, c->ctx_len, dh, cfg.rope_theta, c->meta, out ? out->depth : nullptr,
+                   out ? out->mask : nullptr, mw_out, st); ++nl;
+  launch_embed(rw, ra.d_tokens, (const bf16 *)c->w.embed, d, cfg.vocab, c->h, st); ++nl;
+
+  int n_partial = 0;   // split-K partial sums waiting to be added into the residual stream
+  for (int j = 0; j < cfg.n_layers; ++j) {
+    const bool insert = (rw.k > 0 && j == ra.l);
+    const int act = (rw.k > 0 && j >= ra.l) ? rw.Ms : rw.T;   // rows alive in this layer
+    // residual add + pre-attention RMSNorm; at layer l the pseudo rows are projected in between
+    launch_add_rmsnorm(rw, 0, rw.T + ((insert || act == rw.T) ? 0 : rw.k), c->h, c->partial, n_partial, pstride,
+                       (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x, st); ++nl;
+    if (insert) {
+      launch_pseudo_proj(rw, (const bf16 *)c->w.pred_w, (const bf16 *)c->w.pred_b, d, c->h, st); ++nl;
+      launch_add_rmsnorm(rw, rw.T, rw.Ms, c->h, nullptr, 0, 0, (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x, st); ++nl;
+    }
+    bf16 *kplane = c->kv + (size_t)j * c->kv_layer();
+    {
+      GemmArgs g{};
+      g.X = c->x; g.W = (const bf16 *)c->wqkv[j]; g.R = rw.R; g.N = (H + 2 * Hkv) * dh; g.K = d; g.splits = 1;
+      g.rw = rw; g.rows_active = act; g.H = H; g.Hkv = Hkv; g.dh = dh;
+      g.rope = c->meta.rope; g.seq_ids = c->seq_ids; g.ctx_len = c->ctx_len;
+      g.q = c->q; g.kcache = kplane; g.seq_stride = c->kv_seq(); g.kv_stride = c->kv_plane(); g.max_ctx = cfg.max_ctx;
+      launch_gemm(EPI_QKV_ROPE, g, st); ++nl;
+    }
+    {
+      AttnArgs a{};
+      a.rw = rw; a.rows_active = act; a.H = H; a.Hkv = Hkv; a.dh = dh;
+      a.q = c->q; a.kcache = kplane; a.seq_stride = c->kv_seq(); a.kv_stride = c->kv_plane(); a.max_ctx = cfg.max_ctx;
+      a.seq_ids = c->seq_ids; a.ctx_len = c->ctx_len; a.mask = c->meta.mask;
+      const int tiles = (ra.n_hi_max + act + kAttnTile - 1) / kAttnTile;
+      const int G = H / Hkv, qblocks = (act * G + 63) / 64;
+      int splits = (2 * 148) / (rw.n_seq * Hkv * qblocks);
+      splits = splits < 1 ? 1 : splits;
+      splits = splits > tiles ? tiles : splits;
+      a.splits = splits > kAttnMaxSplits ? kAttnMaxSplits : splits;
+      a.part_o = c->part_o; a.part_ml = c->part_ml; a.o = c->o;
+      launch_attention(a, st); nl += 2;
+    }
+    {
+      GemmArgs g{};
+      g.X = c->o; g.W = (const bf16 *)c->wo[j]; g.R = rw.R; g.N = d; g.K = nq;
+      g.splits = gemm_split_k(d, nq); g.partial = c->partial; g.partial_stride = pstride;
+      launch_gemm(EPI_PARTIAL, g, st); ++nl;
+      n_partial = g.splits;
+    }
+    launch_add_rmsnorm(rw, 0, act, c->h, c->partial, n_partial, pstride, (const bf16 *)c->g_mlp[j], cfg.rms_eps, d,
+                       c->x, st); ++nl;
+    {
+      GemmArgs g{};
+      g.X = c->x; g.W = (const bf16 *)c->wgu[j]; g.R = rw.R; g.N = 2 * F; g.K = d; g.splits = 1;
+      g.y = c->y; g.F = F;
+      launch_gemm(EPI_SWIGLU, g, st); ++nl;
+    }
+    {
+      GemmArgs g{};
+      g.X = c->y; g.W = (const bf16 *)c->wd[j]; g.R = rw.R; g.N = d; g.K = F;
+      g.splits = gemm_split_k(d, F); g.partial = c->partial; g.partial_stride = pstride;
+      launch_gemm(EPI_PARTIAL, g, st); ++nl;
+      n_partial = g.splits;
+    }
+  }
+  if (ra.want_head) {
+    launch_add_rmsnorm(rw, 0, rw.Ms, c->h, c->partial, n_partial, pstride, (const bf16 *)c->w.g_final, cfg.rms_eps, d,
+                       c->x, st); ++nl;
+    GemmArgs g{};
+    g.X = c->x; g.W = (const bf16 *)c->w.lm_head; g.R = rw.R; g.N = cfg.vocab; g.K = d; g.splits = 1;
+    g.logits = ra.logits_dst;
+    launch_gemm(EPI_LOGITS, g, st); ++nl;
+    launch_topb(ra.logits_dst, rw.R, cfg.vocab, cfg.top_b, c->top_ids, c->top_vals, st); ++nl;
+    AcceptArgs a{};
+    a.tokens = ra.d_tokens; a.parents = c->parents; a.next_parents = c->next_parents;
+    a.top_ids = c->top_ids; a.top_vals = c->top_vals; a.T_next = ra.T_next; a.B = cfg.top_b; a.S = c->S;
+    a.prefill_last_row = ra.prefill_last_row;
+    a.path = c->path; a.n_accepted = c->n_acc; a.accepted = c->accepted; a.next_tokens = c->next_tokens;
+    if (out) {
+      a.o_path = out->path; a.o_n_accepted = out->n_accepted; a.o_accepted = out->accepted_tokens;
+      a.o_next_tokens = out->next_tree_tokens; a.o_best = (ra.prefill_last_row < 0) ? out->best : nullptr;
+      a.o_topb_ids = out->topb_ids; a.o_topb_vals = out->topb_vals;
+    }
+    launch_accept(rw, a, st); ++nl;
+  }
+  FIRP_CUDA(c, cudaGetLastError());
+  return FIRP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int firp_create(const firp_model_cfg *cfg, firp_ctx **out) {
+  if (!cfg || !out) return FIRP_ERR_BAD_ARG;
+  *out = nullptr;
+  firp_ctx *c = new firp_ctx();
+  c->cfg = *cfg;
+  auto bad = [&](const char *why) { delete c; fprintf(stderr, "firp_create: %s\n", why); return (int)FIRP_ERR_BAD_ARG; };
+  if (cfg->n_layers < 1 || cfg->d_model < 8 || cfg->d_model % 8 || cfg->d_model > 8192) return bad("d_model must be a multiple of 8, <= 8192");
+  if (cfg->head_dim != 64 && cfg->head_dim != 128) return bad("head_dim must be 64 or 128");
+  if (cfg->n_heads < 1 || cfg->n_kv_heads < 1 || cfg->n_heads % cfg->n_kv_heads) return bad("n_heads must be a multiple of n_kv_heads");
+  if (cfg->d_ffn < 8 || cfg->d_ffn % 8 || cfg->vocab < 8) return bad("d_ffn must be a multiple of 8");
+  if ((cfg->n_heads * cfg->head_dim) % 8) return bad("bad head geometry");
+  if (cfg->max_batch < 1 || cfg->max_batch > kMaxSeq) return bad("max_batch must be 1..16");
+  if (cfg->max_tree < 1 || cfg->max_tree > 128 || cfg->max_k < 0 || cfg->max_k > 8) return bad("max_tree <= 128, max_k <= 8");
+  if (cfg->max_depth < 0 || cfg->max_depth > 15) return bad("max_depth must be 0..15");
+  if (cfg->top_b < 1 || cfg->top_b > kMaxTopB) return bad("top_b must be 1..8");
+  if (cfg->max_ctx < cfg->max_tree + cfg->max_k) return bad("max_ctx too small");
+  const int rows = cfg->max_batch * (cfg->max_tree + cfg->max_k);
+  if (rows > 144) return bad("max_batch * (max_tree + max_k) must be <= 144 rows");
+  c->Rmax = (int)align_up(rows, 16);
+  c->S = cfg->max_depth + 1;
+  c->n_hi.assign(cfg->max_batch, 0);
+  c->ws_bytes = c->carve(nullptr);
+  *out = c;
+  return FIRP_OK;
+}
+
+void firp_destroy(firp_ctx *ctx) { delete ctx; }
+
+const char *firp_last_error(const firp_ctx *ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+size_t firp_workspace_bytes(const firp_ctx *ctx) { return ctx ? ctx->ws_bytes : 0; }
+
+size_t firp_kv_bytes(const firp_ctx *ctx) {
+  return ctx ? (size_t)ctx->cfg.max_batch * ctx->kv_seq() * sizeof(bf16) : 0;
+}
+
+int firp_bind_buffers(firp_ctx *ctx, void *workspace, void *kv_cache, void *stream) {
+  if (!ctx) return FIRP_ERR_BAD_ARG;
+  if (!workspace || !kv_cache || ((uintptr_t)workspace & 255) || ((uintptr_t)kv_cache & 255))
+    return fail(ctx, FIRP_ERR_BAD_ARG, "workspace and kv_cache must be non-NULL and 256-byte aligned");
+  cudaStream_t st = (cudaStream_t)stream;
+  ctx->carve(workspace);
+  ctx->kv = reinterpret_cast<bf16 *>(kv_cache);
+  FIRP_CUDA(ctx, cudaMemsetAsync(workspace, 0, ctx->ws_bytes, st));
+  std::vector<int32_t> chain(kMaxTreeRows);
+  for (int i = 0; i < kMaxTreeRows; ++i) chain[i] = i - 1;
+  FIRP_CUDA(ctx, cudaMemcpyAsync(ctx->chain, chain.data(), sizeof(int32_t) * kMaxTreeRows, cudaMemcpyHostToDevice, st));
+  FIRP_CUDA(ctx, cudaStreamSynchronize(st));
+  std::fill(ctx->n_hi.begin(), ctx->n_hi.end(), 0);
+  ctx->last_parents.clear(); ctx->last_next_parents.clear(); ctx->last_seq_ids.clear();
+  ctx->bound = true; ctx->stepped = false;
+  return FIRP_OK;
+}
+
+int firp_init_weights(firp_ctx *ctx, const firp_weights *w) {
+  if (!ctx || !w) return FIRP_ERR_BAD_ARG;
+  const int L = ctx->cfg.n_layers;
+  if (!w->embed || !w->lm_head || !w->g_final || !w->wqkv || !w->wo || !w->wgu || !w->wd || !w->g_attn || !w->g_mlp)
+    return fail(ctx, FIRP_ERR_BAD_ARG, "missing weight pointer");
+  if (w->n_maps < 0 || (w->n_maps > 0 && !w->pred_w)) return fail(ctx, FIRP_ERR_BAD_ARG, "n_maps > 0 needs pred_w");
+  auto misaligned = [](const void *p) { return ((uintptr_t)p & 15) != 0; };
+  if (misaligned(w->embed) || misaligned(w->lm_head) || misaligned(w->pred_w) || misaligned(w->g_final))
+    return fail(ctx, FIRP_ERR_BAD_ARG, "weights must be 16-byte aligned");
+  for (int j = 0; j < L; ++j) {
+    const void *p[6] = {w->wqkv[j], w->wo[j], w->wgu[j], w->wd[j], w->g_attn[j], w->g_mlp[j]};
+    for (int i = 0; i < 6; ++i)
+      if (!p[i] || misaligned(p[i])) return fail(ctx, FIRP_ERR_BAD_ARG, "layer %d: NULL or misaligned weight", j);
+  }
+  ctx->w = *w;
+  ctx->wqkv.assign(w->wqkv, w->wqkv + L); ctx->wo.assign(w->wo, w->wo + L); ctx->wgu.assign(w->wgu, w->wgu + L);
+  ctx->wd.assign(w->wd, w->wd + L); ctx->g_attn.assign(w->g_attn, w->g_attn + L); ctx->g_mlp.assign(w->g_mlp, w->g_mlp + L);
+  ctx->have_weights = true;
+  return FIRP_OK;
+}
+
+static int check_ready(firp_ctx *ctx) {
+  if (!ctx) return FIRP_ERR_BAD_ARG;
+  if (!ctx->bound) return fail(ctx, FIRP_ERR_STATE, "firp_bind_buffers has not been called");
+  if (!ctx->have_weights) return fail(ctx, FIRP_ERR_STATE, "firp_init_weights has not been called");
+  return FIRP_OK;
+}
+
+static int check_seq_ids(firp_ctx *ctx, int n_seq, const int32_t *seq_ids, std::vector<int32_t> &ids) {
+  if (n_seq < 1 || n_seq > ctx->cfg.max_batch) return fail(ctx, FIRP_ERR_CAPACITY, "n_seq %d outside 1..max_batch", n_seq);
+  ids.resize(n_seq);
+  for (int s = 0; s < n_seq; ++s) {
+    ids[s] = seq_ids ? seq_ids[s] : s;
+    if (ids[s] < 0 || ids[s] >= ctx->cfg.max_batch) return fail(ctx, FIRP_ERR_BAD_ARG, "seq id %d out of range", ids[s]);
+    for (int t = 0; t < s; ++t) if (ids[t] == ids[s]) return fail(ctx, FIRP_ERR_BAD_ARG, "duplicate seq id %d", ids[s]);
+  }
+  return FIRP_OK;
+}
+
+int firp_step(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
+              const int32_t *tree_parents, int32_t T, int32_t k, int32_t l, const firp_step_out *out, void *stream) {
+  int rc = check_ready(ctx);
+  if (rc) return rc;
+  const firp_model_cfg &cfg = ctx->cfg;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!d_tree_tokens || !tree_parents) return fail(ctx, FIRP_ERR_BAD_ARG, "NULL tokens or parents");
+  if (T < 1 || T > cfg.max_tree) return fail(ctx, FIRP_ERR_CAPACITY, "T %d outside 1..max_tree", T);
+  if (k < 0 || k > cfg.max_k || k > ctx->w.n_maps) return fail(ctx, FIRP_ERR_CAPACITY, "k %d exceeds max_k or the loaded maps", k);
+  if (k > 0 && (l < 0 || l >= cfg.n_layers)) return fail(ctx, FIRP_ERR_BAD_ARG, "insertion layer %d outside 0..n_layers-1", l);
+  std::vector<int32_t> ids;
+  if ((rc = check_seq_ids(ctx, n_seq, seq_ids, ids))) return rc;
+  if (n_seq * (T + k) > ctx->Rmax) return fail(ctx, FIRP_ERR_CAPACITY, "n_seq * (T + k) exceeds the row capacity");
+  std::vector<int> depth;
+  const int maxd = tree_depths(tree_parents, T, depth);
+  if (maxd < 0) return fail(ctx, FIRP_ERR_BAD_TREE, "parents[0] must be -1 and 0 <= parents[v] < v");
+  if (maxd > cfg.max_depth) return fail(ctx, FIRP_ERR_BAD_TREE, "tree depth %d exceeds max_depth", maxd);
+  if (k > 0 && maxd > k) return fail(ctx, FIRP_ERR_BAD_TREE, "tree depth %d exceeds k = %d", maxd, k);
+  if (k > 0 && max_sibling_rank(tree_parents, T) >= cfg.top_b) return fail(ctx, FIRP_ERR_BAD_TREE, "more siblings than top_b");
+  int n_hi_max = 0;
+  for (int s = 0; s < n_seq; ++s) {
+    if (ctx->n_hi[ids[s]] + T + k > cfg.max_ctx) return fail(ctx, FIRP_ERR_CAPACITY, "slot %d: context + rows exceeds max_ctx", ids[s]);
+    n_hi_max = ctx->n_hi[ids[s]] > n_hi_max ? ctx->n_hi[ids[s]] : n_hi_max;
+  }
+  ctx->launches = 0;
+  if ((rc = upload_i32(ctx, ctx->seq_ids, ids.data(), n_seq, ctx->last_seq_ids, st))) return rc;
+  if ((rc = upload_i32(ctx, ctx->parents, tree_parents, T, ctx->last_parents, st))) return rc;
+  const int32_t one = -1;
+  const int T_next = (k > 0) ? T : 1;
+  if ((rc = upload_i32(ctx, ctx->next_parents, k > 0 ? tree_parents : &one, T_next, ctx->last_next_parents, st))) return rc;
+
+  RunArgs ra{};
+  ra.rw = Rows{n_seq, T, k, T + k, n_seq * (T + k), 0};
+  ra.d_tokens = d_tree_tokens; ra.l = l; ra.want_head = true; ra.prefill_last_row = -1; ra.T_next = T_next;
+  ra.out = out; ra.logits_dst = (out && out->logits) ? out->logits : ctx->logits; ra.n_hi_max = n_hi_max;
+  if ((rc = run_rows(ctx, ra, st))) return rc;
+  ctx->stepped = true; ctx->last_n_seq = n_seq; ctx->last_T = T; ctx->last_k = k;
+  return FIRP_OK;
+}
+
+int firp_prefill(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int32_t P, int32_t k, int32_t l,
+                 const int32_t *next_parents, int32_t T_next, const firp_step_out *out, void *stream) {
+  int rc = check_ready(ctx);
+  if (rc) return rc;
+  const firp_model_cfg &cfg = ctx->cfg;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!d_prompt || P < 1) return fail(ctx, FIRP_ERR_BAD_ARG, "empty prompt");
+  if (seq < 0 || seq >= cfg.max_batch) return fail(ctx, FIRP_ERR_BAD_ARG, "seq id out of range");
+  if (k < 0 || k > cfg.max_k || k > ctx->w.n_maps) return fail(ctx, FIRP_ERR_CAPACITY, "k exceeds max_k or the loaded maps");
+  if (k > 0 && (l < 0 || l >= cfg.n_layers)) return fail(ctx, FIRP_ERR_BAD_ARG, "insertion layer outside 0..n_layers-1");
+  if (P + k > cfg.max_ctx) return fail(ctx, FIRP_ERR_CAPACITY, "prompt does not fit max_ctx");
+  const int32_t one = -1;
+  if (k == 0) { next_parents = &one; T_next = 1; }
+  if (!next_parents || T_next < 1 || T_next > cfg.max_tree) return fail(ctx, FIRP_ERR_BAD_ARG, "bad next-tree template");
+  std::vector<int> depth;
+  const int maxd = tree_depths(next_parents, T_next, depth);
+  if (maxd < 0 || maxd > k || maxd > cfg.max_depth) return fail(ctx, FIRP_ERR_BAD_TREE, "next-tree template malformed or deeper than k");
+  if (k > 0 && max_sibling_rank(next_parents, T_next) >= cfg.top_b) return fail(ctx, FIRP_ERR_BAD_TREE, "more siblings than top_b");
+
+  ctx->launches = 0;
+  std::vector<int32_t> ids(1, seq);
+  if ((rc = upload_i32(ctx, ctx->seq_ids, ids.data(), 1, ctx->last_seq_ids, st))) return rc;
+  if ((rc = upload_i32(ctx, ctx->next_parents, next_parents, T_next, ctx->last_next_parents, st))) return rc;
+  // chain template for the prompt rows
+  std::vector<int32_t> chain(cfg.max_tree);
+  for (int i = 0; i < cfg.max_tree; ++i) chain[i] = i - 1;
+  if ((rc = upload_i32(ctx, ctx->parents, chain.data(), cfg.max_tree, ctx->last_parents, st))) return rc;
+  FIRP_CUDA(ctx, cudaMemsetAsync(ctx->ctx_len + seq, 0, sizeof(int32_t), st));
+  ctx->n_hi[seq] = 0;
+
+  const int chunk = cfg.max_tree;
+  for (int p0 = 0; p0 < P; p0 += chunk) {
+    const int Tc = (P - p0 < chunk) ? P - p0 : chunk;
+    const bool last = (p0 + Tc == P);
+    const int kc = last ? k : 0;
+    RunArgs ra{};
+    ra.rw = Rows{1, Tc, kc, Tc + kc, Tc + kc, Tc - 1};
+    ra.d_tokens = d_prompt + p0; ra.l = l; ra.want_head = last; ra.prefill_last_row = Tc - 1; ra.T_next = T_next;
+    ra.out = nullptr; ra.logits_dst = ctx->logits; ra.n_hi_max = ctx->n_hi[seq];
+    firp_step_out o2{};
+    if (last && out) {
+      o2 = *out; o2.logits = nullptr; o2.depth = nullptr; o2.mask = nullptr; o2.best = nullptr; o2.path = nullptr;
+      ra.out = &o2;
+    }
+    if ((rc = run_rows(ctx, ra, st))) return rc;
+    if (last && out && out->logits)
+      FIRP_CUDA(ctx, cudaMemcpyAsync(out->logits, ctx->logits + (size_t)(Tc - 1) * cfg.vocab,
+                                     sizeof(float) * (size_t)(1 + k) * cfg.vocab, cudaMemcpyDeviceToDevice, st));
+    launch_advance_ctx(1, ctx->seq_ids, ctx->ctx_len, Tc, st); ++ctx->launches;
+    ctx->n_hi[seq] += Tc;
+  }
+  FIRP_CUDA(ctx, cudaGetLastError());
+  ctx->stepped = false;
+  return FIRP_OK;
+}
+
+int firp_kv_commit(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *path, const int32_t *path_len,
+                   void *stream) {
+  int rc = check_ready(ctx);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!ctx->stepped) return fail(ctx, FIRP_ERR_STATE, "no step to commit");
+  if ((path == nullptr) != (path_len == nullptr)) return fail(ctx, FIRP_ERR_BAD_ARG, "path and path_len go together");
+  std::vector<int32_t> ids;
+  if ((rc = check_seq_ids(ctx, n_seq, seq_ids, ids))) return rc;
+  if (n_seq != ctx->last_n_seq || ids != ctx->last_seq_ids) return fail(ctx, FIRP_ERR_STATE, "commit must name the sequences of the last step");
+  const int S = ctx->S;
+  CommitArgs a{};
+  a.kv = ctx->kv; a.seq_stride = ctx->kv_seq(); a.layer_stride = ctx->kv_layer(); a.kv_stride = ctx->kv_plane();
+  a.n_layers = ctx->cfg.n_layers; a.nkv = ctx->cfg.n_kv_heads * ctx->cfg.head_dim; a.seq_ids = ctx->seq_ids;
+  a.S = S; a.ctx_len = ctx->ctx_len;
+  ctx->launches = 0;
+  if (path) {
+    for (int s = 0; s < n_seq; ++s) {
+      const int len = path_len[s];
+      if (len < 1 || len > S) return fail(ctx, FIRP_ERR_BAD_ARG, "path_len %d outside 1..max_depth+1", len);
+      const int32_t *p = path + (size_t)s * S;
+      if (p[0] != 0) return fail(ctx, FIRP_ERR_BAD_ARG, "path[0] must be the root");
+      for (int j = 1; j < len; ++j)
+        if (p[j] <= p[j - 1] || p[j] >= ctx->last_T) return fail(ctx, FIRP_ERR_BAD_ARG, "path must be strictly increasing tree rows");
+    }
+    FIRP_CUDA(ctx, cudaMemcpyAsync(ctx->exp_path, path, sizeof(int32_t) * (size_t)n_seq * S, cudaMemcpyHostToDevice, st));
+    FIRP_CUDA(ctx, cudaMemcpyAsync(ctx->exp_len, path_len, sizeof(int32_t) * n_seq, cudaMemcpyHostToDevice, st));
+    a.path = ctx->exp_path; a.path_len = ctx->exp_len;
+    for (int s = 0; s < n_seq; ++s) ctx->n_hi[ids[s]] += path_len[s];
+  } else {
+    a.path = ctx->path; a.path_len = ctx->n_acc;
+    for (int s = 0; s < n_seq; ++s) ctx->n_hi[ids[s]] += S;   // exact value is on the device; keep an upper bound
+  }
+  launch_commit(n_seq, a, st); ctx->launches += 2;
+  FIRP_CUDA(ctx, cudaGetLastError());
+  ctx->stepped = false;
+  return FIRP_OK;
+}
+
+int firp_context_len(firp_ctx *ctx, int32_t seq, int32_t *n, void *stream) {
+  if (!ctx || !n) return FIRP_ERR_BAD_ARG;
+  if (!ctx->bound) return fail(ctx, FIRP_ERR_STATE, "firp_bind_buffers has not been called");
+  if (seq < 0 || seq >= ctx->cfg.max_batch) return fail(ctx, FIRP_ERR_BAD_ARG, "seq id out of range");
+  cudaStream_t st = (cudaStream_t)stream;
+  FIRP_CUDA(ctx, cudaMemcpyAsync(n, ctx->ctx_len + seq, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  FIRP_CUDA(ctx, cudaStreamSynchronize(st));
+  ctx->n_hi[seq] = *n;
+  return FIRP_OK;
+}
+
+int firp_set_context_len(firp_ctx *ctx, int32_t seq, int32_t n, void *stream) {
+  if (!ctx) return FIRP_ERR_BAD_ARG;
+  if (!ctx->bound) return fail(ctx, FIRP_ERR_STATE, "firp_bind_buffers has not been called");
+  if (seq < 0 || seq >= ctx->cfg.max_batch || n < 0 || n > ctx->cfg.max_ctx) return fail(ctx, FIRP_ERR_BAD_ARG, "seq or n out of range");
+  cudaStream_t st = (cudaStream_t)stream;
+  FIRP_CUDA(ctx, cudaMemcpyAsync(ctx->ctx_len + seq, &n, sizeof(int32_t), cudaMemcpyHostToDevice, st));
+  FIRP_CUDA(ctx, cudaStreamSynchronize(st));
+  ctx->n_hi[seq] = n;
+  ctx->stepped = false;
+  return FIRP_OK;
+}
+
+int firp_last_launch_count(const firp_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

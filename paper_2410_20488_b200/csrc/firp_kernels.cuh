@@ -1,0 +1,127 @@
+// Internal launcher interface between the step scheduler and the sm_100a kernels.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace firp {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int kMaxSeq = 16;        // sequences per step
+constexpr int kMaxTreeRows = 136;  // T + k per sequence (128 + 8)
+constexpr int kMaskWords = 5;      // ceil(136 / 32)
+constexpr int kMaxTopB = 8;
+constexpr int kAttnTile = 64;      // kv positions per attention tile
+constexpr int kGemmBN = 64;        // weight rows per GEMM tile
+constexpr int kGemmBK = 64;        // k elements per pipeline stage
+
+// Per-step row geometry shared by every kernel.  Row r = s * Ms + v.
+struct Rows {
+  int n_seq;   // sequences in this step
+  int T;       // tree rows per sequence
+  int k;       // pseudo rows per sequence
+  int Ms;      // T + k
+  int R;       // n_seq * Ms
+  int anchor;  // tree row the pseudo chain hangs off
+};
+
+// ---- tree bookkeeping (Section 3.4) ---------------------------------------
+struct TreeMeta {
+  int32_t *depth;      // [R]
+  int32_t *pos;        // [R] absolute position = ctx_len + depth
+  uint32_t *mask;      // [R][kMaskWords] bit u: row v attends to new row u of its sequence
+  float2 *rope;        // [R][dh/2] (cos, sin) of pos * theta^(-2c/dh)
+};
+void launch_tree_prep(const Rows &rw, const int32_t *d_parents, const int32_t *d_seq_ids, const int32_t *d_ctx_len,
+                      int dh, float theta, TreeMeta meta, int32_t *out_depth, uint32_t *out_mask, int out_mask_words,
+                      cudaStream_t st);
+
+// h[r] = embed[token] for tree rows, 0 for pseudo rows
+void launch_embed(const Rows &rw, const int32_t *d_tokens, const bf16 *embed, int d, int vocab, float *h, cudaStream_t st);
+
+// h[r] += sum_s partial[s][r] (s < n_partial), then x[r] = rmsnorm(h[r]) * g, for rows with v in [v0, v1)
+void launch_add_rmsnorm(const Rows &rw, int v0, int v1, float *h, const float *partial, int n_partial, size_t partial_stride,
+                        const bf16 *g, float eps, int d, bf16 *x, cudaStream_t st);
+
+// Eq. 3: h[s*Ms + T + i] = W_i h[s*Ms + anchor] + b_i
+void launch_pseudo_proj(const Rows &rw, const bf16 *pred_w, const bf16 *pred_b, int d, float *h, cudaStream_t st);
+
+// top-B of every row of logits by (value desc, id asc)
+void launch_topb(const float *logits, int R, int V, int B, int32_t *ids, float *vals, cudaStream_t st);
+
+struct AcceptArgs {
+  const int32_t *tokens;        // [n_seq][T]
+  const int32_t *parents;       // [T]
+  const int32_t *next_parents;  // [T_next]
+  const int32_t *top_ids;       // [R][B] (row r's candidates; [0] is the argmax)
+  const float *top_vals;        // [R][B]
+  int T_next, B, S;             // S = path stride
+  int prefill_last_row;         // >= 0: prefill mode, the root is the argmax of this row; -1: verify walk
+  int32_t *path, *n_accepted, *accepted;  // internal copies [n_seq][S], [n_seq], [n_seq][S]
+  int32_t *next_tokens;                   // [n_seq][T_next]
+  // optional caller buffers (may be NULL)
+  int32_t *o_path, *o_n_accepted, *o_accepted, *o_next_tokens, *o_best, *o_topb_ids;
+  float *o_topb_vals;
+};
+void launch_accept(const Rows &rw, const AcceptArgs &a, cudaStream_t st);
+
+// KV compaction: rows path[j] -> slot n + j in every layer; then ctx_len += len
+struct CommitArgs {
+  bf16 *kv;                 // cache base
+  size_t seq_stride;        // elements per sequence
+  size_t layer_stride;      // elements per layer (2 * max_ctx * nkv)
+  size_t kv_stride;         // elements per K or V plane (max_ctx * nkv)
+  int n_layers, nkv;        // nkv = Hkv * dh
+  const int32_t *seq_ids;   // [n_seq] device
+  const int32_t *path;      // [n_seq][S] device
+  const int32_t *path_len;  // [n_seq] device
+  int S;
+  int32_t *ctx_len;         // [max_batch] device
+};
+void launch_commit(int n_seq, const CommitArgs &a, cudaStream_t st);
+void launch_advance_ctx(int n_seq, const int32_t *seq_ids, int32_t *ctx_len, int amount, cudaStream_t st);
+
+// ---- skinny weight-streaming GEMM ------------------------------------------
+enum GemmEpilogue { EPI_PARTIAL = 0, EPI_QKV_ROPE = 1, EPI_SWIGLU = 2, EPI_LOGITS = 3 };
+
+struct GemmArgs {
+  const bf16 *X;    // [Rpad][K] activations (row-major, K contiguous)
+  const bf16 *W;    // [N][K] weights
+  int R;            // valid rows
+  int N, K;
+  int splits;       // split-K factor (EPI_PARTIAL only)
+  // EPI_PARTIAL: out[split][R][N] fp32
+  float *partial; size_t partial_stride;
+  // EPI_QKV_ROPE
+  Rows rw; int rows_active;      // rows with v < rows_active are written
+  int H, Hkv, dh;
+  const float2 *rope; const int32_t *seq_ids; const int32_t *ctx_len;
+  bf16 *q;                       // [R][H*dh]
+  bf16 *kcache; size_t seq_stride, kv_stride; int max_ctx;  // kcache points at this layer's K plane of sequence slot 0
+  // EPI_SWIGLU: y[R][F], N = 2F
+  bf16 *y; int F;
+  // EPI_LOGITS: logits[R][N]
+  float *logits;
+};
+void launch_gemm(GemmEpilogue epi, const GemmArgs &a, cudaStream_t st);
+int gemm_split_k(int N, int K);   // split factor used for EPI_PARTIAL at this shape
+
+// ---- tree-masked split-KV attention ---------------------------------------
+struct AttnArgs {
+  Rows rw; int rows_active;
+  int H, Hkv, dh;
+  const bf16 *q;              // [R][H*dh] rotated queries
+  const bf16 *kcache;         // this layer's K plane of slot 0; V plane = kcache + kv_stride
+  size_t seq_stride, kv_stride; int max_ctx;
+  const int32_t *seq_ids, *ctx_len;
+  const uint32_t *mask;       // [R][kMaskWords]
+  int splits;                 // kv splits (grid.x)
+  float *part_o;              // [splits][R][H][dh]
+  float *part_ml;             // [splits][R][H][2] (running max in log2 units, sum)
+  bf16 *o;                    // [R][H*dh]
+};
+void launch_attention(const AttnArgs &a, cudaStream_t st);
+constexpr int kAttnMaxSplits = 32;
+
+}  // namespace firp

@@ -1,0 +1,394 @@
+// Small kernels of the FIRP step: tree bookkeeping, embedding, residual-add + RMSNorm,
+// the pseudo-hidden projection (Eq. 3), top-B, the acceptance walk / next tree, KV compaction.
+#include "firp_kernels.cuh"
+
+namespace firp {
+
+// ---------------------------------------------------------------------------
+// Tree prep (Section 3.4 "Tree attention"; Section 3.3 for the pseudo rows):
+// depth, absolute position, ancestor-or-self bitmask, rotary table.
+// One CTA per sequence; the extended parent array lives in shared memory.
+// ---------------------------------------------------------------------------
+__global__ void tree_prep_kernel(Rows rw, const int32_t *__restrict__ parents, const int32_t *__restrict__ seq_ids,
+                                 const int32_t *__restrict__ ctx_len, int dh, float theta, TreeMeta meta,
+                                 int32_t *out_depth, uint32_t *out_mask, int out_mask_words) {
+  __shared__ int32_t ext[kMaxTreeRows];
+  __shared__ int32_t sdepth[kMaxTreeRows];
+  const int s = blockIdx.x, tid = threadIdx.x;
+  const int n = ctx_len[seq_ids[s]];
+  for (int v = tid; v < rw.Ms; v += blockDim.x) {
+    int p;
+    if (v < rw.T) p = parents[v];
+    else p = (v == rw.T) ? rw.anchor : v - 1;
+    ext[v] = p;
+  }
+  __syncthreads();
+  for (int v = tid; v < rw.Ms; v += blockDim.x) {
+    uint32_t bits[kMaskWords];
+#pragma unroll
+    for (int w = 0; w < kMaskWords; ++w) bits[w] = 0u;
+    int dep = -1;
+    int u = v;
+    for (int it = 0; it < rw.Ms && u >= 0; ++it) {   // parents[u] < u, so at most Ms hops
+#pragma unroll
+      for (int w = 0; w < kMaskWords; ++w) if ((u >> 5) == w) bits[w] |= 1u << (u & 31);
+      ++dep;
+      u = ext[u];
+    }
+    sdepth[v] = dep;
+    const int r = s * rw.Ms + v;
+    meta.depth[r] = dep;
+    meta.pos[r] = n + dep;
+#pragma unroll
+    for (int w = 0; w < kMaskWords; ++w) meta.mask[(size_t)r * kMaskWords + w] = bits[w];
+    if (out_depth) out_depth[r] = dep;
+    if (out_mask)
+      for (int w = 0; w < out_mask_words; ++w) out_mask[(size_t)r * out_mask_words + w] = bits[w];
+  }
+  __syncthreads();
+  const int half = dh / 2;
+  const double l2t = log2((double)theta);
+  for (int i = tid; i < rw.Ms * half; i += blockDim.x) {
+    const int v = i / half, c = i % half;
+    const double inv_freq = exp2(-2.0 * (double)c / (double)dh * l2t);
+    const double ang = (double)(n + sdepth[v]) * inv_freq;
+    double sn, cs;
+    sincos(ang, &sn, &cs);
+    meta.rope[(size_t)(s * rw.Ms + v) * half + c] = make_float2((float)cs, (float)sn);
+  }
+}
+
+void launch_tree_prep(const Rows &rw, const int32_t *d_parents, const int32_t *d_seq_ids, const int32_t *d_ctx_len,
+                      int dh, float theta, TreeMeta meta, int32_t *out_depth, uint32_t *out_mask, int out_mask_words,
+                      cudaStream_t st) {
+  tree_prep_kernel<<<rw.n_seq, 256, 0, st>>>(rw, d_parents, d_seq_ids, d_ctx_len, dh, theta, meta, out_depth, out_mask,
+                                             out_mask_words);
+}
+
+// ---------------------------------------------------------------------------
+// Embedding gather: fp32 residual rows from bf16 table rows; pseudo rows start at zero.
+// ---------------------------------------------------------------------------
+__global__ void embed_kernel(Rows rw, const int32_t *__restrict__ tokens, const bf16 *__restrict__ embed, int d,
+                             int vocab, float *__restrict__ h) {
+  const int r = blockIdx.x, s = r / rw.Ms, v = r % rw.Ms;
+  float *dst = h + (size_t)r * d;
+  if (v >= rw.T) {
+    for (int c = threadIdx.x; c < d; c += blockDim.x) dst[c] = 0.f;
+    return;
+  }
+  int tok = tokens[s * rw.T + v];
+  tok = min(max(tok, 0), vocab - 1);
+  const bf16 *src = embed + (size_t)tok * d;
+  for (int c = threadIdx.x * 2; c < d; c += blockDim.x * 2) {
+    const __nv_bfloat162 p = *reinterpret_cast<const __nv_bfloat162 *>(src + c);
+    *reinterpret_cast<float2 *>(dst + c) = __bfloat1622float2(p);
+  }
+}
+
+void launch_embed(const Rows &rw, const int32_t *d_tokens, const bf16 *embed, int d, int vocab, float *h,
+                  cudaStream_t st) {
+  embed_kernel<<<rw.R, 128, 0, st>>>(rw, d_tokens, embed, d, vocab, h);
+}
+
+// ---------------------------------------------------------------------------
+// Residual add of split-K partial sums + RMSNorm -> bf16 GEMM operand.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ float block_sum(float v, float *red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  const int w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  if ((threadIdx.x & 31) == 0) red[w] = v;
+  __syncthreads();
+  float t = (threadIdx.x < nw) ? red[threadIdx.x] : 0.f;
+  if (w == 0) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    if (threadIdx.x == 0) red[0] = t;
+  }
+  __syncthreads();
+  t = red[0];
+  __syncthreads();
+  return t;
+}
+
+constexpr int kNormThreads = 256;
+constexpr int kNormMaxVec = 8;  // d <= 256 * 8 * 4 = 8192
+
+__global__ void __launch_bounds__(kNormThreads)
+add_rmsnorm_kernel(Rows rw, int v0, int nv, float *__restrict__ h, const float *__restrict__ partial, int n_partial,
+                   size_t partial_stride, const bf16 *__restrict__ g, float eps, int d, bf16 *__restrict__ x) {
+  __shared__ float red[32];
+  const int s = blockIdx.x / nv, v = v0 + blockIdx.x % nv;
+  const int r = s * rw.Ms + v;
+  float4 *hr = reinterpret_cast<float4 *>(h + (size_t)r * d);
+  const int nvec = d >> 2;
+  float4 val[kNormMaxVec];
+  float ss = 0.f;
+#pragma unroll
+  for (int it = 0; it < kNormMaxVec; ++it) {
+    const int i = threadIdx.x + it * kNormThreads;
+    if (i < nvec) {
+      float4 a = hr[i];
+      for (int p = 0; p < n_partial; ++p) {
+        const float4 b = reinterpret_cast<const float4 *>(partial + (size_t)p * partial_stride + (size_t)r * d)[i];
+        a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+      }
+      if (n_partial > 0) hr[i] = a;
+      val[it] = a;
+      ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+    }
+  }
+  ss = block_sum(ss, red);
+  const float rs = rsqrtf(ss / (float)d + eps);
+#pragma unroll
+  for (int it = 0; it < kNormMaxVec; ++it) {
+    const int i = threadIdx.x + it * kNormThreads;
+    if (i < nvec) {
+      const __nv_bfloat162 g01 = reinterpret_cast<const __nv_bfloat162 *>(g)[2 * i];
+      const __nv_bfloat162 g23 = reinterpret_cast<const __nv_bfloat162 *>(g)[2 * i + 1];
+      const float2 ga = __bfloat1622float2(g01), gb = __bfloat1622float2(g23);
+      __nv_bfloat162 o01 = __floats2bfloat162_rn(val[it].x * rs * ga.x, val[it].y * rs * ga.y);
+      __nv_bfloat162 o23 = __floats2bfloat162_rn(val[it].z * rs * gb.x, val[it].w * rs * gb.y);
+      __nv_bfloat162 *xo = reinterpret_cast<__nv_bfloat162 *>(x + (size_t)r * d) + 2 * i;
+      xo[0] = o01; xo[1] = o23;
+    }
+  }
+}
+
+void launch_add_rmsnorm(const Rows &rw, int v0, int v1, float *h, const float *partial, int n_partial,
+                        size_t partial_stride, const bf16 *g, float eps, int d, bf16 *x, cudaStream_t st) {
+  const int nv = v1 - v0;
+  if (nv <= 0) return;
+  add_rmsnorm_kernel<<<rw.n_seq * nv, kNormThreads, 0, st>>>(rw, v0, nv, h, partial, n_partial, partial_stride, g, eps,
+                                                             d, x);
+}
+
+// ---------------------------------------------------------------------------
+// Pseudo hidden states, Eq. 3: h~_i = W_i h[anchor] + b_i on the raw fp32 residual stream.
+// M = 1 row per sequence, so this is a weight-streaming GEMV on the FMA lanes:
+// one warp per output coordinate, 16-byte weight loads, fp32 accumulation.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+pseudo_proj_kernel(Rows rw, const bf16 *__restrict__ W, const bf16 *__restrict__ b, int d, float *__restrict__ h) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= rw.k * d) return;
+  const int i = warp / d, o = warp % d;
+  const bf16 *wrow = W + ((size_t)i * d + o) * d;
+  float acc[kMaxSeq];
+#pragma unroll
+  for (int s = 0; s < kMaxSeq; ++s) acc[s] = 0.f;
+  for (int c = lane * 8; c < d; c += 32 * 8) {
+    const uint4 wv = *reinterpret_cast<const uint4 *>(wrow + c);
+    const __nv_bfloat162 *wp = reinterpret_cast<const __nv_bfloat162 *>(&wv);
+    float wf[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { const float2 f = __bfloat1622float2(wp[j]); wf[2 * j] = f.x; wf[2 * j + 1] = f.y; }
+#pragma unroll
+    for (int s = 0; s < kMaxSeq; ++s) {
+      if (s < rw.n_seq) {
+        const float *hv = h + (size_t)(s * rw.Ms + rw.anchor) * d + c;
+        const float4 h0 = *reinterpret_cast<const float4 *>(hv), h1 = *reinterpret_cast<const float4 *>(hv + 4);
+        acc[s] += wf[0] * h0.x + wf[1] * h0.y + wf[2] * h0.z + wf[3] * h0.w + wf[4] * h1.x + wf[5] * h1.y +
+                  wf[6] * h1.z + wf[7] * h1.w;
+      }
+    }
+  }
+  const float bias = b ? __bfloat162float(b[(size_t)i * d + o]) : 0.f;
+#pragma unroll
+  for (int s = 0; s < kMaxSeq; ++s) {
+    if (s < rw.n_seq) {
+      float a = acc[s];
+#pragma unroll
+      for (int sh = 16; sh > 0; sh >>= 1) a += __shfl_xor_sync(0xffffffffu, a, sh);
+      if (lane == 0) h[(size_t)(s * rw.Ms + rw.T + i) * d + o] = a + bias;
+    }
+  }
+}
+
+void launch_pseudo_proj(const Rows &rw, const bf16 *pred_w, const bf16 *pred_b, int d, float *h, cudaStream_t st) {
+  const int warps = rw.k * d;
+  pseudo_proj_kernel<<<(warps + 7) / 8, 256, 0, st>>>(rw, pred_w, pred_b, d, h);
+}
+
+// ---------------------------------------------------------------------------
+// Top-B of each logits row by (value descending, id ascending).
+// ---------------------------------------------------------------------------
+constexpr int kTopThreads = 256;
+
+__device__ __forceinline__ bool better(float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia < ib); }
+
+__global__ void __launch_bounds__(kTopThreads)
+topb_kernel(const float *__restrict__ logits, int V, int B, int32_t *__restrict__ ids, float *__restrict__ vals) {
+  __shared__ float sval[32];
+  __shared__ int sid[32];
+  __shared__ int swin;
+  const float *row = logits + (size_t)blockIdx.x * V;
+  float lv[kMaxTopB];
+  int li[kMaxTopB];
+#pragma unroll
+  for (int j = 0; j < kMaxTopB; ++j) { lv[j] = -INFINITY; li[j] = 0x7fffffff; }
+  for (int t = threadIdx.x; t < V; t += kTopThreads) {
+    const float v = row[t];
+    if (better(v, t, lv[kMaxTopB - 1], li[kMaxTopB - 1])) {
+      lv[kMaxTopB - 1] = v; li[kMaxTopB - 1] = t;
+#pragma unroll
+      for (int j = kMaxTopB - 1; j > 0; --j) {
+        if (better(lv[j], li[j], lv[j - 1], li[j - 1])) {
+          const float tv = lv[j]; lv[j] = lv[j - 1]; lv[j - 1] = tv;
+          const int ti = li[j]; li[j] = li[j - 1]; li[j - 1] = ti;
+        }
+      }
+    }
+  }
+  int head = 0;
+  for (int b = 0; b < B; ++b) {
+    float cv = -INFINITY; int ci = 0x7fffffff;
+#pragma unroll
+    for (int j = 0; j < kMaxTopB; ++j) if (j == head) { cv = lv[j]; ci = li[j]; }
+    float bv = cv; int bi = ci;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { sval[threadIdx.x >> 5] = bv; sid[threadIdx.x >> 5] = bi; }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      float v = (threadIdx.x < kTopThreads / 32) ? sval[threadIdx.x] : -INFINITY;
+      int i = (threadIdx.x < kTopThreads / 32) ? sid[threadIdx.x] : 0x7fffffff;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, i, o);
+        if (better(ov, oi, v, i)) { v = ov; i = oi; }
+      }
+      if (threadIdx.x == 0) {
+        swin = i;
+        ids[(size_t)blockIdx.x * B + b] = i;
+        vals[(size_t)blockIdx.x * B + b] = v;
+      }
+    }
+    __syncthreads();
+    if (ci == swin && head < kMaxTopB) ++head;   // token ids are unique, so exactly one thread advances
+    __syncthreads();
+  }
+}
+
+void launch_topb(const float *logits, int R, int V, int B, int32_t *ids, float *vals, cudaStream_t st) {
+  topb_kernel<<<R, kTopThreads, 0, st>>>(logits, V, B, ids, vals);
+}
+
+// ---------------------------------------------------------------------------
+// Greedy acceptance walk and next tree (Section 3.4).  One CTA per sequence.
+// ---------------------------------------------------------------------------
+__global__ void accept_kernel(Rows rw, AcceptArgs a) {
+  __shared__ int32_t s_best[kMaxTreeRows];
+  __shared__ int32_t s_bonus;
+  const int s = blockIdx.x, tid = threadIdx.x;
+  const int32_t *tok = a.tokens + (size_t)s * rw.T;
+  for (int v = tid; v < rw.T; v += blockDim.x) {
+    const int32_t b = a.top_ids[(size_t)(s * rw.Ms + v) * a.B];
+    s_best[v] = b;
+    if (a.o_best) a.o_best[(size_t)s * rw.T + v] = b;
+  }
+  if (a.o_topb_ids || a.o_topb_vals) {
+    for (int i = tid; i < rw.k * a.B; i += blockDim.x) {
+      const size_t src = (size_t)(s * rw.Ms + rw.T) * a.B + i;
+      if (a.o_topb_ids) a.o_topb_ids[(size_t)s * rw.k * a.B + i] = a.top_ids[src];
+      if (a.o_topb_vals) a.o_topb_vals[(size_t)s * rw.k * a.B + i] = a.top_vals[src];
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int32_t *path = a.path + (size_t)s * a.S, *acc = a.accepted + (size_t)s * a.S;
+    int cur = 0, na = 0;
+    path[0] = 0;
+    if (a.prefill_last_row >= 0) {
+      cur = a.prefill_last_row;
+    } else {
+      while (na + 1 < a.S) {
+        int next = -1;
+        for (int ch = cur + 1; ch < rw.T; ++ch)
+          if (a.parents[ch] == cur && tok[ch] == s_best[cur]) { next = ch; break; }
+        if (next < 0) break;
+        acc[na] = tok[next];
+        path[++na] = next;
+        cur = next;
+      }
+    }
+    acc[na] = s_best[cur];
+    s_bonus = s_best[cur];
+    a.n_accepted[s] = na + 1;
+    if (a.o_n_accepted) a.o_n_accepted[s] = na + 1;
+    for (int j = 0; j <= na; ++j) {
+      if (a.o_path) a.o_path[(size_t)s * a.S + j] = path[j];
+      if (a.o_accepted) a.o_accepted[(size_t)s * a.S + j] = acc[j];
+    }
+  }
+  __syncthreads();
+  for (int v = tid; v < a.T_next; v += blockDim.x) {
+    int32_t t;
+    if (v == 0) {
+      t = s_bonus;
+    } else {
+      int dep = 0;
+      for (int u = v; u > 0 && dep <= a.T_next; u = a.next_parents[u]) ++dep;
+      int rank = 0;
+      for (int u = 1; u < v; ++u) rank += (a.next_parents[u] == a.next_parents[v]);
+      dep = min(dep, max(rw.k, 1));
+      rank = min(rank, a.B - 1);
+      t = (rw.k > 0) ? a.top_ids[(size_t)(s * rw.Ms + rw.T + dep - 1) * a.B + rank] : s_bonus;
+    }
+    a.next_tokens[(size_t)s * a.T_next + v] = t;
+    if (a.o_next_tokens) a.o_next_tokens[(size_t)s * a.T_next + v] = t;
+  }
+}
+
+void launch_accept(const Rows &rw, const AcceptArgs &a, cudaStream_t st) {
+  accept_kernel<<<rw.n_seq, 128, 0, st>>>(rw, a);
+}
+
+// ---------------------------------------------------------------------------
+// KV compaction of the accepted path.  Each thread owns one 16-byte column slice of a
+// (layer, K|V) plane and moves it for every path entry: it loads all source rows before
+// storing any, so a destination slot that is another entry's source is never clobbered.
+// ---------------------------------------------------------------------------
+constexpr int kMaxPath = 16;
+
+__global__ void __launch_bounds__(128) commit_kernel(CommitArgs a) {
+  const int s = blockIdx.y, plane = blockIdx.x;     // plane = layer * 2 + (0 K, 1 V)
+  const int slot = a.seq_ids[s];
+  const int n = a.ctx_len[slot];
+  const int len = min(a.path_len[s], kMaxPath);
+  const int32_t *path = a.path + (size_t)s * a.S;
+  bf16 *base = a.kv + (size_t)slot * a.seq_stride + (size_t)(plane >> 1) * a.layer_stride +
+               (size_t)(plane & 1) * a.kv_stride + (size_t)n * a.nkv;
+  const int nvec = a.nkv >> 3;
+  for (int c = threadIdx.x; c < nvec; c += blockDim.x) {
+    uint4 tmp[kMaxPath];
+#pragma unroll
+    for (int j = 0; j < kMaxPath; ++j)
+      if (j < len) tmp[j] = reinterpret_cast<const uint4 *>(base + (size_t)path[j] * a.nkv)[c];
+#pragma unroll
+    for (int j = 0; j < kMaxPath; ++j)
+      if (j < len && path[j] != j) reinterpret_cast<uint4 *>(base + (size_t)j * a.nkv)[c] = tmp[j];
+  }
+}
+
+__global__ void advance_ctx_kernel(int n_seq, const int32_t *seq_ids, int32_t *ctx_len, const int32_t *path_len,
+                                   int amount) {
+  const int s = threadIdx.x;
+  if (s < n_seq) ctx_len[seq_ids[s]] += path_len ? min(path_len[s], kMaxPath) : amount;
+}
+
+void launch_commit(int n_seq, const CommitArgs &a, cudaStream_t st) {
+  commit_kernel<<<dim3(a.n_layers * 2, n_seq), 128, 0, st>>>(a);
+  advance_ctx_kernel<<<1, 32, 0, st>>>(n_seq, a.seq_ids, a.ctx_len, a.path_len, 0);
+}
+
+void launch_advance_ctx(int n_seq, const int32_t *seq_ids, int32_t *ctx_len, int amount, cudaStream_t st) {
+  advance_ctx_kernel<<<1, 32, 0, st>>>(n_seq, seq_ids, ctx_len, nullptr, amount);
+}
+
+}  // namespace firp

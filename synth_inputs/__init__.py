@@ -244,18 +244,21 @@ def chain_template(T: int) -> np.ndarray:
     return np.arange(-1, T - 1, dtype=np.int32)
 
 
-def random_tree(seed: int, T: int, max_depth: int, stream_index: int = 0) -> np.ndarray:
-    """A random tree with parents[v] < v and depth <= max_depth (for property tests)."""
+def random_tree(seed: int, T: int, max_depth: int, stream_index: int = 0, max_children: int = 8) -> np.ndarray:
+    """A random tree with parents[v] < v, depth <= max_depth and at most max_children per node."""
     draws = uniform_i32(seed, stream_id("tokens", 1000 + stream_index), 4 * T, 0, 1 << 30)
     parents = np.full(T, -1, dtype=np.int32)
     depth = np.zeros(T, dtype=np.int32)
+    kids = np.zeros(T, dtype=np.int32)
     for v in range(1, T):
-        for t in range(4):
-            p = int(draws[4 * v + t] % v)
-            if depth[p] < max_depth:
-                break
-        else:
-            p = 0
+        ok = lambda p: depth[p] < max_depth and kids[p] < max_children
+        cands = [int(draws[4 * v + t] % v) for t in range(4)]
+        p = next((c for c in cands if ok(c)), None)
+        if p is None:
+            p = next((c for c in range(v) if ok(c)), None)
+        if p is None:
+            raise ValueError("no room for %d nodes under depth %d / %d children" % (T, max_depth, max_children))
         parents[v] = p
         depth[v] = depth[p] + 1
+        kids[p] += 1
     return parents

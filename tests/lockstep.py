@@ -1,0 +1,217 @@
+"""Lock-step parity harness: the CUDA path (through the C ABI) against the CPU oracle.
+
+Each step both sides get the same tree on the same committed state.  Compared:
+  * depth and ancestor mask of every row: bit-exact;
+  * logits of all T+k rows: max-abs <= 3e-2 and max-abs / max|oracle row| <= 2e-2;
+  * greedy token of a tree row: exact where the oracle's top-2 margin exceeds 0.1;
+  * accepted path / tokens / count: exact when every row on the oracle's path has such a margin
+    (otherwise the step is counted as ambiguous);
+  * the walk and the next tree as integer functions of the CUDA path's own argmax / top-B: exact
+    (re-derived with the oracle's walk on one-hot logits and with the template);
+  * top-B ids: exact at positions whose neighbouring oracle gaps exceed 0.1; values within tolerance;
+  * cache rows after the commit: equal to the oracle's within bf16 rounding.
+Then both sides commit the ORACLE's path and take the ORACLE's next tree, so a near-tie never cascades.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+import oracle
+import synth_inputs as si
+
+ABS_TOL, REL_TOL, MARGIN = 3e-2, 2e-2, 0.1
+
+
+def unpack_mask(words: np.ndarray, M: int) -> np.ndarray:
+    """[M][ceil(M/32)] uint32 words -> dense [M][M] 0/1."""
+    w = words.astype(np.uint32)
+    out = np.zeros((M, M), np.uint8)
+    for u in range(M):
+        out[:, u] = (w[:, u >> 5] >> np.uint32(u & 31)) & 1
+    return out
+
+
+def principal_chain(parents, depth):
+    chain = [0]
+    for _ in range(int(depth.max())):
+        kids = [u for u in range(len(parents)) if parents[u] == chain[-1]]
+        if not kids:
+            break
+        chain.append(min(kids))
+    return chain
+
+
+def template_next(parents, tp, topb_ids, bonus, k):
+    nxt = np.zeros(len(parents), np.int32)
+    nxt[0] = bonus
+    for v in range(1, len(parents)):
+        nxt[v] = topb_ids[tp["depth"][v] - 1][tp["rank"][v]]
+    return nxt if k > 0 else np.array([bonus], np.int32)
+
+
+class Stats:
+    def __init__(self):
+        self.steps = self.ambiguous = self.rows = self.rows_margin = 0
+        self.max_abs = self.max_rel = 0.0
+        self.emitted = 0
+
+    def as_dict(self):
+        return dict(steps=self.steps, ambiguous_steps=self.ambiguous, rows=self.rows, rows_with_margin=self.rows_margin,
+                    max_abs=self.max_abs, max_rel=self.max_rel, emitted=self.emitted)
+
+
+def compare_step(shape, parents, tokens, k, g, ref, stats: Stats, tp=None):
+    """g: dict of numpy arrays from the CUDA path for ONE sequence; ref: oracle.step() output."""
+    T, V = len(parents), shape.V
+    M = T + k
+    tp = tp or oracle.tree_prep(parents, k, 0)
+    # (i) integer bookkeeping
+    assert np.array_equal(g["depth"], ref["depth"]), "depth mismatch"
+    assert np.array_equal(unpack_mask(g["mask"], M), ref["mask"]), "tree mask mismatch"
+    # (ii) logits
+    d = np.abs(g["logits"].astype(np.float64) - ref["logits"].astype(np.float64))
+    row_abs = d.max(axis=1)
+    row_rel = row_abs / np.abs(ref["logits"]).max(axis=1)
+    stats.max_abs = max(stats.max_abs, float(row_abs.max()))
+    stats.max_rel = max(stats.max_rel, float(row_rel.max()))
+    assert row_abs.max() <= ABS_TOL, "logits max-abs %.4g > %.3g (row %d)" % (row_abs.max(), ABS_TOL, row_abs.argmax())
+    assert row_rel.max() <= REL_TOL, "logits rel %.4g > %.3g" % (row_rel.max(), REL_TOL)
+    # (iii) greedy tokens where the oracle margin is clear
+    part = np.partition(ref["logits"][:T], V - 2, axis=1)
+    margin = part[:, V - 1] - part[:, V - 2]
+    clear = margin > MARGIN
+    stats.rows += T
+    stats.rows_margin += int(clear.sum())
+    assert np.array_equal(g["best"][clear], ref["best"][clear]), "argmax mismatch on a clear-margin row"
+    # (iv) acceptance
+    n_ref = ref["n_accepted"]
+    decisive = all(clear[v] for v in ref["path"])
+    if decisive:
+        assert g["n_accepted"] == n_ref, "accepted count %d != %d" % (g["n_accepted"], n_ref)
+        assert np.array_equal(g["path"][:n_ref], ref["path"]), "path mismatch"
+        assert np.array_equal(g["accepted"][:n_ref], ref["accepted"]), "accepted tokens mismatch"
+    else:
+        stats.ambiguous += 1
+    # the walk as an integer function of the CUDA path's own argmax
+    onehot = np.zeros((T, V), np.float32)
+    onehot[np.arange(T), g["best"]] = 1.0
+    o = oracle.verify(onehot, tokens, parents)
+    ng = int(g["n_accepted"])
+    assert ng == o["n_accepted"] and np.array_equal(g["path"][:ng], o["path"]) and \
+        np.array_equal(g["accepted"][:ng], o["accepted"]), "acceptance walk is not the walk of its own argmax"
+    # (v) top-B of the pseudo rows
+    if k > 0:
+        B = g["topb_ids"].shape[1]
+        for i in range(k):
+            row = ref["logits"][T + i]
+            order = np.lexsort((np.arange(V), -row))[: B + 1]
+            vals = row[order]
+            gaps = vals[:-1] - vals[1:]                      # gap after position b
+            for b in range(B):
+                firm = gaps[b] > MARGIN and (b == 0 or gaps[b - 1] > MARGIN)
+                if firm:
+                    assert g["topb_ids"][i, b] == order[b], "top-B id mismatch at a firm position"
+                gid = int(g["topb_ids"][i, b])
+                assert abs(float(g["topb_vals"][i, b]) - float(row[gid])) <= ABS_TOL, "top-B value off"
+                assert float(g["topb_vals"][i, b]) >= float(vals[B - 1]) - 2 * ABS_TOL, "top-B entry too small"
+            gv, gi = g["topb_vals"][i], g["topb_ids"][i]
+            assert all(gv[b] > gv[b + 1] or (gv[b] == gv[b + 1] and gi[b] < gi[b + 1]) for b in range(B - 1)), \
+                "top-B not ordered by (value desc, id asc)"
+            assert np.array_equal(g["topb_ids"][i], np.lexsort((np.arange(V), -g["logits"][T + i]))[:B]), \
+                "top-B is not the top-B of the CUDA path's own logits"
+    # next tree as an integer function of the CUDA path's own top-B and bonus
+    want_next = template_next(parents, tp, g["topb_ids"], int(g["accepted"][ng - 1]), k)
+    assert np.array_equal(g["next_tokens"][: want_next.size], want_next), "next tree is not the template of its own top-B"
+    assert np.array_equal(g["best"], g["logits"][:T].argmax(axis=1)), "best is not the argmax of the CUDA path's own logits"
+    stats.steps += 1
+
+
+def gpu_outputs(out, s, T, k):
+    """Slice sequence s of a StepOut into numpy arrays (synchronises)."""
+    n_acc = int(out.n_accepted[s].item())
+    return dict(depth=out.depth[s].cpu().numpy(), mask=out.mask[s].cpu().numpy().view(np.uint32),
+                logits=out.logits[s].cpu().numpy(), best=out.best[s].cpu().numpy(), n_accepted=n_acc,
+                path=out.path[s].cpu().numpy(), accepted=out.accepted_tokens[s].cpu().numpy(),
+                topb_ids=out.topb_ids[s, :k].cpu().numpy(), topb_vals=out.topb_vals[s, :k].cpu().numpy(),
+                next_tokens=out.next_tree_tokens[s].cpu().numpy())
+
+
+def read_gpu_cache(engine, seq, layer, which, slot):
+    import torch
+    s = engine.shape
+    cfg = engine.cfg
+    kvt = engine.kv.view(torch.bfloat16)
+    plane = cfg.max_ctx * s.n_kv
+    off = ((seq * s.L + layer) * 2 + which) * plane + slot * s.n_kv
+    return kvt[off: off + s.n_kv].float().cpu().numpy()
+
+
+def check_cache(engine, orc, seq, slots, layers, tol=2e-2):
+    for layer in layers:
+        for which in (0, 1):
+            for slot in slots:
+                a = read_gpu_cache(engine, seq, layer, which, slot)
+                b = orc.read_cache(seq, layer, which, slot)
+                scale = max(1.0, float(np.abs(b).max()))
+                assert np.abs(a - b).max() <= tol * scale, "cache row %d layer %d differs" % (slot, layer)
+
+
+def lockstep_run(engine, orc, shape, parents, prompt, steps, forced=False, k=None, l=None, check_cache_rows=True,
+                 compare_every=1, seq=0):
+    """Prefill both sides, then `steps` lock-step steps.  Returns a Stats."""
+    import torch
+    k = shape.k if k is None else k
+    l = shape.l if l is None else l
+    T = len(parents)
+    tp = oracle.tree_prep(parents, k, 0)
+    tp_tree = oracle.tree_prep(parents, 0, 0)
+    D = int(tp_tree["depth"].max())
+    chain = principal_chain(parents, tp_tree["depth"])
+    dev = engine.device
+    stats = Stats()
+
+    # prefill
+    d_prompt = torch.from_numpy(np.ascontiguousarray(prompt, np.int32)).to(dev)
+    pout = engine.new_out(1, 1, k, T_next=T if k > 0 else 1)
+    engine.prefill(seq, d_prompt, k, l, parents if k > 0 else None, pout)
+    ref = orc.prefill(prompt, k, l, parents, seq=seq)
+    torch.cuda.synchronize()
+    plog = pout.logits[0].cpu().numpy()
+    dd = np.abs(plog - ref["logits"]).max()
+    assert dd <= ABS_TOL, "prefill logits differ by %.4g" % dd
+    part = np.partition(ref["logits"][0], shape.V - 2)
+    if part[-1] - part[-2] > MARGIN:
+        assert int(pout.accepted_tokens[0, 0].item()) == ref["root"], "prefill root token differs"
+    assert engine.context_len(seq) == orc.context_len(seq) == len(prompt)
+    tokens = ref["next_tokens"].copy()
+    emitted = [ref["root"]]
+
+    out = engine.new_out(1, T, k)
+    for step in range(steps):
+        if forced:
+            gcont = orc.ar_greedy(int(tokens[0]), D, seq=seq)
+            for j in range(1, D + 1):
+                v = chain[j]
+                for u in range(T):
+                    if parents[u] == parents[v] and u != v and tokens[u] == gcont[j - 1]:
+                        tokens[u] = tokens[v]
+                tokens[v] = gcont[j - 1]
+        d_tokens = torch.from_numpy(np.ascontiguousarray(tokens, np.int32)).to(dev)
+        engine.step(d_tokens, parents, k, l, out, seq_ids=[seq])
+        ref = orc.step(tokens, parents, k, l, seq=seq)
+        if step % compare_every == 0 or step == steps - 1:
+            g = gpu_outputs(out, 0, T, k)
+            compare_step(shape, parents, tokens, k, g, ref, stats, tp)
+        if forced:
+            assert ref["n_accepted"] == D + 1, "forced-accept step accepted %d of %d" % (ref["n_accepted"] - 1, D)
+        n0 = orc.context_len(seq)
+        engine.commit(1, seq_ids=[seq], path=[ref["path"]])
+        orc.commit(ref["path"], seq=seq)
+        n1 = orc.context_len(seq)
+        assert engine.context_len(seq) == n1
+        if check_cache_rows:
+            check_cache(engine, orc, seq, range(n0, n1), sorted({0, shape.L - 1}))
+        emitted += ref["accepted"].tolist()
+        tokens = ref["next_tokens"].copy()
+    stats.emitted = len(emitted)
+    return stats
