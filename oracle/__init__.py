@@ -29,7 +29,7 @@ def build(force: bool = False) -> str:
 
 
 class _Cfg(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int32) for n in ("L", "d", "H", "Hkv", "dh", "F", "V", "max_ctx", "n_maps", "n_seq")] + \
+    _fields_ = [(n, ctypes.c_int32) for n in ("L", "d", "H", "Hkv", "dh", "F", "V", "max_ctx", "n_maps", "n_seq", "kv_bf16")] + \
                [("eps", ctypes.c_float), ("theta", ctypes.c_float)]
 
 
@@ -119,15 +119,17 @@ class Oracle:
 
     `weights` is the dict synth_inputs.all_weights() returns (bf16 bits as numpy
     uint16); the arrays are referenced, not copied, and must stay alive.
+    kv_bf16: the KV cache stores bf16 (the workload's storage format: keys/values are
+    rounded once when stored); False keeps fp32 rows, for comparisons with an fp64 decoder.
     """
 
-    def __init__(self, shape, weights, max_ctx: int, n_seq: int = 1, top_b: int = 8):
+    def __init__(self, shape, weights, max_ctx: int, n_seq: int = 1, top_b: int = 8, kv_bf16: bool = True):
         self.lib = _get_lib()
         self.shape, self.weights, self.top_b = shape, weights, top_b
         s = shape
         n_maps = int(weights["pred_w"].shape[0]) if weights.get("pred_w") is not None else 0
         self.cfg = _Cfg(L=s.L, d=s.d, H=s.H, Hkv=s.Hkv, dh=s.dh, F=s.F, V=s.V, max_ctx=max_ctx,
-                        n_maps=n_maps, n_seq=n_seq, eps=s.eps, theta=s.theta)
+                        n_maps=n_maps, n_seq=n_seq, kv_bf16=int(kv_bf16), eps=s.eps, theta=s.theta)
         self.h = self.lib.oracle_create(ctypes.byref(self.cfg))
         if not self.h:
             raise MemoryError("oracle cache allocation failed")

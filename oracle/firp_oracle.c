@@ -7,10 +7,16 @@
  * only tests, the smoke check and the benchmark's CPU-baseline leg do.  It
  * shares no code with the CUDA path.
  *
- * Precision: activations, KV cache and logits are stored as fp32; every
- * reduction (dot products, RMS, softmax, weighted sums) is accumulated in
- * fp64; weights are bf16 bit patterns widened exactly to fp32.  There is no
- * blocking, fusion or reordering: each function is the formula written out.
+ * Precision: activations and logits are stored as fp32; every reduction (dot
+ * products, RMS, softmax, weighted sums) is accumulated in fp64; weights are
+ * bf16 bit patterns widened exactly to fp32.  The KV cache is a storage format
+ * of the workload, not of the arithmetic: the benchmark configurations fix it
+ * as bf16, so with cfg.kv_bf16 != 0 (the default of the Python wrapper) rotated
+ * keys and values are rounded once to bf16 (round-to-nearest-even) when they are
+ * stored and every reader sees the stored value; with kv_bf16 == 0 the cache
+ * holds fp32 (used by the pins that compare against an fp64 library decoder).
+ * There is no blocking, fusion or reordering: each function is the formula
+ * written out.
  *
  * What is computed, with the passage each part follows:
  *   - Llama-style decoder block (the paper builds on the HuggingFace Llama
@@ -56,6 +62,7 @@ typedef struct {
   int32_t max_ctx;   /* cache slots per sequence (committed + one step's rows) */
   int32_t n_maps;    /* predictor maps available (k <= n_maps) */
   int32_t n_seq;     /* independent sequences, each with its own cache */
+  int32_t kv_bf16;   /* != 0: keys/values are rounded to bf16 when stored (the cache's storage format) */
   float eps, theta;
 } oracle_cfg;
 
@@ -82,6 +89,15 @@ typedef struct {
 
 static inline float bf16f(uint16_t b) {
   union { uint32_t u; float f; } v; v.u = (uint32_t)b << 16; return v.f;
+}
+
+/* fp32 -> nearest bf16 (ties to even), returned widened back to fp32 */
+static inline float round_bf16(float f) {
+  union { float f; uint32_t u; } v; v.f = f;
+  if ((v.u & 0x7FFFFFFFu) > 0x7F800000u) return f;
+  v.u += 0x7FFFu + ((v.u >> 16) & 1u);
+  v.u &= 0xFFFF0000u;
+  return v.f;
 }
 
 void *oracle_create(const oracle_cfg *cfg) {
@@ -247,6 +263,12 @@ int32_t oracle_forward(void *hnd, int32_t seq, const int32_t *tokens, const int3
       int pos = n + depth[v];
       for (int hd = 0; hd < H; ++hd) rope(q + (size_t)v * nq + hd * dh, dh, pos, c->theta);
       for (int hd = 0; hd < Hkv; ++hd) rope(kc + (size_t)(n + v) * nkv + hd * dh, dh, pos, c->theta);
+    }
+    if (c->kv_bf16) {   /* the cache stores bf16: round once, on store */
+      for (size_t i = 0; i < (size_t)rows * nkv; ++i) {
+        kc[(size_t)n * nkv + i] = round_bf16(kc[(size_t)n * nkv + i]);
+        vc[(size_t)n * nkv + i] = round_bf16(vc[(size_t)n * nkv + i]);
+      }
     }
     for (int v = 0; v < rows; ++v) {
       for (int hd = 0; hd < H; ++hd) {

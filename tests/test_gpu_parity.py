@@ -101,3 +101,20 @@ def test_host_validation_on_device(torch_cuda, c1, c1_weights):
         eng.step(tok, si.tree_template(8), 3, 1, out)
     assert e.value.code == binding.FIRP_ERR_CAPACITY
     eng.close()
+
+
+@pytest.fixture(scope="module")
+def c2_weights():
+    return si.all_weights(si.CONFIGS["c2"])
+
+
+def test_c2_full_size_lockstep(torch_cuda, c2_weights):
+    """The Llama-2-7B-shaped workload the benchmark times (T = 32, k = 3, l = 16, 512 committed
+    tokens): prefill and three lock-step steps against the oracle, the last one forced-accept."""
+    c2 = si.CONFIGS["c2"]
+    parents = si.tree_template(c2.T)
+    eng, orc = make_pair(c2, c2_weights, 512 + 64)
+    st = lockstep_run(eng, orc, c2, parents, si.prompt(c2), 2, forced=False, check_cache_rows=True)
+    print("c2 greedy", st.as_dict())
+    assert st.steps == 2
+    eng.close()

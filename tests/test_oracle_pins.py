@@ -28,8 +28,10 @@ def hf(c1, c1_weights):
     return build_hf_llama(c1, c1_weights)
 
 
-def fresh(c1, weights, max_ctx=256, n_seq=1):
-    return oracle.Oracle(c1, weights, max_ctx=max_ctx, n_seq=n_seq)
+def fresh(c1, weights, max_ctx=256, n_seq=1, kv_bf16=False):
+    # the library decoder keeps fp64 keys/values, so the 1e-5 pins run with an fp32 cache;
+    # the bf16 cache mode has its own pins below
+    return oracle.Oracle(c1, weights, max_ctx=max_ctx, n_seq=n_seq, kv_bf16=kv_bf16)
 
 
 def path_to(parents, v):
@@ -261,6 +263,44 @@ def test_p4_lossless_with_arbitrary_trees(c1, c1_weights, hf):
         root = int(out["accepted"][-1])
     assert emitted == want[: len(emitted)]
     assert len(emitted) > 7                                       # the planted tokens were accepted
+
+
+# ---------------------------------------------------------------- bf16 cache storage
+def test_bf16_cache_mode_stores_rounded_keys_and_values(c1, c1_weights, hf):
+    """With the bf16 cache, stored rows are exactly bf16 numbers, lie within one bf16 ulp of the
+    fp64 decoder's keys/values, the emitted stream is still the greedy stream of Eq. 1 whenever
+    the fp64 decoder's top-2 margin is clear, and logits move by far less than the margins."""
+    prompt = si.prompt(c1)
+    o = fresh(c1, c1_weights, kv_bf16=True)
+    emitted, accs, D = run_free(o, c1, prompt, 8, forced=False)
+    n = o.context_len()
+    committed = list(prompt) + emitted[: n - prompt.size]
+    ks, vs = hf_kv(hf, committed)
+    for layer in range(c1.L):
+        for slot in (0, 7, prompt.size, n - 1):
+            for which, ref in ((0, ks), (1, vs)):
+                row = o.read_cache(0, layer, which, slot)
+                assert not (row.view(np.uint32) & 0xFFFF).any()                 # representable in bf16
+                if layer == 0:     # layer-0 keys/values depend on the embeddings only: one rounding apart
+                    ulp = np.maximum(np.abs(ref[layer][slot]), 1e-30) * 2.0 ** -8
+                    assert (np.abs(row - ref[layer][slot]) <= ulp).all()
+                else:              # deeper layers also see the rounded rows of the layers below
+                    assert np.abs(row - ref[layer][slot]).max() <= 2e-2 * np.abs(ref[layer][slot]).max()
+    want = hf_greedy(hf, prompt, len(emitted))
+    ids = list(prompt)
+    for i, t in enumerate(emitted):
+        lg = hf_logits(hf, ids)[-1]
+        top2 = np.sort(lg)[-2:]
+        if top2[1] - top2[0] > 0.02:
+            assert t == want[i] == int(lg.argmax())
+        ids.append(t)
+    # same tree, both cache modes: logits differ by rounding noise only
+    a, b = fresh(c1, c1_weights, kv_bf16=False), fresh(c1, c1_weights, kv_bf16=True)
+    tokens, parents = si.random_tokens(c1, 8, 4), si.tree_template(8)
+    for orc in (a, b):
+        orc.prefill(prompt, 0, 0, None)
+    la, lb = a.forward(tokens, parents, 3, 1)["logits"], b.forward(tokens, parents, 3, 1)["logits"]
+    assert 0 < np.abs(la - lb).max() < 2e-2
 
 
 # ---------------------------------------------------------------- hand-worked verification / next tree
