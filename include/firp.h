@@ -39,7 +39,8 @@ typedef enum {
   FIRP_ERR_BAD_TREE = -2,  /* parents[0] != -1, parents[v] >= v, depth beyond the limit */
   FIRP_ERR_CAPACITY = -3,  /* context + rows would exceed max_ctx, or a max_* of the config */
   FIRP_ERR_CUDA = -4,      /* a CUDA runtime call failed (message has the CUDA error) */
-  FIRP_ERR_STATE = -5      /* call out of order (no buffers bound, no weights, no step to commit) */
+  FIRP_ERR_STATE = -5,     /* call out of order (no buffers bound, no weights, no step to commit) */
+  FIRP_ERR_DEVICE_TIMEOUT = -6 /* a kernel's bounded wait ran out; results since the last check are invalid */
 } firp_status;
 
 typedef struct firp_ctx firp_ctx;
@@ -142,7 +143,8 @@ int firp_step(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_
 int firp_kv_commit(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *path,
                    const int32_t *path_len, void *stream);
 
-/* Committed context length of a slot.  Synchronises `stream` (it reads the device counter). */
+/* Committed context length of a slot.  Synchronises `stream` (it reads the device counter) and
+ * also reads the device status word: FIRP_ERR_DEVICE_TIMEOUT if any kernel gave up a wait. */
 int firp_context_len(firp_ctx *ctx, int32_t seq, int32_t *n, void *stream);
 
 /* Set the committed length of a slot (0 = empty; a smaller value rewinds). */

@@ -20,6 +20,7 @@ class FirpError(RuntimeError):
 
 
 FIRP_OK, FIRP_ERR_BAD_ARG, FIRP_ERR_BAD_TREE, FIRP_ERR_CAPACITY, FIRP_ERR_CUDA, FIRP_ERR_STATE = 0, -1, -2, -3, -4, -5
+FIRP_ERR_DEVICE_TIMEOUT = -6
 
 
 class ModelCfg(ctypes.Structure):

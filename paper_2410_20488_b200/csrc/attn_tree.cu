@@ -7,7 +7,9 @@
 // memory (cp.async, double buffered), each warp owns 16 query rows (row x head-of-group for
 // grouped-query attention), S = Q K^T and O += P V run on the tensor cores with an online
 // softmax in fp32, and each split leaves an unnormalised partial (running max, sum, O) that
-// a small combine kernel merges.
+// a small combine kernel merges.  Queries and probabilities enter the tensor cores as bf16
+// (hi, lo) pairs accumulated into the same fp32 accumulators, so the only bf16 rounding on this
+// path is the cache's own storage format.
 #include "firp_kernels.cuh"
 
 namespace firp {
@@ -51,8 +53,9 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a) {
   constexpr int CH = DH / 8;          // 16-byte chunks per row
   constexpr int TILE_BYTES = KT * DH * 2;
   extern __shared__ __align__(128) uint8_t smem[];
-  uint8_t *sQ = smem;                               // [kQRows][DH]
-  uint8_t *sK = sQ + kQRows * DH * 2;               // [2][KT][DH]
+  uint8_t *sQ = smem;                               // [2 planes][kQRows][DH]
+  constexpr int Q_BYTES = kQRows * DH * 2;
+  uint8_t *sK = sQ + 2 * Q_BYTES;                   // [2][KT][DH]
   uint8_t *sV = sK + 2 * TILE_BYTES;                // [2][KT][DH]
   __shared__ uint32_t s_mask[kQRows][kMaskWords];
   __shared__ int s_row[kQRows];                     // global row index of each query row, -1 = padding
@@ -88,6 +91,7 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a) {
     const bool valid = qr < qrows_total;
     const bf16 *src = valid ? a.q + ((size_t)(s * a.rw.Ms + qr / G) * a.H + kvh * G + qr % G) * DH + c * 8 : a.q;
     cp_async_16(smem_u32(sQ + tile_off<DH>(i, c)), src, valid);
+    cp_async_16(smem_u32(sQ + Q_BYTES + tile_off<DH>(i, c)), valid ? src + a.q_lo_off : a.q, valid);
   }
   auto load_kv = [&](int buf, int t) {
     const int p0 = t * KT;
@@ -108,7 +112,6 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a) {
   float o_acc[DH / 8][4];
 #pragma unroll
   for (int i = 0; i < DH / 8; ++i) { o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f; }
-  uint32_t qf[DH / 16][4];
 
   for (int t = t0; t < t1; ++t) {
     const int buf = (t - t0) & 1;
@@ -116,13 +119,6 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a) {
     cp_async_commit();
     cp_async_wait<1>();
     __syncthreads();
-    if (t == t0) {
-#pragma unroll
-      for (int kk = 0; kk < DH / 16; ++kk) {
-        const int row = warp * 16 + (mi & 1) * 8 + r8, chunk = kk * 2 + (mi >> 1);
-        ldmatrix_x4(qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3], smem_u32(sQ + tile_off<DH>(row, chunk)));
-      }
-    }
     const uint8_t *kt = sK + buf * TILE_BYTES, *vt = sV + buf * TILE_BYTES;
     // S = Q K^T over the 64 positions of the tile
     float sc[KT / 8][4];
@@ -130,13 +126,21 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a) {
     for (int i = 0; i < KT / 8; ++i) { sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f; }
 #pragma unroll
     for (int kk = 0; kk < DH / 16; ++kk) {
+      uint32_t qh[4], ql[4];
+      {
+        const int row = warp * 16 + (mi & 1) * 8 + r8, chunk = kk * 2 + (mi >> 1);
+        ldmatrix_x4(qh[0], qh[1], qh[2], qh[3], smem_u32(sQ + tile_off<DH>(row, chunk)));
+        ldmatrix_x4(ql[0], ql[1], ql[2], ql[3], smem_u32(sQ + Q_BYTES + tile_off<DH>(row, chunk)));
+      }
 #pragma unroll
       for (int p = 0; p < KT / 16; ++p) {
         uint32_t b0, b1, b2, b3;
         const int row = p * 16 + (mi >> 1) * 8 + r8, chunk = kk * 2 + (mi & 1);
         ldmatrix_x4(b0, b1, b2, b3, smem_u32(kt + tile_off<DH>(row, chunk)));
-        mma_bf16(sc[2 * p], qf[kk], b0, b1);
-        mma_bf16(sc[2 * p + 1], qf[kk], b2, b3);
+        mma_bf16(sc[2 * p], qh, b0, b1);
+        mma_bf16(sc[2 * p + 1], qh, b2, b3);
+        mma_bf16(sc[2 * p], ql, b0, b1);
+        mma_bf16(sc[2 * p + 1], ql, b2, b3);
       }
     }
     // mask, scale, online softmax (rows g and g+8 of this warp's 16)
@@ -175,14 +179,18 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a) {
     for (int i = 0; i < DH / 8; ++i) {
       o_acc[i][0] *= corr[0]; o_acc[i][1] *= corr[0]; o_acc[i][2] *= corr[1]; o_acc[i][3] *= corr[1];
     }
-    uint32_t pf[KT / 16][4];
+    uint32_t pf[KT / 16][4], pl[KT / 16][4];   // probabilities as bf16 hi and lo halves
 #pragma unroll
     for (int nt = 0; nt < KT / 8; ++nt) {
       const float e0 = exp2f(sc[nt][0] - msafe[0]), e1 = exp2f(sc[nt][1] - msafe[0]);
       const float e2 = exp2f(sc[nt][2] - msafe[1]), e3 = exp2f(sc[nt][3] - msafe[1]);
       l_run[0] += e0 + e1; l_run[1] += e2 + e3;
-      pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(e0, e1);
-      pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(e2, e3);
+      const __nv_bfloat162 h01 = __floats2bfloat162_rn(e0, e1), h23 = __floats2bfloat162_rn(e2, e3);
+      const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
+      pf[nt >> 1][(nt & 1) * 2 + 0] = *reinterpret_cast<const uint32_t *>(&h01);
+      pf[nt >> 1][(nt & 1) * 2 + 1] = *reinterpret_cast<const uint32_t *>(&h23);
+      pl[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(e0 - f01.x, e1 - f01.y);
+      pl[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(e2 - f23.x, e3 - f23.y);
     }
     // O += P V
 #pragma unroll
@@ -194,6 +202,8 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a) {
         ldmatrix_x4_trans(b0, b1, b2, b3, smem_u32(vt + tile_off<DH>(row, chunk)));
         mma_bf16(o_acc[2 * d2], pf[j], b0, b1);
         mma_bf16(o_acc[2 * d2 + 1], pf[j], b2, b3);
+        mma_bf16(o_acc[2 * d2], pl[j], b0, b1);
+        mma_bf16(o_acc[2 * d2 + 1], pl[j], b2, b3);
       }
     }
     __syncthreads();
@@ -240,12 +250,16 @@ __global__ void attn_combine_kernel(AttnArgs a) {
       const float m = a.part_ml[b * 2];
       if (m != -INFINITY) acc += exp2f(m - M) * a.part_o[b * a.dh + c];
     }
-    a.o[((size_t)r * a.H + head) * a.dh + c] = __float2bfloat16(acc * inv);
+    const float val = acc * inv;
+    const bf16 hi = __float2bfloat16_rn(val);
+    const size_t idx = ((size_t)r * a.H + head) * a.dh + c;
+    a.o[idx] = hi;
+    a.o[a.o_lo_off + idx] = __float2bfloat16_rn(val - __bfloat162float(hi));
   }
 }
 
 template <int DH> void launch_dh(const AttnArgs &a, cudaStream_t st) {
-  constexpr int SMEM = kQRows * DH * 2 + 4 * KT * DH * 2;
+  constexpr int SMEM = 2 * kQRows * DH * 2 + 4 * KT * DH * 2;
   static bool configured = false;
   if (!configured) {
     cudaFuncSetAttribute(tree_attn_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);

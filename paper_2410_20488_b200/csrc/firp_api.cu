@@ -3,6 +3,7 @@
 // the path runs in the kernels declared in firp_kernels.cuh.
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <string>
 #include <vector>
@@ -34,6 +35,8 @@ struct firp_ctx {
   int launches = 0;
   bool bound = false, have_weights = false, stepped = false;
   int Rmax = 0, S = 0, splitk_max = 8;
+  bool use_tc = true, use_pdl = true;   // tcgen05/TMA GEMM, programmatic dependent launch
+  int *dev_status = nullptr;            // device status word (bounded waits report here)
   // weights
   firp_weights w{};
   std::vector<const void *> wqkv, wo, wgu, wd, g_attn, g_mlp;
@@ -60,10 +63,10 @@ struct firp_ctx {
     const int d = cfg.d_model, nq = cfg.n_heads * cfg.head_dim, half = cfg.head_dim / 2;
     const size_t R = Rmax;
     h = c.take<float>(R * d);
-    x = c.take<bf16>(R * d);
-    q = c.take<bf16>(R * nq);
-    o = c.take<bf16>(R * nq);
-    y = c.take<bf16>(R * cfg.d_ffn);
+    x = c.take<bf16>(2 * R * d);            // activations: hi plane, then lo plane
+    q = c.take<bf16>(2 * R * nq);
+    o = c.take<bf16>(2 * R * nq);
+    y = c.take<bf16>(2 * R * cfg.d_ffn);
     partial = c.take<float>((size_t)splitk_max * R * d);
     part_o = c.take<float>((size_t)kAttnMaxSplits * R * nq);
     part_ml = c.take<float>((size_t)kAttnMaxSplits * R * cfg.n_heads * 2);
@@ -85,6 +88,7 @@ struct firp_ctx {
     next_tokens = c.take<int32_t>((size_t)kMaxSeq * kMaxTreeRows);
     exp_path = c.take<int32_t>((size_t)kMaxSeq * S);
     exp_len = c.take<int32_t>(kMaxSeq);
+    dev_status = c.take<int>(1);
     return align_up(c.off, 256);
   }
 };
@@ -157,8 +161,10 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   const int d = cfg.d_model, H = cfg.n_heads, Hkv = cfg.n_kv_heads, dh = cfg.head_dim, F = cfg.d_ffn;
   const int nq = H * dh;
   const size_t pstride = (size_t)rw.R * d;
+  const size_t Rp = (size_t)c->Rmax;          // rows per activation plane
   const firp_step_out *out = ra.out;
   int &nl = c->launches;
+  const bool tc = c->use_tc, pdl = c->use_tc && c->use_pdl;
 
   const int mw_out = (rw.Ms + 31) / 32;
   launch_tree_prep(rw, c->parents, c->seq_ids, c->ctx_len, dh, cfg.rope_theta, c->meta, out ? out->depth : nullptr,
@@ -171,24 +177,26 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     const int act = (rw.k > 0 && j >= ra.l) ? rw.Ms : rw.T;   // rows alive in this layer
     // residual add + pre-attention RMSNorm; at layer l the pseudo rows are projected in between
     launch_add_rmsnorm(rw, 0, rw.T + ((insert || act == rw.T) ? 0 : rw.k), c->h, c->partial, n_partial, pstride,
-                       (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x, st); ++nl;
+                       (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x, Rp * d, st); ++nl;
     if (insert) {
       launch_pseudo_proj(rw, (const bf16 *)c->w.pred_w, (const bf16 *)c->w.pred_b, d, c->h, st); ++nl;
-      launch_add_rmsnorm(rw, rw.T, rw.Ms, c->h, nullptr, 0, 0, (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x, st); ++nl;
+      launch_add_rmsnorm(rw, rw.T, rw.Ms, c->h, nullptr, 0, 0, (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x,
+                         Rp * d, st); ++nl;
     }
     bf16 *kplane = c->kv + (size_t)j * c->kv_layer();
     {
       GemmArgs g{};
-      g.X = c->x; g.W = (const bf16 *)c->wqkv[j]; g.R = rw.R; g.N = (H + 2 * Hkv) * dh; g.K = d; g.splits = 1;
+      g.X = c->x; g.x_lo_off = Rp * d; g.plane_rows = (int)Rp; g.err = c->dev_status;
+      g.W = (const bf16 *)c->wqkv[j]; g.R = rw.R; g.N = (H + 2 * Hkv) * dh; g.K = d; g.splits = 1;
       g.rw = rw; g.rows_active = act; g.H = H; g.Hkv = Hkv; g.dh = dh;
       g.rope = c->meta.rope; g.seq_ids = c->seq_ids; g.ctx_len = c->ctx_len;
-      g.q = c->q; g.kcache = kplane; g.seq_stride = c->kv_seq(); g.kv_stride = c->kv_plane(); g.max_ctx = cfg.max_ctx;
-      launch_gemm(EPI_QKV_ROPE, g, st); ++nl;
+      g.q = c->q; g.q_lo_off = Rp * nq; g.kcache = kplane; g.seq_stride = c->kv_seq(); g.kv_stride = c->kv_plane(); g.max_ctx = cfg.max_ctx;
+      FIRP_CUDA(c, launch_gemm(EPI_QKV_ROPE, g, tc, pdl, st)); ++nl;
     }
     {
       AttnArgs a{};
       a.rw = rw; a.rows_active = act; a.H = H; a.Hkv = Hkv; a.dh = dh;
-      a.q = c->q; a.kcache = kplane; a.seq_stride = c->kv_seq(); a.kv_stride = c->kv_plane(); a.max_ctx = cfg.max_ctx;
+      a.q = c->q; a.q_lo_off = Rp * nq; a.kcache = kplane; a.seq_stride = c->kv_seq(); a.kv_stride = c->kv_plane(); a.max_ctx = cfg.max_ctx;
       a.seq_ids = c->seq_ids; a.ctx_len = c->ctx_len; a.mask = c->meta.mask;
       const int tiles = (ra.n_hi_max + act + kAttnTile - 1) / kAttnTile;
       const int G = H / Hkv, qblocks = (act * G + 63) / 64;
@@ -196,39 +204,43 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       splits = splits < 1 ? 1 : splits;
       splits = splits > tiles ? tiles : splits;
       a.splits = splits > kAttnMaxSplits ? kAttnMaxSplits : splits;
-      a.part_o = c->part_o; a.part_ml = c->part_ml; a.o = c->o;
+      a.part_o = c->part_o; a.part_ml = c->part_ml; a.o = c->o; a.o_lo_off = Rp * nq;
       launch_attention(a, st); nl += 2;
     }
     {
       GemmArgs g{};
-      g.X = c->o; g.W = (const bf16 *)c->wo[j]; g.R = rw.R; g.N = d; g.K = nq;
-      g.splits = gemm_split_k(d, nq); g.partial = c->partial; g.partial_stride = pstride;
-      launch_gemm(EPI_PARTIAL, g, st); ++nl;
+      g.X = c->o; g.x_lo_off = Rp * nq; g.plane_rows = (int)Rp; g.err = c->dev_status;
+      g.W = (const bf16 *)c->wo[j]; g.R = rw.R; g.N = d; g.K = nq;
+      g.splits = gemm_split_k(d, nq, tc); g.partial = c->partial; g.partial_stride = pstride;
+      FIRP_CUDA(c, launch_gemm(EPI_PARTIAL, g, tc, pdl, st)); ++nl;
       n_partial = g.splits;
     }
     launch_add_rmsnorm(rw, 0, act, c->h, c->partial, n_partial, pstride, (const bf16 *)c->g_mlp[j], cfg.rms_eps, d,
-                       c->x, st); ++nl;
+                       c->x, Rp * d, st); ++nl;
     {
       GemmArgs g{};
-      g.X = c->x; g.W = (const bf16 *)c->wgu[j]; g.R = rw.R; g.N = 2 * F; g.K = d; g.splits = 1;
-      g.y = c->y; g.F = F;
-      launch_gemm(EPI_SWIGLU, g, st); ++nl;
+      g.X = c->x; g.x_lo_off = Rp * d; g.plane_rows = (int)Rp; g.err = c->dev_status;
+      g.W = (const bf16 *)c->wgu[j]; g.R = rw.R; g.N = 2 * F; g.K = d; g.splits = 1;
+      g.y = c->y; g.y_lo_off = Rp * F; g.F = F;
+      FIRP_CUDA(c, launch_gemm(EPI_SWIGLU, g, tc, pdl, st)); ++nl;
     }
     {
       GemmArgs g{};
-      g.X = c->y; g.W = (const bf16 *)c->wd[j]; g.R = rw.R; g.N = d; g.K = F;
-      g.splits = gemm_split_k(d, F); g.partial = c->partial; g.partial_stride = pstride;
-      launch_gemm(EPI_PARTIAL, g, st); ++nl;
+      g.X = c->y; g.x_lo_off = Rp * F; g.plane_rows = (int)Rp; g.err = c->dev_status;
+      g.W = (const bf16 *)c->wd[j]; g.R = rw.R; g.N = d; g.K = F;
+      g.splits = gemm_split_k(d, F, tc); g.partial = c->partial; g.partial_stride = pstride;
+      FIRP_CUDA(c, launch_gemm(EPI_PARTIAL, g, tc, pdl, st)); ++nl;
       n_partial = g.splits;
     }
   }
   if (ra.want_head) {
     launch_add_rmsnorm(rw, 0, rw.Ms, c->h, c->partial, n_partial, pstride, (const bf16 *)c->w.g_final, cfg.rms_eps, d,
-                       c->x, st); ++nl;
+                       c->x, Rp * d, st); ++nl;
     GemmArgs g{};
-    g.X = c->x; g.W = (const bf16 *)c->w.lm_head; g.R = rw.R; g.N = cfg.vocab; g.K = d; g.splits = 1;
+    g.X = c->x; g.x_lo_off = Rp * d; g.plane_rows = (int)Rp; g.err = c->dev_status;
+    g.W = (const bf16 *)c->w.lm_head; g.R = rw.R; g.N = cfg.vocab; g.K = d; g.splits = 1;
     g.logits = ra.logits_dst;
-    launch_gemm(EPI_LOGITS, g, st); ++nl;
+    FIRP_CUDA(c, launch_gemm(EPI_LOGITS, g, tc, pdl, st)); ++nl;
     launch_topb(ra.logits_dst, rw.R, cfg.vocab, cfg.top_b, c->top_ids, c->top_vals, st); ++nl;
     AcceptArgs a{};
     a.tokens = ra.d_tokens; a.parents = c->parents; a.next_parents = c->next_parents;
@@ -271,6 +283,10 @@ int firp_create(const firp_model_cfg *cfg, firp_ctx **out) {
   c->Rmax = (int)align_up(rows, 16);
   c->S = cfg->max_depth + 1;
   c->n_hi.assign(cfg->max_batch, 0);
+  // debugging switches: FIRP_GEMM=mma selects the mma.sync GEMM, FIRP_PDL=0 plain stream order
+  const char *eg = getenv("FIRP_GEMM"), *ep = getenv("FIRP_PDL");
+  c->use_tc = !(eg && strcmp(eg, "mma") == 0);
+  c->use_pdl = !(ep && strcmp(ep, "0") == 0);
   c->ws_bytes = c->carve(nullptr);
   *out = c;
   return FIRP_OK;
@@ -300,6 +316,8 @@ int firp_bind_buffers(firp_ctx *ctx, void *workspace, void *kv_cache, void *stre
   FIRP_CUDA(ctx, cudaStreamSynchronize(st));
   std::fill(ctx->n_hi.begin(), ctx->n_hi.end(), 0);
   ctx->last_parents.clear(); ctx->last_next_parents.clear(); ctx->last_seq_ids.clear();
+  if (ctx->use_tc && !gemm_tc_available())
+    return fail(ctx, FIRP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
   ctx->bound = true; ctx->stepped = false;
   return FIRP_OK;
 }
@@ -483,9 +501,12 @@ int firp_context_len(firp_ctx *ctx, int32_t seq, int32_t *n, void *stream) {
   if (!ctx->bound) return fail(ctx, FIRP_ERR_STATE, "firp_bind_buffers has not been called");
   if (seq < 0 || seq >= ctx->cfg.max_batch) return fail(ctx, FIRP_ERR_BAD_ARG, "seq id out of range");
   cudaStream_t st = (cudaStream_t)stream;
+  int status = 0;
   FIRP_CUDA(ctx, cudaMemcpyAsync(n, ctx->ctx_len + seq, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  FIRP_CUDA(ctx, cudaMemcpyAsync(&status, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost, st));
   FIRP_CUDA(ctx, cudaStreamSynchronize(st));
   ctx->n_hi[seq] = *n;
+  if (status != 0) return fail(ctx, FIRP_ERR_DEVICE_TIMEOUT, "a kernel gave up a bounded wait (device status %d)", status);
   return FIRP_OK;
 }
 

@@ -40,9 +40,12 @@ void launch_tree_prep(const Rows &rw, const int32_t *d_parents, const int32_t *d
 // h[r] = embed[token] for tree rows, 0 for pseudo rows
 void launch_embed(const Rows &rw, const int32_t *d_tokens, const bf16 *embed, int d, int vocab, float *h, cudaStream_t st);
 
+// Activations that feed a GEMM or the attention are stored as two bf16 planes (hi, lo) with
+// hi + lo = the fp32 value to ~16 mantissa bits; the lo plane starts *_lo_off elements after hi.
+
 // h[r] += sum_s partial[s][r] (s < n_partial), then x[r] = rmsnorm(h[r]) * g, for rows with v in [v0, v1)
 void launch_add_rmsnorm(const Rows &rw, int v0, int v1, float *h, const float *partial, int n_partial, size_t partial_stride,
-                        const bf16 *g, float eps, int d, bf16 *x, cudaStream_t st);
+                        const bf16 *g, float eps, int d, bf16 *x, size_t x_lo_off, cudaStream_t st);
 
 // Eq. 3: h[s*Ms + T + i] = W_i h[s*Ms + anchor] + b_i
 void launch_pseudo_proj(const Rows &rw, const bf16 *pred_w, const bf16 *pred_b, int d, float *h, cudaStream_t st);
@@ -86,9 +89,12 @@ void launch_advance_ctx(int n_seq, const int32_t *seq_ids, int32_t *ctx_len, int
 enum GemmEpilogue { EPI_PARTIAL = 0, EPI_QKV_ROPE = 1, EPI_SWIGLU = 2, EPI_LOGITS = 3 };
 
 struct GemmArgs {
-  const bf16 *X;    // [Rpad][K] activations (row-major, K contiguous)
+  const bf16 *X;    // [R][K] activations, hi plane (row-major, K contiguous)
+  size_t x_lo_off;  // elements from the hi plane to the lo plane ( = plane_rows * K )
+  int plane_rows;   // rows per plane of X
   const bf16 *W;    // [N][K] weights
   int R;            // valid rows
+  int *err;         // device status word (set to a non-zero code if a bounded wait gives up)
   int N, K;
   int splits;       // split-K factor (EPI_PARTIAL only)
   // EPI_PARTIAL: out[split][R][N] fp32
@@ -97,21 +103,26 @@ struct GemmArgs {
   Rows rw; int rows_active;      // rows with v < rows_active are written
   int H, Hkv, dh;
   const float2 *rope; const int32_t *seq_ids; const int32_t *ctx_len;
-  bf16 *q;                       // [R][H*dh]
+  bf16 *q; size_t q_lo_off;      // [R][H*dh] hi plane, lo plane
   bf16 *kcache; size_t seq_stride, kv_stride; int max_ctx;  // kcache points at this layer's K plane of sequence slot 0
   // EPI_SWIGLU: y[R][F], N = 2F
-  bf16 *y; int F;
+  bf16 *y; size_t y_lo_off; int F;
   // EPI_LOGITS: logits[R][N]
   float *logits;
 };
-void launch_gemm(GemmEpilogue epi, const GemmArgs &a, cudaStream_t st);
-int gemm_split_k(int N, int K);   // split factor used for EPI_PARTIAL at this shape
+// use_tc: tcgen05/TMA kernel (needs pdl-capable launch); otherwise the mma.sync kernel.
+// pdl: launch with programmatic stream serialization (the kernel waits on its predecessor itself).
+cudaError_t launch_gemm(GemmEpilogue epi, const GemmArgs &a, bool use_tc, bool pdl, cudaStream_t st);
+int gemm_split_k(int N, int K, bool use_tc);   // split factor used for EPI_PARTIAL at this shape
+cudaError_t launch_gemm_mma(GemmEpilogue epi, const GemmArgs &a, cudaStream_t st);
+cudaError_t launch_gemm_tc(GemmEpilogue epi, const GemmArgs &a, bool pdl, cudaStream_t st);
+bool gemm_tc_available();         // the driver entry point for tensor-map encoding was found
 
 // ---- tree-masked split-KV attention ---------------------------------------
 struct AttnArgs {
   Rows rw; int rows_active;
   int H, Hkv, dh;
-  const bf16 *q;              // [R][H*dh] rotated queries
+  const bf16 *q; size_t q_lo_off;   // [R][H*dh] rotated queries, hi and lo planes
   const bf16 *kcache;         // this layer's K plane of slot 0; V plane = kcache + kv_stride
   size_t seq_stride, kv_stride; int max_ctx;
   const int32_t *seq_ids, *ctx_len;
@@ -119,7 +130,7 @@ struct AttnArgs {
   int splits;                 // kv splits (grid.x)
   float *part_o;              // [splits][R][H][dh]
   float *part_ml;             // [splits][R][H][2] (running max in log2 units, sum)
-  bf16 *o;                    // [R][H*dh]
+  bf16 *o; size_t o_lo_off;   // [R][H*dh] hi plane, lo plane
 };
 void launch_attention(const AttnArgs &a, cudaStream_t st);
 constexpr int kAttnMaxSplits = 32;

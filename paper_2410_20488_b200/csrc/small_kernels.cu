@@ -116,7 +116,8 @@ constexpr int kNormMaxVec = 8;  // d <= 256 * 8 * 4 = 8192
 
 __global__ void __launch_bounds__(kNormThreads)
 add_rmsnorm_kernel(Rows rw, int v0, int nv, float *__restrict__ h, const float *__restrict__ partial, int n_partial,
-                   size_t partial_stride, const bf16 *__restrict__ g, float eps, int d, bf16 *__restrict__ x) {
+                   size_t partial_stride, const bf16 *__restrict__ g, float eps, int d, bf16 *__restrict__ x,
+                   size_t x_lo_off) {
   __shared__ float red[32];
   const int s = blockIdx.x / nv, v = v0 + blockIdx.x % nv;
   const int r = s * rw.Ms + v;
@@ -147,20 +148,26 @@ add_rmsnorm_kernel(Rows rw, int v0, int nv, float *__restrict__ h, const float *
       const __nv_bfloat162 g01 = reinterpret_cast<const __nv_bfloat162 *>(g)[2 * i];
       const __nv_bfloat162 g23 = reinterpret_cast<const __nv_bfloat162 *>(g)[2 * i + 1];
       const float2 ga = __bfloat1622float2(g01), gb = __bfloat1622float2(g23);
-      __nv_bfloat162 o01 = __floats2bfloat162_rn(val[it].x * rs * ga.x, val[it].y * rs * ga.y);
-      __nv_bfloat162 o23 = __floats2bfloat162_rn(val[it].z * rs * gb.x, val[it].w * rs * gb.y);
+      const float v0 = val[it].x * rs * ga.x, v1 = val[it].y * rs * ga.y;
+      const float v2 = val[it].z * rs * gb.x, v3 = val[it].w * rs * gb.y;
+      const __nv_bfloat162 o01 = __floats2bfloat162_rn(v0, v1), o23 = __floats2bfloat162_rn(v2, v3);
+      const float2 f01 = __bfloat1622float2(o01), f23 = __bfloat1622float2(o23);
       __nv_bfloat162 *xo = reinterpret_cast<__nv_bfloat162 *>(x + (size_t)r * d) + 2 * i;
-      xo[0] = o01; xo[1] = o23;
+      xo[0] = o01; xo[1] = o23;                       // hi plane
+      __nv_bfloat162 *xl = reinterpret_cast<__nv_bfloat162 *>(x + x_lo_off + (size_t)r * d) + 2 * i;
+      xl[0] = __floats2bfloat162_rn(v0 - f01.x, v1 - f01.y);   // lo plane: what the hi half lost
+      xl[1] = __floats2bfloat162_rn(v2 - f23.x, v3 - f23.y);
     }
   }
 }
 
 void launch_add_rmsnorm(const Rows &rw, int v0, int v1, float *h, const float *partial, int n_partial,
-                        size_t partial_stride, const bf16 *g, float eps, int d, bf16 *x, cudaStream_t st) {
+                        size_t partial_stride, const bf16 *g, float eps, int d, bf16 *x, size_t x_lo_off,
+                        cudaStream_t st) {
   const int nv = v1 - v0;
   if (nv <= 0) return;
   add_rmsnorm_kernel<<<rw.n_seq * nv, kNormThreads, 0, st>>>(rw, v0, nv, h, partial, n_partial, partial_stride, g, eps,
-                                                             d, x);
+                                                             d, x, x_lo_off);
 }
 
 // ---------------------------------------------------------------------------
