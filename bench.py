@@ -34,14 +34,14 @@ UNIT = "tokens/s"
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--steps", type=int, default=128)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", help="c1 | c2 | c3 | c4:T:n (sweep point on the c2 weights)")
     ap.add_argument("--layers", type=int, default=0, help="debug only: truncate the decoder (marks the line invalid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--profile-kernels", action="store_true", default=True)
+    ap.add_argument("--no-kernel-times", action="store_true", help="skip the per-kernel event-timed pass")
     return ap.parse_args()
 
 
@@ -73,11 +73,69 @@ def algorithmic_bytes(shape, n_ctx: float) -> dict:
                 total=weights + kv_read + kv_write + 2 * s.T * s.d)
 
 
-def gemm_class_bytes(shape) -> dict:
-    """Algorithmic bytes of each weight-streaming kernel class per launch (weights only)."""
+def class_bytes(shape, n_ctx: float) -> dict:
+    """Algorithmic bytes per launch of each kernel class that streams from HBM: the weight matrix
+    (read once) for the GEMMs and the Eq. 3 maps, the K and V planes of one layer for the attention."""
     s = shape
-    return dict(gemm_qkv=2 * s.n_qkv * s.d, gemm_o=2 * s.d * s.n_q, gemm_gate_up=2 * 2 * s.F * s.d,
-                gemm_down=2 * s.d * s.F, gemm_lm_head=2 * s.V * s.d, pseudo_proj=2 * s.k * s.d * s.d)
+    M = s.T + s.k
+    return dict(gemm_qkv_rope=2 * s.n_qkv * s.d, gemm_o=2 * s.d * s.n_q, gemm_gate_up_swiglu=2 * 2 * s.F * s.d,
+                gemm_down=2 * s.d * s.F, gemm_lm_head=2 * s.V * s.d, pseudo_proj=2 * s.k * s.d * s.d,
+                tree_attention=2 * 2 * s.n_kv * (n_ctx + M))
+
+
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of a kernel class at the
+# c2 shape, from the ncu capture summarised under profiles/; valid only for the kernel sources whose
+# digest is recorded with it (a changed kernel reports traffic = null until it is captured again).
+NCU_TRAFFIC = {
+    "c2-llama2-7b": dict(digest="", per_launch={}),
+}
+
+
+def kernel_source_digest() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2410_20488_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        if name.endswith((".cu", ".cuh")):
+            h.update(open(os.path.join(csrc, name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def kernel_times(eng, shape, parents, tokens, out, steps, n_ctx, peak_gbs, peak_kind):
+    """Second, separately timed pass: the library brackets every launch with CUDA events on the
+    launching stream; per class: launches, average duration, share of the summed kernel time and,
+    for the HBM-streaming classes, achieved GB/s = algorithmic bytes per launch / average duration."""
+    eng.profile(True)
+    for _ in range(steps):
+        eng.step(tokens, parents, shape.k, shape.l, out)
+        eng.commit(1)
+        tokens = out.next_tree_tokens[0]
+    prof = eng.profile_read()
+    eng.profile(False)
+    total = sum(us for _, us in prof.values()) or 1.0
+    cb = class_bytes(shape, n_ctx)
+    kernels = {}
+    for name, (n, us) in prof.items():
+        if n == 0:
+            continue
+        k = dict(launches_per_step=n / steps, avg_us=us / n, share=us / total)
+        if name in cb:
+            k["bytes_per_launch"] = cb[name]
+            k["achieved_gbs"] = cb[name] / (us / n * 1e-6) / 1e9
+            k["frac_of_peak"] = k["achieved_gbs"] / peak_gbs
+        kernels[name] = k
+    top = max((n for n in kernels if n in cb), key=lambda n: kernels[n]["share"])
+    t = kernels[top]
+    rec = NCU_TRAFFIC.get(shape.name)
+    traffic = None
+    if rec and rec["digest"] == kernel_source_digest():
+        traffic = rec["per_launch"].get(top)
+    roofline = dict(bound="hbm", kernel=top, achieved=t["achieved_gbs"], peak=peak_gbs, unit="GB/s",
+                    frac=t["frac_of_peak"], traffic=traffic, peak_kind="%s copy bandwidth" % peak_kind,
+                    avg_us=t["avg_us"], share_of_kernel_time=t["share"], bytes_per_launch=t["bytes_per_launch"],
+                    note="dominant kernel class, event-bracketed launches (bracketing serialises launches that "
+                         "overlap in the timed run)")
+    return dict(roofline=roofline, kernels=kernels, profiled_steps=steps, sum_kernel_ms_per_step=total / steps / 1e3)
 
 
 class ClockSampler:
@@ -301,13 +359,6 @@ def main():
     if e2e:
         e_ms_max, e_units = agg(e2e["ms"], e2e["emitted"])
 
-    # ---- per-kernel-class durations (second, separately timed pass with events in the library) ----
-    prof = None
-    if rank == 0:
-        from paper_2410_20488_b200 import binding
-        if hasattr(binding, "firp_profile_step"):
-            prof = binding.firp_profile_step(eng, tokens, parents, shape, outs[0], steps=min(K, 8))
-
     if rank != 0:
         return
     peaks = {}
@@ -317,6 +368,11 @@ def main():
         pass
     peak_gbs, peak_kind = (peaks["hbm_gbs"], "measured") if "hbm_gbs" in peaks else (6650.0, "fallback")
     n_mid = 0.5 * (n_start + n_end)
+
+    # ---- per-kernel-class durations (second, separately timed pass with events in the library) ----
+    prof = None
+    if not args.no_kernel_times:
+        prof = kernel_times(eng, shape, parents, tokens, outs[0], min(K, 8), n_end, peak_gbs, peak_kind)
     ab = algorithmic_bytes(shape, n_mid)
     ms_step = ms_max / K
     step_gbs = ab["total"] / (ms_step * 1e-3) / 1e9
@@ -340,6 +396,7 @@ def main():
     if prof:
         line["roofline"] = prof["roofline"]
         line["kernels"] = prof["kernels"]
+        line["kernel_pass"] = dict(steps=prof["profiled_steps"], sum_kernel_ms_per_step=prof["sum_kernel_ms_per_step"])
     else:
         line["roofline"] = dict(bound="hbm", achieved=step_gbs, peak=peak_gbs, unit="GB/s", frac=step_gbs / peak_gbs,
                                 traffic=None, note="whole step (all kernels): bytes per step / step time; peak = %s copy bandwidth" % peak_kind)

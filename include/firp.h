@@ -153,6 +153,24 @@ int firp_set_context_len(firp_ctx *ctx, int32_t seq, int32_t n, void *stream);
 /* Number of kernels the last firp_step / firp_prefill / firp_kv_commit call launched. */
 int firp_last_launch_count(const firp_ctx *ctx);
 
+/*
+ * Per-kernel timing aid (measurement only; it changes no result).  While enabled, every kernel
+ * launch of firp_step / firp_prefill / firp_kv_commit is bracketed by a pair of CUDA events on
+ * the call's stream, grouped by kernel class (the steps of Section 3.2-3.4: tree bookkeeping,
+ * embedding, RMSNorm, Eq. 3 projection, the five weight-streaming GEMMs, tree attention, top-B,
+ * acceptance walk, KV compaction).  The events serialise launches that otherwise overlap, so a
+ * profiled step is slower than an unprofiled one: use it for per-kernel durations, not for the
+ * step latency.
+ *   firp_profile_enable  on != 0 starts (and clears) the collection, 0 stops it.
+ *   firp_profile_read    synchronises `stream`, then writes for each class c < n_classes the
+ *                        number of bracketed launches and their summed duration in microseconds
+ *                        (HOST arrays), and clears the collection.  Returns the number of classes.
+ *   firp_kernel_class_name  static name of class c, NULL if c is out of range.
+ */
+int firp_profile_enable(firp_ctx *ctx, int32_t on);
+int firp_profile_read(firp_ctx *ctx, void *stream, int32_t n_classes, int32_t *launches, float *usec);
+const char *firp_kernel_class_name(int32_t c);
+
 #ifdef __cplusplus
 }
 #endif

@@ -44,7 +44,8 @@ class StepOutC(ctypes.Structure):
 
 EXPORTS = ("firp_create", "firp_destroy", "firp_last_error", "firp_workspace_bytes", "firp_kv_bytes",
            "firp_bind_buffers", "firp_init_weights", "firp_prefill", "firp_step", "firp_kv_commit",
-           "firp_context_len", "firp_set_context_len", "firp_last_launch_count")
+           "firp_context_len", "firp_set_context_len", "firp_last_launch_count", "firp_profile_enable",
+           "firp_profile_read", "firp_kernel_class_name")
 
 
 def lib_path() -> str:
@@ -77,8 +78,13 @@ def load_library():
     lib.firp_context_len.argtypes = [vp, i32, ctypes.POINTER(i32), vp]
     lib.firp_set_context_len.argtypes = [vp, i32, i32, vp]
     lib.firp_last_launch_count.argtypes = [vp]
+    lib.firp_profile_enable.argtypes = [vp, i32]
+    lib.firp_profile_read.argtypes = [vp, vp, i32, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_float)]
+    lib.firp_kernel_class_name.argtypes = [i32]
+    lib.firp_kernel_class_name.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name not in ("firp_destroy", "firp_last_error", "firp_workspace_bytes", "firp_kv_bytes"):
+        if name not in ("firp_destroy", "firp_last_error", "firp_workspace_bytes", "firp_kv_bytes",
+                        "firp_kernel_class_name"):
             getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -163,6 +169,25 @@ def firp_set_context_len(ctx, seq: int, n: int, stream: int = 0):
 
 def firp_last_launch_count(ctx) -> int:
     return load_library().firp_last_launch_count(ctx)
+
+
+def firp_profile_enable(ctx, on: bool):
+    _check(ctx, load_library().firp_profile_enable(ctx, 1 if on else 0))
+
+
+def firp_kernel_class_name(c: int):
+    name = load_library().firp_kernel_class_name(c)
+    return name.decode() if name else None
+
+
+def firp_profile_read(ctx, stream: int = 0) -> dict:
+    """{class name: (launches, total microseconds)} since the last read; synchronises the stream."""
+    n = 64
+    launches, usec = (i32 * n)(), (ctypes.c_float * n)()
+    rc = load_library().firp_profile_read(ctx, stream, n, launches, usec)
+    if rc < 0:
+        _check(ctx, rc)
+    return {firp_kernel_class_name(c): (int(launches[c]), float(usec[c])) for c in range(rc)}
 
 
 # ---- convenience: device memory through torch, nothing else ---------------
@@ -264,6 +289,12 @@ class FirpEngine:
 
     def launches(self) -> int:
         return firp_last_launch_count(self.ctx)
+
+    def profile(self, on: bool):
+        firp_profile_enable(self.ctx, on)
+
+    def profile_read(self) -> dict:
+        return firp_profile_read(self.ctx, self.stream)
 
     def close(self):
         if self.ctx:

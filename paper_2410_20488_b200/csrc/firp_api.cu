@@ -29,8 +29,22 @@ struct Carver {
 
 }  // namespace
 
+// Kernel classes of the per-kernel timing aid (firp_profile_*).
+enum KernelClass {
+  KC_TREE_PREP = 0, KC_EMBED, KC_RMSNORM, KC_PSEUDO_PROJ, KC_GEMM_QKV, KC_ATTENTION, KC_GEMM_O, KC_GEMM_GATE_UP,
+  KC_GEMM_DOWN, KC_GEMM_LM_HEAD, KC_TOPB, KC_ACCEPT, KC_COMMIT, KC_COUNT
+};
+static const char *const kClassNames[KC_COUNT] = {
+    "tree_prep", "embed", "add_rmsnorm", "pseudo_proj", "gemm_qkv_rope", "tree_attention", "gemm_o", "gemm_gate_up_swiglu",
+    "gemm_down", "gemm_lm_head", "topb", "accept_next_tree", "kv_commit"};
+
 struct firp_ctx {
   firp_model_cfg cfg{};
+  // per-kernel timing aid: event pairs recorded around launches while enabled
+  bool profiling = false;
+  std::vector<cudaEvent_t> ev_pool;           // events created so far (reused after each read)
+  std::vector<int> ev_class;                  // class of pair i (events 2i, 2i+1)
+  size_t ev_used = 0;                         // pairs in use
   std::string err;
   int launches = 0;
   bool bound = false, have_weights = false, stepped = false;
@@ -111,6 +125,26 @@ int fail(firp_ctx *ctx, int code, const char *fmt, ...) {
     if (e__ != cudaSuccess) return fail(ctx, FIRP_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e__)); \
   } while (0)
 
+// Brackets the launches issued during its lifetime with an event pair when profiling is on.
+struct Bracket {
+  firp_ctx *c; cudaStream_t st; cudaEvent_t stop = nullptr;
+  Bracket(firp_ctx *ctx, int cls, cudaStream_t s) : c(ctx), st(s) {
+    if (!c->profiling) return;
+    while (c->ev_pool.size() < 2 * (c->ev_used + 1)) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return;
+      c->ev_pool.push_back(e);
+    }
+    if (c->ev_class.size() <= c->ev_used) c->ev_class.resize(c->ev_used + 1);
+    c->ev_class[c->ev_used] = cls;
+    cudaEventRecord(c->ev_pool[2 * c->ev_used], st);
+    stop = c->ev_pool[2 * c->ev_used + 1];
+    ++c->ev_used;
+  }
+  ~Bracket() { if (stop) cudaEventRecord(stop, st); }
+};
+#define FIRP_TIMED(cls) Bracket bracket__(c, cls, st)
+
 // depth of every node of a validated tree; returns max depth or -1 if malformed
 int tree_depths(const int32_t *parents, int T, std::vector<int> &depth) {
   depth.assign(T, 0);
@@ -167,19 +201,24 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   const bool tc = c->use_tc, pdl = c->use_tc && c->use_pdl;
 
   const int mw_out = (rw.Ms + 31) / 32;
-  launch_tree_prep(rw, c->parents, c->seq_ids, c->ctx_len, dh, cfg.rope_theta, c->meta, out ? out->depth : nullptr,
-                   out ? out->mask : nullptr, mw_out, st); ++nl;
-  launch_embed(rw, ra.d_tokens, (const bf16 *)c->w.embed, d, cfg.vocab, c->h, st); ++nl;
+  { FIRP_TIMED(KC_TREE_PREP);
+    launch_tree_prep(rw, c->parents, c->seq_ids, c->ctx_len, dh, cfg.rope_theta, c->meta, out ? out->depth : nullptr,
+                     out ? out->mask : nullptr, mw_out, st); ++nl; }
+  { FIRP_TIMED(KC_EMBED);
+    launch_embed(rw, ra.d_tokens, (const bf16 *)c->w.embed, d, cfg.vocab, c->h, st); ++nl; }
 
   int n_partial = 0;   // split-K partial sums waiting to be added into the residual stream
   for (int j = 0; j < cfg.n_layers; ++j) {
     const bool insert = (rw.k > 0 && j == ra.l);
     const int act = (rw.k > 0 && j >= ra.l) ? rw.Ms : rw.T;   // rows alive in this layer
     // residual add + pre-attention RMSNorm; at layer l the pseudo rows are projected in between
-    launch_add_rmsnorm(rw, 0, rw.T + ((insert || act == rw.T) ? 0 : rw.k), c->h, c->partial, n_partial, pstride,
-                       (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x, Rp * d, st); ++nl;
+    { FIRP_TIMED(KC_RMSNORM);
+      launch_add_rmsnorm(rw, 0, rw.T + ((insert || act == rw.T) ? 0 : rw.k), c->h, c->partial, n_partial, pstride,
+                         (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x, Rp * d, st); ++nl; }
     if (insert) {
-      launch_pseudo_proj(rw, (const bf16 *)c->w.pred_w, (const bf16 *)c->w.pred_b, d, c->h, st); ++nl;
+      { FIRP_TIMED(KC_PSEUDO_PROJ);
+        launch_pseudo_proj(rw, (const bf16 *)c->w.pred_w, (const bf16 *)c->w.pred_b, d, c->h, st); ++nl; }
+      FIRP_TIMED(KC_RMSNORM);
       launch_add_rmsnorm(rw, rw.T, rw.Ms, c->h, nullptr, 0, 0, (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x,
                          Rp * d, st); ++nl;
     }
@@ -191,6 +230,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       g.rw = rw; g.rows_active = act; g.H = H; g.Hkv = Hkv; g.dh = dh;
       g.rope = c->meta.rope; g.seq_ids = c->seq_ids; g.ctx_len = c->ctx_len;
       g.q = c->q; g.q_lo_off = Rp * nq; g.kcache = kplane; g.seq_stride = c->kv_seq(); g.kv_stride = c->kv_plane(); g.max_ctx = cfg.max_ctx;
+      FIRP_TIMED(KC_GEMM_QKV);
       FIRP_CUDA(c, launch_gemm(EPI_QKV_ROPE, g, tc, pdl, st)); ++nl;
     }
     {
@@ -205,6 +245,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       splits = splits > tiles ? tiles : splits;
       a.splits = splits > kAttnMaxSplits ? kAttnMaxSplits : splits;
       a.part_o = c->part_o; a.part_ml = c->part_ml; a.o = c->o; a.o_lo_off = Rp * nq;
+      FIRP_TIMED(KC_ATTENTION);
       launch_attention(a, st); nl += 2;
     }
     {
@@ -212,16 +253,19 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       g.X = c->o; g.x_lo_off = Rp * nq; g.plane_rows = (int)Rp; g.err = c->dev_status;
       g.W = (const bf16 *)c->wo[j]; g.R = rw.R; g.N = d; g.K = nq;
       g.splits = gemm_split_k(d, nq, tc); g.partial = c->partial; g.partial_stride = pstride;
+      FIRP_TIMED(KC_GEMM_O);
       FIRP_CUDA(c, launch_gemm(EPI_PARTIAL, g, tc, pdl, st)); ++nl;
       n_partial = g.splits;
     }
-    launch_add_rmsnorm(rw, 0, act, c->h, c->partial, n_partial, pstride, (const bf16 *)c->g_mlp[j], cfg.rms_eps, d,
-                       c->x, Rp * d, st); ++nl;
+    { FIRP_TIMED(KC_RMSNORM);
+      launch_add_rmsnorm(rw, 0, act, c->h, c->partial, n_partial, pstride, (const bf16 *)c->g_mlp[j], cfg.rms_eps, d,
+                         c->x, Rp * d, st); ++nl; }
     {
       GemmArgs g{};
       g.X = c->x; g.x_lo_off = Rp * d; g.plane_rows = (int)Rp; g.err = c->dev_status;
       g.W = (const bf16 *)c->wgu[j]; g.R = rw.R; g.N = 2 * F; g.K = d; g.splits = 1;
       g.y = c->y; g.y_lo_off = Rp * F; g.F = F;
+      FIRP_TIMED(KC_GEMM_GATE_UP);
       FIRP_CUDA(c, launch_gemm(EPI_SWIGLU, g, tc, pdl, st)); ++nl;
     }
     {
@@ -229,19 +273,23 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       g.X = c->y; g.x_lo_off = Rp * F; g.plane_rows = (int)Rp; g.err = c->dev_status;
       g.W = (const bf16 *)c->wd[j]; g.R = rw.R; g.N = d; g.K = F;
       g.splits = gemm_split_k(d, F, tc); g.partial = c->partial; g.partial_stride = pstride;
+      FIRP_TIMED(KC_GEMM_DOWN);
       FIRP_CUDA(c, launch_gemm(EPI_PARTIAL, g, tc, pdl, st)); ++nl;
       n_partial = g.splits;
     }
   }
   if (ra.want_head) {
-    launch_add_rmsnorm(rw, 0, rw.Ms, c->h, c->partial, n_partial, pstride, (const bf16 *)c->w.g_final, cfg.rms_eps, d,
-                       c->x, Rp * d, st); ++nl;
+    { FIRP_TIMED(KC_RMSNORM);
+      launch_add_rmsnorm(rw, 0, rw.Ms, c->h, c->partial, n_partial, pstride, (const bf16 *)c->w.g_final, cfg.rms_eps, d,
+                         c->x, Rp * d, st); ++nl; }
     GemmArgs g{};
     g.X = c->x; g.x_lo_off = Rp * d; g.plane_rows = (int)Rp; g.err = c->dev_status;
     g.W = (const bf16 *)c->w.lm_head; g.R = rw.R; g.N = cfg.vocab; g.K = d; g.splits = 1;
     g.logits = ra.logits_dst;
-    FIRP_CUDA(c, launch_gemm(EPI_LOGITS, g, tc, pdl, st)); ++nl;
-    launch_topb(ra.logits_dst, rw.R, cfg.vocab, cfg.top_b, c->top_ids, c->top_vals, st); ++nl;
+    { FIRP_TIMED(KC_GEMM_LM_HEAD);
+      FIRP_CUDA(c, launch_gemm(EPI_LOGITS, g, tc, pdl, st)); ++nl; }
+    { FIRP_TIMED(KC_TOPB);
+      launch_topb(ra.logits_dst, rw.R, cfg.vocab, cfg.top_b, c->top_ids, c->top_vals, st); ++nl; }
     AcceptArgs a{};
     a.tokens = ra.d_tokens; a.parents = c->parents; a.next_parents = c->next_parents;
     a.top_ids = c->top_ids; a.top_vals = c->top_vals; a.T_next = ra.T_next; a.B = cfg.top_b; a.S = c->S;
@@ -252,6 +300,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       a.o_next_tokens = out->next_tree_tokens; a.o_best = (ra.prefill_last_row < 0) ? out->best : nullptr;
       a.o_topb_ids = out->topb_ids; a.o_topb_vals = out->topb_vals;
     }
+    FIRP_TIMED(KC_ACCEPT);
     launch_accept(rw, a, st); ++nl;
   }
   FIRP_CUDA(c, cudaGetLastError());
@@ -292,7 +341,11 @@ int firp_create(const firp_model_cfg *cfg, firp_ctx **out) {
   return FIRP_OK;
 }
 
-void firp_destroy(firp_ctx *ctx) { delete ctx; }
+void firp_destroy(firp_ctx *ctx) {
+  if (!ctx) return;
+  for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
+  delete ctx;
+}
 
 const char *firp_last_error(const firp_ctx *ctx) { return ctx ? ctx->err.c_str() : "null context"; }
 
@@ -490,7 +543,8 @@ int firp_kv_commit(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const i
     a.path = ctx->path; a.path_len = ctx->n_acc;
     for (int s = 0; s < n_seq; ++s) ctx->n_hi[ids[s]] += S;   // exact value is on the device; keep an upper bound
   }
-  launch_commit(n_seq, a, st); ctx->launches += 2;
+  { firp_ctx *c = ctx; FIRP_TIMED(KC_COMMIT);
+    launch_commit(n_seq, a, st); ctx->launches += 2; }
   FIRP_CUDA(ctx, cudaGetLastError());
   ctx->stepped = false;
   return FIRP_OK;
@@ -523,5 +577,28 @@ int firp_set_context_len(firp_ctx *ctx, int32_t seq, int32_t n, void *stream) {
 }
 
 int firp_last_launch_count(const firp_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int firp_profile_enable(firp_ctx *ctx, int32_t on) {
+  if (!ctx) return FIRP_ERR_BAD_ARG;
+  ctx->profiling = on != 0;
+  ctx->ev_used = 0;
+  return FIRP_OK;
+}
+
+int firp_profile_read(firp_ctx *ctx, void *stream, int32_t n_classes, int32_t *launches, float *usec) {
+  if (!ctx || !launches || !usec || n_classes < 0) return FIRP_ERR_BAD_ARG;
+  FIRP_CUDA(ctx, cudaStreamSynchronize((cudaStream_t)stream));
+  for (int i = 0; i < n_classes; ++i) { launches[i] = 0; usec[i] = 0.f; }
+  for (size_t i = 0; i < ctx->ev_used; ++i) {
+    float ms = 0.f;
+    FIRP_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->ev_pool[2 * i], ctx->ev_pool[2 * i + 1]));
+    const int k = ctx->ev_class[i];
+    if (k < n_classes) { ++launches[k]; usec[k] += ms * 1e3f; }
+  }
+  ctx->ev_used = 0;
+  return KC_COUNT;
+}
+
+const char *firp_kernel_class_name(int32_t c) { return (c >= 0 && c < KC_COUNT) ? kClassNames[c] : nullptr; }
 
 }  // extern "C"
