@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfirp_b200.so")
-SOURCES = ["firp_api.cu", "small_kernels.cu", "gemm_skinny.cu", "gemm_tcgen05.cu", "attn_tree.cu"]
-HEADERS = ["firp_kernels.cuh", "gemm_epilogue.cuh", os.path.join("..", "..", "include", "firp.h")]
+SOURCES = ["firp_api.cu", "small_kernels.cu", "gemm_skinny.cu", "gemm_tcgen05.cu", "finish_kernels.cu", "attn_tree.cu"]
+HEADERS = ["firp_kernels.cuh", "gemm_epilogue.cuh", "launch_util.cuh", os.path.join("..", "..", "include", "firp.h")]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "--use_fast_math", "-shared"]
 

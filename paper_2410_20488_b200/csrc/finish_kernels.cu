@@ -1,0 +1,174 @@
+// Finishers of the stream-K GEMMs: each sums the partial tiles a GEMM left in scratch (fixed
+// order: ascending CTA index) and applies the elementwise step that follows the contraction:
+//   qkv     rotary embedding at the row's tree position (Section 3.4: a tree token keeps its
+//           positional index), queries as (hi, lo) bf16 planes, keys / values into the bf16 cache
+//   swiglu  silu(gate) * up as (hi, lo) bf16 planes
+//   logits  fp32 logits of the lm-head (Section 3.2: the original lm-head on every row)
+// A thread owns 4 neighbouring lanes (weight rows) of one token row of one supertile, so partial
+// tiles are read as float4 and results leave as 8- or 16-byte stores.  The kernels use no shared
+// memory and few registers: they stay resident beside the next GEMM's CTAs, whose weight stream
+// therefore runs while they work.
+#include "firp_kernels.cuh"
+#include "launch_util.cuh"
+
+namespace firp {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+struct Item { int st, m, i4; };
+
+// thread -> (supertile, token row, lane quad); quads vary fastest (coalesced float4 reads)
+__device__ __forceinline__ bool item_of_thread(int n_st, int R, Item &it) {
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= (long long)n_st * R * 32) return false;
+  it.i4 = (int)(t & 31) * 4;
+  const long long r = t >> 5;
+  it.m = (int)(r % R);
+  it.st = (int)(r / R);
+  return true;
+}
+
+// sums of tile 0 and tile 1 of supertile st for token row m, lanes i4 .. i4+3
+__device__ __forceinline__ void sum_partials(const Partials &p, int st, int m, int i4, float4 &v0, float4 &v1) {
+  const size_t plane = (size_t)p.ws_rows * 128, slot = 2 * plane;
+  const int c_first = sk_owner(p.sk, (long long)st * p.sk.KB), c_last = sk_owner(p.sk, (long long)(st + 1) * p.sk.KB - 1);
+  v0 = v1 = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int c0 = c_first; c0 <= c_last; c0 += 4) {      // 4 contributors' loads in flight together
+    float4 a[4], b[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int c = c0 + k;
+      a[k] = b[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (c <= c_last) {
+        const int ord = st - (int)(sk_begin(p.sk, c) / p.sk.KB);
+        const float *src = p.ws + (size_t)(c * kGemmSlots + ord) * slot + (size_t)m * 128 + i4;
+        a[k] = __ldcg(reinterpret_cast<const float4 *>(src));
+        b[k] = __ldcg(reinterpret_cast<const float4 *>(src + plane));
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      v0.x += a[k].x; v0.y += a[k].y; v0.z += a[k].z; v0.w += a[k].w;
+      v1.x += b[k].x; v1.y += b[k].y; v1.z += b[k].z; v1.w += b[k].w;
+    }
+  }
+}
+
+__device__ __forceinline__ void split4(const float v[4], uint2 &hi, uint2 &lo) {
+  const __nv_bfloat162 h01 = __floats2bfloat162_rn(v[0], v[1]), h23 = __floats2bfloat162_rn(v[2], v[3]);
+  const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
+  const __nv_bfloat162 l01 = __floats2bfloat162_rn(v[0] - f01.x, v[1] - f01.y);
+  const __nv_bfloat162 l23 = __floats2bfloat162_rn(v[2] - f23.x, v[3] - f23.y);
+  hi = make_uint2(*reinterpret_cast<const uint32_t *>(&h01), *reinterpret_cast<const uint32_t *>(&h23));
+  lo = make_uint2(*reinterpret_cast<const uint32_t *>(&l01), *reinterpret_cast<const uint32_t *>(&l23));
+}
+__device__ __forceinline__ uint2 round4(const float v[4]) {
+  const __nv_bfloat162 h01 = __floats2bfloat162_rn(v[0], v[1]), h23 = __floats2bfloat162_rn(v[2], v[3]);
+  return make_uint2(*reinterpret_cast<const uint32_t *>(&h01), *reinterpret_cast<const uint32_t *>(&h23));
+}
+
+// ---- q, k, v: rotary embedding, query planes, cache rows --------------------------------------
+// Supertile st holds the first halves (c < dh/2) of 128 / (dh/2) heads in tile 0 and their second
+// halves in tile 1, so lanes i4..i4+3 of the two tiles are 4 rotary pairs (c, c + dh/2) of one head.
+__global__ void __launch_bounds__(kThreads) qkv_finish_kernel(Partials p, GemmArgs a, int n_st, int pdl) {
+  if (pdl) { griddep_launch(); griddep_wait(); }
+  Item it;
+  if (!item_of_thread(n_st, a.R, it)) return;
+  const int half = a.dh >> 1, hp = 128 / half;
+  const int unit = it.st * hp + it.i4 / half, c = it.i4 % half;
+  const int s = it.m / a.rw.Ms, v = it.m - s * a.rw.Ms;
+  if (unit >= a.H + 2 * a.Hkv || v >= a.rows_active) return;
+  float4 v0, v1;
+  sum_partials(p, it.st, it.m, it.i4, v0, v1);
+  float x1[4] = {v0.x, v0.y, v0.z, v0.w}, x2[4] = {v1.x, v1.y, v1.z, v1.w};
+  if (unit < a.H + a.Hkv) {     // queries and keys are rotated at the row's tree position
+    const float4 *cs = reinterpret_cast<const float4 *>(a.rope + (size_t)it.m * half + c);
+    const float4 cs01 = __ldg(cs), cs23 = __ldg(cs + 1);
+    const float co[4] = {cs01.x, cs01.z, cs23.x, cs23.z}, si[4] = {cs01.y, cs01.w, cs23.y, cs23.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float y1 = x1[j] * co[j] - x2[j] * si[j], y2 = x2[j] * co[j] + x1[j] * si[j];
+      x1[j] = y1; x2[j] = y2;
+    }
+  }
+  if (unit < a.H) {
+    uint2 h1, l1, h2, l2;
+    split4(x1, h1, l1); split4(x2, h2, l2);
+    bf16 *dst = a.q + (size_t)it.m * a.H * a.dh + unit * a.dh + c;
+    *reinterpret_cast<uint2 *>(dst) = h1;
+    *reinterpret_cast<uint2 *>(dst + half) = h2;
+    *reinterpret_cast<uint2 *>(dst + a.q_lo_off) = l1;
+    *reinterpret_cast<uint2 *>(dst + a.q_lo_off + half) = l2;
+  } else {                      // the cache stores bf16: one rounding, on store
+    const int is_v = unit >= a.H + a.Hkv;
+    const int kvh = unit - a.H - (is_v ? a.Hkv : 0);
+    const int slot = a.seq_ids[s];
+    const int pos = a.ctx_len[slot] + v;
+    if (pos < a.max_ctx) {
+      bf16 *dst = a.kcache + (size_t)slot * a.seq_stride + (is_v ? a.kv_stride : 0) + ((size_t)pos * a.Hkv + kvh) * a.dh + c;
+      *reinterpret_cast<uint2 *>(dst) = round4(x1);
+      *reinterpret_cast<uint2 *>(dst + half) = round4(x2);
+    }
+  }
+}
+
+// ---- SwiGLU: tile 0 = gate rows st*128 .., tile 1 = the matching up rows ------------------------
+__global__ void __launch_bounds__(kThreads) swiglu_finish_kernel(Partials p, GemmArgs a, int n_st, int pdl) {
+  if (pdl) { griddep_launch(); griddep_wait(); }
+  Item it;
+  if (!item_of_thread(n_st, a.R, it)) return;
+  const int j0 = it.st * 128 + it.i4;
+  const int v = it.m % a.rw.Ms;
+  if (j0 >= a.F || v >= a.rows_active) return;
+  float4 g, u;
+  sum_partials(p, it.st, it.m, it.i4, g, u);
+  const float gg[4] = {g.x, g.y, g.z, g.w}, uu[4] = {u.x, u.y, u.z, u.w};
+  float y[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) y[j] = gg[j] / (1.f + __expf(-gg[j])) * uu[j];
+  uint2 hi, lo;
+  split4(y, hi, lo);
+  bf16 *dst = a.y + (size_t)it.m * a.F + j0;
+  *reinterpret_cast<uint2 *>(dst) = hi;
+  *reinterpret_cast<uint2 *>(dst + a.y_lo_off) = lo;
+}
+
+// ---- logits: tile 0 = rows st*256 .., tile 1 = rows st*256 + 128 .. -----------------------------
+__global__ void __launch_bounds__(kThreads) logits_finish_kernel(Partials p, GemmArgs a, int n_st, int pdl) {
+  if (pdl) { griddep_launch(); griddep_wait(); }
+  Item it;
+  if (!item_of_thread(n_st, a.R, it)) return;
+  const int n0 = it.st * 256 + it.i4, n1 = n0 + 128;
+  if (n0 >= a.N) return;
+  float4 v0, v1;
+  sum_partials(p, it.st, it.m, it.i4, v0, v1);
+  float *row = a.logits + (size_t)it.m * a.N;
+  if ((a.N & 3) == 0) {
+    *reinterpret_cast<float4 *>(row + n0) = v0;
+    if (n1 < a.N) *reinterpret_cast<float4 *>(row + n1) = v1;
+  } else {
+    const float e0[4] = {v0.x, v0.y, v0.z, v0.w}, e1[4] = {v1.x, v1.y, v1.z, v1.w};
+    for (int j = 0; j < 4; ++j) {
+      if (n0 + j < a.N) row[n0 + j] = e0[j];
+      if (n1 + j < a.N) row[n1 + j] = e1[j];
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_finish(GemmEpilogue epi, const Partials &p, const GemmArgs &a, bool pdl, cudaStream_t st) {
+  const int n_st = (int)(p.sk.U / p.sk.KB);
+  const long long threads = (long long)n_st * a.R * 32;
+  const dim3 grid((unsigned)((threads + kThreads - 1) / kThreads)), block(kThreads);
+  switch (epi) {
+    case EPI_QKV_ROPE: return launch_k(qkv_finish_kernel, grid, block, 0, st, pdl, p, a, n_st, pdl ? 1 : 0);
+    case EPI_SWIGLU: return launch_k(swiglu_finish_kernel, grid, block, 0, st, pdl, p, a, n_st, pdl ? 1 : 0);
+    case EPI_LOGITS: return launch_k(logits_finish_kernel, grid, block, 0, st, pdl, p, a, n_st, pdl ? 1 : 0);
+    default: return cudaErrorInvalidValue;   // the residual GEMMs are finished by the RMSNorm kernel
+  }
+}
+
+}  // namespace firp

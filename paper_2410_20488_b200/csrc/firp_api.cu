@@ -48,7 +48,7 @@ struct firp_ctx {
   std::string err;
   int launches = 0;
   bool bound = false, have_weights = false, stepped = false;
-  int Rmax = 0, S = 0, splitk_max = 8;
+  int Rmax = 0, S = 0;
   bool use_tc = true, use_pdl = true;   // tcgen05/TMA GEMM, programmatic dependent launch
   int *dev_status = nullptr;            // device status word (bounded waits report here)
   // weights
@@ -56,7 +56,7 @@ struct firp_ctx {
   std::vector<const void *> wqkv, wo, wgu, wd, g_attn, g_mlp;
   // device buffers (carved from the caller's workspace)
   bf16 *kv = nullptr;
-  float *h = nullptr, *partial = nullptr, *part_o = nullptr, *part_ml = nullptr, *logits = nullptr, *top_vals = nullptr;
+  float *h = nullptr, *gemm_ws = nullptr, *part_o = nullptr, *part_ml = nullptr, *logits = nullptr, *top_vals = nullptr;
   bf16 *x = nullptr, *q = nullptr, *o = nullptr, *y = nullptr;
   int32_t *ctx_len = nullptr, *seq_ids = nullptr, *parents = nullptr, *next_parents = nullptr, *chain = nullptr;
   int32_t *top_ids = nullptr, *path = nullptr, *n_acc = nullptr, *accepted = nullptr, *next_tokens = nullptr;
@@ -81,7 +81,7 @@ struct firp_ctx {
     q = c.take<bf16>(2 * R * nq);
     o = c.take<bf16>(2 * R * nq);
     y = c.take<bf16>(2 * R * cfg.d_ffn);
-    partial = c.take<float>((size_t)splitk_max * R * d);
+    gemm_ws = c.take<float>((size_t)kGemmMaxCtas * kGemmSlots * 2 * R * 128);
     part_o = c.take<float>((size_t)kAttnMaxSplits * R * nq);
     part_ml = c.take<float>((size_t)kAttnMaxSplits * R * cfg.n_heads * 2);
     logits = c.take<float>(R * cfg.vocab);
@@ -194,7 +194,6 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   const Rows &rw = ra.rw;
   const int d = cfg.d_model, H = cfg.n_heads, Hkv = cfg.n_kv_heads, dh = cfg.head_dim, F = cfg.d_ffn;
   const int nq = H * dh;
-  const size_t pstride = (size_t)rw.R * d;
   const size_t Rp = (size_t)c->Rmax;          // rows per activation plane
   const firp_step_out *out = ra.out;
   int &nl = c->launches;
@@ -207,31 +206,41 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   { FIRP_TIMED(KC_EMBED);
     launch_embed(rw, ra.d_tokens, (const bf16 *)c->w.embed, d, cfg.vocab, c->h, st); ++nl; }
 
-  int n_partial = 0;   // split-K partial sums waiting to be added into the residual stream
+  auto gemm_base = [&](const bf16 *X, size_t lo_off, const void *W, int N, int K, int act) {
+    GemmArgs g{};
+    g.X = X; g.x_lo_off = lo_off; g.plane_rows = (int)Rp; g.err = c->dev_status;
+    g.W = (const bf16 *)W; g.R = rw.R; g.N = N; g.K = K; g.rw = rw; g.rows_active = act;
+    g.ws = c->gemm_ws;
+    return g;
+  };
+  // partial tiles a residual GEMM left behind: the next RMSNorm adds them into the residual stream
+  Partials pending{};
+  pending.ws = c->gemm_ws; pending.ws_rows = (int)Rp;
+  const Partials none{};
   for (int j = 0; j < cfg.n_layers; ++j) {
     const bool insert = (rw.k > 0 && j == ra.l);
     const int act = (rw.k > 0 && j >= ra.l) ? rw.Ms : rw.T;   // rows alive in this layer
-    // residual add + pre-attention RMSNorm; at layer l the pseudo rows are projected in between
+    // the rows that took part in the last residual GEMM get its pending sums; new pseudo rows have none
+    const int carried = insert ? rw.T : act;
     { FIRP_TIMED(KC_RMSNORM);
-      launch_add_rmsnorm(rw, 0, rw.T + ((insert || act == rw.T) ? 0 : rw.k), c->h, c->partial, n_partial, pstride,
-                         (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x, Rp * d, st); ++nl; }
-    if (insert) {
+      FIRP_CUDA(c, launch_rmsnorm(rw, 0, carried, c->h, pending, (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x, Rp * d, pdl, st)); ++nl; }
+    pending.sk.U = 0;
+    if (insert) {   // Eq. 3 on the raw (now complete) residual row of the root, then the norm of the new rows
       { FIRP_TIMED(KC_PSEUDO_PROJ);
         launch_pseudo_proj(rw, (const bf16 *)c->w.pred_w, (const bf16 *)c->w.pred_b, d, c->h, st); ++nl; }
       FIRP_TIMED(KC_RMSNORM);
-      launch_add_rmsnorm(rw, rw.T, rw.Ms, c->h, nullptr, 0, 0, (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x,
-                         Rp * d, st); ++nl;
+      FIRP_CUDA(c, launch_rmsnorm(rw, rw.T, rw.Ms, c->h, none, (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x, Rp * d, pdl, st)); ++nl;
     }
     bf16 *kplane = c->kv + (size_t)j * c->kv_layer();
     {
-      GemmArgs g{};
-      g.X = c->x; g.x_lo_off = Rp * d; g.plane_rows = (int)Rp; g.err = c->dev_status;
-      g.W = (const bf16 *)c->wqkv[j]; g.R = rw.R; g.N = (H + 2 * Hkv) * dh; g.K = d; g.splits = 1;
-      g.rw = rw; g.rows_active = act; g.H = H; g.Hkv = Hkv; g.dh = dh;
+      GemmArgs g = gemm_base(c->x, Rp * d, c->wqkv[j], (H + 2 * Hkv) * dh, d, act);
+      g.H = H; g.Hkv = Hkv; g.dh = dh;
       g.rope = c->meta.rope; g.seq_ids = c->seq_ids; g.ctx_len = c->ctx_len;
       g.q = c->q; g.q_lo_off = Rp * nq; g.kcache = kplane; g.seq_stride = c->kv_seq(); g.kv_stride = c->kv_plane(); g.max_ctx = cfg.max_ctx;
       FIRP_TIMED(KC_GEMM_QKV);
-      FIRP_CUDA(c, launch_gemm(EPI_QKV_ROPE, g, tc, pdl, st)); ++nl;
+      Partials p = pending;
+      FIRP_CUDA(c, launch_gemm(EPI_QKV_ROPE, g, tc, pdl, st, &p.sk)); ++nl;
+      if (p.sk.U > 0) { FIRP_CUDA(c, launch_gemm_finish(EPI_QKV_ROPE, p, g, pdl, st)); ++nl; }
     }
     {
       AttnArgs a{};
@@ -249,45 +258,38 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       launch_attention(a, st); nl += 2;
     }
     {
-      GemmArgs g{};
-      g.X = c->o; g.x_lo_off = Rp * nq; g.plane_rows = (int)Rp; g.err = c->dev_status;
-      g.W = (const bf16 *)c->wo[j]; g.R = rw.R; g.N = d; g.K = nq;
-      g.splits = gemm_split_k(d, nq, tc); g.partial = c->partial; g.partial_stride = pstride;
+      GemmArgs g = gemm_base(c->o, Rp * nq, c->wo[j], d, nq, act);
+      g.h_out = c->h;
       FIRP_TIMED(KC_GEMM_O);
-      FIRP_CUDA(c, launch_gemm(EPI_PARTIAL, g, tc, pdl, st)); ++nl;
-      n_partial = g.splits;
+      FIRP_CUDA(c, launch_gemm(EPI_RESIDUAL, g, tc, pdl, st, &pending.sk)); ++nl;
     }
     { FIRP_TIMED(KC_RMSNORM);
-      launch_add_rmsnorm(rw, 0, act, c->h, c->partial, n_partial, pstride, (const bf16 *)c->g_mlp[j], cfg.rms_eps, d,
-                         c->x, Rp * d, st); ++nl; }
+      FIRP_CUDA(c, launch_rmsnorm(rw, 0, act, c->h, pending, (const bf16 *)c->g_mlp[j], cfg.rms_eps, d, c->x, Rp * d, pdl, st)); ++nl; }
+    pending.sk.U = 0;
     {
-      GemmArgs g{};
-      g.X = c->x; g.x_lo_off = Rp * d; g.plane_rows = (int)Rp; g.err = c->dev_status;
-      g.W = (const bf16 *)c->wgu[j]; g.R = rw.R; g.N = 2 * F; g.K = d; g.splits = 1;
+      GemmArgs g = gemm_base(c->x, Rp * d, c->wgu[j], 2 * F, d, act);
       g.y = c->y; g.y_lo_off = Rp * F; g.F = F;
       FIRP_TIMED(KC_GEMM_GATE_UP);
-      FIRP_CUDA(c, launch_gemm(EPI_SWIGLU, g, tc, pdl, st)); ++nl;
+      Partials p = pending;
+      FIRP_CUDA(c, launch_gemm(EPI_SWIGLU, g, tc, pdl, st, &p.sk)); ++nl;
+      if (p.sk.U > 0) { FIRP_CUDA(c, launch_gemm_finish(EPI_SWIGLU, p, g, pdl, st)); ++nl; }
     }
     {
-      GemmArgs g{};
-      g.X = c->y; g.x_lo_off = Rp * F; g.plane_rows = (int)Rp; g.err = c->dev_status;
-      g.W = (const bf16 *)c->wd[j]; g.R = rw.R; g.N = d; g.K = F;
-      g.splits = gemm_split_k(d, F, tc); g.partial = c->partial; g.partial_stride = pstride;
+      GemmArgs g = gemm_base(c->y, Rp * F, c->wd[j], d, F, act);
+      g.h_out = c->h;
       FIRP_TIMED(KC_GEMM_DOWN);
-      FIRP_CUDA(c, launch_gemm(EPI_PARTIAL, g, tc, pdl, st)); ++nl;
-      n_partial = g.splits;
+      FIRP_CUDA(c, launch_gemm(EPI_RESIDUAL, g, tc, pdl, st, &pending.sk)); ++nl;
     }
   }
   if (ra.want_head) {
     { FIRP_TIMED(KC_RMSNORM);
-      launch_add_rmsnorm(rw, 0, rw.Ms, c->h, c->partial, n_partial, pstride, (const bf16 *)c->w.g_final, cfg.rms_eps, d,
-                         c->x, Rp * d, st); ++nl; }
-    GemmArgs g{};
-    g.X = c->x; g.x_lo_off = Rp * d; g.plane_rows = (int)Rp; g.err = c->dev_status;
-    g.W = (const bf16 *)c->w.lm_head; g.R = rw.R; g.N = cfg.vocab; g.K = d; g.splits = 1;
+      FIRP_CUDA(c, launch_rmsnorm(rw, 0, rw.Ms, c->h, pending, (const bf16 *)c->w.g_final, cfg.rms_eps, d, c->x, Rp * d, pdl, st)); ++nl; }
+    GemmArgs g = gemm_base(c->x, Rp * d, c->w.lm_head, cfg.vocab, d, rw.Ms);
     g.logits = ra.logits_dst;
     { FIRP_TIMED(KC_GEMM_LM_HEAD);
-      FIRP_CUDA(c, launch_gemm(EPI_LOGITS, g, tc, pdl, st)); ++nl; }
+      Partials p = pending;
+      FIRP_CUDA(c, launch_gemm(EPI_LOGITS, g, tc, pdl, st, &p.sk)); ++nl;
+      if (p.sk.U > 0) { FIRP_CUDA(c, launch_gemm_finish(EPI_LOGITS, p, g, pdl, st)); ++nl; } }
     { FIRP_TIMED(KC_TOPB);
       launch_topb(ra.logits_dst, rw.R, cfg.vocab, cfg.top_b, c->top_ids, c->top_vals, st); ++nl; }
     AcceptArgs a{};
@@ -336,6 +338,7 @@ int firp_create(const firp_model_cfg *cfg, firp_ctx **out) {
   const char *eg = getenv("FIRP_GEMM"), *ep = getenv("FIRP_PDL");
   c->use_tc = !(eg && strcmp(eg, "mma") == 0);
   c->use_pdl = !(ep && strcmp(ep, "0") == 0);
+
   c->ws_bytes = c->carve(nullptr);
   *out = c;
   return FIRP_OK;

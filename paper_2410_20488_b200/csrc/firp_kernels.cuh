@@ -26,6 +26,25 @@ struct Rows {
   int anchor;  // tree row the pseudo chain hangs off
 };
 
+constexpr int kGemmMaxCtas = 192;         // scratch slots are provided for this many CTAs
+constexpr int kGemmSlots = 3;             // partial tiles (segments) per CTA
+
+// Stream-K schedule of one GEMM launch.  Unit u = supertile * KB + k block (supertile = 256 weight
+// rows, k block = 64 elements); CTA c owns units [sk_begin(c), sk_begin(c + 1)) and its s-th segment
+// is the part of supertile sk_begin(c) / KB + s inside that range.
+struct StreamK {
+  long long U;  // units
+  int KB;       // k blocks per supertile
+  int G;        // CTAs (<= U, so no range is empty)
+};
+__host__ __device__ __forceinline__ long long sk_begin(const StreamK &s, int c) { return (s.U * c) / s.G; }
+__host__ __device__ __forceinline__ int sk_owner(const StreamK &s, long long u) {   // CTA whose range holds unit u
+  int c = (int)((u * s.G) / s.U);
+  while (c + 1 < s.G && sk_begin(s, c + 1) <= u) ++c;
+  while (c > 0 && sk_begin(s, c) > u) --c;
+  return c;
+}
+
 // ---- tree bookkeeping (Section 3.4) ---------------------------------------
 struct TreeMeta {
   int32_t *depth;      // [R]
@@ -43,9 +62,17 @@ void launch_embed(const Rows &rw, const int32_t *d_tokens, const bf16 *embed, in
 // Activations that feed a GEMM or the attention are stored as two bf16 planes (hi, lo) with
 // hi + lo = the fp32 value to ~16 mantissa bits; the lo plane starts *_lo_off elements after hi.
 
-// h[r] += sum_s partial[s][r] (s < n_partial), then x[r] = rmsnorm(h[r]) * g, for rows with v in [v0, v1)
-void launch_add_rmsnorm(const Rows &rw, int v0, int v1, float *h, const float *partial, int n_partial, size_t partial_stride,
-                        const bf16 *g, float eps, int d, bf16 *x, size_t x_lo_off, cudaStream_t st);
+// Partial tiles a stream-K GEMM left in scratch: slot (c, s) = segment s of CTA c, laid out
+// [2 tiles][ws_rows token rows][128 lanes] fp32; whoever consumes the GEMM sums them in CTA order.
+struct Partials {
+  StreamK sk;        // schedule of the GEMM that wrote the tiles (U = 0: nothing pending)
+  const float *ws;   // its scratch slots
+  int ws_rows;       // token rows per scratch tile
+};
+// For rows with v in [v0, v1): if `pending` has units, first h[r] += the partial tiles of a residual GEMM;
+// then x[r] = rmsnorm(h[r]) * g as a (hi, lo) bf16 pair.
+cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Partials &pending, const bf16 *g, float eps,
+                           int d, bf16 *x, size_t x_lo_off, bool pdl, cudaStream_t st);
 
 // Eq. 3: h[s*Ms + T + i] = W_i h[s*Ms + anchor] + b_i
 void launch_pseudo_proj(const Rows &rw, const bf16 *pred_w, const bf16 *pred_b, int d, float *h, cudaStream_t st);
@@ -86,7 +113,7 @@ void launch_commit(int n_seq, const CommitArgs &a, cudaStream_t st);
 void launch_advance_ctx(int n_seq, const int32_t *seq_ids, int32_t *ctx_len, int amount, cudaStream_t st);
 
 // ---- skinny weight-streaming GEMM ------------------------------------------
-enum GemmEpilogue { EPI_PARTIAL = 0, EPI_QKV_ROPE = 1, EPI_SWIGLU = 2, EPI_LOGITS = 3 };
+enum GemmEpilogue { EPI_RESIDUAL = 0, EPI_QKV_ROPE = 1, EPI_SWIGLU = 2, EPI_LOGITS = 3 };
 
 struct GemmArgs {
   const bf16 *X;    // [R][K] activations, hi plane (row-major, K contiguous)
@@ -96,11 +123,13 @@ struct GemmArgs {
   int R;            // valid rows
   int *err;         // device status word (set to a non-zero code if a bounded wait gives up)
   int N, K;
-  int splits;       // split-K factor (EPI_PARTIAL only)
-  // EPI_PARTIAL: out[split][R][N] fp32
-  float *partial; size_t partial_stride;
+  Rows rw; int rows_active;      // rows with v < rows_active are written, the others skipped
+  // stream-K scratch of the tcgen05 kernel: partial tiles [kGemmMaxCtas][kGemmSlots][2][plane_rows][128] fp32
+  float *ws;
+  // EPI_RESIDUAL: the result is to be added to h_out[R][N] (the mma.sync kernel adds it itself; the
+  // tcgen05 kernel leaves partial tiles for the RMSNorm kernel that follows)
+  float *h_out;
   // EPI_QKV_ROPE
-  Rows rw; int rows_active;      // rows with v < rows_active are written
   int H, Hkv, dh;
   const float2 *rope; const int32_t *seq_ids; const int32_t *ctx_len;
   bf16 *q; size_t q_lo_off;      // [R][H*dh] hi plane, lo plane
@@ -110,12 +139,14 @@ struct GemmArgs {
   // EPI_LOGITS: logits[R][N]
   float *logits;
 };
-// use_tc: tcgen05/TMA kernel (needs pdl-capable launch); otherwise the mma.sync kernel.
+// use_tc: tcgen05/TMA kernel: leaves partial tiles in a.ws under the schedule *sk_out, to be finished by
+// launch_gemm_finish (or, for EPI_RESIDUAL, by launch_rmsnorm).  Otherwise the mma.sync kernel (a debugging
+// cross-check) with the epilogue fused: *sk_out gets U = 0, nothing is pending.
 // pdl: launch with programmatic stream serialization (the kernel waits on its predecessor itself).
-cudaError_t launch_gemm(GemmEpilogue epi, const GemmArgs &a, bool use_tc, bool pdl, cudaStream_t st);
-int gemm_split_k(int N, int K, bool use_tc);   // split factor used for EPI_PARTIAL at this shape
+cudaError_t launch_gemm(GemmEpilogue epi, const GemmArgs &a, bool use_tc, bool pdl, cudaStream_t st, StreamK *sk_out);
+cudaError_t launch_gemm_finish(GemmEpilogue epi, const Partials &p, const GemmArgs &a, bool pdl, cudaStream_t st);
 cudaError_t launch_gemm_mma(GemmEpilogue epi, const GemmArgs &a, cudaStream_t st);
-cudaError_t launch_gemm_tc(GemmEpilogue epi, const GemmArgs &a, bool pdl, cudaStream_t st);
+cudaError_t launch_gemm_tc(GemmEpilogue epi, const GemmArgs &a, bool pdl, cudaStream_t st, StreamK *sk_out);
 bool gemm_tc_available();         // the driver entry point for tensor-map encoding was found
 
 // ---- tree-masked split-KV attention ---------------------------------------

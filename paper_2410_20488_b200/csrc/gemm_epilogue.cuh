@@ -45,11 +45,10 @@ template <int EPI, int BN>
 __device__ __forceinline__ void gemm_epilogue(const float *C, int ldc, int tile, int split, const GemmArgs &a,
                                               const TileMap &tm, int tid, int nthreads) {
   constexpr int G = BN / 2;
-  if (EPI == EPI_PARTIAL) {
-    float *out = a.partial + (size_t)split * a.partial_stride;
+  if (EPI == EPI_RESIDUAL) {   // every k split adds its partial sums into the residual stream
     for (int idx = tid; idx < a.R * BN; idx += nthreads) {
       const int m = idx / BN, col = idx % BN, n = tile * BN + col;
-      if (n < a.N) out[(size_t)m * a.N + n] = C[m * ldc + col];
+      if (n < a.N && (m % a.rw.Ms) < a.rows_active) atomicAdd(a.h_out + (size_t)m * a.N + n, C[m * ldc + col]);
     }
   } else if (EPI == EPI_LOGITS) {
     for (int idx = tid; idx < a.R * BN; idx += nthreads) {

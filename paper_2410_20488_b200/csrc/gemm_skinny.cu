@@ -44,7 +44,7 @@ __device__ __forceinline__ void mma_bf16(float *c, const uint32_t *a, uint32_t b
 // MT = number of 8-token MMA n-tiles (token rows padded to MT*8)
 template <int MT, int EPI, int STAGES>
 __global__ void __launch_bounds__(kThreads)
-gemm_skinny_mma_kernel(GemmArgs a, TileMap tm) {
+gemm_skinny_mma_kernel(GemmArgs a, TileMap tm, int splits) {
   constexpr int MT2 = (MT + 1) / 2;                 // ldmatrix.x4 covers two n-tiles
   constexpr int XROWS = MT2 * 16;
   constexpr int W_BYTES = BN * 128, X_BYTES = XROWS * 128, STAGE_BYTES = W_BYTES + 2 * X_BYTES;   // W, X hi, X lo
@@ -52,7 +52,7 @@ gemm_skinny_mma_kernel(GemmArgs a, TileMap tm) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
   const int kb_total = (a.K + BK - 1) / BK;
-  const int kb_per = (kb_total + a.splits - 1) / a.splits;
+  const int kb_per = (kb_total + splits - 1) / splits;
   const int kb0 = split * kb_per, kb1 = min(kb_total, kb0 + kb_per);
   const int nkb = max(kb1 - kb0, 0);
 
@@ -135,6 +135,17 @@ gemm_skinny_mma_kernel(GemmArgs a, TileMap tm) {
   gemm_epilogue<EPI, BN>(C, LDC, tile, split, a, tm, tid, kThreads);
 }
 
+// split-K factor of the residual GEMMs: enough CTAs to cover the SMs about twice, at least
+// 8 k-blocks per split, and no empty split
+int split_k(int N, int K) {
+  const int tiles = (N + BN - 1) / BN, kb = (K + BK - 1) / BK;
+  int s = (2 * 148 + tiles - 1) / tiles;
+  s = s < 1 ? 1 : (s > 8 ? 8 : s);
+  while (s > 1 && kb / s < 8) --s;
+  const int per = (kb + s - 1) / s;
+  return (kb + per - 1) / per;
+}
+
 template <int MT, int EPI>
 cudaError_t launch_mt(const GemmArgs &a, const TileMap &tm, int tiles, cudaStream_t st) {
   constexpr int MT2 = (MT + 1) / 2;
@@ -147,10 +158,8 @@ cudaError_t launch_mt(const GemmArgs &a, const TileMap &tm, int tiles, cudaStrea
     cudaFuncSetAttribute(gemm_skinny_mma_kernel<MT, EPI, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
     configured = true;
   }
-  const int splits = (EPI == EPI_PARTIAL) ? a.splits : 1;
-  GemmArgs b = a;
-  b.splits = splits;
-  gemm_skinny_mma_kernel<MT, EPI, STAGES><<<dim3(tiles, splits), kThreads, SMEM, st>>>(b, tm);
+  const int splits = (EPI == EPI_RESIDUAL) ? split_k(a.N, a.K) : 1;
+  gemm_skinny_mma_kernel<MT, EPI, STAGES><<<dim3(tiles, splits), kThreads, SMEM, st>>>(a, tm, splits);
   return cudaGetLastError();
 }
 
@@ -164,17 +173,6 @@ cudaError_t launch_epi(const GemmArgs &a, const TileMap &tm, int tiles, cudaStre
 }
 
 }  // namespace
-
-int gemm_split_k(int N, int K, bool use_tc) {
-  // enough CTAs to cover the SMs about twice, at least 8 k-blocks per split, and no empty split
-  const int bn = use_tc ? 128 : BN;
-  const int tiles = (N + bn - 1) / bn, kb = (K + BK - 1) / BK;
-  int s = (2 * 148 + tiles - 1) / tiles;
-  s = s < 1 ? 1 : (s > 8 ? 8 : s);
-  while (s > 1 && kb / s < 8) --s;
-  const int per = (kb + s - 1) / s;
-  return (kb + per - 1) / per;
-}
 
 cudaError_t launch_gemm_mma(GemmEpilogue epi, const GemmArgs &a, cudaStream_t st) {
   TileMap tm{};
@@ -190,12 +188,14 @@ cudaError_t launch_gemm_mma(GemmEpilogue epi, const GemmArgs &a, cudaStream_t st
     case EPI_LOGITS:
       return launch_epi<EPI_LOGITS>(a, tm, (a.N + BN - 1) / BN, st);
     default:
-      return launch_epi<EPI_PARTIAL>(a, tm, (a.N + BN - 1) / BN, st);
+      return launch_epi<EPI_RESIDUAL>(a, tm, (a.N + BN - 1) / BN, st);
   }
 }
 
-cudaError_t launch_gemm(GemmEpilogue epi, const GemmArgs &a, bool use_tc, bool pdl, cudaStream_t st) {
-  return use_tc ? launch_gemm_tc(epi, a, pdl, st) : launch_gemm_mma(epi, a, st);
+cudaError_t launch_gemm(GemmEpilogue epi, const GemmArgs &a, bool use_tc, bool pdl, cudaStream_t st, StreamK *sk_out) {
+  if (use_tc) return launch_gemm_tc(epi, a, pdl, st, sk_out);
+  if (sk_out) *sk_out = StreamK{0, 1, 1};   // the mma.sync kernel adds into the residual stream itself
+  return launch_gemm_mma(epi, a, st);
 }
 
 }  // namespace firp

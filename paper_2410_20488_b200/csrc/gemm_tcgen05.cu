@@ -1,21 +1,37 @@
 // Skinny weight-streaming GEMM on the 5th-generation tensor cores (tcgen05 + TMEM), operands
 // staged by TMA.  out[m][n] = sum_k X[m][k] * W[n][k], M = T + k token rows, W read once.
 //
-// Roles are swapped: a tile is 128 weight rows (the MMA M dimension, one TMEM lane each) by all
-// token rows (the MMA N dimension, one TMEM column each).  Per CTA:
-//   warp 0   : weight producer.  One thread streams [128 rows x 64 k] bf16 tiles (two 64-row TMA
-//              boxes, 128-byte swizzle) through a deep ring.  Weights never depend on the previous
-//              kernel, so this warp does not wait for it: under programmatic dependent launch the
-//              weight stream of this GEMM starts while its predecessor drains.
-//   warp 6   : activation producer.  Streams the matching [NPAD x 64] hi and lo activation tiles
-//              (L2-resident) through a short ring, after waiting for the previous kernel.
-//   warp 1   : MMA issuer.  One thread issues tcgen05.mma (M=128, N=NPAD, K=16, bf16 x bf16 -> fp32
-//              in TMEM): per 64-wide k block 4 steps x {hi, lo} activations into one accumulator;
-//              tcgen05.commit hands ring slots back to the producers.
-//   warps 2-5: epilogue.  tcgen05.ld the accumulator (lane = weight row, column = token), stage it
-//              as C[token][row] in shared memory and run the fused epilogue.
-// Every mbarrier wait is bounded: after ~2 s it sets the status word and falls through, so a
-// broken pipeline ends with an error code instead of a hang; TMEM is always released.
+// Roles are swapped: weight rows are the MMA M dimension (one TMEM lane each), token rows the
+// MMA N dimension (one TMEM column each).  A "supertile" is 2 x 128 weight rows that share one
+// activation tile per k block, chosen so that both operands of a fused epilogue meet in one
+// thread: lane i of the first 128 rows and lane i of the second are a rotary pair (c, c + dh/2),
+// a gate row and its up row, or simply rows n and n + 128.
+//
+// Persistent stream-K schedule: the (supertile, k block) units of the whole matrix, 32 KB of
+// weights each, are cut into one contiguous range per SM, so every SM streams the same number of
+// bytes whatever the matrix shape.  A range crosses supertile boundaries; each piece ("segment")
+// accumulates in TMEM and its fp32 partial tile is stored to the CTA's scratch slot.  The kernel
+// that consumes the GEMM (RMSNorm for the residual GEMMs, the rotary / SwiGLU / logits finishers
+// otherwise) sums the slots of a supertile in CTA order, so every sum has a fixed order and results
+// are identical from run to run; no CTA ever waits for another.  The finishers are small-footprint
+// kernels that stay resident beside the next GEMM's CTAs: under programmatic dependent launch the
+// next weight stream starts while they run.
+//
+// Per CTA (one per SM):
+//   warp 0   : weight producer (one thread, TMA, 128-byte swizzle, deep ring).  Weights never
+//              depend on the previous kernel, so under programmatic dependent launch this stream
+//              starts while the predecessor drains.
+//   warp 6   : activation producer: the (hi, lo) bf16 planes of the matching k block (L2
+//              resident, own shorter ring), after waiting for the previous kernel.
+//   warp 1   : MMA issuer: tcgen05.mma kind::f16, M = 128, K = 16; the hi and lo planes sit one
+//              after the other in shared memory and are multiplied as ONE operand of N = 2 NPAD
+//              token columns (hi sums and lo sums land in neighbouring TMEM columns and are added
+//              in the epilogue); tcgen05.commit releases ring slots.
+//   warps 2-5: epilogue: tcgen05.ld (lane = weight row, column = token), hi + lo, store of the
+//              partial tile; overlapped with the next segment's main loop through a second
+//              accumulator buffer.
+// Every mbarrier wait is bounded (~2 s): on expiry the status word is set and the kernel runs to
+// its end; TMEM is always released.
 #include <cuda.h>
 
 #include <map>
@@ -23,15 +39,18 @@
 
 #include "firp_kernels.cuh"
 #include "gemm_epilogue.cuh"
+#include "launch_util.cuh"
 
 namespace firp {
 
 namespace {
 
-constexpr int BM = 128;           // weight rows per tile
-constexpr int BK = kGemmBK;       // 64 bf16 = 128 bytes = one swizzle row
-constexpr int kThreads = 224;     // 7 warps
-constexpr int W_TILE = BM * 128;  // bytes per weight stage
+constexpr int BM = 128;            // weight rows per MMA tile
+constexpr int TM = 2;              // MMA tiles per supertile
+constexpr int BK = kGemmBK;        // 64 bf16 = 128 bytes = one swizzle row
+constexpr int kThreads = 224;      // 7 warps
+constexpr int W_TILE = BM * 128;   // bytes of one 128-row weight tile of a k block
+constexpr int W_STAGE = TM * W_TILE;
 constexpr int kErrTimeout = 100;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -45,6 +64,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -71,9 +93,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm,
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
       ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
 }
-__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm, int x, int y, int z, int w, uint32_t bar,
+                                            uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -83,13 +108,15 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t
   asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t *r) {
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float *r) {
+  uint32_t *u = reinterpret_cast<uint32_t *>(r);
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                 "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+               : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+                 "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15])
                : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // Shared-memory operand descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups
 // 1024 bytes apart (start address >> 4 in bits 0-13, leading offset 1 in bits 16-29 (unused for
@@ -105,49 +132,68 @@ __host__ __device__ constexpr uint32_t instr_desc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
 
+constexpr int pow2_cols(int c) { return c <= 32 ? 32 : c <= 64 ? 64 : c <= 128 ? 128 : c <= 256 ? 256 : 512; }
+
+// NPAD = token rows padded to a multiple of 8 (16 when the planes cannot be merged).
 template <int NPAD> struct TcCfg {
-  static constexpr int X_TILE = NPAD * 128;                      // bytes of one activation plane per stage
-  static constexpr int WS = (NPAD <= 48) ? 5 : (NPAD <= 80 ? 4 : 8);  // weight ring depth (two CTAs per SM up to NPAD = 80)
-  static constexpr int XS = 2;                                   // activation ring depth
-  static constexpr int TMEM_COLS = NPAD <= 32 ? 32 : (NPAD <= 64 ? 64 : (NPAD <= 128 ? 128 : 256));
-  static constexpr int RING_BYTES = WS * W_TILE + XS * 2 * X_TILE;
-  static constexpr int C_BYTES = NPAD * BM * 4;
-  static constexpr int DATA_BYTES = RING_BYTES > C_BYTES ? RING_BYTES : C_BYTES;
-  static constexpr int SMEM = DATA_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+  static constexpr int X_PLANE = NPAD * 128;                   // bytes of one activation plane per stage
+  static constexpr int X_STAGE = 2 * X_PLANE;                  // hi plane, then lo plane
+  static constexpr bool MERGE = (2 * NPAD <= 256);             // hi and lo as one MMA operand of N = 2 NPAD
+  static constexpr int ACC_COLS = MERGE ? 2 * NPAD : NPAD;     // accumulator columns per weight tile
+  static constexpr int NBUF = (2 * TM * ACC_COLS <= 512) ? 2 : 1;   // accumulator buffers
+  static constexpr int TMEM_COLS = pow2_cols(NBUF * TM * ACC_COLS);
+  static constexpr int SW = NPAD <= 40 ? 6 : (NPAD <= 80 ? 5 : 4);  // weight ring depth (32 KB stages)
+  static constexpr int SX = NPAD <= 16 ? 4 : (NPAD <= 40 ? 3 : (NPAD <= 48 ? 4 : (NPAD <= 80 ? 3 : 2)));
+  static constexpr int RING_BYTES = SW * W_STAGE + SX * X_STAGE;
+  static constexpr int SMEM = RING_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+  static_assert(SMEM <= 227 * 1024, "shared memory budget");
+  static_assert((2 * SW + 2 * SX + 2 * NBUF) * 8 + 8 <= 256, "barrier area");
 };
 
-struct TcArgs {
-  int box1_off;   // rows from the first 64-row box of a tile to the second (64, or pair_off)
-  int tile_rows;  // rows a tile advances the first box by (128 contiguous, 64 paired)
-  int pdl;        // launched with programmatic stream serialization
+// How the 2 x 128 rows of supertile `st` map to weight rows.
+//   ROWS_LINEAR   rows st*256 .. +255 (two boxes of 128 rows)
+//   ROWS_GATE_UP  gate rows st*128 .. +127, then the matching up rows F + st*128 ..
+//   ROWS_ROTARY   first halves (c < dh/2) of 128/(dh/2) heads, then their second halves, fetched
+//                 through a 4-D view [head][half][c][k] of the weight so that each is one box
+enum RowMode { ROWS_LINEAR = 0, ROWS_GATE_UP = 1, ROWS_ROTARY = 2 };
+struct Sched {
+  StreamK sk;      // units, k blocks per supertile, CTAs
+  int mode;        // RowMode
+  int F;           // ROWS_GATE_UP: rows of the gate matrix
+  int half;        // ROWS_ROTARY: dh / 2
+  int n_st;        // supertiles
+  int pdl;         // launched with programmatic stream serialization
+  int ws_rows;     // token rows per scratch tile
 };
 
-template <int NPAD, int EPI>
+template <int NPAD>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, GemmArgs a,
-               TileMap tm, TcArgs t) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, GemmArgs a, Sched sc) {
   using Cfg = TcCfg<NPAD>;
-  constexpr int WS = Cfg::WS, XS = Cfg::XS, X_TILE = Cfg::X_TILE;
+  constexpr int SW = Cfg::SW, SX = Cfg::SX, X_STAGE = Cfg::X_STAGE, X_PLANE = Cfg::X_PLANE, NBUF = Cfg::NBUF;
+  constexpr int ACC = Cfg::ACC_COLS;
+  constexpr bool MERGE = Cfg::MERGE;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;      // swizzled tiles need 1024-byte alignment
   uint8_t *data = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t w_ring = base, x_ring = base + WS * W_TILE;
-  const uint32_t bars = base + Cfg::DATA_BYTES;                     // 8-byte barriers
-  const uint32_t full_w = bars, empty_w = bars + 8 * WS, full_x = bars + 16 * WS, empty_x = full_x + 8 * XS,
-                 accum_bar = empty_x + 8 * XS, tmem_slot = accum_bar + 8;
-  volatile uint32_t *tmem_slot_ptr = reinterpret_cast<volatile uint32_t *>(data + Cfg::DATA_BYTES + 16 * WS + 16 * XS + 8);
+  const uint32_t w_ring = base, x_ring = base + SW * W_STAGE;
+  const uint32_t bars = base + Cfg::RING_BYTES;                     // 8-byte barriers
+  const uint32_t full_w = bars, empty_w = full_w + 8 * SW, full_x = empty_w + 8 * SW, empty_x = full_x + 8 * SX,
+                 acc_full = empty_x + 8 * SX, acc_empty = acc_full + 8 * NBUF, tmem_slot = acc_empty + 8 * NBUF;
+  volatile uint32_t *tmem_slot_ptr =
+      reinterpret_cast<volatile uint32_t *>(data + Cfg::RING_BYTES + 16 * SW + 16 * SX + 16 * NBUF);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile = blockIdx.x, split = blockIdx.y;
-  const int kb_total = (a.K + BK - 1) / BK;
-  const int kb_per = (kb_total + a.splits - 1) / a.splits;
-  const int kb0 = split * kb_per;
-  const int nkb = max(min(kb_total, kb0 + kb_per) - kb0, 0);
+  const int cta = blockIdx.x;
+  const StreamK sk = sc.sk;
+  const int KB = sk.KB;
+  const long long u0 = sk_begin(sk, cta), u1 = sk_begin(sk, cta + 1);
+  const int n_units = (int)(u1 - u0);
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < WS; ++i) { mbar_init(full_w + 8 * i, 1); mbar_init(empty_w + 8 * i, 1); }
-    for (int i = 0; i < XS; ++i) { mbar_init(full_x + 8 * i, 1); mbar_init(empty_x + 8 * i, 1); }
-    mbar_init(accum_bar, 1);
+    for (int i = 0; i < SW; ++i) { mbar_init(full_w + 8 * i, 1); mbar_init(empty_w + 8 * i, 1); }
+    for (int i = 0; i < SX; ++i) { mbar_init(full_x + 8 * i, 1); mbar_init(empty_x + 8 * i, 1); }
+    for (int i = 0; i < NBUF; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {   // TMEM: one warp allocates (and later frees) the accumulator columns
@@ -157,85 +203,136 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_acc = *tmem_slot_ptr;
-  if (t.pdl) griddep_launch();   // the next kernel may start its own weight stream
+  const uint32_t tmem_base = *tmem_slot_ptr;
+  if (sc.pdl) griddep_launch();   // the next kernel may start its own weight stream as SMs free up
 
   bool dead = false;
   if (warp == 0) {
     if (lane == 0) {             // ---- weight producer: does not wait for the previous kernel
       uint64_t pol;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-      const int r0 = tile * t.tile_rows, r1 = r0 + t.box1_off;
-      for (int it = 0; it < nkb; ++it) {
-        const int st = it % WS;
-        mbar_wait(empty_w + 8 * st, ((it / WS) & 1) ^ 1, a.err, dead);
-        mbar_expect_tx(full_w + 8 * st, W_TILE);
-        const int k0 = (kb0 + it) * BK;
-        tma_load_2d(w_ring + st * W_TILE, &tmW, k0, r0, full_w + 8 * st, pol);
-        tma_load_2d(w_ring + st * W_TILE + W_TILE / 2, &tmW, k0, r1, full_w + 8 * st, pol);
+      for (int it = 0; it < n_units; ++it) {
+        const long long u = u0 + it;
+        const int st = (int)(u / KB), kb = (int)(u - (long long)st * KB);
+        const int sl = it % SW;
+        mbar_wait(empty_w + 8 * sl, ((it / SW) & 1) ^ 1, a.err, dead);
+        mbar_expect_tx(full_w + 8 * sl, W_STAGE);
+        const uint32_t dst = w_ring + sl * W_STAGE, bar = full_w + 8 * sl;
+        if (sc.mode == ROWS_ROTARY) {
+          const int hp = BM / sc.half;               // heads per supertile
+          tma_load_4d(dst, &tmW, kb * BK, 0, 0, st * hp, bar, pol);
+          tma_load_4d(dst + W_TILE, &tmW, kb * BK, 0, 1, st * hp, bar, pol);
+        } else if (sc.mode == ROWS_GATE_UP) {
+          tma_load_2d(dst, &tmW, kb * BK, st * BM, bar, pol);
+          tma_load_2d(dst + W_TILE, &tmW, kb * BK, sc.F + st * BM, bar, pol);
+        } else {
+          tma_load_2d(dst, &tmW, kb * BK, st * (TM * BM), bar, pol);
+          tma_load_2d(dst + W_TILE, &tmW, kb * BK, st * (TM * BM) + BM, bar, pol);
+        }
       }
     }
   } else if (warp == 6) {
     if (lane == 0) {             // ---- activation producer
       uint64_t pol;
       asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-      if (t.pdl) griddep_wait();
-      for (int it = 0; it < nkb; ++it) {
-        const int st = it % XS;
-        mbar_wait(empty_x + 8 * st, ((it / XS) & 1) ^ 1, a.err, dead);
-        mbar_expect_tx(full_x + 8 * st, 2 * X_TILE);
-        const int k0 = (kb0 + it) * BK;
-        tma_load_2d(x_ring + st * 2 * X_TILE, &tmX, k0, 0, full_x + 8 * st, pol);
-        tma_load_2d(x_ring + st * 2 * X_TILE + X_TILE, &tmX, k0, a.plane_rows, full_x + 8 * st, pol);
+      if (sc.pdl) griddep_wait();
+      const int xrows = min((a.R + 7) & ~7, NPAD);
+      for (int it = 0; it < n_units; ++it) {
+        const int kb = (int)((u0 + it) % KB);
+        const int sl = it % SX;
+        mbar_wait(empty_x + 8 * sl, ((it / SX) & 1) ^ 1, a.err, dead);
+        mbar_expect_tx(full_x + 8 * sl, 2 * xrows * 128);
+        const uint32_t dst = x_ring + sl * X_STAGE;
+        tma_load_2d(dst, &tmX, kb * BK, 0, full_x + 8 * sl, pol);
+        tma_load_2d(dst + X_PLANE, &tmX, kb * BK, a.plane_rows, full_x + 8 * sl, pol);
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {             // ---- MMA issuer
-      constexpr uint32_t idesc = instr_desc(NPAD);
-      for (int it = 0; it < nkb; ++it) {
-        const int sw = it % WS, sx = it % XS;
-        mbar_wait(full_w + 8 * sw, (it / WS) & 1, a.err, dead);
-        mbar_wait(full_x + 8 * sx, (it / XS) & 1, a.err, dead);
+      constexpr uint32_t idesc = instr_desc(MERGE ? 2 * NPAD : NPAD);
+      int it = 0, seg = 0;
+      long long u = u0;
+      while (u < u1) {
+        const int st = (int)(u / KB), kb0 = (int)(u - (long long)st * KB);
+        const int kb1 = (int)min((long long)KB, kb0 + (u1 - u));
+        const int buf = seg % NBUF;
+        mbar_wait(acc_empty + 8 * buf, ((seg / NBUF) & 1) ^ 1, a.err, dead);   // epilogue has drained this buffer
         tc_fence_after();
-        const uint64_t da = smem_desc(w_ring + sw * W_TILE);
-        const uint64_t dhi = smem_desc(x_ring + sx * 2 * X_TILE), dlo = smem_desc(x_ring + sx * 2 * X_TILE + X_TILE);
+        const uint32_t acc = tmem_base + (uint32_t)(buf * TM * ACC);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+          const int sw = it % SW, sx = it % SX;
+          mbar_wait(full_w + 8 * sw, (it / SW) & 1, a.err, dead);
+          mbar_wait(full_x + 8 * sx, (it / SX) & 1, a.err, dead);
+          tc_fence_after();
+          const uint32_t wst = w_ring + sw * W_STAGE, xst = x_ring + sx * X_STAGE;
+          const uint64_t dhi = smem_desc(xst), dlo = smem_desc(xst + X_PLANE);
 #pragma unroll
-        for (int kk = 0; kk < BK / 16; ++kk) {
-          tc_mma(tmem_acc, da + 2 * kk, dhi + 2 * kk, idesc, (it | kk) != 0);
-          tc_mma(tmem_acc, da + 2 * kk, dlo + 2 * kk, idesc, 1u);
+          for (int kk = 0; kk < BK / 16; ++kk) {
+#pragma unroll
+            for (int t = 0; t < TM; ++t) {
+              const uint64_t da = smem_desc(wst + t * W_TILE) + 2 * kk;
+              tc_mma(acc + t * ACC, da, dhi + 2 * kk, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+              if (!MERGE) tc_mma(acc + t * ACC, da, dlo + 2 * kk, idesc, 1u);
+            }
+          }
+          tc_commit(empty_w + 8 * sw);   // the slots are free once these MMAs have read them
+          tc_commit(empty_x + 8 * sx);
         }
-        tc_commit(empty_w + 8 * sw);   // slots are free once these MMAs have read them
-        tc_commit(empty_x + 8 * sx);
+        tc_commit(acc_full + 8 * buf);
+        u += kb1 - kb0;
+        ++seg;
       }
-      tc_commit(accum_bar);
     }
   } else {                       // ---- epilogue warps 2..5: TMEM lane quarter = warp % 4
-    if (t.pdl) griddep_wait();
+    if (sc.pdl) griddep_wait();
     const int quarter = warp & 3;
-    const int row = quarter * 32 + lane;          // tile-local weight row = TMEM lane
-    float *C = reinterpret_cast<float *>(data);   // C[token][BM], reuses the rings
-    if (nkb > 0) {
-      mbar_wait(accum_bar, 0, a.err, dead);
+    const int i = quarter * 32 + lane;            // row within each 128-row tile = TMEM lane
+    const size_t plane_elems = (size_t)sc.ws_rows * BM, slot_elems = TM * plane_elems;
+    int seg = 0;
+    long long u = u0;
+    while (u < u1) {
+      const int st = (int)(u / KB), kb0 = (int)(u - (long long)st * KB);
+      const int kb1 = (int)min((long long)KB, kb0 + (u1 - u));
+      const int buf = seg % NBUF;
+      mbar_wait(acc_full + 8 * buf, (seg / NBUF) & 1, a.err, dead);
       tc_fence_after();
+      const uint32_t tacc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * TM * ACC);
+      float *my_ws = a.ws + (size_t)(cta * kGemmSlots + seg) * slot_elems + i;
+      for (int c0 = 0; c0 < a.R && seg < kGemmSlots; c0 += 16) {
+        float r0[16], r1[16];
+        tc_ld16(tacc + c0, r0);
+        tc_ld16(tacc + ACC + c0, r1);
+        if (MERGE) {             // columns NPAD.. hold the sums over the lo plane
+          float l0[16], l1[16];
+          tc_ld16(tacc + NPAD + c0, l0);
+          tc_ld16(tacc + ACC + NPAD + c0, l1);
+          tc_ld_wait();
 #pragma unroll
-      for (int c0 = 0; c0 < NPAD; c0 += 16) {
-        uint32_t r[16];
-        tc_ld16(tmem_acc + ((uint32_t)(quarter * 32) << 16) + c0, r);
-        tc_ld_wait();
+          for (int j = 0; j < 16; ++j) { r0[j] += l0[j]; r1[j] += l1[j]; }
+        } else {
+          tc_ld_wait();
+        }
 #pragma unroll
-        for (int j = 0; j < 16; ++j) C[(c0 + j) * BM + row] = __uint_as_float(r[j]);
+        for (int j = 0; j < 16; ++j) {
+          const int m = c0 + j;
+          if (m < a.R) {
+            __stcg(my_ws + (size_t)m * BM, r0[j]);
+            __stcg(my_ws + plane_elems + (size_t)m * BM, r1[j]);
+          }
+        }
       }
-    } else {
-      for (int m = 0; m < NPAD; ++m) C[m * BM + row] = 0.f;
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty + 8 * buf);   // the MMA warp may reuse this accumulator
+      u += kb1 - kb0;
+      ++seg;
     }
-    tc_fence_before();
-    asm volatile("bar.sync 1, 128;" ::: "memory");
-    gemm_epilogue<EPI, BM>(C, BM, tile, split, a, tm, threadIdx.x - 64, 128);
   }
+  tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(Cfg::TMEM_COLS) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(Cfg::TMEM_COLS) : "memory");
   }
 }
 
@@ -258,43 +355,67 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// 2-D bf16 tensor [rows][K] (K contiguous), box [box_rows][64], 128-byte swizzle, zero fill out of bounds.
+// bf16 tensor maps with 64-element (128-byte) inner boxes, 128-byte swizzle, zero fill out of bounds.
+//   half == 0: 2-D [rows][K], box [box_rows][64]
+//   half  > 0: 4-D view [rows / (2 half)][2][half][K] of a QKV weight, box [128 / half][1][half][64]:
+//              the same half of 128 / half neighbouring heads
 // Encoded maps are cached: the same few (pointer, shape) pairs recur every step.
-bool make_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t K, uint32_t box_rows) {
-  typedef std::tuple<const void *, uint64_t, uint64_t, uint32_t> Key;
+bool make_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t K, uint32_t box_rows, uint32_t half) {
+  typedef std::tuple<const void *, uint64_t, uint64_t, uint32_t, uint32_t> Key;
   static std::map<Key, CUtensorMap> cache;
-  const Key key(ptr, rows, K, box_rows);
+  const Key key(ptr, rows, K, box_rows, half);
   auto it = cache.find(key);
   if (it != cache.end()) { *m = it->second; return true; }
-  const cuuint64_t dims[2] = {K, rows};
-  const cuuint64_t strides[1] = {K * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  if (encode_fn()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return false;
+  CUresult rc;
+  if (half == 0) {
+    const cuuint64_t dims[2] = {K, rows};
+    const cuuint64_t strides[1] = {K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    rc = encode_fn()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else {
+    const cuuint64_t dims[4] = {K, half, 2, rows / (2 * half)};
+    const cuuint64_t strides[3] = {K * 2, (cuuint64_t)half * K * 2, (cuuint64_t)2 * half * K * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)BK, half, 1, (cuuint32_t)BM / half};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    rc = encode_fn()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(ptr), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
+  if (rc != CUDA_SUCCESS) return false;
   if (cache.size() > 4096) cache.clear();
   cache[key] = *m;
   return true;
 }
 
-template <int NPAD, int EPI>
-cudaError_t launch_np(const GemmArgs &a, const TileMap &tm, const TcArgs &t, int tiles, cudaStream_t st) {
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 1;
+  }
+  return n;
+}
+
+template <int NPAD>
+cudaError_t launch_np(const GemmArgs &a, const Sched &sc, cudaStream_t st) {
   using Cfg = TcCfg<NPAD>;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<NPAD, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<NPAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
     if (e != cudaSuccess) return e;
     configured = true;
   }
+  const int xrows = std::min((a.R + 7) & ~7, NPAD);
   CUtensorMap tmW, tmX;
-  if (!make_map(&tmW, a.W, (uint64_t)a.N, (uint64_t)a.K, 64)) return cudaErrorInvalidValue;
-  if (!make_map(&tmX, a.X, (uint64_t)a.plane_rows + a.R, (uint64_t)a.K, NPAD)) return cudaErrorInvalidValue;
-  GemmArgs b = a;
-  b.splits = (EPI == EPI_PARTIAL) ? a.splits : 1;
+  if (!make_map(&tmW, a.W, (uint64_t)a.N, (uint64_t)a.K, BM, sc.mode == ROWS_ROTARY ? (uint32_t)sc.half : 0u))
+    return cudaErrorInvalidValue;
+  if (!make_map(&tmX, a.X, (uint64_t)a.plane_rows + a.R, (uint64_t)a.K, (uint32_t)xrows, 0)) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(tiles, b.splits);
+  cfg.gridDim = dim3((unsigned)sc.sk.G);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = Cfg::SMEM;
   cfg.stream = st;
@@ -302,38 +423,49 @@ cudaError_t launch_np(const GemmArgs &a, const TileMap &tm, const TcArgs &t, int
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = t.pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<NPAD, EPI>, tmW, tmX, b, tm, t);
+  cfg.numAttrs = sc.pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<NPAD>, tmW, tmX, a, sc);
 }
 
-template <int EPI>
-cudaError_t launch_epi(const GemmArgs &a, const TileMap &tm, const TcArgs &t, int tiles, cudaStream_t st) {
-  if (a.R <= 16) return launch_np<16, EPI>(a, tm, t, tiles, st);
-  if (a.R <= 48) return launch_np<48, EPI>(a, tm, t, tiles, st);
-  if (a.R <= 80) return launch_np<80, EPI>(a, tm, t, tiles, st);
-  return launch_np<144, EPI>(a, tm, t, tiles, st);
+cudaError_t launch_rows(const GemmArgs &a, const Sched &sc, cudaStream_t st) {
+  if (a.R <= 16) return launch_np<16>(a, sc, st);
+  if (a.R <= 40) return launch_np<40>(a, sc, st);
+  if (a.R <= 48) return launch_np<48>(a, sc, st);
+  if (a.R <= 80) return launch_np<80>(a, sc, st);
+  return launch_np<144>(a, sc, st);
+}
+
+Sched make_sched(GemmEpilogue epi, const GemmArgs &a, bool pdl) {
+  Sched sc{};
+  sc.pdl = pdl ? 1 : 0;
+  sc.ws_rows = a.plane_rows;
+  sc.mode = ROWS_LINEAR; sc.n_st = (a.N + TM * BM - 1) / (TM * BM);
+  if (epi == EPI_SWIGLU) {
+    sc.mode = ROWS_GATE_UP; sc.F = a.F; sc.n_st = (a.F + BM - 1) / BM;
+  } else if (epi == EPI_QKV_ROPE) {
+    sc.mode = ROWS_ROTARY; sc.half = a.dh / 2;
+    const int hp = BM / sc.half;
+    sc.n_st = (a.H + 2 * a.Hkv + hp - 1) / hp;
+  }
+  sc.sk.KB = (a.K + BK - 1) / BK;
+  sc.sk.U = (long long)sc.n_st * sc.sk.KB;
+  sc.sk.G = (int)std::min<long long>(sm_count(), sc.sk.U);
+  return sc;
 }
 
 }  // namespace
 
 bool gemm_tc_available() { return encode_fn() != nullptr; }
 
-cudaError_t launch_gemm_tc(GemmEpilogue epi, const GemmArgs &a, bool pdl, cudaStream_t st) {
+cudaError_t launch_gemm_tc(GemmEpilogue epi, const GemmArgs &a, bool pdl, cudaStream_t st, StreamK *sk_out) {
   if (!encode_fn()) return cudaErrorNotSupported;
-  TileMap tm{};
-  TcArgs t{64, BM, pdl ? 1 : 0};
-  switch (epi) {
-    case EPI_QKV_ROPE:   // contiguous tiles of 128 / dh whole heads
-      return launch_epi<EPI_QKV_ROPE>(a, tm, t, (a.N + BM - 1) / BM, st);
-    case EPI_SWIGLU:     // 64 gate rows + the matching 64 up rows
-      tm.paired = 1; tm.tiles_per_unit = (a.F + 63) / 64; tm.unit_stride = 0; tm.pair_off = a.F; tm.group_rows = a.F;
-      t.box1_off = a.F; t.tile_rows = 64;
-      return launch_epi<EPI_SWIGLU>(a, tm, t, tm.tiles_per_unit, st);
-    case EPI_LOGITS:
-      return launch_epi<EPI_LOGITS>(a, tm, t, (a.N + BM - 1) / BM, st);
-    default:
-      return launch_epi<EPI_PARTIAL>(a, tm, t, (a.N + BM - 1) / BM, st);
-  }
+  const Sched sc = make_sched(epi, a, pdl);
+  // a CTA's range of U / G units touches at most this many supertiles, each needing a scratch slot
+  const long long per = (sc.sk.U + sc.sk.G - 1) / sc.sk.G;
+  if (sc.sk.G > kGemmMaxCtas || (per + sc.sk.KB - 2) / sc.sk.KB + 1 > kGemmSlots)
+    return cudaErrorInvalidConfiguration;
+  if (sk_out) *sk_out = sc.sk;
+  return launch_rows(a, sc, st);
 }
 
 }  // namespace firp

@@ -1,6 +1,11 @@
 // Small kernels of the FIRP step: tree bookkeeping, embedding, residual-add + RMSNorm,
 // the pseudo-hidden projection (Eq. 3), top-B, the acceptance walk / next tree, KV compaction.
+#include <cooperative_groups.h>
+
 #include "firp_kernels.cuh"
+#include "launch_util.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace firp {
 
@@ -91,7 +96,7 @@ void launch_embed(const Rows &rw, const int32_t *d_tokens, const bf16 *embed, in
 }
 
 // ---------------------------------------------------------------------------
-// Residual add of split-K partial sums + RMSNorm -> bf16 GEMM operand.
+// RMSNorm of the fp32 residual rows -> bf16 (hi, lo) GEMM operand.
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ float block_sum(float v, float *red) {
 #pragma unroll
@@ -112,39 +117,71 @@ __device__ __forceinline__ float block_sum(float v, float *red) {
 }
 
 constexpr int kNormThreads = 256;
-constexpr int kNormMaxVec = 8;  // d <= 256 * 8 * 4 = 8192
+constexpr int kNormCluster = 4;   // CTAs per token row, each owns a quarter of the columns
+constexpr int kNormMaxVec = 2;    // float4 per thread: d <= 4 * 256 * 2 * 4 = 8192
 
-__global__ void __launch_bounds__(kNormThreads)
-add_rmsnorm_kernel(Rows rw, int v0, int nv, float *__restrict__ h, const float *__restrict__ partial, int n_partial,
-                   size_t partial_stride, const bf16 *__restrict__ g, float eps, int d, bf16 *__restrict__ x,
-                   size_t x_lo_off) {
+// One cluster of 4 CTAs per token row.  If a residual GEMM left partial tiles behind, they are summed
+// into the residual stream first (fixed order: ascending CTA index of the GEMM); the sum of squares
+// is combined across the cluster through distributed shared memory.
+__global__ void __cluster_dims__(kNormCluster, 1, 1) __launch_bounds__(kNormThreads)
+rmsnorm_kernel(Rows rw, int v0, int nv, float *__restrict__ h, Partials pend, const bf16 *__restrict__ g, float eps,
+               int d, bf16 *__restrict__ x, size_t x_lo_off, int pdl) {
   __shared__ float red[32];
-  const int s = blockIdx.x / nv, v = v0 + blockIdx.x % nv;
+  __shared__ float cl_ss;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int q = (int)cluster.block_rank();
+  if (pdl) { griddep_launch(); griddep_wait(); }
+  const int rowi = blockIdx.x / kNormCluster;
+  const int s = rowi / nv, v = v0 + rowi % nv;
   const int r = s * rw.Ms + v;
   float4 *hr = reinterpret_cast<float4 *>(h + (size_t)r * d);
-  const int nvec = d >> 2;
+  const int nvec = d >> 2, per = (nvec + kNormCluster - 1) / kNormCluster;
+  const int f0 = q * per, f1 = min(nvec, f0 + per);
+  const size_t plane_elems = (size_t)pend.ws_rows * 128;
   float4 val[kNormMaxVec];
   float ss = 0.f;
 #pragma unroll
   for (int it = 0; it < kNormMaxVec; ++it) {
-    const int i = threadIdx.x + it * kNormThreads;
-    if (i < nvec) {
-      float4 a = hr[i];
-      for (int p = 0; p < n_partial; ++p) {
-        const float4 b = reinterpret_cast<const float4 *>(partial + (size_t)p * partial_stride + (size_t)r * d)[i];
-        a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+    const int idx = f0 + threadIdx.x + it * kNormThreads;
+    if (idx < f1) {
+      float4 a = __ldcg(hr + idx);
+      if (pend.sk.U > 0) {
+        const int n = idx * 4, st = n >> 8, t = (n >> 7) & 1, i = n & 127;
+        const int c_first = sk_owner(pend.sk, (long long)st * pend.sk.KB);
+        const int c_last = sk_owner(pend.sk, (long long)(st + 1) * pend.sk.KB - 1);
+        for (int c0 = c_first; c0 <= c_last; c0 += 8) {     // 8 contributors' loads in flight together
+          float4 p[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const int c = c0 + k;
+            p[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c <= c_last) {
+              const int ord = st - (int)(sk_begin(pend.sk, c) / pend.sk.KB);
+              const float *src = pend.ws + ((size_t)(c * kGemmSlots + ord) * 2 + t) * plane_elems + (size_t)r * 128 + i;
+              p[k] = __ldcg(reinterpret_cast<const float4 *>(src));
+            }
+          }
+#pragma unroll
+          for (int k = 0; k < 8; ++k) { a.x += p[k].x; a.y += p[k].y; a.z += p[k].z; a.w += p[k].w; }
+        }
+        hr[idx] = a;
       }
-      if (n_partial > 0) hr[i] = a;
       val[it] = a;
       ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
     }
   }
   ss = block_sum(ss, red);
-  const float rs = rsqrtf(ss / (float)d + eps);
+  if (threadIdx.x == 0) cl_ss = ss;
+  cluster.sync();
+  float total = 0.f;
+#pragma unroll
+  for (int k = 0; k < kNormCluster; ++k) total += *cluster.map_shared_rank(&cl_ss, k);
+  cluster.sync();                     // peers have read cl_ss before anyone may exit
+  const float rs = rsqrtf(total / (float)d + eps);
 #pragma unroll
   for (int it = 0; it < kNormMaxVec; ++it) {
-    const int i = threadIdx.x + it * kNormThreads;
-    if (i < nvec) {
+    const int i = f0 + threadIdx.x + it * kNormThreads;
+    if (i < f1) {
       const __nv_bfloat162 g01 = reinterpret_cast<const __nv_bfloat162 *>(g)[2 * i];
       const __nv_bfloat162 g23 = reinterpret_cast<const __nv_bfloat162 *>(g)[2 * i + 1];
       const float2 ga = __bfloat1622float2(g01), gb = __bfloat1622float2(g23);
@@ -161,13 +198,12 @@ add_rmsnorm_kernel(Rows rw, int v0, int nv, float *__restrict__ h, const float *
   }
 }
 
-void launch_add_rmsnorm(const Rows &rw, int v0, int v1, float *h, const float *partial, int n_partial,
-                        size_t partial_stride, const bf16 *g, float eps, int d, bf16 *x, size_t x_lo_off,
-                        cudaStream_t st) {
+cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Partials &pending, const bf16 *g, float eps,
+                           int d, bf16 *x, size_t x_lo_off, bool pdl, cudaStream_t st) {
   const int nv = v1 - v0;
-  if (nv <= 0) return;
-  add_rmsnorm_kernel<<<rw.n_seq * nv, kNormThreads, 0, st>>>(rw, v0, nv, h, partial, n_partial, partial_stride, g, eps,
-                                                             d, x, x_lo_off);
+  if (nv <= 0) return cudaSuccess;
+  return launch_k(rmsnorm_kernel, dim3(rw.n_seq * nv * kNormCluster), dim3(kNormThreads), 0, st, pdl, rw, v0, nv, h,
+                  pending, g, eps, d, x, x_lo_off, pdl ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------
