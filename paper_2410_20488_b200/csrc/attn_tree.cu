@@ -3,14 +3,22 @@
 // Every new row attends to the whole committed prefix [0, n) and, among the new rows of its
 // own sequence (cache slots n .. n+rows-1), only to its ancestors and itself; the visibility
 // bits come from the parent array (built once per step).  Grid = (kv split, kv head,
-// sequence x query block).  A CTA stages 64-position K and V tiles of its split in shared
-// memory (cp.async, double buffered), each warp owns 16 query rows (row x head-of-group for
-// grouped-query attention), S = Q K^T and O += P V run on the tensor cores with an online
-// softmax in fp32, and each split leaves an unnormalised partial (running max, sum, O) that
-// a small combine kernel merges.  Queries and probabilities enter the tensor cores as bf16
-// (hi, lo) pairs accumulated into the same fp32 accumulators, so the only bf16 rounding on this
-// path is the cache's own storage format.
+// sequence x query block); the CTAs of one (kv head, query block) form a thread-block cluster.
+// A CTA stages 64-position K and V tiles of its split in shared memory (cp.async, double
+// buffered), each warp owns 16 query rows (row x head-of-group for grouped-query attention),
+// S = Q K^T and O += P V run on the tensor cores with an online softmax in fp32.  Each split
+// leaves its unnormalised (running max, sum, O) in its own shared memory; after a cluster
+// barrier every CTA merges a share of the query rows by reading its peers' partials through
+// distributed shared memory and writes the final rows, so there is no second kernel and the
+// merge order is fixed.  Queries and probabilities enter the tensor cores as bf16 (hi, lo)
+// pairs accumulated into the same fp32 accumulators, so the only bf16 rounding on this path is
+// the cache's own storage format.
+#include <cooperative_groups.h>
+
 #include "firp_kernels.cuh"
+#include "launch_util.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace firp {
 
@@ -49,7 +57,7 @@ template <int DH> __device__ __forceinline__ int tile_off(int r, int c) {
 }
 
 template <int DH>
-__global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a) {
+__global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a, int pdl) {
   constexpr int CH = DH / 8;          // 16-byte chunks per row
   constexpr int TILE_BYTES = KT * DH * 2;
   extern __shared__ __align__(128) uint8_t smem[];
@@ -59,6 +67,9 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a) {
   uint8_t *sV = sK + 2 * TILE_BYTES;                // [2][KT][DH]
   __shared__ uint32_t s_mask[kQRows][kMaskWords];
   __shared__ int s_row[kQRows];                     // global row index of each query row, -1 = padding
+  __shared__ float s_m[kQRows], s_l[kQRows];        // this split's running max (log2 units) and sum per query row
+  __shared__ float p_m[kAttnMaxSplits][kQRows], p_l[kAttnMaxSplits][kQRows];   // every split's, gathered for the merge
+  if (pdl) { griddep_launch(); griddep_wait(); }
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int split = blockIdx.x, kvh = blockIdx.y;
@@ -70,8 +81,7 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a) {
   const int n = a.ctx_len[slot];
   const int kv_len = min(n + a.rows_active, a.max_ctx);
   const int tiles_total = (kv_len + KT - 1) / KT;
-  const int tiles_per = (tiles_total + a.splits - 1) / a.splits;
-  const int t0 = split * tiles_per, t1 = min(tiles_total, t0 + tiles_per);
+  const int t0 = split * tiles_total / a.splits, t1 = (split + 1) * tiles_total / a.splits;   // balanced ranges
 
   const bf16 *kbase = a.kcache + (size_t)slot * a.seq_stride + (size_t)kvh * DH;
   const bf16 *vbase = kbase + a.kv_stride;
@@ -210,72 +220,110 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a) {
   }
   cp_async_wait<0>();
 
-  // partial result of this split
+  // this split's partial result -> own shared memory (the K buffers are free now)
+  float *sO = reinterpret_cast<float *>(sK);        // [kQRows][DH]
+  static_assert(2 * TILE_BYTES >= kQRows * DH * 4, "partial O must fit the K buffers");
+  __syncthreads();
 #pragma unroll
   for (int rr = 0; rr < 2; ++rr) {
     float l = l_run[rr];
     l += __shfl_xor_sync(0xffffffffu, l, 1);
     l += __shfl_xor_sync(0xffffffffu, l, 2);
     const int i = warp * 16 + g + rr * 8;
-    const int qr = qb * kQRows + i;
-    if (qr >= qrows_total) continue;
-    const int r = s * a.rw.Ms + qr / G, head = kvh * G + qr % G;
-    const size_t base = ((size_t)split * a.rw.R + r) * a.H + head;
-    if (t4 == 0) { a.part_ml[base * 2] = m_run[rr]; a.part_ml[base * 2 + 1] = l; }
-    float *po = a.part_o + base * DH;
+    if (t4 == 0) { s_m[i] = m_run[rr]; s_l[i] = l; }
 #pragma unroll
     for (int nt = 0; nt < DH / 8; ++nt)
-      *reinterpret_cast<float2 *>(po + nt * 8 + t4 * 2) = make_float2(o_acc[nt][rr * 2], o_acc[nt][rr * 2 + 1]);
+      *reinterpret_cast<float2 *>(sO + i * DH + nt * 8 + t4 * 2) = make_float2(o_acc[nt][rr * 2], o_acc[nt][rr * 2 + 1]);
   }
-}
-
-// Merge the splits: o = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s
-__global__ void attn_combine_kernel(AttnArgs a) {
-  const int r = blockIdx.x / a.H, head = blockIdx.x % a.H;
-  const int v = r % a.rw.Ms;
-  if (v >= a.rows_active) return;
-  float M = -INFINITY;
-  for (int sp = 0; sp < a.splits; ++sp) M = fmaxf(M, a.part_ml[(((size_t)sp * a.rw.R + r) * a.H + head) * 2]);
-  float L = 0.f;
-  for (int sp = 0; sp < a.splits; ++sp) {
-    const size_t b = (((size_t)sp * a.rw.R + r) * a.H + head) * 2;
-    const float m = a.part_ml[b];
-    if (m != -INFINITY) L += exp2f(m - M) * a.part_ml[b + 1];
+  // merge: o = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s; CTA `rank` finalises rows rank, rank + splits, ...
+  cg::cluster_group cluster = cg::this_cluster();
+  cluster.sync();
+  const int rank = (int)cluster.block_rank(), nsp = (int)cluster.num_blocks();
+#pragma unroll 4
+  for (int idx = tid; idx < nsp * kQRows; idx += kThreads) {     // all peers' (max, sum): independent remote loads
+    const int sp = idx / kQRows, i = idx % kQRows;
+    p_m[sp][i] = *cluster.map_shared_rank(&s_m[i], sp);
+    p_l[sp][i] = *cluster.map_shared_rank(&s_l[i], sp);
   }
-  const float inv = (L > 0.f) ? 1.f / L : 0.f;
-  for (int c = threadIdx.x; c < a.dh; c += blockDim.x) {
-    float acc = 0.f;
-    for (int sp = 0; sp < a.splits; ++sp) {
-      const size_t b = ((size_t)sp * a.rw.R + r) * a.H + head;
-      const float m = a.part_ml[b * 2];
-      if (m != -INFINITY) acc += exp2f(m - M) * a.part_o[b * a.dh + c];
+  __syncthreads();
+  constexpr int RPP = kThreads / DH;                // rows finalised per pass (1 for dh = 128, 2 for dh = 64)
+  const int c = tid % DH, sub = tid / DH;
+  for (int i0 = rank * RPP; i0 < kQRows; i0 += 2 * nsp * RPP) {   // two passes at a time: 16 remote loads in flight
+    float ov[2][kAttnMaxSplits];
+    int row[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int i = i0 + u * nsp * RPP + sub;
+      row[u] = (i < kQRows && qb * kQRows + i < qrows_total) ? i : -1;
+#pragma unroll
+      for (int sp = 0; sp < kAttnMaxSplits; ++sp)
+        ov[u][sp] = (row[u] >= 0 && sp < nsp) ? *cluster.map_shared_rank(sO + row[u] * DH + c, sp) : 0.f;
     }
-    const float val = acc * inv;
-    const bf16 hi = __float2bfloat16_rn(val);
-    const size_t idx = ((size_t)r * a.H + head) * a.dh + c;
-    a.o[idx] = hi;
-    a.o[a.o_lo_off + idx] = __float2bfloat16_rn(val - __bfloat162float(hi));
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int i = row[u];
+      if (i < 0) continue;
+      float M = -INFINITY;
+#pragma unroll
+      for (int sp = 0; sp < kAttnMaxSplits; ++sp) if (sp < nsp) M = fmaxf(M, p_m[sp][i]);
+      float L = 0.f, acc = 0.f;
+#pragma unroll
+      for (int sp = 0; sp < kAttnMaxSplits; ++sp) {
+        if (sp < nsp && p_m[sp][i] != -INFINITY) {
+          const float w = exp2f(p_m[sp][i] - M);
+          L += w * p_l[sp][i];
+          acc += w * ov[u][sp];
+        }
+      }
+      const float val = (L > 0.f) ? acc / L : 0.f;
+      const int qr = qb * kQRows + i;
+      const int r = s * a.rw.Ms + qr / G, head = kvh * G + qr % G;
+      const bf16 hi = __float2bfloat16_rn(val);
+      const size_t idx = ((size_t)r * a.H + head) * DH + c;
+      a.o[idx] = hi;
+      a.o[a.o_lo_off + idx] = __float2bfloat16_rn(val - __bfloat162float(hi));
+    }
   }
+  cluster.sync();                                   // peers may still be reading this CTA's partials
 }
 
-template <int DH> void launch_dh(const AttnArgs &a, cudaStream_t st) {
+template <int DH> cudaError_t launch_dh(const AttnArgs &a, bool pdl, cudaStream_t st) {
   constexpr int SMEM = 2 * kQRows * DH * 2 + 4 * KT * DH * 2;
   static bool configured = false;
   if (!configured) {
-    cudaFuncSetAttribute(tree_attn_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+    cudaError_t e = cudaFuncSetAttribute(tree_attn_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+    if (e != cudaSuccess) return e;
     configured = true;
   }
   const int G = a.H / a.Hkv;
   const int qblocks = (a.rows_active * G + kQRows - 1) / kQRows;
-  tree_attn_kernel<DH><<<dim3(a.splits, a.Hkv, a.rw.n_seq * qblocks), kThreads, SMEM, st>>>(a);
-  attn_combine_kernel<<<a.rw.R * a.H, DH, 0, st>>>(a);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(a.splits, a.Hkv, a.rw.n_seq * qblocks);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = SMEM;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = a.splits; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, tree_attn_kernel<DH>, a, pdl ? 1 : 0);
 }
 
 }  // namespace
 
-void launch_attention(const AttnArgs &a, cudaStream_t st) {
-  if (a.dh == 128) launch_dh<128>(a, st);
-  else launch_dh<64>(a, st);
+int attention_splits(int groups, int kv_tiles) {
+  // CTAs of one (kv head, query block) = one cluster (<= 8): about two CTAs per SM over the whole grid,
+  // never more splits than 64-position tiles
+  int s = 1;
+  while (s < kAttnMaxSplits && 2 * s * groups <= 2 * 148 && 2 * s <= kv_tiles) s *= 2;
+  return s;
+}
+
+cudaError_t launch_attention(const AttnArgs &a, bool pdl, cudaStream_t st) {
+  return a.dh == 128 ? launch_dh<128>(a, pdl, st) : launch_dh<64>(a, pdl, st);
 }
 
 }  // namespace firp

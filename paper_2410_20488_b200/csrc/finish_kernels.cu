@@ -85,7 +85,7 @@ __global__ void __launch_bounds__(kThreads) qkv_finish_kernel(Partials p, GemmAr
   float x1[4] = {v0.x, v0.y, v0.z, v0.w}, x2[4] = {v1.x, v1.y, v1.z, v1.w};
   if (unit < a.H + a.Hkv) {     // queries and keys are rotated at the row's tree position
     const float4 *cs = reinterpret_cast<const float4 *>(a.rope + (size_t)it.m * half + c);
-    const float4 cs01 = __ldg(cs), cs23 = __ldg(cs + 1);
+    const float4 cs01 = __ldcg(cs), cs23 = __ldcg(cs + 1);
     const float co[4] = {cs01.x, cs01.z, cs23.x, cs23.z}, si[4] = {cs01.y, cs01.w, cs23.y, cs23.w};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {

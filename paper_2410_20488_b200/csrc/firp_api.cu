@@ -56,7 +56,7 @@ struct firp_ctx {
   std::vector<const void *> wqkv, wo, wgu, wd, g_attn, g_mlp;
   // device buffers (carved from the caller's workspace)
   bf16 *kv = nullptr;
-  float *h = nullptr, *gemm_ws = nullptr, *part_o = nullptr, *part_ml = nullptr, *logits = nullptr, *top_vals = nullptr;
+  float *h = nullptr, *gemm_ws = nullptr, *logits = nullptr, *top_vals = nullptr;
   bf16 *x = nullptr, *q = nullptr, *o = nullptr, *y = nullptr;
   int32_t *ctx_len = nullptr, *seq_ids = nullptr, *parents = nullptr, *next_parents = nullptr, *chain = nullptr;
   int32_t *top_ids = nullptr, *path = nullptr, *n_acc = nullptr, *accepted = nullptr, *next_tokens = nullptr;
@@ -82,8 +82,6 @@ struct firp_ctx {
     o = c.take<bf16>(2 * R * nq);
     y = c.take<bf16>(2 * R * cfg.d_ffn);
     gemm_ws = c.take<float>((size_t)kGemmMaxCtas * kGemmSlots * 2 * R * 128);
-    part_o = c.take<float>((size_t)kAttnMaxSplits * R * nq);
-    part_ml = c.take<float>((size_t)kAttnMaxSplits * R * cfg.n_heads * 2);
     logits = c.take<float>(R * cfg.vocab);
     top_ids = c.take<int32_t>(R * kMaxTopB);
     top_vals = c.take<float>(R * kMaxTopB);
@@ -197,14 +195,14 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   const size_t Rp = (size_t)c->Rmax;          // rows per activation plane
   const firp_step_out *out = ra.out;
   int &nl = c->launches;
-  const bool tc = c->use_tc, pdl = c->use_tc && c->use_pdl;
+  const bool tc = c->use_tc, pdl = c->use_pdl;
 
   const int mw_out = (rw.Ms + 31) / 32;
   { FIRP_TIMED(KC_TREE_PREP);
     launch_tree_prep(rw, c->parents, c->seq_ids, c->ctx_len, dh, cfg.rope_theta, c->meta, out ? out->depth : nullptr,
-                     out ? out->mask : nullptr, mw_out, st); ++nl; }
+                     out ? out->mask : nullptr, mw_out, pdl, st); ++nl; }
   { FIRP_TIMED(KC_EMBED);
-    launch_embed(rw, ra.d_tokens, (const bf16 *)c->w.embed, d, cfg.vocab, c->h, st); ++nl; }
+    launch_embed(rw, ra.d_tokens, (const bf16 *)c->w.embed, d, cfg.vocab, c->h, pdl, st); ++nl; }
 
   auto gemm_base = [&](const bf16 *X, size_t lo_off, const void *W, int N, int K, int act) {
     GemmArgs g{};
@@ -227,7 +225,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     pending.sk.U = 0;
     if (insert) {   // Eq. 3 on the raw (now complete) residual row of the root, then the norm of the new rows
       { FIRP_TIMED(KC_PSEUDO_PROJ);
-        launch_pseudo_proj(rw, (const bf16 *)c->w.pred_w, (const bf16 *)c->w.pred_b, d, c->h, st); ++nl; }
+        launch_pseudo_proj(rw, (const bf16 *)c->w.pred_w, (const bf16 *)c->w.pred_b, d, c->h, pdl, st); ++nl; }
       FIRP_TIMED(KC_RMSNORM);
       FIRP_CUDA(c, launch_rmsnorm(rw, rw.T, rw.Ms, c->h, none, (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x, Rp * d, pdl, st)); ++nl;
     }
@@ -249,13 +247,10 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       a.seq_ids = c->seq_ids; a.ctx_len = c->ctx_len; a.mask = c->meta.mask;
       const int tiles = (ra.n_hi_max + act + kAttnTile - 1) / kAttnTile;
       const int G = H / Hkv, qblocks = (act * G + 63) / 64;
-      int splits = (2 * 148) / (rw.n_seq * Hkv * qblocks);
-      splits = splits < 1 ? 1 : splits;
-      splits = splits > tiles ? tiles : splits;
-      a.splits = splits > kAttnMaxSplits ? kAttnMaxSplits : splits;
-      a.part_o = c->part_o; a.part_ml = c->part_ml; a.o = c->o; a.o_lo_off = Rp * nq;
+      a.splits = attention_splits(rw.n_seq * Hkv * qblocks, tiles);
+      a.o = c->o; a.o_lo_off = Rp * nq;
       FIRP_TIMED(KC_ATTENTION);
-      launch_attention(a, st); nl += 2;
+      FIRP_CUDA(c, launch_attention(a, pdl, st)); ++nl;
     }
     {
       GemmArgs g = gemm_base(c->o, Rp * nq, c->wo[j], d, nq, act);
@@ -291,7 +286,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       FIRP_CUDA(c, launch_gemm(EPI_LOGITS, g, tc, pdl, st, &p.sk)); ++nl;
       if (p.sk.U > 0) { FIRP_CUDA(c, launch_gemm_finish(EPI_LOGITS, p, g, pdl, st)); ++nl; } }
     { FIRP_TIMED(KC_TOPB);
-      launch_topb(ra.logits_dst, rw.R, cfg.vocab, cfg.top_b, c->top_ids, c->top_vals, st); ++nl; }
+      launch_topb(ra.logits_dst, rw.R, cfg.vocab, cfg.top_b, c->top_ids, c->top_vals, pdl, st); ++nl; }
     AcceptArgs a{};
     a.tokens = ra.d_tokens; a.parents = c->parents; a.next_parents = c->next_parents;
     a.top_ids = c->top_ids; a.top_vals = c->top_vals; a.T_next = ra.T_next; a.B = cfg.top_b; a.S = c->S;
@@ -303,7 +298,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       a.o_topb_ids = out->topb_ids; a.o_topb_vals = out->topb_vals;
     }
     FIRP_TIMED(KC_ACCEPT);
-    launch_accept(rw, a, st); ++nl;
+    launch_accept(rw, a, pdl, st); ++nl;
   }
   FIRP_CUDA(c, cudaGetLastError());
   return FIRP_OK;
@@ -505,7 +500,7 @@ int firp_prefill(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int32_t P,
     if (last && out && out->logits)
       FIRP_CUDA(ctx, cudaMemcpyAsync(out->logits, ctx->logits + (size_t)(Tc - 1) * cfg.vocab,
                                      sizeof(float) * (size_t)(1 + k) * cfg.vocab, cudaMemcpyDeviceToDevice, st));
-    launch_advance_ctx(1, ctx->seq_ids, ctx->ctx_len, Tc, st); ++ctx->launches;
+    launch_advance_ctx(1, ctx->seq_ids, ctx->ctx_len, Tc, ctx->use_pdl, st); ++ctx->launches;
     ctx->n_hi[seq] += Tc;
   }
   FIRP_CUDA(ctx, cudaGetLastError());
@@ -547,7 +542,7 @@ int firp_kv_commit(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const i
     for (int s = 0; s < n_seq; ++s) ctx->n_hi[ids[s]] += S;   // exact value is on the device; keep an upper bound
   }
   { firp_ctx *c = ctx; FIRP_TIMED(KC_COMMIT);
-    launch_commit(n_seq, a, st); ctx->launches += 2; }
+    launch_commit(n_seq, a, ctx->use_pdl, st); ctx->launches += 2; }
   FIRP_CUDA(ctx, cudaGetLastError());
   ctx->stepped = false;
   return FIRP_OK;

@@ -54,10 +54,11 @@ struct TreeMeta {
 };
 void launch_tree_prep(const Rows &rw, const int32_t *d_parents, const int32_t *d_seq_ids, const int32_t *d_ctx_len,
                       int dh, float theta, TreeMeta meta, int32_t *out_depth, uint32_t *out_mask, int out_mask_words,
-                      cudaStream_t st);
+                      bool pdl, cudaStream_t st);
 
 // h[r] = embed[token] for tree rows, 0 for pseudo rows
-void launch_embed(const Rows &rw, const int32_t *d_tokens, const bf16 *embed, int d, int vocab, float *h, cudaStream_t st);
+void launch_embed(const Rows &rw, const int32_t *d_tokens, const bf16 *embed, int d, int vocab, float *h, bool pdl,
+                  cudaStream_t st);
 
 // Activations that feed a GEMM or the attention are stored as two bf16 planes (hi, lo) with
 // hi + lo = the fp32 value to ~16 mantissa bits; the lo plane starts *_lo_off elements after hi.
@@ -75,10 +76,10 @@ cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Parti
                            int d, bf16 *x, size_t x_lo_off, bool pdl, cudaStream_t st);
 
 // Eq. 3: h[s*Ms + T + i] = W_i h[s*Ms + anchor] + b_i
-void launch_pseudo_proj(const Rows &rw, const bf16 *pred_w, const bf16 *pred_b, int d, float *h, cudaStream_t st);
+void launch_pseudo_proj(const Rows &rw, const bf16 *pred_w, const bf16 *pred_b, int d, float *h, bool pdl, cudaStream_t st);
 
 // top-B of every row of logits by (value desc, id asc)
-void launch_topb(const float *logits, int R, int V, int B, int32_t *ids, float *vals, cudaStream_t st);
+void launch_topb(const float *logits, int R, int V, int B, int32_t *ids, float *vals, bool pdl, cudaStream_t st);
 
 struct AcceptArgs {
   const int32_t *tokens;        // [n_seq][T]
@@ -94,7 +95,7 @@ struct AcceptArgs {
   int32_t *o_path, *o_n_accepted, *o_accepted, *o_next_tokens, *o_best, *o_topb_ids;
   float *o_topb_vals;
 };
-void launch_accept(const Rows &rw, const AcceptArgs &a, cudaStream_t st);
+void launch_accept(const Rows &rw, const AcceptArgs &a, bool pdl, cudaStream_t st);
 
 // KV compaction: rows path[j] -> slot n + j in every layer; then ctx_len += len
 struct CommitArgs {
@@ -109,8 +110,8 @@ struct CommitArgs {
   int S;
   int32_t *ctx_len;         // [max_batch] device
 };
-void launch_commit(int n_seq, const CommitArgs &a, cudaStream_t st);
-void launch_advance_ctx(int n_seq, const int32_t *seq_ids, int32_t *ctx_len, int amount, cudaStream_t st);
+void launch_commit(int n_seq, const CommitArgs &a, bool pdl, cudaStream_t st);
+void launch_advance_ctx(int n_seq, const int32_t *seq_ids, int32_t *ctx_len, int amount, bool pdl, cudaStream_t st);
 
 // ---- skinny weight-streaming GEMM ------------------------------------------
 enum GemmEpilogue { EPI_RESIDUAL = 0, EPI_QKV_ROPE = 1, EPI_SWIGLU = 2, EPI_LOGITS = 3 };
@@ -150,6 +151,7 @@ cudaError_t launch_gemm_tc(GemmEpilogue epi, const GemmArgs &a, bool pdl, cudaSt
 bool gemm_tc_available();         // the driver entry point for tensor-map encoding was found
 
 // ---- tree-masked split-KV attention ---------------------------------------
+constexpr int kAttnMaxSplits = 8;   // kv splits = CTAs per cluster (portable cluster size limit)
 struct AttnArgs {
   Rows rw; int rows_active;
   int H, Hkv, dh;
@@ -158,12 +160,11 @@ struct AttnArgs {
   size_t seq_stride, kv_stride; int max_ctx;
   const int32_t *seq_ids, *ctx_len;
   const uint32_t *mask;       // [R][kMaskWords]
-  int splits;                 // kv splits (grid.x)
-  float *part_o;              // [splits][R][H][dh]
-  float *part_ml;             // [splits][R][H][2] (running max in log2 units, sum)
+  int splits;                 // kv splits (grid.x = cluster size): 1, 2, 4 or 8
   bf16 *o; size_t o_lo_off;   // [R][H*dh] hi plane, lo plane
 };
-void launch_attention(const AttnArgs &a, cudaStream_t st);
-constexpr int kAttnMaxSplits = 32;
+// kv splits for `groups` = sequences x kv heads x query blocks and `kv_tiles` 64-position tiles
+int attention_splits(int groups, int kv_tiles);
+cudaError_t launch_attention(const AttnArgs &a, bool pdl, cudaStream_t st);
 
 }  // namespace firp

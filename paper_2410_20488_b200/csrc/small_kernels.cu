@@ -14,11 +14,12 @@ namespace firp {
 // depth, absolute position, ancestor-or-self bitmask, rotary table.
 // One CTA per sequence; the extended parent array lives in shared memory.
 // ---------------------------------------------------------------------------
-__global__ void tree_prep_kernel(Rows rw, const int32_t *__restrict__ parents, const int32_t *__restrict__ seq_ids,
-                                 const int32_t *__restrict__ ctx_len, int dh, float theta, TreeMeta meta,
-                                 int32_t *out_depth, uint32_t *out_mask, int out_mask_words) {
+__global__ void tree_prep_kernel(Rows rw, const int32_t *parents, const int32_t *seq_ids,
+                                 const int32_t *ctx_len, int dh, float theta, TreeMeta meta,
+                                 int32_t *out_depth, uint32_t *out_mask, int out_mask_words, int pdl) {
   __shared__ int32_t ext[kMaxTreeRows];
   __shared__ int32_t sdepth[kMaxTreeRows];
+  if (pdl) { griddep_launch(); griddep_wait(); }
   const int s = blockIdx.x, tid = threadIdx.x;
   const int n = ctx_len[seq_ids[s]];
   for (int v = tid; v < rw.Ms; v += blockDim.x) {
@@ -65,16 +66,17 @@ __global__ void tree_prep_kernel(Rows rw, const int32_t *__restrict__ parents, c
 
 void launch_tree_prep(const Rows &rw, const int32_t *d_parents, const int32_t *d_seq_ids, const int32_t *d_ctx_len,
                       int dh, float theta, TreeMeta meta, int32_t *out_depth, uint32_t *out_mask, int out_mask_words,
-                      cudaStream_t st) {
-  tree_prep_kernel<<<rw.n_seq, 256, 0, st>>>(rw, d_parents, d_seq_ids, d_ctx_len, dh, theta, meta, out_depth, out_mask,
-                                             out_mask_words);
+                      bool pdl, cudaStream_t st) {
+  launch_k(tree_prep_kernel, dim3(rw.n_seq), dim3(256), 0, st, pdl, rw, d_parents, d_seq_ids, d_ctx_len, dh, theta, meta,
+           out_depth, out_mask, out_mask_words, pdl ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------
 // Embedding gather: fp32 residual rows from bf16 table rows; pseudo rows start at zero.
 // ---------------------------------------------------------------------------
-__global__ void embed_kernel(Rows rw, const int32_t *__restrict__ tokens, const bf16 *__restrict__ embed, int d,
-                             int vocab, float *__restrict__ h) {
+__global__ void embed_kernel(Rows rw, const int32_t *tokens, const bf16 *__restrict__ embed, int d,
+                             int vocab, float *h, int pdl) {
+  if (pdl) { griddep_launch(); griddep_wait(); }
   const int r = blockIdx.x, s = r / rw.Ms, v = r % rw.Ms;
   float *dst = h + (size_t)r * d;
   if (v >= rw.T) {
@@ -90,9 +92,9 @@ __global__ void embed_kernel(Rows rw, const int32_t *__restrict__ tokens, const 
   }
 }
 
-void launch_embed(const Rows &rw, const int32_t *d_tokens, const bf16 *embed, int d, int vocab, float *h,
+void launch_embed(const Rows &rw, const int32_t *d_tokens, const bf16 *embed, int d, int vocab, float *h, bool pdl,
                   cudaStream_t st) {
-  embed_kernel<<<rw.R, 128, 0, st>>>(rw, d_tokens, embed, d, vocab, h);
+  launch_k(embed_kernel, dim3(rw.R), dim3(128), 0, st, pdl, rw, d_tokens, embed, d, vocab, h, pdl ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------
@@ -124,8 +126,8 @@ constexpr int kNormMaxVec = 2;    // float4 per thread: d <= 4 * 256 * 2 * 4 = 8
 // into the residual stream first (fixed order: ascending CTA index of the GEMM); the sum of squares
 // is combined across the cluster through distributed shared memory.
 __global__ void __cluster_dims__(kNormCluster, 1, 1) __launch_bounds__(kNormThreads)
-rmsnorm_kernel(Rows rw, int v0, int nv, float *__restrict__ h, Partials pend, const bf16 *__restrict__ g, float eps,
-               int d, bf16 *__restrict__ x, size_t x_lo_off, int pdl) {
+rmsnorm_kernel(Rows rw, int v0, int nv, float *h, Partials pend, const bf16 *__restrict__ g, float eps,
+               int d, bf16 *x, size_t x_lo_off, int pdl) {
   __shared__ float red[32];
   __shared__ float cl_ss;
   cg::cluster_group cluster = cg::this_cluster();
@@ -212,7 +214,8 @@ cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Parti
 // one warp per output coordinate, 16-byte weight loads, fp32 accumulation.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-pseudo_proj_kernel(Rows rw, const bf16 *__restrict__ W, const bf16 *__restrict__ b, int d, float *__restrict__ h) {
+pseudo_proj_kernel(Rows rw, const bf16 *__restrict__ W, const bf16 *__restrict__ b, int d, float *h, int pdl) {
+  if (pdl) { griddep_launch(); griddep_wait(); }
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= rw.k * d) return;
   const int i = warp / d, o = warp % d;
@@ -248,9 +251,9 @@ pseudo_proj_kernel(Rows rw, const bf16 *__restrict__ W, const bf16 *__restrict__
   }
 }
 
-void launch_pseudo_proj(const Rows &rw, const bf16 *pred_w, const bf16 *pred_b, int d, float *h, cudaStream_t st) {
+void launch_pseudo_proj(const Rows &rw, const bf16 *pred_w, const bf16 *pred_b, int d, float *h, bool pdl, cudaStream_t st) {
   const int warps = rw.k * d;
-  pseudo_proj_kernel<<<(warps + 7) / 8, 256, 0, st>>>(rw, pred_w, pred_b, d, h);
+  launch_k(pseudo_proj_kernel, dim3((warps + 7) / 8), dim3(256), 0, st, pdl, rw, pred_w, pred_b, d, h, pdl ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------
@@ -261,10 +264,11 @@ constexpr int kTopThreads = 256;
 __device__ __forceinline__ bool better(float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia < ib); }
 
 __global__ void __launch_bounds__(kTopThreads)
-topb_kernel(const float *__restrict__ logits, int V, int B, int32_t *__restrict__ ids, float *__restrict__ vals) {
+topb_kernel(const float *logits, int V, int B, int32_t *ids, float *vals, int pdl) {
   __shared__ float sval[32];
   __shared__ int sid[32];
   __shared__ int swin;
+  if (pdl) { griddep_launch(); griddep_wait(); }
   const float *row = logits + (size_t)blockIdx.x * V;
   float lv[kMaxTopB];
   int li[kMaxTopB];
@@ -318,16 +322,17 @@ topb_kernel(const float *__restrict__ logits, int V, int B, int32_t *__restrict_
   }
 }
 
-void launch_topb(const float *logits, int R, int V, int B, int32_t *ids, float *vals, cudaStream_t st) {
-  topb_kernel<<<R, kTopThreads, 0, st>>>(logits, V, B, ids, vals);
+void launch_topb(const float *logits, int R, int V, int B, int32_t *ids, float *vals, bool pdl, cudaStream_t st) {
+  launch_k(topb_kernel, dim3(R), dim3(kTopThreads), 0, st, pdl, logits, V, B, ids, vals, pdl ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------
 // Greedy acceptance walk and next tree (Section 3.4).  One CTA per sequence.
 // ---------------------------------------------------------------------------
-__global__ void accept_kernel(Rows rw, AcceptArgs a) {
+__global__ void accept_kernel(Rows rw, AcceptArgs a, int pdl) {
   __shared__ int32_t s_best[kMaxTreeRows];
   __shared__ int32_t s_bonus;
+  if (pdl) { griddep_launch(); griddep_wait(); }
   const int s = blockIdx.x, tid = threadIdx.x;
   const int32_t *tok = a.tokens + (size_t)s * rw.T;
   for (int v = tid; v < rw.T; v += blockDim.x) {
@@ -388,8 +393,8 @@ __global__ void accept_kernel(Rows rw, AcceptArgs a) {
   }
 }
 
-void launch_accept(const Rows &rw, const AcceptArgs &a, cudaStream_t st) {
-  accept_kernel<<<rw.n_seq, 128, 0, st>>>(rw, a);
+void launch_accept(const Rows &rw, const AcceptArgs &a, bool pdl, cudaStream_t st) {
+  launch_k(accept_kernel, dim3(rw.n_seq), dim3(128), 0, st, pdl, rw, a, pdl ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------
@@ -399,7 +404,8 @@ void launch_accept(const Rows &rw, const AcceptArgs &a, cudaStream_t st) {
 // ---------------------------------------------------------------------------
 constexpr int kMaxPath = 16;
 
-__global__ void __launch_bounds__(128) commit_kernel(CommitArgs a) {
+__global__ void __launch_bounds__(128) commit_kernel(CommitArgs a, int pdl) {
+  if (pdl) { griddep_launch(); griddep_wait(); }
   const int s = blockIdx.y, plane = blockIdx.x;     // plane = layer * 2 + (0 K, 1 V)
   const int slot = a.seq_ids[s];
   const int n = a.ctx_len[slot];
@@ -420,18 +426,20 @@ __global__ void __launch_bounds__(128) commit_kernel(CommitArgs a) {
 }
 
 __global__ void advance_ctx_kernel(int n_seq, const int32_t *seq_ids, int32_t *ctx_len, const int32_t *path_len,
-                                   int amount) {
+                                   int amount, int pdl) {
+  if (pdl) { griddep_launch(); griddep_wait(); }
   const int s = threadIdx.x;
   if (s < n_seq) ctx_len[seq_ids[s]] += path_len ? min(path_len[s], kMaxPath) : amount;
 }
 
-void launch_commit(int n_seq, const CommitArgs &a, cudaStream_t st) {
-  commit_kernel<<<dim3(a.n_layers * 2, n_seq), 128, 0, st>>>(a);
-  advance_ctx_kernel<<<1, 32, 0, st>>>(n_seq, a.seq_ids, a.ctx_len, a.path_len, 0);
+void launch_commit(int n_seq, const CommitArgs &a, bool pdl, cudaStream_t st) {
+  launch_k(commit_kernel, dim3(a.n_layers * 2, n_seq), dim3(128), 0, st, pdl, a, pdl ? 1 : 0);
+  launch_k(advance_ctx_kernel, dim3(1), dim3(32), 0, st, pdl, n_seq, a.seq_ids, a.ctx_len, a.path_len, 0, pdl ? 1 : 0);
 }
 
-void launch_advance_ctx(int n_seq, const int32_t *seq_ids, int32_t *ctx_len, int amount, cudaStream_t st) {
-  advance_ctx_kernel<<<1, 32, 0, st>>>(n_seq, seq_ids, ctx_len, nullptr, amount);
+void launch_advance_ctx(int n_seq, const int32_t *seq_ids, int32_t *ctx_len, int amount, bool pdl, cudaStream_t st) {
+  launch_k(advance_ctx_kernel, dim3(1), dim3(32), 0, st, pdl, n_seq, seq_ids, ctx_len, (const int32_t *)nullptr, amount,
+           pdl ? 1 : 0);
 }
 
 }  // namespace firp
