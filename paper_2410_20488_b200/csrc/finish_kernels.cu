@@ -21,37 +21,37 @@ struct Item { int st, m, i4; };
 
 // thread -> (supertile, token row, lane quad); quads vary fastest (coalesced float4 reads)
 __device__ __forceinline__ bool item_of_thread(int n_st, int R, Item &it) {
-  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= (long long)n_st * R * 32) return false;
-  it.i4 = (int)(t & 31) * 4;
-  const long long r = t >> 5;
-  it.m = (int)(r % R);
-  it.st = (int)(r / R);
+  const unsigned t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= (unsigned)(n_st * R * 32)) return false;
+  it.i4 = (int)(t & 31u) * 4;
+  const unsigned r = t >> 5;
+  it.m = (int)(r % (unsigned)R);
+  it.st = (int)(r / (unsigned)R);
   return true;
 }
 
 // sums of tile 0 and tile 1 of supertile st for token row m, lanes i4 .. i4+3
 __device__ __forceinline__ void sum_partials(const Partials &p, int st, int m, int i4, float4 &v0, float4 &v1) {
   const size_t plane = (size_t)p.ws_rows * 128, slot = 2 * plane;
-  const int c_first = sk_owner(p.sk, (long long)st * p.sk.KB), c_last = sk_owner(p.sk, (long long)(st + 1) * p.sk.KB - 1);
+  const SkContrib k = sk_contributors(p.sk, st);
+  const float *base = p.ws + (size_t)m * 128 + i4;
   v0 = v1 = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int c0 = c_first; c0 <= c_last; c0 += 4) {      // 4 contributors' loads in flight together
+  for (int c0 = k.c_first; c0 <= k.c_last; c0 += 4) {      // 4 contributors' loads in flight together
     float4 a[4], b[4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const int c = c0 + k;
-      a[k] = b[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (c <= c_last) {
-        const int ord = st - (int)(sk_begin(p.sk, c) / p.sk.KB);
-        const float *src = p.ws + (size_t)(c * kGemmSlots + ord) * slot + (size_t)m * 128 + i4;
-        a[k] = __ldcg(reinterpret_cast<const float4 *>(src));
-        b[k] = __ldcg(reinterpret_cast<const float4 *>(src + plane));
+    for (int j = 0; j < 4; ++j) {
+      const int c = c0 + j;
+      a[j] = b[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (c <= k.c_last) {
+        const float *src = base + (size_t)(c * kGemmSlots + (c == k.c_first ? k.ord_first : 0)) * slot;
+        a[j] = __ldcg(reinterpret_cast<const float4 *>(src));
+        b[j] = __ldcg(reinterpret_cast<const float4 *>(src + plane));
       }
     }
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      v0.x += a[k].x; v0.y += a[k].y; v0.z += a[k].z; v0.w += a[k].w;
-      v1.x += b[k].x; v1.y += b[k].y; v1.z += b[k].z; v1.w += b[k].w;
+    for (int j = 0; j < 4; ++j) {
+      v0.x += a[j].x; v0.y += a[j].y; v0.z += a[j].z; v0.w += a[j].w;
+      v1.x += b[j].x; v1.y += b[j].y; v1.z += b[j].z; v1.w += b[j].w;
     }
   }
 }
@@ -160,7 +160,7 @@ __global__ void __launch_bounds__(kThreads) logits_finish_kernel(Partials p, Gem
 }  // namespace
 
 cudaError_t launch_gemm_finish(GemmEpilogue epi, const Partials &p, const GemmArgs &a, bool pdl, cudaStream_t st) {
-  const int n_st = (int)(p.sk.U / p.sk.KB);
+  const int n_st = p.sk.U / p.sk.KB;
   const long long threads = (long long)n_st * a.R * 32;
   const dim3 grid((unsigned)((threads + kThreads - 1) / kThreads)), block(kThreads);
   switch (epi) {

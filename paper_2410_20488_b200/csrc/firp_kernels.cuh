@@ -33,16 +33,24 @@ constexpr int kGemmSlots = 3;             // partial tiles (segments) per CTA
 // rows, k block = 64 elements); CTA c owns units [sk_begin(c), sk_begin(c + 1)) and its s-th segment
 // is the part of supertile sk_begin(c) / KB + s inside that range.
 struct StreamK {
-  long long U;  // units
+  int U;        // units (supertiles x k blocks; U * G stays far below 2^31 for every supported shape)
   int KB;       // k blocks per supertile
   int G;        // CTAs (<= U, so no range is empty)
 };
-__host__ __device__ __forceinline__ long long sk_begin(const StreamK &s, int c) { return (s.U * c) / s.G; }
-__host__ __device__ __forceinline__ int sk_owner(const StreamK &s, long long u) {   // CTA whose range holds unit u
-  int c = (int)((u * s.G) / s.U);
-  while (c + 1 < s.G && sk_begin(s, c + 1) <= u) ++c;
-  while (c > 0 && sk_begin(s, c) > u) --c;
-  return c;
+__host__ __device__ __forceinline__ int sk_begin(const StreamK &s, int c) { return (int)(((unsigned)s.U * (unsigned)c) / (unsigned)s.G); }
+// CTA whose range holds unit u: the largest c with floor(U c / G) <= u, i.e. c < (u + 1) G / U
+__host__ __device__ __forceinline__ int sk_owner(const StreamK &s, int u) {
+  return (int)((((unsigned)u + 1u) * (unsigned)s.G + (unsigned)s.U - 1u) / (unsigned)s.U) - 1;
+}
+// The CTAs c_first..c_last that hold a piece of supertile st.  Every one but the first starts its range
+// inside st, so its piece is its segment 0; the first one's piece is segment ord_first.
+struct SkContrib { int c_first, c_last, ord_first; };
+__host__ __device__ __forceinline__ SkContrib sk_contributors(const StreamK &s, int st) {
+  SkContrib k;
+  k.c_first = sk_owner(s, st * s.KB);
+  k.c_last = sk_owner(s, (st + 1) * s.KB - 1);
+  k.ord_first = st - sk_begin(s, k.c_first) / s.KB;
+  return k;
 }
 
 // ---- tree bookkeeping (Section 3.4) ---------------------------------------

@@ -34,6 +34,7 @@
 // its end; TMEM is always released.
 #include <cuda.h>
 
+#include <cstdlib>
 #include <map>
 #include <tuple>
 
@@ -98,6 +99,13 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm,
   asm volatile(
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
       ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap *tm, int x, int y) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tm), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap *tm, int x, int y, int z, int w) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];"
+               ::"l"(tm), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -164,6 +172,7 @@ struct Sched {
   int n_st;        // supertiles
   int pdl;         // launched with programmatic stream serialization
   int ws_rows;     // token rows per scratch tile
+  int l2_ahead;    // units each CTA prefetches into L2 beyond its shared-memory ring
 };
 
 template <int NPAD>
@@ -187,8 +196,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const int cta = blockIdx.x;
   const StreamK sk = sc.sk;
   const int KB = sk.KB;
-  const long long u0 = sk_begin(sk, cta), u1 = sk_begin(sk, cta + 1);
-  const int n_units = (int)(u1 - u0);
+  const int u0 = sk_begin(sk, cta), u1 = sk_begin(sk, cta + 1);
+  const int n_units = u1 - u0;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < SW; ++i) { mbar_init(full_w + 8 * i, 1); mbar_init(empty_w + 8 * i, 1); }
@@ -211,9 +220,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (lane == 0) {             // ---- weight producer: does not wait for the previous kernel
       uint64_t pol;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+      // While the ring is full (typically: the activations are not there yet because the previous kernel is
+      // still running) the stream goes on into L2: units up to l2_ahead beyond the ring are prefetched, so
+      // HBM stays busy during the small kernels between two GEMMs and the ring later refills from L2.
+      int pf = SW;
       for (int it = 0; it < n_units; ++it) {
-        const long long u = u0 + it;
-        const int st = (int)(u / KB), kb = (int)(u - (long long)st * KB);
+        for (const int upto = min(n_units, it + SW + sc.l2_ahead); pf < upto; ++pf) {
+          const int up = u0 + pf;
+          const int pst = up / KB, pkb = up - pst * KB;
+          if (sc.mode == ROWS_ROTARY) {
+            const int hp = BM / sc.half;
+            tma_prefetch_4d(&tmW, pkb * BK, 0, 0, pst * hp);
+            tma_prefetch_4d(&tmW, pkb * BK, 0, 1, pst * hp);
+          } else if (sc.mode == ROWS_GATE_UP) {
+            tma_prefetch_2d(&tmW, pkb * BK, pst * BM);
+            tma_prefetch_2d(&tmW, pkb * BK, sc.F + pst * BM);
+          } else {
+            tma_prefetch_2d(&tmW, pkb * BK, pst * (TM * BM));
+            tma_prefetch_2d(&tmW, pkb * BK, pst * (TM * BM) + BM);
+          }
+        }
+        const int u = u0 + it;
+        const int st = u / KB, kb = u - st * KB;
         const int sl = it % SW;
         mbar_wait(empty_w + 8 * sl, ((it / SW) & 1) ^ 1, a.err, dead);
         mbar_expect_tx(full_w + 8 * sl, W_STAGE);
@@ -251,10 +279,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (lane == 0) {             // ---- MMA issuer
       constexpr uint32_t idesc = instr_desc(MERGE ? 2 * NPAD : NPAD);
       int it = 0, seg = 0;
-      long long u = u0;
+      int u = u0;
       while (u < u1) {
-        const int st = (int)(u / KB), kb0 = (int)(u - (long long)st * KB);
-        const int kb1 = (int)min((long long)KB, kb0 + (u1 - u));
+        const int st = u / KB, kb0 = u - st * KB;
+        const int kb1 = min(KB, kb0 + (u1 - u));
         const int buf = seg % NBUF;
         mbar_wait(acc_empty + 8 * buf, ((seg / NBUF) & 1) ^ 1, a.err, dead);   // epilogue has drained this buffer
         tc_fence_after();
@@ -289,10 +317,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const int i = quarter * 32 + lane;            // row within each 128-row tile = TMEM lane
     const size_t plane_elems = (size_t)sc.ws_rows * BM, slot_elems = TM * plane_elems;
     int seg = 0;
-    long long u = u0;
+    int u = u0;
     while (u < u1) {
-      const int st = (int)(u / KB), kb0 = (int)(u - (long long)st * KB);
-      const int kb1 = (int)min((long long)KB, kb0 + (u1 - u));
+      const int st = u / KB, kb0 = u - st * KB;
+      const int kb1 = min(KB, kb0 + (u1 - u));
       const int buf = seg % NBUF;
       mbar_wait(acc_full + 8 * buf, (seg / NBUF) & 1, a.err, dead);
       tc_fence_after();
@@ -439,6 +467,8 @@ Sched make_sched(GemmEpilogue epi, const GemmArgs &a, bool pdl) {
   Sched sc{};
   sc.pdl = pdl ? 1 : 0;
   sc.ws_rows = a.plane_rows;
+  static const int l2_ahead = [] { const char *e = getenv("FIRP_L2_AHEAD"); return e ? atoi(e) : 48; }();
+  sc.l2_ahead = l2_ahead < 0 ? 0 : l2_ahead;
   sc.mode = ROWS_LINEAR; sc.n_st = (a.N + TM * BM - 1) / (TM * BM);
   if (epi == EPI_SWIGLU) {
     sc.mode = ROWS_GATE_UP; sc.F = a.F; sc.n_st = (a.F + BM - 1) / BM;
@@ -448,8 +478,8 @@ Sched make_sched(GemmEpilogue epi, const GemmArgs &a, bool pdl) {
     sc.n_st = (a.H + 2 * a.Hkv + hp - 1) / hp;
   }
   sc.sk.KB = (a.K + BK - 1) / BK;
-  sc.sk.U = (long long)sc.n_st * sc.sk.KB;
-  sc.sk.G = (int)std::min<long long>(sm_count(), sc.sk.U);
+  sc.sk.U = sc.n_st * sc.sk.KB;
+  sc.sk.G = std::min(sm_count(), sc.sk.U);
   return sc;
 }
 
@@ -461,8 +491,9 @@ cudaError_t launch_gemm_tc(GemmEpilogue epi, const GemmArgs &a, bool pdl, cudaSt
   if (!encode_fn()) return cudaErrorNotSupported;
   const Sched sc = make_sched(epi, a, pdl);
   // a CTA's range of U / G units touches at most this many supertiles, each needing a scratch slot
-  const long long per = (sc.sk.U + sc.sk.G - 1) / sc.sk.G;
-  if (sc.sk.G > kGemmMaxCtas || (per + sc.sk.KB - 2) / sc.sk.KB + 1 > kGemmSlots)
+  const int per = (sc.sk.U + sc.sk.G - 1) / sc.sk.G;
+  if (sc.sk.G > kGemmMaxCtas || (per + sc.sk.KB - 2) / sc.sk.KB + 1 > kGemmSlots ||
+      (long long)(sc.sk.U + 1) * (sc.sk.G + 1) >= (1ll << 31))   // the schedule arithmetic is 32-bit
     return cudaErrorInvalidConfiguration;
   if (sk_out) *sk_out = sc.sk;
   return launch_rows(a, sc, st);

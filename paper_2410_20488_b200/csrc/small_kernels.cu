@@ -149,22 +149,20 @@ rmsnorm_kernel(Rows rw, int v0, int nv, float *h, Partials pend, const bf16 *__r
       float4 a = __ldcg(hr + idx);
       if (pend.sk.U > 0) {
         const int n = idx * 4, st = n >> 8, t = (n >> 7) & 1, i = n & 127;
-        const int c_first = sk_owner(pend.sk, (long long)st * pend.sk.KB);
-        const int c_last = sk_owner(pend.sk, (long long)(st + 1) * pend.sk.KB - 1);
-        for (int c0 = c_first; c0 <= c_last; c0 += 8) {     // 8 contributors' loads in flight together
-          float4 p[8];
+        const SkContrib k = sk_contributors(pend.sk, st);
+        const float *base = pend.ws + (size_t)t * plane_elems + (size_t)r * 128 + i;
+        for (int c0 = k.c_first; c0 <= k.c_last; c0 += 12) {    // 12 contributors' loads in flight together
+          float4 p[12];
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const int c = c0 + k;
-            p[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (c <= c_last) {
-              const int ord = st - (int)(sk_begin(pend.sk, c) / pend.sk.KB);
-              const float *src = pend.ws + ((size_t)(c * kGemmSlots + ord) * 2 + t) * plane_elems + (size_t)r * 128 + i;
-              p[k] = __ldcg(reinterpret_cast<const float4 *>(src));
-            }
+          for (int j = 0; j < 12; ++j) {
+            const int c = c0 + j;
+            p[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c <= k.c_last)
+              p[j] = __ldcg(reinterpret_cast<const float4 *>(
+                  base + (size_t)(c * kGemmSlots + (c == k.c_first ? k.ord_first : 0)) * 2 * plane_elems));
           }
 #pragma unroll
-          for (int k = 0; k < 8; ++k) { a.x += p[k].x; a.y += p[k].y; a.z += p[k].z; a.w += p[k].w; }
+          for (int j = 0; j < 12; ++j) { a.x += p[j].x; a.y += p[j].y; a.z += p[j].z; a.w += p[j].w; }
         }
         hr[idx] = a;
       }
