@@ -39,21 +39,32 @@ __device__ __forceinline__ void sum_partials(const Partials &p, int st, int m, i
   for (int c0 = k.c_first; c0 <= k.c_last; c0 += 4) {      // 4 contributors' loads in flight together
     float4 a[4], b[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int c = c0 + j;
-      a[j] = b[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (c <= k.c_last) {
-        const float *src = base + (size_t)(c * kGemmSlots + (c == k.c_first ? k.ord_first : 0)) * slot;
-        a[j] = __ldcg(reinterpret_cast<const float4 *>(src));
-        b[j] = __ldcg(reinterpret_cast<const float4 *>(src + plane));
-      }
+    for (int j = 0; j < 4; ++j) {         // unconditional loads (index clamped) so that they issue back to back
+      const int c = min(c0 + j, k.c_last);
+      const float *src = base + (size_t)(c * kGemmSlots + (c == k.c_first ? k.ord_first : 0)) * slot;
+      a[j] = __ldcg(reinterpret_cast<const float4 *>(src));
+      b[j] = __ldcg(reinterpret_cast<const float4 *>(src + plane));
     }
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      v0.x += a[j].x; v0.y += a[j].y; v0.z += a[j].z; v0.w += a[j].w;
-      v1.x += b[j].x; v1.y += b[j].y; v1.z += b[j].z; v1.w += b[j].w;
+      if (c0 + j <= k.c_last) {
+        v0.x += a[j].x; v0.y += a[j].y; v0.z += a[j].z; v0.w += a[j].w;
+        v1.x += b[j].x; v1.y += b[j].y; v1.z += b[j].z; v1.w += b[j].w;
+      }
     }
   }
+}
+
+// 1 / sqrt(mean(h^2) + eps) of token row m from the per-warp sums of squares the RMSNorm kernel left;
+// all 32 lanes of a warp work on the same row, and the butterfly adds in a fixed order
+__device__ __forceinline__ float row_rms_scale(const GemmArgs &a, int m) {
+  if (a.ss == nullptr) return 1.f;
+  const int lane = threadIdx.x & 31, nw = a.K >> 7;
+  const float *p = a.ss + (size_t)m * kNormMaxWarps;
+  float v = (lane < nw ? __ldcg(p + lane) : 0.f) + (lane + 32 < nw ? __ldcg(p + lane + 32) : 0.f);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return rsqrtf(v / (float)a.K + a.eps);
 }
 
 __device__ __forceinline__ void split4(const float v[4], uint2 &hi, uint2 &lo) {
@@ -79,10 +90,11 @@ __global__ void __launch_bounds__(kThreads) qkv_finish_kernel(Partials p, GemmAr
   const int half = a.dh >> 1, hp = 128 / half;
   const int unit = it.st * hp + it.i4 / half, c = it.i4 % half;
   const int s = it.m / a.rw.Ms, v = it.m - s * a.rw.Ms;
+  const float rs = row_rms_scale(a, it.m);          // before any lane drops out: the warp adds together
   if (unit >= a.H + 2 * a.Hkv || v >= a.rows_active) return;
   float4 v0, v1;
   sum_partials(p, it.st, it.m, it.i4, v0, v1);
-  float x1[4] = {v0.x, v0.y, v0.z, v0.w}, x2[4] = {v1.x, v1.y, v1.z, v1.w};
+  float x1[4] = {v0.x * rs, v0.y * rs, v0.z * rs, v0.w * rs}, x2[4] = {v1.x * rs, v1.y * rs, v1.z * rs, v1.w * rs};
   if (unit < a.H + a.Hkv) {     // queries and keys are rotated at the row's tree position
     const float4 *cs = reinterpret_cast<const float4 *>(a.rope + (size_t)it.m * half + c);
     const float4 cs01 = __ldcg(cs), cs23 = __ldcg(cs + 1);
@@ -121,10 +133,11 @@ __global__ void __launch_bounds__(kThreads) swiglu_finish_kernel(Partials p, Gem
   if (!item_of_thread(n_st, a.R, it)) return;
   const int j0 = it.st * 128 + it.i4;
   const int v = it.m % a.rw.Ms;
+  const float rs = row_rms_scale(a, it.m);
   if (j0 >= a.F || v >= a.rows_active) return;
   float4 g, u;
   sum_partials(p, it.st, it.m, it.i4, g, u);
-  const float gg[4] = {g.x, g.y, g.z, g.w}, uu[4] = {u.x, u.y, u.z, u.w};
+  const float gg[4] = {g.x * rs, g.y * rs, g.z * rs, g.w * rs}, uu[4] = {u.x * rs, u.y * rs, u.z * rs, u.w * rs};
   float y[4];
 #pragma unroll
   for (int j = 0; j < 4; ++j) y[j] = gg[j] / (1.f + __expf(-gg[j])) * uu[j];
@@ -141,9 +154,12 @@ __global__ void __launch_bounds__(kThreads) logits_finish_kernel(Partials p, Gem
   Item it;
   if (!item_of_thread(n_st, a.R, it)) return;
   const int n0 = it.st * 256 + it.i4, n1 = n0 + 128;
+  const float rs = row_rms_scale(a, it.m);
   if (n0 >= a.N) return;
   float4 v0, v1;
   sum_partials(p, it.st, it.m, it.i4, v0, v1);
+  v0.x *= rs; v0.y *= rs; v0.z *= rs; v0.w *= rs;
+  v1.x *= rs; v1.y *= rs; v1.z *= rs; v1.w *= rs;
   float *row = a.logits + (size_t)it.m * a.N;
   if ((a.N & 3) == 0) {
     *reinterpret_cast<float4 *>(row + n0) = v0;

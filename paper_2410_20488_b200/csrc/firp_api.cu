@@ -49,14 +49,14 @@ struct firp_ctx {
   int launches = 0;
   bool bound = false, have_weights = false, stepped = false;
   int Rmax = 0, S = 0;
-  bool use_tc = true, use_pdl = true;   // tcgen05/TMA GEMM, programmatic dependent launch
+  bool use_pdl = true;                  // programmatic dependent launch
   int *dev_status = nullptr;            // device status word (bounded waits report here)
   // weights
   firp_weights w{};
   std::vector<const void *> wqkv, wo, wgu, wd, g_attn, g_mlp;
   // device buffers (carved from the caller's workspace)
   bf16 *kv = nullptr;
-  float *h = nullptr, *gemm_ws = nullptr, *logits = nullptr, *top_vals = nullptr;
+  float *h = nullptr, *gemm_ws = nullptr, *ss = nullptr, *logits = nullptr, *top_vals = nullptr;
   bf16 *x = nullptr, *q = nullptr, *o = nullptr, *y = nullptr;
   int32_t *ctx_len = nullptr, *seq_ids = nullptr, *parents = nullptr, *next_parents = nullptr, *chain = nullptr;
   int32_t *top_ids = nullptr, *path = nullptr, *n_acc = nullptr, *accepted = nullptr, *next_tokens = nullptr;
@@ -82,6 +82,7 @@ struct firp_ctx {
     o = c.take<bf16>(2 * R * nq);
     y = c.take<bf16>(2 * R * cfg.d_ffn);
     gemm_ws = c.take<float>((size_t)kGemmMaxCtas * kGemmSlots * 2 * R * 128);
+    ss = c.take<float>(R * kNormMaxWarps);
     logits = c.take<float>(R * cfg.vocab);
     top_ids = c.take<int32_t>(R * kMaxTopB);
     top_vals = c.take<float>(R * kMaxTopB);
@@ -195,7 +196,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   const size_t Rp = (size_t)c->Rmax;          // rows per activation plane
   const firp_step_out *out = ra.out;
   int &nl = c->launches;
-  const bool tc = c->use_tc, pdl = c->use_pdl;
+  const bool pdl = c->use_pdl;
 
   const int mw_out = (rw.Ms + 31) / 32;
   { FIRP_TIMED(KC_TREE_PREP);
@@ -209,6 +210,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     g.X = X; g.x_lo_off = lo_off; g.plane_rows = (int)Rp; g.err = c->dev_status;
     g.W = (const bf16 *)W; g.R = rw.R; g.N = N; g.K = K; g.rw = rw; g.rows_active = act;
     g.ws = c->gemm_ws;
+    if (X == c->x) { g.ss = c->ss; g.eps = cfg.rms_eps; }   // x = h * g: the finisher divides by the row's RMS
     return g;
   };
   // partial tiles a residual GEMM left behind: the next RMSNorm adds them into the residual stream
@@ -221,13 +223,13 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     // the rows that took part in the last residual GEMM get its pending sums; new pseudo rows have none
     const int carried = insert ? rw.T : act;
     { FIRP_TIMED(KC_RMSNORM);
-      FIRP_CUDA(c, launch_rmsnorm(rw, 0, carried, c->h, pending, (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x, Rp * d, pdl, st)); ++nl; }
+      FIRP_CUDA(c, launch_rmsnorm(rw, 0, carried, c->h, pending, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, c->ss, pdl, st)); ++nl; }
     pending.sk.U = 0;
     if (insert) {   // Eq. 3 on the raw (now complete) residual row of the root, then the norm of the new rows
       { FIRP_TIMED(KC_PSEUDO_PROJ);
         launch_pseudo_proj(rw, (const bf16 *)c->w.pred_w, (const bf16 *)c->w.pred_b, d, c->h, pdl, st); ++nl; }
       FIRP_TIMED(KC_RMSNORM);
-      FIRP_CUDA(c, launch_rmsnorm(rw, rw.T, rw.Ms, c->h, none, (const bf16 *)c->g_attn[j], cfg.rms_eps, d, c->x, Rp * d, pdl, st)); ++nl;
+      FIRP_CUDA(c, launch_rmsnorm(rw, rw.T, rw.Ms, c->h, none, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, c->ss, pdl, st)); ++nl;
     }
     bf16 *kplane = c->kv + (size_t)j * c->kv_layer();
     {
@@ -237,7 +239,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       g.q = c->q; g.q_lo_off = Rp * nq; g.kcache = kplane; g.seq_stride = c->kv_seq(); g.kv_stride = c->kv_plane(); g.max_ctx = cfg.max_ctx;
       FIRP_TIMED(KC_GEMM_QKV);
       Partials p = pending;
-      FIRP_CUDA(c, launch_gemm(EPI_QKV_ROPE, g, tc, pdl, st, &p.sk)); ++nl;
+      FIRP_CUDA(c, launch_gemm_tc(EPI_QKV_ROPE, g, pdl, st, &p.sk)); ++nl;
       if (p.sk.U > 0) { FIRP_CUDA(c, launch_gemm_finish(EPI_QKV_ROPE, p, g, pdl, st)); ++nl; }
     }
     {
@@ -254,36 +256,34 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     }
     {
       GemmArgs g = gemm_base(c->o, Rp * nq, c->wo[j], d, nq, act);
-      g.h_out = c->h;
       FIRP_TIMED(KC_GEMM_O);
-      FIRP_CUDA(c, launch_gemm(EPI_RESIDUAL, g, tc, pdl, st, &pending.sk)); ++nl;
+      FIRP_CUDA(c, launch_gemm_tc(EPI_RESIDUAL, g, pdl, st, &pending.sk)); ++nl;
     }
     { FIRP_TIMED(KC_RMSNORM);
-      FIRP_CUDA(c, launch_rmsnorm(rw, 0, act, c->h, pending, (const bf16 *)c->g_mlp[j], cfg.rms_eps, d, c->x, Rp * d, pdl, st)); ++nl; }
+      FIRP_CUDA(c, launch_rmsnorm(rw, 0, act, c->h, pending, (const bf16 *)c->g_mlp[j], d, c->x, Rp * d, c->ss, pdl, st)); ++nl; }
     pending.sk.U = 0;
     {
       GemmArgs g = gemm_base(c->x, Rp * d, c->wgu[j], 2 * F, d, act);
       g.y = c->y; g.y_lo_off = Rp * F; g.F = F;
       FIRP_TIMED(KC_GEMM_GATE_UP);
       Partials p = pending;
-      FIRP_CUDA(c, launch_gemm(EPI_SWIGLU, g, tc, pdl, st, &p.sk)); ++nl;
+      FIRP_CUDA(c, launch_gemm_tc(EPI_SWIGLU, g, pdl, st, &p.sk)); ++nl;
       if (p.sk.U > 0) { FIRP_CUDA(c, launch_gemm_finish(EPI_SWIGLU, p, g, pdl, st)); ++nl; }
     }
     {
       GemmArgs g = gemm_base(c->y, Rp * F, c->wd[j], d, F, act);
-      g.h_out = c->h;
       FIRP_TIMED(KC_GEMM_DOWN);
-      FIRP_CUDA(c, launch_gemm(EPI_RESIDUAL, g, tc, pdl, st, &pending.sk)); ++nl;
+      FIRP_CUDA(c, launch_gemm_tc(EPI_RESIDUAL, g, pdl, st, &pending.sk)); ++nl;
     }
   }
   if (ra.want_head) {
     { FIRP_TIMED(KC_RMSNORM);
-      FIRP_CUDA(c, launch_rmsnorm(rw, 0, rw.Ms, c->h, pending, (const bf16 *)c->w.g_final, cfg.rms_eps, d, c->x, Rp * d, pdl, st)); ++nl; }
+      FIRP_CUDA(c, launch_rmsnorm(rw, 0, rw.Ms, c->h, pending, (const bf16 *)c->w.g_final, d, c->x, Rp * d, c->ss, pdl, st)); ++nl; }
     GemmArgs g = gemm_base(c->x, Rp * d, c->w.lm_head, cfg.vocab, d, rw.Ms);
     g.logits = ra.logits_dst;
     { FIRP_TIMED(KC_GEMM_LM_HEAD);
       Partials p = pending;
-      FIRP_CUDA(c, launch_gemm(EPI_LOGITS, g, tc, pdl, st, &p.sk)); ++nl;
+      FIRP_CUDA(c, launch_gemm_tc(EPI_LOGITS, g, pdl, st, &p.sk)); ++nl;
       if (p.sk.U > 0) { FIRP_CUDA(c, launch_gemm_finish(EPI_LOGITS, p, g, pdl, st)); ++nl; } }
     { FIRP_TIMED(KC_TOPB);
       launch_topb(ra.logits_dst, rw.R, cfg.vocab, cfg.top_b, c->top_ids, c->top_vals, pdl, st); ++nl; }
@@ -314,7 +314,7 @@ int firp_create(const firp_model_cfg *cfg, firp_ctx **out) {
   firp_ctx *c = new firp_ctx();
   c->cfg = *cfg;
   auto bad = [&](const char *why) { delete c; fprintf(stderr, "firp_create: %s\n", why); return (int)FIRP_ERR_BAD_ARG; };
-  if (cfg->n_layers < 1 || cfg->d_model < 8 || cfg->d_model % 8 || cfg->d_model > 8192) return bad("d_model must be a multiple of 8, <= 8192");
+  if (cfg->n_layers < 1 || cfg->d_model < 128 || cfg->d_model % 128 || cfg->d_model > 8192) return bad("d_model must be a multiple of 128, <= 8192");
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return bad("head_dim must be 64 or 128");
   if (cfg->n_heads < 1 || cfg->n_kv_heads < 1 || cfg->n_heads % cfg->n_kv_heads) return bad("n_heads must be a multiple of n_kv_heads");
   if (cfg->d_ffn < 8 || cfg->d_ffn % 8 || cfg->vocab < 8) return bad("d_ffn must be a multiple of 8");
@@ -329,9 +329,8 @@ int firp_create(const firp_model_cfg *cfg, firp_ctx **out) {
   c->Rmax = (int)align_up(rows, 16);
   c->S = cfg->max_depth + 1;
   c->n_hi.assign(cfg->max_batch, 0);
-  // debugging switches: FIRP_GEMM=mma selects the mma.sync GEMM, FIRP_PDL=0 plain stream order
-  const char *eg = getenv("FIRP_GEMM"), *ep = getenv("FIRP_PDL");
-  c->use_tc = !(eg && strcmp(eg, "mma") == 0);
+  // debugging switch: FIRP_PDL=0 launches every kernel in plain stream order
+  const char *ep = getenv("FIRP_PDL");
   c->use_pdl = !(ep && strcmp(ep, "0") == 0);
 
   c->ws_bytes = c->carve(nullptr);
@@ -367,7 +366,7 @@ int firp_bind_buffers(firp_ctx *ctx, void *workspace, void *kv_cache, void *stre
   FIRP_CUDA(ctx, cudaStreamSynchronize(st));
   std::fill(ctx->n_hi.begin(), ctx->n_hi.end(), 0);
   ctx->last_parents.clear(); ctx->last_next_parents.clear(); ctx->last_seq_ids.clear();
-  if (ctx->use_tc && !gemm_tc_available())
+  if (!gemm_tc_available())
     return fail(ctx, FIRP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
   ctx->bound = true; ctx->stepped = false;
   return FIRP_OK;

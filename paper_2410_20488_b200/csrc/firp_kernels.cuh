@@ -79,9 +79,11 @@ struct Partials {
   int ws_rows;       // token rows per scratch tile
 };
 // For rows with v in [v0, v1): if `pending` has units, first h[r] += the partial tiles of a residual GEMM;
-// then x[r] = rmsnorm(h[r]) * g as a (hi, lo) bf16 pair.
-cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Partials &pending, const bf16 *g, float eps,
-                           int d, bf16 *x, size_t x_lo_off, bool pdl, cudaStream_t st);
+// then x[r] = h[r] * g as a (hi, lo) bf16 pair and ss[r][w] = sum of squares of the 128 columns of warp w.
+// The 1 / sqrt(mean(h^2) + eps) of RMSNorm is applied by the finisher of the GEMM that consumes x.
+constexpr int kNormMaxWarps = 64;   // d <= 8192
+cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Partials &pending, const bf16 *g, int d,
+                           bf16 *x, size_t x_lo_off, float *ss, bool pdl, cudaStream_t st);
 
 // Eq. 3: h[s*Ms + T + i] = W_i h[s*Ms + anchor] + b_i
 void launch_pseudo_proj(const Rows &rw, const bf16 *pred_w, const bf16 *pred_b, int d, float *h, bool pdl, cudaStream_t st);
@@ -133,11 +135,11 @@ struct GemmArgs {
   int *err;         // device status word (set to a non-zero code if a bounded wait gives up)
   int N, K;
   Rows rw; int rows_active;      // rows with v < rows_active are written, the others skipped
-  // stream-K scratch of the tcgen05 kernel: partial tiles [kGemmMaxCtas][kGemmSlots][2][plane_rows][128] fp32
+  // stream-K scratch: partial tiles [kGemmMaxCtas][kGemmSlots][2][plane_rows][128] fp32
   float *ws;
-  // EPI_RESIDUAL: the result is to be added to h_out[R][N] (the mma.sync kernel adds it itself; the
-  // tcgen05 kernel leaves partial tiles for the RMSNorm kernel that follows)
-  float *h_out;
+  // finishers: X holds h * g, not yet divided by the RMS: row m of the result is scaled by
+  // 1 / sqrt(sum_w ss[m][w] / K + eps) (ss == NULL: X is used as it is)
+  const float *ss; float eps;
   // EPI_QKV_ROPE
   int H, Hkv, dh;
   const float2 *rope; const int32_t *seq_ids; const int32_t *ctx_len;
@@ -148,14 +150,11 @@ struct GemmArgs {
   // EPI_LOGITS: logits[R][N]
   float *logits;
 };
-// use_tc: tcgen05/TMA kernel: leaves partial tiles in a.ws under the schedule *sk_out, to be finished by
-// launch_gemm_finish (or, for EPI_RESIDUAL, by launch_rmsnorm).  Otherwise the mma.sync kernel (a debugging
-// cross-check) with the epilogue fused: *sk_out gets U = 0, nothing is pending.
+// The GEMM leaves partial tiles in a.ws under the schedule *sk_out, to be finished by launch_gemm_finish
+// (or, for EPI_RESIDUAL, by launch_rmsnorm).  `epi` only selects how weight rows are grouped into supertiles.
 // pdl: launch with programmatic stream serialization (the kernel waits on its predecessor itself).
-cudaError_t launch_gemm(GemmEpilogue epi, const GemmArgs &a, bool use_tc, bool pdl, cudaStream_t st, StreamK *sk_out);
-cudaError_t launch_gemm_finish(GemmEpilogue epi, const Partials &p, const GemmArgs &a, bool pdl, cudaStream_t st);
-cudaError_t launch_gemm_mma(GemmEpilogue epi, const GemmArgs &a, cudaStream_t st);
 cudaError_t launch_gemm_tc(GemmEpilogue epi, const GemmArgs &a, bool pdl, cudaStream_t st, StreamK *sk_out);
+cudaError_t launch_gemm_finish(GemmEpilogue epi, const Partials &p, const GemmArgs &a, bool pdl, cudaStream_t st);
 bool gemm_tc_available();         // the driver entry point for tensor-map encoding was found
 
 // ---- tree-masked split-KV attention ---------------------------------------

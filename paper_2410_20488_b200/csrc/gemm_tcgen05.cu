@@ -39,7 +39,6 @@
 #include <tuple>
 
 #include "firp_kernels.cuh"
-#include "gemm_epilogue.cuh"
 #include "launch_util.cuh"
 
 namespace firp {
@@ -100,12 +99,13 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm,
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
       ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar), "l"(policy) : "memory");
 }
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap *tm, int x, int y) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tm), "r"(x), "r"(y) : "memory");
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap *tm, int x, int y, uint64_t policy) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile.L2::cache_hint [%0, {%1, %2}], %3;"
+               ::"l"(tm), "r"(x), "r"(y), "l"(policy) : "memory");
 }
-__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap *tm, int x, int y, int z, int w) {
-  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];"
-               ::"l"(tm), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap *tm, int x, int y, int z, int w, uint64_t policy) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile.L2::cache_hint [%0, {%1, %2, %3, %4}], %5;"
+               ::"l"(tm), "r"(x), "r"(y), "r"(z), "r"(w), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -230,14 +230,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           const int pst = up / KB, pkb = up - pst * KB;
           if (sc.mode == ROWS_ROTARY) {
             const int hp = BM / sc.half;
-            tma_prefetch_4d(&tmW, pkb * BK, 0, 0, pst * hp);
-            tma_prefetch_4d(&tmW, pkb * BK, 0, 1, pst * hp);
+            tma_prefetch_4d(&tmW, pkb * BK, 0, 0, pst * hp, pol);
+            tma_prefetch_4d(&tmW, pkb * BK, 0, 1, pst * hp, pol);
           } else if (sc.mode == ROWS_GATE_UP) {
-            tma_prefetch_2d(&tmW, pkb * BK, pst * BM);
-            tma_prefetch_2d(&tmW, pkb * BK, sc.F + pst * BM);
+            tma_prefetch_2d(&tmW, pkb * BK, pst * BM, pol);
+            tma_prefetch_2d(&tmW, pkb * BK, sc.F + pst * BM, pol);
           } else {
-            tma_prefetch_2d(&tmW, pkb * BK, pst * (TM * BM));
-            tma_prefetch_2d(&tmW, pkb * BK, pst * (TM * BM) + BM);
+            tma_prefetch_2d(&tmW, pkb * BK, pst * (TM * BM), pol);
+            tma_prefetch_2d(&tmW, pkb * BK, pst * (TM * BM) + BM, pol);
           }
         }
         const int u = u0 + it;

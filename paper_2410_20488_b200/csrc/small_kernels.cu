@@ -1,11 +1,8 @@
 // Small kernels of the FIRP step: tree bookkeeping, embedding, residual-add + RMSNorm,
 // the pseudo-hidden projection (Eq. 3), top-B, the acceptance walk / next tree, KV compaction.
-#include <cooperative_groups.h>
-
 #include "firp_kernels.cuh"
 #include "launch_util.cuh"
 
-namespace cg = cooperative_groups;
 
 namespace firp {
 
@@ -98,112 +95,75 @@ void launch_embed(const Rows &rw, const int32_t *d_tokens, const bf16 *embed, in
 }
 
 // ---------------------------------------------------------------------------
-// RMSNorm of the fp32 residual rows -> bf16 (hi, lo) GEMM operand.
+// Residual update + first half of RMSNorm, as a flat elementwise kernel.
+//   h[r] += the partial tiles a residual GEMM left in scratch (fixed order: ascending CTA index)
+//   x[r]  = h[r] * g as a (hi, lo) bf16 pair -- NOT yet divided by the row's RMS
+//   ss[r][w] = sum of h[r][c]^2 over the 128 columns of warp w
+// The division by sqrt(mean(h^2) + eps) commutes with the GEMM that consumes x, so that GEMM's
+// finisher applies it to the fp32 sums (it adds the ss[r][*] in a fixed order).  This kernel then
+// has no reduction across threads beyond a warp, no barrier, and every thread is independent.
+// A thread owns 4 neighbouring columns of one row; d must be a multiple of 128.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ float block_sum(float v, float *red) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  const int w = threadIdx.x >> 5, nw = blockDim.x >> 5;
-  if ((threadIdx.x & 31) == 0) red[w] = v;
-  __syncthreads();
-  float t = (threadIdx.x < nw) ? red[threadIdx.x] : 0.f;
-  if (w == 0) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-    if (threadIdx.x == 0) red[0] = t;
-  }
-  __syncthreads();
-  t = red[0];
-  __syncthreads();
-  return t;
-}
-
 constexpr int kNormThreads = 256;
-constexpr int kNormCluster = 4;   // CTAs per token row, each owns a quarter of the columns
-constexpr int kNormMaxVec = 2;    // float4 per thread: d <= 4 * 256 * 2 * 4 = 8192
 
-// One cluster of 4 CTAs per token row.  If a residual GEMM left partial tiles behind, they are summed
-// into the residual stream first (fixed order: ascending CTA index of the GEMM); the sum of squares
-// is combined across the cluster through distributed shared memory.
-__global__ void __cluster_dims__(kNormCluster, 1, 1) __launch_bounds__(kNormThreads)
-rmsnorm_kernel(Rows rw, int v0, int nv, float *h, Partials pend, const bf16 *__restrict__ g, float eps,
-               int d, bf16 *x, size_t x_lo_off, int pdl) {
-  __shared__ float red[32];
-  __shared__ float cl_ss;
-  cg::cluster_group cluster = cg::this_cluster();
-  const int q = (int)cluster.block_rank();
+__global__ void __launch_bounds__(kNormThreads)
+rmsnorm_kernel(Rows rw, int v0, int nv, float *h, Partials pend, const bf16 *__restrict__ g, int d, bf16 *x,
+               size_t x_lo_off, float *ss, int pdl) {
   if (pdl) { griddep_launch(); griddep_wait(); }
-  const int rowi = blockIdx.x / kNormCluster;
+  const int nvec = d >> 2;                                  // float4 per row, a multiple of 32
+  const unsigned t = blockIdx.x * kNormThreads + threadIdx.x;
+  if (t >= (unsigned)(rw.n_seq * nv * nvec)) return;        // whole warps drop out together
+  const int rowi = (int)(t / (unsigned)nvec), idx = (int)(t % (unsigned)nvec);
   const int s = rowi / nv, v = v0 + rowi % nv;
   const int r = s * rw.Ms + v;
   float4 *hr = reinterpret_cast<float4 *>(h + (size_t)r * d);
-  const int nvec = d >> 2, per = (nvec + kNormCluster - 1) / kNormCluster;
-  const int f0 = q * per, f1 = min(nvec, f0 + per);
-  const size_t plane_elems = (size_t)pend.ws_rows * 128;
-  float4 val[kNormMaxVec];
-  float ss = 0.f;
+  float4 a = __ldcg(hr + idx);
+  if (pend.sk.U > 0) {
+    const size_t plane_elems = (size_t)pend.ws_rows * 128;
+    const int n = idx * 4, st = n >> 8, tl = (n >> 7) & 1, i = n & 127;
+    const SkContrib k = sk_contributors(pend.sk, st);
+    const float *base = pend.ws + (size_t)tl * plane_elems + (size_t)r * 128 + i;
+    for (int c0 = k.c_first; c0 <= k.c_last; c0 += 12) {    // 12 contributors' loads in flight together
+      float4 p[12];
 #pragma unroll
-  for (int it = 0; it < kNormMaxVec; ++it) {
-    const int idx = f0 + threadIdx.x + it * kNormThreads;
-    if (idx < f1) {
-      float4 a = __ldcg(hr + idx);
-      if (pend.sk.U > 0) {
-        const int n = idx * 4, st = n >> 8, t = (n >> 7) & 1, i = n & 127;
-        const SkContrib k = sk_contributors(pend.sk, st);
-        const float *base = pend.ws + (size_t)t * plane_elems + (size_t)r * 128 + i;
-        for (int c0 = k.c_first; c0 <= k.c_last; c0 += 12) {    // 12 contributors' loads in flight together
-          float4 p[12];
-#pragma unroll
-          for (int j = 0; j < 12; ++j) {
-            const int c = c0 + j;
-            p[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (c <= k.c_last)
-              p[j] = __ldcg(reinterpret_cast<const float4 *>(
-                  base + (size_t)(c * kGemmSlots + (c == k.c_first ? k.ord_first : 0)) * 2 * plane_elems));
-          }
-#pragma unroll
-          for (int j = 0; j < 12; ++j) { a.x += p[j].x; a.y += p[j].y; a.z += p[j].z; a.w += p[j].w; }
-        }
-        hr[idx] = a;
+      for (int j = 0; j < 12; ++j) {      // unconditional loads (index clamped) so that they issue back to back
+        const int c = min(c0 + j, k.c_last);
+        p[j] = __ldcg(reinterpret_cast<const float4 *>(
+            base + (size_t)(c * kGemmSlots + (c == k.c_first ? k.ord_first : 0)) * 2 * plane_elems));
       }
-      val[it] = a;
-      ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
-    }
-  }
-  ss = block_sum(ss, red);
-  if (threadIdx.x == 0) cl_ss = ss;
-  cluster.sync();
-  float total = 0.f;
 #pragma unroll
-  for (int k = 0; k < kNormCluster; ++k) total += *cluster.map_shared_rank(&cl_ss, k);
-  cluster.sync();                     // peers have read cl_ss before anyone may exit
-  const float rs = rsqrtf(total / (float)d + eps);
-#pragma unroll
-  for (int it = 0; it < kNormMaxVec; ++it) {
-    const int i = f0 + threadIdx.x + it * kNormThreads;
-    if (i < f1) {
-      const __nv_bfloat162 g01 = reinterpret_cast<const __nv_bfloat162 *>(g)[2 * i];
-      const __nv_bfloat162 g23 = reinterpret_cast<const __nv_bfloat162 *>(g)[2 * i + 1];
-      const float2 ga = __bfloat1622float2(g01), gb = __bfloat1622float2(g23);
-      const float v0 = val[it].x * rs * ga.x, v1 = val[it].y * rs * ga.y;
-      const float v2 = val[it].z * rs * gb.x, v3 = val[it].w * rs * gb.y;
-      const __nv_bfloat162 o01 = __floats2bfloat162_rn(v0, v1), o23 = __floats2bfloat162_rn(v2, v3);
-      const float2 f01 = __bfloat1622float2(o01), f23 = __bfloat1622float2(o23);
-      __nv_bfloat162 *xo = reinterpret_cast<__nv_bfloat162 *>(x + (size_t)r * d) + 2 * i;
-      xo[0] = o01; xo[1] = o23;                       // hi plane
-      __nv_bfloat162 *xl = reinterpret_cast<__nv_bfloat162 *>(x + x_lo_off + (size_t)r * d) + 2 * i;
-      xl[0] = __floats2bfloat162_rn(v0 - f01.x, v1 - f01.y);   // lo plane: what the hi half lost
-      xl[1] = __floats2bfloat162_rn(v2 - f23.x, v3 - f23.y);
+      for (int j = 0; j < 12; ++j) {
+        if (c0 + j <= k.c_last) { a.x += p[j].x; a.y += p[j].y; a.z += p[j].z; a.w += p[j].w; }
+      }
     }
+    hr[idx] = a;
   }
+  float sq = a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+  if ((threadIdx.x & 31) == 0) ss[(size_t)r * kNormMaxWarps + (idx >> 5)] = sq;
+  const __nv_bfloat162 g01 = reinterpret_cast<const __nv_bfloat162 *>(g)[2 * idx];
+  const __nv_bfloat162 g23 = reinterpret_cast<const __nv_bfloat162 *>(g)[2 * idx + 1];
+  const float2 ga = __bfloat1622float2(g01), gb = __bfloat1622float2(g23);
+  const float y0 = a.x * ga.x, y1 = a.y * ga.y, y2 = a.z * gb.x, y3 = a.w * gb.y;
+  const __nv_bfloat162 o01 = __floats2bfloat162_rn(y0, y1), o23 = __floats2bfloat162_rn(y2, y3);
+  const float2 f01 = __bfloat1622float2(o01), f23 = __bfloat1622float2(o23);
+  const __nv_bfloat162 l01 = __floats2bfloat162_rn(y0 - f01.x, y1 - f01.y);     // lo plane: what the hi half lost
+  const __nv_bfloat162 l23 = __floats2bfloat162_rn(y2 - f23.x, y3 - f23.y);
+  uint2 hi2, lo2;
+  hi2.x = *reinterpret_cast<const uint32_t *>(&o01); hi2.y = *reinterpret_cast<const uint32_t *>(&o23);
+  lo2.x = *reinterpret_cast<const uint32_t *>(&l01); lo2.y = *reinterpret_cast<const uint32_t *>(&l23);
+  *reinterpret_cast<uint2 *>(x + (size_t)r * d + 4 * idx) = hi2;
+  *reinterpret_cast<uint2 *>(x + x_lo_off + (size_t)r * d + 4 * idx) = lo2;
 }
 
-cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Partials &pending, const bf16 *g, float eps,
-                           int d, bf16 *x, size_t x_lo_off, bool pdl, cudaStream_t st) {
+cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Partials &pending, const bf16 *g, int d,
+                           bf16 *x, size_t x_lo_off, float *ss, bool pdl, cudaStream_t st) {
   const int nv = v1 - v0;
   if (nv <= 0) return cudaSuccess;
-  return launch_k(rmsnorm_kernel, dim3(rw.n_seq * nv * kNormCluster), dim3(kNormThreads), 0, st, pdl, rw, v0, nv, h,
-                  pending, g, eps, d, x, x_lo_off, pdl ? 1 : 0);
+  const int threads = rw.n_seq * nv * (d >> 2);
+  return launch_k(rmsnorm_kernel, dim3((threads + kNormThreads - 1) / kNormThreads), dim3(kNormThreads), 0, st, pdl, rw,
+                  v0, nv, h, pending, g, d, x, x_lo_off, ss, pdl ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------

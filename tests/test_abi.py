@@ -45,7 +45,7 @@ def test_create_validates_configuration(lib):
     assert firp.firp_kv_bytes(ctx) == 1 * 2 * 2 * 256 * 4 * 64 * 2
     firp.firp_destroy(ctx)
     for bad in (dict(head_dim=96), dict(n_heads=3, n_kv_heads=2), dict(max_tree=129), dict(max_k=9), dict(top_b=0),
-                dict(top_b=9), dict(max_batch=0), dict(max_batch=4, max_tree=64), dict(d_model=250),
+                dict(top_b=9), dict(max_batch=0), dict(max_batch=4, max_tree=64), dict(d_model=192),
                 dict(max_depth=16), dict(max_ctx=4)):
         with pytest.raises(firp.FirpError):
             firp.firp_create(good_cfg(**bad))
