@@ -78,7 +78,7 @@ def class_bytes(shape, n_ctx: float) -> dict:
     (read once) for the GEMMs and the Eq. 3 maps, the K and V planes of one layer for the attention."""
     s = shape
     M = s.T + s.k
-    return dict(gemm_qkv_rope=2 * s.n_qkv * s.d, gemm_o=2 * s.d * s.n_q, gemm_gate_up_swiglu=2 * 2 * s.F * s.d,
+    return dict(gemm_qkv=2 * s.n_qkv * s.d, gemm_o=2 * s.d * s.n_q, gemm_gate_up=2 * 2 * s.F * s.d,
                 gemm_down=2 * s.d * s.F, gemm_lm_head=2 * s.V * s.d, pseudo_proj=2 * s.k * s.d * s.d,
                 tree_attention=2 * 2 * s.n_kv * (n_ctx + M))
 

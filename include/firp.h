@@ -157,8 +157,8 @@ int firp_last_launch_count(const firp_ctx *ctx);
  * Per-kernel timing aid (measurement only; it changes no result).  While enabled, every kernel
  * launch of firp_step / firp_prefill / firp_kv_commit is bracketed by a pair of CUDA events on
  * the call's stream, grouped by kernel class (the steps of Section 3.2-3.4: tree bookkeeping,
- * embedding, RMSNorm, Eq. 3 projection, the five weight-streaming GEMMs, tree attention, top-B,
- * acceptance walk, KV compaction).  The events serialise launches that otherwise overlap, so a
+ * embedding, residual + RMSNorm, Eq. 3 projection, the five weight-streaming GEMMs and their
+ * finishers, tree attention, top-B, acceptance walk, KV compaction).  The events serialise launches that otherwise overlap, so a
  * profiled step is slower than an unprofiled one: use it for per-kernel durations, not for the
  * step latency.
  *   firp_profile_enable  on != 0 starts (and clears) the collection, 0 stops it.

@@ -31,12 +31,12 @@ struct Carver {
 
 // Kernel classes of the per-kernel timing aid (firp_profile_*).
 enum KernelClass {
-  KC_TREE_PREP = 0, KC_EMBED, KC_RMSNORM, KC_PSEUDO_PROJ, KC_GEMM_QKV, KC_ATTENTION, KC_GEMM_O, KC_GEMM_GATE_UP,
-  KC_GEMM_DOWN, KC_GEMM_LM_HEAD, KC_TOPB, KC_ACCEPT, KC_COMMIT, KC_COUNT
+  KC_TREE_PREP = 0, KC_EMBED, KC_RMSNORM, KC_PSEUDO_PROJ, KC_GEMM_QKV, KC_QKV_FINISH, KC_ATTENTION, KC_GEMM_O,
+  KC_GEMM_GATE_UP, KC_SWIGLU_FINISH, KC_GEMM_DOWN, KC_GEMM_LM_HEAD, KC_LOGITS_FINISH, KC_TOPB, KC_ACCEPT, KC_COMMIT, KC_COUNT
 };
 static const char *const kClassNames[KC_COUNT] = {
-    "tree_prep", "embed", "add_rmsnorm", "pseudo_proj", "gemm_qkv_rope", "tree_attention", "gemm_o", "gemm_gate_up_swiglu",
-    "gemm_down", "gemm_lm_head", "topb", "accept_next_tree", "kv_commit"};
+    "tree_prep", "embed", "residual_rmsnorm", "pseudo_proj", "gemm_qkv", "qkv_rope_finish", "tree_attention", "gemm_o",
+    "gemm_gate_up", "swiglu_finish", "gemm_down", "gemm_lm_head", "logits_finish", "topb", "accept_next_tree", "kv_commit"};
 
 struct firp_ctx {
   firp_model_cfg cfg{};
@@ -77,7 +77,7 @@ struct firp_ctx {
     const int d = cfg.d_model, nq = cfg.n_heads * cfg.head_dim, half = cfg.head_dim / 2;
     const size_t R = Rmax;
     h = c.take<float>(R * d);
-    x = c.take<bf16>(2 * R * d);            // activations: hi plane, then lo plane
+    x = c.take<bf16>(3 * R * d);            // normalised activations: hi plane, lo plane, third plane (QKV input)
     q = c.take<bf16>(2 * R * nq);
     o = c.take<bf16>(2 * R * nq);
     y = c.take<bf16>(2 * R * cfg.d_ffn);
@@ -208,7 +208,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   auto gemm_base = [&](const bf16 *X, size_t lo_off, const void *W, int N, int K, int act) {
     GemmArgs g{};
     g.X = X; g.x_lo_off = lo_off; g.plane_rows = (int)Rp; g.err = c->dev_status;
-    g.W = (const bf16 *)W; g.R = rw.R; g.N = N; g.K = K; g.rw = rw; g.rows_active = act;
+    g.W = (const bf16 *)W; g.R = rw.R; g.N = N; g.K = K; g.rw = rw; g.rows_active = act; g.planes = 2;
     g.ws = c->gemm_ws;
     if (X == c->x) { g.ss = c->ss; g.eps = cfg.rms_eps; }   // x = h * g: the finisher divides by the row's RMS
     return g;
@@ -223,24 +223,26 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     // the rows that took part in the last residual GEMM get its pending sums; new pseudo rows have none
     const int carried = insert ? rw.T : act;
     { FIRP_TIMED(KC_RMSNORM);
-      FIRP_CUDA(c, launch_rmsnorm(rw, 0, carried, c->h, pending, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, c->ss, pdl, st)); ++nl; }
+      FIRP_CUDA(c, launch_rmsnorm(rw, 0, carried, c->h, pending, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, 3, c->ss, pdl, st)); ++nl; }
     pending.sk.U = 0;
     if (insert) {   // Eq. 3 on the raw (now complete) residual row of the root, then the norm of the new rows
       { FIRP_TIMED(KC_PSEUDO_PROJ);
         launch_pseudo_proj(rw, (const bf16 *)c->w.pred_w, (const bf16 *)c->w.pred_b, d, c->h, pdl, st); ++nl; }
       FIRP_TIMED(KC_RMSNORM);
-      FIRP_CUDA(c, launch_rmsnorm(rw, rw.T, rw.Ms, c->h, none, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, c->ss, pdl, st)); ++nl;
+      FIRP_CUDA(c, launch_rmsnorm(rw, rw.T, rw.Ms, c->h, none, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, 3, c->ss, pdl, st)); ++nl;
     }
     bf16 *kplane = c->kv + (size_t)j * c->kv_layer();
     {
       GemmArgs g = gemm_base(c->x, Rp * d, c->wqkv[j], (H + 2 * Hkv) * dh, d, act);
       g.H = H; g.Hkv = Hkv; g.dh = dh;
+      g.planes = 3;   // keys and values are rounded to bf16 for the cache: their inputs carry ~24 mantissa bits
       g.rope = c->meta.rope; g.seq_ids = c->seq_ids; g.ctx_len = c->ctx_len;
       g.q = c->q; g.q_lo_off = Rp * nq; g.kcache = kplane; g.seq_stride = c->kv_seq(); g.kv_stride = c->kv_plane(); g.max_ctx = cfg.max_ctx;
-      FIRP_TIMED(KC_GEMM_QKV);
       Partials p = pending;
-      FIRP_CUDA(c, launch_gemm_tc(EPI_QKV_ROPE, g, pdl, st, &p.sk)); ++nl;
-      if (p.sk.U > 0) { FIRP_CUDA(c, launch_gemm_finish(EPI_QKV_ROPE, p, g, pdl, st)); ++nl; }
+      { FIRP_TIMED(KC_GEMM_QKV);
+        FIRP_CUDA(c, launch_gemm_tc(EPI_QKV_ROPE, g, pdl, st, &p.sk)); ++nl; }
+      FIRP_TIMED(KC_QKV_FINISH);
+      FIRP_CUDA(c, launch_gemm_finish(EPI_QKV_ROPE, p, g, pdl, st)); ++nl;
     }
     {
       AttnArgs a{};
@@ -260,15 +262,16 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       FIRP_CUDA(c, launch_gemm_tc(EPI_RESIDUAL, g, pdl, st, &pending.sk)); ++nl;
     }
     { FIRP_TIMED(KC_RMSNORM);
-      FIRP_CUDA(c, launch_rmsnorm(rw, 0, act, c->h, pending, (const bf16 *)c->g_mlp[j], d, c->x, Rp * d, c->ss, pdl, st)); ++nl; }
+      FIRP_CUDA(c, launch_rmsnorm(rw, 0, act, c->h, pending, (const bf16 *)c->g_mlp[j], d, c->x, Rp * d, 2, c->ss, pdl, st)); ++nl; }
     pending.sk.U = 0;
     {
       GemmArgs g = gemm_base(c->x, Rp * d, c->wgu[j], 2 * F, d, act);
       g.y = c->y; g.y_lo_off = Rp * F; g.F = F;
-      FIRP_TIMED(KC_GEMM_GATE_UP);
       Partials p = pending;
-      FIRP_CUDA(c, launch_gemm_tc(EPI_SWIGLU, g, pdl, st, &p.sk)); ++nl;
-      if (p.sk.U > 0) { FIRP_CUDA(c, launch_gemm_finish(EPI_SWIGLU, p, g, pdl, st)); ++nl; }
+      { FIRP_TIMED(KC_GEMM_GATE_UP);
+        FIRP_CUDA(c, launch_gemm_tc(EPI_SWIGLU, g, pdl, st, &p.sk)); ++nl; }
+      FIRP_TIMED(KC_SWIGLU_FINISH);
+      FIRP_CUDA(c, launch_gemm_finish(EPI_SWIGLU, p, g, pdl, st)); ++nl;
     }
     {
       GemmArgs g = gemm_base(c->y, Rp * F, c->wd[j], d, F, act);
@@ -278,13 +281,14 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   }
   if (ra.want_head) {
     { FIRP_TIMED(KC_RMSNORM);
-      FIRP_CUDA(c, launch_rmsnorm(rw, 0, rw.Ms, c->h, pending, (const bf16 *)c->w.g_final, d, c->x, Rp * d, c->ss, pdl, st)); ++nl; }
+      FIRP_CUDA(c, launch_rmsnorm(rw, 0, rw.Ms, c->h, pending, (const bf16 *)c->w.g_final, d, c->x, Rp * d, 2, c->ss, pdl, st)); ++nl; }
     GemmArgs g = gemm_base(c->x, Rp * d, c->w.lm_head, cfg.vocab, d, rw.Ms);
     g.logits = ra.logits_dst;
-    { FIRP_TIMED(KC_GEMM_LM_HEAD);
-      Partials p = pending;
-      FIRP_CUDA(c, launch_gemm_tc(EPI_LOGITS, g, pdl, st, &p.sk)); ++nl;
-      if (p.sk.U > 0) { FIRP_CUDA(c, launch_gemm_finish(EPI_LOGITS, p, g, pdl, st)); ++nl; } }
+    { Partials p = pending;
+      { FIRP_TIMED(KC_GEMM_LM_HEAD);
+        FIRP_CUDA(c, launch_gemm_tc(EPI_LOGITS, g, pdl, st, &p.sk)); ++nl; }
+      FIRP_TIMED(KC_LOGITS_FINISH);
+      FIRP_CUDA(c, launch_gemm_finish(EPI_LOGITS, p, g, pdl, st)); ++nl; }
     { FIRP_TIMED(KC_TOPB);
       launch_topb(ra.logits_dst, rw.R, cfg.vocab, cfg.top_b, c->top_ids, c->top_vals, pdl, st); ++nl; }
     AcceptArgs a{};

@@ -79,11 +79,12 @@ struct Partials {
   int ws_rows;       // token rows per scratch tile
 };
 // For rows with v in [v0, v1): if `pending` has units, first h[r] += the partial tiles of a residual GEMM;
-// then x[r] = h[r] * g as a (hi, lo) bf16 pair and ss[r][w] = sum of squares of the 128 columns of warp w.
+// then x[r] = h[r] * g as `planes` bf16 planes (hi, lo or hi, mid, lo) and ss[r][w] = sum of squares of the
+// 128 columns of warp w.
 // The 1 / sqrt(mean(h^2) + eps) of RMSNorm is applied by the finisher of the GEMM that consumes x.
 constexpr int kNormMaxWarps = 64;   // d <= 8192
 cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Partials &pending, const bf16 *g, int d,
-                           bf16 *x, size_t x_lo_off, float *ss, bool pdl, cudaStream_t st);
+                           bf16 *x, size_t x_lo_off, int planes, float *ss, bool pdl, cudaStream_t st);
 
 // Eq. 3: h[s*Ms + T + i] = W_i h[s*Ms + anchor] + b_i
 void launch_pseudo_proj(const Rows &rw, const bf16 *pred_w, const bf16 *pred_b, int d, float *h, bool pdl, cudaStream_t st);
@@ -127,9 +128,10 @@ void launch_advance_ctx(int n_seq, const int32_t *seq_ids, int32_t *ctx_len, int
 enum GemmEpilogue { EPI_RESIDUAL = 0, EPI_QKV_ROPE = 1, EPI_SWIGLU = 2, EPI_LOGITS = 3 };
 
 struct GemmArgs {
-  const bf16 *X;    // [R][K] activations, hi plane (row-major, K contiguous)
-  size_t x_lo_off;  // elements from the hi plane to the lo plane ( = plane_rows * K )
+  const bf16 *X;    // [R][K] activations, first (hi) plane (row-major, K contiguous)
+  size_t x_lo_off;  // elements from one plane to the next ( = plane_rows * K )
   int plane_rows;   // rows per plane of X
+  int planes;       // 2: hi + lo (~16 mantissa bits), 3: hi + mid + lo (~24 bits)
   const bf16 *W;    // [N][K] weights
   int R;            // valid rows
   int *err;         // device status word (set to a non-zero code if a bounded wait gives up)

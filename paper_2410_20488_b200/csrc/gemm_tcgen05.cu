@@ -23,10 +23,11 @@
 //              starts while the predecessor drains.
 //   warp 6   : activation producer: the (hi, lo) bf16 planes of the matching k block (L2
 //              resident, own shorter ring), after waiting for the previous kernel.
-//   warp 1   : MMA issuer: tcgen05.mma kind::f16, M = 128, K = 16; the hi and lo planes sit one
-//              after the other in shared memory and are multiplied as ONE operand of N = 2 NPAD
-//              token columns (hi sums and lo sums land in neighbouring TMEM columns and are added
-//              in the epilogue); tcgen05.commit releases ring slots.
+//   warp 1   : MMA issuer: tcgen05.mma kind::f16, M = 128, K = 16; the bf16 planes of the
+//              activations (hi, lo, or hi, mid, lo) sit one after the other in shared memory and are
+//              multiplied as ONE operand of N = planes x NPAD token columns (the sums over each
+//              plane land in neighbouring TMEM columns and are added in the epilogue);
+//              tcgen05.commit releases ring slots.
 //   warps 2-5: epilogue: tcgen05.ld (lane = weight row, column = token), hi + lo, store of the
 //              partial tile; overlapped with the next segment's main loop through a second
 //              accumulator buffer.
@@ -142,19 +143,24 @@ __host__ __device__ constexpr uint32_t instr_desc(int n) {
 
 constexpr int pow2_cols(int c) { return c <= 32 ? 32 : c <= 64 ? 64 : c <= 128 ? 128 : c <= 256 ? 256 : 512; }
 
-// NPAD = token rows padded to a multiple of 8 (16 when the planes cannot be merged).
-template <int NPAD> struct TcCfg {
+// NPAD = token rows padded to a multiple of 8; P = bf16 planes of the activations (2: hi + lo,
+// 3: hi + mid + lo).  The planes of a stage sit one after the other in shared memory; when P * NPAD is
+// a legal MMA N (a multiple of 16, <= 256) they are multiplied as one operand, otherwise plane by plane.
+template <int NPAD, int P> struct TcCfg {
   static constexpr int X_PLANE = NPAD * 128;                   // bytes of one activation plane per stage
-  static constexpr int X_STAGE = 2 * X_PLANE;                  // hi plane, then lo plane
-  static constexpr bool MERGE = (2 * NPAD <= 256);             // hi and lo as one MMA operand of N = 2 NPAD
-  static constexpr int ACC_COLS = MERGE ? 2 * NPAD : NPAD;     // accumulator columns per weight tile
+  static constexpr int X_STAGE = P * X_PLANE;
+  static constexpr bool MERGE = (P * NPAD <= 256) && ((P * NPAD) % 16 == 0);
+  static constexpr int ACC_COLS = MERGE ? P * NPAD : NPAD;     // accumulator columns per weight tile
   static constexpr int NBUF = (2 * TM * ACC_COLS <= 512) ? 2 : 1;   // accumulator buffers
   static constexpr int TMEM_COLS = pow2_cols(NBUF * TM * ACC_COLS);
-  static constexpr int SW = NPAD <= 40 ? 6 : (NPAD <= 80 ? 5 : 4);  // weight ring depth (32 KB stages)
-  static constexpr int SX = NPAD <= 16 ? 4 : (NPAD <= 40 ? 3 : (NPAD <= 48 ? 4 : (NPAD <= 80 ? 3 : 2)));
+  // ring depths: as many 32 KB weight stages as fit beside two to four activation stages
+  static constexpr int SX = X_STAGE <= 8 * 1024 ? 4 : (X_STAGE <= 20 * 1024 ? 3 : 2);
+  static constexpr int SW = (227 * 1024 - 1280 - SX * X_STAGE) / W_STAGE > 6 ? 6 : (227 * 1024 - 1280 - SX * X_STAGE) / W_STAGE;
   static constexpr int RING_BYTES = SW * W_STAGE + SX * X_STAGE;
   static constexpr int SMEM = RING_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
-  static_assert(SMEM <= 227 * 1024, "shared memory budget");
+  static_assert(!MERGE || NPAD % 8 == 0, "planes must start on a swizzle atom");
+  static_assert(MERGE || NPAD % 16 == 0, "MMA N must be a multiple of 16");
+  static_assert(SW >= 3 && SMEM <= 227 * 1024, "shared memory budget");
   static_assert((2 * SW + 2 * SX + 2 * NBUF) * 8 + 8 <= 256, "barrier area");
 };
 
@@ -175,10 +181,10 @@ struct Sched {
   int l2_ahead;    // units each CTA prefetches into L2 beyond its shared-memory ring
 };
 
-template <int NPAD>
+template <int NPAD, int P>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, GemmArgs a, Sched sc) {
-  using Cfg = TcCfg<NPAD>;
+  using Cfg = TcCfg<NPAD, P>;
   constexpr int SW = Cfg::SW, SX = Cfg::SX, X_STAGE = Cfg::X_STAGE, X_PLANE = Cfg::X_PLANE, NBUF = Cfg::NBUF;
   constexpr int ACC = Cfg::ACC_COLS;
   constexpr bool MERGE = Cfg::MERGE;
@@ -269,15 +275,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const int kb = (int)((u0 + it) % KB);
         const int sl = it % SX;
         mbar_wait(empty_x + 8 * sl, ((it / SX) & 1) ^ 1, a.err, dead);
-        mbar_expect_tx(full_x + 8 * sl, 2 * xrows * 128);
+        mbar_expect_tx(full_x + 8 * sl, P * xrows * 128);
         const uint32_t dst = x_ring + sl * X_STAGE;
-        tma_load_2d(dst, &tmX, kb * BK, 0, full_x + 8 * sl, pol);
-        tma_load_2d(dst + X_PLANE, &tmX, kb * BK, a.plane_rows, full_x + 8 * sl, pol);
+#pragma unroll
+        for (int pl = 0; pl < P; ++pl)
+          tma_load_2d(dst + pl * X_PLANE, &tmX, kb * BK, pl * a.plane_rows, full_x + 8 * sl, pol);
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {             // ---- MMA issuer
-      constexpr uint32_t idesc = instr_desc(MERGE ? 2 * NPAD : NPAD);
+      constexpr uint32_t idesc = instr_desc(MERGE ? P * NPAD : NPAD);
       int it = 0, seg = 0;
       int u = u0;
       while (u < u1) {
@@ -293,14 +300,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           mbar_wait(full_x + 8 * sx, (it / SX) & 1, a.err, dead);
           tc_fence_after();
           const uint32_t wst = w_ring + sw * W_STAGE, xst = x_ring + sx * X_STAGE;
-          const uint64_t dhi = smem_desc(xst), dlo = smem_desc(xst + X_PLANE);
+          const uint64_t dx = smem_desc(xst);
 #pragma unroll
           for (int kk = 0; kk < BK / 16; ++kk) {
 #pragma unroll
             for (int t = 0; t < TM; ++t) {
               const uint64_t da = smem_desc(wst + t * W_TILE) + 2 * kk;
-              tc_mma(acc + t * ACC, da, dhi + 2 * kk, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
-              if (!MERGE) tc_mma(acc + t * ACC, da, dlo + 2 * kk, idesc, 1u);
+              tc_mma(acc + t * ACC, da, dx + 2 * kk, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+              if (!MERGE) {
+#pragma unroll
+                for (int pl = 1; pl < P; ++pl) tc_mma(acc + t * ACC, da, dx + (pl * X_PLANE >> 4) + 2 * kk, idesc, 1u);
+              }
             }
           }
           tc_commit(empty_w + 8 * sw);   // the slots are free once these MMAs have read them
@@ -330,15 +340,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         float r0[16], r1[16];
         tc_ld16(tacc + c0, r0);
         tc_ld16(tacc + ACC + c0, r1);
-        if (MERGE) {             // columns NPAD.. hold the sums over the lo plane
-          float l0[16], l1[16];
-          tc_ld16(tacc + NPAD + c0, l0);
-          tc_ld16(tacc + ACC + NPAD + c0, l1);
-          tc_ld_wait();
+        tc_ld_wait();
+        if (MERGE) {             // columns pl * NPAD .. hold the sums over plane pl
 #pragma unroll
-          for (int j = 0; j < 16; ++j) { r0[j] += l0[j]; r1[j] += l1[j]; }
-        } else {
-          tc_ld_wait();
+          for (int pl = 1; pl < P; ++pl) {
+            float l0[16], l1[16];
+            tc_ld16(tacc + pl * NPAD + c0, l0);
+            tc_ld16(tacc + ACC + pl * NPAD + c0, l1);
+            tc_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) { r0[j] += l0[j]; r1[j] += l1[j]; }
+          }
         }
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
@@ -428,12 +440,12 @@ int sm_count() {
   return n;
 }
 
-template <int NPAD>
+template <int NPAD, int P>
 cudaError_t launch_np(const GemmArgs &a, const Sched &sc, cudaStream_t st) {
-  using Cfg = TcCfg<NPAD>;
+  using Cfg = TcCfg<NPAD, P>;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<NPAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<NPAD, P>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
     if (e != cudaSuccess) return e;
     configured = true;
   }
@@ -441,7 +453,7 @@ cudaError_t launch_np(const GemmArgs &a, const Sched &sc, cudaStream_t st) {
   CUtensorMap tmW, tmX;
   if (!make_map(&tmW, a.W, (uint64_t)a.N, (uint64_t)a.K, BM, sc.mode == ROWS_ROTARY ? (uint32_t)sc.half : 0u))
     return cudaErrorInvalidValue;
-  if (!make_map(&tmX, a.X, (uint64_t)a.plane_rows + a.R, (uint64_t)a.K, (uint32_t)xrows, 0)) return cudaErrorInvalidValue;
+  if (!make_map(&tmX, a.X, (uint64_t)(P - 1) * a.plane_rows + a.R, (uint64_t)a.K, (uint32_t)xrows, 0)) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)sc.sk.G);
   cfg.blockDim = dim3(kThreads);
@@ -452,15 +464,21 @@ cudaError_t launch_np(const GemmArgs &a, const Sched &sc, cudaStream_t st) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = sc.pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<NPAD>, tmW, tmX, a, sc);
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<NPAD, P>, tmW, tmX, a, sc);
 }
 
 cudaError_t launch_rows(const GemmArgs &a, const Sched &sc, cudaStream_t st) {
-  if (a.R <= 16) return launch_np<16>(a, sc, st);
-  if (a.R <= 40) return launch_np<40>(a, sc, st);
-  if (a.R <= 48) return launch_np<48>(a, sc, st);
-  if (a.R <= 80) return launch_np<80>(a, sc, st);
-  return launch_np<144>(a, sc, st);
+  if (a.planes == 3) {   // N = 3 NPAD must be a multiple of 16
+    if (a.R <= 16) return launch_np<16, 3>(a, sc, st);
+    if (a.R <= 48) return launch_np<48, 3>(a, sc, st);
+    if (a.R <= 80) return launch_np<80, 3>(a, sc, st);
+    return launch_np<144, 3>(a, sc, st);
+  }
+  if (a.R <= 16) return launch_np<16, 2>(a, sc, st);
+  if (a.R <= 40) return launch_np<40, 2>(a, sc, st);
+  if (a.R <= 48) return launch_np<48, 2>(a, sc, st);
+  if (a.R <= 80) return launch_np<80, 2>(a, sc, st);
+  return launch_np<144, 2>(a, sc, st);
 }
 
 Sched make_sched(GemmEpilogue epi, const GemmArgs &a, bool pdl) {

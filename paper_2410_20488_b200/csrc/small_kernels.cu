@@ -97,7 +97,7 @@ void launch_embed(const Rows &rw, const int32_t *d_tokens, const bf16 *embed, in
 // ---------------------------------------------------------------------------
 // Residual update + first half of RMSNorm, as a flat elementwise kernel.
 //   h[r] += the partial tiles a residual GEMM left in scratch (fixed order: ascending CTA index)
-//   x[r]  = h[r] * g as a (hi, lo) bf16 pair -- NOT yet divided by the row's RMS
+//   x[r]  = h[r] * g as bf16 planes (hi, lo; plus a third plane on request) -- NOT yet divided by the row's RMS
 //   ss[r][w] = sum of h[r][c]^2 over the 128 columns of warp w
 // The division by sqrt(mean(h^2) + eps) commutes with the GEMM that consumes x, so that GEMM's
 // finisher applies it to the fp32 sums (it adds the ss[r][*] in a fixed order).  This kernel then
@@ -108,7 +108,7 @@ constexpr int kNormThreads = 256;
 
 __global__ void __launch_bounds__(kNormThreads)
 rmsnorm_kernel(Rows rw, int v0, int nv, float *h, Partials pend, const bf16 *__restrict__ g, int d, bf16 *x,
-               size_t x_lo_off, float *ss, int pdl) {
+               size_t x_lo_off, int planes, float *ss, int pdl) {
   if (pdl) { griddep_launch(); griddep_wait(); }
   const int nvec = d >> 2;                                  // float4 per row, a multiple of 32
   const unsigned t = blockIdx.x * kNormThreads + threadIdx.x;
@@ -155,15 +155,23 @@ rmsnorm_kernel(Rows rw, int v0, int nv, float *h, Partials pend, const bf16 *__r
   lo2.x = *reinterpret_cast<const uint32_t *>(&l01); lo2.y = *reinterpret_cast<const uint32_t *>(&l23);
   *reinterpret_cast<uint2 *>(x + (size_t)r * d + 4 * idx) = hi2;
   *reinterpret_cast<uint2 *>(x + x_lo_off + (size_t)r * d + 4 * idx) = lo2;
+  if (planes == 3) {   // third plane: what hi + mid still miss (the K/V projections need fp32-grade inputs)
+    const float2 m01 = __bfloat1622float2(l01), m23 = __bfloat1622float2(l23);
+    const __nv_bfloat162 t01 = __floats2bfloat162_rn(y0 - f01.x - m01.x, y1 - f01.y - m01.y);
+    const __nv_bfloat162 t23 = __floats2bfloat162_rn(y2 - f23.x - m23.x, y3 - f23.y - m23.y);
+    uint2 t2;
+    t2.x = *reinterpret_cast<const uint32_t *>(&t01); t2.y = *reinterpret_cast<const uint32_t *>(&t23);
+    *reinterpret_cast<uint2 *>(x + 2 * x_lo_off + (size_t)r * d + 4 * idx) = t2;
+  }
 }
 
 cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Partials &pending, const bf16 *g, int d,
-                           bf16 *x, size_t x_lo_off, float *ss, bool pdl, cudaStream_t st) {
+                           bf16 *x, size_t x_lo_off, int planes, float *ss, bool pdl, cudaStream_t st) {
   const int nv = v1 - v0;
   if (nv <= 0) return cudaSuccess;
   const int threads = rw.n_seq * nv * (d >> 2);
   return launch_k(rmsnorm_kernel, dim3((threads + kNormThreads - 1) / kNormThreads), dim3(kNormThreads), 0, st, pdl, rw,
-                  v0, nv, h, pending, g, d, x, x_lo_off, ss, pdl ? 1 : 0);
+                  v0, nv, h, pending, g, d, x, x_lo_off, planes, ss, pdl ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------
