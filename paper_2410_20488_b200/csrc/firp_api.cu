@@ -56,7 +56,8 @@ struct firp_ctx {
   std::vector<const void *> wqkv, wo, wgu, wd, g_attn, g_mlp;
   // device buffers (carved from the caller's workspace)
   bf16 *kv = nullptr;
-  float *h = nullptr, *gemm_ws = nullptr, *ss = nullptr, *logits = nullptr, *top_vals = nullptr;
+  float *h = nullptr, *gemm_ws = nullptr, *ss = nullptr, *logits = nullptr, *top_vals = nullptr, *cand_vals = nullptr;
+  int32_t *cand_ids = nullptr;
   bf16 *x = nullptr, *q = nullptr, *o = nullptr, *y = nullptr;
   int32_t *ctx_len = nullptr, *seq_ids = nullptr, *parents = nullptr, *next_parents = nullptr, *chain = nullptr;
   int32_t *top_ids = nullptr, *path = nullptr, *n_acc = nullptr, *accepted = nullptr, *next_tokens = nullptr;
@@ -86,6 +87,8 @@ struct firp_ctx {
     logits = c.take<float>(R * cfg.vocab);
     top_ids = c.take<int32_t>(R * kMaxTopB);
     top_vals = c.take<float>(R * kMaxTopB);
+    cand_ids = c.take<int32_t>(R * (size_t)topb_segments(cfg.vocab) * kMaxTopB);
+    cand_vals = c.take<float>(R * (size_t)topb_segments(cfg.vocab) * kMaxTopB);
     meta.depth = c.take<int32_t>(R);
     meta.pos = c.take<int32_t>(R);
     meta.mask = c.take<uint32_t>(R * kMaskWords);
@@ -290,7 +293,8 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       FIRP_TIMED(KC_LOGITS_FINISH);
       FIRP_CUDA(c, launch_gemm_finish(EPI_LOGITS, p, g, pdl, st)); ++nl; }
     { FIRP_TIMED(KC_TOPB);
-      launch_topb(ra.logits_dst, rw.R, cfg.vocab, cfg.top_b, c->top_ids, c->top_vals, pdl, st); ++nl; }
+      launch_topb(ra.logits_dst, rw.R, cfg.vocab, cfg.top_b, c->cand_ids, c->cand_vals, c->top_ids, c->top_vals, pdl, st);
+      nl += 2; }
     AcceptArgs a{};
     a.tokens = ra.d_tokens; a.parents = c->parents; a.next_parents = c->next_parents;
     a.top_ids = c->top_ids; a.top_vals = c->top_vals; a.T_next = ra.T_next; a.B = cfg.top_b; a.S = c->S;

@@ -90,7 +90,11 @@ cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Parti
 void launch_pseudo_proj(const Rows &rw, const bf16 *pred_w, const bf16 *pred_b, int d, float *h, bool pdl, cudaStream_t st);
 
 // top-B of every row of logits by (value desc, id asc)
-void launch_topb(const float *logits, int R, int V, int B, int32_t *ids, float *vals, bool pdl, cudaStream_t st);
+// Two passes: per 2048-logit segment candidates (scratch cand_*: [R][topb_segments(V)][B]), then the row's top-B.
+constexpr int kTopSeg = 2048;
+int topb_segments(int V);
+void launch_topb(const float *logits, int R, int V, int B, int32_t *cand_ids, float *cand_vals, int32_t *ids, float *vals,
+                 bool pdl, cudaStream_t st);
 
 struct AcceptArgs {
   const int32_t *tokens;        // [n_seq][T]

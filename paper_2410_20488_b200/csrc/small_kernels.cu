@@ -223,27 +223,37 @@ void launch_pseudo_proj(const Rows &rw, const bf16 *pred_w, const bf16 *pred_b, 
 }
 
 // ---------------------------------------------------------------------------
-// Top-B of each logits row by (value descending, id ascending).
+// Top-B of each logits row by (value descending, id ascending), in two passes of one kernel:
+//   pass 1  every (row, segment of kTopSeg logits) leaves its B best as candidates in scratch
+//   pass 2  every row picks its B best among its candidates
+// Selecting by the same total order in both passes gives exactly the top-B of the whole row.
 // ---------------------------------------------------------------------------
 constexpr int kTopThreads = 256;
 
 __device__ __forceinline__ bool better(float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia < ib); }
 
+// grid = (segments, rows).  Element t of the segment has value vals[row * row_stride + seg * seg_len + t] and
+// id ids[same index] (ids == NULL: its position in the row).  Output slot (row * segments + seg) gets B pairs;
+// a segment with fewer than B elements pads with (-inf, INT_MAX).
 __global__ void __launch_bounds__(kTopThreads)
-topb_kernel(const float *logits, int V, int B, int32_t *ids, float *vals, int pdl) {
+topb_kernel(const float *vals, const int32_t *ids, int row_stride, int seg_len, int row_len, int B, int32_t *out_ids,
+            float *out_vals, int pdl) {
   __shared__ float sval[32];
   __shared__ int sid[32];
   __shared__ int swin;
   if (pdl) { griddep_launch(); griddep_wait(); }
-  const float *row = logits + (size_t)blockIdx.x * V;
+  const int seg = blockIdx.x, r = blockIdx.y;
+  const size_t base = (size_t)r * row_stride + (size_t)seg * seg_len;
+  const int n = min(seg_len, row_len - seg * seg_len);
   float lv[kMaxTopB];
   int li[kMaxTopB];
 #pragma unroll
   for (int j = 0; j < kMaxTopB; ++j) { lv[j] = -INFINITY; li[j] = 0x7fffffff; }
-  for (int t = threadIdx.x; t < V; t += kTopThreads) {
-    const float v = row[t];
-    if (better(v, t, lv[kMaxTopB - 1], li[kMaxTopB - 1])) {
-      lv[kMaxTopB - 1] = v; li[kMaxTopB - 1] = t;
+  for (int t = threadIdx.x; t < n; t += kTopThreads) {
+    const float v = vals[base + t];
+    const int id = ids ? ids[base + t] : seg * seg_len + t;
+    if (better(v, id, lv[kMaxTopB - 1], li[kMaxTopB - 1])) {
+      lv[kMaxTopB - 1] = v; li[kMaxTopB - 1] = id;
 #pragma unroll
       for (int j = kMaxTopB - 1; j > 0; --j) {
         if (better(lv[j], li[j], lv[j - 1], li[j - 1])) {
@@ -253,6 +263,7 @@ topb_kernel(const float *logits, int V, int B, int32_t *ids, float *vals, int pd
       }
     }
   }
+  const size_t o = ((size_t)r * gridDim.x + seg) * B;
   int head = 0;
   for (int b = 0; b < B; ++b) {
     float cv = -INFINITY; int ci = 0x7fffffff;
@@ -260,9 +271,9 @@ topb_kernel(const float *logits, int V, int B, int32_t *ids, float *vals, int pd
     for (int j = 0; j < kMaxTopB; ++j) if (j == head) { cv = lv[j]; ci = li[j]; }
     float bv = cv; int bi = ci;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    for (int s = 16; s > 0; s >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, s);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, s);
       if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
     }
     if ((threadIdx.x & 31) == 0) { sval[threadIdx.x >> 5] = bv; sid[threadIdx.x >> 5] = bi; }
@@ -271,25 +282,32 @@ topb_kernel(const float *logits, int V, int B, int32_t *ids, float *vals, int pd
       float v = (threadIdx.x < kTopThreads / 32) ? sval[threadIdx.x] : -INFINITY;
       int i = (threadIdx.x < kTopThreads / 32) ? sid[threadIdx.x] : 0x7fffffff;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, v, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, i, o);
+      for (int s = 16; s > 0; s >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, v, s);
+        const int oi = __shfl_xor_sync(0xffffffffu, i, s);
         if (better(ov, oi, v, i)) { v = ov; i = oi; }
       }
       if (threadIdx.x == 0) {
         swin = i;
-        ids[(size_t)blockIdx.x * B + b] = i;
-        vals[(size_t)blockIdx.x * B + b] = v;
+        out_ids[o + b] = i;
+        out_vals[o + b] = v;
       }
     }
     __syncthreads();
-    if (ci == swin && head < kMaxTopB) ++head;   // token ids are unique, so exactly one thread advances
+    if (ci == swin && ci != 0x7fffffff && head < kMaxTopB) ++head;   // ids are unique: exactly one thread advances
     __syncthreads();
   }
 }
 
-void launch_topb(const float *logits, int R, int V, int B, int32_t *ids, float *vals, bool pdl, cudaStream_t st) {
-  launch_k(topb_kernel, dim3(R), dim3(kTopThreads), 0, st, pdl, logits, V, B, ids, vals, pdl ? 1 : 0);
+int topb_segments(int V) { return (V + kTopSeg - 1) / kTopSeg; }
+
+void launch_topb(const float *logits, int R, int V, int B, int32_t *cand_ids, float *cand_vals, int32_t *ids, float *vals,
+                 bool pdl, cudaStream_t st) {
+  const int segs = topb_segments(V);
+  launch_k(topb_kernel, dim3(segs, R), dim3(kTopThreads), 0, st, pdl, logits, (const int32_t *)nullptr, V, kTopSeg, V, B,
+           cand_ids, cand_vals, pdl ? 1 : 0);
+  launch_k(topb_kernel, dim3(1, R), dim3(kTopThreads), 0, st, pdl, (const float *)cand_vals, (const int32_t *)cand_ids,
+           segs * B, segs * B, segs * B, B, ids, vals, pdl ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------
