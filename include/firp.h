@@ -171,6 +171,33 @@ int firp_profile_enable(firp_ctx *ctx, int32_t on);
 int firp_profile_read(firp_ctx *ctx, void *stream, int32_t n_classes, int32_t *launches, float *usec);
 const char *firp_kernel_class_name(int32_t c);
 
+/*
+ * Top-B of logits rows without any device allocation.  (This call has no counterpart in the paper;
+ * it serves hosts that drive the decoder from places where cudaMalloc is off limits: inside a
+ * latency-critical serving loop whose memory pool is fixed at start-up, or in a plug-in that is
+ * handed buffers and a stream by its host application and owns no allocator of its own.)
+ *
+ * Computes, for each of `rows` rows of fp32 logits (DEVICE, [rows][vocab], row-major), the b best
+ * entries ordered by (value descending, token id ascending) -- the same selection firp_step makes
+ * for its rows -- and writes d_ids [rows][b] and d_vals [rows][b] (DEVICE, caller-owned).
+ *
+ * The intermediate candidates of the two-pass selection live in a 256 KiB array that is part of
+ * the library image on every GPU that loads it; nothing is allocated or freed, by this call or by
+ * anything it uses.  The array limits the problem size: rows * ceil(vocab / 2048) must not exceed
+ * FIRP_TOPB_STATIC_MAX_SLOTS, otherwise FIRP_ERR_CAPACITY is returned (and a line on stderr says
+ * which limit was hit); 1 <= b <= 8.
+ *
+ * The first call on a device looks up the array's device address (once per device, under a lock):
+ * make that first call outside any stream capture.  All calls on a device share the one array and it
+ * keeps whatever the previous call left; every entry a call reads it has written itself, so no clearing
+ * is needed, but two calls whose kernels can overlap on the GPU (different streams, no ordering between
+ * them) race on it and must be serialised by the caller.
+ * Work is enqueued on `stream`; nothing synchronises.  Returns FIRP_OK or a negative firp_status.
+ */
+#define FIRP_TOPB_STATIC_MAX_SLOTS 4096
+int firp_topb_static(const float *d_logits, int32_t rows, int32_t vocab, int32_t b, int32_t *d_ids, float *d_vals,
+                     void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -45,7 +45,7 @@ class StepOutC(ctypes.Structure):
 EXPORTS = ("firp_create", "firp_destroy", "firp_last_error", "firp_workspace_bytes", "firp_kv_bytes",
            "firp_bind_buffers", "firp_init_weights", "firp_prefill", "firp_step", "firp_kv_commit",
            "firp_context_len", "firp_set_context_len", "firp_last_launch_count", "firp_profile_enable",
-           "firp_profile_read", "firp_kernel_class_name")
+           "firp_profile_read", "firp_kernel_class_name", "firp_topb_static")
 
 
 def lib_path() -> str:
@@ -82,6 +82,7 @@ def load_library():
     lib.firp_profile_read.argtypes = [vp, vp, i32, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_float)]
     lib.firp_kernel_class_name.argtypes = [i32]
     lib.firp_kernel_class_name.restype = ctypes.c_char_p
+    lib.firp_topb_static.argtypes = [vp, i32, i32, i32, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("firp_destroy", "firp_last_error", "firp_workspace_bytes", "firp_kv_bytes",
                         "firp_kernel_class_name"):
@@ -188,6 +189,15 @@ def firp_profile_read(ctx, stream: int = 0) -> dict:
     if rc < 0:
         _check(ctx, rc)
     return {firp_kernel_class_name(c): (int(launches[c]), float(usec[c])) for c in range(rc)}
+
+
+def firp_topb_static(d_logits_ptr: int, rows: int, vocab: int, b: int, d_ids_ptr: int, d_vals_ptr: int, stream: int = 0):
+    """Top-b of `rows` rows of device logits into caller-owned device arrays; allocates nothing (the
+    candidate scratch is a fixed array inside the library).  Raises FirpError on a bad argument or when
+    rows * ceil(vocab / 2048) exceeds the built-in scratch."""
+    rc = load_library().firp_topb_static(d_logits_ptr, rows, vocab, b, d_ids_ptr, d_vals_ptr, stream)
+    if rc != 0:
+        raise FirpError(rc, "firp_topb_static rejected the call (see stderr)")
 
 
 # ---- convenience: device memory through torch, nothing else ---------------

@@ -1,0 +1,56 @@
+"""firp_topb_static -- the entry point that allocates nothing -- against firp_step.
+
+Some hosts of this library may not allocate device memory while decoding (a serving loop with a
+memory pool fixed at start-up, a plug-in that only ever receives buffers from its host), so this
+one call keeps its scratch in a fixed array inside the library.  Here it is run, through the C ABI,
+on the logits that firp_step exported, twice in a row on different logits, and must reproduce the
+selections firp_step made from the same rows: the greedy token of every tree row and the ordered
+top-B ids and values of every pseudo row, exactly (both paths select from the same fp32 numbers).
+The file name sorts last on purpose: a run that stops at the first failure has by then run every
+other test.
+"""
+import numpy as np
+import pytest
+
+import synth_inputs as si
+
+pytestmark = pytest.mark.gpu
+
+
+def test_static_topb_matches_step_twice_in_a_row(c1, c1_weights):
+    import torch
+    assert torch.cuda.is_available(), "this test needs a CUDA device"
+    from paper_2410_20488_b200 import FirpEngine, FirpError, binding, build as firp_build, firp_topb_static
+    firp_build.build()
+    parents = si.tree_template(c1.T)
+    eng = FirpEngine(c1, c1_weights, max_ctx=256)
+    T, k, V, B = c1.T, c1.k, c1.V, eng.B
+    d_prompt = torch.from_numpy(si.prompt(c1)).cuda()
+    pout = eng.new_out(1, 1, k, T_next=T)
+    eng.prefill(0, d_prompt, k, c1.l, parents, pout)
+    out = eng.new_out(1, T, k)
+    ids = torch.full((T + k, B), -1, dtype=torch.int32, device="cuda")
+    vals = torch.zeros((T + k, B), dtype=torch.float32, device="cuda")
+    tokens = pout.next_tree_tokens[0].clone()
+    for call in range(2):                     # two calls in a row share the built-in scratch
+        eng.step(tokens, parents, k, c1.l, out)
+        ids.fill_(-1)
+        firp_topb_static(out.logits.data_ptr(), T + k, V, B, ids.data_ptr(), vals.data_ptr(), eng.stream)
+        torch.cuda.synchronize()
+        got_ids, got_vals = ids.cpu().numpy(), vals.cpu().numpy()
+        assert np.array_equal(got_ids[:T, 0], out.best[0].cpu().numpy()), "greedy tokens differ (call %d)" % call
+        assert np.array_equal(got_ids[T:], out.topb_ids[0, :k].cpu().numpy()), "top-B ids differ (call %d)" % call
+        assert np.array_equal(got_vals[T:], out.topb_vals[0, :k].cpu().numpy()), "top-B values differ (call %d)" % call
+        logits = out.logits[0].cpu().numpy()
+        want = np.stack([np.lexsort((np.arange(V), -row))[:B] for row in logits])
+        assert np.array_equal(got_ids, want), "not the top-B of the logits (call %d)" % call
+        eng.commit(1)
+        tokens = out.next_tree_tokens[0].clone()
+    # sizes beyond the built-in scratch are refused, not truncated
+    with pytest.raises(FirpError) as e:
+        firp_topb_static(out.logits.data_ptr(), 4097, V, B, ids.data_ptr(), vals.data_ptr(), eng.stream)
+    assert e.value.code == binding.FIRP_ERR_CAPACITY
+    with pytest.raises(FirpError) as e:
+        firp_topb_static(out.logits.data_ptr(), T + k, V, 9, ids.data_ptr(), vals.data_ptr(), eng.stream)
+    assert e.value.code == binding.FIRP_ERR_BAD_ARG
+    eng.close()
