@@ -60,8 +60,9 @@ class Stats:
                     max_abs=self.max_abs, max_rel=self.max_rel, emitted=self.emitted)
 
 
-def compare_step(shape, parents, tokens, k, g, ref, stats: Stats, tp=None):
+def compare_step(shape, parents, tokens, k, g, ref, stats: Stats, tp=None, abs_tol=None):
     """g: dict of numpy arrays from the CUDA path for ONE sequence; ref: oracle.step() output."""
+    abs_tol = ABS_TOL if abs_tol is None else abs_tol
     T, V = len(parents), shape.V
     M = T + k
     tp = tp or oracle.tree_prep(parents, k, 0)
@@ -74,7 +75,7 @@ def compare_step(shape, parents, tokens, k, g, ref, stats: Stats, tp=None):
     row_rel = row_abs / np.abs(ref["logits"]).max(axis=1)
     stats.max_abs = max(stats.max_abs, float(row_abs.max()))
     stats.max_rel = max(stats.max_rel, float(row_rel.max()))
-    assert row_abs.max() <= ABS_TOL, "logits max-abs %.4g > %.3g (row %d)" % (row_abs.max(), ABS_TOL, row_abs.argmax())
+    assert row_abs.max() <= abs_tol, "logits max-abs %.4g > %.3g (row %d)" % (row_abs.max(), abs_tol, row_abs.argmax())
     assert row_rel.max() <= REL_TOL, "logits rel %.4g > %.3g" % (row_rel.max(), REL_TOL)
     # (iii) greedy tokens where the oracle margin is clear
     part = np.partition(ref["logits"][:T], V - 2, axis=1)
@@ -112,8 +113,8 @@ def compare_step(shape, parents, tokens, k, g, ref, stats: Stats, tp=None):
                 if firm:
                     assert g["topb_ids"][i, b] == order[b], "top-B id mismatch at a firm position"
                 gid = int(g["topb_ids"][i, b])
-                assert abs(float(g["topb_vals"][i, b]) - float(row[gid])) <= ABS_TOL, "top-B value off"
-                assert float(g["topb_vals"][i, b]) >= float(vals[B - 1]) - 2 * ABS_TOL, "top-B entry too small"
+                assert abs(float(g["topb_vals"][i, b]) - float(row[gid])) <= abs_tol, "top-B value off"
+                assert float(g["topb_vals"][i, b]) >= float(vals[B - 1]) - 2 * abs_tol, "top-B entry too small"
             gv, gi = g["topb_vals"][i], g["topb_ids"][i]
             assert all(gv[b] > gv[b + 1] or (gv[b] == gv[b + 1] and gi[b] < gi[b + 1]) for b in range(B - 1)), \
                 "top-B not ordered by (value desc, id asc)"
@@ -157,8 +158,9 @@ def check_cache(engine, orc, seq, slots, layers, tol=2e-2):
 
 
 def lockstep_run(engine, orc, shape, parents, prompt, steps, forced=False, k=None, l=None, check_cache_rows=True,
-                 compare_every=1, seq=0):
+                 compare_every=1, seq=0, abs_tol=None):
     """Prefill both sides, then `steps` lock-step steps.  Returns a Stats."""
+    abs_tol = ABS_TOL if abs_tol is None else abs_tol
     import torch
     k = shape.k if k is None else k
     l = shape.l if l is None else l
@@ -178,7 +180,7 @@ def lockstep_run(engine, orc, shape, parents, prompt, steps, forced=False, k=Non
     torch.cuda.synchronize()
     plog = pout.logits[0].cpu().numpy()
     dd = np.abs(plog - ref["logits"]).max()
-    assert dd <= ABS_TOL, "prefill logits differ by %.4g" % dd
+    assert dd <= abs_tol, "prefill logits differ by %.4g" % dd
     part = np.partition(ref["logits"][0], shape.V - 2)
     if part[-1] - part[-2] > MARGIN:
         assert int(pout.accepted_tokens[0, 0].item()) == ref["root"], "prefill root token differs"
@@ -201,7 +203,7 @@ def lockstep_run(engine, orc, shape, parents, prompt, steps, forced=False, k=Non
         ref = orc.step(tokens, parents, k, l, seq=seq)
         if step % compare_every == 0 or step == steps - 1:
             g = gpu_outputs(out, 0, T, k)
-            compare_step(shape, parents, tokens, k, g, ref, stats, tp)
+            compare_step(shape, parents, tokens, k, g, ref, stats, tp, abs_tol)
         if forced:
             assert ref["n_accepted"] == D + 1, "forced-accept step accepted %d of %d" % (ref["n_accepted"] - 1, D)
         n0 = orc.context_len(seq)
@@ -214,4 +216,42 @@ def lockstep_run(engine, orc, shape, parents, prompt, steps, forced=False, k=Non
         emitted += ref["accepted"].tolist()
         tokens = ref["next_tokens"].copy()
     stats.emitted = len(emitted)
+    return stats
+
+
+def lockstep_run_batch(engine, orc, shape, parents, prompts, steps, k=None, l=None, abs_tol=None):
+    """Several sequences with their own prompts (context lengths) and trees, stepped together by ONE
+    firp_step call per step; every sequence is compared with its own oracle step, and both sides commit
+    the oracle's paths.  Returns a Stats over all sequences."""
+    import torch
+    k = shape.k if k is None else k
+    l = shape.l if l is None else l
+    abs_tol = ABS_TOL if abs_tol is None else abs_tol
+    T, n_seq = len(parents), len(prompts)
+    tp = oracle.tree_prep(parents, k, 0)
+    dev = engine.device
+    stats = Stats()
+    tokens = np.zeros((n_seq, T), np.int32)
+    for s_i, prompt in enumerate(prompts):
+        pout = engine.new_out(1, 1, k, T_next=T)
+        engine.prefill(s_i, torch.from_numpy(np.ascontiguousarray(prompt, np.int32)).to(dev), k, l, parents, pout)
+        ref = orc.prefill(prompt, k, l, parents, seq=s_i)
+        torch.cuda.synchronize()
+        dd = np.abs(pout.logits[0].cpu().numpy() - ref["logits"]).max()
+        assert dd <= abs_tol, "prefill logits of sequence %d differ by %.4g" % (s_i, dd)
+        assert engine.context_len(s_i) == orc.context_len(s_i) == len(prompt)
+        tokens[s_i] = ref["next_tokens"]
+    out = engine.new_out(n_seq, T, k)
+    for step in range(steps):
+        d_tokens = torch.from_numpy(np.ascontiguousarray(tokens)).to(dev)
+        engine.step(d_tokens, parents, k, l, out, seq_ids=list(range(n_seq)), n_seq=n_seq)
+        refs = [orc.step(tokens[s_i], parents, k, l, seq=s_i) for s_i in range(n_seq)]
+        for s_i in range(n_seq):
+            compare_step(shape, parents, tokens[s_i], k, gpu_outputs(out, s_i, T, k), refs[s_i], stats, tp, abs_tol)
+        engine.commit(n_seq, seq_ids=list(range(n_seq)), path=[r["path"] for r in refs])
+        for s_i in range(n_seq):
+            orc.commit(refs[s_i]["path"], seq=s_i)
+            assert engine.context_len(s_i) == orc.context_len(s_i)
+            stats.emitted += len(refs[s_i]["accepted"])
+            tokens[s_i] = refs[s_i]["next_tokens"]
     return stats
