@@ -138,6 +138,20 @@ def kernel_times(eng, shape, parents, tokens, out, steps, n_ctx, peak_gbs, peak_
     return dict(roofline=roofline, kernels=kernels, profiled_steps=steps, sum_kernel_ms_per_step=total / steps / 1e3)
 
 
+def aggregate_over_ranks(ms: float, units: float, device=None):
+    """Whole-job figures of N independent replicas: the slowest rank's device time and the units of all
+    ranks.  With one process (no process group) the inputs come back unchanged."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms), float(units)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    u = torch.tensor([units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
 class ClockSampler:
     FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -346,18 +360,9 @@ def main():
                    d2h=int((h_acc.numel() + 1 + h_next.numel()) * 4))
 
     # ---- aggregate over ranks: max time, summed units ----------------------------------------
-    def agg(ms, units):
-        if world == 1:
-            return ms, units
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        u = torch.tensor([units], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.all_reduce(u, op=dist.ReduceOp.SUM)
-        return float(t.item()), float(u.item())
-
-    ms_max, units = agg(ms_total, emitted)
+    ms_max, units = aggregate_over_ranks(ms_total, emitted, dev)
     if e2e:
-        e_ms_max, e_units = agg(e2e["ms"], e2e["emitted"])
+        e_ms_max, e_units = aggregate_over_ranks(e2e["ms"], e2e["emitted"], dev)
 
     if rank != 0:
         return
