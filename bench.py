@@ -87,7 +87,8 @@ def class_bytes(shape, n_ctx: float) -> dict:
 # c2 shape, from the ncu capture summarised under profiles/; valid only for the kernel sources whose
 # digest is recorded with it (a changed kernel reports traffic = null until it is captured again).
 NCU_TRAFFIC = {
-    "c2-llama2-7b": dict(digest="", per_launch={}),
+    "c2-llama2-7b": dict(digest="67fb5953f2b07334", per_launch={"gemm_gate_up": 197948160, "gemm_qkv": 108428032,
+                                                             "gemm_o": 34111488, "gemm_down": 96498688}),
 }
 
 
@@ -309,10 +310,10 @@ def main():
         launches += eng.launches()
         return o
 
-    for i in range(W):
+    sampler = ClockSampler(local_rank) if rank == 0 else None    # nvidia-smi takes a while to start: the warm-up
+    for i in range(W):                                           # steps (same load) are sampled as well
         tokens = one_step(i, tokens).next_tree_tokens[0]
     barrier()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     launches = 0
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     acc_counts = torch.zeros(K, dtype=torch.int32, device=dev)
