@@ -15,6 +15,8 @@
 // the cache's own storage format.
 #include <cooperative_groups.h>
 
+#include <cstdlib>
+
 #include "firp_kernels.cuh"
 #include "launch_util.cuh"
 
@@ -77,24 +79,7 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a, int pdl
   const int qrows_total = a.rows_active * G;
   const int qblocks = (qrows_total + kQRows - 1) / kQRows;
   const int s = blockIdx.z / qblocks, qb = blockIdx.z % qblocks;
-  const int slot = a.seq_ids[s];
-  const int n = a.ctx_len[slot];
-  const int kv_len = min(n + a.rows_active, a.max_ctx);
-  const int tiles_total = (kv_len + KT - 1) / KT;
-  const int t0 = split * tiles_total / a.splits, t1 = (split + 1) * tiles_total / a.splits;   // balanced ranges
-
-  const bf16 *kbase = a.kcache + (size_t)slot * a.seq_stride + (size_t)kvh * DH;
-  const bf16 *vbase = kbase + a.kv_stride;
-  const size_t pos_stride = (size_t)a.Hkv * DH;
-
-  // query rows of this block: qr -> (tree row v = qr / G, head = kvh * G + qr % G)
-  for (int i = tid; i < kQRows; i += kThreads) {
-    const int qr = qb * kQRows + i;
-    int r = -1;
-    if (qr < qrows_total) r = s * a.rw.Ms + qr / G;
-    s_row[i] = r;
-    for (int w = 0; w < kMaskWords; ++w) s_mask[i][w] = (r >= 0) ? a.mask[(size_t)r * kMaskWords + w] : 0u;
-  }
+  // the query tile does not depend on the context length: its loads go out first
   for (int ch = tid; ch < kQRows * CH; ch += kThreads) {
     const int i = ch / CH, c = ch % CH;
     const int qr = qb * kQRows + i;
@@ -103,6 +88,16 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a, int pdl
     cp_async_16(smem_u32(sQ + tile_off<DH>(i, c)), src, valid);
     cp_async_16(smem_u32(sQ + Q_BYTES + tile_off<DH>(i, c)), valid ? src + a.q_lo_off : a.q, valid);
   }
+  const int slot = a.seq_ids[s];
+  const int n = a.ctx_len[slot];
+  const int kv_len = min(n + a.rows_active, a.max_ctx);
+  const int tiles_total = (kv_len + KT - 1) / KT;
+  // balanced ranges; a remainder goes to the first splits, the last one owns the (slower) masked tiles
+  const int t0 = (split * tiles_total + a.splits - 1) / a.splits, t1 = ((split + 1) * tiles_total + a.splits - 1) / a.splits;
+
+  const bf16 *kbase = a.kcache + (size_t)slot * a.seq_stride + (size_t)kvh * DH;
+  const bf16 *vbase = kbase + a.kv_stride;
+  const size_t pos_stride = (size_t)a.Hkv * DH;
   auto load_kv = [&](int buf, int t) {
     const int p0 = t * KT;
     for (int ch = tid; ch < KT * CH; ch += kThreads) {
@@ -115,6 +110,14 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a, int pdl
   };
   if (t0 < t1) load_kv(0, t0);
   cp_async_commit();
+  // query rows of this block: qr -> (tree row v = qr / G, head = kvh * G + qr % G), and their visibility words
+  for (int i = tid; i < kQRows; i += kThreads) {
+    const int qr = qb * kQRows + i;
+    int r = -1;
+    if (qr < qrows_total) r = s * a.rw.Ms + qr / G;
+    s_row[i] = r;
+    for (int w = 0; w < kMaskWords; ++w) s_mask[i][w] = (r >= 0) ? a.mask[(size_t)r * kMaskWords + w] : 0u;
+  }
 
   const int g = lane >> 2, t4 = lane & 3, mi = lane >> 3, r8 = lane & 7;
   const float scale_log2 = rsqrtf((float)DH) * 1.4426950408889634f;
@@ -156,21 +159,36 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a, int pdl
     // mask, scale, online softmax (rows g and g+8 of this warp's 16)
     const int p0 = t * KT;
     const bool need_mask = (p0 + KT > n);
+    // visibility of the tile's 64 positions for this thread's two rows: bit j = position p0 + j;
+    // positions below n are the committed prefix (visible), position n + u is new row u (mask bit u)
+    uint32_t vis[2][2] = {{~0u, ~0u}, {~0u, ~0u}};
+    if (need_mask) {
+#pragma unroll
+      for (int rr = 0; rr < 2; ++rr) {
+        const uint32_t *mw = s_mask[warp * 16 + g + rr * 8];
+#pragma unroll
+        for (int hw = 0; hw < 2; ++hw) {
+          const int sh = p0 + 32 * hw - n;             // mask bit of this word's bit 0
+          uint32_t bits;
+          if (sh <= -32) bits = ~0u;
+          else if (sh < 0) bits = (mw[0] << (-sh)) | ((1u << (-sh)) - 1u);
+          else {
+            const int w = sh >> 5, bsh = sh & 31;
+            const uint32_t lo = (w < kMaskWords) ? mw[w] : 0u, hi = (w + 1 < kMaskWords) ? mw[w + 1] : 0u;
+            bits = bsh ? ((lo >> bsh) | (hi << (32 - bsh))) : lo;
+          }
+          vis[rr][hw] = bits;
+        }
+      }
+    }
     float mx[2] = {m_run[0], m_run[1]};
 #pragma unroll
     for (int nt = 0; nt < KT / 8; ++nt) {
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const int rr = e >> 1, pos = p0 + nt * 8 + t4 * 2 + (e & 1);
+        const int rr = e >> 1, j = nt * 8 + t4 * 2 + (e & 1);
         float v = sc[nt][e] * scale_log2;
-        if (need_mask) {
-          bool vis = pos < n;
-          if (!vis && pos < kv_len) {
-            const int u = pos - n;
-            vis = (s_mask[warp * 16 + g + rr * 8][u >> 5] >> (u & 31)) & 1u;
-          }
-          if (!vis) v = -INFINITY;
-        }
+        if (!((vis[rr][j >> 5] >> (j & 31)) & 1u)) v = -INFINITY;
         sc[nt][e] = v;
         mx[rr] = fmaxf(mx[rr], v);
       }
@@ -246,18 +264,21 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a, int pdl
     p_l[sp][i] = *cluster.map_shared_rank(&s_l[i], sp);
   }
   __syncthreads();
-  constexpr int RPP = kThreads / DH;                // rows finalised per pass (1 for dh = 128, 2 for dh = 64)
-  const int c = tid % DH, sub = tid / DH;
-  for (int i0 = rank * RPP; i0 < kQRows; i0 += 2 * nsp * RPP) {   // two passes at a time: 16 remote loads in flight
-    float ov[2][kAttnMaxSplits];
+  // a thread finalises 4 neighbouring dims of a row; rows rank, rank + nsp, ... belong to this CTA
+  constexpr int TPR = DH / 4, RP = kThreads / TPR;  // threads per row, rows per pass
+  const int c4 = (tid % TPR) * 4, sub = tid / TPR;
+  for (int q0 = 0; rank + q0 * nsp < kQRows; q0 += 2 * RP) {     // two passes at a time: 16 remote float4 loads in flight
+    float4 ov[2][kAttnMaxSplits];
     int row[2];
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
-      const int i = i0 + u * nsp * RPP + sub;
+      const int i = rank + (q0 + u * RP + sub) * nsp;
       row[u] = (i < kQRows && qb * kQRows + i < qrows_total) ? i : -1;
 #pragma unroll
       for (int sp = 0; sp < kAttnMaxSplits; ++sp)
-        ov[u][sp] = (row[u] >= 0 && sp < nsp) ? *cluster.map_shared_rank(sO + row[u] * DH + c, sp) : 0.f;
+        ov[u][sp] = (row[u] >= 0 && sp < nsp)
+                        ? *reinterpret_cast<const float4 *>(cluster.map_shared_rank(sO + row[u] * DH + c4, sp))
+                        : make_float4(0.f, 0.f, 0.f, 0.f);
     }
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
@@ -266,22 +287,29 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a, int pdl
       float M = -INFINITY;
 #pragma unroll
       for (int sp = 0; sp < kAttnMaxSplits; ++sp) if (sp < nsp) M = fmaxf(M, p_m[sp][i]);
-      float L = 0.f, acc = 0.f;
+      float L = 0.f;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int sp = 0; sp < kAttnMaxSplits; ++sp) {
         if (sp < nsp && p_m[sp][i] != -INFINITY) {
           const float w = exp2f(p_m[sp][i] - M);
           L += w * p_l[sp][i];
-          acc += w * ov[u][sp];
+          acc.x += w * ov[u][sp].x; acc.y += w * ov[u][sp].y; acc.z += w * ov[u][sp].z; acc.w += w * ov[u][sp].w;
         }
       }
-      const float val = (L > 0.f) ? acc / L : 0.f;
+      const float inv = (L > 0.f) ? 1.f / L : 0.f;
+      const float val[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
       const int qr = qb * kQRows + i;
       const int r = s * a.rw.Ms + qr / G, head = kvh * G + qr % G;
-      const bf16 hi = __float2bfloat16_rn(val);
-      const size_t idx = ((size_t)r * a.H + head) * DH + c;
-      a.o[idx] = hi;
-      a.o[a.o_lo_off + idx] = __float2bfloat16_rn(val - __bfloat162float(hi));
+      const __nv_bfloat162 h01 = __floats2bfloat162_rn(val[0], val[1]), h23 = __floats2bfloat162_rn(val[2], val[3]);
+      const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
+      const __nv_bfloat162 l01 = __floats2bfloat162_rn(val[0] - f01.x, val[1] - f01.y);
+      const __nv_bfloat162 l23 = __floats2bfloat162_rn(val[2] - f23.x, val[3] - f23.y);
+      const size_t idx = ((size_t)r * a.H + head) * DH + c4;
+      *reinterpret_cast<uint2 *>(a.o + idx) =
+          make_uint2(*reinterpret_cast<const uint32_t *>(&h01), *reinterpret_cast<const uint32_t *>(&h23));
+      *reinterpret_cast<uint2 *>(a.o + a.o_lo_off + idx) =
+          make_uint2(*reinterpret_cast<const uint32_t *>(&l01), *reinterpret_cast<const uint32_t *>(&l23));
     }
   }
   cluster.sync();                                   // peers may still be reading this CTA's partials
@@ -317,8 +345,9 @@ template <int DH> cudaError_t launch_dh(const AttnArgs &a, bool pdl, cudaStream_
 int attention_splits(int groups, int kv_tiles) {
   // CTAs of one (kv head, query block) = one cluster (<= 8): about two CTAs per SM over the whole grid,
   // never more splits than 64-position tiles
+  static const int budget = [] { const char *e = getenv("FIRP_ATTN_CTAS"); return e ? atoi(e) : 296; }();
   int s = 1;
-  while (s < kAttnMaxSplits && 2 * s * groups <= 2 * 148 && 2 * s <= kv_tiles) s *= 2;
+  while (s < kAttnMaxSplits && 2 * s * groups <= budget && 2 * s <= kv_tiles) s *= 2;
   return s;
 }
 
