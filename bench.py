@@ -42,6 +42,7 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-kernel-times", action="store_true", help="skip the per-kernel event-timed pass")
+    ap.add_argument("--sweep", action="store_true", help="config-4 sweep on the c2 weights: T x context, one JSON line per point")
     return ap.parse_args()
 
 
@@ -57,20 +58,20 @@ def pick_shape(name: str, layers: int):
     return shape
 
 
-def algorithmic_bytes(shape, n_ctx: float) -> dict:
+def algorithmic_bytes(shape, n_ctx: float, batch: int = 1) -> dict:
     """Bytes one step must move: every weight once, the KV cache read once per layer, the new
     rows' KV written once, the embedding rows (logits stay on the device and are not exported)."""
     s = shape
     M_lo, M_hi = s.T, s.T + s.k
     weights = s.weight_bytes()
-    kv_row = 2 * 2 * s.n_kv                       # K and V, bf16
+    kv_row = 2 * 2 * s.n_kv * batch               # K and V, bf16, every sequence
     kv_read = kv_write = 0
     for j in range(s.L):
         M = M_hi if (s.k > 0 and j >= s.l) else M_lo
         kv_read += kv_row * (n_ctx + M)
         kv_write += kv_row * M
-    return dict(weights=weights, kv_read=kv_read, kv_write=kv_write, embed=2 * s.T * s.d,
-                total=weights + kv_read + kv_write + 2 * s.T * s.d)
+    return dict(weights=weights, kv_read=kv_read, kv_write=kv_write, embed=2 * s.T * s.d * batch,
+                total=weights + kv_read + kv_write + 2 * s.T * s.d * batch)
 
 
 def class_bytes(shape, n_ctx: float) -> dict:
@@ -102,15 +103,16 @@ def kernel_source_digest() -> str:
     return h.hexdigest()[:16]
 
 
-def kernel_times(eng, shape, parents, tokens, out, steps, n_ctx, peak_gbs, peak_kind):
+def kernel_times(eng, shape, parents, tokens, out, steps, n_ctx, peak_gbs, peak_kind, seq_ids=None):
     """Second, separately timed pass: the library brackets every launch with CUDA events on the
     launching stream; per class: launches, average duration, share of the summed kernel time and,
     for the HBM-streaming classes, achieved GB/s = algorithmic bytes per launch / average duration."""
+    seq_ids = seq_ids or [0]
     eng.profile(True)
     for _ in range(steps):
-        eng.step(tokens, parents, shape.k, shape.l, out)
-        eng.commit(1)
-        tokens = out.next_tree_tokens[0]
+        eng.step(tokens, parents, shape.k, shape.l, out, seq_ids=seq_ids, n_seq=len(seq_ids))
+        eng.commit(len(seq_ids), seq_ids=seq_ids)
+        tokens = out.next_tree_tokens
     prof = eng.profile_read()
     eng.profile(False)
     total = sum(us for _, us in prof.values()) or 1.0
@@ -253,6 +255,54 @@ def run_reference(args, shape):
     print(json.dumps(line))
 
 
+def run_sweep(args, shape, weights, dev, rank):
+    """Config 4: tree size x committed context on the c2 weights, `--steps` steps per point (default 64 there),
+    device-resident timing only.  One engine serves every point; one JSON line per point."""
+    import torch
+    import synth_inputs as si
+    from paper_2410_20488_b200 import FirpEngine
+    K, W = args.steps, max(args.warmup, 3)
+    eng = FirpEngine(shape, weights, max_ctx=max(si.C4_CONTEXTS) + (K + W + 2) * 4 + 128 + 3 + 64, max_tree=128, max_k=3,
+                     max_depth=3, device=str(dev))
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except OSError:
+        pass
+    peak_gbs = peaks.get("hbm_gbs", 6650.0)
+    for n_ctx in si.C4_CONTEXTS:
+        prompt = torch.from_numpy(si.prompt(shape, length=n_ctx)).to(dev)
+        for T in si.C4_TREE_SIZES:
+            pt = si.c4_point(T, n_ctx)
+            parents = si.tree_template(T)
+            T_next = T if pt.k > 0 else 1
+            pout = eng.new_out(1, 1, pt.k, T_next=T_next, want_logits=False)
+            eng.prefill(0, prompt, pt.k, pt.l, parents if pt.k > 0 else None, pout)
+            outs = [eng.new_out(1, T, pt.k, want_logits=False) for _ in range(2)]
+            tokens = pout.next_tree_tokens
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n_w = n_ctx
+            for i in range(W + K):
+                if i == W:
+                    n_w = eng.context_len(0)        # synchronises
+                    ev0.record()
+                o = outs[i & 1]
+                eng.step(tokens, parents, pt.k, pt.l, o)
+                eng.commit(1)
+                tokens = o.next_tree_tokens
+            ev1.record()
+            torch.cuda.synchronize()
+            ms = ev0.elapsed_time(ev1) / K
+            n_end = eng.context_len(0)
+            ab = algorithmic_bytes(pt, 0.5 * (n_ctx + n_end))
+            gbs = ab["total"] / (ms * 1e-3) / 1e9
+            print(json.dumps(dict(workload=pt.name, T=T, k=pt.k, context=n_ctx, steps=K, ms_per_step=ms,
+                                  tokens_per_s=(n_end - n_w) / (ms * K * 1e-3), bytes_per_step=ab["total"],
+                                  achieved_gbs=gbs, frac_of_measured_peak=gbs / peak_gbs, frac_of_8tbs=gbs / 8000.0)),
+                  flush=True)
+    eng.close()
+
+
 def main():
     args = parse()
     shape = pick_shape(args.workload, args.layers)
@@ -280,18 +330,29 @@ def main():
 
     K, W = args.steps, max(args.warmup, 3)
     weights = load_weights(shape, local_rank, world)
+    if args.sweep:
+        return run_sweep(args, shape, weights, dev, rank)
     parents = si.tree_template(shape.T)
-    depth_max = {1: 0}.get(shape.T, 3)
+    B = shape.batch
     S = max(shape.k, 1) + 1
     total_steps = 2 * (K + W) + 16
-    max_ctx = shape.prompt_len + total_steps * S + shape.T + shape.k + 64
-    eng = FirpEngine(shape, weights, max_ctx=max_ctx, device=str(dev))
-    prompt = torch.from_numpy(si.prompt(shape, seq=rank)).to(dev)
-    outs = [eng.new_out(1, shape.T, shape.k, want_logits=False) for _ in range(2)]
-    pout = eng.new_out(1, 1, shape.k, T_next=shape.T if shape.k > 0 else 1, want_logits=False)
-    eng.prefill(0, prompt, shape.k, shape.l, parents if shape.k > 0 else None, pout)
+    if B > 1:       # config 5: every sequence has its own committed context length, uniform in [256, 4096]
+        lengths = [int(n) for n in si.context_lengths(shape)]
+    else:
+        lengths = [shape.prompt_len]
+    max_ctx = max(lengths) + total_steps * S + shape.T + shape.k + 64
+    eng = FirpEngine(shape, weights, max_ctx=max_ctx, max_batch=B, device=str(dev))
+    T_next = shape.T if shape.k > 0 else 1
+    outs = [eng.new_out(B, shape.T, shape.k, want_logits=False) for _ in range(2)]
+    first = torch.zeros(B, T_next, dtype=torch.int32, device=dev)
+    for b_i, n in enumerate(lengths):
+        prompt = torch.from_numpy(si.prompt(shape, seq=rank * B + b_i, length=n)).to(dev)
+        pout = eng.new_out(1, 1, shape.k, T_next=T_next, want_logits=False)
+        eng.prefill(b_i, prompt, shape.k, shape.l, parents if shape.k > 0 else None, pout)
+        first[b_i] = pout.next_tree_tokens[0]
     torch.cuda.synchronize()
-    n_start = eng.context_len(0)
+    n_start = sum(eng.context_len(b_i) for b_i in range(B)) / B
+    seq_ids = list(range(B))
 
     def barrier():
         if world > 1:
@@ -299,66 +360,65 @@ def main():
         torch.cuda.synchronize()
 
     # ---- device-resident timing: next tree tokens never leave the GPU -----------------------
-    tokens = pout.next_tree_tokens[0]
+    tokens = first
     launches = 0
     def one_step(i, tokens):
         nonlocal launches
         o = outs[i & 1]
-        eng.step(tokens, parents, shape.k, shape.l, o)
+        eng.step(tokens, parents, shape.k, shape.l, o, seq_ids=seq_ids, n_seq=B)
         launches += eng.launches()
-        eng.commit(1)
+        eng.commit(B, seq_ids=seq_ids)
         launches += eng.launches()
         return o
 
     sampler = ClockSampler(local_rank) if rank == 0 else None    # nvidia-smi takes a while to start: the warm-up
     for i in range(W):                                           # steps (same load) are sampled as well
-        tokens = one_step(i, tokens).next_tree_tokens[0]
+        tokens = one_step(i, tokens).next_tree_tokens
     barrier()
     launches = 0
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    acc_counts = torch.zeros(K, dtype=torch.int32, device=dev)
+    n_before = [eng.context_len(b_i) for b_i in range(B)]
+    barrier()
     ev0.record()
     for i in range(K):
-        o = one_step(i, tokens)
-        acc_counts[i] = o.n_accepted[0]
-        tokens = o.next_tree_tokens[0]
+        tokens = one_step(i, tokens).next_tree_tokens
     ev1.record()
     barrier()
     clocks = sampler.stop() if sampler else None
     ms_total = ev0.elapsed_time(ev1)
-    emitted = int(acc_counts.sum().item())
-    n_end = eng.context_len(0)
+    # every commit advances a context by the tokens that step emitted, so the growth counts them exactly
+    n_after = [eng.context_len(b_i) for b_i in range(B)]
+    emitted = sum(n_after) - sum(n_before)
+    n_end = sum(n_after) / B
 
     # ---- end to end: host buffers in, host results out, every step -------------------------
     e2e = None
     if not args.no_e2e:
-        h_tokens = torch.empty(shape.T, dtype=torch.int32).pin_memory()
+        h_tokens = torch.empty(B, T_next, dtype=torch.int32).pin_memory()
         h_tokens.copy_(tokens.cpu())
-        d_tokens = torch.empty(shape.T, dtype=torch.int32, device=dev)
+        d_tokens = torch.empty(B, T_next, dtype=torch.int32, device=dev)
         o = outs[0]
-        h_acc = torch.empty(S, dtype=torch.int32).pin_memory()
-        h_n = torch.empty(1, dtype=torch.int32).pin_memory()
-        h_next = torch.empty(shape.T if shape.k > 0 else 1, dtype=torch.int32).pin_memory()
+        h_acc = torch.empty(B, S, dtype=torch.int32).pin_memory()
+        h_n = torch.empty(B, dtype=torch.int32).pin_memory()
+        h_next = torch.empty(B, T_next, dtype=torch.int32).pin_memory()
         e_emitted = 0
         barrier()
-        t0 = time.perf_counter()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for i in range(K):
             d_tokens.copy_(h_tokens, non_blocking=True)
-            eng.step(d_tokens, parents, shape.k, shape.l, o)
-            eng.commit(1)
-            h_acc.copy_(o.accepted_tokens[0], non_blocking=True)
+            eng.step(d_tokens, parents, shape.k, shape.l, o, seq_ids=seq_ids, n_seq=B)
+            eng.commit(B, seq_ids=seq_ids)
+            h_acc.copy_(o.accepted_tokens, non_blocking=True)
             h_n.copy_(o.n_accepted, non_blocking=True)
-            h_next.copy_(o.next_tree_tokens[0], non_blocking=True)
+            h_next.copy_(o.next_tree_tokens, non_blocking=True)
             torch.cuda.current_stream().synchronize()
-            e_emitted += int(h_n[0])
-            h_tokens[: h_next.numel()].copy_(h_next)
+            e_emitted += int(h_n.sum())
+            h_tokens.copy_(h_next)
         e1.record()
         barrier()
-        e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3 * 0.0)
-        e2e = dict(ms=e_ms, emitted=e_emitted, h2d=int(h_tokens.numel() * 4),
-                   d2h=int((h_acc.numel() + 1 + h_next.numel()) * 4))
+        e2e = dict(ms=e0.elapsed_time(e1), emitted=e_emitted, h2d=int(h_tokens.numel() * 4),
+                   d2h=int((h_acc.numel() + h_n.numel() + h_next.numel()) * 4))
 
     # ---- aggregate over ranks: max time, summed units ----------------------------------------
     ms_max, units = aggregate_over_ranks(ms_total, emitted, dev)
@@ -378,18 +438,18 @@ def main():
     # ---- per-kernel-class durations (second, separately timed pass with events in the library) ----
     prof = None
     if not args.no_kernel_times:
-        prof = kernel_times(eng, shape, parents, tokens, outs[0], min(K, 8), n_end, peak_gbs, peak_kind)
-    ab = algorithmic_bytes(shape, n_mid)
+        prof = kernel_times(eng, shape, parents, tokens, outs[0], min(K, 8), n_end, peak_gbs, peak_kind, seq_ids)
+    ab = algorithmic_bytes(shape, n_mid, B)
     ms_step = ms_max / K
     step_gbs = ab["total"] / (ms_step * 1e-3) / 1e9
     line = dict(metric=METRIC, value=units / (ms_max * 1e-3), unit=UNIT, n_gpus=world, steps=K, warmup=W,
                 ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                 data="synthetic", gpu_launches=launches,
                 config=dict(workload=shape.name, T=shape.T, k=shape.k, l=shape.l, context_start=n_start,
-                            context_end=n_end, batch=1, l2="inputs_larger_than_l2 (%.1f GB of weights per step)" %
+                            context_end=n_end, batch=B, l2="inputs_larger_than_l2 (%.1f GB of weights per step)" %
                             (ab["weights"] / 1e9), parallelism="replicas x%d" % world,
                             mode="free-running greedy (random weights accept ~0 drafts per step)"),
-                step_latency_us=ms_step * 1e3, tokens_per_step=units / (K * world),
+                step_latency_us=ms_step * 1e3, tokens_per_step=units / (K * world), tokens_per_step_per_sequence=units / (K * world * B),
                 step_hbm=dict(bytes_per_step=ab["total"], weights=ab["weights"], kv_read=ab["kv_read"],
                               achieved_gbs=step_gbs, frac_of_measured_peak=step_gbs / peak_gbs,
                               frac_of_8tbs=step_gbs / 8000.0, peak_gbs=peak_gbs, peak=peak_kind),
