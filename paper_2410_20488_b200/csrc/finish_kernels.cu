@@ -83,7 +83,7 @@ __device__ __forceinline__ uint2 round4(const float v[4]) {
 // ---- q, k, v: rotary embedding, query planes, cache rows --------------------------------------
 // Supertile st holds the first halves (c < dh/2) of 128 / (dh/2) heads in tile 0 and their second
 // halves in tile 1, so lanes i4..i4+3 of the two tiles are 4 rotary pairs (c, c + dh/2) of one head.
-__global__ void __launch_bounds__(kThreads) qkv_finish_kernel(Partials p, GemmArgs a, int n_st, int pdl) {
+__global__ void __launch_bounds__(kThreads, 5) qkv_finish_kernel(Partials p, GemmArgs a, int n_st, int pdl) {
   if (pdl) { griddep_launch(); griddep_wait(); }
   Item it;
   if (!item_of_thread(n_st, a.R, it)) return;
@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(kThreads) qkv_finish_kernel(Partials p, GemmAr
 }
 
 // ---- SwiGLU: tile 0 = gate rows st*128 .., tile 1 = the matching up rows ------------------------
-__global__ void __launch_bounds__(kThreads) swiglu_finish_kernel(Partials p, GemmArgs a, int n_st, int pdl) {
+__global__ void __launch_bounds__(kThreads, 5) swiglu_finish_kernel(Partials p, GemmArgs a, int n_st, int pdl) {
   if (pdl) { griddep_launch(); griddep_wait(); }
   Item it;
   if (!item_of_thread(n_st, a.R, it)) return;
@@ -173,6 +173,30 @@ __global__ void __launch_bounds__(kThreads) logits_finish_kernel(Partials p, Gem
   }
 }
 
+// ---- Eq. 3: the k maps stacked into one [k d][d] matrix; token row m = sequence m ------------------------
+__global__ void __launch_bounds__(kThreads) pseudo_finish_kernel(Partials p, GemmArgs a, int n_st, int pdl) {
+  if (pdl) { griddep_launch(); griddep_wait(); }
+  Item it;
+  if (!item_of_thread(n_st, a.R, it)) return;
+  const int n0 = it.st * 256 + it.i4;
+  if (n0 >= a.N) return;
+  float4 v0, v1;
+  sum_partials(p, it.st, it.m, it.i4, v0, v1);
+  const float e[2][4] = {{v0.x, v0.y, v0.z, v0.w}, {v1.x, v1.y, v1.z, v1.w}};
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    const int n = n0 + 128 * t;                   // d is a multiple of 128: the 4 outputs belong to one map
+    if (n >= a.N) continue;
+    const int i = n / a.K, o = n - i * a.K;
+    float4 r = make_float4(e[t][0], e[t][1], e[t][2], e[t][3]);
+    if (a.pred_b) {
+      r.x += __bfloat162float(a.pred_b[n]); r.y += __bfloat162float(a.pred_b[n + 1]);
+      r.z += __bfloat162float(a.pred_b[n + 2]); r.w += __bfloat162float(a.pred_b[n + 3]);
+    }
+    *reinterpret_cast<float4 *>(a.h_rows + (size_t)(it.m * a.rw.Ms + a.rw.T + i) * a.K + o) = r;
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_gemm_finish(GemmEpilogue epi, const Partials &p, const GemmArgs &a, bool pdl, cudaStream_t st) {
@@ -183,6 +207,7 @@ cudaError_t launch_gemm_finish(GemmEpilogue epi, const Partials &p, const GemmAr
     case EPI_QKV_ROPE: return launch_k(qkv_finish_kernel, grid, block, 0, st, pdl, p, a, n_st, pdl ? 1 : 0);
     case EPI_SWIGLU: return launch_k(swiglu_finish_kernel, grid, block, 0, st, pdl, p, a, n_st, pdl ? 1 : 0);
     case EPI_LOGITS: return launch_k(logits_finish_kernel, grid, block, 0, st, pdl, p, a, n_st, pdl ? 1 : 0);
+    case EPI_PSEUDO: return launch_k(pseudo_finish_kernel, grid, block, 0, st, pdl, p, a, n_st, pdl ? 1 : 0);
     default: return cudaErrorInvalidValue;   // the residual GEMMs are finished by the RMSNorm kernel
   }
 }

@@ -58,7 +58,7 @@ struct firp_ctx {
   bf16 *kv = nullptr;
   float *h = nullptr, *gemm_ws = nullptr, *ss = nullptr, *logits = nullptr, *top_vals = nullptr, *cand_vals = nullptr;
   int32_t *cand_ids = nullptr;
-  bf16 *x = nullptr, *q = nullptr, *o = nullptr, *y = nullptr;
+  bf16 *x = nullptr, *xp = nullptr, *q = nullptr, *o = nullptr, *y = nullptr;
   int32_t *ctx_len = nullptr, *seq_ids = nullptr, *parents = nullptr, *next_parents = nullptr, *chain = nullptr;
   int32_t *top_ids = nullptr, *path = nullptr, *n_acc = nullptr, *accepted = nullptr, *next_tokens = nullptr;
   int32_t *exp_path = nullptr, *exp_len = nullptr;
@@ -78,6 +78,7 @@ struct firp_ctx {
     const int d = cfg.d_model, nq = cfg.n_heads * cfg.head_dim, half = cfg.head_dim / 2;
     const size_t R = Rmax;
     h = c.take<float>(R * d);
+    xp = c.take<bf16>(2 * (size_t)kMaxSeq * d);   // anchor rows of Eq. 3: hi plane, lo plane
     x = c.take<bf16>(3 * R * d);            // normalised activations: hi plane, lo plane, third plane (QKV input)
     q = c.take<bf16>(2 * R * nq);
     o = c.take<bf16>(2 * R * nq);
@@ -229,8 +230,16 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       FIRP_CUDA(c, launch_rmsnorm(rw, 0, carried, c->h, pending, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, 3, c->ss, pdl, st)); ++nl; }
     pending.sk.U = 0;
     if (insert) {   // Eq. 3 on the raw (now complete) residual row of the root, then the norm of the new rows
-      { FIRP_TIMED(KC_PSEUDO_PROJ);
-        launch_pseudo_proj(rw, (const bf16 *)c->w.pred_w, (const bf16 *)c->w.pred_b, d, c->h, pdl, st); ++nl; }
+      { FIRP_TIMED(KC_PSEUDO_PROJ);      // the k maps as one [k d][d] GEMM on the anchor rows (one row per sequence)
+        launch_root_split(rw, c->h, d, c->xp, (size_t)kMaxSeq * d, pdl, st); ++nl;
+        GemmArgs g{};
+        g.X = c->xp; g.x_lo_off = (size_t)kMaxSeq * d; g.plane_rows = kMaxSeq; g.planes = 2; g.err = c->dev_status;
+        g.W = (const bf16 *)c->w.pred_w; g.R = rw.n_seq; g.N = rw.k * d; g.K = d; g.rw = rw; g.rows_active = rw.Ms;
+        g.ws = c->gemm_ws; g.h_rows = c->h; g.pred_b = (const bf16 *)c->w.pred_b;
+        Partials p = pending;
+        FIRP_CUDA(c, launch_gemm_tc(EPI_PSEUDO, g, pdl, st, &p.sk)); ++nl;
+        p.ws_rows = kMaxSeq;
+        FIRP_CUDA(c, launch_gemm_finish(EPI_PSEUDO, p, g, pdl, st)); ++nl; }
       FIRP_TIMED(KC_RMSNORM);
       FIRP_CUDA(c, launch_rmsnorm(rw, rw.T, rw.Ms, c->h, none, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, 3, c->ss, pdl, st)); ++nl;
     }

@@ -86,8 +86,11 @@ constexpr int kNormMaxWarps = 64;   // d <= 8192
 cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Partials &pending, const bf16 *g, int d,
                            bf16 *x, size_t x_lo_off, int planes, float *ss, bool pdl, cudaStream_t st);
 
-// Eq. 3: h[s*Ms + T + i] = W_i h[s*Ms + anchor] + b_i
-void launch_pseudo_proj(const Rows &rw, const bf16 *pred_w, const bf16 *pred_b, int d, float *h, bool pdl, cudaStream_t st);
+// Eq. 3, h[s*Ms + T + i] = W_i h[s*Ms + anchor] + b_i, as a GEMM of the k maps stacked into one [k d][d] matrix:
+// launch_root_split writes the raw residual row of every sequence's anchor as (hi, lo) bf16 planes into row s of
+// xp; the GEMM (EPI_PSEUDO) multiplies; launch_gemm_finish(EPI_PSEUDO) sums the partial tiles, adds the bias and
+// stores the k new residual rows (GemmArgs: h_rows = residual stream, pred_b = bias or NULL, R = n_seq).
+void launch_root_split(const Rows &rw, const float *h, int d, bf16 *xp, size_t xp_lo_off, bool pdl, cudaStream_t st);
 
 // top-B of every row of logits by (value desc, id asc)
 // Two passes: per 2048-logit segment candidates (scratch cand_*: [R][topb_segments(V)][B]), then the row's top-B.
@@ -129,7 +132,7 @@ void launch_commit(int n_seq, const CommitArgs &a, bool pdl, cudaStream_t st);
 void launch_advance_ctx(int n_seq, const int32_t *seq_ids, int32_t *ctx_len, int amount, bool pdl, cudaStream_t st);
 
 // ---- skinny weight-streaming GEMM ------------------------------------------
-enum GemmEpilogue { EPI_RESIDUAL = 0, EPI_QKV_ROPE = 1, EPI_SWIGLU = 2, EPI_LOGITS = 3 };
+enum GemmEpilogue { EPI_RESIDUAL = 0, EPI_QKV_ROPE = 1, EPI_SWIGLU = 2, EPI_LOGITS = 3, EPI_PSEUDO = 4 };
 
 struct GemmArgs {
   const bf16 *X;    // [R][K] activations, first (hi) plane (row-major, K contiguous)
@@ -155,6 +158,8 @@ struct GemmArgs {
   bf16 *y; size_t y_lo_off; int F;
   // EPI_LOGITS: logits[R][N]
   float *logits;
+  // EPI_PSEUDO: row m = sequence m; output n = i * K + o goes to h_rows[(m * Ms + T + i) * K + o] (+ pred_b[n])
+  float *h_rows; const bf16 *pred_b;
 };
 // The GEMM leaves partial tiles in a.ws under the schedule *sk_out, to be finished by launch_gemm_finish
 // (or, for EPI_RESIDUAL, by launch_rmsnorm).  `epi` only selects how weight rows are grouped into supertiles.

@@ -175,51 +175,31 @@ cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Parti
 }
 
 // ---------------------------------------------------------------------------
-// Pseudo hidden states, Eq. 3: h~_i = W_i h[anchor] + b_i on the raw fp32 residual stream.
-// M = 1 row per sequence, so this is a weight-streaming GEMV on the FMA lanes:
-// one warp per output coordinate, 16-byte weight loads, fp32 accumulation.
+// Pseudo hidden states, Eq. 3: h~_i = W_i h[anchor] + b_i on the raw fp32 residual stream.  The k maps are
+// one [k d][d] weight matrix for the stream-K GEMM; this kernel prepares its operand: the anchor row of every
+// sequence, untouched by any norm, as (hi, lo) bf16 planes in row s of xp.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-pseudo_proj_kernel(Rows rw, const bf16 *__restrict__ W, const bf16 *__restrict__ b, int d, float *h, int pdl) {
+root_split_kernel(Rows rw, const float *h, int d, bf16 *xp, size_t xp_lo_off, int pdl) {
   if (pdl) { griddep_launch(); griddep_wait(); }
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (warp >= rw.k * d) return;
-  const int i = warp / d, o = warp % d;
-  const bf16 *wrow = W + ((size_t)i * d + o) * d;
-  float acc[kMaxSeq];
-#pragma unroll
-  for (int s = 0; s < kMaxSeq; ++s) acc[s] = 0.f;
-  for (int c = lane * 8; c < d; c += 32 * 8) {
-    const uint4 wv = *reinterpret_cast<const uint4 *>(wrow + c);
-    const __nv_bfloat162 *wp = reinterpret_cast<const __nv_bfloat162 *>(&wv);
-    float wf[8];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) { const float2 f = __bfloat1622float2(wp[j]); wf[2 * j] = f.x; wf[2 * j + 1] = f.y; }
-#pragma unroll
-    for (int s = 0; s < kMaxSeq; ++s) {
-      if (s < rw.n_seq) {
-        const float *hv = h + (size_t)(s * rw.Ms + rw.anchor) * d + c;
-        const float4 h0 = *reinterpret_cast<const float4 *>(hv), h1 = *reinterpret_cast<const float4 *>(hv + 4);
-        acc[s] += wf[0] * h0.x + wf[1] * h0.y + wf[2] * h0.z + wf[3] * h0.w + wf[4] * h1.x + wf[5] * h1.y +
-                  wf[6] * h1.z + wf[7] * h1.w;
-      }
-    }
-  }
-  const float bias = b ? __bfloat162float(b[(size_t)i * d + o]) : 0.f;
-#pragma unroll
-  for (int s = 0; s < kMaxSeq; ++s) {
-    if (s < rw.n_seq) {
-      float a = acc[s];
-#pragma unroll
-      for (int sh = 16; sh > 0; sh >>= 1) a += __shfl_xor_sync(0xffffffffu, a, sh);
-      if (lane == 0) h[(size_t)(s * rw.Ms + rw.T + i) * d + o] = a + bias;
-    }
-  }
+  const int nvec = d >> 2;
+  const unsigned t = blockIdx.x * 256 + threadIdx.x;
+  if (t >= (unsigned)(rw.n_seq * nvec)) return;
+  const int s = (int)(t / (unsigned)nvec), idx = (int)(t % (unsigned)nvec);
+  const float4 a = __ldcg(reinterpret_cast<const float4 *>(h + (size_t)(s * rw.Ms + rw.anchor) * d) + idx);
+  const __nv_bfloat162 o01 = __floats2bfloat162_rn(a.x, a.y), o23 = __floats2bfloat162_rn(a.z, a.w);
+  const float2 f01 = __bfloat1622float2(o01), f23 = __bfloat1622float2(o23);
+  const __nv_bfloat162 l01 = __floats2bfloat162_rn(a.x - f01.x, a.y - f01.y), l23 = __floats2bfloat162_rn(a.z - f23.x, a.w - f23.y);
+  uint2 hi2, lo2;
+  hi2.x = *reinterpret_cast<const uint32_t *>(&o01); hi2.y = *reinterpret_cast<const uint32_t *>(&o23);
+  lo2.x = *reinterpret_cast<const uint32_t *>(&l01); lo2.y = *reinterpret_cast<const uint32_t *>(&l23);
+  *reinterpret_cast<uint2 *>(xp + (size_t)s * d + 4 * idx) = hi2;
+  *reinterpret_cast<uint2 *>(xp + xp_lo_off + (size_t)s * d + 4 * idx) = lo2;
 }
 
-void launch_pseudo_proj(const Rows &rw, const bf16 *pred_w, const bf16 *pred_b, int d, float *h, bool pdl, cudaStream_t st) {
-  const int warps = rw.k * d;
-  launch_k(pseudo_proj_kernel, dim3((warps + 7) / 8), dim3(256), 0, st, pdl, rw, pred_w, pred_b, d, h, pdl ? 1 : 0);
+void launch_root_split(const Rows &rw, const float *h, int d, bf16 *xp, size_t xp_lo_off, bool pdl, cudaStream_t st) {
+  const int threads = rw.n_seq * (d >> 2);
+  launch_k(root_split_kernel, dim3((threads + 255) / 256), dim3(256), 0, st, pdl, rw, h, d, xp, xp_lo_off, pdl ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------

@@ -56,6 +56,17 @@ def test_c1_random_trees_and_layers(torch_cuda, c1, c1_weights, case):
     eng.close()
 
 
+def test_c1_predictor_with_bias(torch_cuda, c1, c1_weights):
+    """Eq. 3 with a non-zero bias b_i (the synthetic configurations use b = 0)."""
+    w = dict(c1_weights)
+    w["pred_b"] = si.normal_bf16(c1.seed, si.stream_id("pred_w", 7), c1.k * c1.d, 0.5).reshape(c1.k, c1.d)
+    parents = si.tree_template(c1.T)
+    eng, orc = make_pair(c1, w, 256)
+    st = lockstep_run(eng, orc, c1, parents, si.prompt(c1, length=19), 3)
+    assert st.steps == 3
+    eng.close()
+
+
 def test_device_side_commit_matches_explicit(torch_cuda, c1, c1_weights):
     """firp_kv_commit(NULL path) uses the path found on the device."""
     import torch
