@@ -70,7 +70,6 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a, int pdl
   __shared__ uint32_t s_mask[kQRows][kMaskWords];
   __shared__ int s_row[kQRows];                     // global row index of each query row, -1 = padding
   __shared__ float s_m[kQRows], s_l[kQRows];        // this split's running max (log2 units) and sum per query row
-  __shared__ float p_m[kAttnMaxSplits][kQRows], p_l[kAttnMaxSplits][kQRows];   // every split's, gathered for the merge
   if (pdl) { griddep_launch(); griddep_wait(); }
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -89,7 +88,7 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a, int pdl
     cp_async_16(smem_u32(sQ + Q_BYTES + tile_off<DH>(i, c)), valid ? src + a.q_lo_off : a.q, valid);
   }
   const int slot = a.seq_ids[s];
-  const int n = a.ctx_len[slot];
+  const int n = a.pos[s * a.rw.Ms];                 // position of the root row = committed length (no dependent load)
   const int kv_len = min(n + a.rows_active, a.max_ctx);
   const int tiles_total = (kv_len + KT - 1) / KT;
   // balanced ranges; a remainder goes to the first splits, the last one owns the (slower) masked tiles
@@ -257,28 +256,25 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a, int pdl
   cg::cluster_group cluster = cg::this_cluster();
   cluster.sync();
   const int rank = (int)cluster.block_rank(), nsp = (int)cluster.num_blocks();
-#pragma unroll 4
-  for (int idx = tid; idx < nsp * kQRows; idx += kThreads) {     // all peers' (max, sum): independent remote loads
-    const int sp = idx / kQRows, i = idx % kQRows;
-    p_m[sp][i] = *cluster.map_shared_rank(&s_m[i], sp);
-    p_l[sp][i] = *cluster.map_shared_rank(&s_l[i], sp);
-  }
-  __syncthreads();
   // a thread finalises 4 neighbouring dims of a row; rows rank, rank + nsp, ... belong to this CTA
   constexpr int TPR = DH / 4, RP = kThreads / TPR;  // threads per row, rows per pass
   const int c4 = (tid % TPR) * 4, sub = tid / TPR;
   for (int q0 = 0; rank + q0 * nsp < kQRows; q0 += 2 * RP) {     // two passes at a time: 16 remote float4 loads in flight
     float4 ov[2][kAttnMaxSplits];
+    float pm[2][kAttnMaxSplits], pl[2][kAttnMaxSplits];   // every split's (max, sum) of the row, fetched with its O
     int row[2];
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
       const int i = rank + (q0 + u * RP + sub) * nsp;
       row[u] = (i < kQRows && qb * kQRows + i < qrows_total) ? i : -1;
 #pragma unroll
-      for (int sp = 0; sp < kAttnMaxSplits; ++sp)
-        ov[u][sp] = (row[u] >= 0 && sp < nsp)
-                        ? *reinterpret_cast<const float4 *>(cluster.map_shared_rank(sO + row[u] * DH + c4, sp))
-                        : make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int sp = 0; sp < kAttnMaxSplits; ++sp) {
+        const bool on = row[u] >= 0 && sp < nsp;
+        ov[u][sp] = on ? *reinterpret_cast<const float4 *>(cluster.map_shared_rank(sO + row[u] * DH + c4, sp))
+                       : make_float4(0.f, 0.f, 0.f, 0.f);
+        pm[u][sp] = on ? *cluster.map_shared_rank(&s_m[row[u]], sp) : -INFINITY;
+        pl[u][sp] = on ? *cluster.map_shared_rank(&s_l[row[u]], sp) : 0.f;
+      }
     }
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
@@ -286,14 +282,14 @@ __global__ void __launch_bounds__(kThreads) tree_attn_kernel(AttnArgs a, int pdl
       if (i < 0) continue;
       float M = -INFINITY;
 #pragma unroll
-      for (int sp = 0; sp < kAttnMaxSplits; ++sp) if (sp < nsp) M = fmaxf(M, p_m[sp][i]);
+      for (int sp = 0; sp < kAttnMaxSplits; ++sp) M = fmaxf(M, pm[u][sp]);
       float L = 0.f;
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int sp = 0; sp < kAttnMaxSplits; ++sp) {
-        if (sp < nsp && p_m[sp][i] != -INFINITY) {
-          const float w = exp2f(p_m[sp][i] - M);
-          L += w * p_l[sp][i];
+        if (pm[u][sp] != -INFINITY) {
+          const float w = exp2f(pm[u][sp] - M);
+          L += w * pl[u][sp];
           acc.x += w * ov[u][sp].x; acc.y += w * ov[u][sp].y; acc.z += w * ov[u][sp].z; acc.w += w * ov[u][sp].w;
         }
       }

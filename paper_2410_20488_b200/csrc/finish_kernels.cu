@@ -117,7 +117,7 @@ __global__ void __launch_bounds__(kThreads, 5) qkv_finish_kernel(Partials p, Gem
     const int is_v = unit >= a.H + a.Hkv;
     const int kvh = unit - a.H - (is_v ? a.Hkv : 0);
     const int slot = a.seq_ids[s];
-    const int pos = a.ctx_len[slot] + v;
+    const int pos = a.pos[s * a.rw.Ms] + v;        // committed length (position of the root row) + row index
     if (pos < a.max_ctx) {
       bf16 *dst = a.kcache + (size_t)slot * a.seq_stride + (is_v ? a.kv_stride : 0) + ((size_t)pos * a.Hkv + kvh) * a.dh + c;
       *reinterpret_cast<uint2 *>(dst) = round4(x1);

@@ -248,7 +248,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       GemmArgs g = gemm_base(c->x, Rp * d, c->wqkv[j], (H + 2 * Hkv) * dh, d, act);
       g.H = H; g.Hkv = Hkv; g.dh = dh;
       g.planes = 3;   // keys and values are rounded to bf16 for the cache: their inputs carry ~24 mantissa bits
-      g.rope = c->meta.rope; g.seq_ids = c->seq_ids; g.ctx_len = c->ctx_len;
+      g.rope = c->meta.rope; g.seq_ids = c->seq_ids; g.ctx_len = c->ctx_len; g.pos = c->meta.pos;
       g.q = c->q; g.q_lo_off = Rp * nq; g.kcache = kplane; g.seq_stride = c->kv_seq(); g.kv_stride = c->kv_plane(); g.max_ctx = cfg.max_ctx;
       Partials p = pending;
       { FIRP_TIMED(KC_GEMM_QKV);
@@ -260,7 +260,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       AttnArgs a{};
       a.rw = rw; a.rows_active = act; a.H = H; a.Hkv = Hkv; a.dh = dh;
       a.q = c->q; a.q_lo_off = Rp * nq; a.kcache = kplane; a.seq_stride = c->kv_seq(); a.kv_stride = c->kv_plane(); a.max_ctx = cfg.max_ctx;
-      a.seq_ids = c->seq_ids; a.ctx_len = c->ctx_len; a.mask = c->meta.mask;
+      a.seq_ids = c->seq_ids; a.ctx_len = c->ctx_len; a.pos = c->meta.pos; a.mask = c->meta.mask;
       const int tiles = (ra.n_hi_max + act + kAttnTile - 1) / kAttnTile;
       const int G = H / Hkv, qblocks = (act * G + 63) / 64;
       a.splits = attention_splits(rw.n_seq * Hkv * qblocks, tiles);

@@ -151,7 +151,7 @@ struct GemmArgs {
   const float *ss; float eps;
   // EPI_QKV_ROPE
   int H, Hkv, dh;
-  const float2 *rope; const int32_t *seq_ids; const int32_t *ctx_len;
+  const float2 *rope; const int32_t *seq_ids; const int32_t *ctx_len; const int32_t *pos;   // pos[R]: row positions
   bf16 *q; size_t q_lo_off;      // [R][H*dh] hi plane, lo plane
   bf16 *kcache; size_t seq_stride, kv_stride; int max_ctx;  // kcache points at this layer's K plane of sequence slot 0
   // EPI_SWIGLU: y[R][F], N = 2F
@@ -177,6 +177,7 @@ struct AttnArgs {
   const bf16 *kcache;         // this layer's K plane of slot 0; V plane = kcache + kv_stride
   size_t seq_stride, kv_stride; int max_ctx;
   const int32_t *seq_ids, *ctx_len;
+  const int32_t *pos;         // [R] absolute position of every row (row 0 of a sequence: its committed length)
   const uint32_t *mask;       // [R][kMaskWords]
   int splits;                 // kv splits (grid.x = cluster size): 1, 2, 4 or 8
   bf16 *o; size_t o_lo_off;   // [R][H*dh] hi plane, lo plane
