@@ -249,7 +249,9 @@ def run_reference(args, shape):
     line = dict(metric=METRIC, value=tps, unit=UNIT, n_gpus=args.gpus, steps=steps, warmup=warmup, ms_per_step=ms,
                 higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32 storage, f64 accumulation",
                 data="synthetic", impl="reference",
-                config=dict(workload=shape.name, T=shape.T, k=shape.k, l=shape.l, context=32),
+                config=dict(workload=shape.name, T=shape.T, k=shape.k, l=shape.l, context_start=shape.prompt_len,
+                            batch=1, sample="oracle steps on a 32-token context instead of %d tokens (its prefill "
+                            "cost grows with the context; the step's GEMM work does not)" % shape.prompt_len),
                 cpu_baseline=dict(value=tps, unit=UNIT, cores=host_cores(), kind="oracle", sample=sample),
                 e2e=dict(value=tps, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line))
