@@ -125,7 +125,6 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float *r) {
                : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // Shared-memory operand descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups
 // 1024 bytes apart (start address >> 4 in bits 0-13, leading offset 1 in bits 16-29 (unused for
