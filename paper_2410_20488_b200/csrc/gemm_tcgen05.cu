@@ -148,7 +148,10 @@ constexpr int pow2_cols(int c) { return c <= 32 ? 32 : c <= 64 ? 64 : c <= 128 ?
 template <int NPAD, int P> struct TcCfg {
   static constexpr int X_PLANE = NPAD * 128;                   // bytes of one activation plane per stage
   static constexpr int X_STAGE = P * X_PLANE;
-  static constexpr bool MERGE = (P * NPAD <= 256) && ((P * NPAD) % 16 == 0);
+  // two planes are merged only while two accumulator buffers still fit the 512 TMEM columns (measured: the
+  // second buffer -- epilogue of one segment under the main loop of the next -- is worth more than one MMA
+  // instead of two); three planes are always merged when legal (measured the other way round)
+  static constexpr bool MERGE = (P * NPAD <= 256) && ((P * NPAD) % 16 == 0) && (2 * TM * P * NPAD <= 512 || NPAD % 16 != 0 || P > 2);
   static constexpr int ACC_COLS = MERGE ? P * NPAD : NPAD;     // accumulator columns per weight tile
   static constexpr int NBUF = (2 * TM * ACC_COLS <= 512) ? 2 : 1;   // accumulator buffers
   static constexpr int TMEM_COLS = pow2_cols(NBUF * TM * ACC_COLS);
