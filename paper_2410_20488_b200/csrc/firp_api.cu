@@ -201,6 +201,16 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   const firp_step_out *out = ra.out;
   int &nl = c->launches;
   const bool pdl = c->use_pdl;
+  // L2 lookahead per GEMM class (32 KB units beyond the ring): qkv, o, gate/up, down, lm-head.  Measured at the
+  // 7B shape: it pays before the GEMMs whose predecessor is short or cannot share the SM (o, gate/up) and
+  // costs before the down projection, whose finisher it slows by more than it saves.  FIRP_L2_AHEAD=a,b,c,d,e
+  // overrides (tuning aid).
+  static int ahead[5] = {0, 48, 48, 0, 48};
+  static bool ahead_init = false;
+  if (!ahead_init) {
+    ahead_init = true;
+    if (const char *e = getenv("FIRP_L2_AHEAD")) sscanf(e, "%d,%d,%d,%d,%d", &ahead[0], &ahead[1], &ahead[2], &ahead[3], &ahead[4]);
+  }
 
   const int mw_out = (rw.Ms + 31) / 32;
   { FIRP_TIMED(KC_TREE_PREP);
@@ -213,7 +223,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     GemmArgs g{};
     g.X = X; g.x_lo_off = lo_off; g.plane_rows = (int)Rp; g.err = c->dev_status;
     g.W = (const bf16 *)W; g.R = rw.R; g.N = N; g.K = K; g.rw = rw; g.rows_active = act; g.planes = 2;
-    g.ws = c->gemm_ws;
+    g.ws = c->gemm_ws; g.l2_ahead = 48;
     if (X == c->x) { g.ss = c->ss; g.eps = cfg.rms_eps; }   // x = h * g: the finisher divides by the row's RMS
     return g;
   };
@@ -235,7 +245,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
         GemmArgs g{};
         g.X = c->xp; g.x_lo_off = (size_t)kMaxSeq * d; g.plane_rows = kMaxSeq; g.planes = 2; g.err = c->dev_status;
         g.W = (const bf16 *)c->w.pred_w; g.R = rw.n_seq; g.N = rw.k * d; g.K = d; g.rw = rw; g.rows_active = rw.Ms;
-        g.ws = c->gemm_ws; g.h_rows = c->h; g.pred_b = (const bf16 *)c->w.pred_b;
+        g.ws = c->gemm_ws; g.l2_ahead = 48; g.h_rows = c->h; g.pred_b = (const bf16 *)c->w.pred_b;
         Partials p = pending;
         FIRP_CUDA(c, launch_gemm_tc(EPI_PSEUDO, g, pdl, st, &p.sk)); ++nl;
         p.ws_rows = kMaxSeq;
@@ -247,6 +257,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     {
       GemmArgs g = gemm_base(c->x, Rp * d, c->wqkv[j], (H + 2 * Hkv) * dh, d, act);
       g.H = H; g.Hkv = Hkv; g.dh = dh;
+      g.l2_ahead = ahead[0];
       g.planes = 3;   // keys and values are rounded to bf16 for the cache: their inputs carry ~24 mantissa bits
       g.rope = c->meta.rope; g.seq_ids = c->seq_ids; g.ctx_len = c->ctx_len; g.pos = c->meta.pos;
       g.q = c->q; g.q_lo_off = Rp * nq; g.kcache = kplane; g.seq_stride = c->kv_seq(); g.kv_stride = c->kv_plane(); g.max_ctx = cfg.max_ctx;
@@ -270,6 +281,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     }
     {
       GemmArgs g = gemm_base(c->o, Rp * nq, c->wo[j], d, nq, act);
+      g.l2_ahead = ahead[1];
       FIRP_TIMED(KC_GEMM_O);
       FIRP_CUDA(c, launch_gemm_tc(EPI_RESIDUAL, g, pdl, st, &pending.sk)); ++nl;
     }
@@ -278,7 +290,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     pending.sk.U = 0;
     {
       GemmArgs g = gemm_base(c->x, Rp * d, c->wgu[j], 2 * F, d, act);
-      g.y = c->y; g.y_lo_off = Rp * F; g.F = F;
+      g.y = c->y; g.y_lo_off = Rp * F; g.F = F; g.l2_ahead = ahead[2];
       Partials p = pending;
       { FIRP_TIMED(KC_GEMM_GATE_UP);
         FIRP_CUDA(c, launch_gemm_tc(EPI_SWIGLU, g, pdl, st, &p.sk)); ++nl; }
@@ -287,6 +299,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     }
     {
       GemmArgs g = gemm_base(c->y, Rp * F, c->wd[j], d, F, act);
+      g.l2_ahead = ahead[3];
       FIRP_TIMED(KC_GEMM_DOWN);
       FIRP_CUDA(c, launch_gemm_tc(EPI_RESIDUAL, g, pdl, st, &pending.sk)); ++nl;
     }
@@ -295,7 +308,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     { FIRP_TIMED(KC_RMSNORM);
       FIRP_CUDA(c, launch_rmsnorm(rw, 0, rw.Ms, c->h, pending, (const bf16 *)c->w.g_final, d, c->x, Rp * d, 2, c->ss, pdl, st)); ++nl; }
     GemmArgs g = gemm_base(c->x, Rp * d, c->w.lm_head, cfg.vocab, d, rw.Ms);
-    g.logits = ra.logits_dst;
+    g.logits = ra.logits_dst; g.l2_ahead = ahead[4];
     { Partials p = pending;
       { FIRP_TIMED(KC_GEMM_LM_HEAD);
         FIRP_CUDA(c, launch_gemm_tc(EPI_LOGITS, g, pdl, st, &p.sk)); ++nl; }

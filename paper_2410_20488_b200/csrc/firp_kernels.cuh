@@ -146,6 +146,7 @@ struct GemmArgs {
   Rows rw; int rows_active;      // rows with v < rows_active are written, the others skipped
   // stream-K scratch: partial tiles [kGemmMaxCtas][kGemmSlots][2][plane_rows][128] fp32
   float *ws;
+  int l2_ahead;     // 32 KB units each CTA prefetches into L2 beyond its shared-memory ring while it waits
   // finishers: X holds h * g, not yet divided by the RMS: row m of the result is scaled by
   // 1 / sqrt(sum_w ss[m][w] / K + eps) (ss == NULL: X is used as it is)
   const float *ss; float eps;

@@ -487,8 +487,7 @@ Sched make_sched(GemmEpilogue epi, const GemmArgs &a, bool pdl) {
   Sched sc{};
   sc.pdl = pdl ? 1 : 0;
   sc.ws_rows = a.plane_rows;
-  static const int l2_ahead = [] { const char *e = getenv("FIRP_L2_AHEAD"); return e ? atoi(e) : 48; }();
-  sc.l2_ahead = l2_ahead < 0 ? 0 : l2_ahead;
+  sc.l2_ahead = a.l2_ahead < 0 ? 0 : a.l2_ahead;
   sc.mode = ROWS_LINEAR; sc.n_st = (a.N + TM * BM - 1) / (TM * BM);
   if (epi == EPI_SWIGLU) {
     sc.mode = ROWS_GATE_UP; sc.F = a.F; sc.n_st = (a.F + BM - 1) / BM;
