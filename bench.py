@@ -88,7 +88,7 @@ def class_bytes(shape, n_ctx: float) -> dict:
 # c2 shape, from the ncu capture summarised under profiles/; valid only for the kernel sources whose
 # digest is recorded with it (a changed kernel reports traffic = null until it is captured again).
 NCU_TRAFFIC = {
-    "c2-llama2-7b": dict(digest="a88bcbe29712560e", per_launch={"gemm_gate_up": 197948160, "gemm_qkv": 108428032,
+    "c2-llama2-7b": dict(digest="3c40eb62a7f6c388", per_launch={"gemm_gate_up": 197948160, "gemm_qkv": 108428032,
                                                              "gemm_o": 34111488, "gemm_down": 96498688}),
 }
 

@@ -147,6 +147,10 @@ struct GemmArgs {
   // stream-K scratch: partial tiles [kGemmMaxCtas][kGemmSlots][2][plane_rows][128] fp32
   float *ws;
   int l2_ahead;     // 32 KB units each CTA prefetches into L2 beyond its shared-memory ring while it waits
+  // The GEMM that follows this one in the step (NULL: none).  Once a CTA has issued its own last load it
+  // prefetches the first next_units units of the same CTA's range of THAT GEMM into L2, so that HBM keeps
+  // streaming through this kernel's tail and the hand-over, and the next kernel's ring fills from L2.
+  const bf16 *next_W; int next_epi, next_N, next_K, next_F, next_heads, next_dh, next_units;
   // finishers: X holds h * g, not yet divided by the RMS: row m of the result is scaled by
   // 1 / sqrt(sum_w ss[m][w] / K + eps) (ss == NULL: X is used as it is)
   const float *ss; float eps;

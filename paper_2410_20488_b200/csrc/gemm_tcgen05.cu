@@ -183,9 +183,25 @@ struct Sched {
   int l2_ahead;    // units each CTA prefetches into L2 beyond its shared-memory ring
 };
 
+// L2 prefetch of the two weight tiles of unit (supertile st, k block kb) under schedule sc
+__device__ __forceinline__ void prefetch_unit(const CUtensorMap *tm, const Sched &sc, int st, int kb, uint64_t pol) {
+  if (sc.mode == ROWS_ROTARY) {
+    const int hp = BM / sc.half;
+    tma_prefetch_4d(tm, kb * BK, 0, 0, st * hp, pol);
+    tma_prefetch_4d(tm, kb * BK, 0, 1, st * hp, pol);
+  } else if (sc.mode == ROWS_GATE_UP) {
+    tma_prefetch_2d(tm, kb * BK, st * BM, pol);
+    tma_prefetch_2d(tm, kb * BK, sc.F + st * BM, pol);
+  } else {
+    tma_prefetch_2d(tm, kb * BK, st * (TM * BM), pol);
+    tma_prefetch_2d(tm, kb * BK, st * (TM * BM) + BM, pol);
+  }
+}
+
 template <int NPAD, int P>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, GemmArgs a, Sched sc) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
+               const __grid_constant__ CUtensorMap tmNext, GemmArgs a, Sched sc, Sched nx) {
   using Cfg = TcCfg<NPAD, P>;
   constexpr int SW = Cfg::SW, SX = Cfg::SX, X_STAGE = Cfg::X_STAGE, X_PLANE = Cfg::X_PLANE, NBUF = Cfg::NBUF;
   constexpr int ACC = Cfg::ACC_COLS;
@@ -235,18 +251,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       for (int it = 0; it < n_units; ++it) {
         for (const int upto = min(n_units, it + SW + sc.l2_ahead); pf < upto; ++pf) {
           const int up = u0 + pf;
-          const int pst = up / KB, pkb = up - pst * KB;
-          if (sc.mode == ROWS_ROTARY) {
-            const int hp = BM / sc.half;
-            tma_prefetch_4d(&tmW, pkb * BK, 0, 0, pst * hp, pol);
-            tma_prefetch_4d(&tmW, pkb * BK, 0, 1, pst * hp, pol);
-          } else if (sc.mode == ROWS_GATE_UP) {
-            tma_prefetch_2d(&tmW, pkb * BK, pst * BM, pol);
-            tma_prefetch_2d(&tmW, pkb * BK, sc.F + pst * BM, pol);
-          } else {
-            tma_prefetch_2d(&tmW, pkb * BK, pst * (TM * BM), pol);
-            tma_prefetch_2d(&tmW, pkb * BK, pst * (TM * BM) + BM, pol);
-          }
+          prefetch_unit(&tmW, sc, up / KB, up % KB, pol);
         }
         const int u = u0 + it;
         const int st = u / KB, kb = u - st * KB;
@@ -265,6 +270,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           tma_load_2d(dst, &tmW, kb * BK, st * (TM * BM), bar, pol);
           tma_load_2d(dst + W_TILE, &tmW, kb * BK, st * (TM * BM) + BM, bar, pol);
         }
+      }
+      // all own loads are out: bring the head of the next GEMM's range of this CTA into L2
+      if (nx.l2_ahead > 0 && cta < nx.sk.G) {
+        const int v0 = sk_begin(nx.sk, cta), v1 = min(sk_begin(nx.sk, cta + 1), v0 + nx.l2_ahead);
+        for (int v = v0; v < v1; ++v) prefetch_unit(&tmNext, nx, v / nx.sk.KB, v % nx.sk.KB, pol);
       }
     }
   } else if (warp == 6) {
@@ -442,6 +452,8 @@ int sm_count() {
   return n;
 }
 
+Sched make_sched(GemmEpilogue epi, const GemmArgs &a, bool pdl);
+
 template <int NPAD, int P>
 cudaError_t launch_np(const GemmArgs &a, const Sched &sc, cudaStream_t st) {
   using Cfg = TcCfg<NPAD, P>;
@@ -456,6 +468,18 @@ cudaError_t launch_np(const GemmArgs &a, const Sched &sc, cudaStream_t st) {
   if (!make_map(&tmW, a.W, (uint64_t)a.N, (uint64_t)a.K, BM, sc.mode == ROWS_ROTARY ? (uint32_t)sc.half : 0u))
     return cudaErrorInvalidValue;
   if (!make_map(&tmX, a.X, (uint64_t)(P - 1) * a.plane_rows + a.R, (uint64_t)a.K, (uint32_t)xrows, 0)) return cudaErrorInvalidValue;
+  // the GEMM that follows (if any): its weight map and schedule, for the tail prefetch
+  CUtensorMap tmNext = tmW;
+  Sched nx{};
+  if (a.next_W && a.next_units > 0) {
+    GemmArgs b{};
+    b.W = a.next_W; b.N = a.next_N; b.K = a.next_K; b.F = a.next_F; b.dh = a.next_dh; b.plane_rows = a.plane_rows;
+    b.H = a.next_heads; b.Hkv = 0;
+    nx = make_sched((GemmEpilogue)a.next_epi, b, false);
+    nx.l2_ahead = a.next_units;
+    if (!make_map(&tmNext, b.W, (uint64_t)b.N, (uint64_t)b.K, BM, nx.mode == ROWS_ROTARY ? (uint32_t)nx.half : 0u))
+      return cudaErrorInvalidValue;
+  }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)sc.sk.G);
   cfg.blockDim = dim3(kThreads);
@@ -466,7 +490,7 @@ cudaError_t launch_np(const GemmArgs &a, const Sched &sc, cudaStream_t st) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = sc.pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<NPAD, P>, tmW, tmX, a, sc);
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<NPAD, P>, tmW, tmX, tmNext, a, sc, nx);
 }
 
 cudaError_t launch_rows(const GemmArgs &a, const Sched &sc, cudaStream_t st) {
