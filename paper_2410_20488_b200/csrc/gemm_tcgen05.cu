@@ -229,21 +229,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     for (int i = 0; i < NBUF; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {   // TMEM: one warp allocates (and later frees) the accumulator columns
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(Cfg::TMEM_COLS) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  __syncthreads();                 // barriers are initialised
+  if (sc.pdl) griddep_launch();    // the next kernel may start its own weight stream as SMs free up
+  // The two producers start at once; the warps that touch TMEM (MMA issuer and epilogue) meet on their own
+  // barrier once warp 1 has allocated (and later frees) the accumulator columns.
+  uint32_t tmem_base = 0;
+  if (warp >= 1 && warp <= 5) {
+    if (warp == 1) {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(Cfg::TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    asm volatile("bar.sync 2, 160;" ::: "memory");
+    tc_fence_after();
+    tmem_base = *tmem_slot_ptr;
   }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot_ptr;
-  if (sc.pdl) griddep_launch();   // the next kernel may start its own weight stream as SMs free up
 
   bool dead = false;
   if (warp == 0) {
     if (lane == 0) {             // ---- weight producer: does not wait for the previous kernel
       uint64_t pol;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
       // While the ring is full (typically: the activations are not there yet because the previous kernel is
       // still running) the stream goes on into L2: units up to l2_ahead beyond the ring are prefetched, so
       // HBM stays busy during the small kernels between two GEMMs and the ring later refills from L2.
