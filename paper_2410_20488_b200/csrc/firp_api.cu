@@ -232,10 +232,16 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   pending.ws = c->gemm_ws; pending.ws_rows = (int)Rp;
   const Partials none{};
   // every GEMM names its successor, whose first units it prefetches into L2 at its own tail
-  static const int next_units = [] { const char *e = getenv("FIRP_NEXT_UNITS"); return e ? atoi(e) : 5; }();
-  auto set_next = [&](GemmArgs &g, GemmEpilogue epi, const void *W, int N, int K) {
+  // (32 KB units per CTA, by the GEMM that issues the prefetch: qkv, o, gate/up, down; FIRP_NEXT_UNITS=a,b,c,d overrides)
+  static int next_units[4] = {5, 5, 5, 5};
+  static bool next_init = false;
+  if (!next_init) {
+    next_init = true;
+    if (const char *e = getenv("FIRP_NEXT_UNITS")) sscanf(e, "%d,%d,%d,%d", &next_units[0], &next_units[1], &next_units[2], &next_units[3]);
+  }
+  auto set_next = [&](GemmArgs &g, int cls, GemmEpilogue epi, const void *W, int N, int K) {
     g.next_W = (const bf16 *)W; g.next_epi = epi; g.next_N = N; g.next_K = K; g.next_F = F; g.next_heads = H + 2 * Hkv;
-    g.next_dh = dh; g.next_units = next_units;
+    g.next_dh = dh; g.next_units = next_units[cls];
   };
   for (int j = 0; j < cfg.n_layers; ++j) {
     const bool insert = (rw.k > 0 && j == ra.l);
@@ -264,7 +270,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       GemmArgs g = gemm_base(c->x, Rp * d, c->wqkv[j], (H + 2 * Hkv) * dh, d, act);
       g.H = H; g.Hkv = Hkv; g.dh = dh;
       g.l2_ahead = ahead[0];
-      set_next(g, EPI_RESIDUAL, c->wo[j], d, nq);
+      set_next(g, 0, EPI_RESIDUAL, c->wo[j], d, nq);
       g.planes = 3;   // keys and values are rounded to bf16 for the cache: their inputs carry ~24 mantissa bits
       g.rope = c->meta.rope; g.seq_ids = c->seq_ids; g.ctx_len = c->ctx_len; g.pos = c->meta.pos;
       g.q = c->q; g.q_lo_off = Rp * nq; g.kcache = kplane; g.seq_stride = c->kv_seq(); g.kv_stride = c->kv_plane(); g.max_ctx = cfg.max_ctx;
@@ -289,7 +295,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     {
       GemmArgs g = gemm_base(c->o, Rp * nq, c->wo[j], d, nq, act);
       g.l2_ahead = ahead[1];
-      set_next(g, EPI_SWIGLU, c->wgu[j], 2 * F, d);
+      set_next(g, 1, EPI_SWIGLU, c->wgu[j], 2 * F, d);
       FIRP_TIMED(KC_GEMM_O);
       FIRP_CUDA(c, launch_gemm_tc(EPI_RESIDUAL, g, pdl, st, &pending.sk)); ++nl;
     }
@@ -299,7 +305,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     {
       GemmArgs g = gemm_base(c->x, Rp * d, c->wgu[j], 2 * F, d, act);
       g.y = c->y; g.y_lo_off = Rp * F; g.F = F; g.l2_ahead = ahead[2];
-      set_next(g, EPI_RESIDUAL, c->wd[j], d, F);
+      set_next(g, 2, EPI_RESIDUAL, c->wd[j], d, F);
       Partials p = pending;
       { FIRP_TIMED(KC_GEMM_GATE_UP);
         FIRP_CUDA(c, launch_gemm_tc(EPI_SWIGLU, g, pdl, st, &p.sk)); ++nl; }
@@ -309,8 +315,8 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     {
       GemmArgs g = gemm_base(c->y, Rp * F, c->wd[j], d, F, act);
       g.l2_ahead = ahead[3];
-      if (j + 1 < cfg.n_layers) set_next(g, EPI_QKV_ROPE, c->wqkv[j + 1], (H + 2 * Hkv) * dh, d);
-      else if (ra.want_head) set_next(g, EPI_LOGITS, c->w.lm_head, cfg.vocab, d);
+      if (j + 1 < cfg.n_layers) set_next(g, 3, EPI_QKV_ROPE, c->wqkv[j + 1], (H + 2 * Hkv) * dh, d);
+      else if (ra.want_head) set_next(g, 3, EPI_LOGITS, c->w.lm_head, cfg.vocab, d);
       FIRP_TIMED(KC_GEMM_DOWN);
       FIRP_CUDA(c, launch_gemm_tc(EPI_RESIDUAL, g, pdl, st, &pending.sk)); ++nl;
     }
