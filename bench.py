@@ -87,9 +87,9 @@ def class_bytes(shape, n_ctx: float) -> dict:
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of a kernel class at the
 # c2 shape, from the ncu capture summarised under profiles/; valid only for the kernel sources whose
 # digest is recorded with it (a changed kernel reports traffic = null until it is captured again).
-NCU_TRAFFIC = {
-    "c2-llama2-7b": dict(digest="3c40eb62a7f6c388", per_launch={"gemm_gate_up": 197948160, "gemm_qkv": 108428032,
-                                                             "gemm_o": 34111488, "gemm_down": 96498688}),
+NCU_TRAFFIC = {  # dram read+write per launch; includes the ~24 MB successor head each GEMM prefetches
+    "c2-llama2-7b": dict(digest="3ff401c2cc32be01", per_launch={"gemm_gate_up": 221068288, "gemm_qkv": 129246464,
+                                                             "gemm_o": 49970688, "gemm_down": 117008128}),
 }
 
 
