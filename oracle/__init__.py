@@ -57,6 +57,8 @@ def _get_lib():
         lib.oracle_tree_prep.restype = i32
         lib.oracle_forward.argtypes = [vp, i32, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
         lib.oracle_forward.restype = i32
+        lib.oracle_forward_layers.argtypes = [vp, i32, vp, vp, i32, i32, vp, i32, i32, vp, vp, vp, i32, vp, vp]
+        lib.oracle_forward_layers.restype = i32
         lib.oracle_verify.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
         lib.oracle_verify.restype = i32
         lib.oracle_next_tree.argtypes = [vp, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp]
@@ -181,9 +183,14 @@ class Oracle:
         return out
 
     # -- the step ------------------------------------------------------------
-    def forward(self, tokens, parents, k: int, l: int, anchor: int = 0, seq: int = 0,
+    def forward(self, tokens, parents, k: int, l, anchor: int = 0, seq: int = 0,
                 logit_row0: int = 0, want_h_at_l: bool = False):
+        """l: one insertion layer for all k prediction steps, or a non-decreasing sequence of k
+        layers t_1..t_k (Section 3.3); with a sequence, want_h_at_l returns `h_ins` [k, d], every
+        pseudo row as it was appended, instead of the residual stream at one layer."""
         tokens, parents = _i32(tokens), _i32(parents)
+        if not np.isscalar(l):
+            return self._forward_layers(tokens, parents, k, _i32(l), anchor, seq, logit_row0, want_h_at_l)
         T = tokens.size
         M = T + k
         s = self.shape
@@ -198,6 +205,25 @@ class Oracle:
         out = dict(logits=logits, depth=depth, mask=mask, pos=depth + self.context_len(seq))
         if want_h_at_l:
             out["h_at_l"] = h_at_l
+        return out
+
+    def _forward_layers(self, tokens, parents, k, layers, anchor, seq, logit_row0, want_h_ins):
+        if layers.size != k:
+            raise ValueError("need one insertion layer per prediction step")
+        T = tokens.size
+        M = T + k
+        s = self.shape
+        logits = np.zeros((M, s.V), np.float32)
+        depth = np.zeros(M, np.int32)
+        mask = np.zeros((M, M), np.uint8)
+        h_ins = np.zeros((k, s.d), np.float32) if want_h_ins else None
+        rc = self.lib.oracle_forward_layers(self.h, seq, _ptr(tokens), _ptr(parents), T, k, _ptr(layers), anchor,
+                                            logit_row0, _ptr(logits), _ptr(depth), _ptr(mask), -1, None, _ptr(h_ins))
+        if rc != 0:
+            raise ValueError("oracle_forward_layers failed: %d" % rc)
+        out = dict(logits=logits, depth=depth, mask=mask, pos=depth + self.context_len(seq))
+        if want_h_ins:
+            out["h_ins"] = h_ins
         return out
 
     def verify(self, logits, tokens, parents):

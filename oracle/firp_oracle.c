@@ -28,7 +28,11 @@
  *     each token's positional index n + depth, and a row attends to the
  *     committed prefix plus its own ancestors and itself.
  *   - Pseudo hidden states (Section 3.2, Section 3.3 Eq. 3): at the input of
- *     layer l, k rows h~_i = W_i h[anchor] + b_i are appended.  Pseudo row i
+ *     layer l, k rows h~_i = W_i h[anchor] + b_i are appended.  Section 3.3
+ *     gives every prediction step i its own layer t_i (Section 4 "Setup" uses
+ *     15/20/25 and 25/30/35): oracle_forward_layers() appends row i at the
+ *     input of layer t_i, t_1 <= ... <= t_k, from the anchor's residual there;
+ *     oracle_forward() is the case t_1 = ... = t_k = l.  Pseudo row i
  *     stands for position pos[anchor] + i; it sees the prefix, the anchor's
  *     ancestors and the anchor, the earlier pseudo rows ("No masked" setting
  *     of Section 4.3) and itself (Section 3.3, paragraph after Eq. 3).
@@ -199,23 +203,29 @@ int32_t oracle_tree_prep(const int32_t *parents, int32_t T, int32_t k, int32_t a
 }
 
 /*
- * One forward pass over the T tree rows (+ k pseudo rows from layer l on) of
+ * One forward pass over the T tree rows (+ pseudo row i from layer tl[i] on) of
  * sequence `seq`, on top of its committed cache of n positions.  Cache slots
- * n..n+T+k-1 receive the rows' keys/values (scratch until oracle_commit).
+ * n..n+T+k-1 receive the rows' keys/values (scratch until oracle_commit; a
+ * pseudo row has none below its own layer).
  *
+ * tl          [k] insertion layer of each prediction step, non-decreasing, 0 <= tl[i] < L
  * logits      [(T+k)][V] fp32 out; rows < logit_row0 are skipped (left untouched)
- * h_at_l      optional [(T+k)][d]: residual stream entering layer l, after insertion
- * Returns 0, -1 malformed tree, -2 capacity.
+ * dump_layer, h_dump   optional [(T+k)][d]: residual stream entering layer dump_layer,
+ *             after that layer's insertions (rows not yet alive are zero)
+ * h_ins       optional [k][d]: every pseudo row as it was appended
+ * Returns 0, -1 malformed tree or layers, -2 capacity.
  */
-int32_t oracle_forward(void *hnd, int32_t seq, const int32_t *tokens, const int32_t *parents,
-                       int32_t T, int32_t k, int32_t l, int32_t anchor, int32_t logit_row0,
-                       float *logits, int32_t *depth_out, uint8_t *mask_out, float *h_at_l) {
+int32_t oracle_forward_layers(void *hnd, int32_t seq, const int32_t *tokens, const int32_t *parents,
+                              int32_t T, int32_t k, const int32_t *tl, int32_t anchor, int32_t logit_row0,
+                              float *logits, int32_t *depth_out, uint8_t *mask_out,
+                              int32_t dump_layer, float *h_dump, float *h_ins) {
   oracle_t *o = (oracle_t *)hnd;
   const oracle_cfg *c = &o->cfg;
   const oracle_weights *w = &o->w;
   const int d = c->d, H = c->H, Hkv = c->Hkv, dh = c->dh, F = c->F, V = c->V;
   const int nq = H * dh, nkv = Hkv * dh, M = T + k, n = o->n[seq];
-  if (k < 0 || k > c->n_maps || (k > 0 && (l < 0 || l >= c->L))) return -1;
+  if (k < 0 || k > c->n_maps) return -1;
+  for (int i = 0; i < k; ++i) if (tl[i] < 0 || tl[i] >= c->L || (i > 0 && tl[i] < tl[i - 1])) return -1;
   if (n + M > c->max_ctx) return -2;
 
   int32_t *ext_parent = (int32_t *)malloc(sizeof(int32_t) * M);
@@ -238,18 +248,18 @@ int32_t oracle_forward(void *hnd, int32_t seq, const int32_t *tokens, const int3
   for (int v = 0; v < T; ++v)
     for (int cc = 0; cc < d; ++cc) h[(size_t)v * d + cc] = bf16f(w->embed[(size_t)tokens[v] * d + cc]);
 
-  int rows = T;  /* rows alive: T before layer l, T+k from layer l on */
+  int rows = T;  /* rows alive: the tree rows and the pseudo rows whose layer has been reached */
   for (int j = 0; j < c->L; ++j) {
-    if (k > 0 && j == l) {
-      /* Eq. 3: h~_i = W_i h[anchor] + b_i, appended as rows T..T+k-1 */
-      for (int i = 0; i < k; ++i) {
-        float *dst = h + (size_t)(T + i) * d;
-        linear(w->pred_w + (size_t)i * d * d, h + (size_t)anchor * d, d, dst, d, 1, d, d);
-        if (w->pred_b) for (int cc = 0; cc < d; ++cc) dst[cc] += bf16f(w->pred_b[(size_t)i * d + cc]);
-      }
-      rows = M;
+    for (int i = 0; i < k; ++i) {
+      if (tl[i] != j) continue;
+      /* Eq. 3: h~_i = W_i h[anchor] + b_i on the residual entering layer t_i, appended as row T+i */
+      float *dst = h + (size_t)(T + i) * d;
+      linear(w->pred_w + (size_t)i * d * d, h + (size_t)anchor * d, d, dst, d, 1, d, d);
+      if (w->pred_b) for (int cc = 0; cc < d; ++cc) dst[cc] += bf16f(w->pred_b[(size_t)i * d + cc]);
+      if (h_ins) memcpy(h_ins + (size_t)i * d, dst, sizeof(float) * d);
+      rows = T + i + 1;
     }
-    if (h_at_l && j == l) memcpy(h_at_l, h, sizeof(float) * (size_t)M * d);
+    if (h_dump && j == dump_layer) memcpy(h_dump, h, sizeof(float) * (size_t)M * d);
 
     float *kc = o->kc[seq] + (size_t)j * c->max_ctx * nkv;
     float *vc = o->vc[seq] + (size_t)j * c->max_ctx * nkv;
@@ -320,6 +330,17 @@ int32_t oracle_forward(void *hnd, int32_t seq, const int32_t *tokens, const int3
   free(ext_parent); free(depth); free(mask);
   free(h); free(x); free(q); free(att); free(delta); free(gate); free(up); free(p);
   return 0;
+}
+
+/* The single-layer case of the paper's overview (Section 3.2): every prediction step at layer l. */
+int32_t oracle_forward(void *hnd, int32_t seq, const int32_t *tokens, const int32_t *parents,
+                       int32_t T, int32_t k, int32_t l, int32_t anchor, int32_t logit_row0,
+                       float *logits, int32_t *depth_out, uint8_t *mask_out, float *h_at_l) {
+  int32_t tl[64];
+  if (k < 0 || k > 64) return -1;
+  for (int i = 0; i < k; ++i) tl[i] = l;
+  return oracle_forward_layers(hnd, seq, tokens, parents, T, k, tl, anchor, logit_row0, logits, depth_out, mask_out,
+                               l, h_at_l, NULL);
 }
 
 /* argmax with ties to the lowest index */

@@ -75,21 +75,31 @@ def hf_kv(model, token_ids):
 
 def hf_logits_with_replaced_rows(model, token_ids, layer, first_row, maps_w, maps_b, anchor_row):
     """Causal forward in which, at the input of decoder layer `layer`, rows
-    first_row.. are replaced by W_i h[anchor_row] + b_i (i = 0..len(maps_w)-1)."""
-    def hook(module, args, kwargs):
-        hs = args[0] if args else kwargs["hidden_states"]
-        hs = hs.clone()
-        src = hs[0, anchor_row]
-        for i, W in enumerate(maps_w):
-            hs[0, first_row + i] = torch.from_numpy(W) @ src + torch.from_numpy(maps_b[i])
-        if args:
-            return (hs,) + tuple(args[1:]), kwargs
-        kwargs = dict(kwargs)
-        kwargs["hidden_states"] = hs
-        return args, kwargs
+    first_row.. are replaced by W_i h[anchor_row] + b_i (i = 0..len(maps_w)-1).
+    `layer` may be a sequence with one layer per row: row first_row + i is then
+    replaced at the input of layer[i] (what it held before is never read by a row
+    that matters, because the sequence is causal and the layers do not decrease)."""
+    layers = [int(layer)] * len(maps_w) if np.isscalar(layer) else [int(t) for t in layer]
+    assert len(layers) == len(maps_w) and layers == sorted(layers)
 
-    handle = model.model.layers[layer].register_forward_pre_hook(hook, with_kwargs=True)
+    def make_hook(at):
+        def hook(module, args, kwargs):
+            hs = args[0] if args else kwargs["hidden_states"]
+            hs = hs.clone()
+            src = hs[0, anchor_row]
+            for i, W in enumerate(maps_w):
+                if layers[i] == at:
+                    hs[0, first_row + i] = torch.from_numpy(W) @ src + torch.from_numpy(maps_b[i])
+            if args:
+                return (hs,) + tuple(args[1:]), kwargs
+            kwargs = dict(kwargs)
+            kwargs["hidden_states"] = hs
+            return args, kwargs
+        return hook
+
+    handles = [model.model.layers[at].register_forward_pre_hook(make_hook(at), with_kwargs=True) for at in sorted(set(layers))]
     try:
         return hf_logits(model, token_ids)
     finally:
-        handle.remove()
+        for h in handles:
+            h.remove()

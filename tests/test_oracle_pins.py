@@ -9,6 +9,8 @@
   P7  forced-accept mode accepts the full depth every step
   P8  the pseudo chain == a causal forward whose rows are replaced at layer l
   P9  predictor size k*d^2 equals the draft-module sizes printed in the paper's Table 1
+  P10 one insertion layer per prediction step (Section 3.3): the chain == a causal forward whose row i is
+      replaced at layer t_i; step i does not depend on the layers of later steps; W = I closed form
 plus hand-worked cases for the mask, the acceptance walk, the tie rules and the next tree.
 """
 import os
@@ -177,6 +179,64 @@ def test_p8_pseudo_chain_is_causal_forward_with_replaced_rows(c1, c1_weights, hf
     ids = list(prompt) + [int(tokens[0])] + [0] * k
     ref = hf_logits_with_replaced_rows(hf, ids, l, prompt.size + 1, list(Wf), list(bf), prompt.size)
     assert np.abs(out["logits"][8:] - ref[prompt.size + 1:]).max() < 1e-5
+
+
+# ---------------------------------------------------------------- P10
+@pytest.fixture(scope="module")
+def c1_deep():
+    shape = si.scaled(si.CONFIGS["c1"], L=4, l=1)
+    return shape, si.all_weights(shape)
+
+
+@pytest.mark.parametrize("layers", [(0, 1, 3), (1, 1, 2), (2, 3, 3), (0, 0, 0)])
+def test_p10_per_step_layers_chain_is_causal_forward_with_rows_replaced_at_their_layers(c1_deep, layers):
+    shape, weights = c1_deep
+    hf4 = build_hf_llama(shape, weights)
+    k = 3
+    prompt = si.prompt(shape, length=13)
+    Wf = si.bf16_bits_to_f32(weights["pred_w"]).astype(np.float64)
+    bf = np.zeros((k, shape.d))
+    o = fresh(shape, weights)
+    o.forward(prompt, si.chain_template(prompt.size), 0, 0)
+    o.commit(np.arange(prompt.size))
+    tokens, parents = si.random_tokens(shape, 8, 9), si.tree_template(8)
+    out = o.forward(tokens, parents, k, list(layers), anchor=0)
+    ids = list(prompt) + [int(tokens[0])] + [0] * k
+    ref = hf_logits_with_replaced_rows(hf4, ids, layers, prompt.size + 1, list(Wf), list(bf), prompt.size)
+    assert np.abs(out["logits"][8:] - ref[prompt.size + 1:]).max() < 1e-5
+    # the tree rows are those of a plain tree step
+    plain = o.forward(tokens, parents, 0, 0)["logits"]
+    assert np.array_equal(out["logits"][:8], plain)
+    # the same layer for every step is the single-layer call
+    if len(set(layers)) == 1:
+        assert np.array_equal(out["logits"], o.forward(tokens, parents, k, layers[0])["logits"])
+
+
+def test_p10_a_step_ignores_the_layers_of_later_steps_and_identity_maps_copy_the_anchor(c1_deep):
+    shape, weights = c1_deep
+    d, k = shape.d, 3
+    prompt = si.prompt(shape)
+    tokens, parents = si.random_tokens(shape, 8, 4), si.tree_template(8)
+    o = fresh(shape, weights)
+    o.prefill(prompt, 0, 0, None)
+    a = o.forward(tokens, parents, k, [1, 2, 3])["logits"]
+    b = o.forward(tokens, parents, k, [1, 3, 3])["logits"]
+    c = o.forward(tokens, parents, 1, 1)["logits"]
+    assert np.array_equal(a[8], b[8]) and np.array_equal(a[8], c[8])          # step 1 sees no later step
+    assert not np.array_equal(a[9], b[9])                                      # step 2 moved from layer 2 to 3
+    with pytest.raises(ValueError):
+        o.forward(tokens, parents, k, [2, 1, 3])                               # layers must not decrease
+    with pytest.raises(ValueError):
+        o.forward(tokens, parents, k, [1, 2, 4])                               # layer outside the decoder
+    # W = I, b = 0: pseudo row i is the anchor's residual entering layer t_i
+    wI = with_maps(weights, np.stack([np.eye(d, dtype=np.float32)] * k), np.zeros((k, d), np.float32))
+    oI = fresh(shape, wI)
+    oI.prefill(prompt, 0, 0, None)
+    for anchor in (0, 3):
+        h_ins = oI.forward(tokens, parents, k, [0, 2, 3], anchor=anchor, want_h_at_l=True)["h_ins"]
+        for i, t in enumerate((0, 2, 3)):
+            h_t = oI.forward(tokens, parents, 0, t, want_h_at_l=True)["h_at_l"]   # k = 0: plain residual at layer t
+            assert np.array_equal(h_ins[i], h_t[anchor])
 
 
 # ---------------------------------------------------------------- P5
