@@ -39,11 +39,22 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", help="c1 | c2 | c3 | c4:T:n (sweep point on the c2 weights)")
     ap.add_argument("--layers", type=int, default=0, help="debug only: truncate the decoder (marks the line invalid)")
+    ap.add_argument("--insert-layers", default="", help="one insertion layer per prediction step, e.g. 15,20,25 "
+                    "(the paper's 7B setting); default: the workload's single layer l")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-kernel-times", action="store_true", help="skip the per-kernel event-timed pass")
     ap.add_argument("--sweep", action="store_true", help="config-4 sweep on the c2 weights: T x context, one JSON line per point")
     return ap.parse_args()
+
+
+# One insertion layer per prediction step (--insert-layers), or None: the workload's single layer l.
+INSERT_LAYERS = None
+
+
+def ins_l(shape):
+    """What the step and prefill calls get as `l`: the per-step layers if given, else shape.l."""
+    return list(INSERT_LAYERS) if INSERT_LAYERS else shape.l
 
 
 def pick_shape(name: str, layers: int):
@@ -67,7 +78,10 @@ def algorithmic_bytes(shape, n_ctx: float, batch: int = 1) -> dict:
     kv_row = 2 * 2 * s.n_kv * batch               # K and V, bf16, every sequence
     kv_read = kv_write = 0
     for j in range(s.L):
-        M = M_hi if (s.k > 0 and j >= s.l) else M_lo
+        if INSERT_LAYERS:
+            M = s.T + sum(1 for t in INSERT_LAYERS if t <= j)
+        else:
+            M = M_hi if (s.k > 0 and j >= s.l) else M_lo
         kv_read += kv_row * (n_ctx + M)
         kv_write += kv_row * M
     return dict(weights=weights, kv_read=kv_read, kv_write=kv_write, embed=2 * s.T * s.d * batch,
@@ -110,7 +124,7 @@ def kernel_times(eng, shape, parents, tokens, out, steps, n_ctx, peak_gbs, peak_
     seq_ids = seq_ids or [0]
     eng.profile(True)
     for _ in range(steps):
-        eng.step(tokens, parents, shape.k, shape.l, out, seq_ids=seq_ids, n_seq=len(seq_ids))
+        eng.step(tokens, parents, shape.k, ins_l(shape), out, seq_ids=seq_ids, n_seq=len(seq_ids))
         eng.commit(len(seq_ids), seq_ids=seq_ids)
         tokens = out.next_tree_tokens
     prof = eng.profile_read()
@@ -212,12 +226,12 @@ def time_oracle(shape, weights, steps: int, warmup: int, n_ctx: int = 32):
     import synth_inputs as si
     parents = si.tree_template(shape.T)
     orc = oracle.Oracle(shape, weights, max_ctx=n_ctx + (steps + warmup + 1) * (shape.k + 1) + shape.T + shape.k + 8)
-    r = orc.prefill(si.prompt(shape, length=n_ctx), shape.k, shape.l, parents)
+    r = orc.prefill(si.prompt(shape, length=n_ctx), shape.k, ins_l(shape), parents)
     tokens = r["next_tokens"]
     emitted, t_total = 0, 0.0
     for i in range(warmup + steps):
         t0 = time.perf_counter()
-        out = orc.step(tokens, parents, shape.k, shape.l)
+        out = orc.step(tokens, parents, shape.k, ins_l(shape))
         orc.commit(out["path"])
         dt = time.perf_counter() - t0
         if i >= warmup:
@@ -244,12 +258,12 @@ def run_reference(args, shape):
     weights = si.all_weights(shape)
     steps, warmup = max(1, min(args.steps, 3)), min(args.warmup, 1)
     tps, ms = time_oracle(shape, weights, steps, warmup)
-    sample = "%d oracle steps (+%d warm-up) of T=%d,k=%d,l=%d over all %d layers on a 32-token context" % (
-        steps, warmup, shape.T, shape.k, shape.l, shape.L)
+    sample = "%d oracle steps (+%d warm-up) of T=%d,k=%d,l=%s over all %d layers on a 32-token context" % (
+        steps, warmup, shape.T, shape.k, ins_l(shape), shape.L)
     line = dict(metric=METRIC, value=tps, unit=UNIT, n_gpus=args.gpus, steps=steps, warmup=warmup, ms_per_step=ms,
                 higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32 storage, f64 accumulation",
                 data="synthetic", impl="reference",
-                config=dict(workload=shape.name, T=shape.T, k=shape.k, l=shape.l, context_start=shape.prompt_len,
+                config=dict(workload=shape.name, T=shape.T, k=shape.k, l=ins_l(shape), context_start=shape.prompt_len,
                             batch=1, sample="oracle steps on a 32-token context instead of %d tokens (its prefill "
                             "cost grows with the context; the step's GEMM work does not)" % shape.prompt_len),
                 cpu_baseline=dict(value=tps, unit=UNIT, cores=host_cores(), kind="oracle", sample=sample),
@@ -308,6 +322,11 @@ def run_sweep(args, shape, weights, dev, rank):
 def main():
     args = parse()
     shape = pick_shape(args.workload, args.layers)
+    if args.insert_layers:
+        global INSERT_LAYERS
+        INSERT_LAYERS = [int(t) for t in args.insert_layers.split(",")]
+        if len(INSERT_LAYERS) != shape.k or INSERT_LAYERS != sorted(INSERT_LAYERS) or not all(0 <= t < shape.L for t in INSERT_LAYERS):
+            raise SystemExit("--insert-layers needs k non-decreasing layers inside the decoder")
     if args.impl == "reference":
         return run_reference(args, shape)
 
@@ -350,7 +369,7 @@ def main():
     for b_i, n in enumerate(lengths):
         prompt = torch.from_numpy(si.prompt(shape, seq=rank * B + b_i, length=n)).to(dev)
         pout = eng.new_out(1, 1, shape.k, T_next=T_next, want_logits=False)
-        eng.prefill(b_i, prompt, shape.k, shape.l, parents if shape.k > 0 else None, pout)
+        eng.prefill(b_i, prompt, shape.k, ins_l(shape), parents if shape.k > 0 else None, pout)
         first[b_i] = pout.next_tree_tokens[0]
     torch.cuda.synchronize()
     n_start = sum(eng.context_len(b_i) for b_i in range(B)) / B
@@ -367,7 +386,7 @@ def main():
     def one_step(i, tokens):
         nonlocal launches
         o = outs[i & 1]
-        eng.step(tokens, parents, shape.k, shape.l, o, seq_ids=seq_ids, n_seq=B)
+        eng.step(tokens, parents, shape.k, ins_l(shape), o, seq_ids=seq_ids, n_seq=B)
         launches += eng.launches()
         eng.commit(B, seq_ids=seq_ids)
         launches += eng.launches()
@@ -409,7 +428,7 @@ def main():
         e0.record()
         for i in range(K):
             d_tokens.copy_(h_tokens, non_blocking=True)
-            eng.step(d_tokens, parents, shape.k, shape.l, o, seq_ids=seq_ids, n_seq=B)
+            eng.step(d_tokens, parents, shape.k, ins_l(shape), o, seq_ids=seq_ids, n_seq=B)
             eng.commit(B, seq_ids=seq_ids)
             h_acc.copy_(o.accepted_tokens, non_blocking=True)
             h_n.copy_(o.n_accepted, non_blocking=True)
@@ -447,7 +466,7 @@ def main():
     line = dict(metric=METRIC, value=units / (ms_max * 1e-3), unit=UNIT, n_gpus=world, steps=K, warmup=W,
                 ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                 data="synthetic", gpu_launches=launches,
-                config=dict(workload=shape.name, T=shape.T, k=shape.k, l=shape.l, context_start=n_start,
+                config=dict(workload=shape.name, T=shape.T, k=shape.k, l=ins_l(shape), context_start=n_start,
                             context_end=n_end, batch=B, l2="inputs_larger_than_l2 (%.1f GB of weights per step)" %
                             (ab["weights"] / 1e9), parallelism="replicas x%d" % world,
                             mode="free-running greedy (random weights accept ~0 drafts per step)"),
@@ -472,8 +491,8 @@ def main():
         cb_steps = 1
         tps, ms = time_oracle(shape, weights, cb_steps, 0)
         line["cpu_baseline"] = dict(value=tps, unit=UNIT, cores=host_cores(), kind="oracle", ms_per_step=ms,
-                                    sample="%d oracle step of T=%d,k=%d,l=%d over all %d layers on a 32-token context "
-                                           "(plus its 32-token prefill, untimed)" % (cb_steps, shape.T, shape.k, shape.l, shape.L))
+                                    sample="%d oracle step of T=%d,k=%d,l=%s over all %d layers on a 32-token context "
+                                           "(plus its 32-token prefill, untimed)" % (cb_steps, shape.T, shape.k, ins_l(shape), shape.L))
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -135,6 +135,23 @@ int firp_step(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_
               void *stream);
 
 /*
+ * The same two calls with one insertion layer per prediction step (Section 3.3: step i is
+ * trained on, and its pseudo hidden state predicted at, its own layer t_i; Section 4 "Setup"
+ * uses 15/20/25 for the 7B and 25/30/35 for the 13B models).
+ *   layers   HOST [k], non-decreasing, 0 <= layers[i] < n_layers: pseudo row i is appended at the
+ *            input of layer layers[i] as W_i h[anchor] + b_i on the anchor's residual entering that
+ *            layer, and takes part in every layer from there on (it has no keys/values below it).
+ * layers[i] = l for every i is firp_step / firp_prefill with that l.  FIRP_ERR_BAD_ARG if the
+ * layers decrease or leave the decoder; everything else as in the calls above.
+ */
+int firp_prefill_layers(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int32_t P, int32_t k,
+                        const int32_t *layers, const int32_t *next_parents, int32_t T_next,
+                        const firp_step_out *out, void *stream);
+int firp_step_layers(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
+                     const int32_t *tree_parents, int32_t T, int32_t k, const int32_t *layers,
+                     const firp_step_out *out, void *stream);
+
+/*
  * Commit after a step: for each sequence move the cache rows of path[j] to slot n + j
  * (every layer, K and V) and advance n by path_len.  path (HOST [n_seq][max_depth+1]) and
  * path_len (HOST [n_seq]) give an explicit path (strictly increasing, path[0] = 0); NULL

@@ -45,7 +45,7 @@ class StepOutC(ctypes.Structure):
 EXPORTS = ("firp_create", "firp_destroy", "firp_last_error", "firp_workspace_bytes", "firp_kv_bytes",
            "firp_bind_buffers", "firp_init_weights", "firp_prefill", "firp_step", "firp_kv_commit",
            "firp_context_len", "firp_set_context_len", "firp_last_launch_count", "firp_profile_enable",
-           "firp_profile_read", "firp_kernel_class_name", "firp_topb_static")
+           "firp_profile_read", "firp_kernel_class_name", "firp_topb_static", "firp_prefill_layers", "firp_step_layers")
 
 
 def lib_path() -> str:
@@ -74,6 +74,8 @@ def load_library():
     lib.firp_init_weights.argtypes = [vp, ctypes.POINTER(Weights)]
     lib.firp_prefill.argtypes = [vp, i32, vp, i32, i32, i32, vp, i32, ctypes.POINTER(StepOutC), vp]
     lib.firp_step.argtypes = [vp, i32, vp, vp, vp, i32, i32, i32, ctypes.POINTER(StepOutC), vp]
+    lib.firp_prefill_layers.argtypes = [vp, i32, vp, i32, i32, vp, vp, i32, ctypes.POINTER(StepOutC), vp]
+    lib.firp_step_layers.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp, ctypes.POINTER(StepOutC), vp]
     lib.firp_kv_commit.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.firp_context_len.argtypes = [vp, i32, ctypes.POINTER(i32), vp]
     lib.firp_set_context_len.argtypes = [vp, i32, i32, vp]
@@ -141,6 +143,27 @@ def firp_prefill(ctx, seq: int, d_prompt_ptr: int, P: int, k: int, l: int, next_
     arr, ptr = _host_i32(next_parents)
     _check(ctx, load_library().firp_prefill(ctx, seq, d_prompt_ptr, P, k, l, ptr, 0 if arr is None else arr.size,
                                             ctypes.byref(out) if out is not None else None, stream))
+
+
+def firp_prefill_layers(ctx, seq: int, d_prompt_ptr: int, P: int, k: int, layers, next_parents, out: StepOutC,
+                        stream: int = 0):
+    arr, ptr = _host_i32(next_parents)
+    lay, lay_ptr = _host_i32(layers)
+    if lay is None or lay.size != k:
+        raise ValueError("need one insertion layer per prediction step")
+    _check(ctx, load_library().firp_prefill_layers(ctx, seq, d_prompt_ptr, P, k, lay_ptr, ptr, 0 if arr is None else arr.size,
+                                                   ctypes.byref(out) if out is not None else None, stream))
+
+
+def firp_step_layers(ctx, n_seq: int, seq_ids, d_tokens_ptr: int, tree_parents, T: int, k: int, layers, out: StepOutC,
+                     stream: int = 0):
+    ids, ids_ptr = _host_i32(seq_ids)
+    par, par_ptr = _host_i32(tree_parents)
+    lay, lay_ptr = _host_i32(layers)
+    if lay is None or lay.size != k:
+        raise ValueError("need one insertion layer per prediction step")
+    _check(ctx, load_library().firp_step_layers(ctx, n_seq, ids_ptr, d_tokens_ptr, par_ptr, T, k, lay_ptr,
+                                                ctypes.byref(out) if out is not None else None, stream))
 
 
 def firp_step(ctx, n_seq: int, seq_ids, d_tokens_ptr: int, tree_parents, T: int, k: int, l: int, out: StepOutC,
@@ -273,13 +296,16 @@ class FirpEngine:
         return StepOut(self.torch, self.device, n_seq, T, k, self.shape.V, self.S, self.B, T_next, want_logits)
 
     def prefill(self, seq, d_prompt, k, l, next_parents, out: StepOut):
-        firp_prefill(self.ctx, seq, d_prompt.data_ptr(), d_prompt.numel(), k, l, next_parents,
-                     out.c if out is not None else None, self.stream)
+        """l: one insertion layer, or a sequence of k layers (one per prediction step)."""
+        fn = firp_prefill if np.isscalar(l) else firp_prefill_layers
+        fn(self.ctx, seq, d_prompt.data_ptr(), d_prompt.numel(), k, l, next_parents,
+           out.c if out is not None else None, self.stream)
 
     def step(self, d_tokens, parents, k, l, out: StepOut, seq_ids=None, n_seq=1):
+        """l: one insertion layer, or a sequence of k layers (one per prediction step)."""
         T = len(parents)
-        firp_step(self.ctx, n_seq, seq_ids, d_tokens.data_ptr(), parents, T, k, l, out.c if out is not None else None,
-                  self.stream)
+        fn = firp_step if np.isscalar(l) else firp_step_layers
+        fn(self.ctx, n_seq, seq_ids, d_tokens.data_ptr(), parents, T, k, l, out.c if out is not None else None, self.stream)
 
     def commit(self, n_seq=1, seq_ids=None, path=None, path_len=None):
         if path is not None:

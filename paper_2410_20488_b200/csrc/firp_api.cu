@@ -183,7 +183,7 @@ int upload_i32(firp_ctx *ctx, int32_t *dst, const int32_t *src, int n, std::vect
 struct RunArgs {
   Rows rw;
   const int32_t *d_tokens;   // [n_seq][T]
-  int l;
+  int tl[8];                 // insertion layer of each prediction step (non-decreasing), Section 3.3
   bool want_head;            // run final norm + lm-head + top-B + accept
   int prefill_last_row;      // -1: verify walk
   int T_next;
@@ -243,27 +243,34 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     g.next_W = (const bf16 *)W; g.next_epi = epi; g.next_N = N; g.next_K = K; g.next_F = F; g.next_heads = H + 2 * Hkv;
     g.next_dh = dh; g.next_units = next_units[cls];
   };
+  int alive = 0;   // pseudo rows appended below this layer
   for (int j = 0; j < cfg.n_layers; ++j) {
-    const bool insert = (rw.k > 0 && j == ra.l);
-    const int act = (rw.k > 0 && j >= ra.l) ? rw.Ms : rw.T;   // rows alive in this layer
+    int ins = 0;     // prediction steps whose layer this is
+    while (alive + ins < rw.k && ra.tl[alive + ins] == j) ++ins;
+    const bool insert = ins > 0;
     // the rows that took part in the last residual GEMM get its pending sums; new pseudo rows have none
-    const int carried = insert ? rw.T : act;
+    const int carried = rw.T + alive;
+    const int act = carried + ins;                             // rows alive in this layer
     { FIRP_TIMED(KC_RMSNORM);
       FIRP_CUDA(c, launch_rmsnorm(rw, 0, carried, c->h, pending, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, 3, c->ss, pdl, st)); ++nl; }
     pending.sk.U = 0;
     if (insert) {   // Eq. 3 on the raw (now complete) residual row of the root, then the norm of the new rows
-      { FIRP_TIMED(KC_PSEUDO_PROJ);      // the k maps as one [k d][d] GEMM on the anchor rows (one row per sequence)
+      { FIRP_TIMED(KC_PSEUDO_PROJ);      // this layer's maps as one [ins d][d] GEMM on the anchor rows (one row per sequence)
         launch_root_split(rw, c->h, d, c->xp, (size_t)kMaxSeq * d, pdl, st); ++nl;
         GemmArgs g{};
         g.X = c->xp; g.x_lo_off = (size_t)kMaxSeq * d; g.plane_rows = kMaxSeq; g.planes = 2; g.err = c->dev_status;
-        g.W = (const bf16 *)c->w.pred_w; g.R = rw.n_seq; g.N = rw.k * d; g.K = d; g.rw = rw; g.rows_active = rw.Ms;
-        g.ws = c->gemm_ws; g.l2_ahead = 48; g.h_rows = c->h; g.pred_b = (const bf16 *)c->w.pred_b;
+        g.W = (const bf16 *)c->w.pred_w + (size_t)alive * d * d; g.R = rw.n_seq; g.N = ins * d; g.K = d; g.rw = rw;
+        g.rows_active = act;
+        g.ws = c->gemm_ws; g.l2_ahead = 48;
+        g.h_rows = c->h + (size_t)alive * d;     // map i of this GEMM fills pseudo row alive + i
+        g.pred_b = c->w.pred_b ? (const bf16 *)c->w.pred_b + (size_t)alive * d : nullptr;
         Partials p = pending;
         FIRP_CUDA(c, launch_gemm_tc(EPI_PSEUDO, g, pdl, st, &p.sk)); ++nl;
         p.ws_rows = kMaxSeq;
         FIRP_CUDA(c, launch_gemm_finish(EPI_PSEUDO, p, g, pdl, st)); ++nl; }
       FIRP_TIMED(KC_RMSNORM);
-      FIRP_CUDA(c, launch_rmsnorm(rw, rw.T, rw.Ms, c->h, none, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, 3, c->ss, pdl, st)); ++nl;
+      FIRP_CUDA(c, launch_rmsnorm(rw, carried, act, c->h, none, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, 3, c->ss, pdl, st)); ++nl;
+      alive += ins;
     }
     bf16 *kplane = c->kv + (size_t)j * c->kv_layer();
     {
@@ -458,8 +465,26 @@ static int check_seq_ids(firp_ctx *ctx, int n_seq, const int32_t *seq_ids, std::
   return FIRP_OK;
 }
 
+// layers of the prediction steps: non-decreasing and inside the decoder
+static int check_layers(firp_ctx *ctx, int k, const int32_t *layers) {
+  if (k > 0 && !layers) return fail(ctx, FIRP_ERR_BAD_ARG, "NULL insertion layers");
+  for (int i = 0; i < k; ++i) {
+    if (layers[i] < 0 || layers[i] >= ctx->cfg.n_layers) return fail(ctx, FIRP_ERR_BAD_ARG, "insertion layer %d outside 0..n_layers-1", layers[i]);
+    if (i > 0 && layers[i] < layers[i - 1]) return fail(ctx, FIRP_ERR_BAD_ARG, "insertion layers must not decrease");
+  }
+  return FIRP_OK;
+}
+
 int firp_step(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
               const int32_t *tree_parents, int32_t T, int32_t k, int32_t l, const firp_step_out *out, void *stream) {
+  int32_t layers[8];
+  for (int i = 0; i < 8; ++i) layers[i] = l;
+  return firp_step_layers(ctx, n_seq, seq_ids, d_tree_tokens, tree_parents, T, k, layers, out, stream);
+}
+
+int firp_step_layers(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
+                     const int32_t *tree_parents, int32_t T, int32_t k, const int32_t *layers, const firp_step_out *out,
+                     void *stream) {
   int rc = check_ready(ctx);
   if (rc) return rc;
   const firp_model_cfg &cfg = ctx->cfg;
@@ -467,7 +492,7 @@ int firp_step(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_
   if (!d_tree_tokens || !tree_parents) return fail(ctx, FIRP_ERR_BAD_ARG, "NULL tokens or parents");
   if (T < 1 || T > cfg.max_tree) return fail(ctx, FIRP_ERR_CAPACITY, "T %d outside 1..max_tree", T);
   if (k < 0 || k > cfg.max_k || k > ctx->w.n_maps) return fail(ctx, FIRP_ERR_CAPACITY, "k %d exceeds max_k or the loaded maps", k);
-  if (k > 0 && (l < 0 || l >= cfg.n_layers)) return fail(ctx, FIRP_ERR_BAD_ARG, "insertion layer %d outside 0..n_layers-1", l);
+  if ((rc = check_layers(ctx, k, layers))) return rc;
   std::vector<int32_t> ids;
   if ((rc = check_seq_ids(ctx, n_seq, seq_ids, ids))) return rc;
   if (n_seq * (T + k) > ctx->Rmax) return fail(ctx, FIRP_ERR_CAPACITY, "n_seq * (T + k) exceeds the row capacity");
@@ -491,7 +516,8 @@ int firp_step(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_
 
   RunArgs ra{};
   ra.rw = Rows{n_seq, T, k, T + k, n_seq * (T + k), 0};
-  ra.d_tokens = d_tree_tokens; ra.l = l; ra.want_head = true; ra.prefill_last_row = -1; ra.T_next = T_next;
+  for (int i = 0; i < k; ++i) ra.tl[i] = layers[i];
+  ra.d_tokens = d_tree_tokens; ra.want_head = true; ra.prefill_last_row = -1; ra.T_next = T_next;
   ra.out = out; ra.logits_dst = (out && out->logits) ? out->logits : ctx->logits; ra.n_hi_max = n_hi_max;
   if ((rc = run_rows(ctx, ra, st))) return rc;
   ctx->stepped = true; ctx->last_n_seq = n_seq; ctx->last_T = T; ctx->last_k = k;
@@ -500,6 +526,13 @@ int firp_step(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_
 
 int firp_prefill(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int32_t P, int32_t k, int32_t l,
                  const int32_t *next_parents, int32_t T_next, const firp_step_out *out, void *stream) {
+  int32_t layers[8];
+  for (int i = 0; i < 8; ++i) layers[i] = l;
+  return firp_prefill_layers(ctx, seq, d_prompt, P, k, layers, next_parents, T_next, out, stream);
+}
+
+int firp_prefill_layers(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int32_t P, int32_t k, const int32_t *layers,
+                        const int32_t *next_parents, int32_t T_next, const firp_step_out *out, void *stream) {
   int rc = check_ready(ctx);
   if (rc) return rc;
   const firp_model_cfg &cfg = ctx->cfg;
@@ -507,7 +540,7 @@ int firp_prefill(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int32_t P,
   if (!d_prompt || P < 1) return fail(ctx, FIRP_ERR_BAD_ARG, "empty prompt");
   if (seq < 0 || seq >= cfg.max_batch) return fail(ctx, FIRP_ERR_BAD_ARG, "seq id out of range");
   if (k < 0 || k > cfg.max_k || k > ctx->w.n_maps) return fail(ctx, FIRP_ERR_CAPACITY, "k exceeds max_k or the loaded maps");
-  if (k > 0 && (l < 0 || l >= cfg.n_layers)) return fail(ctx, FIRP_ERR_BAD_ARG, "insertion layer outside 0..n_layers-1");
+  if ((rc = check_layers(ctx, k, layers))) return rc;
   if (P + k > cfg.max_ctx) return fail(ctx, FIRP_ERR_CAPACITY, "prompt does not fit max_ctx");
   const int32_t one = -1;
   if (k == 0) { next_parents = &one; T_next = 1; }
@@ -535,7 +568,8 @@ int firp_prefill(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int32_t P,
     const int kc = last ? k : 0;
     RunArgs ra{};
     ra.rw = Rows{1, Tc, kc, Tc + kc, Tc + kc, Tc - 1};
-    ra.d_tokens = d_prompt + p0; ra.l = l; ra.want_head = last; ra.prefill_last_row = Tc - 1; ra.T_next = T_next;
+    for (int i = 0; i < kc; ++i) ra.tl[i] = layers[i];
+    ra.d_tokens = d_prompt + p0; ra.want_head = last; ra.prefill_last_row = Tc - 1; ra.T_next = T_next;
     ra.out = nullptr; ra.logits_dst = ctx->logits; ra.n_hi_max = ctx->n_hi[seq];
     firp_step_out o2{};
     if (last && out) {

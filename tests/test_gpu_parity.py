@@ -56,6 +56,57 @@ def test_c1_random_trees_and_layers(torch_cuda, c1, c1_weights, case):
     eng.close()
 
 
+@pytest.mark.parametrize("layers", [(0, 1, 1), (0, 0, 1), (0, 1, 3), (1, 2, 3), (2, 2, 3), (3, 3, 3)])
+def test_c1_one_insertion_layer_per_prediction_step(torch_cuda, c1, layers):
+    """Section 3.3: prediction step i has its own layer t_i (firp_step_layers / firp_prefill_layers):
+    lock-step against the oracle on the small shape, two or four layers deep, greedy and forced."""
+    shape = si.scaled(c1, L=2 if max(layers) < 2 else 4, l=layers[0])
+    weights = si.all_weights(shape)
+    parents = si.random_tree(5, 19, 3, sum(layers))
+    for forced in (False, True):
+        eng, orc = make_pair(shape, weights, 256, max_tree=32, max_k=3, max_depth=3)
+        st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=45), 4, forced=forced, k=3, l=list(layers))
+        assert st.steps == 4
+        eng.close()
+
+
+def test_c1_equal_layers_are_the_single_layer_call_bit_for_bit(torch_cuda, c1, c1_weights):
+    import torch
+    parents = si.tree_template(8)
+    tokens = torch.from_numpy(si.random_tokens(c1, 8, 3)).cuda()
+    prompt = torch.from_numpy(si.prompt(c1)).cuda()
+    logits = []
+    for l in (1, [1, 1, 1]):
+        eng, _ = make_pair(c1, c1_weights, 128)
+        pout = eng.new_out(1, 1, 3, T_next=8)
+        eng.prefill(0, prompt, 3, l, parents, pout)
+        out = eng.new_out(1, 8, 3)
+        eng.step(tokens, parents, 3, l, out)
+        torch.cuda.synchronize()
+        logits.append((pout.logits.cpu().numpy().copy(), out.logits.cpu().numpy().copy(), out.next_tree_tokens.cpu().numpy().copy()))
+        eng.close()
+    for a, b in zip(logits[0], logits[1]):
+        assert np.array_equal(a, b)
+
+
+def test_layers_are_validated_on_the_host(torch_cuda, c1, c1_weights):
+    import torch
+    from paper_2410_20488_b200 import FirpError, binding
+    eng, _ = make_pair(c1, c1_weights, 128)
+    tok = torch.zeros(8, dtype=torch.int32, device="cuda")
+    out = eng.new_out(1, 8, 3)
+    pout = eng.new_out(1, 1, 3, T_next=8)
+    eng.prefill(0, torch.from_numpy(si.prompt(c1)).cuda(), 3, [0, 1, 1], si.tree_template(8), pout)
+    for layers in ([1, 0, 1], [0, 1, 2], [-1, 0, 1]):
+        with pytest.raises(FirpError) as e:
+            eng.step(tok, si.tree_template(8), 3, layers, out)
+        assert e.value.code == binding.FIRP_ERR_BAD_ARG
+        with pytest.raises(FirpError) as e:
+            eng.prefill(0, torch.from_numpy(si.prompt(c1)).cuda(), 3, layers, si.tree_template(8), pout)
+        assert e.value.code == binding.FIRP_ERR_BAD_ARG
+    eng.close()
+
+
 def test_c1_predictor_with_bias(torch_cuda, c1, c1_weights):
     """Eq. 3 with a non-zero bias b_i (the synthetic configurations use b = 0)."""
     w = dict(c1_weights)
@@ -127,6 +178,18 @@ def test_c2_full_size_lockstep(torch_cuda, c2_weights):
     eng, orc = make_pair(c2, c2_weights, 512 + 64)
     st = lockstep_run(eng, orc, c2, parents, si.prompt(c2), 2, forced=False, check_cache_rows=True)
     print("c2 greedy", st.as_dict())
+    assert st.steps == 2
+    eng.close()
+
+
+def test_c2_layers_15_20_25_full_size(torch_cuda, c2_weights):
+    """The prediction layers the paper uses for its 7B models (Section 4 "Setup": 15, 20, 25) on the
+    7B-shaped workload: prefill and two lock-step steps against the oracle."""
+    c2 = si.CONFIGS["c2"]
+    parents = si.tree_template(c2.T)
+    eng, orc = make_pair(c2, c2_weights, 512 + 64)
+    st = lockstep_run(eng, orc, c2, parents, si.prompt(c2), 2, forced=False, check_cache_rows=False, l=[15, 20, 25])
+    print("c2 layers 15/20/25", st.as_dict())
     assert st.steps == 2
     eng.close()
 
