@@ -59,6 +59,10 @@ def _get_lib():
         lib.oracle_forward.restype = i32
         lib.oracle_forward_layers.argtypes = [vp, i32, vp, vp, i32, i32, vp, i32, i32, vp, vp, vp, i32, vp, vp]
         lib.oracle_forward_layers.restype = i32
+        lib.oracle_forward_chains.argtypes = [vp, i32, vp, vp, i32, i32, vp, i32, vp, vp, vp, vp]
+        lib.oracle_forward_chains.restype = i32
+        lib.oracle_tree_prep_chains.argtypes = [vp, i32, i32, vp, vp, vp, vp]
+        lib.oracle_tree_prep_chains.restype = i32
         lib.oracle_verify.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
         lib.oracle_verify.restype = i32
         lib.oracle_next_tree.argtypes = [vp, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp]
@@ -89,6 +93,25 @@ def tree_prep(parents, k: int = 0, anchor: int = 0):
     if rc != 0:
         raise ValueError("malformed tree")
     return dict(ext_parent=ext, depth=depth, mask=mask, rank=rank)
+
+
+def tree_prep_chains(parents, k: int):
+    """The same for a chain of k pseudo rows under every node: M = T*(1+k) rows, chain row i
+    (1-based) of node v at row T + (i-1)*T + v."""
+    parents = _i32(parents)
+    T = parents.size
+    M = T * (1 + k)
+    ext = np.zeros(M, np.int32); depth = np.zeros(M, np.int32)
+    mask = np.zeros((M, M), np.uint8); rank = np.zeros(T, np.int32)
+    rc = _get_lib().oracle_tree_prep_chains(_ptr(parents), T, k, _ptr(ext), _ptr(depth), _ptr(mask), _ptr(rank))
+    if rc != 0:
+        raise ValueError("malformed tree")
+    return dict(ext_parent=ext, depth=depth, mask=mask, rank=rank)
+
+
+def chain_row(T: int, v: int, i: int) -> int:
+    """Row of chain step i (1-based) of tree node v in the every-node-chains layout."""
+    return T + (i - 1) * T + v
 
 
 def verify(logits, tokens, parents):
@@ -224,6 +247,46 @@ class Oracle:
         out = dict(logits=logits, depth=depth, mask=mask, pos=depth + self.context_len(seq))
         if want_h_ins:
             out["h_ins"] = h_ins
+        return out
+
+    def forward_chains(self, tokens, parents, k: int, l, seq: int = 0, logit_row0: int = 0, want_h_ins: bool = False):
+        """The step with a chain of k pseudo rows under every tree node (rows as in tree_prep_chains);
+        l: one insertion layer or one per prediction step."""
+        tokens, parents = _i32(tokens), _i32(parents)
+        layers = _i32([l] * k) if np.isscalar(l) else _i32(l)
+        if layers.size != k:
+            raise ValueError("need one insertion layer per prediction step")
+        T = tokens.size
+        M = T * (1 + k)
+        s = self.shape
+        logits = np.zeros((M, s.V), np.float32)
+        depth = np.zeros(M, np.int32)
+        mask = np.zeros((M, M), np.uint8)
+        h_ins = np.zeros((T * k, s.d), np.float32) if want_h_ins else None
+        rc = self.lib.oracle_forward_chains(self.h, seq, _ptr(tokens), _ptr(parents), T, k, _ptr(layers), logit_row0,
+                                            _ptr(logits), _ptr(depth), _ptr(mask), _ptr(h_ins))
+        if rc != 0:
+            raise ValueError("oracle_forward_chains failed: %d" % rc)
+        out = dict(logits=logits, depth=depth, mask=mask, pos=depth + self.context_len(seq))
+        if want_h_ins:
+            out["h_ins"] = h_ins
+        return out
+
+    def step_chains(self, tokens, parents, k: int, l, seq: int = 0, next_parents=None):
+        """Forward with a chain under every node + greedy verification + the next tree read from the
+        chain of the node the walk ended on (its row i gives the candidates of depth i).  Does not commit."""
+        tokens, parents = _i32(tokens), _i32(parents)
+        T = tokens.size
+        out = self.forward_chains(tokens, parents, k, l, seq)
+        out.update(self.verify(out["logits"][:T], tokens, parents))
+        end = int(out["path"][-1])
+        bonus = int(out["accepted"][-1])
+        rows = [chain_row(T, end, i) for i in range(1, k + 1)]
+        picked = np.concatenate([out["logits"][:T], out["logits"][rows]]) if k > 0 else out["logits"][:T]
+        if next_parents is None:
+            next_parents = parents if k > 0 else np.array([-1], np.int32)
+        out.update(self.next_tree(picked, T, k, bonus, next_parents))
+        out["end_node"] = end
         return out
 
     def verify(self, logits, tokens, parents):

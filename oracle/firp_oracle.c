@@ -36,6 +36,12 @@
  *     stands for position pos[anchor] + i; it sees the prefix, the anchor's
  *     ancestors and the anchor, the earlier pseudo rows ("No masked" setting
  *     of Section 4.3) and itself (Section 3.3, paragraph after Eq. 3).
+ *     With one chain (oracle_forward, oracle_forward_layers) the rows hang off
+ *     one tree node, the root by default.  oracle_forward_chains keeps such a
+ *     chain under every tree node, so that the next candidates can be read from
+ *     the chain of the node the acceptance walk ends on (Section 3.4 produces
+ *     them from the accepted sequence; the paper does not say how a tree step
+ *     does that before the sequence is known).
  *   - Greedy verification (Section 3.4, Section 4 "greedy sampling"): walk
  *     from the root, following the child whose token equals the argmax of the
  *     current row; the walk's nodes are the accepted path, the last argmax is
@@ -180,60 +186,81 @@ static void rope(float *x, int dh, int p, double theta) {
  * among its parent's children in index order (tree rows only; rank[0] = 0).
  * Returns 0, or -1 for a malformed tree.
  */
-int32_t oracle_tree_prep(const int32_t *parents, int32_t T, int32_t k, int32_t anchor,
-                         int32_t *ext_parent, int32_t *depth, uint8_t *mask, int32_t *rank) {
-  int M = T + k;
-  if (T < 1 || parents[0] != -1 || anchor < 0 || anchor >= T) return -1;
-  for (int v = 1; v < T; ++v) if (parents[v] < 0 || parents[v] >= v) return -1;
-  for (int v = 0; v < T; ++v) ext_parent[v] = parents[v];
-  for (int i = 1; i <= k; ++i) ext_parent[T + i - 1] = (i == 1) ? anchor : T + i - 2;
+static int tree_ok(const int32_t *parents, int32_t T) {
+  if (T < 1 || parents[0] != -1) return 0;
+  for (int v = 1; v < T; ++v) if (parents[v] < 0 || parents[v] >= v) return 0;
+  return 1;
+}
+
+/* depth and ancestor-or-self mask of M rows whose extended parents precede them */
+static void closure(const int32_t *ext_parent, int M, int32_t *depth, uint8_t *mask) {
   memset(mask, 0, (size_t)M * M);
   for (int v = 0; v < M; ++v) {
     depth[v] = (ext_parent[v] < 0) ? 0 : depth[ext_parent[v]] + 1;
     for (int u = v; u >= 0; u = ext_parent[u]) mask[(size_t)v * M + u] = 1;
   }
-  if (rank) {
-    for (int v = 0; v < T; ++v) {
-      int r = 0;
-      for (int u = 1; u < v; ++u) if (parents[u] == parents[v]) ++r;
-      rank[v] = (v == 0) ? 0 : r;
-    }
+}
+
+static void sibling_ranks(const int32_t *parents, int32_t T, int32_t *rank) {
+  for (int v = 0; v < T; ++v) {
+    int r = 0;
+    for (int u = 1; u < v; ++u) if (parents[u] == parents[v]) ++r;
+    rank[v] = (v == 0) ? 0 : r;
   }
+}
+
+int32_t oracle_tree_prep(const int32_t *parents, int32_t T, int32_t k, int32_t anchor,
+                         int32_t *ext_parent, int32_t *depth, uint8_t *mask, int32_t *rank) {
+  if (!tree_ok(parents, T) || anchor < 0 || anchor >= T) return -1;
+  for (int v = 0; v < T; ++v) ext_parent[v] = parents[v];
+  for (int i = 1; i <= k; ++i) ext_parent[T + i - 1] = (i == 1) ? anchor : T + i - 2;
+  closure(ext_parent, T + k, depth, mask);
+  if (rank) sibling_ranks(parents, T, rank);
   return 0;
 }
 
 /*
- * One forward pass over the T tree rows (+ pseudo row i from layer tl[i] on) of
- * sequence `seq`, on top of its committed cache of n positions.  Cache slots
- * n..n+T+k-1 receive the rows' keys/values (scratch until oracle_commit; a
- * pseudo row has none below its own layer).
- *
- * tl          [k] insertion layer of each prediction step, non-decreasing, 0 <= tl[i] < L
- * logits      [(T+k)][V] fp32 out; rows < logit_row0 are skipped (left untouched)
- * dump_layer, h_dump   optional [(T+k)][d]: residual stream entering layer dump_layer,
- *             after that layer's insertions (rows not yet alive are zero)
- * h_ins       optional [k][d]: every pseudo row as it was appended
- * Returns 0, -1 malformed tree or layers, -2 capacity.
+ * The same bookkeeping when EVERY tree node v carries its own chain of k pseudo rows
+ * (Section 3.4 generates the next candidates from the accepted sequence, which is only
+ * known after the pass, so a chain is kept for every node the walk may end on; Section
+ * 3.3: chain row i of node v stands for position pos[v] + i and sees what v sees, the
+ * earlier rows of its own chain and itself).  Rows: 0..T-1 tree nodes, then step-major
+ * row(v, i) = T + (i-1)*T + v for i = 1..k, so M = T*(1+k).
  */
-int32_t oracle_forward_layers(void *hnd, int32_t seq, const int32_t *tokens, const int32_t *parents,
-                              int32_t T, int32_t k, const int32_t *tl, int32_t anchor, int32_t logit_row0,
-                              float *logits, int32_t *depth_out, uint8_t *mask_out,
-                              int32_t dump_layer, float *h_dump, float *h_ins) {
-  oracle_t *o = (oracle_t *)hnd;
+int32_t oracle_tree_prep_chains(const int32_t *parents, int32_t T, int32_t k,
+                                int32_t *ext_parent, int32_t *depth, uint8_t *mask, int32_t *rank) {
+  if (!tree_ok(parents, T) || k < 0) return -1;
+  for (int v = 0; v < T; ++v) ext_parent[v] = parents[v];
+  for (int i = 1; i <= k; ++i)
+    for (int v = 0; v < T; ++v) ext_parent[T + (i - 1) * T + v] = (i == 1) ? v : T + (i - 2) * T + v;
+  closure(ext_parent, T * (1 + k), depth, mask);
+  if (rank) sibling_ranks(parents, T, rank);
+  return 0;
+}
+
+/*
+ * One forward pass over the T tree rows and pn pseudo rows of sequence `seq`, on top of
+ * its committed cache of n positions.  Pseudo row r (row T + r) is W_step h[src] + b_step
+ * (Eq. 3) on the residual entering layer tl[step[r]] and is alive from that layer on; the
+ * rows are ordered by that layer.  Cache slots n..n+T+pn-1 receive the rows' keys/values
+ * (scratch until oracle_commit; a pseudo row has none below its own layer).
+ *
+ * depth, mask [M], [M][M]: position offset and visibility of every row (M = T + pn)
+ * logits      [M][V] fp32 out; rows < logit_row0 are skipped (left untouched)
+ * dump_layer, h_dump   optional [M][d]: residual stream entering layer dump_layer,
+ *             after that layer's insertions (rows not yet alive are zero)
+ * h_ins       optional [pn][d]: every pseudo row as it was appended
+ * Returns 0 or -2 (capacity).
+ */
+static int32_t forward_core(oracle_t *o, int32_t seq, const int32_t *tokens, int32_t T, int32_t pn,
+                            const int32_t *p_src, const int32_t *p_step, const int32_t *tl,
+                            const int32_t *depth, const uint8_t *mask, int32_t logit_row0, float *logits,
+                            int32_t dump_layer, float *h_dump, float *h_ins) {
   const oracle_cfg *c = &o->cfg;
   const oracle_weights *w = &o->w;
   const int d = c->d, H = c->H, Hkv = c->Hkv, dh = c->dh, F = c->F, V = c->V;
-  const int nq = H * dh, nkv = Hkv * dh, M = T + k, n = o->n[seq];
-  if (k < 0 || k > c->n_maps) return -1;
-  for (int i = 0; i < k; ++i) if (tl[i] < 0 || tl[i] >= c->L || (i > 0 && tl[i] < tl[i - 1])) return -1;
+  const int nq = H * dh, nkv = Hkv * dh, M = T + pn, n = o->n[seq];
   if (n + M > c->max_ctx) return -2;
-
-  int32_t *ext_parent = (int32_t *)malloc(sizeof(int32_t) * M);
-  int32_t *depth = (int32_t *)malloc(sizeof(int32_t) * M);
-  uint8_t *mask = (uint8_t *)malloc((size_t)M * M);
-  if (oracle_tree_prep(parents, T, k, anchor, ext_parent, depth, mask, NULL) != 0) {
-    free(ext_parent); free(depth); free(mask); return -1;
-  }
 
   float *h = (float *)calloc((size_t)M * d, sizeof(float));
   float *x = (float *)calloc((size_t)M * d, sizeof(float));
@@ -250,14 +277,15 @@ int32_t oracle_forward_layers(void *hnd, int32_t seq, const int32_t *tokens, con
 
   int rows = T;  /* rows alive: the tree rows and the pseudo rows whose layer has been reached */
   for (int j = 0; j < c->L; ++j) {
-    for (int i = 0; i < k; ++i) {
+    for (int r = 0; r < pn; ++r) {
+      const int i = p_step[r];
       if (tl[i] != j) continue;
-      /* Eq. 3: h~_i = W_i h[anchor] + b_i on the residual entering layer t_i, appended as row T+i */
-      float *dst = h + (size_t)(T + i) * d;
-      linear(w->pred_w + (size_t)i * d * d, h + (size_t)anchor * d, d, dst, d, 1, d, d);
+      /* Eq. 3: h~ = W_i h[src] + b_i on the residual entering layer t_i, appended as row T+r */
+      float *dst = h + (size_t)(T + r) * d;
+      linear(w->pred_w + (size_t)i * d * d, h + (size_t)p_src[r] * d, d, dst, d, 1, d, d);
       if (w->pred_b) for (int cc = 0; cc < d; ++cc) dst[cc] += bf16f(w->pred_b[(size_t)i * d + cc]);
-      if (h_ins) memcpy(h_ins + (size_t)i * d, dst, sizeof(float) * d);
-      rows = T + i + 1;
+      if (h_ins) memcpy(h_ins + (size_t)r * d, dst, sizeof(float) * d);
+      rows = T + r + 1;
     }
     if (h_dump && j == dump_layer) memcpy(h_dump, h, sizeof(float) * (size_t)M * d);
 
@@ -325,11 +353,68 @@ int32_t oracle_forward_layers(void *hnd, int32_t seq, const int32_t *tokens, con
   if (logits && logit_row0 < M)
     linear(w->lm_head, x + (size_t)logit_row0 * d, d, logits + (size_t)logit_row0 * V, V, M - logit_row0, d, V);
 
-  if (depth_out) memcpy(depth_out, depth, sizeof(int32_t) * M);
-  if (mask_out) memcpy(mask_out, mask, (size_t)M * M);
-  free(ext_parent); free(depth); free(mask);
   free(h); free(x); free(q); free(att); free(delta); free(gate); free(up); free(p);
   return 0;
+}
+
+static int layers_ok(const oracle_cfg *c, int32_t k, const int32_t *tl) {
+  if (k < 0 || k > c->n_maps) return 0;
+  for (int i = 0; i < k; ++i) if (tl[i] < 0 || tl[i] >= c->L || (i > 0 && tl[i] < tl[i - 1])) return 0;
+  return 1;
+}
+
+/*
+ * The step with one chain of k pseudo rows hanging off tree node `anchor`: pseudo row i
+ * (row T+i) is appended at the input of layer tl[i] (non-decreasing, 0 <= tl[i] < L).
+ * h_ins optional [k][d].  Returns 0, -1 malformed tree or layers, -2 capacity.
+ */
+int32_t oracle_forward_layers(void *hnd, int32_t seq, const int32_t *tokens, const int32_t *parents,
+                              int32_t T, int32_t k, const int32_t *tl, int32_t anchor, int32_t logit_row0,
+                              float *logits, int32_t *depth_out, uint8_t *mask_out,
+                              int32_t dump_layer, float *h_dump, float *h_ins) {
+  oracle_t *o = (oracle_t *)hnd;
+  if (!layers_ok(&o->cfg, k, tl)) return -1;
+  const int M = T + k;
+  int32_t *ext_parent = (int32_t *)malloc(sizeof(int32_t) * M);
+  int32_t *depth = (int32_t *)malloc(sizeof(int32_t) * M);
+  uint8_t *mask = (uint8_t *)malloc((size_t)M * M);
+  int32_t *src = (int32_t *)malloc(sizeof(int32_t) * (k + 1)), *step = (int32_t *)malloc(sizeof(int32_t) * (k + 1));
+  int32_t rc = -1;
+  if (oracle_tree_prep(parents, T, k, anchor, ext_parent, depth, mask, NULL) == 0) {
+    for (int i = 0; i < k; ++i) { src[i] = anchor; step[i] = i; }
+    rc = forward_core(o, seq, tokens, T, k, src, step, tl, depth, mask, logit_row0, logits, dump_layer, h_dump, h_ins);
+    if (depth_out) memcpy(depth_out, depth, sizeof(int32_t) * M);
+    if (mask_out) memcpy(mask_out, mask, (size_t)M * M);
+  }
+  free(ext_parent); free(depth); free(mask); free(src); free(step);
+  return rc;
+}
+
+/*
+ * The step with a chain of k pseudo rows under EVERY tree node (see oracle_tree_prep_chains
+ * for the row order): chain row i of node v is W_i h[v] + b_i on v's residual entering
+ * layer tl[i].  logits [T*(1+k)][V].  Returns 0, -1 malformed tree or layers, -2 capacity.
+ */
+int32_t oracle_forward_chains(void *hnd, int32_t seq, const int32_t *tokens, const int32_t *parents,
+                              int32_t T, int32_t k, const int32_t *tl, int32_t logit_row0,
+                              float *logits, int32_t *depth_out, uint8_t *mask_out, float *h_ins) {
+  oracle_t *o = (oracle_t *)hnd;
+  if (!layers_ok(&o->cfg, k, tl)) return -1;
+  const int pn = T * k, M = T + pn;
+  int32_t *ext_parent = (int32_t *)malloc(sizeof(int32_t) * M);
+  int32_t *depth = (int32_t *)malloc(sizeof(int32_t) * M);
+  uint8_t *mask = (uint8_t *)malloc((size_t)M * M);
+  int32_t *src = (int32_t *)malloc(sizeof(int32_t) * (pn + 1)), *step = (int32_t *)malloc(sizeof(int32_t) * (pn + 1));
+  int32_t rc = -1;
+  if (oracle_tree_prep_chains(parents, T, k, ext_parent, depth, mask, NULL) == 0) {
+    for (int i = 0; i < k; ++i)
+      for (int v = 0; v < T; ++v) { src[i * T + v] = v; step[i * T + v] = i; }
+    rc = forward_core(o, seq, tokens, T, pn, src, step, tl, depth, mask, logit_row0, logits, -1, NULL, h_ins);
+    if (depth_out) memcpy(depth_out, depth, sizeof(int32_t) * M);
+    if (mask_out) memcpy(mask_out, mask, (size_t)M * M);
+  }
+  free(ext_parent); free(depth); free(mask); free(src); free(step);
+  return rc;
 }
 
 /* The single-layer case of the paper's overview (Section 3.2): every prediction step at layer l. */

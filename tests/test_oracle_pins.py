@@ -11,6 +11,9 @@
   P9  predictor size k*d^2 equals the draft-module sizes printed in the paper's Table 1
   P10 one insertion layer per prediction step (Section 3.3): the chain == a causal forward whose row i is
       replaced at layer t_i; step i does not depend on the layers of later steps; W = I closed form
+  P11 a chain of k pseudo rows under every tree node: every chain row == a causal forward over prefix + the
+      node's root path with rows replaced at the insertion layer(s); the root's chain == the single chain;
+      mask == brute-force closure; the free-running decode stays lossless
 plus hand-worked cases for the mask, the acceptance walk, the tie rules and the next tree.
 """
 import os
@@ -237,6 +240,75 @@ def test_p10_a_step_ignores_the_layers_of_later_steps_and_identity_maps_copy_the
         for i, t in enumerate((0, 2, 3)):
             h_t = oI.forward(tokens, parents, 0, t, want_h_at_l=True)["h_at_l"]   # k = 0: plain residual at layer t
             assert np.array_equal(h_ins[i], h_t[anchor])
+
+
+# ---------------------------------------------------------------- P11
+def test_p11_chain_bookkeeping_is_the_closure_of_its_parents():
+    parents = si.tree_template(8)
+    T, k = 8, 3
+    tp = oracle.tree_prep_chains(parents, k)
+    M = T * (1 + k)
+    base = oracle.tree_prep(parents)
+    for v in range(T):
+        for i in range(1, k + 1):
+            r = oracle.chain_row(T, v, i)
+            assert tp["depth"][r] == base["depth"][v] + i                      # position id pos[v] + i (Section 3.3)
+            want = np.zeros(M, np.uint8)
+            want[:T] = base["mask"][v]                                         # what v sees among the tree rows
+            for j in range(1, i + 1):
+                want[oracle.chain_row(T, v, j)] = 1                            # earlier rows of its own chain, itself
+            assert np.array_equal(tp["mask"][r], want)
+    assert np.array_equal(tp["mask"][:T, :T], base["mask"]) and not tp["mask"][:T, T:].any()   # tree rows see no chain
+
+
+@pytest.mark.parametrize("layers", [1, (0, 1, 3), (2, 2, 3)])
+def test_p11_every_chain_row_is_a_causal_forward_over_its_nodes_path(c1_deep, layers):
+    shape, weights = c1_deep
+    hf4 = build_hf_llama(shape, weights)
+    k, T = 3, 8
+    prompt = si.prompt(shape, length=11)
+    Wf = si.bf16_bits_to_f32(weights["pred_w"]).astype(np.float64)
+    bf = np.zeros((k, shape.d))
+    o = fresh(shape, weights)
+    o.forward(prompt, si.chain_template(prompt.size), 0, 0)
+    o.commit(np.arange(prompt.size))
+    tokens, parents = si.random_tokens(shape, T, 6), si.tree_template(T)
+    out = o.forward_chains(tokens, parents, k, layers if np.isscalar(layers) else list(layers))
+    for v in range(T):
+        path = path_to(parents, v)
+        ids = list(prompt) + [int(tokens[u]) for u in path] + [0] * k
+        first = prompt.size + len(path)
+        ref = hf_logits_with_replaced_rows(hf4, ids, layers, first, list(Wf), list(bf), first - 1)
+        got = out["logits"][[oracle.chain_row(T, v, i) for i in (1, 2, 3)]]
+        assert np.abs(got - ref[first:]).max() < 1e-5, "chain of node %d" % v
+        assert np.abs(out["logits"][v] - ref[first - 1]).max() < 1e-5
+    # the root's chain is the single chain of the plain step; tree rows do not depend on the chains
+    one = o.forward(tokens, parents, k, layers if np.isscalar(layers) else list(layers), anchor=0)["logits"]
+    assert np.array_equal(out["logits"][:T], one[:T])
+    assert np.array_equal(out["logits"][[oracle.chain_row(T, 0, i) for i in (1, 2, 3)]], one[T:])
+    assert np.array_equal(o.forward(tokens, parents, k, 1, anchor=5)["logits"][T:],
+                          o.forward_chains(tokens, parents, k, 1)["logits"][[oracle.chain_row(T, 5, i) for i in (1, 2, 3)]])
+
+
+def test_p11_decoding_with_chains_is_lossless_and_reads_the_end_nodes_chain(c1, c1_weights, hf):
+    prompt = si.prompt(c1)
+    want = hf_greedy(hf, prompt, 40)
+    parents = si.tree_template(c1.T)
+    o = fresh(c1, c1_weights)
+    r = o.prefill(prompt, c1.k, c1.l, parents)
+    tokens, emitted = r["next_tokens"].copy(), [r["root"]]
+    for _ in range(10):
+        out = o.step_chains(tokens, parents, c1.k, c1.l)
+        end = out["end_node"]
+        assert end == out["path"][-1]
+        rows = [oracle.chain_row(c1.T, end, i) for i in (1, 2, 3)]
+        for i, rr in enumerate(rows):                      # candidates of depth i+1 come from row i+1 of the end node's chain
+            order = np.lexsort((np.arange(c1.V), -out["logits"][rr]))[:8]
+            assert np.array_equal(out["topb_ids"][i], order)
+        o.commit(out["path"])
+        emitted += out["accepted"].tolist()
+        tokens = out["next_tokens"].copy()
+    assert emitted == want[: len(emitted)]                 # Eq. 1: the stream is the greedy stream
 
 
 # ---------------------------------------------------------------- P5
