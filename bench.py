@@ -41,6 +41,8 @@ def parse():
     ap.add_argument("--layers", type=int, default=0, help="debug only: truncate the decoder (marks the line invalid)")
     ap.add_argument("--insert-layers", default="", help="one insertion layer per prediction step, e.g. 15,20,25 "
                     "(the paper's 7B setting); default: the workload's single layer l")
+    ap.add_argument("--chains", action="store_true", help="a chain of k pseudo rows under every tree node "
+                    "(firp_step_chains; T (1 + k) rows) instead of the workload's single chain")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-kernel-times", action="store_true", help="skip the per-kernel event-timed pass")
@@ -50,6 +52,8 @@ def parse():
 
 # One insertion layer per prediction step (--insert-layers), or None: the workload's single layer l.
 INSERT_LAYERS = None
+# A chain of pseudo rows under every tree node (--chains) instead of one chain under the root.
+CHAINS = False
 
 
 def ins_l(shape):
@@ -73,15 +77,13 @@ def algorithmic_bytes(shape, n_ctx: float, batch: int = 1) -> dict:
     """Bytes one step must move: every weight once, the KV cache read once per layer, the new
     rows' KV written once, the embedding rows (logits stay on the device and are not exported)."""
     s = shape
-    M_lo, M_hi = s.T, s.T + s.k
     weights = s.weight_bytes()
     kv_row = 2 * 2 * s.n_kv * batch               # K and V, bf16, every sequence
     kv_read = kv_write = 0
     for j in range(s.L):
-        if INSERT_LAYERS:
-            M = s.T + sum(1 for t in INSERT_LAYERS if t <= j)
-        else:
-            M = M_hi if (s.k > 0 and j >= s.l) else M_lo
+        per_step = s.T if CHAINS else 1            # pseudo rows one prediction step adds
+        alive = sum(1 for t in INSERT_LAYERS if t <= j) if INSERT_LAYERS else (s.k if j >= s.l else 0)
+        M = s.T + per_step * alive
         kv_read += kv_row * (n_ctx + M)
         kv_write += kv_row * M
     return dict(weights=weights, kv_read=kv_read, kv_write=kv_write, embed=2 * s.T * s.d * batch,
@@ -117,14 +119,15 @@ def kernel_source_digest() -> str:
     return h.hexdigest()[:16]
 
 
-def kernel_times(eng, shape, parents, tokens, out, steps, n_ctx, peak_gbs, peak_kind, seq_ids=None):
+def kernel_times(eng, shape, parents, tokens, out, steps, n_ctx, peak_gbs, peak_kind, seq_ids=None, step_fn=None):
     """Second, separately timed pass: the library brackets every launch with CUDA events on the
     launching stream; per class: launches, average duration, share of the summed kernel time and,
     for the HBM-streaming classes, achieved GB/s = algorithmic bytes per launch / average duration."""
     seq_ids = seq_ids or [0]
+    step_fn = step_fn or eng.step
     eng.profile(True)
     for _ in range(steps):
-        eng.step(tokens, parents, shape.k, ins_l(shape), out, seq_ids=seq_ids, n_seq=len(seq_ids))
+        step_fn(tokens, parents, shape.k, ins_l(shape), out, seq_ids=seq_ids, n_seq=len(seq_ids))
         eng.commit(len(seq_ids), seq_ids=seq_ids)
         tokens = out.next_tree_tokens
     prof = eng.profile_read()
@@ -225,13 +228,14 @@ def time_oracle(shape, weights, steps: int, warmup: int, n_ctx: int = 32):
     import oracle
     import synth_inputs as si
     parents = si.tree_template(shape.T)
-    orc = oracle.Oracle(shape, weights, max_ctx=n_ctx + (steps + warmup + 1) * (shape.k + 1) + shape.T + shape.k + 8)
+    rows = shape.T * (1 + shape.k) if CHAINS else shape.T + shape.k
+    orc = oracle.Oracle(shape, weights, max_ctx=n_ctx + (steps + warmup + 1) * (shape.k + 1) + rows + 8)
     r = orc.prefill(si.prompt(shape, length=n_ctx), shape.k, ins_l(shape), parents)
     tokens = r["next_tokens"]
     emitted, t_total = 0, 0.0
     for i in range(warmup + steps):
         t0 = time.perf_counter()
-        out = orc.step(tokens, parents, shape.k, ins_l(shape))
+        out = (orc.step_chains if CHAINS else orc.step)(tokens, parents, shape.k, ins_l(shape))
         orc.commit(out["path"])
         dt = time.perf_counter() - t0
         if i >= warmup:
@@ -327,6 +331,8 @@ def main():
         INSERT_LAYERS = [int(t) for t in args.insert_layers.split(",")]
         if len(INSERT_LAYERS) != shape.k or INSERT_LAYERS != sorted(INSERT_LAYERS) or not all(0 <= t < shape.L for t in INSERT_LAYERS):
             raise SystemExit("--insert-layers needs k non-decreasing layers inside the decoder")
+    global CHAINS
+    CHAINS = bool(args.chains)
     if args.impl == "reference":
         return run_reference(args, shape)
 
@@ -361,10 +367,13 @@ def main():
         lengths = [int(n) for n in si.context_lengths(shape)]
     else:
         lengths = [shape.prompt_len]
-    max_ctx = max(lengths) + total_steps * S + shape.T + shape.k + 64
-    eng = FirpEngine(shape, weights, max_ctx=max_ctx, max_batch=B, device=str(dev))
+    chains = bool(args.chains)
+    rows_per_seq = shape.T * (1 + shape.k) if chains else shape.T + shape.k
+    max_ctx = max(lengths) + total_steps * S + rows_per_seq + 64
+    eng = FirpEngine(shape, weights, max_ctx=max_ctx, max_batch=B, device=str(dev), max_rows=B * rows_per_seq if chains else 0)
+    step_fn = eng.step_chains if chains else eng.step
     T_next = shape.T if shape.k > 0 else 1
-    outs = [eng.new_out(B, shape.T, shape.k, want_logits=False) for _ in range(2)]
+    outs = [eng.new_out(B, shape.T, shape.k, want_logits=False, chains=chains) for _ in range(2)]
     first = torch.zeros(B, T_next, dtype=torch.int32, device=dev)
     for b_i, n in enumerate(lengths):
         prompt = torch.from_numpy(si.prompt(shape, seq=rank * B + b_i, length=n)).to(dev)
@@ -386,7 +395,7 @@ def main():
     def one_step(i, tokens):
         nonlocal launches
         o = outs[i & 1]
-        eng.step(tokens, parents, shape.k, ins_l(shape), o, seq_ids=seq_ids, n_seq=B)
+        step_fn(tokens, parents, shape.k, ins_l(shape), o, seq_ids=seq_ids, n_seq=B)
         launches += eng.launches()
         eng.commit(B, seq_ids=seq_ids)
         launches += eng.launches()
@@ -428,7 +437,7 @@ def main():
         e0.record()
         for i in range(K):
             d_tokens.copy_(h_tokens, non_blocking=True)
-            eng.step(d_tokens, parents, shape.k, ins_l(shape), o, seq_ids=seq_ids, n_seq=B)
+            step_fn(d_tokens, parents, shape.k, ins_l(shape), o, seq_ids=seq_ids, n_seq=B)
             eng.commit(B, seq_ids=seq_ids)
             h_acc.copy_(o.accepted_tokens, non_blocking=True)
             h_n.copy_(o.n_accepted, non_blocking=True)
@@ -459,7 +468,7 @@ def main():
     # ---- per-kernel-class durations (second, separately timed pass with events in the library) ----
     prof = None
     if not args.no_kernel_times:
-        prof = kernel_times(eng, shape, parents, tokens, outs[0], min(K, 8), n_end, peak_gbs, peak_kind, seq_ids)
+        prof = kernel_times(eng, shape, parents, tokens, outs[0], min(K, 8), n_end, peak_gbs, peak_kind, seq_ids, step_fn)
     ab = algorithmic_bytes(shape, n_mid, B)
     ms_step = ms_max / K
     step_gbs = ab["total"] / (ms_step * 1e-3) / 1e9
@@ -467,7 +476,7 @@ def main():
                 ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                 data="synthetic", gpu_launches=launches,
                 config=dict(workload=shape.name, T=shape.T, k=shape.k, l=ins_l(shape), context_start=n_start,
-                            context_end=n_end, batch=B, l2="inputs_larger_than_l2 (%.1f GB of weights per step)" %
+                            context_end=n_end, batch=B, pseudo_rows="a chain under every node" if chains else "one chain under the root", l2="inputs_larger_than_l2 (%.1f GB of weights per step)" %
                             (ab["weights"] / 1e9), parallelism="replicas x%d" % world,
                             mode="free-running greedy (random weights accept ~0 drafts per step)"),
                 step_latency_us=ms_step * 1e3, tokens_per_step=units / (K * world), tokens_per_step_per_sequence=units / (K * world * B),

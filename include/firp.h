@@ -56,6 +56,8 @@ typedef struct {
   int32_t max_k;      /* largest k (pseudo rows per sequence), <= 8 */
   int32_t max_depth;  /* largest tree depth; paths and accepted lists hold max_depth+1 entries */
   int32_t top_b;      /* candidates kept per pseudo row, 1..8 */
+  int32_t max_rows;   /* rows one step may carry over all its sequences, <= 144; 0 = max_batch * (max_tree +
+                         max_k).  firp_step_chains needs n_seq * T * (1 + k) rows: raise it for that call. */
 } firp_model_cfg;
 
 /* Device pointers to bf16 weights.  wqkv..g_mlp are HOST arrays of n_layers device pointers.
@@ -148,6 +150,25 @@ int firp_prefill_layers(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int
                         const int32_t *layers, const int32_t *next_parents, int32_t T_next,
                         const firp_step_out *out, void *stream);
 int firp_step_layers(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
+                     const int32_t *tree_parents, int32_t T, int32_t k, const int32_t *layers,
+                     const firp_step_out *out, void *stream);
+
+/*
+ * The step with a chain of k pseudo rows under EVERY tree node instead of one chain under the
+ * root.  Section 3.4 draws the next candidates from the accepted sequence, which a tree step only
+ * knows after the pass; with a chain per node the next tree is read from the chain of the node the
+ * acceptance walk ends on, so depth-j candidates are predictions for exactly the position they
+ * will occupy (with the single chain of firp_step they are predictions made from the root).
+ * Rows per sequence: T tree rows, then chain row i (1-based) of node v at row T + (i-1) T + v,
+ * T (1 + k) in all (depth, mask, logits of `out` have that many rows; best, path, accepted,
+ * next_tree_tokens as in firp_step; topb_ids / topb_vals [n_seq][k][B] are those of the end node's
+ * chain).  Chain row i of node v is W_i h[v] + b_i (Eq. 3) on v's residual entering layer
+ * layers[i-1], stands for position pos[v] + i and sees what v sees, rows 1..i-1 of its own chain
+ * and itself (Section 3.3).  layers as in firp_step_layers.  Needs n_seq * T * (1 + k) <= max_rows
+ * and context + T (1 + k) <= max_ctx; prefill is firp_prefill / firp_prefill_layers (only the last
+ * prompt row needs a chain).  firp_kv_commit follows as after firp_step.
+ */
+int firp_step_chains(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
                      const int32_t *tree_parents, int32_t T, int32_t k, const int32_t *layers,
                      const firp_step_out *out, void *stream);
 

@@ -26,7 +26,7 @@ FIRP_ERR_DEVICE_TIMEOUT = -6
 class ModelCfg(ctypes.Structure):
     _fields_ = [(n, i32) for n in ("n_layers", "d_model", "n_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab")] + \
                [("rms_eps", ctypes.c_float), ("rope_theta", ctypes.c_float)] + \
-               [(n, i32) for n in ("max_batch", "max_ctx", "max_tree", "max_k", "max_depth", "top_b")]
+               [(n, i32) for n in ("max_batch", "max_ctx", "max_tree", "max_k", "max_depth", "top_b", "max_rows")]
 
 
 _PP = ctypes.POINTER(vp)
@@ -45,7 +45,7 @@ class StepOutC(ctypes.Structure):
 EXPORTS = ("firp_create", "firp_destroy", "firp_last_error", "firp_workspace_bytes", "firp_kv_bytes",
            "firp_bind_buffers", "firp_init_weights", "firp_prefill", "firp_step", "firp_kv_commit",
            "firp_context_len", "firp_set_context_len", "firp_last_launch_count", "firp_profile_enable",
-           "firp_profile_read", "firp_kernel_class_name", "firp_topb_static", "firp_prefill_layers", "firp_step_layers")
+           "firp_profile_read", "firp_kernel_class_name", "firp_topb_static", "firp_prefill_layers", "firp_step_layers", "firp_step_chains")
 
 
 def lib_path() -> str:
@@ -76,6 +76,7 @@ def load_library():
     lib.firp_step.argtypes = [vp, i32, vp, vp, vp, i32, i32, i32, ctypes.POINTER(StepOutC), vp]
     lib.firp_prefill_layers.argtypes = [vp, i32, vp, i32, i32, vp, vp, i32, ctypes.POINTER(StepOutC), vp]
     lib.firp_step_layers.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp, ctypes.POINTER(StepOutC), vp]
+    lib.firp_step_chains.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp, ctypes.POINTER(StepOutC), vp]
     lib.firp_kv_commit.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.firp_context_len.argtypes = [vp, i32, ctypes.POINTER(i32), vp]
     lib.firp_set_context_len.argtypes = [vp, i32, i32, vp]
@@ -174,6 +175,18 @@ def firp_step(ctx, n_seq: int, seq_ids, d_tokens_ptr: int, tree_parents, T: int,
                                          ctypes.byref(out) if out is not None else None, stream))
 
 
+def firp_step_chains(ctx, n_seq: int, seq_ids, d_tokens_ptr: int, tree_parents, T: int, k: int, layers, out: StepOutC,
+                     stream: int = 0):
+    """A chain of k pseudo rows under every tree node; layers: one insertion layer per prediction step."""
+    ids, ids_ptr = _host_i32(seq_ids)
+    par, par_ptr = _host_i32(tree_parents)
+    lay, lay_ptr = _host_i32(layers)
+    if k > 0 and (lay is None or lay.size != k):
+        raise ValueError("need one insertion layer per prediction step")
+    _check(ctx, load_library().firp_step_chains(ctx, n_seq, ids_ptr, d_tokens_ptr, par_ptr, T, k, lay_ptr,
+                                                ctypes.byref(out) if out is not None else None, stream))
+
+
 def firp_kv_commit(ctx, n_seq: int, seq_ids=None, path=None, path_len=None, stream: int = 0):
     ids, ids_ptr = _host_i32(seq_ids)
     p, p_ptr = _host_i32(path)
@@ -227,15 +240,16 @@ def firp_topb_static(d_logits_ptr: int, rows: int, vocab: int, b: int, d_ids_ptr
 class StepOut:
     """Device output buffers of one step (torch tensors) and their C view."""
 
-    def __init__(self, torch, device, n_seq, T, k, V, S, B, T_next=None, want_logits=True):
+    def __init__(self, torch, device, n_seq, T, k, V, S, B, T_next=None, want_logits=True, chains=False):
         T_next = T if T_next is None else T_next
+        M = T * (1 + k) if chains else T + k          # rows per sequence
         z = lambda *shape, dt=torch.int32: torch.zeros(*shape, dtype=dt, device=device)
         self.accepted_tokens, self.n_accepted, self.path = z(n_seq, S), z(n_seq), z(n_seq, S)
         self.next_tree_tokens, self.best = z(n_seq, max(T_next, 1)), z(n_seq, T)
         self.topb_ids, self.topb_vals = z(n_seq, max(k, 1), B), z(n_seq, max(k, 1), B, dt=torch.float32)
-        self.logits = z(n_seq, T + k, V, dt=torch.float32) if want_logits else None
-        self.depth = z(n_seq, T + k)
-        self.mask = z(n_seq, T + k, (T + k + 31) // 32)
+        self.logits = z(n_seq, M, V, dt=torch.float32) if want_logits else None
+        self.depth = z(n_seq, M)
+        self.mask = z(n_seq, M, (M + 31) // 32)
         self.c = StepOutC(**{n: (getattr(self, n).data_ptr() if getattr(self, n) is not None else None)
                              for n, _ in StepOutC._fields_})
 
@@ -244,7 +258,7 @@ class FirpEngine:
     """Owns a context plus the torch tensors backing its workspace, KV cache and weights."""
 
     def __init__(self, shape, weights, max_ctx, max_batch=1, max_tree=None, max_k=None, max_depth=None, top_b=8,
-                 device="cuda:0"):
+                 device="cuda:0", max_rows=0):
         import torch
         self.torch, self.device, self.shape = torch, torch.device(device), shape
         s = shape
@@ -253,7 +267,7 @@ class FirpEngine:
         max_depth = max(max_k, 1) if max_depth is None else max_depth
         self.cfg = ModelCfg(n_layers=s.L, d_model=s.d, n_heads=s.H, n_kv_heads=s.Hkv, head_dim=s.dh, d_ffn=s.F,
                             vocab=s.V, rms_eps=s.eps, rope_theta=s.theta, max_batch=max_batch, max_ctx=max_ctx,
-                            max_tree=max_tree, max_k=max_k, max_depth=max_depth, top_b=top_b)
+                            max_tree=max_tree, max_k=max_k, max_depth=max_depth, top_b=top_b, max_rows=max_rows)
         self.S, self.B = max_depth + 1, top_b
         self.ctx = firp_create(self.cfg)
         with torch.cuda.device(self.device):
@@ -292,8 +306,8 @@ class FirpEngine:
         self.w = w
         firp_init_weights(self.ctx, w)
 
-    def new_out(self, n_seq, T, k, T_next=None, want_logits=True) -> StepOut:
-        return StepOut(self.torch, self.device, n_seq, T, k, self.shape.V, self.S, self.B, T_next, want_logits)
+    def new_out(self, n_seq, T, k, T_next=None, want_logits=True, chains=False) -> StepOut:
+        return StepOut(self.torch, self.device, n_seq, T, k, self.shape.V, self.S, self.B, T_next, want_logits, chains)
 
     def prefill(self, seq, d_prompt, k, l, next_parents, out: StepOut):
         """l: one insertion layer, or a sequence of k layers (one per prediction step)."""
@@ -306,6 +320,13 @@ class FirpEngine:
         T = len(parents)
         fn = firp_step if np.isscalar(l) else firp_step_layers
         fn(self.ctx, n_seq, seq_ids, d_tokens.data_ptr(), parents, T, k, l, out.c if out is not None else None, self.stream)
+
+    def step_chains(self, d_tokens, parents, k, l, out: StepOut, seq_ids=None, n_seq=1):
+        """The step with a chain of k pseudo rows under every tree node (out from new_out(..., chains=True));
+        l: one insertion layer, or one per prediction step."""
+        layers = [l] * k if np.isscalar(l) else l
+        firp_step_chains(self.ctx, n_seq, seq_ids, d_tokens.data_ptr(), parents, len(parents), k, layers,
+                         out.c if out is not None else None, self.stream)
 
     def commit(self, n_seq=1, seq_ids=None, path=None, path_len=None):
         if path is not None:

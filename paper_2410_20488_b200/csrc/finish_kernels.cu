@@ -193,7 +193,14 @@ __global__ void __launch_bounds__(kThreads) pseudo_finish_kernel(Partials p, Gem
       r.x += __bfloat162float(a.pred_b[n]); r.y += __bfloat162float(a.pred_b[n + 1]);
       r.z += __bfloat162float(a.pred_b[n + 2]); r.w += __bfloat162float(a.pred_b[n + 3]);
     }
-    *reinterpret_cast<float4 *>(a.h_rows + (size_t)(it.m * a.rw.Ms + a.rw.T + i) * a.K + o) = r;
+    size_t row;
+    if (a.rw.chains) {
+      const int s = it.m / a.rw.T, v = it.m - s * a.rw.T;
+      row = (size_t)s * a.rw.Ms + a.rw.T + (size_t)(a.pseudo0 + i) * a.rw.T + v;
+    } else {
+      row = (size_t)it.m * a.rw.Ms + a.rw.T + a.pseudo0 + i;
+    }
+    *reinterpret_cast<float4 *>(a.h_rows + row * a.K + o) = r;
   }
 }
 

@@ -78,7 +78,7 @@ struct firp_ctx {
     const int d = cfg.d_model, nq = cfg.n_heads * cfg.head_dim, half = cfg.head_dim / 2;
     const size_t R = Rmax;
     h = c.take<float>(R * d);
-    xp = c.take<bf16>(2 * (size_t)kMaxSeq * d);   // anchor rows of Eq. 3: hi plane, lo plane
+    xp = c.take<bf16>(2 * R * d);           // the rows Eq. 3 reads (anchor of each sequence, or all tree rows): hi plane, lo plane
     x = c.take<bf16>(3 * R * d);            // normalised activations: hi plane, lo plane, third plane (QKV input)
     q = c.take<bf16>(2 * R * nq);
     o = c.take<bf16>(2 * R * nq);
@@ -243,30 +243,32 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     g.next_W = (const bf16 *)W; g.next_epi = epi; g.next_N = N; g.next_K = K; g.next_F = F; g.next_heads = H + 2 * Hkv;
     g.next_dh = dh; g.next_units = next_units[cls];
   };
-  int alive = 0;   // pseudo rows appended below this layer
+  int alive = 0;   // prediction steps appended below this layer
+  const int per_step = rw.chains ? rw.T : 1;                   // pseudo rows one prediction step adds per sequence
   for (int j = 0; j < cfg.n_layers; ++j) {
     int ins = 0;     // prediction steps whose layer this is
-    while (alive + ins < rw.k && ra.tl[alive + ins] == j) ++ins;
+    while (alive + ins < rw.kc && ra.tl[alive + ins] == j) ++ins;
     const bool insert = ins > 0;
     // the rows that took part in the last residual GEMM get its pending sums; new pseudo rows have none
-    const int carried = rw.T + alive;
-    const int act = carried + ins;                             // rows alive in this layer
+    const int carried = rw.T + alive * per_step;
+    const int act = carried + ins * per_step;                  // rows alive in this layer
     { FIRP_TIMED(KC_RMSNORM);
       FIRP_CUDA(c, launch_rmsnorm(rw, 0, carried, c->h, pending, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, 3, c->ss, pdl, st)); ++nl; }
     pending.sk.U = 0;
     if (insert) {   // Eq. 3 on the raw (now complete) residual row of the root, then the norm of the new rows
-      { FIRP_TIMED(KC_PSEUDO_PROJ);      // this layer's maps as one [ins d][d] GEMM on the anchor rows (one row per sequence)
-        launch_root_split(rw, c->h, d, c->xp, (size_t)kMaxSeq * d, pdl, st); ++nl;
+      { FIRP_TIMED(KC_PSEUDO_PROJ);      // this layer's maps as one [ins d][d] GEMM on the source rows (the anchor of
+                                         // each sequence, or every tree row when each node carries a chain)
+        launch_root_split(rw, c->h, d, c->xp, Rp * d, pdl, st); ++nl;
         GemmArgs g{};
-        g.X = c->xp; g.x_lo_off = (size_t)kMaxSeq * d; g.plane_rows = kMaxSeq; g.planes = 2; g.err = c->dev_status;
-        g.W = (const bf16 *)c->w.pred_w + (size_t)alive * d * d; g.R = rw.n_seq; g.N = ins * d; g.K = d; g.rw = rw;
+        g.X = c->xp; g.x_lo_off = Rp * d; g.plane_rows = (int)Rp; g.planes = 2; g.err = c->dev_status;
+        g.W = (const bf16 *)c->w.pred_w + (size_t)alive * d * d; g.R = rw.n_seq * per_step; g.N = ins * d; g.K = d; g.rw = rw;
         g.rows_active = act;
         g.ws = c->gemm_ws; g.l2_ahead = 48;
-        g.h_rows = c->h + (size_t)alive * d;     // map i of this GEMM fills pseudo row alive + i
+        g.h_rows = c->h; g.pseudo0 = alive;      // map i of this GEMM is prediction step alive + i
         g.pred_b = c->w.pred_b ? (const bf16 *)c->w.pred_b + (size_t)alive * d : nullptr;
         Partials p = pending;
         FIRP_CUDA(c, launch_gemm_tc(EPI_PSEUDO, g, pdl, st, &p.sk)); ++nl;
-        p.ws_rows = kMaxSeq;
+        p.ws_rows = (int)Rp;
         FIRP_CUDA(c, launch_gemm_finish(EPI_PSEUDO, p, g, pdl, st)); ++nl; }
       FIRP_TIMED(KC_RMSNORM);
       FIRP_CUDA(c, launch_rmsnorm(rw, carried, act, c->h, none, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, 3, c->ss, pdl, st)); ++nl;
@@ -378,8 +380,10 @@ int firp_create(const firp_model_cfg *cfg, firp_ctx **out) {
   if (cfg->max_depth < 0 || cfg->max_depth > 15) return bad("max_depth must be 0..15");
   if (cfg->top_b < 1 || cfg->top_b > kMaxTopB) return bad("top_b must be 1..8");
   if (cfg->max_ctx < cfg->max_tree + cfg->max_k) return bad("max_ctx too small");
-  const int rows = cfg->max_batch * (cfg->max_tree + cfg->max_k);
+  int rows = cfg->max_batch * (cfg->max_tree + cfg->max_k);
   if (rows > 144) return bad("max_batch * (max_tree + max_k) must be <= 144 rows");
+  if (cfg->max_rows < 0 || cfg->max_rows > 144) return bad("max_rows must be 0..144");
+  if (cfg->max_rows > rows) rows = cfg->max_rows;
   c->Rmax = (int)align_up(rows, 16);
   c->S = cfg->max_depth + 1;
   c->n_hi.assign(cfg->max_batch, 0);
@@ -482,9 +486,26 @@ int firp_step(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_
   return firp_step_layers(ctx, n_seq, seq_ids, d_tree_tokens, tree_parents, T, k, layers, out, stream);
 }
 
+// One chain of k pseudo rows under the root (chains = false) or under every tree node (chains = true).
+static int step_impl(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
+                     const int32_t *tree_parents, int32_t T, int32_t k, const int32_t *layers, bool chains,
+                     const firp_step_out *out, void *stream);
+
 int firp_step_layers(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
                      const int32_t *tree_parents, int32_t T, int32_t k, const int32_t *layers, const firp_step_out *out,
                      void *stream) {
+  return step_impl(ctx, n_seq, seq_ids, d_tree_tokens, tree_parents, T, k, layers, false, out, stream);
+}
+
+int firp_step_chains(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
+                     const int32_t *tree_parents, int32_t T, int32_t k, const int32_t *layers, const firp_step_out *out,
+                     void *stream) {
+  return step_impl(ctx, n_seq, seq_ids, d_tree_tokens, tree_parents, T, k, layers, true, out, stream);
+}
+
+static int step_impl(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
+                     const int32_t *tree_parents, int32_t T, int32_t k, const int32_t *layers, bool chains,
+                     const firp_step_out *out, void *stream) {
   int rc = check_ready(ctx);
   if (rc) return rc;
   const firp_model_cfg &cfg = ctx->cfg;
@@ -495,7 +516,10 @@ int firp_step_layers(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const
   if ((rc = check_layers(ctx, k, layers))) return rc;
   std::vector<int32_t> ids;
   if ((rc = check_seq_ids(ctx, n_seq, seq_ids, ids))) return rc;
-  if (n_seq * (T + k) > ctx->Rmax) return fail(ctx, FIRP_ERR_CAPACITY, "n_seq * (T + k) exceeds the row capacity");
+  const int pseudo = chains ? T * k : k;       // pseudo rows per sequence
+  const int Ms = T + pseudo;
+  if (Ms > kMaxTreeRows || n_seq * Ms > ctx->Rmax)
+    return fail(ctx, FIRP_ERR_CAPACITY, "%d sequences x %d rows exceed the row capacity %d (max_rows of the configuration)", n_seq, Ms, ctx->Rmax);
   std::vector<int> depth;
   const int maxd = tree_depths(tree_parents, T, depth);
   if (maxd < 0) return fail(ctx, FIRP_ERR_BAD_TREE, "parents[0] must be -1 and 0 <= parents[v] < v");
@@ -504,7 +528,7 @@ int firp_step_layers(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const
   if (k > 0 && max_sibling_rank(tree_parents, T) >= cfg.top_b) return fail(ctx, FIRP_ERR_BAD_TREE, "more siblings than top_b");
   int n_hi_max = 0;
   for (int s = 0; s < n_seq; ++s) {
-    if (ctx->n_hi[ids[s]] + T + k > cfg.max_ctx) return fail(ctx, FIRP_ERR_CAPACITY, "slot %d: context + rows exceeds max_ctx", ids[s]);
+    if (ctx->n_hi[ids[s]] + Ms > cfg.max_ctx) return fail(ctx, FIRP_ERR_CAPACITY, "slot %d: context + rows exceeds max_ctx", ids[s]);
     n_hi_max = ctx->n_hi[ids[s]] > n_hi_max ? ctx->n_hi[ids[s]] : n_hi_max;
   }
   ctx->launches = 0;
@@ -515,7 +539,7 @@ int firp_step_layers(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const
   if ((rc = upload_i32(ctx, ctx->next_parents, k > 0 ? tree_parents : &one, T_next, ctx->last_next_parents, st))) return rc;
 
   RunArgs ra{};
-  ra.rw = Rows{n_seq, T, k, T + k, n_seq * (T + k), 0};
+  ra.rw = Rows{n_seq, T, pseudo, Ms, n_seq * Ms, 0, chains ? 1 : 0, k};
   for (int i = 0; i < k; ++i) ra.tl[i] = layers[i];
   ra.d_tokens = d_tree_tokens; ra.want_head = true; ra.prefill_last_row = -1; ra.T_next = T_next;
   ra.out = out; ra.logits_dst = (out && out->logits) ? out->logits : ctx->logits; ra.n_hi_max = n_hi_max;
@@ -567,7 +591,7 @@ int firp_prefill_layers(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int
     const bool last = (p0 + Tc == P);
     const int kc = last ? k : 0;
     RunArgs ra{};
-    ra.rw = Rows{1, Tc, kc, Tc + kc, Tc + kc, Tc - 1};
+    ra.rw = Rows{1, Tc, kc, Tc + kc, Tc + kc, Tc - 1, 0, kc};
     for (int i = 0; i < kc; ++i) ra.tl[i] = layers[i];
     ra.d_tokens = d_prompt + p0; ra.want_head = last; ra.prefill_last_row = Tc - 1; ra.T_next = T_next;
     ra.out = nullptr; ra.logits_dst = ctx->logits; ra.n_hi_max = ctx->n_hi[seq];

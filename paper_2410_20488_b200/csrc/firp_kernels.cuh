@@ -9,7 +9,7 @@ namespace firp {
 typedef __nv_bfloat16 bf16;
 
 constexpr int kMaxSeq = 16;        // sequences per step
-constexpr int kMaxTreeRows = 136;  // T + k per sequence (128 + 8)
+constexpr int kMaxTreeRows = 144;  // rows per sequence: T + k (128 + 8), or T (1 + k) with a chain under every node
 constexpr int kMaskWords = 5;      // ceil(136 / 32)
 constexpr int kMaxTopB = 8;
 constexpr int kAttnTile = 64;      // kv positions per attention tile
@@ -23,7 +23,9 @@ struct Rows {
   int k;       // pseudo rows per sequence
   int Ms;      // T + k
   int R;       // n_seq * Ms
-  int anchor;  // tree row the pseudo chain hangs off
+  int anchor;  // tree row the pseudo chain hangs off (one chain)
+  int chains;  // != 0: a chain under every tree node; chain row i (1-based) of node v is row T + (i-1) T + v
+  int kc;      // prediction steps per chain (k = kc with one chain, k = T * kc with a chain per node)
 };
 
 constexpr int kGemmMaxCtas = 192;         // scratch slots are provided for this many CTAs
@@ -87,7 +89,8 @@ cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Parti
                            bf16 *x, size_t x_lo_off, int planes, float *ss, bool pdl, cudaStream_t st);
 
 // Eq. 3, h[s*Ms + T + i] = W_i h[s*Ms + anchor] + b_i, as a GEMM of the k maps stacked into one [k d][d] matrix:
-// launch_root_split writes the raw residual row of every sequence's anchor as (hi, lo) bf16 planes into row s of
+// launch_root_split writes the raw residual rows Eq. 3 reads (every sequence's anchor, or all its T tree rows when
+// every node carries a chain: row s * T + v) as (hi, lo) bf16 planes; one chain: into row s of
 // xp; the GEMM (EPI_PSEUDO) multiplies; launch_gemm_finish(EPI_PSEUDO) sums the partial tiles, adds the bias and
 // stores the k new residual rows (GemmArgs: h_rows = residual stream, pred_b = bias or NULL, R = n_seq).
 void launch_root_split(const Rows &rw, const float *h, int d, bf16 *xp, size_t xp_lo_off, bool pdl, cudaStream_t st);
@@ -163,8 +166,10 @@ struct GemmArgs {
   bf16 *y; size_t y_lo_off; int F;
   // EPI_LOGITS: logits[R][N]
   float *logits;
-  // EPI_PSEUDO: row m = sequence m; output n = i * K + o goes to h_rows[(m * Ms + T + i) * K + o] (+ pred_b[n])
-  float *h_rows; const bf16 *pred_b;
+  // EPI_PSEUDO: output n = i * K + o of map pseudo0 + i (+ pred_b[n]).  One chain: row m = sequence m, result to
+  // h_rows[(m * Ms + T + pseudo0 + i) * K + o].  A chain per node: row m = s * T + v, result to
+  // h_rows[(s * Ms + T + (pseudo0 + i) * T + v) * K + o].
+  float *h_rows; const bf16 *pred_b; int pseudo0;
 };
 // The GEMM leaves partial tiles in a.ws under the schedule *sk_out, to be finished by launch_gemm_finish
 // (or, for EPI_RESIDUAL, by launch_rmsnorm).  `epi` only selects how weight rows are grouped into supertiles.

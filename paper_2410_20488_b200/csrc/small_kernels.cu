@@ -22,6 +22,7 @@ __global__ void tree_prep_kernel(Rows rw, const int32_t *parents, const int32_t 
   for (int v = tid; v < rw.Ms; v += blockDim.x) {
     int p;
     if (v < rw.T) p = parents[v];
+    else if (rw.chains) p = v - rw.T;   // step 1 of node u (row T + u) hangs off u, step i off step i-1 of the same node
     else p = (v == rw.T) ? rw.anchor : v - 1;
     ext[v] = p;
   }
@@ -184,9 +185,12 @@ root_split_kernel(Rows rw, const float *h, int d, bf16 *xp, size_t xp_lo_off, in
   if (pdl) { griddep_launch(); griddep_wait(); }
   const int nvec = d >> 2;
   const unsigned t = blockIdx.x * 256 + threadIdx.x;
-  if (t >= (unsigned)(rw.n_seq * nvec)) return;
-  const int s = (int)(t / (unsigned)nvec), idx = (int)(t % (unsigned)nvec);
-  const float4 a = __ldcg(reinterpret_cast<const float4 *>(h + (size_t)(s * rw.Ms + rw.anchor) * d) + idx);
+  const int per_seq = rw.chains ? rw.T : 1;                 // source rows per sequence
+  if (t >= (unsigned)(rw.n_seq * per_seq * nvec)) return;
+  const int m = (int)(t / (unsigned)nvec), idx = (int)(t % (unsigned)nvec);
+  const int sq = m / per_seq, v = rw.chains ? m - sq * per_seq : rw.anchor;
+  const int s = m;                                          // destination row in xp
+  const float4 a = __ldcg(reinterpret_cast<const float4 *>(h + (size_t)(sq * rw.Ms + v) * d) + idx);
   const __nv_bfloat162 o01 = __floats2bfloat162_rn(a.x, a.y), o23 = __floats2bfloat162_rn(a.z, a.w);
   const float2 f01 = __bfloat1622float2(o01), f23 = __bfloat1622float2(o23);
   const __nv_bfloat162 l01 = __floats2bfloat162_rn(a.x - f01.x, a.y - f01.y), l23 = __floats2bfloat162_rn(a.z - f23.x, a.w - f23.y);
@@ -198,7 +202,7 @@ root_split_kernel(Rows rw, const float *h, int d, bf16 *xp, size_t xp_lo_off, in
 }
 
 void launch_root_split(const Rows &rw, const float *h, int d, bf16 *xp, size_t xp_lo_off, bool pdl, cudaStream_t st) {
-  const int threads = rw.n_seq * (d >> 2);
+  const int threads = rw.n_seq * (rw.chains ? rw.T : 1) * (d >> 2);
   launch_k(root_split_kernel, dim3((threads + 255) / 256), dim3(256), 0, st, pdl, rw, h, d, xp, xp_lo_off, pdl ? 1 : 0);
 }
 
@@ -295,7 +299,7 @@ void launch_topb(const float *logits, int R, int V, int B, int32_t *cand_ids, fl
 // ---------------------------------------------------------------------------
 __global__ void accept_kernel(Rows rw, AcceptArgs a, int pdl) {
   __shared__ int32_t s_best[kMaxTreeRows];
-  __shared__ int32_t s_bonus;
+  __shared__ int32_t s_bonus, s_end;
   if (pdl) { griddep_launch(); griddep_wait(); }
   const int s = blockIdx.x, tid = threadIdx.x;
   const int32_t *tok = a.tokens + (size_t)s * rw.T;
@@ -303,13 +307,6 @@ __global__ void accept_kernel(Rows rw, AcceptArgs a, int pdl) {
     const int32_t b = a.top_ids[(size_t)(s * rw.Ms + v) * a.B];
     s_best[v] = b;
     if (a.o_best) a.o_best[(size_t)s * rw.T + v] = b;
-  }
-  if (a.o_topb_ids || a.o_topb_vals) {
-    for (int i = tid; i < rw.k * a.B; i += blockDim.x) {
-      const size_t src = (size_t)(s * rw.Ms + rw.T) * a.B + i;
-      if (a.o_topb_ids) a.o_topb_ids[(size_t)s * rw.k * a.B + i] = a.top_ids[src];
-      if (a.o_topb_vals) a.o_topb_vals[(size_t)s * rw.k * a.B + i] = a.top_vals[src];
-    }
   }
   __syncthreads();
   if (tid == 0) {
@@ -331,6 +328,7 @@ __global__ void accept_kernel(Rows rw, AcceptArgs a, int pdl) {
     }
     acc[na] = s_best[cur];
     s_bonus = s_best[cur];
+    s_end = cur;
     a.n_accepted[s] = na + 1;
     if (a.o_n_accepted) a.o_n_accepted[s] = na + 1;
     for (int j = 0; j <= na; ++j) {
@@ -339,6 +337,18 @@ __global__ void accept_kernel(Rows rw, AcceptArgs a, int pdl) {
     }
   }
   __syncthreads();
+  // the pseudo row that holds the candidates of depth j (1-based): row j of the one chain, or of the chain
+  // under the node the walk ended on
+  const int steps = rw.chains ? rw.kc : rw.k;
+  const size_t row0 = (size_t)s * rw.Ms + rw.T + (rw.chains ? s_end : 0);
+  const int row_step = rw.chains ? rw.T : 1;
+  if (a.o_topb_ids || a.o_topb_vals) {
+    for (int i = tid; i < steps * a.B; i += blockDim.x) {
+      const size_t src = (row0 + (size_t)(i / a.B) * row_step) * a.B + i % a.B;
+      if (a.o_topb_ids) a.o_topb_ids[(size_t)s * steps * a.B + i] = a.top_ids[src];
+      if (a.o_topb_vals) a.o_topb_vals[(size_t)s * steps * a.B + i] = a.top_vals[src];
+    }
+  }
   for (int v = tid; v < a.T_next; v += blockDim.x) {
     int32_t t;
     if (v == 0) {
@@ -348,9 +358,9 @@ __global__ void accept_kernel(Rows rw, AcceptArgs a, int pdl) {
       for (int u = v; u > 0 && dep <= a.T_next; u = a.next_parents[u]) ++dep;
       int rank = 0;
       for (int u = 1; u < v; ++u) rank += (a.next_parents[u] == a.next_parents[v]);
-      dep = min(dep, max(rw.k, 1));
+      dep = min(dep, max(steps, 1));
       rank = min(rank, a.B - 1);
-      t = (rw.k > 0) ? a.top_ids[(size_t)(s * rw.Ms + rw.T + dep - 1) * a.B + rank] : s_bonus;
+      t = (steps > 0) ? a.top_ids[(row0 + (size_t)(dep - 1) * row_step) * a.B + rank] : s_bonus;
     }
     a.next_tokens[(size_t)s * a.T_next + v] = t;
     if (a.o_next_tokens) a.o_next_tokens[(size_t)s * a.T_next + v] = t;

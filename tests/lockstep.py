@@ -60,12 +60,14 @@ class Stats:
                     max_abs=self.max_abs, max_rel=self.max_rel, emitted=self.emitted)
 
 
-def compare_step(shape, parents, tokens, k, g, ref, stats: Stats, tp=None, abs_tol=None):
-    """g: dict of numpy arrays from the CUDA path for ONE sequence; ref: oracle.step() output."""
+def compare_step(shape, parents, tokens, k, g, ref, stats: Stats, tp=None, abs_tol=None, chains=False):
+    """g: dict of numpy arrays from the CUDA path for ONE sequence; ref: oracle.step() output
+    (oracle.step_chains() with chains=True: a chain of k pseudo rows under every node, the candidates
+    are those of the chain under the node the walk ended on)."""
     abs_tol = ABS_TOL if abs_tol is None else abs_tol
     T, V = len(parents), shape.V
-    M = T + k
-    tp = tp or oracle.tree_prep(parents, k, 0)
+    M = T * (1 + k) if chains else T + k
+    tp = tp or (oracle.tree_prep_chains(parents, k) if chains else oracle.tree_prep(parents, k, 0))
     # (i) integer bookkeeping
     assert np.array_equal(g["depth"], ref["depth"]), "depth mismatch"
     assert np.array_equal(unpack_mask(g["mask"], M), ref["mask"]), "tree mask mismatch"
@@ -100,11 +102,14 @@ def compare_step(shape, parents, tokens, k, g, ref, stats: Stats, tp=None, abs_t
     ng = int(g["n_accepted"])
     assert ng == o["n_accepted"] and np.array_equal(g["path"][:ng], o["path"]) and \
         np.array_equal(g["accepted"][:ng], o["accepted"]), "acceptance walk is not the walk of its own argmax"
-    # (v) top-B of the pseudo rows
+    # (v) top-B of the pseudo rows (of the chain under the CUDA path's own end node; compared with the
+    # oracle's values of the same rows, which are its candidates too whenever the walks agree)
+    g_end = int(g["path"][ng - 1])
+    prow = (lambda i: oracle.chain_row(T, g_end, i + 1)) if chains else (lambda i: T + i)
     if k > 0:
         B = g["topb_ids"].shape[1]
         for i in range(k):
-            row = ref["logits"][T + i]
+            row = ref["logits"][prow(i)]
             order = np.lexsort((np.arange(V), -row))[: B + 1]
             vals = row[order]
             gaps = vals[:-1] - vals[1:]                      # gap after position b
@@ -118,7 +123,7 @@ def compare_step(shape, parents, tokens, k, g, ref, stats: Stats, tp=None, abs_t
             gv, gi = g["topb_vals"][i], g["topb_ids"][i]
             assert all(gv[b] > gv[b + 1] or (gv[b] == gv[b + 1] and gi[b] < gi[b + 1]) for b in range(B - 1)), \
                 "top-B not ordered by (value desc, id asc)"
-            assert np.array_equal(g["topb_ids"][i], np.lexsort((np.arange(V), -g["logits"][T + i]))[:B]), \
+            assert np.array_equal(g["topb_ids"][i], np.lexsort((np.arange(V), -g["logits"][prow(i)]))[:B]), \
                 "top-B is not the top-B of the CUDA path's own logits"
     # next tree as an integer function of the CUDA path's own top-B and bonus
     want_next = template_next(parents, tp, g["topb_ids"], int(g["accepted"][ng - 1]), k)
@@ -158,14 +163,15 @@ def check_cache(engine, orc, seq, slots, layers, tol=2e-2):
 
 
 def lockstep_run(engine, orc, shape, parents, prompt, steps, forced=False, k=None, l=None, check_cache_rows=True,
-                 compare_every=1, seq=0, abs_tol=None):
-    """Prefill both sides, then `steps` lock-step steps.  Returns a Stats."""
+                 compare_every=1, seq=0, abs_tol=None, chains=False):
+    """Prefill both sides, then `steps` lock-step steps (chains: with a chain of k pseudo rows under
+    every tree node, firp_step_chains against oracle.step_chains).  Returns a Stats."""
     abs_tol = ABS_TOL if abs_tol is None else abs_tol
     import torch
     k = shape.k if k is None else k
     l = shape.l if l is None else l
     T = len(parents)
-    tp = oracle.tree_prep(parents, k, 0)
+    tp = oracle.tree_prep_chains(parents, k) if chains else oracle.tree_prep(parents, k, 0)
     tp_tree = oracle.tree_prep(parents, 0, 0)
     D = int(tp_tree["depth"].max())
     chain = principal_chain(parents, tp_tree["depth"])
@@ -188,7 +194,7 @@ def lockstep_run(engine, orc, shape, parents, prompt, steps, forced=False, k=Non
     tokens = ref["next_tokens"].copy()
     emitted = [ref["root"]]
 
-    out = engine.new_out(1, T, k)
+    out = engine.new_out(1, T, k, chains=chains)
     for step in range(steps):
         if forced:
             gcont = orc.ar_greedy(int(tokens[0]), D, seq=seq)
@@ -199,11 +205,15 @@ def lockstep_run(engine, orc, shape, parents, prompt, steps, forced=False, k=Non
                         tokens[u] = tokens[v]
                 tokens[v] = gcont[j - 1]
         d_tokens = torch.from_numpy(np.ascontiguousarray(tokens, np.int32)).to(dev)
-        engine.step(d_tokens, parents, k, l, out, seq_ids=[seq])
-        ref = orc.step(tokens, parents, k, l, seq=seq)
+        if chains:
+            engine.step_chains(d_tokens, parents, k, l, out, seq_ids=[seq])
+            ref = orc.step_chains(tokens, parents, k, l, seq=seq)
+        else:
+            engine.step(d_tokens, parents, k, l, out, seq_ids=[seq])
+            ref = orc.step(tokens, parents, k, l, seq=seq)
         if step % compare_every == 0 or step == steps - 1:
             g = gpu_outputs(out, 0, T, k)
-            compare_step(shape, parents, tokens, k, g, ref, stats, tp, abs_tol)
+            compare_step(shape, parents, tokens, k, g, ref, stats, tp, abs_tol, chains=chains)
         if forced:
             assert ref["n_accepted"] == D + 1, "forced-accept step accepted %d of %d" % (ref["n_accepted"] - 1, D)
         n0 = orc.context_len(seq)

@@ -107,6 +107,39 @@ def test_layers_are_validated_on_the_host(torch_cuda, c1, c1_weights):
     eng.close()
 
 
+@pytest.mark.parametrize("case", range(4))
+def test_c1_a_chain_under_every_node(torch_cuda, c1, case):
+    """firp_step_chains: k pseudo rows under every tree node, next tree from the end node's chain;
+    lock-step against the oracle, greedy and forced, single and per-step insertion layers."""
+    T = (8, 5, 19, 36)[case]
+    k = (3, 1, 3, 3)[case]
+    layers = (1, 0, [0, 1, 3], [1, 2, 2])[case]
+    deep = not np.isscalar(layers)
+    shape = si.scaled(c1, L=4 if deep else 2, l=1)
+    weights = si.all_weights(shape)
+    parents = si.tree_template(8) if case == 0 else si.random_tree(9, T, k, case)
+    for forced in (False, True):
+        eng, orc = make_pair(shape, weights, 512, max_tree=64, max_k=3, max_depth=3, max_rows=T * (1 + k))
+        st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=(32, 3, 70, 131)[case]), 4, forced=forced,
+                          k=k, l=layers, chains=True)
+        assert st.steps == 4
+        eng.close()
+
+
+def test_chains_need_the_row_capacity(torch_cuda, c1, c1_weights):
+    import torch
+    from paper_2410_20488_b200 import FirpError, binding
+    eng, _ = make_pair(c1, c1_weights, 128)                                   # max_rows defaults to T + k = 11
+    tok = torch.zeros(8, dtype=torch.int32, device="cuda")
+    out = eng.new_out(1, 8, 3, chains=True)
+    pout = eng.new_out(1, 1, 3, T_next=8)
+    eng.prefill(0, torch.from_numpy(si.prompt(c1)).cuda(), 3, 1, si.tree_template(8), pout)
+    with pytest.raises(FirpError) as e:
+        eng.step_chains(tok, si.tree_template(8), 3, 1, out)
+    assert e.value.code == binding.FIRP_ERR_CAPACITY and "max_rows" in str(e.value)
+    eng.close()
+
+
 def test_c1_predictor_with_bias(torch_cuda, c1, c1_weights):
     """Eq. 3 with a non-zero bias b_i (the synthetic configurations use b = 0)."""
     w = dict(c1_weights)
@@ -191,6 +224,18 @@ def test_c2_layers_15_20_25_full_size(torch_cuda, c2_weights):
     st = lockstep_run(eng, orc, c2, parents, si.prompt(c2), 2, forced=False, check_cache_rows=False, l=[15, 20, 25])
     print("c2 layers 15/20/25", st.as_dict())
     assert st.steps == 2
+    eng.close()
+
+
+def test_c2_chain_under_every_node_full_size(torch_cuda, c2_weights):
+    """T = 32 nodes each with a chain of k = 3 pseudo rows (128 rows from layer 16 on) at the 7B shape:
+    prefill and one lock-step step against the oracle."""
+    c2 = si.CONFIGS["c2"]
+    parents = si.tree_template(c2.T)
+    eng, orc = make_pair(c2, c2_weights, 512 + 160, max_rows=c2.T * (1 + c2.k))
+    st = lockstep_run(eng, orc, c2, parents, si.prompt(c2), 1, forced=False, check_cache_rows=False, chains=True)
+    print("c2 chains", st.as_dict())
+    assert st.steps == 1
     eng.close()
 
 
