@@ -530,6 +530,10 @@ Sched make_sched(GemmEpilogue epi, const GemmArgs &a, bool pdl) {
   sc.sk.KB = (a.K + BK - 1) / BK;
   sc.sk.U = sc.n_st * sc.sk.KB;
   sc.sk.G = std::min(sm_count(), sc.sk.U);
+  // With more than 80 rows the MMAs fall behind the weight stream, and a lookahead beyond the ring only fills L2
+  // with tiles that are evicted before they are read and then fetched twice (measured at 140 rows: 1.8x the weight
+  // bytes from DRAM, step 10 % slower).  With few rows the stream is the bound and the deep lookahead pays.
+  if (a.R > 80) sc.l2_ahead = 0;
   return sc;
 }
 
