@@ -156,7 +156,9 @@ template <int NPAD, int P> struct TcCfg {
   static constexpr int NBUF = (2 * TM * ACC_COLS <= 512) ? 2 : 1;   // accumulator buffers
   static constexpr int TMEM_COLS = pow2_cols(NBUF * TM * ACC_COLS);
   // ring depths: as many 32 KB weight stages as fit beside two to four activation stages
-  static constexpr int SX = X_STAGE <= 8 * 1024 ? 4 : (X_STAGE <= 20 * 1024 ? 3 : 2);
+  // (an activation stage of the 144-row variant is 36 KB and comes from L2 in ~2 us: with two stages that
+  // latency, not the weight stream or the MMAs, set the pace of a unit; three stages beside three weight stages)
+  static constexpr int SX = X_STAGE <= 8 * 1024 ? 4 : (X_STAGE <= 40 * 1024 ? 3 : 2);
   static constexpr int SW = (227 * 1024 - 1280 - SX * X_STAGE) / W_STAGE > 6 ? 6 : (227 * 1024 - 1280 - SX * X_STAGE) / W_STAGE;
   static constexpr int RING_BYTES = SW * W_STAGE + SX * X_STAGE;
   static constexpr int SMEM = RING_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
@@ -533,7 +535,8 @@ Sched make_sched(GemmEpilogue epi, const GemmArgs &a, bool pdl) {
   // With more than 80 rows the MMAs fall behind the weight stream, and a lookahead beyond the ring only fills L2
   // with tiles that are evicted before they are read and then fetched twice (measured at 140 rows: 1.8x the weight
   // bytes from DRAM, step 10 % slower).  With few rows the stream is the bound and the deep lookahead pays.
-  if (a.R > 80) sc.l2_ahead = 0;
+  static const int big_ahead = [] { const char *e = getenv("FIRP_BIG_AHEAD"); return e ? atoi(e) : 0; }();   // tuning aid
+  if (a.R > 80) sc.l2_ahead = std::min(sc.l2_ahead, big_ahead);
   return sc;
 }
 
