@@ -63,6 +63,8 @@ def _get_lib():
         lib.oracle_forward_chains.restype = i32
         lib.oracle_tree_prep_chains.argtypes = [vp, i32, i32, vp, vp, vp, vp]
         lib.oracle_tree_prep_chains.restype = i32
+        lib.oracle_set_masked.argtypes = [vp, i32]
+        lib.oracle_mask_pseudo.argtypes = [vp, i32, i32]
         lib.oracle_verify.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
         lib.oracle_verify.restype = i32
         lib.oracle_next_tree.argtypes = [vp, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp]
@@ -148,7 +150,9 @@ class Oracle:
     rounded once when stored); False keeps fp32 rows, for comparisons with an fp64 decoder.
     """
 
-    def __init__(self, shape, weights, max_ctx: int, n_seq: int = 1, top_b: int = 8, kv_bf16: bool = True):
+    def __init__(self, shape, weights, max_ctx: int, n_seq: int = 1, top_b: int = 8, kv_bf16: bool = True,
+                 masked: bool = False):
+        """masked: the "Masked" setting of Section 4.3 (a pseudo row sees no other pseudo row)."""
         self.lib = _get_lib()
         self.shape, self.weights, self.top_b = shape, weights, top_b
         s = shape
@@ -186,6 +190,7 @@ class Oracle:
         w.g_mlp = per_layer(lambda lw: lw["g_mlp"])
         self._w = w
         self.lib.oracle_set_weights(self.h, ctypes.byref(w))
+        self.lib.oracle_set_masked(self.h, int(masked))
 
     def __del__(self):
         if getattr(self, "h", None):

@@ -92,6 +92,7 @@ typedef struct {
 typedef struct {
   oracle_cfg cfg;
   oracle_weights w;
+  int32_t masked;  /* != 0: the "Masked" setting of Section 4.3: a pseudo row does not see other pseudo rows */
   int32_t *n;      /* committed length per sequence */
   float **kc;      /* per sequence: [L][max_ctx][Hkv*dh] */
   float **vc;
@@ -133,6 +134,16 @@ void oracle_destroy(void *h) {
 }
 
 void oracle_set_weights(void *h, const oracle_weights *w) { ((oracle_t *)h)->w = *w; }
+/* Section 4.3 compares "No masked" (a pseudo row sees the earlier rows of its chain; the default, what the paper
+ * adopts) with "Masked" (it sees none of them: only the prefix, its node's ancestors and node, and itself). */
+void oracle_set_masked(void *h, int32_t masked) { ((oracle_t *)h)->masked = masked; }
+
+/* The "Masked" setting applied to a visibility matrix of T tree rows + pseudo rows: pseudo rows keep what they
+ * see among the tree rows and themselves, and lose every other pseudo row. */
+void oracle_mask_pseudo(uint8_t *mask, int32_t T, int32_t M) {
+  for (int v = T; v < M; ++v)
+    for (int u = T; u < M; ++u) if (u != v) mask[(size_t)v * M + u] = 0;
+}
 int32_t oracle_context_len(void *h, int32_t seq) { return ((oracle_t *)h)->n[seq]; }
 /* Rewind the committed length (rows >= n become scratch again); n = 0 empties the cache. */
 void oracle_set_context_len(void *h, int32_t seq, int32_t n) { ((oracle_t *)h)->n[seq] = n; }
@@ -381,6 +392,7 @@ int32_t oracle_forward_layers(void *hnd, int32_t seq, const int32_t *tokens, con
   int32_t *src = (int32_t *)malloc(sizeof(int32_t) * (k + 1)), *step = (int32_t *)malloc(sizeof(int32_t) * (k + 1));
   int32_t rc = -1;
   if (oracle_tree_prep(parents, T, k, anchor, ext_parent, depth, mask, NULL) == 0) {
+    if (o->masked) oracle_mask_pseudo(mask, T, M);
     for (int i = 0; i < k; ++i) { src[i] = anchor; step[i] = i; }
     rc = forward_core(o, seq, tokens, T, k, src, step, tl, depth, mask, logit_row0, logits, dump_layer, h_dump, h_ins);
     if (depth_out) memcpy(depth_out, depth, sizeof(int32_t) * M);
@@ -407,6 +419,7 @@ int32_t oracle_forward_chains(void *hnd, int32_t seq, const int32_t *tokens, con
   int32_t *src = (int32_t *)malloc(sizeof(int32_t) * (pn + 1)), *step = (int32_t *)malloc(sizeof(int32_t) * (pn + 1));
   int32_t rc = -1;
   if (oracle_tree_prep_chains(parents, T, k, ext_parent, depth, mask, NULL) == 0) {
+    if (o->masked) oracle_mask_pseudo(mask, T, M);
     for (int i = 0; i < k; ++i)
       for (int v = 0; v < T; ++v) { src[i * T + v] = v; step[i * T + v] = i; }
     rc = forward_core(o, seq, tokens, T, pn, src, step, tl, depth, mask, logit_row0, logits, -1, NULL, h_ins);

@@ -38,11 +38,16 @@ def build_hf_llama(shape, weights):
     return model
 
 
-def hf_logits(model, token_ids):
-    """Plain causal forward, no cache: logits [len, V] as float64 numpy."""
+def hf_logits(model, token_ids, visible=None):
+    """Causal forward, no cache: logits [len, V] as float64 numpy.  visible: optional [len, len] 0/1
+    matrix replacing the causal mask (row r attends to column c iff visible[r, c])."""
     with torch.no_grad():
         ids = torch.as_tensor(np.asarray(token_ids, dtype=np.int64))[None]
-        return model(ids, use_cache=False).logits[0].numpy()
+        mask = None
+        if visible is not None:
+            vis = torch.as_tensor(np.asarray(visible, dtype=bool))
+            mask = torch.zeros(vis.shape, dtype=torch.float64).masked_fill(~vis, float("-inf"))[None, None]
+        return model(ids, attention_mask=mask, use_cache=False).logits[0].numpy()
 
 
 def hf_greedy(model, prompt_ids, count):
@@ -73,7 +78,7 @@ def hf_kv(model, token_ids):
     return ks, vs
 
 
-def hf_logits_with_replaced_rows(model, token_ids, layer, first_row, maps_w, maps_b, anchor_row):
+def hf_logits_with_replaced_rows(model, token_ids, layer, first_row, maps_w, maps_b, anchor_row, visible=None):
     """Causal forward in which, at the input of decoder layer `layer`, rows
     first_row.. are replaced by W_i h[anchor_row] + b_i (i = 0..len(maps_w)-1).
     `layer` may be a sequence with one layer per row: row first_row + i is then
@@ -99,7 +104,7 @@ def hf_logits_with_replaced_rows(model, token_ids, layer, first_row, maps_w, map
 
     handles = [model.model.layers[at].register_forward_pre_hook(make_hook(at), with_kwargs=True) for at in sorted(set(layers))]
     try:
-        return hf_logits(model, token_ids)
+        return hf_logits(model, token_ids, visible)
     finally:
         for h in handles:
             h.remove()

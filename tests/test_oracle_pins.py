@@ -14,6 +14,8 @@
   P11 a chain of k pseudo rows under every tree node: every chain row == a causal forward over prefix + the
       node's root path with rows replaced at the insertion layer(s); the root's chain == the single chain;
       mask == brute-force closure; the free-running decode stays lossless
+  P12 the "Masked" setting of Section 4.3: the chain == a forward over prefix + root + k rows replaced at the
+      insertion layer whose mask hides the pseudo rows from one another; step 1 and the tree rows are unchanged
 plus hand-worked cases for the mask, the acceptance walk, the tie rules and the next tree.
 """
 import os
@@ -309,6 +311,36 @@ def test_p11_decoding_with_chains_is_lossless_and_reads_the_end_nodes_chain(c1, 
         emitted += out["accepted"].tolist()
         tokens = out["next_tokens"].copy()
     assert emitted == want[: len(emitted)]                 # Eq. 1: the stream is the greedy stream
+
+
+# ---------------------------------------------------------------- P12
+def test_p12_masked_pseudo_rows_see_no_other_pseudo_row(c1, c1_weights, hf):
+    k, l = 3, 1
+    prompt = si.prompt(c1, length=15)
+    Wf = si.bf16_bits_to_f32(c1_weights["pred_w"]).astype(np.float64)
+    tokens, parents = si.random_tokens(c1, 8, 11), si.tree_template(8)
+    om = oracle.Oracle(c1, c1_weights, max_ctx=256, kv_bf16=False, masked=True)
+    on = fresh(c1, c1_weights)
+    for o in (om, on):
+        o.forward(prompt, si.chain_template(prompt.size), 0, 0)
+        o.commit(np.arange(prompt.size))
+    masked, plain = om.forward(tokens, parents, k, l), on.forward(tokens, parents, k, l)
+    n = prompt.size
+    # prefix, root and the k pseudo rows at positions n+1..n+k: causal, except that a pseudo row sees no other one
+    ids = list(prompt) + [int(tokens[0])] + [0] * k
+    L = len(ids)
+    vis = np.tril(np.ones((L, L), np.uint8))
+    vis[n + 1:, n + 1:] = np.eye(k, dtype=np.uint8)
+    ref = hf_logits_with_replaced_rows(hf, ids, l, n + 1, list(Wf), list(np.zeros((k, c1.d))), n, visible=vis)
+    assert np.abs(masked["logits"][8:] - ref[n + 1:]).max() < 1e-5
+    causal = hf_logits_with_replaced_rows(hf, ids, l, n + 1, list(Wf), list(np.zeros((k, c1.d))), n,
+                                          visible=np.tril(np.ones((L, L), np.uint8)))
+    assert np.abs(plain["logits"][8:] - causal[n + 1:]).max() < 1e-5            # the explicit causal mask is the default one
+    assert np.array_equal(masked["logits"][:9], plain["logits"][:9])          # tree rows and step 1 are the same
+    assert not np.array_equal(masked["logits"][9:], plain["logits"][9:])      # steps 2, 3 lost what they saw
+    want = plain["mask"].copy()
+    want[8:, 8:] = np.eye(k, dtype=np.uint8)
+    assert np.array_equal(masked["mask"], want) and np.array_equal(masked["depth"], plain["depth"])
 
 
 # ---------------------------------------------------------------- P5
