@@ -173,6 +173,14 @@ int firp_step_chains(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const
                      const firp_step_out *out, void *stream);
 
 /*
+ * Visibility among the pseudo rows (Section 4.3, ablation).  masked = 0 (default, the "No masked"
+ * setting the paper adopts): chain row i sees rows 1..i-1 of its chain.  masked != 0 ("Masked"): a
+ * pseudo row sees no other pseudo row, only the prefix, its node with its ancestors, and itself;
+ * positions are unchanged.  Applies to every later firp_prefill* / firp_step* call of the context.
+ */
+int firp_set_pseudo_masked(firp_ctx *ctx, int32_t masked);
+
+/*
  * Commit after a step: for each sequence move the cache rows of path[j] to slot n + j
  * (every layer, K and V) and advance n by path_len.  path (HOST [n_seq][max_depth+1]) and
  * path_len (HOST [n_seq]) give an explicit path (strictly increasing, path[0] = 0); NULL

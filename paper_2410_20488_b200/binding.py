@@ -45,7 +45,7 @@ class StepOutC(ctypes.Structure):
 EXPORTS = ("firp_create", "firp_destroy", "firp_last_error", "firp_workspace_bytes", "firp_kv_bytes",
            "firp_bind_buffers", "firp_init_weights", "firp_prefill", "firp_step", "firp_kv_commit",
            "firp_context_len", "firp_set_context_len", "firp_last_launch_count", "firp_profile_enable",
-           "firp_profile_read", "firp_kernel_class_name", "firp_topb_static", "firp_prefill_layers", "firp_step_layers", "firp_step_chains")
+           "firp_profile_read", "firp_kernel_class_name", "firp_topb_static", "firp_prefill_layers", "firp_step_layers", "firp_step_chains", "firp_set_pseudo_masked")
 
 
 def lib_path() -> str:
@@ -77,6 +77,7 @@ def load_library():
     lib.firp_prefill_layers.argtypes = [vp, i32, vp, i32, i32, vp, vp, i32, ctypes.POINTER(StepOutC), vp]
     lib.firp_step_layers.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp, ctypes.POINTER(StepOutC), vp]
     lib.firp_step_chains.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp, ctypes.POINTER(StepOutC), vp]
+    lib.firp_set_pseudo_masked.argtypes = [vp, i32]
     lib.firp_kv_commit.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.firp_context_len.argtypes = [vp, i32, ctypes.POINTER(i32), vp]
     lib.firp_set_context_len.argtypes = [vp, i32, i32, vp]
@@ -185,6 +186,11 @@ def firp_step_chains(ctx, n_seq: int, seq_ids, d_tokens_ptr: int, tree_parents, 
         raise ValueError("need one insertion layer per prediction step")
     _check(ctx, load_library().firp_step_chains(ctx, n_seq, ids_ptr, d_tokens_ptr, par_ptr, T, k, lay_ptr,
                                                 ctypes.byref(out) if out is not None else None, stream))
+
+
+def firp_set_pseudo_masked(ctx, masked: bool):
+    """Section 4.3 "Masked" ablation: pseudo rows do not see one another."""
+    _check(ctx, load_library().firp_set_pseudo_masked(ctx, int(bool(masked))))
 
 
 def firp_kv_commit(ctx, n_seq: int, seq_ids=None, path=None, path_len=None, stream: int = 0):
@@ -327,6 +333,9 @@ class FirpEngine:
         layers = [l] * k if np.isscalar(l) else l
         firp_step_chains(self.ctx, n_seq, seq_ids, d_tokens.data_ptr(), parents, len(parents), k, layers,
                          out.c if out is not None else None, self.stream)
+
+    def set_pseudo_masked(self, masked: bool):
+        firp_set_pseudo_masked(self.ctx, masked)
 
     def commit(self, n_seq=1, seq_ids=None, path=None, path_len=None):
         if path is not None:

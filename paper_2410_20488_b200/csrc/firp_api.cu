@@ -68,6 +68,7 @@ struct firp_ctx {
   std::vector<int32_t> n_hi;           // upper bound of each slot's committed length
   std::vector<int32_t> last_parents, last_next_parents, last_seq_ids;
   int last_n_seq = 0, last_T = 0, last_k = 0;
+  int pseudo_masked = 0;     // Section 4.3 "Masked": pseudo rows do not see one another
 
   size_t kv_plane() const { return (size_t)cfg.max_ctx * cfg.n_kv_heads * cfg.head_dim; }
   size_t kv_layer() const { return 2 * kv_plane(); }
@@ -539,7 +540,7 @@ static int step_impl(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const
   if ((rc = upload_i32(ctx, ctx->next_parents, k > 0 ? tree_parents : &one, T_next, ctx->last_next_parents, st))) return rc;
 
   RunArgs ra{};
-  ra.rw = Rows{n_seq, T, pseudo, Ms, n_seq * Ms, 0, chains ? 1 : 0, k};
+  ra.rw = Rows{n_seq, T, pseudo, Ms, n_seq * Ms, 0, chains ? 1 : 0, k, ctx->pseudo_masked};
   for (int i = 0; i < k; ++i) ra.tl[i] = layers[i];
   ra.d_tokens = d_tree_tokens; ra.want_head = true; ra.prefill_last_row = -1; ra.T_next = T_next;
   ra.out = out; ra.logits_dst = (out && out->logits) ? out->logits : ctx->logits; ra.n_hi_max = n_hi_max;
@@ -591,7 +592,7 @@ int firp_prefill_layers(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int
     const bool last = (p0 + Tc == P);
     const int kc = last ? k : 0;
     RunArgs ra{};
-    ra.rw = Rows{1, Tc, kc, Tc + kc, Tc + kc, Tc - 1, 0, kc};
+    ra.rw = Rows{1, Tc, kc, Tc + kc, Tc + kc, Tc - 1, 0, kc, ctx->pseudo_masked};
     for (int i = 0; i < kc; ++i) ra.tl[i] = layers[i];
     ra.d_tokens = d_prompt + p0; ra.want_head = last; ra.prefill_last_row = Tc - 1; ra.T_next = T_next;
     ra.out = nullptr; ra.logits_dst = ctx->logits; ra.n_hi_max = ctx->n_hi[seq];
@@ -609,6 +610,12 @@ int firp_prefill_layers(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int
   }
   FIRP_CUDA(ctx, cudaGetLastError());
   ctx->stepped = false;
+  return FIRP_OK;
+}
+
+int firp_set_pseudo_masked(firp_ctx *ctx, int32_t masked) {
+  if (!ctx) return FIRP_ERR_BAD_ARG;
+  ctx->pseudo_masked = masked ? 1 : 0;
   return FIRP_OK;
 }
 

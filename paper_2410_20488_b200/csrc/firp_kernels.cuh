@@ -26,6 +26,7 @@ struct Rows {
   int anchor;  // tree row the pseudo chain hangs off (one chain)
   int chains;  // != 0: a chain under every tree node; chain row i (1-based) of node v is row T + (i-1) T + v
   int kc;      // prediction steps per chain (k = kc with one chain, k = T * kc with a chain per node)
+  int masked;  // != 0: a pseudo row sees no other pseudo row (the "Masked" ablation of Section 4.3)
 };
 
 constexpr int kGemmMaxCtas = 192;         // scratch slots are provided for this many CTAs

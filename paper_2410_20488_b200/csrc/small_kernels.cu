@@ -34,8 +34,10 @@ __global__ void tree_prep_kernel(Rows rw, const int32_t *parents, const int32_t 
     int dep = -1;
     int u = v;
     for (int it = 0; it < rw.Ms && u >= 0; ++it) {   // parents[u] < u, so at most Ms hops
+      if (!(rw.masked && u >= rw.T && u != v)) {     // "Masked": other pseudo rows stay invisible, depth still counts them
 #pragma unroll
-      for (int w = 0; w < kMaskWords; ++w) if ((u >> 5) == w) bits[w] |= 1u << (u & 31);
+        for (int w = 0; w < kMaskWords; ++w) if ((u >> 5) == w) bits[w] |= 1u << (u & 31);
+      }
       ++dep;
       u = ext[u];
     }

@@ -18,10 +18,12 @@ def torch_cuda():
     return torch
 
 
-def make_pair(shape, weights, max_ctx, **kw):
+def make_pair(shape, weights, max_ctx, masked=False, **kw):
     from paper_2410_20488_b200 import FirpEngine
     eng = FirpEngine(shape, weights, max_ctx=max_ctx, **kw)
-    orc = oracle.Oracle(shape, weights, max_ctx=max_ctx, n_seq=kw.get("max_batch", 1))
+    orc = oracle.Oracle(shape, weights, max_ctx=max_ctx, n_seq=kw.get("max_batch", 1), masked=masked)
+    if masked:
+        eng.set_pseudo_masked(True)
     return eng, orc
 
 
@@ -124,6 +126,16 @@ def test_c1_a_chain_under_every_node(torch_cuda, c1, case):
                           k=k, l=layers, chains=True)
         assert st.steps == 4
         eng.close()
+
+
+@pytest.mark.parametrize("chains", [False, True])
+def test_c1_masked_pseudo_rows(torch_cuda, c1, c1_weights, chains):
+    """The "Masked" ablation of Section 4.3 (firp_set_pseudo_masked): pseudo rows do not see one another."""
+    parents = si.random_tree(3, 13, 3, 2)
+    eng, orc = make_pair(c1, c1_weights, 256, masked=True, max_tree=16, max_k=3, max_depth=3, max_rows=13 * 4)
+    st = lockstep_run(eng, orc, c1, parents, si.prompt(c1, length=40), 4, k=3, l=1 if chains else [0, 1, 1], chains=chains)
+    assert st.steps == 4
+    eng.close()
 
 
 def test_chains_need_the_row_capacity(torch_cuda, c1, c1_weights):
