@@ -580,13 +580,14 @@ int firp_prefill_layers(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int
   if ((rc = upload_i32(ctx, ctx->seq_ids, ids.data(), 1, ctx->last_seq_ids, st))) return rc;
   if ((rc = upload_i32(ctx, ctx->next_parents, next_parents, T_next, ctx->last_next_parents, st))) return rc;
   // chain template for the prompt rows
-  std::vector<int32_t> chain(cfg.max_tree);
-  for (int i = 0; i < cfg.max_tree; ++i) chain[i] = i - 1;
-  if ((rc = upload_i32(ctx, ctx->parents, chain.data(), cfg.max_tree, ctx->last_parents, st))) return rc;
+  // the prompt runs in chunks of as many rows as one step may carry (fewer passes over the weights)
+  const int chunk = std::min(ctx->Rmax, kMaxTreeRows) - k;
+  std::vector<int32_t> chain(chunk);
+  for (int i = 0; i < chunk; ++i) chain[i] = i - 1;
+  if ((rc = upload_i32(ctx, ctx->parents, chain.data(), chunk, ctx->last_parents, st))) return rc;
   FIRP_CUDA(ctx, cudaMemsetAsync(ctx->ctx_len + seq, 0, sizeof(int32_t), st));
   ctx->n_hi[seq] = 0;
 
-  const int chunk = cfg.max_tree;
   for (int p0 = 0; p0 < P; p0 += chunk) {
     const int Tc = (P - p0 < chunk) ? P - p0 : chunk;
     const bool last = (p0 + Tc == P);
