@@ -535,8 +535,7 @@ Sched make_sched(GemmEpilogue epi, const GemmArgs &a, bool pdl) {
   // With more than 80 rows the MMAs fall behind the weight stream, and a lookahead beyond the ring only fills L2
   // with tiles that are evicted before they are read and then fetched twice (measured at 140 rows: 1.8x the weight
   // bytes from DRAM, step 10 % slower).  With few rows the stream is the bound and the deep lookahead pays.
-  static const int big_ahead = [] { const char *e = getenv("FIRP_BIG_AHEAD"); return e ? atoi(e) : 0; }();   // tuning aid
-  if (a.R > 80) sc.l2_ahead = std::min(sc.l2_ahead, big_ahead);
+  if (a.R > 80) sc.l2_ahead = 0;
   return sc;
 }
 
