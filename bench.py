@@ -104,8 +104,8 @@ def class_bytes(shape, n_ctx: float) -> dict:
 # c2 shape, from the ncu capture summarised under profiles/; valid only for the kernel sources whose
 # digest is recorded with it (a changed kernel reports traffic = null until it is captured again).
 NCU_TRAFFIC = {  # dram read+write per launch; includes the ~24 MB successor head each GEMM prefetches
-    "c2-llama2-7b": dict(digest="d7d94813c05b5992", per_launch={"gemm_gate_up": 222732800, "gemm_qkv": 129425920,
-                                                             "gemm_o": 50531584, "gemm_down": 117035776}),
+    "c2-llama2-7b": dict(digest="a2bb6d50dd07d0bc", per_launch={"gemm_gate_up": 221511168, "gemm_qkv": 129046016,
+                                                             "gemm_o": 52361472, "gemm_down": 119311872}),
 }
 
 
