@@ -54,3 +54,32 @@ def test_reference_arm_other_ranks_do_no_work():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
                        env=env, capture_output=True, text=True, timeout=120)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_byte_model_counts_the_rows_of_every_variant():
+    """Algorithmic KV bytes follow the rows alive per layer: one chain at one layer, one layer per
+    prediction step, a chain under every node."""
+    sys.path.insert(0, ROOT)
+    import bench
+    import synth_inputs as si
+    s = si.CONFIGS["c2"]
+    kv_row = 2 * 2 * s.n_kv
+    try:
+        bench.INSERT_LAYERS, bench.CHAINS = None, False
+        base = bench.algorithmic_bytes(s, 512)
+        assert base["kv_write"] == kv_row * (s.l * s.T + (s.L - s.l) * (s.T + s.k))
+        bench.INSERT_LAYERS = [15, 20, 25]
+        per_step = bench.algorithmic_bytes(s, 512)
+        rows = sum(s.T + sum(1 for t in (15, 20, 25) if t <= j) for j in range(s.L))
+        assert per_step["kv_write"] == kv_row * rows and per_step["weights"] == base["weights"]
+        bench.INSERT_LAYERS, bench.CHAINS = None, True
+        chains = bench.algorithmic_bytes(s, 512)
+        assert chains["kv_write"] == kv_row * (s.l * s.T + (s.L - s.l) * s.T * (1 + s.k))
+    finally:
+        bench.INSERT_LAYERS, bench.CHAINS = None, False
+
+
+def test_reference_arm_rejects_bad_insert_layers():
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "c1",
+                        "--insert-layers", "1,0,1"], capture_output=True, text=True, timeout=120)
+    assert r.returncode != 0 and "non-decreasing" in (r.stderr + r.stdout)
