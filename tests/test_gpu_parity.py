@@ -280,6 +280,21 @@ def c2_width_2_layers():
     return shape, si.all_weights(shape)
 
 
+def test_c2_width_chains_with_one_layer_per_step(torch_cuda):
+    """A chain under every node with the prediction steps at layers 1, 2, 3 of a 4-layer decoder of the 7B width:
+    32, 64, 96 and 128 rows in successive layers, so one step runs the 40-, 80- and 144-row GEMM variants and
+    the Eq. 3 GEMM on all 32 tree rows."""
+    shape = si.scaled(si.CONFIGS["c2"], L=4, l=1, name="c2-width-4-layers")
+    weights = si.all_weights(shape)
+    parents = si.tree_template(shape.T)
+    eng, orc = make_pair(shape, weights, 256 + 160, max_rows=shape.T * (1 + shape.k))
+    st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=200), 3, k=3, l=[1, 2, 3], chains=True,
+                      check_cache_rows=True)
+    print("c2 width, chains, layers 1/2/3", st.as_dict())
+    assert st.steps == 3
+    eng.close()
+
+
 def test_c4_long_context_2048(torch_cuda, c2_width_2_layers):
     """Sweep point with a 2048-token committed context (prefilled through the chunked step path on both sides)
     at the full Llama-2-7B width, with the depth cut to 2 layers so that the oracle's prefill stays affordable:
