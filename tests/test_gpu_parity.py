@@ -232,8 +232,8 @@ def test_c2_layers_15_20_25_full_size(torch_cuda, c2_weights):
     7B-shaped workload: prefill and two lock-step steps against the oracle."""
     c2 = si.CONFIGS["c2"]
     parents = si.tree_template(c2.T)
-    eng, orc = make_pair(c2, c2_weights, 512 + 64)
-    st = lockstep_run(eng, orc, c2, parents, si.prompt(c2), 2, forced=False, check_cache_rows=False, l=[15, 20, 25])
+    eng, orc = make_pair(c2, c2_weights, 128 + 64)          # a 128-token context keeps the oracle's prefill short
+    st = lockstep_run(eng, orc, c2, parents, si.prompt(c2, length=128), 2, forced=False, check_cache_rows=False, l=[15, 20, 25])
     print("c2 layers 15/20/25", st.as_dict())
     assert st.steps == 2
     eng.close()
@@ -244,8 +244,8 @@ def test_c2_chain_under_every_node_full_size(torch_cuda, c2_weights):
     prefill and one lock-step step against the oracle."""
     c2 = si.CONFIGS["c2"]
     parents = si.tree_template(c2.T)
-    eng, orc = make_pair(c2, c2_weights, 512 + 160, max_rows=c2.T * (1 + c2.k))
-    st = lockstep_run(eng, orc, c2, parents, si.prompt(c2), 1, forced=False, check_cache_rows=False, chains=True)
+    eng, orc = make_pair(c2, c2_weights, 128 + 160, max_rows=c2.T * (1 + c2.k))
+    st = lockstep_run(eng, orc, c2, parents, si.prompt(c2, length=128), 1, forced=False, check_cache_rows=False, chains=True)
     print("c2 chains", st.as_dict())
     assert st.steps == 1
     eng.close()
