@@ -18,13 +18,18 @@ _LIB = os.path.join(_HERE, "_firp_oracle.so")
 _lib = None
 
 
+def compile_source(src: str, out: str) -> str:
+    """gcc (OpenMP) a copy of the oracle's C source into the shared object `out`."""
+    tmp = out + ".%d.tmp" % os.getpid()
+    subprocess.check_call(["gcc", "-O3", "-march=x86-64-v3", "-fopenmp", "-shared", "-fPIC", "-o", tmp, src, "-lm"])
+    os.replace(tmp, out)
+    return out
+
+
 def build(force: bool = False) -> str:
-    """Compile firp_oracle.c (gcc, OpenMP) into a shared object next to it."""
+    """Compile firp_oracle.c into a shared object next to it."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        tmp = _LIB + ".%d.tmp" % os.getpid()
-        subprocess.check_call(["gcc", "-O3", "-march=x86-64-v3", "-fopenmp", "-shared", "-fPIC",
-                               "-o", tmp, _SRC, "-lm"])
-        os.replace(tmp, _LIB)
+        compile_source(_SRC, _LIB)
     return _LIB
 
 
@@ -41,38 +46,43 @@ class _Weights(ctypes.Structure):
                [(n, _PP) for n in ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown", "g_attn", "g_mlp")]
 
 
+def bind(lib):
+    """Declare the C signatures on a loaded oracle library (the built one, or a test's altered copy)."""
+    i32, vp = ctypes.c_int32, ctypes.c_void_p
+    lib.oracle_create.argtypes = [ctypes.POINTER(_Cfg)]
+    lib.oracle_create.restype = vp
+    lib.oracle_destroy.argtypes = [vp]
+    lib.oracle_set_weights.argtypes = [vp, ctypes.POINTER(_Weights)]
+    lib.oracle_context_len.argtypes = [vp, i32]
+    lib.oracle_context_len.restype = i32
+    lib.oracle_set_context_len.argtypes = [vp, i32, i32]
+    lib.oracle_tree_prep.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
+    lib.oracle_tree_prep.restype = i32
+    lib.oracle_forward.argtypes = [vp, i32, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+    lib.oracle_forward.restype = i32
+    lib.oracle_forward_layers.argtypes = [vp, i32, vp, vp, i32, i32, vp, i32, i32, vp, vp, vp, i32, vp, vp]
+    lib.oracle_forward_layers.restype = i32
+    lib.oracle_forward_chains.argtypes = [vp, i32, vp, vp, i32, i32, vp, i32, vp, vp, vp, vp]
+    lib.oracle_forward_chains.restype = i32
+    lib.oracle_tree_prep_chains.argtypes = [vp, i32, i32, vp, vp, vp, vp]
+    lib.oracle_tree_prep_chains.restype = i32
+    lib.oracle_set_masked.argtypes = [vp, i32]
+    lib.oracle_mask_pseudo.argtypes = [vp, i32, i32]
+    lib.oracle_verify.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
+    lib.oracle_verify.restype = i32
+    lib.oracle_next_tree.argtypes = [vp, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp]
+    lib.oracle_next_tree.restype = i32
+    lib.oracle_commit.argtypes = [vp, i32, vp, i32]
+    lib.oracle_commit.restype = i32
+    lib.oracle_read_cache.argtypes = [vp, i32, i32, i32, i32, vp]
+    lib.oracle_write_cache.argtypes = [vp, i32, i32, i32, i32, i32, vp]
+    return lib
+
+
 def _get_lib():
     global _lib
     if _lib is None:
-        lib = ctypes.CDLL(build())
-        i32, vp = ctypes.c_int32, ctypes.c_void_p
-        lib.oracle_create.argtypes = [ctypes.POINTER(_Cfg)]
-        lib.oracle_create.restype = vp
-        lib.oracle_destroy.argtypes = [vp]
-        lib.oracle_set_weights.argtypes = [vp, ctypes.POINTER(_Weights)]
-        lib.oracle_context_len.argtypes = [vp, i32]
-        lib.oracle_context_len.restype = i32
-        lib.oracle_set_context_len.argtypes = [vp, i32, i32]
-        lib.oracle_tree_prep.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
-        lib.oracle_tree_prep.restype = i32
-        lib.oracle_forward.argtypes = [vp, i32, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
-        lib.oracle_forward.restype = i32
-        lib.oracle_forward_layers.argtypes = [vp, i32, vp, vp, i32, i32, vp, i32, i32, vp, vp, vp, i32, vp, vp]
-        lib.oracle_forward_layers.restype = i32
-        lib.oracle_forward_chains.argtypes = [vp, i32, vp, vp, i32, i32, vp, i32, vp, vp, vp, vp]
-        lib.oracle_forward_chains.restype = i32
-        lib.oracle_tree_prep_chains.argtypes = [vp, i32, i32, vp, vp, vp, vp]
-        lib.oracle_tree_prep_chains.restype = i32
-        lib.oracle_set_masked.argtypes = [vp, i32]
-        lib.oracle_mask_pseudo.argtypes = [vp, i32, i32]
-        lib.oracle_verify.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
-        lib.oracle_verify.restype = i32
-        lib.oracle_next_tree.argtypes = [vp, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp]
-        lib.oracle_next_tree.restype = i32
-        lib.oracle_commit.argtypes = [vp, i32, vp, i32]
-        lib.oracle_commit.restype = i32
-        lib.oracle_read_cache.argtypes = [vp, i32, i32, i32, i32, vp]
-        _lib = lib
+        _lib = bind(ctypes.CDLL(build()))
     return _lib
 
 
@@ -209,6 +219,13 @@ class Oracle:
         out = np.zeros(self.shape.n_kv, np.float32)
         self.lib.oracle_read_cache(self.h, seq, layer, which, slot, _ptr(out))
         return out
+
+    def write_cache(self, seq: int, layer: int, which: int, slot0: int, rows_bf16: np.ndarray) -> None:
+        """Overwrite cache rows slot0.. of one layer (which: 0 keys, 1 values) with bf16 bit patterns
+        [count, Hkv*dh]: a seeded stand-in for a committed prefix, written into both implementations."""
+        rows = np.ascontiguousarray(rows_bf16, dtype=np.uint16)
+        assert rows.ndim == 2 and rows.shape[1] == self.shape.n_kv and slot0 + rows.shape[0] <= self.max_ctx
+        self.lib.oracle_write_cache(self.h, seq, layer, which, slot0, rows.shape[0], _ptr(rows))
 
     # -- the step ------------------------------------------------------------
     def forward(self, tokens, parents, k: int, l, anchor: int = 0, seq: int = 0,

@@ -541,3 +541,15 @@ void oracle_read_cache(void *hnd, int32_t seq, int32_t layer, int32_t which, int
   const float *base = (which ? o->vc[seq] : o->kc[seq]) + ((size_t)layer * c->max_ctx + slot) * nkv;
   memcpy(out, base, sizeof(float) * nkv);
 }
+
+/* Test aid: overwrite cache rows slot0 .. slot0+count-1 of one layer with given bf16 rows (widened exactly).
+ * Lets a harness start both implementations from the same seeded prefix without running a prefill;
+ * no arithmetic of the method is involved.  which: 0 keys, 1 values. */
+void oracle_write_cache(void *hnd, int32_t seq, int32_t layer, int32_t which, int32_t slot0, int32_t count,
+                        const uint16_t *rows) {
+  oracle_t *o = (oracle_t *)hnd;
+  const oracle_cfg *c = &o->cfg;
+  const int nkv = c->Hkv * c->dh;
+  float *base = (which ? o->vc[seq] : o->kc[seq]) + ((size_t)layer * c->max_ctx + slot0) * nkv;
+  for (size_t i = 0; i < (size_t)count * nkv; ++i) base[i] = bf16f(rows[i]);
+}

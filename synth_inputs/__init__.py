@@ -8,7 +8,8 @@ sharing any computation.
 Recipe (all counter-based, see gen.c for the bit-level definition):
   * weight matrices  ~ N(0, std=0.02), rounded once to bf16 (RNE)
   * predictor maps   ~ N(0, variance=1/d)  (std d^-1/2), bias = 0
-  * RMSNorm gains    = 1.0
+  * RMSNorm gains    = 1.0 (the workload configurations); `gains=True` draws three kinds of
+                       non-unit gains, 1 + 0.25 N(0,1), each from a stream of its own
   * prompts          = uniform token ids in [0, V)
   * tree templates   = the first T nodes of a per-depth-width product tree,
                        ordered by (sum of sibling ranks, depth, rank tuple)
@@ -78,9 +79,21 @@ def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
 
 BF16_ONE = np.uint16(0x3F80)
 
+
+def f32_to_bf16_bits(a: np.ndarray) -> np.ndarray:
+    """Round float32 values to bf16 bit patterns (round to nearest even; finite inputs)."""
+    u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+    return ((u + np.uint32(0x7FFF) + ((u >> 16) & np.uint32(1))) >> 16).astype(np.uint16)
+
+
+def gain_vector(shape: "Shape", kind: str, index: int = 0) -> np.ndarray:
+    """A non-unit RMSNorm gain, 1 + 0.25 N(0,1), as bf16 bits; kind = g_attn | g_mlp | g_final."""
+    noise = bf16_bits_to_f32(normal_bf16(shape.seed, stream_id(kind, index), shape.d, 0.25))
+    return f32_to_bf16_bits(np.float32(1.0) + noise)
+
 # stream ids: kind + 32 * (index + 1); index = layer or map number (0 for globals)
 _KIND = dict(embed=1, lm_head=2, pred_w=3, wq=4, wk=5, wv=6, wo=7, wgate=8, wup=9, wdown=10,
-             prompt=20, ctxlen=21, tokens=22)
+             g_attn=11, g_mlp=12, g_final=13, prompt=20, ctxlen=21, tokens=22, cache_k=23, cache_v=24)
 
 
 def stream_id(kind: str, index: int = 0) -> int:
@@ -152,12 +165,12 @@ def scaled(shape: Shape, **kw) -> Shape:
 # ----------------------------------------------------------------------------
 # weights
 # ----------------------------------------------------------------------------
-def layer_weights(shape: Shape, layer: int) -> dict:
+def layer_weights(shape: Shape, layer: int, gains: bool = False) -> dict:
     """bf16 bits of one decoder layer.
 
     wqkv [(H+2Hkv)*dh, d]: q rows, then k rows, then v rows (each its own stream);
-    wo [d, H*dh]; wgu [2F, d]: gate rows then up rows; wd [d, F]; gains = 1.
-    All matrices are [out, in] row-major.
+    wo [d, H*dh]; wgu [2F, d]: gate rows then up rows; wd [d, F]; gains = 1
+    unless `gains` asks for the seeded non-unit ones.  All matrices are [out, in] row-major.
     """
     s = shape
     wqkv = np.empty((s.n_qkv, s.d), dtype=np.uint16)
@@ -170,10 +183,12 @@ def layer_weights(shape: Shape, layer: int) -> dict:
     normal_bf16(s.seed, stream_id("wup", layer), s.F * s.d, 0.02, out=wgu[s.F:].reshape(-1))
     wd = normal_bf16(s.seed, stream_id("wdown", layer), s.d * s.F, 0.02).reshape(s.d, s.F)
     ones = np.full(s.d, BF16_ONE, dtype=np.uint16)
-    return dict(wqkv=wqkv, wo=wo, wgu=wgu, wd=wd, g_attn=ones.copy(), g_mlp=ones.copy())
+    g_attn = gain_vector(s, "g_attn", layer) if gains else ones.copy()
+    g_mlp = gain_vector(s, "g_mlp", layer) if gains else ones.copy()
+    return dict(wqkv=wqkv, wo=wo, wgu=wgu, wd=wd, g_attn=g_attn, g_mlp=g_mlp)
 
 
-def global_weights(shape: Shape, n_maps: int | None = None) -> dict:
+def global_weights(shape: Shape, n_maps: int | None = None, gains: bool = False) -> dict:
     """embed [V,d], lm_head [V,d] (untied), g_final [d], pred_w [k,d,d], pred_b [k,d] (zeros)."""
     s = shape
     k = s.k if n_maps is None else n_maps
@@ -184,15 +199,25 @@ def global_weights(shape: Shape, n_maps: int | None = None) -> dict:
         normal_bf16(s.seed, stream_id("pred_w", i), s.d * s.d, s.d ** -0.5, out=pred_w[i].reshape(-1))
     pred_w = pred_w[:k]
     pred_b = np.zeros((k, s.d), dtype=np.uint16)
-    return dict(embed=embed, lm_head=lm_head, g_final=np.full(s.d, BF16_ONE, dtype=np.uint16),
-                pred_w=pred_w, pred_b=pred_b)
+    g_final = gain_vector(s, "g_final") if gains else np.full(s.d, BF16_ONE, dtype=np.uint16)
+    return dict(embed=embed, lm_head=lm_head, g_final=g_final, pred_w=pred_w, pred_b=pred_b)
 
 
-def all_weights(shape: Shape) -> dict:
-    """{'layers': [layer dicts], **globals}; host memory = shape.weight_bytes()."""
-    w = global_weights(shape)
-    w["layers"] = [layer_weights(shape, i) for i in range(shape.L)]
+def all_weights(shape: Shape, gains: bool = False) -> dict:
+    """{'layers': [layer dicts], **globals}; host memory = shape.weight_bytes().
+    gains: non-unit RMSNorm gains, different for the attention, MLP and final norms."""
+    w = global_weights(shape, gains=gains)
+    w["layers"] = [layer_weights(shape, i, gains) for i in range(shape.L)]
     return w
+
+
+def cache_rows(shape: Shape, seq: int, layer: int, n: int, std_k: float = 1.0, std_v: float = 0.5) -> tuple:
+    """Seeded key and value rows for cache positions 0..n-1 of one layer, as bf16 bits [n, Hkv*dh]:
+    a stand-in for the committed prefix of a long context (data only; nobody computed them)."""
+    idx = seq * 4096 + layer
+    ks = normal_bf16(shape.seed, stream_id("cache_k", idx), n * shape.n_kv, std_k).reshape(n, shape.n_kv)
+    vs = normal_bf16(shape.seed, stream_id("cache_v", idx), n * shape.n_kv, std_v).reshape(n, shape.n_kv)
+    return ks, vs
 
 
 # ----------------------------------------------------------------------------

@@ -511,3 +511,88 @@ def test_p9_predictor_size_matches_paper_table1():
         n_params = int(k) * int(d) ** 2
         assert round(n_params / 1e9, 2) == float(billions), name
     assert 3 * si.CONFIGS["c2"].d ** 2 == 50331648 and 3 * si.CONFIGS["c3"].d ** 2 == 78643200
+
+
+# ---------------------------------------------------------------- RMSNorm gains and grouped-query attention
+# The workload configurations have unit gains and (on the tiny shape) as many key/value heads as query heads,
+# which would leave the gain factor, the routing of the three gain vectors and the query-head -> kv-head map
+# pinned by nothing.  These variants repeat P1, P2, P6 and P8 against the library decoder (the architecture of
+# Section 4 "Setup": learned gains in every RMSNorm; grouped-query attention in the larger models).
+VARIANTS = {
+    "gains": (dict(), True),              # three different seeded gain vectors per layer kind
+    "gqa2": (dict(Hkv=2), False),         # 4 query heads on 2 key/value heads
+    "gqa1": (dict(Hkv=1), True),          # multi-query, and gains on top
+}
+
+
+@pytest.fixture(scope="module", params=sorted(VARIANTS))
+def variant(request):
+    over, gains = VARIANTS[request.param]
+    shape = si.scaled(si.CONFIGS["c1"], **over)
+    weights = si.all_weights(shape, gains=gains)
+    return shape, weights, build_hf_llama(shape, weights)
+
+
+def test_variants_p1_p2_p6_against_the_library_decoder(variant):
+    shape, weights, hfv = variant
+    prompt = si.prompt(shape, length=19)
+    o = fresh(shape, weights)
+    r = o.prefill(prompt, 0, 0, None)
+    # P1: T = 1, k = 0 stepping is cache-free greedy decoding
+    want = hf_greedy(hfv, prompt, 6)
+    got, tok, ids = [r["root"]], r["root"], list(prompt)
+    one = np.array([-1], np.int32)
+    for _ in range(5):
+        out = o.step([tok], one, 0, 0)
+        ids.append(tok)
+        assert np.abs(out["logits"][0] - hf_logits(hfv, ids)[-1]).max() < 1e-5
+        o.commit([0])
+        tok = int(out["accepted"][0])
+        got.append(tok)
+    assert got == want
+    # P6: the committed cache rows are the keys/values of a from-scratch forward (pins the kv-head layout)
+    n = o.context_len()
+    ks, vs = hf_kv(hfv, ids)
+    for layer in range(shape.L):
+        for slot in (0, prompt.size, n - 1):
+            assert np.abs(o.read_cache(0, layer, 0, slot) - ks[layer][slot]).max() < 1e-5
+            assert np.abs(o.read_cache(0, layer, 1, slot) - vs[layer][slot]).max() < 1e-5
+    # P2: every row of a random tree is a causal forward over prefix + its root path
+    T = 11
+    parents = si.random_tree(5, T, 3, 2)
+    tokens = si.random_tokens(shape, T, 3)
+    out = o.forward(tokens, parents, 3, 1)
+    for v in range(T):
+        ref = hf_logits(hfv, ids + [int(tokens[u]) for u in path_to(parents, v)])[-1]
+        assert np.abs(out["logits"][v] - ref).max() < 1e-5, v
+
+
+def test_variants_p8_pseudo_chain(variant):
+    shape, weights, hfv = variant
+    k, l = 3, 1
+    prompt = si.prompt(shape, length=14)
+    Wf = si.bf16_bits_to_f32(weights["pred_w"]).astype(np.float64)
+    bf = np.zeros((k, shape.d))
+    o = fresh(shape, weights)
+    o.forward(prompt, si.chain_template(prompt.size), 0, 0)
+    o.commit(np.arange(prompt.size))
+    tokens, parents = si.random_tokens(shape, 8, 9), si.tree_template(8)
+    out = o.forward(tokens, parents, k, l, anchor=0)
+    ids = list(prompt) + [int(tokens[0])] + [0] * k
+    ref = hf_logits_with_replaced_rows(hfv, ids, l, prompt.size + 1, list(Wf), list(bf), prompt.size)
+    assert np.abs(out["logits"][8:] - ref[prompt.size + 1:]).max() < 1e-5
+
+
+def test_gain_vectors_differ_and_matter(c1):
+    """The variant really exercises the gains: the three kinds differ, and the logits move with them."""
+    w = si.all_weights(c1, gains=True)
+    g = [si.bf16_bits_to_f32(w["layers"][0]["g_attn"]), si.bf16_bits_to_f32(w["layers"][0]["g_mlp"]),
+         si.bf16_bits_to_f32(w["g_final"]), si.bf16_bits_to_f32(w["layers"][1]["g_attn"])]
+    for i in range(4):
+        assert np.abs(g[i] - 1).max() > 0.3
+        for j in range(i):
+            assert np.abs(g[i] - g[j]).max() > 0.3
+    a, b = fresh(c1, w), fresh(c1, si.all_weights(c1))
+    la = a.forward(si.prompt(c1, length=5), si.chain_template(5), 0, 0)["logits"]
+    lb = b.forward(si.prompt(c1, length=5), si.chain_template(5), 0, 0)["logits"]
+    assert np.abs(la - lb).max() > 0.05
