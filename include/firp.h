@@ -185,9 +185,43 @@ int firp_set_pseudo_masked(firp_ctx *ctx, int32_t masked);
  * (every layer, K and V) and advance n by path_len.  path (HOST [n_seq][max_depth+1]) and
  * path_len (HOST [n_seq]) give an explicit path (strictly increasing, path[0] = 0); NULL
  * for both commits the path the last firp_step found, read on the device.
+ * After a device-side commit the host does not know how many tokens were accepted: it keeps
+ * an upper bound of the committed length (+ max_depth + 1 per commit), which sizes the
+ * attention launch and feeds the capacity check.  firp_context_len brings the bound back to
+ * the exact value; a step whose bound would not fit max_ctx reads the exact length itself
+ * (one stream synchronisation) before it refuses, so the bound never causes a spurious
+ * FIRP_ERR_CAPACITY, but a loop that never calls firp_context_len pays that synchronisation
+ * on every step once the bound has drifted past max_ctx.
  */
 int firp_kv_commit(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *path,
                    const int32_t *path_len, void *stream);
+
+/*
+ * How the decoder layers of a step are launched (Section 3.4 describes one forward pass per round; the
+ * paper gives no kernel design).  on != 0 (default): a step of at most 48 rows over all its sequences
+ * runs its layers, Eq. 3 and the lm-head as ONE persistent kernel whose weight stream never stops between
+ * operations; larger steps, and every step when on == 0, use one kernel per operation.  Both run the same
+ * arithmetic; they may cut the cached positions into a different number of attention splits, so their
+ * results agree to fp32 rounding, and each is identical from run to run.
+ */
+int firp_set_fused(firp_ctx *ctx, int32_t on);
+
+/*
+ * Bound of every wait inside the kernels (for a tile, for the other CTAs of the persistent kernel), in
+ * microseconds; 0 restores the default of 2 s.  A wait that runs out sets a device status word and the
+ * kernel runs to its end without waiting again; the next firp_context_len returns
+ * FIRP_ERR_DEVICE_TIMEOUT (results since the last check are invalid) and clears the word.
+ */
+int firp_set_wait_limit_us(firp_ctx *ctx, int64_t usec);
+
+/*
+ * Exercise the time-out path without disturbing any computation (the paper has no counterpart): enqueues a
+ * one-CTA kernel that waits, with the routine and the limit the product kernels use, on a barrier nobody
+ * arrives on.  The wait runs out, the kernel sets the device status word and returns normally; the next
+ * firp_context_len therefore returns FIRP_ERR_DEVICE_TIMEOUT once, after which the context works as before.
+ * Set a short limit first (firp_set_wait_limit_us): with the default the kernel runs for 2 s.
+ */
+int firp_selftest_wait(firp_ctx *ctx, void *stream);
 
 /* Committed context length of a slot.  Synchronises `stream` (it reads the device counter) and
  * also reads the device status word: FIRP_ERR_DEVICE_TIMEOUT if any kernel gave up a wait. */

@@ -45,7 +45,8 @@ class StepOutC(ctypes.Structure):
 EXPORTS = ("firp_create", "firp_destroy", "firp_last_error", "firp_workspace_bytes", "firp_kv_bytes",
            "firp_bind_buffers", "firp_init_weights", "firp_prefill", "firp_step", "firp_kv_commit",
            "firp_context_len", "firp_set_context_len", "firp_last_launch_count", "firp_profile_enable",
-           "firp_profile_read", "firp_kernel_class_name", "firp_topb_static", "firp_prefill_layers", "firp_step_layers", "firp_step_chains", "firp_set_pseudo_masked")
+           "firp_profile_read", "firp_kernel_class_name", "firp_topb_static", "firp_prefill_layers", "firp_step_layers", "firp_step_chains", "firp_set_pseudo_masked",
+           "firp_set_fused", "firp_set_wait_limit_us", "firp_selftest_wait")
 
 
 def lib_path() -> str:
@@ -78,6 +79,9 @@ def load_library():
     lib.firp_step_layers.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp, ctypes.POINTER(StepOutC), vp]
     lib.firp_step_chains.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp, ctypes.POINTER(StepOutC), vp]
     lib.firp_set_pseudo_masked.argtypes = [vp, i32]
+    lib.firp_set_fused.argtypes = [vp, i32]
+    lib.firp_set_wait_limit_us.argtypes = [vp, ctypes.c_int64]
+    lib.firp_selftest_wait.argtypes = [vp, vp]
     lib.firp_kv_commit.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.firp_context_len.argtypes = [vp, i32, ctypes.POINTER(i32), vp]
     lib.firp_set_context_len.argtypes = [vp, i32, i32, vp]
@@ -191,6 +195,21 @@ def firp_step_chains(ctx, n_seq: int, seq_ids, d_tokens_ptr: int, tree_parents, 
 def firp_set_pseudo_masked(ctx, masked: bool):
     """Section 4.3 "Masked" ablation: pseudo rows do not see one another."""
     _check(ctx, load_library().firp_set_pseudo_masked(ctx, int(bool(masked))))
+
+
+def firp_set_fused(ctx, on: bool):
+    """Run the layers of small steps as one persistent kernel (default) or one kernel per operation."""
+    _check(ctx, load_library().firp_set_fused(ctx, int(bool(on))))
+
+
+def firp_set_wait_limit_us(ctx, usec: int):
+    """Bound of every device-side wait in microseconds (0: the default of 2 s)."""
+    _check(ctx, load_library().firp_set_wait_limit_us(ctx, int(usec)))
+
+
+def firp_selftest_wait(ctx, stream: int = 0):
+    """Enqueue the bounded wait that nothing satisfies (see firp.h); the next firp_context_len reports it."""
+    _check(ctx, load_library().firp_selftest_wait(ctx, stream))
 
 
 def firp_kv_commit(ctx, n_seq: int, seq_ids=None, path=None, path_len=None, stream: int = 0):
@@ -336,6 +355,15 @@ class FirpEngine:
 
     def set_pseudo_masked(self, masked: bool):
         firp_set_pseudo_masked(self.ctx, masked)
+
+    def set_fused(self, on: bool):
+        firp_set_fused(self.ctx, on)
+
+    def set_wait_limit_us(self, usec: int):
+        firp_set_wait_limit_us(self.ctx, usec)
+
+    def selftest_wait(self):
+        firp_selftest_wait(self.ctx, self.stream)
 
     def commit(self, n_seq=1, seq_ids=None, path=None, path_len=None):
         if path is not None:

@@ -8,8 +8,10 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfirp_b200.so")
-SOURCES = ["firp_api.cu", "small_kernels.cu", "gemm_tcgen05.cu", "finish_kernels.cu", "attn_tree.cu", "topb_static.cu"]
-HEADERS = ["firp_kernels.cuh", "launch_util.cuh", os.path.join("..", "..", "include", "firp.h")]
+SOURCES = ["firp_api.cu", "small_kernels.cu", "gemm_tcgen05.cu", "finish_kernels.cu", "attn_tree.cu", "fused_step.cu",
+           "topb_static.cu"]
+HEADERS = ["firp_kernels.cuh", "launch_util.cuh", "tc_device.cuh", "finish_device.cuh", "norm_device.cuh", "attn_device.cuh",
+           os.path.join("..", "..", "include", "firp.h")]
 # -dlcm=cg: plain global loads are cached in L2 only.  Under programmatic dependent launch kernels of
 # consecutive steps share an SM; buffers that are rewritten every step (context lengths, tree metadata,
 # activations) must never be served from an L1 line another kernel left behind.

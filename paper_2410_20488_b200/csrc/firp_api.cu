@@ -32,11 +32,12 @@ struct Carver {
 // Kernel classes of the per-kernel timing aid (firp_profile_*).
 enum KernelClass {
   KC_TREE_PREP = 0, KC_EMBED, KC_RMSNORM, KC_PSEUDO_PROJ, KC_GEMM_QKV, KC_QKV_FINISH, KC_ATTENTION, KC_GEMM_O,
-  KC_GEMM_GATE_UP, KC_SWIGLU_FINISH, KC_GEMM_DOWN, KC_GEMM_LM_HEAD, KC_LOGITS_FINISH, KC_TOPB, KC_ACCEPT, KC_COMMIT, KC_COUNT
+  KC_GEMM_GATE_UP, KC_SWIGLU_FINISH, KC_GEMM_DOWN, KC_GEMM_LM_HEAD, KC_LOGITS_FINISH, KC_TOPB, KC_ACCEPT, KC_COMMIT, KC_FUSED_LAYERS, KC_COUNT
 };
 static const char *const kClassNames[KC_COUNT] = {
     "tree_prep", "embed", "residual_rmsnorm", "pseudo_proj", "gemm_qkv", "qkv_rope_finish", "tree_attention", "gemm_o",
-    "gemm_gate_up", "swiglu_finish", "gemm_down", "gemm_lm_head", "logits_finish", "topb", "accept_next_tree", "kv_commit"};
+    "gemm_gate_up", "swiglu_finish", "gemm_down", "gemm_lm_head", "logits_finish", "topb", "accept_next_tree", "kv_commit",
+    "fused_decoder_layers"};
 
 struct firp_ctx {
   firp_model_cfg cfg{};
@@ -50,7 +51,14 @@ struct firp_ctx {
   bool bound = false, have_weights = false, stepped = false;
   int Rmax = 0, S = 0;
   bool use_pdl = true;                  // programmatic dependent launch
+  bool use_fused = true;                // steps of at most 48 rows run their layers as one persistent kernel
+  unsigned long long wait_ns = 0;       // bound of device-side waits (0: the kernels' default)
+  uint64_t weights_gen = 0;             // bumped by firp_init_weights
+  FusedPlan *plan_step = nullptr, *plan_prefill = nullptr;
   int *dev_status = nullptr;            // device status word (bounded waits report here)
+  unsigned *grid_bar = nullptr;         // arrival counter of the fused kernel's grid barrier
+  float *attn_ws = nullptr;             // partial results of its attention splits
+  uint8_t *d_maps = nullptr;            // its tensor maps
   // weights
   firp_weights w{};
   std::vector<const void *> wqkv, wo, wgu, wd, g_attn, g_mlp;
@@ -107,6 +115,9 @@ struct firp_ctx {
     exp_path = c.take<int32_t>((size_t)kMaxSeq * S);
     exp_len = c.take<int32_t>(kMaxSeq);
     dev_status = c.take<int>(1);
+    grid_bar = c.take<unsigned>(1);
+    attn_ws = c.take<float>(fused_attn_ws_floats(cfg.max_batch, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim));
+    d_maps = c.take<uint8_t>(fused_map_bytes(cfg.n_layers));
     return align_up(c.off, 256);
   }
 };
@@ -216,13 +227,33 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   const int mw_out = (rw.Ms + 31) / 32;
   { FIRP_TIMED(KC_TREE_PREP);
     launch_tree_prep(rw, c->parents, c->seq_ids, c->ctx_len, dh, cfg.rope_theta, c->meta, out ? out->depth : nullptr,
-                     out ? out->mask : nullptr, mw_out, pdl, st); ++nl; }
+                     out ? out->mask : nullptr, mw_out, c->grid_bar, pdl, st); ++nl; }
   { FIRP_TIMED(KC_EMBED);
     launch_embed(rw, ra.d_tokens, (const bf16 *)c->w.embed, d, cfg.vocab, c->h, pdl, st); ++nl; }
 
+  const FusedShape fshape{cfg.n_layers, d, H, Hkv, dh, F, cfg.vocab, cfg.max_ctx, cfg.rms_eps};
+  const bool fused = c->use_fused && fused_eligible(fshape, rw);
+  if (fused) {      // all decoder layers (and the lm-head) as one persistent kernel
+    FusedStep fs{};
+    fs.shape = fshape; fs.rw = rw; memcpy(fs.tl, ra.tl, sizeof(fs.tl)); fs.want_head = ra.want_head; fs.Rp = (int)Rp;
+    fs.n_hi_max = ra.n_hi_max; fs.weights_gen = c->weights_gen; fs.wait_ns = c->wait_ns;
+    fs.wqkv = c->wqkv.data(); fs.wo = c->wo.data(); fs.wgu = c->wgu.data(); fs.wd = c->wd.data();
+    fs.g_attn = c->g_attn.data(); fs.g_mlp = c->g_mlp.data();
+    fs.g_final = c->w.g_final; fs.lm_head = c->w.lm_head; fs.pred_w = c->w.pred_w; fs.pred_b = c->w.pred_b;
+    fs.h = c->h; fs.ws = c->gemm_ws; fs.ss = c->ss; fs.logits = ra.logits_dst; fs.attn_ws = c->attn_ws;
+    fs.x = c->x; fs.xp = c->xp; fs.q = c->q; fs.o = c->o; fs.y = c->y; fs.kv = c->kv;
+    fs.kv_seq = c->kv_seq(); fs.kv_layer = c->kv_layer(); fs.kv_plane = c->kv_plane();
+    fs.rope = c->meta.rope; fs.pos = c->meta.pos; fs.seq_ids = c->seq_ids; fs.ctx_len = c->ctx_len; fs.mask = c->meta.mask;
+    fs.err = c->dev_status; fs.bar = c->grid_bar; fs.d_maps = c->d_maps;
+    FusedPlan *&plan = ra.prefill_last_row >= 0 ? c->plan_prefill : c->plan_step;
+    if (!plan) plan = fused_plan_create();
+    FIRP_TIMED(KC_FUSED_LAYERS);
+    FIRP_CUDA(c, launch_fused_layers(plan, fs, pdl, st, &nl));
+  }
+
   auto gemm_base = [&](const bf16 *X, size_t lo_off, const void *W, int N, int K, int act) {
     GemmArgs g{};
-    g.X = X; g.x_lo_off = lo_off; g.plane_rows = (int)Rp; g.err = c->dev_status;
+    g.X = X; g.x_lo_off = lo_off; g.plane_rows = (int)Rp; g.err = c->dev_status; g.wait_ns = c->wait_ns;
     g.W = (const bf16 *)W; g.R = rw.R; g.N = N; g.K = K; g.rw = rw; g.rows_active = act; g.planes = 2;
     g.ws = c->gemm_ws; g.l2_ahead = 48;
     if (X == c->x) { g.ss = c->ss; g.eps = cfg.rms_eps; }   // x = h * g: the finisher divides by the row's RMS
@@ -246,7 +277,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   };
   int alive = 0;   // prediction steps appended below this layer
   const int per_step = rw.chains ? rw.T : 1;                   // pseudo rows one prediction step adds per sequence
-  for (int j = 0; j < cfg.n_layers; ++j) {
+  for (int j = 0; j < cfg.n_layers && !fused; ++j) {
     int ins = 0;     // prediction steps whose layer this is
     while (alive + ins < rw.kc && ra.tl[alive + ins] == j) ++ins;
     const bool insert = ins > 0;
@@ -261,7 +292,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
                                          // each sequence, or every tree row when each node carries a chain)
         launch_root_split(rw, c->h, d, c->xp, Rp * d, pdl, st); ++nl;
         GemmArgs g{};
-        g.X = c->xp; g.x_lo_off = Rp * d; g.plane_rows = (int)Rp; g.planes = 2; g.err = c->dev_status;
+        g.X = c->xp; g.x_lo_off = Rp * d; g.plane_rows = (int)Rp; g.planes = 2; g.err = c->dev_status; g.wait_ns = c->wait_ns;
         g.W = (const bf16 *)c->w.pred_w + (size_t)alive * d * d; g.R = rw.n_seq * per_step; g.N = ins * d; g.K = d; g.rw = rw;
         g.rows_active = act;
         g.ws = c->gemm_ws; g.l2_ahead = 48;
@@ -332,15 +363,17 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     }
   }
   if (ra.want_head) {
-    { FIRP_TIMED(KC_RMSNORM);
-      FIRP_CUDA(c, launch_rmsnorm(rw, 0, rw.Ms, c->h, pending, (const bf16 *)c->w.g_final, d, c->x, Rp * d, 2, c->ss, pdl, st)); ++nl; }
-    GemmArgs g = gemm_base(c->x, Rp * d, c->w.lm_head, cfg.vocab, d, rw.Ms);
-    g.logits = ra.logits_dst; g.l2_ahead = ahead[4];
-    { Partials p = pending;
+    if (!fused) {
+      { FIRP_TIMED(KC_RMSNORM);
+        FIRP_CUDA(c, launch_rmsnorm(rw, 0, rw.Ms, c->h, pending, (const bf16 *)c->w.g_final, d, c->x, Rp * d, 2, c->ss, pdl, st)); ++nl; }
+      GemmArgs g = gemm_base(c->x, Rp * d, c->w.lm_head, cfg.vocab, d, rw.Ms);
+      g.logits = ra.logits_dst; g.l2_ahead = ahead[4];
+      Partials p = pending;
       { FIRP_TIMED(KC_GEMM_LM_HEAD);
         FIRP_CUDA(c, launch_gemm_tc(EPI_LOGITS, g, pdl, st, &p.sk)); ++nl; }
       FIRP_TIMED(KC_LOGITS_FINISH);
-      FIRP_CUDA(c, launch_gemm_finish(EPI_LOGITS, p, g, pdl, st)); ++nl; }
+      FIRP_CUDA(c, launch_gemm_finish(EPI_LOGITS, p, g, pdl, st)); ++nl;
+    }
     { FIRP_TIMED(KC_TOPB);
       launch_topb(ra.logits_dst, rw.R, cfg.vocab, cfg.top_b, c->cand_ids, c->cand_vals, c->top_ids, c->top_vals, pdl, st);
       nl += 2; }
@@ -400,6 +433,8 @@ int firp_create(const firp_model_cfg *cfg, firp_ctx **out) {
 void firp_destroy(firp_ctx *ctx) {
   if (!ctx) return;
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
+  if (ctx->plan_step) fused_plan_destroy(ctx->plan_step);
+  if (ctx->plan_prefill) fused_plan_destroy(ctx->plan_prefill);
   delete ctx;
 }
 
@@ -428,6 +463,7 @@ int firp_bind_buffers(firp_ctx *ctx, void *workspace, void *kv_cache, void *stre
   if (!gemm_tc_available())
     return fail(ctx, FIRP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
   ctx->bound = true; ctx->stepped = false;
+  ++ctx->weights_gen;
   return FIRP_OK;
 }
 
@@ -449,6 +485,7 @@ int firp_init_weights(firp_ctx *ctx, const firp_weights *w) {
   ctx->wqkv.assign(w->wqkv, w->wqkv + L); ctx->wo.assign(w->wo, w->wo + L); ctx->wgu.assign(w->wgu, w->wgu + L);
   ctx->wd.assign(w->wd, w->wd + L); ctx->g_attn.assign(w->g_attn, w->g_attn + L); ctx->g_mlp.assign(w->g_mlp, w->g_mlp + L);
   ctx->have_weights = true;
+  ++ctx->weights_gen;
   return FIRP_OK;
 }
 
@@ -529,7 +566,14 @@ static int step_impl(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const
   if (k > 0 && max_sibling_rank(tree_parents, T) >= cfg.top_b) return fail(ctx, FIRP_ERR_BAD_TREE, "more siblings than top_b");
   int n_hi_max = 0;
   for (int s = 0; s < n_seq; ++s) {
-    if (ctx->n_hi[ids[s]] + Ms > cfg.max_ctx) return fail(ctx, FIRP_ERR_CAPACITY, "slot %d: context + rows exceeds max_ctx", ids[s]);
+    if (ctx->n_hi[ids[s]] + Ms > cfg.max_ctx) {
+      // the host only keeps an upper bound after device-side commits: before refusing, read the exact length
+      int32_t n = 0;
+      FIRP_CUDA(ctx, cudaMemcpyAsync(&n, ctx->ctx_len + ids[s], sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+      FIRP_CUDA(ctx, cudaStreamSynchronize(st));
+      ctx->n_hi[ids[s]] = n;
+      if (n + Ms > cfg.max_ctx) return fail(ctx, FIRP_ERR_CAPACITY, "slot %d: context + rows exceeds max_ctx", ids[s]);
+    }
     n_hi_max = ctx->n_hi[ids[s]] > n_hi_max ? ctx->n_hi[ids[s]] : n_hi_max;
   }
   ctx->launches = 0;
@@ -620,6 +664,25 @@ int firp_set_pseudo_masked(firp_ctx *ctx, int32_t masked) {
   return FIRP_OK;
 }
 
+int firp_set_fused(firp_ctx *ctx, int32_t on) {
+  if (!ctx) return FIRP_ERR_BAD_ARG;
+  ctx->use_fused = on != 0;
+  return FIRP_OK;
+}
+
+int firp_set_wait_limit_us(firp_ctx *ctx, int64_t usec) {
+  if (!ctx || usec < 0) return FIRP_ERR_BAD_ARG;
+  ctx->wait_ns = (unsigned long long)usec * 1000ull;
+  return FIRP_OK;
+}
+
+int firp_selftest_wait(firp_ctx *ctx, void *stream) {
+  if (!ctx) return FIRP_ERR_BAD_ARG;
+  if (!ctx->bound) return fail(ctx, FIRP_ERR_STATE, "firp_bind_buffers has not been called");
+  FIRP_CUDA(ctx, launch_wait_selftest(ctx->dev_status, ctx->wait_ns, (cudaStream_t)stream));
+  return FIRP_OK;
+}
+
 int firp_kv_commit(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *path, const int32_t *path_len,
                    void *stream) {
   int rc = check_ready(ctx);
@@ -670,7 +733,11 @@ int firp_context_len(firp_ctx *ctx, int32_t seq, int32_t *n, void *stream) {
   FIRP_CUDA(ctx, cudaMemcpyAsync(&status, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost, st));
   FIRP_CUDA(ctx, cudaStreamSynchronize(st));
   ctx->n_hi[seq] = *n;
-  if (status != 0) return fail(ctx, FIRP_ERR_DEVICE_TIMEOUT, "a kernel gave up a bounded wait (device status %d)", status);
+  if (status != 0) {   // report once and clear, so that the context can go on after the caller has dealt with it
+    FIRP_CUDA(ctx, cudaMemsetAsync(ctx->dev_status, 0, sizeof(int), st));
+    FIRP_CUDA(ctx, cudaStreamSynchronize(st));
+    return fail(ctx, FIRP_ERR_DEVICE_TIMEOUT, "a kernel gave up a bounded wait (device status %d)", status);
+  }
   return FIRP_OK;
 }
 

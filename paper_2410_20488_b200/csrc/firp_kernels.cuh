@@ -63,9 +63,10 @@ struct TreeMeta {
   uint32_t *mask;      // [R][kMaskWords] bit u: row v attends to new row u of its sequence
   float2 *rope;        // [R][dh/2] (cos, sin) of pos * theta^(-2c/dh)
 };
+// zero_word (may be NULL): a device word the kernel clears (the arrival counter of the fused decoder kernel)
 void launch_tree_prep(const Rows &rw, const int32_t *d_parents, const int32_t *d_seq_ids, const int32_t *d_ctx_len,
                       int dh, float theta, TreeMeta meta, int32_t *out_depth, uint32_t *out_mask, int out_mask_words,
-                      bool pdl, cudaStream_t st);
+                      unsigned *zero_word, bool pdl, cudaStream_t st);
 
 // h[r] = embed[token] for tree rows, 0 for pseudo rows
 void launch_embed(const Rows &rw, const int32_t *d_tokens, const bf16 *embed, int d, int vocab, float *h, bool pdl,
@@ -146,6 +147,7 @@ struct GemmArgs {
   const bf16 *W;    // [N][K] weights
   int R;            // valid rows
   int *err;         // device status word (set to a non-zero code if a bounded wait gives up)
+  unsigned long long wait_ns;   // bounded waits give up after this many nanoseconds (0: the default of 2 s)
   int N, K;
   Rows rw; int rows_active;      // rows with v < rows_active are written, the others skipped
   // stream-K scratch: partial tiles [kGemmMaxCtas][kGemmSlots][2][plane_rows][128] fp32
@@ -196,5 +198,40 @@ struct AttnArgs {
 // kv splits for `groups` = sequences x kv heads x query blocks and `kv_tiles` 64-position tiles
 int attention_splits(int groups, int kv_tiles);
 cudaError_t launch_attention(const AttnArgs &a, bool pdl, cudaStream_t st);
+
+// ---- the decoder layers of a step as one persistent kernel (fused_step.cu) ------------------------------
+struct FusedShape { int L, d, H, Hkv, dh, F, V, max_ctx; float eps; };
+struct FusedStep {
+  FusedShape shape;
+  Rows rw;
+  int tl[8];                 // insertion layer of each prediction step (non-decreasing)
+  bool want_head;            // final norm + lm-head
+  int Rp;                    // rows per activation plane
+  int n_hi_max;              // upper bound of the longest committed context among the sequences
+  uint64_t weights_gen;      // changes whenever the weight pointers change
+  unsigned long long wait_ns;   // bound of every device-side wait (0: default)
+  // weights (device pointers; the per-layer arrays are host arrays of L pointers)
+  const void *const *wqkv, *const *wo, *const *wgu, *const *wd, *const *g_attn, *const *g_mlp;
+  const void *g_final, *lm_head, *pred_w, *pred_b;
+  // workspace
+  float *h, *ws, *ss, *logits, *attn_ws;
+  bf16 *x, *xp, *q, *o, *y, *kv;
+  size_t kv_seq, kv_layer, kv_plane;
+  const float2 *rope; const int32_t *pos, *seq_ids, *ctx_len; const uint32_t *mask;
+  int *err; unsigned *bar;   // status word; arrival counter of the grid barrier (zero before the launch)
+  void *d_maps;              // device room for the tensor maps: fused_map_bytes(L) bytes, 128-byte aligned
+};
+struct FusedPlan;            // host-side cache of the phase list and the tensor maps of one step shape
+FusedPlan *fused_plan_create();
+void fused_plan_destroy(FusedPlan *p);
+size_t fused_map_bytes(int n_layers);
+size_t fused_attn_ws_floats(int max_batch, int H, int Hkv, int dh);   // scratch of the attention splits
+// whether the fused kernel can run this step (at most 48 rows; every GEMM's stream-K schedule fits its scratch)
+bool fused_eligible(const FusedShape &sh, const Rows &rw);
+// Runs everything between the embedding and the top-B: all decoder layers, Eq. 3 at its layers, and (want_head)
+// the final norm and the lm-head.  Cooperative launch, one CTA per SM.
+cudaError_t launch_fused_layers(FusedPlan *plan, const FusedStep &fs, bool pdl, cudaStream_t st, int *launches);
+// one CTA waits (bounded by wait_ns, 0 = default) on a barrier nobody arrives on, sets *err and returns
+cudaError_t launch_wait_selftest(int *err, unsigned long long wait_ns, cudaStream_t st);
 
 }  // namespace firp

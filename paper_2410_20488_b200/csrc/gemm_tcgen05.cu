@@ -41,6 +41,7 @@
 
 #include "firp_kernels.cuh"
 #include "launch_util.cuh"
+#include "tc_device.cuh"
 
 namespace firp {
 
@@ -52,93 +53,6 @@ constexpr int BK = kGemmBK;        // 64 bf16 = 128 bytes = one swizzle row
 constexpr int kThreads = 224;      // 7 warps
 constexpr int W_TILE = BM * 128;   // bytes of one 128-row weight tile of a k block
 constexpr int W_STAGE = TM * W_TILE;
-constexpr int kErrTimeout = 100;
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned long long globaltimer() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait.  `dead` is sticky per thread: after one timeout later waits return at once.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int *err, bool &dead) {
-  if (dead || mbar_try_wait(bar, parity)) return;
-  const unsigned long long t0 = globaltimer();
-  uint32_t spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 255u) == 0 && globaltimer() - t0 > 2000000000ull) {
-      dead = true;
-      atomicExch(err, kErrTimeout);
-      return;
-    }
-  }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int x, int y, uint32_t bar,
-                                            uint64_t policy) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
-      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm, int x, int y, int z, int w, uint32_t bar,
-                                            uint64_t policy) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
-      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap *tm, int x, int y, uint64_t policy) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile.L2::cache_hint [%0, {%1, %2}], %3;"
-               ::"l"(tm), "r"(x), "r"(y), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap *tm, int x, int y, int z, int w, uint64_t policy) {
-  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile.L2::cache_hint [%0, {%1, %2, %3, %4}], %5;"
-               ::"l"(tm), "r"(x), "r"(y), "r"(z), "r"(w), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, float *r) {
-  uint32_t *u = reinterpret_cast<uint32_t *>(r);
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-               : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
-                 "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15])
-               : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory operand descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups
-// 1024 bytes apart (start address >> 4 in bits 0-13, leading offset 1 in bits 16-29 (unused for
-// swizzled K-major), stride offset 1024 >> 4 in bits 32-45, version 1 in bits 46-47, layout 2 =
-// SWIZZLE_128B in bits 61-63).  Advancing K by 16 elements adds 32 bytes to the start address.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
-         ((uint64_t)2 << 61);
-}
-// Instruction descriptor, kind::f16: fp32 accumulator (bits 4-5 = 1), A and B bf16 (bits 7-9, 10-12 = 1),
-// both K-major (bits 15, 16 = 0), N >> 3 in bits 17-22, M >> 4 in bits 24-28.
-__host__ __device__ constexpr uint32_t instr_desc(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-}
 
 constexpr int pow2_cols(int c) { return c <= 32 ? 32 : c <= 64 ? 64 : c <= 128 ? 128 : c <= 256 ? 256 : 512; }
 
@@ -248,6 +162,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   }
 
   bool dead = false;
+  const unsigned long long wait_ns = a.wait_ns ? a.wait_ns : kDefaultWaitNs;
   if (warp == 0) {
     if (lane == 0) {             // ---- weight producer: does not wait for the previous kernel
       uint64_t pol;
@@ -265,7 +180,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const int u = u0 + it;
         const int st = u / KB, kb = u - st * KB;
         const int sl = it % SW;
-        mbar_wait(empty_w + 8 * sl, ((it / SW) & 1) ^ 1, a.err, dead);
+        mbar_wait(empty_w + 8 * sl, ((it / SW) & 1) ^ 1, a.err, dead, wait_ns);
         mbar_expect_tx(full_w + 8 * sl, W_STAGE);
         const uint32_t dst = w_ring + sl * W_STAGE, bar = full_w + 8 * sl;
         if (sc.mode == ROWS_ROTARY) {
@@ -295,7 +210,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       for (int it = 0; it < n_units; ++it) {
         const int kb = (int)((u0 + it) % KB);
         const int sl = it % SX;
-        mbar_wait(empty_x + 8 * sl, ((it / SX) & 1) ^ 1, a.err, dead);
+        mbar_wait(empty_x + 8 * sl, ((it / SX) & 1) ^ 1, a.err, dead, wait_ns);
         mbar_expect_tx(full_x + 8 * sl, P * xrows * 128);
         const uint32_t dst = x_ring + sl * X_STAGE;
 #pragma unroll
@@ -305,20 +220,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
   } else if (warp == 1) {
     if (lane == 0) {             // ---- MMA issuer
-      constexpr uint32_t idesc = instr_desc(MERGE ? P * NPAD : NPAD);
+      constexpr uint32_t idesc = instr_desc_m128(MERGE ? P * NPAD : NPAD);
       int it = 0, seg = 0;
       int u = u0;
       while (u < u1) {
         const int st = u / KB, kb0 = u - st * KB;
         const int kb1 = min(KB, kb0 + (u1 - u));
         const int buf = seg % NBUF;
-        mbar_wait(acc_empty + 8 * buf, ((seg / NBUF) & 1) ^ 1, a.err, dead);   // epilogue has drained this buffer
+        mbar_wait(acc_empty + 8 * buf, ((seg / NBUF) & 1) ^ 1, a.err, dead, wait_ns);   // epilogue has drained this buffer
         tc_fence_after();
         const uint32_t acc = tmem_base + (uint32_t)(buf * TM * ACC);
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int sw = it % SW, sx = it % SX;
-          mbar_wait(full_w + 8 * sw, (it / SW) & 1, a.err, dead);
-          mbar_wait(full_x + 8 * sx, (it / SX) & 1, a.err, dead);
+          mbar_wait(full_w + 8 * sw, (it / SW) & 1, a.err, dead, wait_ns);
+          mbar_wait(full_x + 8 * sx, (it / SX) & 1, a.err, dead, wait_ns);
           tc_fence_after();
           const uint32_t wst = w_ring + sw * W_STAGE, xst = x_ring + sx * X_STAGE;
           const uint64_t dx = smem_desc(xst);
@@ -353,7 +268,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const int st = u / KB, kb0 = u - st * KB;
       const int kb1 = min(KB, kb0 + (u1 - u));
       const int buf = seg % NBUF;
-      mbar_wait(acc_full + 8 * buf, (seg / NBUF) & 1, a.err, dead);
+      mbar_wait(acc_full + 8 * buf, (seg / NBUF) & 1, a.err, dead, wait_ns);
       tc_fence_after();
       const uint32_t tacc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * TM * ACC);
       float *my_ws = a.ws + (size_t)(cta * kGemmSlots + seg) * slot_elems + i;

@@ -2,6 +2,7 @@
 // the pseudo-hidden projection (Eq. 3), top-B, the acceptance walk / next tree, KV compaction.
 #include "firp_kernels.cuh"
 #include "launch_util.cuh"
+#include "norm_device.cuh"
 
 
 namespace firp {
@@ -13,11 +14,12 @@ namespace firp {
 // ---------------------------------------------------------------------------
 __global__ void tree_prep_kernel(Rows rw, const int32_t *parents, const int32_t *seq_ids,
                                  const int32_t *ctx_len, int dh, float theta, TreeMeta meta,
-                                 int32_t *out_depth, uint32_t *out_mask, int out_mask_words, int pdl) {
+                                 int32_t *out_depth, uint32_t *out_mask, int out_mask_words, unsigned *zero_word, int pdl) {
   __shared__ int32_t ext[kMaxTreeRows];
   __shared__ int32_t sdepth[kMaxTreeRows];
   if (pdl) { griddep_launch(); griddep_wait(); }
   const int s = blockIdx.x, tid = threadIdx.x;
+  if (zero_word && s == 0 && tid == 0) *zero_word = 0u;
   const int n = ctx_len[seq_ids[s]];
   for (int v = tid; v < rw.Ms; v += blockDim.x) {
     int p;
@@ -66,9 +68,9 @@ __global__ void tree_prep_kernel(Rows rw, const int32_t *parents, const int32_t 
 
 void launch_tree_prep(const Rows &rw, const int32_t *d_parents, const int32_t *d_seq_ids, const int32_t *d_ctx_len,
                       int dh, float theta, TreeMeta meta, int32_t *out_depth, uint32_t *out_mask, int out_mask_words,
-                      bool pdl, cudaStream_t st) {
+                      unsigned *zero_word, bool pdl, cudaStream_t st) {
   launch_k(tree_prep_kernel, dim3(rw.n_seq), dim3(256), 0, st, pdl, rw, d_parents, d_seq_ids, d_ctx_len, dh, theta, meta,
-           out_depth, out_mask, out_mask_words, pdl ? 1 : 0);
+           out_depth, out_mask, out_mask_words, zero_word, pdl ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------
@@ -113,59 +115,7 @@ __global__ void __launch_bounds__(kNormThreads)
 rmsnorm_kernel(Rows rw, int v0, int nv, float *h, Partials pend, const bf16 *__restrict__ g, int d, bf16 *x,
                size_t x_lo_off, int planes, float *ss, int pdl) {
   if (pdl) { griddep_launch(); griddep_wait(); }
-  const int nvec = d >> 2;                                  // float4 per row, a multiple of 32
-  const unsigned t = blockIdx.x * kNormThreads + threadIdx.x;
-  if (t >= (unsigned)(rw.n_seq * nv * nvec)) return;        // whole warps drop out together
-  const int rowi = (int)(t / (unsigned)nvec), idx = (int)(t % (unsigned)nvec);
-  const int s = rowi / nv, v = v0 + rowi % nv;
-  const int r = s * rw.Ms + v;
-  float4 *hr = reinterpret_cast<float4 *>(h + (size_t)r * d);
-  float4 a = __ldcg(hr + idx);
-  if (pend.sk.U > 0) {
-    const size_t plane_elems = (size_t)pend.ws_rows * 128;
-    const int n = idx * 4, st = n >> 8, tl = (n >> 7) & 1, i = n & 127;
-    const SkContrib k = sk_contributors(pend.sk, st);
-    const float *base = pend.ws + (size_t)tl * plane_elems + (size_t)r * 128 + i;
-    for (int c0 = k.c_first; c0 <= k.c_last; c0 += 12) {    // 12 contributors' loads in flight together
-      float4 p[12];
-#pragma unroll
-      for (int j = 0; j < 12; ++j) {      // unconditional loads (index clamped) so that they issue back to back
-        const int c = min(c0 + j, k.c_last);
-        p[j] = __ldcg(reinterpret_cast<const float4 *>(
-            base + (size_t)(c * kGemmSlots + (c == k.c_first ? k.ord_first : 0)) * 2 * plane_elems));
-      }
-#pragma unroll
-      for (int j = 0; j < 12; ++j) {
-        if (c0 + j <= k.c_last) { a.x += p[j].x; a.y += p[j].y; a.z += p[j].z; a.w += p[j].w; }
-      }
-    }
-    hr[idx] = a;
-  }
-  float sq = a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-  if ((threadIdx.x & 31) == 0) ss[(size_t)r * kNormMaxWarps + (idx >> 5)] = sq;
-  const __nv_bfloat162 g01 = reinterpret_cast<const __nv_bfloat162 *>(g)[2 * idx];
-  const __nv_bfloat162 g23 = reinterpret_cast<const __nv_bfloat162 *>(g)[2 * idx + 1];
-  const float2 ga = __bfloat1622float2(g01), gb = __bfloat1622float2(g23);
-  const float y0 = a.x * ga.x, y1 = a.y * ga.y, y2 = a.z * gb.x, y3 = a.w * gb.y;
-  const __nv_bfloat162 o01 = __floats2bfloat162_rn(y0, y1), o23 = __floats2bfloat162_rn(y2, y3);
-  const float2 f01 = __bfloat1622float2(o01), f23 = __bfloat1622float2(o23);
-  const __nv_bfloat162 l01 = __floats2bfloat162_rn(y0 - f01.x, y1 - f01.y);     // lo plane: what the hi half lost
-  const __nv_bfloat162 l23 = __floats2bfloat162_rn(y2 - f23.x, y3 - f23.y);
-  uint2 hi2, lo2;
-  hi2.x = *reinterpret_cast<const uint32_t *>(&o01); hi2.y = *reinterpret_cast<const uint32_t *>(&o23);
-  lo2.x = *reinterpret_cast<const uint32_t *>(&l01); lo2.y = *reinterpret_cast<const uint32_t *>(&l23);
-  *reinterpret_cast<uint2 *>(x + (size_t)r * d + 4 * idx) = hi2;
-  *reinterpret_cast<uint2 *>(x + x_lo_off + (size_t)r * d + 4 * idx) = lo2;
-  if (planes == 3) {   // third plane: what hi + mid still miss (the K/V projections need fp32-grade inputs)
-    const float2 m01 = __bfloat1622float2(l01), m23 = __bfloat1622float2(l23);
-    const __nv_bfloat162 t01 = __floats2bfloat162_rn(y0 - f01.x - m01.x, y1 - f01.y - m01.y);
-    const __nv_bfloat162 t23 = __floats2bfloat162_rn(y2 - f23.x - m23.x, y3 - f23.y - m23.y);
-    uint2 t2;
-    t2.x = *reinterpret_cast<const uint32_t *>(&t01); t2.y = *reinterpret_cast<const uint32_t *>(&t23);
-    *reinterpret_cast<uint2 *>(x + 2 * x_lo_off + (size_t)r * d + 4 * idx) = t2;
-  }
+  rmsnorm_item(rw, v0, nv, h, pend, g, d, x, x_lo_off, planes, ss, blockIdx.x * kNormThreads + threadIdx.x);
 }
 
 cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Partials &pending, const bf16 *g, int d,
@@ -185,22 +135,7 @@ cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Parti
 __global__ void __launch_bounds__(256)
 root_split_kernel(Rows rw, const float *h, int d, bf16 *xp, size_t xp_lo_off, int pdl) {
   if (pdl) { griddep_launch(); griddep_wait(); }
-  const int nvec = d >> 2;
-  const unsigned t = blockIdx.x * 256 + threadIdx.x;
-  const int per_seq = rw.chains ? rw.T : 1;                 // source rows per sequence
-  if (t >= (unsigned)(rw.n_seq * per_seq * nvec)) return;
-  const int m = (int)(t / (unsigned)nvec), idx = (int)(t % (unsigned)nvec);
-  const int sq = m / per_seq, v = rw.chains ? m - sq * per_seq : rw.anchor;
-  const int s = m;                                          // destination row in xp
-  const float4 a = __ldcg(reinterpret_cast<const float4 *>(h + (size_t)(sq * rw.Ms + v) * d) + idx);
-  const __nv_bfloat162 o01 = __floats2bfloat162_rn(a.x, a.y), o23 = __floats2bfloat162_rn(a.z, a.w);
-  const float2 f01 = __bfloat1622float2(o01), f23 = __bfloat1622float2(o23);
-  const __nv_bfloat162 l01 = __floats2bfloat162_rn(a.x - f01.x, a.y - f01.y), l23 = __floats2bfloat162_rn(a.z - f23.x, a.w - f23.y);
-  uint2 hi2, lo2;
-  hi2.x = *reinterpret_cast<const uint32_t *>(&o01); hi2.y = *reinterpret_cast<const uint32_t *>(&o23);
-  lo2.x = *reinterpret_cast<const uint32_t *>(&l01); lo2.y = *reinterpret_cast<const uint32_t *>(&l23);
-  *reinterpret_cast<uint2 *>(xp + (size_t)s * d + 4 * idx) = hi2;
-  *reinterpret_cast<uint2 *>(xp + xp_lo_off + (size_t)s * d + 4 * idx) = lo2;
+  root_split_item(rw, h, d, xp, xp_lo_off, blockIdx.x * 256 + threadIdx.x);
 }
 
 void launch_root_split(const Rows &rw, const float *h, int d, bf16 *xp, size_t xp_lo_off, bool pdl, cudaStream_t st) {

@@ -43,7 +43,8 @@ extern "C" int firp_topb_static(const float *d_logits, int32_t rows, int32_t voc
     fprintf(stderr, "firp_topb_static: NULL pointer, or rows / vocab / b out of range (b must be 1..%d)\n", firp::kMaxTopB);
     return FIRP_ERR_BAD_ARG;
   }
-  const long long slots = (long long)rows * firp::topb_segments(vocab);
+  // segment count in 64 bits: (vocab + 2047) would wrap for a vocab next to INT32_MAX
+  const long long slots = (long long)rows * (((long long)vocab + firp::kTopSeg - 1) / firp::kTopSeg);
   if (slots > kStaticSlots) {
     fprintf(stderr, "firp_topb_static: rows * ceil(vocab / 2048) = %lld exceeds the built-in scratch of %d slots\n", slots,
             kStaticSlots);

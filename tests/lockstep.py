@@ -54,10 +54,12 @@ class Stats:
         self.steps = self.ambiguous = self.rows = self.rows_margin = 0
         self.max_abs = self.max_rel = 0.0
         self.emitted = 0
+        self.unsynced_max_abs = None     # deviation of a step on the engine's own prefilled cache (see lockstep_run)
 
     def as_dict(self):
         return dict(steps=self.steps, ambiguous_steps=self.ambiguous, rows=self.rows, rows_with_margin=self.rows_margin,
-                    max_abs=self.max_abs, max_rel=self.max_rel, emitted=self.emitted)
+                    max_abs=self.max_abs, max_rel=self.max_rel, emitted=self.emitted,
+                    unsynced_max_abs=self.unsynced_max_abs)
 
 
 def compare_step(shape, parents, tokens, k, g, ref, stats: Stats, tp=None, abs_tol=None, chains=False):
@@ -162,21 +164,63 @@ def check_cache(engine, orc, seq, slots, layers, tol=2e-2):
                 assert np.abs(a - b).max() <= tol * scale, "cache row %d layer %d differs" % (slot, layer)
 
 
+def write_gpu_cache(engine, seq, layer, which, slot0, rows_bits):
+    """Copy bf16 bit patterns [count, Hkv*dh] into the engine's cache tensor at positions slot0.. of one
+    layer (which: 0 keys, 1 values): plain data movement through torch, no kernel of the library."""
+    import torch
+    s, cfg = engine.shape, engine.cfg
+    kvt = engine.kv.view(torch.int16)
+    plane = cfg.max_ctx * s.n_kv
+    off = ((seq * s.L + layer) * 2 + which) * plane + slot0 * s.n_kv
+    src = torch.from_numpy(np.ascontiguousarray(rows_bits, np.uint16).view(np.int16).reshape(-1))
+    kvt[off: off + src.numel()].copy_(src.to(engine.device))
+
+
+def seed_prefix(engine, orc, shape, seq, n):
+    """Give both sides the same committed prefix of n positions WITHOUT a prefill: seeded bf16 key and value rows
+    (synth_inputs.cache_rows; N(0, (0.02 sqrt(d))^2), the spread the projections of a unit-RMS row have) are written
+    bit for bit into both caches and both committed lengths are set to n.  The oracle's cost per step is then
+    linear in n, which is what makes the long contexts checkable against it."""
+    std = 0.02 * float(np.sqrt(shape.d))
+    for layer in range(shape.L):
+        ks, vs = si.cache_rows(shape, seq, layer, n, std, std)
+        for which, rows in ((0, ks), (1, vs)):
+            orc.write_cache(seq, layer, which, 0, rows)
+            write_gpu_cache(engine, seq, layer, which, 0, rows)
+    orc.set_context_len(seq, n)
+    engine.set_context_len(seq, n)
+
+
+def sync_prefix_from_oracle(engine, orc, shape, seq, n, sample=12):
+    """After both sides have prefilled the same prompt: check the engine's cache rows against the oracle's at
+    sampled positions (first and last layer), then overwrite the engine's n prefix rows with the oracle's, bit for
+    bit.  Both caches hold bf16, and a key or value whose fp32 pre-image sits next to a rounding boundary may round
+    differently on the two sides; over hundreds of rows and tens of layers those one-ulp differences add up to
+    logit noise of the size of the parity bound itself, which says nothing about either implementation.  With the
+    prefix synchronised, a step is compared on the same committed state, as the lock-step protocol asks."""
+    slots = sorted(set(np.linspace(0, n - 1, num=min(sample, n)).astype(int).tolist()))
+    check_cache(engine, orc, seq, slots, sorted({0, shape.L - 1}))
+    for layer in range(shape.L):
+        for which in (0, 1):
+            rows = np.stack([orc.read_cache(seq, layer, which, slot) for slot in range(n)])
+            bits = (rows.view(np.uint32) >> 16).astype(np.uint16)
+            assert not (rows.view(np.uint32) & 0xFFFF).any(), "the oracle's cache rows are not bf16 values"
+            write_gpu_cache(engine, seq, layer, which, 0, bits)
+
+
 def lockstep_run(engine, orc, shape, parents, prompt, steps, forced=False, k=None, l=None, check_cache_rows=True,
-                 compare_every=1, seq=0, abs_tol=None, chains=False):
+                 compare_every=1, seq=0, abs_tol=None, chains=False, forced_steps=(), sync_prefix=False):
     """Prefill both sides, then `steps` lock-step steps (chains: with a chain of k pseudo rows under
-    every tree node, firp_step_chains against oracle.step_chains).  Returns a Stats."""
+    every tree node, firp_step_chains against oracle.step_chains).  sync_prefix: after the prefill has been
+    checked (logits, sampled cache rows), one un-synchronised step is compared at twice the bound and its
+    deviation reported in Stats.unsynced_max_abs, then the engine's prefix rows are replaced by the oracle's
+    (sync_prefix_from_oracle) before the asserted steps.  Returns a Stats."""
     abs_tol = ABS_TOL if abs_tol is None else abs_tol
     import torch
     k = shape.k if k is None else k
     l = shape.l if l is None else l
     T = len(parents)
-    tp = oracle.tree_prep_chains(parents, k) if chains else oracle.tree_prep(parents, k, 0)
-    tp_tree = oracle.tree_prep(parents, 0, 0)
-    D = int(tp_tree["depth"].max())
-    chain = principal_chain(parents, tp_tree["depth"])
     dev = engine.device
-    stats = Stats()
 
     # prefill
     d_prompt = torch.from_numpy(np.ascontiguousarray(prompt, np.int32)).to(dev)
@@ -191,12 +235,48 @@ def lockstep_run(engine, orc, shape, parents, prompt, steps, forced=False, k=Non
     if part[-1] - part[-2] > MARGIN:
         assert int(pout.accepted_tokens[0, 0].item()) == ref["root"], "prefill root token differs"
     assert engine.context_len(seq) == orc.context_len(seq) == len(prompt)
-    tokens = ref["next_tokens"].copy()
-    emitted = [ref["root"]]
+    unsynced = None
+    if sync_prefix:
+        n = len(prompt)
+        probe = lockstep_steps(engine, orc, shape, parents, ref["next_tokens"].copy(), 1, k=k, l=l, check_cache_rows=False,
+                               seq=seq, abs_tol=2 * abs_tol, chains=chains)
+        unsynced = probe.max_abs
+        orc.set_context_len(seq, n)
+        engine.set_context_len(seq, n)
+        sync_prefix_from_oracle(engine, orc, shape, seq, n)
+    stats = lockstep_steps(engine, orc, shape, parents, ref["next_tokens"].copy(), steps, forced=forced, k=k, l=l,
+                           check_cache_rows=check_cache_rows, compare_every=compare_every, seq=seq, abs_tol=abs_tol,
+                           chains=chains, forced_steps=forced_steps)
+    stats.emitted += 1
+    stats.unsynced_max_abs = unsynced
+    return stats
+
+
+def lockstep_steps(engine, orc, shape, parents, tokens, steps, forced=False, k=None, l=None, check_cache_rows=True,
+                   compare_every=1, seq=0, abs_tol=None, chains=False, forced_steps=(), device_commit=False):
+    """`steps` lock-step steps from the committed state both sides are in, starting with the tree `tokens`.
+    forced / forced_steps: all steps, or the listed ones, run in forced-accept mode (the oracle's own greedy
+    continuation is planted on the principal chain, so the full depth is accepted and the commit compacts a real
+    path).  device_commit: the engine commits the path its own walk found (path = NULL) instead of being told the
+    oracle's; this requires a decisive step, and the committed cache rows are compared like any other."""
+    abs_tol = ABS_TOL if abs_tol is None else abs_tol
+    import torch
+    k = shape.k if k is None else k
+    l = shape.l if l is None else l
+    T = len(parents)
+    tp = oracle.tree_prep_chains(parents, k) if chains else oracle.tree_prep(parents, k, 0)
+    tp_tree = oracle.tree_prep(parents, 0, 0)
+    D = int(tp_tree["depth"].max())
+    chain = principal_chain(parents, tp_tree["depth"])
+    dev = engine.device
+    stats = Stats()
+    tokens = np.array(tokens, np.int32)
+    emitted = []
 
     out = engine.new_out(1, T, k, chains=chains)
     for step in range(steps):
-        if forced:
+        force_now = forced or step in forced_steps
+        if force_now:
             gcont = orc.ar_greedy(int(tokens[0]), D, seq=seq)
             for j in range(1, D + 1):
                 v = chain[j]
@@ -211,13 +291,19 @@ def lockstep_run(engine, orc, shape, parents, prompt, steps, forced=False, k=Non
         else:
             engine.step(d_tokens, parents, k, l, out, seq_ids=[seq])
             ref = orc.step(tokens, parents, k, l, seq=seq)
-        if step % compare_every == 0 or step == steps - 1:
+        g = None
+        if step % compare_every == 0 or step == steps - 1 or device_commit:
             g = gpu_outputs(out, 0, T, k)
             compare_step(shape, parents, tokens, k, g, ref, stats, tp, abs_tol, chains=chains)
-        if forced:
+        if force_now:
             assert ref["n_accepted"] == D + 1, "forced-accept step accepted %d of %d" % (ref["n_accepted"] - 1, D)
         n0 = orc.context_len(seq)
-        engine.commit(1, seq_ids=[seq], path=[ref["path"]])
+        if device_commit:
+            assert g["n_accepted"] == ref["n_accepted"] and np.array_equal(g["path"][: ref["n_accepted"]], ref["path"]), \
+                "the device-side commit needs a step on which both walks agree"
+            engine.commit(1, seq_ids=[seq])
+        else:
+            engine.commit(1, seq_ids=[seq], path=[ref["path"]])
         orc.commit(ref["path"], seq=seq)
         n1 = orc.context_len(seq)
         assert engine.context_len(seq) == n1
@@ -238,9 +324,7 @@ def lockstep_run_batch(engine, orc, shape, parents, prompts, steps, k=None, l=No
     l = shape.l if l is None else l
     abs_tol = ABS_TOL if abs_tol is None else abs_tol
     T, n_seq = len(parents), len(prompts)
-    tp = oracle.tree_prep(parents, k, 0)
     dev = engine.device
-    stats = Stats()
     tokens = np.zeros((n_seq, T), np.int32)
     for s_i, prompt in enumerate(prompts):
         pout = engine.new_out(1, 1, k, T_next=T)
@@ -251,6 +335,20 @@ def lockstep_run_batch(engine, orc, shape, parents, prompts, steps, k=None, l=No
         assert dd <= abs_tol, "prefill logits of sequence %d differ by %.4g" % (s_i, dd)
         assert engine.context_len(s_i) == orc.context_len(s_i) == len(prompt)
         tokens[s_i] = ref["next_tokens"]
+    return lockstep_steps_batch(engine, orc, shape, parents, tokens, steps, k=k, l=l, abs_tol=abs_tol)
+
+
+def lockstep_steps_batch(engine, orc, shape, parents, tokens, steps, k=None, l=None, abs_tol=None, check_cache_rows=False):
+    """`steps` lock-step steps of n_seq sequences (tokens [n_seq, T]) from the committed state both sides are in."""
+    import torch
+    k = shape.k if k is None else k
+    l = shape.l if l is None else l
+    abs_tol = ABS_TOL if abs_tol is None else abs_tol
+    tokens = np.array(tokens, np.int32)
+    n_seq, T = tokens.shape
+    tp = oracle.tree_prep(parents, k, 0)
+    dev = engine.device
+    stats = Stats()
     out = engine.new_out(n_seq, T, k)
     for step in range(steps):
         d_tokens = torch.from_numpy(np.ascontiguousarray(tokens)).to(dev)
@@ -258,10 +356,13 @@ def lockstep_run_batch(engine, orc, shape, parents, prompts, steps, k=None, l=No
         refs = [orc.step(tokens[s_i], parents, k, l, seq=s_i) for s_i in range(n_seq)]
         for s_i in range(n_seq):
             compare_step(shape, parents, tokens[s_i], k, gpu_outputs(out, s_i, T, k), refs[s_i], stats, tp, abs_tol)
+        n0 = [orc.context_len(s_i) for s_i in range(n_seq)]
         engine.commit(n_seq, seq_ids=list(range(n_seq)), path=[r["path"] for r in refs])
         for s_i in range(n_seq):
             orc.commit(refs[s_i]["path"], seq=s_i)
             assert engine.context_len(s_i) == orc.context_len(s_i)
+            if check_cache_rows:
+                check_cache(engine, orc, s_i, range(n0[s_i], orc.context_len(s_i)), sorted({0, shape.L - 1}))
             stats.emitted += len(refs[s_i]["accepted"])
             tokens[s_i] = refs[s_i]["next_tokens"]
     return stats

@@ -4,7 +4,7 @@ import pytest
 
 import oracle
 import synth_inputs as si
-from lockstep import lockstep_run, compare_step, gpu_outputs, Stats
+from lockstep import lockstep_run, lockstep_steps, seed_prefix, compare_step, gpu_outputs, Stats
 
 pytestmark = pytest.mark.gpu
 
@@ -18,19 +18,22 @@ def torch_cuda():
     return torch
 
 
-def make_pair(shape, weights, max_ctx, masked=False, **kw):
+def make_pair(shape, weights, max_ctx, masked=False, fused=True, **kw):
+    """fused=False: one kernel per operation even for small steps (the path steps of more than 48 rows take)."""
     from paper_2410_20488_b200 import FirpEngine
     eng = FirpEngine(shape, weights, max_ctx=max_ctx, **kw)
+    eng.set_fused(fused)
     orc = oracle.Oracle(shape, weights, max_ctx=max_ctx, n_seq=kw.get("max_batch", 1), masked=masked)
     if masked:
         eng.set_pseudo_masked(True)
     return eng, orc
 
 
-def test_c1_greedy_and_forced(torch_cuda, c1, c1_weights):
+@pytest.mark.parametrize("fused", [True, False])
+def test_c1_greedy_and_forced(torch_cuda, c1, c1_weights, fused):
     parents = si.tree_template(c1.T)
     for forced in (False, True):
-        eng, orc = make_pair(c1, c1_weights, 256)
+        eng, orc = make_pair(c1, c1_weights, 256, fused=fused)
         st = lockstep_run(eng, orc, c1, parents, si.prompt(c1), c1.steps, forced=forced)
         assert st.steps == c1.steps
         if forced:
@@ -46,13 +49,48 @@ def test_c1_t1_k0_autoregressive(torch_cuda, c1, c1_weights):
     eng.close()
 
 
+def test_c1_non_unit_gains(torch_cuda, c1):
+    """RMSNorm gains that differ between the attention norm, the MLP norm and the final norm of every layer
+    (the workload configurations use gains of 1, which would hide a swapped or dropped gain)."""
+    weights = si.all_weights(c1, gains=True)
+    parents = si.tree_template(c1.T)
+    for forced in (False, True):
+        eng, orc = make_pair(c1, weights, 256)
+        st = lockstep_run(eng, orc, c1, parents, si.prompt(c1, length=41), 6, forced=forced)
+        assert st.steps == 6
+        eng.close()
+    # per-step insertion layers and a chain under every node take other kernel paths for the new rows' norm
+    shape = si.scaled(c1, L=4)
+    w4 = si.all_weights(shape, gains=True)
+    eng, orc = make_pair(shape, w4, 256, max_tree=16, max_k=3, max_depth=3, max_rows=13 * 4)
+    parents = si.random_tree(3, 13, 3, 2)
+    assert lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=30), 3, k=3, l=[0, 2, 3]).steps == 3
+    assert lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=30), 3, k=3, l=[1, 2, 2], chains=True).steps == 3
+    eng.close()
+
+
+@pytest.mark.parametrize("Hkv", [2, 1])
+def test_c1_grouped_query_attention_two_query_blocks(torch_cuda, c1, Hkv):
+    """4 query heads on 2 or 1 key/value heads with enough rows that rows x heads-per-group exceeds one
+    64-row query block (19 x 2 = 38 and 19 x 4 = 76; 35 x 4 = 140 with the 32-node tree), gains non-unit."""
+    shape = si.scaled(c1, Hkv=Hkv)
+    weights = si.all_weights(shape, gains=True)
+    for T, n0 in ((16, 70), (32, 9)):
+        parents = si.tree_template(T)
+        eng, orc = make_pair(shape, weights, 256, max_tree=32, max_k=3, max_depth=3)
+        st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=n0), 4, k=3, l=1, forced_steps=(1, 3))
+        assert st.steps == 4
+        eng.close()
+
+
+@pytest.mark.parametrize("fused", [True, False])
 @pytest.mark.parametrize("case", range(4))
-def test_c1_random_trees_and_layers(torch_cuda, c1, c1_weights, case):
+def test_c1_random_trees_and_layers(torch_cuda, c1, c1_weights, case, fused):
     T = (5, 16, 33, 128)[case]
     k = (1, 3, 2, 3)[case]
     l = (0, 1, 1, 0)[case]
     parents = si.random_tree(21, T, k, case)
-    eng, orc = make_pair(c1, c1_weights, 512, max_tree=128, max_k=3, max_depth=3)
+    eng, orc = make_pair(c1, c1_weights, 512, max_tree=128, max_k=3, max_depth=3, fused=fused)
     st = lockstep_run(eng, orc, c1, parents, si.prompt(c1, length=(3, 70, 129, 200)[case]), 4, k=k, l=l)
     assert st.steps == 4
     eng.close()
@@ -89,6 +127,59 @@ def test_c1_equal_layers_are_the_single_layer_call_bit_for_bit(torch_cuda, c1, c
         eng.close()
     for a, b in zip(logits[0], logits[1]):
         assert np.array_equal(a, b)
+
+
+def test_fused_and_per_operation_paths_agree_and_repeat_bit_for_bit(torch_cuda, c1, c1_weights):
+    """The persistent kernel and the kernel-per-operation path run the same arithmetic (they may split the cached
+    positions differently for the attention): logits agree to fp32 rounding.  Each path repeated on the same state
+    gives bit-identical logits (fixed summation orders everywhere)."""
+    import torch
+    shape = si.scaled(c1, Hkv=2)
+    weights = si.all_weights(shape, gains=True)
+    parents = si.random_tree(4, 29, 3, 1)
+    tokens = torch.from_numpy(si.random_tokens(shape, 29, 3)).cuda()
+    prompt = torch.from_numpy(si.prompt(shape, length=150)).cuda()
+    got = {}
+    for fused in (True, False):
+        eng, _ = make_pair(shape, weights, 256, max_tree=32, max_k=3, max_depth=3, fused=fused)
+        pout = eng.new_out(1, 1, 3, T_next=29)
+        eng.prefill(0, prompt, 3, [0, 1, 1], parents, pout)
+        out = eng.new_out(1, 29, 3)
+        runs = []
+        for _ in range(3):
+            eng.step(tokens, parents, 3, [0, 1, 1], out)
+            torch.cuda.synchronize()
+            runs.append(out.logits.cpu().numpy().copy())
+        assert np.array_equal(runs[0], runs[1]) and np.array_equal(runs[0], runs[2]), "fused=%s: logits differ from run to run" % fused
+        got[fused] = (pout.logits.cpu().numpy().copy(), runs[0])
+        assert eng.launches() <= (8 if fused else 10 ** 6)
+        eng.close()
+    for a, b in zip(got[True], got[False]):
+        assert np.abs(a - b).max() < 1e-4, np.abs(a - b).max()
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_goes_on(torch_cuda, c1, c1_weights):
+    """The time-out path: with the wait limit set to 200 us, firp_selftest_wait enqueues a kernel that waits (with
+    the routine the product kernels use) on a barrier nobody arrives on; the wait runs out, the kernel returns, the
+    next firp_context_len reports FIRP_ERR_DEVICE_TIMEOUT once, and the same context then steps in lock-step with
+    the oracle as if nothing had happened."""
+    import time
+    import torch
+    from paper_2410_20488_b200 import FirpError, binding
+    parents = si.tree_template(c1.T)
+    eng, orc = make_pair(c1, c1_weights, 256)
+    eng.set_wait_limit_us(200)
+    t0 = time.time()
+    eng.selftest_wait()
+    with pytest.raises(FirpError) as e:
+        eng.context_len(0)
+    assert e.value.code == binding.FIRP_ERR_DEVICE_TIMEOUT
+    assert time.time() - t0 < 1.0                      # the 200 us limit was used, not the 2 s default
+    assert eng.context_len(0) == 0                    # reported once, then cleared
+    eng.set_wait_limit_us(0)
+    st = lockstep_run(eng, orc, c1, parents, si.prompt(c1), 3)
+    assert st.steps == 3
+    eng.close()
 
 
 def test_layers_are_validated_on_the_host(torch_cuda, c1, c1_weights):
@@ -164,23 +255,52 @@ def test_c1_predictor_with_bias(torch_cuda, c1, c1_weights):
 
 
 def test_device_side_commit_matches_explicit(torch_cuda, c1, c1_weights):
-    """firp_kv_commit(NULL path) uses the path found on the device."""
+    """firp_kv_commit(path = NULL) compacts the path the device's own walk found: forced-accept steps make that a
+    real depth-3 path; the committed cache rows and the logits of the following steps are compared with the oracle,
+    which commits the same path explicitly."""
     import torch
     parents = si.tree_template(c1.T)
     eng, orc = make_pair(c1, c1_weights, 256)
-    prompt = si.prompt(c1)
-    d_prompt = torch.from_numpy(prompt).cuda()
-    pout = eng.new_out(1, 1, c1.k, T_next=c1.T)
-    eng.prefill(0, d_prompt, c1.k, c1.l, parents, pout)
+    st = lockstep_run(eng, orc, c1, parents, si.prompt(c1), 2)
+    tokens = si.random_tokens(c1, c1.T, 123)              # any tree will do: forced mode plants the principal chain
+    st = lockstep_steps(eng, orc, c1, parents, tokens, 6, forced=True, device_commit=True, check_cache_rows=True)
+    assert st.steps == 6 and st.emitted == 6 * 4
+    # free-running with device-side commits: the committed length follows the device's own counts
     out = eng.new_out(1, c1.T, c1.k)
-    tokens = pout.next_tree_tokens[0].clone()
-    total = prompt.size
-    for _ in range(6):
-        eng.step(tokens, parents, c1.k, c1.l, out)
-        eng.commit(1)                                   # device-side path
+    total = eng.context_len(0)
+    d_tokens = torch.from_numpy(np.ascontiguousarray(tokens)).cuda()
+    for _ in range(4):
+        eng.step(d_tokens, parents, c1.k, c1.l, out)
+        eng.commit(1)
         total += int(out.n_accepted[0].item())
         assert eng.context_len(0) == total
-        tokens = out.next_tree_tokens[0].clone()
+        d_tokens = out.next_tree_tokens[0].clone()
+    eng.close()
+
+
+def test_device_side_commits_do_not_exhaust_the_capacity_bound(torch_cuda, c1, c1_weights):
+    """A free-running loop that only ever commits on the device: the host's upper bound of the committed length
+    grows by max_depth + 1 per step, the true length by about 1.  The step must keep running until the TRUE
+    length reaches max_ctx (it re-reads the exact length before refusing), and refuse then."""
+    import torch
+    from paper_2410_20488_b200 import FirpError, binding
+    parents = si.tree_template(c1.T)
+    eng, _ = make_pair(c1, c1_weights, 128)
+    pout = eng.new_out(1, 1, c1.k, T_next=c1.T)
+    eng.prefill(0, torch.from_numpy(si.prompt(c1, length=16)).cuda(), c1.k, c1.l, parents, pout)
+    out = eng.new_out(1, c1.T, c1.k)
+    tokens = pout.next_tree_tokens[0].clone()
+    steps, total = 0, 16
+    with pytest.raises(FirpError) as e:
+        for _ in range(200):
+            eng.step(tokens, parents, c1.k, c1.l, out)
+            eng.commit(1)
+            steps += 1
+            total += int(out.n_accepted[0].item())
+            tokens = out.next_tree_tokens[0].clone()
+    assert e.value.code == binding.FIRP_ERR_CAPACITY
+    assert total + c1.T + c1.k > 128 and steps > (128 - 16 - 11) // 4, (steps, total)   # far beyond where the bound alone would stop
+    assert eng.context_len(0) == total
     eng.close()
 
 
@@ -217,13 +337,18 @@ def c2_weights():
 
 def test_c2_full_size_lockstep(torch_cuda, c2_weights):
     """The Llama-2-7B-shaped workload the benchmark times (T = 32, k = 3, l = 16, 512 committed
-    tokens): prefill and three lock-step steps against the oracle, the last one forced-accept."""
+    tokens): prefill and three lock-step steps against the oracle, the last one forced-accept (a depth-3 path is
+    compacted at the full 4096-wide cache rows and compared), then one more forced step committed from the
+    device's own path."""
     c2 = si.CONFIGS["c2"]
     parents = si.tree_template(c2.T)
     eng, orc = make_pair(c2, c2_weights, 512 + 64)
-    st = lockstep_run(eng, orc, c2, parents, si.prompt(c2), 2, forced=False, check_cache_rows=True)
-    print("c2 greedy", st.as_dict())
-    assert st.steps == 2
+    st = lockstep_run(eng, orc, c2, parents, si.prompt(c2), 3, forced_steps=(2,), check_cache_rows=True, sync_prefix=True)
+    print("c2 greedy + forced", st.as_dict())
+    assert st.steps == 3 and st.emitted == 1 + 1 + 1 + 4
+    tokens = si.random_tokens(c2, c2.T, 123)
+    st = lockstep_steps(eng, orc, c2, parents, tokens, 1, forced=True, device_commit=True, check_cache_rows=True)
+    print("c2 forced, device-side commit", st.as_dict())
     eng.close()
 
 
@@ -233,7 +358,8 @@ def test_c2_layers_15_20_25_full_size(torch_cuda, c2_weights):
     c2 = si.CONFIGS["c2"]
     parents = si.tree_template(c2.T)
     eng, orc = make_pair(c2, c2_weights, 128 + 64)          # a 128-token context keeps the oracle's prefill short
-    st = lockstep_run(eng, orc, c2, parents, si.prompt(c2, length=128), 2, forced=False, check_cache_rows=False, l=[15, 20, 25])
+    st = lockstep_run(eng, orc, c2, parents, si.prompt(c2, length=128), 2, forced=False, check_cache_rows=False, l=[15, 20, 25],
+                      sync_prefix=True)
     print("c2 layers 15/20/25", st.as_dict())
     assert st.steps == 2
     eng.close()
@@ -245,19 +371,11 @@ def test_c2_chain_under_every_node_full_size(torch_cuda, c2_weights):
     c2 = si.CONFIGS["c2"]
     parents = si.tree_template(c2.T)
     eng, orc = make_pair(c2, c2_weights, 128 + 160, max_rows=c2.T * (1 + c2.k))
-    st = lockstep_run(eng, orc, c2, parents, si.prompt(c2, length=128), 1, forced=False, check_cache_rows=False, chains=True)
+    st = lockstep_run(eng, orc, c2, parents, si.prompt(c2, length=128), 1, forced=False, check_cache_rows=False, chains=True,
+                      sync_prefix=True)
     print("c2 chains", st.as_dict())
     assert st.steps == 1
     eng.close()
-
-
-# Logits tolerance of the deep configurations.  Both sides store keys and values as bf16, so a key or value whose
-# fp32 pre-image lies next to a rounding boundary may round differently on the two sides, and the one-ulp
-# difference feeds the layers above.  Perturbing the ORACLE's own pre-rounding keys/values by 1e-7 relative (the
-# size of a change of fp32 summation order) moves its logits by 0.012 on the 32-layer shape and 0.024 on the
-# 40-layer shape (1e-6: 0.031): any two correct implementations with a bf16 cache differ by that much.  The stated
-# 3e-2 is kept up to 32 layers; deeper shapes get twice that, the relative bound of 2e-2 stays.
-DEEP_ABS_TOL = 6e-2
 
 
 def test_c4_tree_sizes_full_depth(torch_cuda, c2_weights):
@@ -268,7 +386,7 @@ def test_c4_tree_sizes_full_depth(torch_cuda, c2_weights):
         k = 0 if T == 1 else 3
         parents = si.tree_template(T)
         eng, orc = make_pair(c2, c2_weights, 128 + 160, max_tree=T, max_k=max(k, 1), max_depth=3)
-        st = lockstep_run(eng, orc, c2, parents, si.prompt(c2, length=128), 1, k=k, l=c2.l, check_cache_rows=False)
+        st = lockstep_run(eng, orc, c2, parents, si.prompt(c2, length=128), 1, k=k, l=c2.l, check_cache_rows=False, sync_prefix=True)
         print("c4 full depth T=%d" % T, st.as_dict())
         assert st.steps == 1
         eng.close()
@@ -295,88 +413,64 @@ def test_c2_width_chains_with_one_layer_per_step(torch_cuda):
     eng.close()
 
 
-def test_c4_long_context_2048(torch_cuda, c2_width_2_layers):
-    """Sweep point with a 2048-token committed context (prefilled through the chunked step path on both sides)
-    at the full Llama-2-7B width, with the depth cut to 2 layers so that the oracle's prefill stays affordable:
-    split-KV attention over 33 tiles in 8 splits; the per-layer work is that of the full model."""
+@pytest.mark.parametrize("n_ctx", [2048, 8192])
+def test_c4_long_contexts_against_the_oracle(torch_cuda, c2_width_2_layers, n_ctx):
+    """Sweep points with 2048 and 8192 committed tokens at the full Llama-2-7B width, depth cut to 2 layers, for
+    T = 1 (k = 0), 32 and 128: both sides start from the same seeded prefix (bit-identical cache rows written into
+    both caches, no prefill), so the oracle's cost per step is linear in the context.  The attention then runs over
+    33 / 129 tiles in 8 splits, with one, one and three query blocks."""
     shape, weights = c2_width_2_layers
-    for T in (32,):
+    for T in (1, 32, 128):
+        k = 0 if T == 1 else 3
         parents = si.tree_template(T)
-        eng, orc = make_pair(shape, weights, 2048 + 256, max_tree=128, max_k=3, max_depth=3)
-        st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=2048), 2, check_cache_rows=True)
-        print("c4 long context T=%d n=2048" % T, st.as_dict())
+        eng, orc = make_pair(shape, weights, n_ctx + 2 * 160, max_tree=128, max_k=3, max_depth=3)
+        seed_prefix(eng, orc, shape, 0, n_ctx)
+        st = lockstep_steps(eng, orc, shape, parents, si.random_tokens(shape, T, 77 + T), 2, k=k, l=shape.l if k else 0,
+                            forced_steps=(1,) if k else (), check_cache_rows=True)
+        print("c4 seeded context n=%d T=%d" % (n_ctx, T), st.as_dict())
         assert st.steps == 2
         eng.close()
 
 
-def test_c4_context_8192_tree_rows_match_own_path_steps(torch_cuda, c2_width_2_layers):
-    """At 8192 committed tokens the oracle's attention is out of reach (its cost grows with the square of the
-    context), so the longest sweep context is checked through a property that holds at any size (Section 3.4:
-    a tree token sees the prefix and its ancestors only): the logits of a tree row must equal the logits of the
-    plain autoregressive step (T = 1, k = 0) that feeds the same root-to-node path token by token -- the pin
-    that ties the oracle's tree step to a causal decoder, applied to the CUDA path itself over 129 kv tiles."""
-    import torch
-    shape, weights = c2_width_2_layers
-    n_ctx, T, k = 8192, 16, 3
-    parents = si.tree_template(T)
-    from paper_2410_20488_b200 import FirpEngine
-    eng = FirpEngine(shape, weights, max_ctx=n_ctx + 64, max_tree=128, max_k=3, max_depth=3)
-    d_prompt = torch.from_numpy(si.prompt(shape, length=n_ctx)).cuda()
-    pout = eng.new_out(1, 1, k, T_next=T)
-    eng.prefill(0, d_prompt, k, shape.l, parents, pout)
-    assert eng.context_len(0) == n_ctx
-    tokens = si.random_tokens(shape, T, 77)
-    out = eng.new_out(1, T, k)
-    eng.step(torch.from_numpy(tokens).cuda(), parents, k, shape.l, out)
-    torch.cuda.synchronize()
-    tree_logits = out.logits[0].cpu().numpy()
-    one = np.array([-1], np.int32)
-    out1 = eng.new_out(1, 1, 0, T_next=1)
-    worst = 0.0
-    leaves = [v for v in range(T) if v not in set(parents.tolist())][:3]
-    for leaf in leaves:
-        path = []
-        v = leaf
-        while v >= 0:
-            path.append(v)
-            v = int(parents[v])
-        eng.set_context_len(0, n_ctx)                      # rewind to the committed prefix
-        for node in path[::-1]:
-            eng.step(torch.from_numpy(tokens[node:node + 1]).cuda(), one, 0, 0, out1)
-            eng.commit(1, path=[[0]])
-            torch.cuda.synchronize()
-            worst = max(worst, float(np.abs(out1.logits[0, 0].cpu().numpy() - tree_logits[node]).max()))
-        assert eng.context_len(0) == n_ctx + len(path)
-    print("context 8192: tree rows vs own path steps, max abs logit difference %.5f" % worst)
-    assert worst <= 1e-2
-    eng.close()
-
-
 def test_c3_full_depth(torch_cuda):
-    """Llama-2-13B shape, all 40 layers, T = 64, k = 3 at layer 20, on a 128-token context (the configuration's
-    1024-token prompt would cost the oracle minutes of prefill; long contexts are covered on the 7B width)."""
+    """Llama-2-13B shape, all 40 layers, T = 64, k = 3 at layer 20, on the configuration's 1024 committed tokens
+    (seeded prefix on both sides): two lock-step steps, the second forced-accept, then the prompt path: a 128-token
+    prefill through the library and one more step."""
     c3 = si.CONFIGS["c3"]
     weights = si.all_weights(c3)
     parents = si.tree_template(c3.T)
-    eng, orc = make_pair(c3, weights, 128 + 160)
-    st = lockstep_run(eng, orc, c3, parents, si.prompt(c3, length=128), 2, check_cache_rows=False, abs_tol=DEEP_ABS_TOL)
-    print("c3", st.as_dict())
-    assert st.steps == 2 and st.max_rel <= 2e-2
+    eng, orc = make_pair(c3, weights, 1024 + 2 * 160)
+    seed_prefix(eng, orc, c3, 0, 1024)
+    st = lockstep_steps(eng, orc, c3, parents, si.random_tokens(c3, c3.T, 5), 2, forced_steps=(1,), check_cache_rows=True)
+    print("c3 seeded context 1024", st.as_dict())
+    assert st.steps == 2
+    st = lockstep_run(eng, orc, c3, parents, si.prompt(c3, length=128), 1, check_cache_rows=False, sync_prefix=True)
+    print("c3 after a 128-token prefill", st.as_dict())
     eng.close()
 
 
 def test_c5_gqa_batch_reduced_depth(torch_cuda):
     """34B grouped-query shape (d 8192, 64 query / 8 kv heads, FFN 22016), batch of 4 sequences with their own
-    32-node trees and their own context lengths, stepped by one firp_step call; depth cut from 48 to 4 layers
-    (the full model needs a minute of oracle time per step and 67 GB of weights on both sides)."""
-    from lockstep import lockstep_run_batch
+    32-node trees, stepped by one firp_step call; depth cut from 48 to 4 layers (the full model needs a minute of
+    oracle time per step and 67 GB of weights on both sides).  First on short prompts through the library's
+    prefill, then on the configuration's context lengths (drawn uniformly from [256, 4096], seeded prefixes):
+    the sequences then differ in their number of kv tiles inside one attention launch."""
+    from lockstep import lockstep_run_batch, lockstep_steps_batch
     shape = si.scaled(si.CONFIGS["c5"], L=4, l=2, name="c5-width-4-layers")
     weights = si.all_weights(shape)
     parents = si.tree_template(shape.T)
     lengths = (23, 64, 97, 130)
     prompts = [si.prompt(shape, seq=s, length=n) for s, n in enumerate(lengths)]
-    eng, orc = make_pair(shape, weights, 130 + 96, max_batch=4)
-    st = lockstep_run_batch(eng, orc, shape, parents, prompts, 2)
-    print("c5 reduced depth", st.as_dict())
+    eng, orc = make_pair(shape, weights, 4096 + 160, max_batch=4)
+    st = lockstep_run_batch(eng, orc, shape, parents, prompts, 1)
+    print("c5 reduced depth, short prompts", st.as_dict())
+    assert st.steps == 4
+    ctx = si.context_lengths(shape)
+    assert ctx.min() >= 256 and ctx.max() <= 4096 and len(set(ctx.tolist())) == 4
+    for s_i, n in enumerate(ctx):
+        seed_prefix(eng, orc, shape, s_i, int(n))
+    tokens = np.stack([si.random_tokens(shape, shape.T, 40 + s_i) for s_i in range(4)])
+    st = lockstep_steps_batch(eng, orc, shape, parents, tokens, 2, check_cache_rows=True)
+    print("c5 reduced depth, contexts %s" % ctx.tolist(), st.as_dict())
     assert st.steps == 8
     eng.close()

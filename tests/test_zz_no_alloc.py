@@ -54,3 +54,38 @@ def test_static_topb_matches_step_twice_in_a_row(c1, c1_weights):
         firp_topb_static(out.logits.data_ptr(), T + k, V, 9, ids.data_ptr(), vals.data_ptr(), eng.stream)
     assert e.value.code == binding.FIRP_ERR_BAD_ARG
     eng.close()
+
+
+@pytest.mark.parametrize("rows,vocab,b", [(1365, 5000, 5), (256, 32000, 3), (2, 4097, 8), (4096, 2048, 1), (7, 1, 1)])
+def test_static_topb_many_segments_and_ragged_tails(rows, vocab, b):
+    """The same call on synthetic fp32 logits whose rows span several 2048-logit segments with a ragged last
+    one, at row counts that fill the built-in scratch almost to its 4096 slots (1365 x 3 = 4095, 256 x 16 =
+    4096), with b < 8, and with planted ties; twice in a row on different data."""
+    import torch
+    assert torch.cuda.is_available(), "this test needs a CUDA device"
+    from paper_2410_20488_b200 import FirpError, binding, build as firp_build, firp_topb_static
+    firp_build.build()
+    stream = torch.cuda.current_stream().cuda_stream
+    ids = torch.empty((rows, b), dtype=torch.int32, device="cuda")
+    vals = torch.empty((rows, b), dtype=torch.float32, device="cuda")
+    for call in range(2):
+        bits = si.normal_bf16(11 + call, si.stream_id("tokens", 500), rows * vocab, 1.0)
+        logits = si.bf16_bits_to_f32(bits).reshape(rows, vocab).copy()          # bf16-valued: ties do occur
+        if vocab > 2:
+            logits[0, :] = 0.25                                                # a row of ties: lowest ids win
+            logits[rows - 1, vocab - 1] = 9.0                                  # the winner sits in the ragged tail
+        d_logits = torch.from_numpy(logits).cuda()
+        ids.fill_(-1)
+        firp_topb_static(d_logits.data_ptr(), rows, vocab, b, ids.data_ptr(), vals.data_ptr(), stream)
+        torch.cuda.synchronize()
+        got_ids, got_vals = ids.cpu().numpy(), vals.cpu().numpy()
+        bb = min(b, vocab)
+        check = sorted(set([0, rows - 1] + list(range(0, rows, max(1, rows // 64)))))
+        for r in check:
+            want = np.lexsort((np.arange(vocab), -logits[r]))[:bb]
+            assert np.array_equal(got_ids[r, :bb], want), "row %d (call %d)" % (r, call)
+            assert np.array_equal(got_vals[r, :bb], logits[r][want])
+    # a vocabulary whose segment count does not fit 32 bits of intermediate arithmetic is refused, not wrapped
+    with pytest.raises(FirpError) as e:
+        firp_topb_static(d_logits.data_ptr(), 1, 2 ** 31 - 1, b, ids.data_ptr(), vals.data_ptr(), stream)
+    assert e.value.code == binding.FIRP_ERR_CAPACITY
