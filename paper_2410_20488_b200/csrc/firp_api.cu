@@ -236,7 +236,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   if (fused) {      // all decoder layers (and the lm-head) as one persistent kernel
     FusedStep fs{};
     fs.shape = fshape; fs.rw = rw; memcpy(fs.tl, ra.tl, sizeof(fs.tl)); fs.want_head = ra.want_head; fs.Rp = (int)Rp;
-    fs.n_hi_max = ra.n_hi_max; fs.weights_gen = c->weights_gen; fs.wait_ns = c->wait_ns;
+    fs.n_hi_max = ra.n_hi_max; fs.max_batch = cfg.max_batch; fs.weights_gen = c->weights_gen; fs.wait_ns = c->wait_ns;
     fs.wqkv = c->wqkv.data(); fs.wo = c->wo.data(); fs.wgu = c->wgu.data(); fs.wd = c->wd.data();
     fs.g_attn = c->g_attn.data(); fs.g_mlp = c->g_mlp.data();
     fs.g_final = c->w.g_final; fs.lm_head = c->w.lm_head; fs.pred_w = c->w.pred_w; fs.pred_b = c->w.pred_b;

@@ -208,6 +208,7 @@ struct FusedStep {
   bool want_head;            // final norm + lm-head
   int Rp;                    // rows per activation plane
   int n_hi_max;              // upper bound of the longest committed context among the sequences
+  int max_batch;             // of the configuration (sizes the attention scratch)
   uint64_t weights_gen;      // changes whenever the weight pointers change
   unsigned long long wait_ns;   // bound of every device-side wait (0: default)
   // weights (device pointers; the per-layer arrays are host arrays of L pointers)

@@ -41,10 +41,11 @@ namespace {
 
 constexpr int BM = 128, TM = 2, BK = kGemmBK;
 constexpr int W_TILE = BM * 128, W_STAGE = TM * W_TILE;   // one unit: 2 x 128 weight rows x 64 k = 32 KB
-constexpr int kFThreads = 224;
-constexpr int SW = 4;                                     // weight stages (128 KB in flight per SM)
-constexpr int SX = 4;                                     // activation stages
-constexpr int kRegion = 96 * 1024;                        // activation ring, reused by the attention phases
+constexpr int kFThreads = 352;                            // 11 warps: 3 single-thread roles + 8 worker warps
+constexpr int kWorkers = 256;
+constexpr int SW = 5;                                     // weight stages (160 KB in flight per SM)
+constexpr int SX = 3;                                     // activation stages
+constexpr int kRegion = 64 * 1024;                        // activation ring, reused by the attention phases
 constexpr int kSmallBytes = kAttnQRows * kMaskWords * 4 + kAttnQRows * 4;   // s_mask, s_row
 constexpr int kBarBytes = 256;
 constexpr int kFusedSmem = SW * W_STAGE + kRegion + kSmallBytes + kBarBytes;
@@ -60,7 +61,7 @@ enum RowMode { ROWS_LINEAR = 0, ROWS_GATE_UP = 1, ROWS_ROTARY = 2 };
 
 struct GemmClass {
   int mode, F, half;   // how a supertile maps to weight rows
-  int U, KB;           // stream-K schedule over gridDim.x CTAs
+  int U, KB, G;        // stream-K schedule: CTAs 0..G-1 share the units (G = min(grid, U)), the others have none
   int P;               // activation planes
   int xmap;            // tensor map of the activations
   int N, K;
@@ -93,20 +94,28 @@ struct FusedParams {
 };
 static_assert(sizeof(FusedParams) <= 32000, "kernel parameter space");
 
-struct WorkerSync { static __device__ __forceinline__ void sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); } };
+#ifdef FIRP_TRACE     // development aid, not part of the product build: per-CTA time stamps of every phase
+__device__ unsigned long long *g_trace = nullptr;
+#define FIRP_STAMP(slot) do { if (wtid == 0 && g_trace) g_trace[((size_t)cta * kMaxFusedOps + oi) * 2 + (slot)] = globaltimer(); } while (0)
+#else
+#define FIRP_STAMP(slot) do { } while (0)
+#endif
+
+struct WorkerSync { static __device__ __forceinline__ void sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); } };      // all 8 worker warps
+struct AttnGroupSync { static __device__ __forceinline__ void sync() { asm volatile("bar.sync 3, 128;" ::: "memory"); } };   // warps 2..5
 
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 // Grid-wide barrier of the worker warps (128 threads per CTA).  Monotonic arrival counter; `epoch` counts the
 // barriers passed.  The wait is bounded: on expiry the status word is set and this thread stops waiting for good.
 __device__ __forceinline__ void grid_sync(unsigned *ctr, unsigned &epoch, int wtid, int *err, bool &dead,
-                                          unsigned long long wait_ns) {
-  fence_proxy_async();            // what this thread wrote must also be visible to TMA reads of other CTAs
-  __threadfence();
+                                          unsigned long long wait_ns, bool tma_reads_follow) {
+  if (tma_reads_follow) fence_proxy_async();   // what this thread wrote will be read by TMA loads of other CTAs
   WorkerSync::sync();
   ++epoch;
   if (wtid == 0 && !dead) {
     const unsigned target = epoch * gridDim.x;
+    // release at gpu scope, cumulative: it also orders what the other workers wrote before the block barrier
     asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ctr) : "memory");
     const unsigned long long t0 = globaltimer();
     uint32_t spins = 0;
@@ -120,9 +129,8 @@ __device__ __forceinline__ void grid_sync(unsigned *ctr, unsigned &epoch, int wt
         break;
       }
     }
-    __threadfence();
   }
-  WorkerSync::sync();
+  WorkerSync::sync();             // the acquire of thread 0 reaches the other workers through this barrier
 }
 
 template <int NPAD>
@@ -152,23 +160,20 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
   if (threadIdx.x == 0) {
     for (int i = 0; i < SW; ++i) { mbar_init(full_w + 8 * i, 1); mbar_init(empty_w + 8 * i, 1); }
     for (int i = 0; i < SX; ++i) { mbar_init(full_x + 8 * i, 1); mbar_init(empty_x + 8 * i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 8); }
     mbar_init(xgo, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
   griddep_launch();
-  uint32_t tmem_base = 0;
-  if (warp >= 1 && warp <= 5) {
-    if (warp == 1) {
-      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512) : "memory");
-      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    asm volatile("bar.sync 2, 160;" ::: "memory");
-    tc_fence_after();
-    tmem_base = *tmem_slot_ptr;
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
 
   bool dead = false;
   if (warp == 0) {
@@ -179,8 +184,8 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
       for (int g = 0; g < P.n_gemm; ++g) {
         const GemmClass &c = P.cls[P.gemm_cls[g]];
         const CUtensorMap *tm = P.maps + P.gemm_map[g];
-        const StreamK sk{c.U, c.KB, G};
-        const int u0 = sk_begin(sk, cta), n_units = sk_begin(sk, cta + 1) - u0;
+        const StreamK sk{c.U, c.KB, c.G};
+        const int u0 = cta < c.G ? sk_begin(sk, cta) : 0, n_units = cta < c.G ? sk_begin(sk, cta + 1) - u0 : 0;
         for (int it = 0; it < n_units; ++it, ++k) {
           const int u = u0 + it;
           const int st = u / c.KB, kb = u - st * c.KB;
@@ -211,8 +216,8 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
       for (int g = 0; g < P.n_gemm; ++g) {
         const GemmClass &c = P.cls[P.gemm_cls[g]];
         const CUtensorMap *tm = P.maps + c.xmap;
-        const StreamK sk{c.U, c.KB, G};
-        const int u0 = sk_begin(sk, cta), n_units = sk_begin(sk, cta + 1) - u0;
+        const StreamK sk{c.U, c.KB, c.G};
+        const int u0 = cta < c.G ? sk_begin(sk, cta) : 0, n_units = cta < c.G ? sk_begin(sk, cta + 1) - u0 : 0;
         mbar_wait(xgo, g & 1, P.err, dead, wait_ns);     // the workers have passed the barrier before this GEMM
         fence_proxy_async();
         for (int it = 0; it < n_units; ++it, ++k) {
@@ -232,8 +237,8 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
       unsigned use[2] = {0u, 0u};
       for (int g = 0; g < P.n_gemm; ++g) {
         const GemmClass &c = P.cls[P.gemm_cls[g]];
-        const StreamK sk{c.U, c.KB, G};
-        const int u0 = sk_begin(sk, cta), u1 = sk_begin(sk, cta + 1);
+        const StreamK sk{c.U, c.KB, c.G};
+        const int u0 = cta < c.G ? sk_begin(sk, cta) : 0, u1 = cta < c.G ? sk_begin(sk, cta + 1) : 0;
         const int ACC = c.P * NPAD;                       // accumulator columns per weight tile
         const int nbuf = (2 * TM * ACC <= 512) ? 2 : 1;
         const uint32_t idesc = instr_desc_m128(ACC);
@@ -271,11 +276,12 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
         }
       }
     }
-  } else {                       // ---- workers, warps 2..5
-    const int wtid = threadIdx.x - 64;              // 0..127
+  } else {                       // ---- workers: warps 2..5 (group A) and 7..10 (group B)
+    const int wgroup = warp >= 7 ? 1 : 0;
+    const int wtid = wgroup ? threadIdx.x - 224 + 128 : threadIdx.x - 64;   // 0..255
     const int quarter = warp & 3;                   // TMEM lane quarter this warp may read
     const int li = quarter * 32 + lane;             // row within each 128-row tile = TMEM lane
-    const unsigned tbase = (unsigned)cta * 128u + (unsigned)wtid, tstride = (unsigned)G * 128u;
+    const unsigned tbase = (unsigned)cta * (unsigned)kWorkers + (unsigned)wtid, tstride = (unsigned)G * (unsigned)kWorkers;
     unsigned epoch = 0;
     unsigned use[2] = {0u, 0u};
     const int nq = P.H * P.dh;
@@ -284,11 +290,12 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
     if (P.n_ops > 0 && P.ops[0].type == OP_GEMM && wtid == 0) mbar_arrive(xgo);
     for (int oi = 0; oi < P.n_ops; ++oi) {
       const FusedOp &op = P.ops[oi];
+      FIRP_STAMP(0);
       switch (op.type) {
         case OP_GEMM: {          // TMEM -> partial tiles of this CTA's segments
           const GemmClass &c = P.cls[op.cls];
-          const StreamK sk{c.U, c.KB, G};
-          const int u0 = sk_begin(sk, cta), u1 = sk_begin(sk, cta + 1);
+          const StreamK sk{c.U, c.KB, c.G};
+          const int u0 = cta < c.G ? sk_begin(sk, cta) : 0, u1 = cta < c.G ? sk_begin(sk, cta + 1) : 0;
           const int ACC = c.P * NPAD;
           const int nbuf = (2 * TM * ACC <= 512) ? 2 : 1;
           int seg = 0;
@@ -299,28 +306,24 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
             const int buf = seg % nbuf;
             mbar_wait(acc_full + 8 * buf, use[buf] & 1u, P.err, dead, wait_ns);
             tc_fence_after();
-            const uint32_t tacc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * TM * ACC);
-            float *my_ws = P.ws + (size_t)(cta * kGemmSlots + seg) * slot_elems + li;
+            // group A drains the first weight tile of the supertile, group B the second
+            const uint32_t tacc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * TM * ACC + wgroup * ACC);
+            float *my_ws = P.ws + (size_t)(cta * kGemmSlots + seg) * slot_elems + (size_t)wgroup * plane_elems + li;
             for (int c0 = 0; c0 < P.rw.R && seg < kGemmSlots; c0 += 16) {
-              float r0[16], r1[16];
+              float r0[16];
               tc_ld16(tacc + c0, r0);
-              tc_ld16(tacc + ACC + c0, r1);
               tc_ld_wait();
               for (int pl = 1; pl < c.P; ++pl) {      // columns pl * NPAD .. hold the sums over plane pl
-                float l0[16], l1[16];
+                float l0[16];
                 tc_ld16(tacc + pl * NPAD + c0, l0);
-                tc_ld16(tacc + ACC + pl * NPAD + c0, l1);
                 tc_ld_wait();
 #pragma unroll
-                for (int j = 0; j < 16; ++j) { r0[j] += l0[j]; r1[j] += l1[j]; }
+                for (int j = 0; j < 16; ++j) r0[j] += l0[j];
               }
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
                 const int m = c0 + j;
-                if (m < P.rw.R) {
-                  __stcg(my_ws + (size_t)m * BM, r0[j]);
-                  __stcg(my_ws + plane_elems + (size_t)m * BM, r1[j]);
-                }
+                if (m < P.rw.R) __stcg(my_ws + (size_t)m * BM, r0[j]);
               }
             }
             tc_fence_before();
@@ -335,7 +338,7 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
         case OP_NORM: {
           Partials pend{};
           pend.ws = P.ws; pend.ws_rows = P.Rp;
-          if (op.aux >= 0) { const GemmClass &c = P.cls[op.aux]; pend.sk = StreamK{c.U, c.KB, G}; }
+          if (op.aux >= 0) { const GemmClass &c = P.cls[op.aux]; pend.sk = StreamK{c.U, c.KB, c.G}; }
           const unsigned total = (unsigned)(P.rw.n_seq * op.nv * (P.d >> 2));
           for (unsigned t = tbase; t < total; t += tstride)
             rmsnorm_item(P.rw, op.v0, op.nv, P.h, pend, (const bf16 *)op.ptr, P.d, P.x, (size_t)P.Rp * P.d, op.planes, P.ss, t);
@@ -349,7 +352,7 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
         case OP_FINISH: {
           const GemmClass &c = P.cls[op.cls];
           Partials p{};
-          p.sk = StreamK{c.U, c.KB, G}; p.ws = P.ws; p.ws_rows = P.Rp;
+          p.sk = StreamK{c.U, c.KB, c.G}; p.ws = P.ws; p.ws_rows = P.Rp;
           GemmArgs a{};
           a.R = P.rw.R; a.rw = P.rw; a.rows_active = op.act; a.N = c.N; a.K = c.K; a.eps = P.eps;
           const int n_st = c.U / c.KB;
@@ -384,15 +387,15 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
           const int qblocks = (op.act * Gq + kAttnQRows - 1) / kAttnQRows;
           const int n_items = P.rw.n_seq * qblocks * P.Hkv * P.splits;
           const size_t item_floats = (size_t)kAttnQRows * (P.dh + 2);
-          for (int item = cta; item < n_items; item += G) {
+          for (int item = cta; item < n_items && wgroup == 0; item += G) {      // group A's four warps; group B waits at the barrier
             const int split = item % P.splits, rest = item / P.splits;
             const int kvh = rest % P.Hkv, z = rest / P.Hkv;
             float *out = P.attn_ws + (size_t)item * item_floats;
             if (P.dh == 128)
-              attn_split_item<128, WorkerSync>(a, region, s_mask, s_row, wtid, z / qblocks, kvh, z % qblocks, split, P.splits,
+              attn_split_item<128, AttnGroupSync>(a, region, s_mask, s_row, wtid, z / qblocks, kvh, z % qblocks, split, P.splits,
                                                out, out + kAttnQRows, out + 2 * kAttnQRows);
             else
-              attn_split_item<64, WorkerSync>(a, region, s_mask, s_row, wtid, z / qblocks, kvh, z % qblocks, split, P.splits,
+              attn_split_item<64, AttnGroupSync>(a, region, s_mask, s_row, wtid, z / qblocks, kvh, z % qblocks, split, P.splits,
                                               out, out + kAttnQRows, out + 2 * kAttnQRows);
           }
           break;
@@ -437,8 +440,11 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
         }
         default: break;
       }
-      grid_sync(P.bar, epoch, wtid, P.err, dead, wait_ns);
-      if (oi + 1 < P.n_ops && P.ops[oi + 1].type == OP_GEMM && wtid == 0) mbar_arrive(xgo);
+      FIRP_STAMP(1);
+      if (oi + 1 == P.n_ops) break;      // nothing in this kernel reads what the last phase wrote
+      const bool gemm_next = P.ops[oi + 1].type == OP_GEMM;
+      grid_sync(P.bar, epoch, wtid, P.err, dead, wait_ns, gemm_next);
+      if (gemm_next && wtid == 0) mbar_arrive(xgo);
     }
   }
   tc_fence_before();
@@ -515,7 +521,8 @@ int fused_sm_count() {
   return n;
 }
 
-GemmClass make_class(int epi, int N, int K, int P, int xmap, int F, int H, int Hkv, int dh) {
+GemmClass make_class(int epi, int N, int K, int P, int xmap, int F, int H, int Hkv, int dh, int grid = 0) {
+  if (grid == 0) grid = fused_sm_count();
   GemmClass c{};
   c.epi = epi; c.N = N; c.K = K; c.P = P; c.xmap = xmap;
   c.mode = ROWS_LINEAR;
@@ -524,14 +531,14 @@ GemmClass make_class(int epi, int N, int K, int P, int xmap, int F, int H, int H
   else if (epi == EPI_QKV_ROPE) { c.mode = ROWS_ROTARY; c.half = dh / 2; const int hp = BM / c.half; n_st = (H + 2 * Hkv + hp - 1) / hp; }
   c.KB = (K + BK - 1) / BK;
   c.U = n_st * c.KB;
+  c.G = c.U < grid ? c.U : grid;
   return c;
 }
 
-// every CTA must own a non-empty range that touches at most kGemmSlots supertiles
-bool class_fits(const GemmClass &c, int G) {
-  if (c.U < G) return false;
-  const int per = (c.U + G - 1) / G;
-  return (per + c.KB - 2) / c.KB + 1 <= kGemmSlots && (long long)(c.U + 1) * (G + 1) < (1ll << 31);
+// a CTA's range must touch at most kGemmSlots supertiles (one scratch slot each)
+bool class_fits(const GemmClass &c, int) {
+  const int per = (c.U + c.G - 1) / c.G;
+  return (per + c.KB - 2) / c.KB + 1 <= kGemmSlots && (long long)(c.U + 1) * (c.G + 1) < (1ll << 31);
 }
 
 }  // namespace
@@ -550,7 +557,7 @@ size_t fused_map_bytes(int n_layers) { return sizeof(CUtensorMap) * (size_t)(4 *
 size_t fused_attn_ws_floats(int max_batch, int H, int Hkv, int dh) {
   const int Gq = H / Hkv;
   const int groups = max_batch * Hkv * ((48 * Gq + kAttnQRows - 1) / kAttnQRows);
-  const int items = groups > 192 ? groups : 192;
+  const int items = groups > 320 ? groups : 320;
   return (size_t)items * kAttnQRows * (dh + 2);
 }
 
@@ -558,6 +565,13 @@ cudaError_t launch_wait_selftest(int *err, unsigned long long wait_ns, cudaStrea
   wait_selftest_kernel<<<1, 32, 0, st>>>(err, wait_ns ? wait_ns : kDefaultWaitNs);
   return cudaGetLastError();
 }
+
+#ifdef FIRP_TRACE
+extern "C" int firp_debug_set_trace(unsigned long long *buf) {
+  return (int)cudaMemcpyToSymbol(g_trace, &buf, sizeof(buf));
+}
+extern "C" int firp_debug_max_ops() { return kMaxFusedOps; }
+#endif
 
 bool fused_eligible(const FusedShape &sh, const Rows &rw) {
   if (!fused_encode_fn()) return false;
@@ -680,14 +694,22 @@ cudaError_t launch_fused_layers(FusedPlan *plan, const FusedStep &fs, bool pdl, 
   P.logits = fs.logits;
   P.wait_ns = fs.wait_ns;
   {
+    // kv splits: every (sequence x query block, kv head, split) is one work item, a CTA takes items cta, cta + G, ...
+    // Pick the split count that minimises the 64-position tiles the busiest CTA walks through (rounds x tiles per
+    // split), with a charge per round for the latency of an item's first loads (measured: about 2.5 tiles' worth).
     const int Gq = H / Hkv;
     const int tiles = (fs.n_hi_max + rw.Ms + kAttnTile - 1) / kAttnTile;
     const int groups = rw.n_seq * Hkv * ((rw.Ms * Gq + kAttnQRows - 1) / kAttnQRows);
-    int s = G / groups;
-    s = s < 1 ? 1 : s;
-    s = s > tiles ? tiles : s;
-    s = s > kMaxSplitsFused ? kMaxSplitsFused : s;
-    P.splits = s < 1 ? 1 : s;
+    const size_t cap_items = fused_attn_ws_floats(fs.max_batch, H, Hkv, dh) / ((size_t)kAttnQRows * (dh + 2));
+    int best = 1;
+    float best_cost = 1e30f;
+    for (int s = 1; s <= kMaxSplitsFused && s <= tiles; ++s) {
+      if ((size_t)groups * s > cap_items) break;
+      const int rounds = (groups * s + G - 1) / G, per = (tiles + s - 1) / s;
+      const float cost = (float)rounds * ((float)per + 2.5f);   // an item costs about 2.5 tiles' worth before its first tile
+      if (cost < best_cost - 1e-6f) { best_cost = cost; best = s; }
+    }
+    P.splits = best;
   }
   static bool configured[2] = {false, false};
   auto kernel = NPAD == 16 ? fused_layers_kernel<16> : fused_layers_kernel<48>;
