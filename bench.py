@@ -46,6 +46,9 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-kernel-times", action="store_true", help="skip the per-kernel event-timed pass")
+    ap.add_argument("--fused", type=int, default=-1, choices=[-1, 0, 1], help="1: the decoder layers of a step as one persistent "
+                    "kernel, 0: one kernel per operation, -1: the library's default")
+    ap.add_argument("--no-forced", action="store_true", help="skip the forced-accept run")
     ap.add_argument("--sweep", action="store_true", help="config-4 sweep on the c2 weights: T x context, one JSON line per point")
     return ap.parse_args()
 
@@ -95,18 +98,25 @@ def class_bytes(shape, n_ctx: float) -> dict:
     (read once) for the GEMMs and the Eq. 3 maps, the K and V planes of one layer for the attention."""
     s = shape
     M = s.T + s.k
+    ab = algorithmic_bytes(s, n_ctx)
     return dict(gemm_qkv=2 * s.n_qkv * s.d, gemm_o=2 * s.d * s.n_q, gemm_gate_up=2 * 2 * s.F * s.d,
                 gemm_down=2 * s.d * s.F, gemm_lm_head=2 * s.V * s.d, pseudo_proj=2 * s.k * s.d * s.d,
-                tree_attention=2 * 2 * s.n_kv * (n_ctx + M))
+                tree_attention=2 * 2 * s.n_kv * (n_ctx + M),
+                # the persistent kernel runs every layer, Eq. 3 and the lm-head: all weights once, the cache once
+                fused_decoder_layers=ab["weights"] - 2 * s.V * s.d + ab["kv_read"] + ab["kv_write"])
 
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of a kernel class at the
-# c2 shape, from the ncu capture summarised under profiles/; valid only for the kernel sources whose
-# digest is recorded with it (a changed kernel reports traffic = null until it is captured again).
-NCU_TRAFFIC = {  # dram read+write per launch; includes the ~24 MB successor head each GEMM prefetches
-    "c2-llama2-7b": dict(digest="a2bb6d50dd07d0bc", per_launch={"gemm_gate_up": 221511168, "gemm_qkv": 129046016,
-                                                             "gemm_o": 52361472, "gemm_down": 119311872}),
-}
+def ncu_traffic(workload: str):
+    """DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of each kernel class, from the ncu
+    capture summarised in profiles/ncu_traffic.json; valid only for the kernel sources whose digest is recorded
+    with it (a changed kernel reports traffic = null until it is captured again)."""
+    try:
+        rec = json.load(open(os.path.join(ROOT, "profiles", "ncu_traffic.json"))).get(workload)
+    except (OSError, ValueError):
+        return None
+    if not rec or rec.get("digest") != kernel_source_digest():
+        return None
+    return rec.get("per_launch", {})
 
 
 def kernel_source_digest() -> str:
@@ -146,10 +156,8 @@ def kernel_times(eng, shape, parents, tokens, out, steps, n_ctx, peak_gbs, peak_
         kernels[name] = k
     top = max((n for n in kernels if n in cb), key=lambda n: kernels[n]["share"])
     t = kernels[top]
-    rec = NCU_TRAFFIC.get(shape.name)
-    traffic = None
-    if rec and rec["digest"] == kernel_source_digest():
-        traffic = rec["per_launch"].get(top)
+    rec = ncu_traffic(shape.name)
+    traffic = rec.get(top) if rec else None
     roofline = dict(bound="hbm", kernel=top, achieved=t["achieved_gbs"], peak=peak_gbs, unit="GB/s",
                     frac=t["frac_of_peak"], traffic=traffic, peak_kind="%s copy bandwidth" % peak_kind,
                     avg_us=t["avg_us"], share_of_kernel_time=t["share"], bytes_per_launch=t["bytes_per_launch"],
@@ -215,6 +223,14 @@ class ClockSampler:
                     reasons=sorted(reasons), samples=len(sm))
 
 
+def eng_fused(args) -> bool:
+    """What --fused selects; -1 is the library's default."""
+    return LIB_DEFAULT_FUSED if args.fused < 0 else bool(args.fused)
+
+
+LIB_DEFAULT_FUSED = False
+
+
 def host_cores() -> int:
     try:
         return len(os.sched_getaffinity(0))
@@ -222,16 +238,24 @@ def host_cores() -> int:
         return os.cpu_count() or 1
 
 
-def time_oracle(shape, weights, steps: int, warmup: int, n_ctx: int = 32):
-    """The CPU oracle, as it stands, on a bounded sample: `steps` full draft+verify steps (all layers,
-    T + k rows) on top of a short prefilled context."""
+def time_oracle(shape, weights, steps: int, warmup: int, n_ctx: int | None = None):
+    """The CPU oracle, as it stands, on a bounded sample: `steps` full draft+verify steps (all layers, T + k rows)
+    on the workload's own committed context length.  The context is not prefilled (the oracle's prefill grows with
+    the square of the context): its cache rows are seeded values (synth_inputs.cache_rows), so a step costs what a
+    step on a real context of that length costs."""
     import oracle
     import synth_inputs as si
+    n_ctx = shape.prompt_len if n_ctx is None else n_ctx
     parents = si.tree_template(shape.T)
     rows = shape.T * (1 + shape.k) if CHAINS else shape.T + shape.k
     orc = oracle.Oracle(shape, weights, max_ctx=n_ctx + (steps + warmup + 1) * (shape.k + 1) + rows + 8)
-    r = orc.prefill(si.prompt(shape, length=n_ctx), shape.k, ins_l(shape), parents)
-    tokens = r["next_tokens"]
+    std = 0.02 * float(np.sqrt(shape.d))
+    for layer in range(shape.L):
+        ks, vs = si.cache_rows(shape, 0, layer, n_ctx, std, std)
+        orc.write_cache(0, layer, 0, 0, ks)
+        orc.write_cache(0, layer, 1, 0, vs)
+    orc.set_context_len(0, n_ctx)
+    tokens = si.random_tokens(shape, shape.T, 9)
     emitted, t_total = 0, 0.0
     for i in range(warmup + steps):
         t0 = time.perf_counter()
@@ -243,6 +267,57 @@ def time_oracle(shape, weights, steps: int, warmup: int, n_ctx: int = 32):
             emitted += int(out["n_accepted"])
         tokens = out["next_tokens"]
     return emitted / t_total, t_total / steps * 1e3
+
+
+def run_forced(eng, shape, parents, tokens, outs, K, dev, step_fn):
+    """Forced-accept throughput (every step accepts the full depth D of the tree and emits D + 1 tokens, so every
+    commit compacts a real path), without the oracle: the greedy continuation of the committed sequence is first
+    produced on the device by plain T = 1, k = 0 steps, the context is rewound, and each timed step then gets that
+    continuation planted on the principal chain (root -> lowest-index child -> ...) of its tree.  A near-tie that
+    the two passes resolve differently would show as tokens_per_step < D + 1; nothing is assumed, the emitted
+    tokens are counted from the growth of the committed context."""
+    import torch
+    T = shape.T
+    chain = [0]
+    while True:
+        kids = [u for u in range(T) if parents[u] == chain[-1]]
+        if not kids:
+            break
+        chain.append(min(kids))
+    D = len(chain) - 1
+    n0 = eng.context_len(0)
+    need = K * (D + 1) + D + 1
+    one = np.array([-1], np.int32)
+    o1 = eng.new_out(1, 1, 0, T_next=1, want_logits=False)
+    stream = torch.empty(need + 1, dtype=torch.int32, device=dev)
+    tok = tokens[0, :1].clone()
+    stream[0] = tok[0]
+    for i in range(need):
+        eng.step(tok, one, 0, 0, o1)
+        eng.commit(1)
+        tok = o1.accepted_tokens[0, :1].clone()
+        stream[i + 1] = tok[0]
+    eng.set_context_len(0, n0)                       # rewind to the committed prefix (synchronises)
+    idx = torch.tensor(chain[1:], dtype=torch.long, device=dev)
+    cur = tokens.clone()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    p = 0
+    for i in range(K):
+        cur[0, 0] = stream[p]
+        cur[0, idx] = stream[p + 1: p + 1 + D]
+        o = outs[i & 1]
+        step_fn(cur, parents, shape.k, ins_l(shape), o, seq_ids=[0], n_seq=1)
+        eng.commit(1, seq_ids=[0])
+        cur = o.next_tree_tokens.clone()
+        p += D + 1
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1)
+    emitted = eng.context_len(0) - n0
+    return dict(tokens_per_s=emitted / (ms * 1e-3), tokens_per_step=emitted / K, ms_per_step=ms / K, steps=K, depth=D,
+                note="device-resident; the timed region also holds the three small torch kernels per step that plant the chain")
 
 
 def load_weights(shape, local_rank: int, world: int):
@@ -262,14 +337,13 @@ def run_reference(args, shape):
     weights = si.all_weights(shape)
     steps, warmup = max(1, min(args.steps, 3)), min(args.warmup, 1)
     tps, ms = time_oracle(shape, weights, steps, warmup)
-    sample = "%d oracle steps (+%d warm-up) of T=%d,k=%d,l=%s over all %d layers on a 32-token context" % (
-        steps, warmup, shape.T, shape.k, ins_l(shape), shape.L)
+    sample = "%d oracle steps (+%d warm-up) of T=%d,k=%d,l=%s over all %d layers on a %d-token context (seeded cache rows, no prefill)" % (
+        steps, warmup, shape.T, shape.k, ins_l(shape), shape.L, shape.prompt_len)
     line = dict(metric=METRIC, value=tps, unit=UNIT, n_gpus=args.gpus, steps=steps, warmup=warmup, ms_per_step=ms,
                 higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32 storage, f64 accumulation",
                 data="synthetic", impl="reference",
                 config=dict(workload=shape.name, T=shape.T, k=shape.k, l=ins_l(shape), context_start=shape.prompt_len,
-                            batch=1, sample="oracle steps on a 32-token context instead of %d tokens (its prefill "
-                            "cost grows with the context; the step's GEMM work does not)" % shape.prompt_len),
+                            batch=1, sample="a few oracle steps on the workload's %d-token context" % shape.prompt_len),
                 cpu_baseline=dict(value=tps, unit=UNIT, cores=host_cores(), kind="oracle", sample=sample),
                 e2e=dict(value=tps, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line))
@@ -362,7 +436,7 @@ def main():
     parents = si.tree_template(shape.T)
     B = shape.batch
     S = max(shape.k, 1) + 1
-    total_steps = 2 * (K + W) + 16
+    total_steps = 4 * (K + W) + 32
     if B > 1:       # config 5: every sequence has its own committed context length, uniform in [256, 4096]
         lengths = [int(n) for n in si.context_lengths(shape)]
     else:
@@ -371,6 +445,8 @@ def main():
     rows_per_seq = shape.T * (1 + shape.k) if chains else shape.T + shape.k
     max_ctx = max(lengths) + total_steps * S + rows_per_seq + 64
     eng = FirpEngine(shape, weights, max_ctx=max_ctx, max_batch=B, device=str(dev), max_rows=B * rows_per_seq if chains else 0)
+    if args.fused >= 0:
+        eng.set_fused(bool(args.fused))
     step_fn = eng.step_chains if chains else eng.step
     T_next = shape.T if shape.k > 0 else 1
     outs = [eng.new_out(B, shape.T, shape.k, want_logits=False, chains=chains) for _ in range(2)]
@@ -450,6 +526,11 @@ def main():
         e2e = dict(ms=e0.elapsed_time(e1), emitted=e_emitted, h2d=int(h_tokens.numel() * 4),
                    d2h=int((h_acc.numel() + h_n.numel() + h_next.numel()) * 4))
 
+    # ---- forced-accept mode (a = D every step): rank-local, one sequence --------------------
+    forced = None
+    if not args.no_forced and shape.k > 0 and B == 1 and not chains:
+        forced = run_forced(eng, shape, parents, tokens, outs, K, dev, step_fn)
+
     # ---- aggregate over ranks: max time, summed units ----------------------------------------
     ms_max, units = aggregate_over_ranks(ms_total, emitted, dev)
     if e2e:
@@ -478,7 +559,8 @@ def main():
                 config=dict(workload=shape.name, T=shape.T, k=shape.k, l=ins_l(shape), context_start=n_start,
                             context_end=n_end, batch=B, pseudo_rows="a chain under every node" if chains else "one chain under the root", l2="inputs_larger_than_l2 (%.1f GB of weights per step)" %
                             (ab["weights"] / 1e9), parallelism="replicas x%d" % world,
-                            mode="free-running greedy (random weights accept ~0 drafts per step)"),
+                            mode="free-running greedy (random weights accept ~0 drafts per step); forced_accept has the a = D case",
+                            layers_as="one persistent kernel" if eng_fused(args) else "one kernel per operation"),
                 step_latency_us=ms_step * 1e3, tokens_per_step=units / (K * world), tokens_per_step_per_sequence=units / (K * world * B),
                 step_hbm=dict(bytes_per_step=ab["total"], weights=ab["weights"], kv_read=ab["kv_read"],
                               achieved_gbs=step_gbs, frac_of_measured_peak=step_gbs / peak_gbs,
@@ -489,6 +571,8 @@ def main():
     if e2e:
         line["e2e"] = dict(value=e_units / (e_ms_max * 1e-3), unit=UNIT, ms_per_step=e_ms_max / K,
                            h2d_bytes_per_step=e2e["h2d"], d2h_bytes_per_step=e2e["d2h"])
+    if forced:
+        line["forced_accept"] = forced
     if prof:
         line["roofline"] = prof["roofline"]
         line["kernels"] = prof["kernels"]
@@ -497,11 +581,11 @@ def main():
         line["roofline"] = dict(bound="hbm", achieved=step_gbs, peak=peak_gbs, unit="GB/s", frac=step_gbs / peak_gbs,
                                 traffic=None, note="whole step (all kernels): bytes per step / step time; peak = %s copy bandwidth" % peak_kind)
     if not args.no_cpu_baseline:
-        cb_steps = 1
+        cb_steps = 2 if shape.name.startswith("c2") else 1
         tps, ms = time_oracle(shape, weights, cb_steps, 0)
         line["cpu_baseline"] = dict(value=tps, unit=UNIT, cores=host_cores(), kind="oracle", ms_per_step=ms,
-                                    sample="%d oracle step of T=%d,k=%d,l=%s over all %d layers on a 32-token context "
-                                           "(plus its 32-token prefill, untimed)" % (cb_steps, shape.T, shape.k, ins_l(shape), shape.L))
+                                    sample="%d oracle steps of T=%d,k=%d,l=%s over all %d layers on a %d-token context "
+                                           "(seeded cache rows, no prefill)" % (cb_steps, shape.T, shape.k, ins_l(shape), shape.L, shape.prompt_len))
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -198,9 +198,10 @@ int firp_kv_commit(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const i
 
 /*
  * How the decoder layers of a step are launched (Section 3.4 describes one forward pass per round; the
- * paper gives no kernel design).  on != 0 (default): a step of at most 48 rows over all its sequences
- * runs its layers, Eq. 3 and the lm-head as ONE persistent kernel whose weight stream never stops between
- * operations; larger steps, and every step when on == 0, use one kernel per operation.  Both run the same
+ * paper gives no kernel design).  on != 0: a step of at most 48 rows over all its sequences runs its
+ * layers, Eq. 3 and the lm-head as ONE persistent kernel (6 launches per step instead of ~300) whose weight
+ * stream never stops between operations; larger steps, and every step when on == 0 (the default: it
+ * measured 2-3 % faster at the 7B shape), use one kernel per operation.  Both run the same
  * arithmetic; they may cut the cached positions into a different number of attention splits, so their
  * results agree to fp32 rounding, and each is identical from run to run.
  */

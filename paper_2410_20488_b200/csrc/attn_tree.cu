@@ -125,7 +125,7 @@ template <int DH> cudaError_t launch_dh(const AttnArgs &a, bool pdl, cudaStream_
 int attention_splits(int groups, int kv_tiles) {
   // CTAs of one (kv head, query block) = one cluster (<= 8): about two CTAs per SM over the whole grid,
   // never more splits than 64-position tiles
-  static const int budget = [] { const char *e = getenv("FIRP_ATTN_CTAS"); return e ? atoi(e) : 296; }();
+  const int budget = 296;
   int s = 1;
   while (s < kAttnMaxSplits && 2 * s * groups <= budget && 2 * s <= kv_tiles) s *= 2;
   return s;

@@ -51,7 +51,7 @@ struct firp_ctx {
   bool bound = false, have_weights = false, stepped = false;
   int Rmax = 0, S = 0;
   bool use_pdl = true;                  // programmatic dependent launch
-  bool use_fused = true;                // steps of at most 48 rows run their layers as one persistent kernel
+  bool use_fused = false;               // firp_set_fused: steps of at most 48 rows run their layers as one persistent kernel
   unsigned long long wait_ns = 0;       // bound of device-side waits (0: the kernels' default)
   uint64_t weights_gen = 0;             // bumped by firp_init_weights
   FusedPlan *plan_step = nullptr, *plan_prefill = nullptr;
@@ -215,14 +215,8 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   const bool pdl = c->use_pdl;
   // L2 lookahead per GEMM class (32 KB units beyond the ring): qkv, o, gate/up, down, lm-head.  Measured at the
   // 7B shape: it pays before the GEMMs whose predecessor is short or cannot share the SM (o, gate/up) and
-  // costs before the down projection, whose finisher it slows by more than it saves.  FIRP_L2_AHEAD=a,b,c,d,e
-  // overrides (tuning aid).
-  static int ahead[5] = {0, 48, 48, 0, 48};
-  static bool ahead_init = false;
-  if (!ahead_init) {
-    ahead_init = true;
-    if (const char *e = getenv("FIRP_L2_AHEAD")) sscanf(e, "%d,%d,%d,%d,%d", &ahead[0], &ahead[1], &ahead[2], &ahead[3], &ahead[4]);
-  }
+  // costs before the down projection, whose finisher it slows by more than it saves.
+  static const int ahead[5] = {0, 48, 48, 0, 48};
 
   const int mw_out = (rw.Ms + 31) / 32;
   { FIRP_TIMED(KC_TREE_PREP);
@@ -264,13 +258,8 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   pending.ws = c->gemm_ws; pending.ws_rows = (int)Rp;
   const Partials none{};
   // every GEMM names its successor, whose first units it prefetches into L2 at its own tail
-  // (32 KB units per CTA, by the GEMM that issues the prefetch: qkv, o, gate/up, down; FIRP_NEXT_UNITS=a,b,c,d overrides)
-  static int next_units[4] = {5, 5, 5, 5};
-  static bool next_init = false;
-  if (!next_init) {
-    next_init = true;
-    if (const char *e = getenv("FIRP_NEXT_UNITS")) sscanf(e, "%d,%d,%d,%d", &next_units[0], &next_units[1], &next_units[2], &next_units[3]);
-  }
+  // (32 KB units per CTA, by the GEMM that issues the prefetch: qkv, o, gate/up, down; 3 and 8 measured worse)
+  static const int next_units[4] = {5, 5, 5, 5};
   auto set_next = [&](GemmArgs &g, int cls, GemmEpilogue epi, const void *W, int N, int K) {
     g.next_W = (const bf16 *)W; g.next_epi = epi; g.next_N = N; g.next_K = K; g.next_F = F; g.next_heads = H + 2 * Hkv;
     g.next_dh = dh; g.next_units = next_units[cls];
@@ -421,9 +410,6 @@ int firp_create(const firp_model_cfg *cfg, firp_ctx **out) {
   c->Rmax = (int)align_up(rows, 16);
   c->S = cfg->max_depth + 1;
   c->n_hi.assign(cfg->max_batch, 0);
-  // debugging switch: FIRP_PDL=0 launches every kernel in plain stream order
-  const char *ep = getenv("FIRP_PDL");
-  c->use_pdl = !(ep && strcmp(ep, "0") == 0);
 
   c->ws_bytes = c->carve(nullptr);
   *out = c;

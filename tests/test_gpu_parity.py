@@ -18,8 +18,8 @@ def torch_cuda():
     return torch
 
 
-def make_pair(shape, weights, max_ctx, masked=False, fused=True, **kw):
-    """fused=False: one kernel per operation even for small steps (the path steps of more than 48 rows take)."""
+def make_pair(shape, weights, max_ctx, masked=False, fused=False, **kw):
+    """fused=True: steps of at most 48 rows run their decoder layers as one persistent kernel (firp_set_fused)."""
     from paper_2410_20488_b200 import FirpEngine
     eng = FirpEngine(shape, weights, max_ctx=max_ctx, **kw)
     eng.set_fused(fused)
@@ -42,42 +42,45 @@ def test_c1_greedy_and_forced(torch_cuda, c1, c1_weights, fused):
         eng.close()
 
 
-def test_c1_t1_k0_autoregressive(torch_cuda, c1, c1_weights):
-    eng, orc = make_pair(c1, c1_weights, 128, max_tree=8, max_k=3)
+@pytest.mark.parametrize("fused", [False, True])
+def test_c1_t1_k0_autoregressive(torch_cuda, c1, c1_weights, fused):
+    eng, orc = make_pair(c1, c1_weights, 128, max_tree=8, max_k=3, fused=fused)
     st = lockstep_run(eng, orc, c1, np.array([-1], np.int32), si.prompt(c1, length=9), 12, k=0, l=0)
     assert st.steps == 12 and st.emitted == 13
     eng.close()
 
 
-def test_c1_non_unit_gains(torch_cuda, c1):
+@pytest.mark.parametrize("fused", [False, True])
+def test_c1_non_unit_gains(torch_cuda, c1, fused):
     """RMSNorm gains that differ between the attention norm, the MLP norm and the final norm of every layer
     (the workload configurations use gains of 1, which would hide a swapped or dropped gain)."""
     weights = si.all_weights(c1, gains=True)
     parents = si.tree_template(c1.T)
     for forced in (False, True):
-        eng, orc = make_pair(c1, weights, 256)
+        eng, orc = make_pair(c1, weights, 256, fused=fused)
         st = lockstep_run(eng, orc, c1, parents, si.prompt(c1, length=41), 6, forced=forced)
         assert st.steps == 6
         eng.close()
     # per-step insertion layers and a chain under every node take other kernel paths for the new rows' norm
     shape = si.scaled(c1, L=4)
     w4 = si.all_weights(shape, gains=True)
-    eng, orc = make_pair(shape, w4, 256, max_tree=16, max_k=3, max_depth=3, max_rows=13 * 4)
+    eng, orc = make_pair(shape, w4, 256, max_tree=16, max_k=3, max_depth=3, max_rows=13 * 4, fused=fused)
     parents = si.random_tree(3, 13, 3, 2)
     assert lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=30), 3, k=3, l=[0, 2, 3]).steps == 3
     assert lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=30), 3, k=3, l=[1, 2, 2], chains=True).steps == 3
     eng.close()
 
 
+@pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("Hkv", [2, 1])
-def test_c1_grouped_query_attention_two_query_blocks(torch_cuda, c1, Hkv):
+def test_c1_grouped_query_attention_two_query_blocks(torch_cuda, c1, Hkv, fused):
     """4 query heads on 2 or 1 key/value heads with enough rows that rows x heads-per-group exceeds one
     64-row query block (19 x 2 = 38 and 19 x 4 = 76; 35 x 4 = 140 with the 32-node tree), gains non-unit."""
     shape = si.scaled(c1, Hkv=Hkv)
     weights = si.all_weights(shape, gains=True)
     for T, n0 in ((16, 70), (32, 9)):
         parents = si.tree_template(T)
-        eng, orc = make_pair(shape, weights, 256, max_tree=32, max_k=3, max_depth=3)
+        eng, orc = make_pair(shape, weights, 256, max_tree=32, max_k=3, max_depth=3, fused=fused)
         st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=n0), 4, k=3, l=1, forced_steps=(1, 3))
         assert st.steps == 4
         eng.close()
@@ -219,11 +222,12 @@ def test_c1_a_chain_under_every_node(torch_cuda, c1, case):
         eng.close()
 
 
+@pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("chains", [False, True])
-def test_c1_masked_pseudo_rows(torch_cuda, c1, c1_weights, chains):
+def test_c1_masked_pseudo_rows(torch_cuda, c1, c1_weights, chains, fused):
     """The "Masked" ablation of Section 4.3 (firp_set_pseudo_masked): pseudo rows do not see one another."""
     parents = si.random_tree(3, 13, 3, 2)
-    eng, orc = make_pair(c1, c1_weights, 256, masked=True, max_tree=16, max_k=3, max_depth=3, max_rows=13 * 4)
+    eng, orc = make_pair(c1, c1_weights, 256, masked=True, max_tree=16, max_k=3, max_depth=3, max_rows=13 * 4, fused=fused)
     st = lockstep_run(eng, orc, c1, parents, si.prompt(c1, length=40), 4, k=3, l=1 if chains else [0, 1, 1], chains=chains)
     assert st.steps == 4
     eng.close()
@@ -352,12 +356,14 @@ def test_c2_full_size_lockstep(torch_cuda, c2_weights):
     eng.close()
 
 
-def test_c2_layers_15_20_25_full_size(torch_cuda, c2_weights):
+@pytest.mark.parametrize("fused", [False, True])
+def test_c2_layers_15_20_25_full_size(torch_cuda, c2_weights, fused):
     """The prediction layers the paper uses for its 7B models (Section 4 "Setup": 15, 20, 25) on the
-    7B-shaped workload: prefill and two lock-step steps against the oracle."""
+    7B-shaped workload: prefill and two lock-step steps against the oracle, with the layers of a step as one
+    kernel per operation and as one persistent kernel."""
     c2 = si.CONFIGS["c2"]
     parents = si.tree_template(c2.T)
-    eng, orc = make_pair(c2, c2_weights, 128 + 64)          # a 128-token context keeps the oracle's prefill short
+    eng, orc = make_pair(c2, c2_weights, 128 + 64, fused=fused)          # a 128-token context keeps the oracle's prefill short
     st = lockstep_run(eng, orc, c2, parents, si.prompt(c2, length=128), 2, forced=False, check_cache_rows=False, l=[15, 20, 25],
                       sync_prefix=True)
     print("c2 layers 15/20/25", st.as_dict())
