@@ -67,6 +67,7 @@ def bind(lib):
     lib.oracle_tree_prep_chains.argtypes = [vp, i32, i32, vp, vp, vp, vp]
     lib.oracle_tree_prep_chains.restype = i32
     lib.oracle_set_masked.argtypes = [vp, i32]
+    lib.oracle_set_prenorm.argtypes = [vp, i32]
     lib.oracle_mask_pseudo.argtypes = [vp, i32, i32]
     lib.oracle_verify.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
     lib.oracle_verify.restype = i32
@@ -161,8 +162,9 @@ class Oracle:
     """
 
     def __init__(self, shape, weights, max_ctx: int, n_seq: int = 1, top_b: int = 8, kv_bf16: bool = True,
-                 masked: bool = False):
-        """masked: the "Masked" setting of Section 4.3 (a pseudo row sees no other pseudo row)."""
+                 masked: bool = False, prenorm: bool = False):
+        """masked: the "Masked" setting of Section 4.3 (a pseudo row sees no other pseudo row).
+        prenorm: Eq. 3 reads the anchor's state through the input RMSNorm of the insertion layer."""
         self.lib = _get_lib()
         self.shape, self.weights, self.top_b = shape, weights, top_b
         s = shape
@@ -201,6 +203,7 @@ class Oracle:
         self._w = w
         self.lib.oracle_set_weights(self.h, ctypes.byref(w))
         self.lib.oracle_set_masked(self.h, int(masked))
+        self.lib.oracle_set_prenorm(self.h, int(prenorm))
 
     def __del__(self):
         if getattr(self, "h", None):

@@ -93,6 +93,7 @@ typedef struct {
   oracle_cfg cfg;
   oracle_weights w;
   int32_t masked;  /* != 0: the "Masked" setting of Section 4.3: a pseudo row does not see other pseudo rows */
+  int32_t prenorm; /* != 0: Eq. 3 reads the anchor's state through the RMSNorm of the layer it is inserted at */
   int32_t *n;      /* committed length per sequence */
   float **kc;      /* per sequence: [L][max_ctx][Hkv*dh] */
   float **vc;
@@ -137,6 +138,11 @@ void oracle_set_weights(void *h, const oracle_weights *w) { ((oracle_t *)h)->w =
 /* Section 4.3 compares "No masked" (a pseudo row sees the earlier rows of its chain; the default, what the paper
  * adopts) with "Masked" (it sees none of them: only the prefix, its node's ancestors and node, and itself). */
 void oracle_set_masked(void *h, int32_t masked) { ((oracle_t *)h)->masked = masked; }
+
+/* Eq. 3 applies the map to the hidden state h^{t_i} as it stands (Section 3.3; the default here).  A variant the
+ * equation's wording leaves open feeds the map what the decoder layer itself would read: the state after the
+ * input RMSNorm of layer t_i, h~_i = W_i rmsnorm(h^{t_i}; g_attn[t_i]) + b_i.  prenorm != 0 selects it. */
+void oracle_set_prenorm(void *h, int32_t prenorm) { ((oracle_t *)h)->prenorm = prenorm; }
 
 /* The "Masked" setting applied to a visibility matrix of T tree rows + pseudo rows: pseudo rows keep what they
  * see among the tree rows and themselves, and lose every other pseudo row. */
@@ -293,7 +299,12 @@ static int32_t forward_core(oracle_t *o, int32_t seq, const int32_t *tokens, int
       if (tl[i] != j) continue;
       /* Eq. 3: h~ = W_i h[src] + b_i on the residual entering layer t_i, appended as row T+r */
       float *dst = h + (size_t)(T + r) * d;
-      linear(w->pred_w + (size_t)i * d * d, h + (size_t)p_src[r] * d, d, dst, d, 1, d, d);
+      const float *src = h + (size_t)p_src[r] * d;
+      if (o->prenorm) {   /* variant: the map reads the anchor through layer j's input norm */
+        rmsnorm(src, w->g_attn[j], c->eps, x, 1, d);
+        src = x;
+      }
+      linear(w->pred_w + (size_t)i * d * d, src, d, dst, d, 1, d, d);
       if (w->pred_b) for (int cc = 0; cc < d; ++cc) dst[cc] += bf16f(w->pred_b[(size_t)i * d + cc]);
       if (h_ins) memcpy(h_ins + (size_t)r * d, dst, sizeof(float) * d);
       rows = T + r + 1;

@@ -78,12 +78,14 @@ def hf_kv(model, token_ids):
     return ks, vs
 
 
-def hf_logits_with_replaced_rows(model, token_ids, layer, first_row, maps_w, maps_b, anchor_row, visible=None):
+def hf_logits_with_replaced_rows(model, token_ids, layer, first_row, maps_w, maps_b, anchor_row, visible=None,
+                                 prenorm=False):
     """Causal forward in which, at the input of decoder layer `layer`, rows
     first_row.. are replaced by W_i h[anchor_row] + b_i (i = 0..len(maps_w)-1).
     `layer` may be a sequence with one layer per row: row first_row + i is then
     replaced at the input of layer[i] (what it held before is never read by a row
-    that matters, because the sequence is causal and the layers do not decrease)."""
+    that matters, because the sequence is causal and the layers do not decrease).
+    prenorm: the maps read the anchor row through that layer's own input RMSNorm module."""
     layers = [int(layer)] * len(maps_w) if np.isscalar(layer) else [int(t) for t in layer]
     assert len(layers) == len(maps_w) and layers == sorted(layers)
 
@@ -92,6 +94,8 @@ def hf_logits_with_replaced_rows(model, token_ids, layer, first_row, maps_w, map
             hs = args[0] if args else kwargs["hidden_states"]
             hs = hs.clone()
             src = hs[0, anchor_row]
+            if prenorm:
+                src = module.input_layernorm(src[None])[0]
             for i, W in enumerate(maps_w):
                 if layers[i] == at:
                     hs[0, first_row + i] = torch.from_numpy(W) @ src + torch.from_numpy(maps_b[i])

@@ -596,3 +596,30 @@ def test_gain_vectors_differ_and_matter(c1):
     la = a.forward(si.prompt(c1, length=5), si.chain_template(5), 0, 0)["logits"]
     lb = b.forward(si.prompt(c1, length=5), si.chain_template(5), 0, 0)["logits"]
     assert np.abs(la - lb).max() > 0.05
+
+
+# ---------------------------------------------------------------- P13: Eq. 3 on the normalised state (variant)
+@pytest.mark.parametrize("layers", [1, (0, 1, 1)])
+def test_p13_prenorm_variant_reads_the_anchor_through_the_layers_input_norm(variant, layers):
+    """The variant of Eq. 3 that feeds the map the anchor's state after the input RMSNorm of the insertion layer:
+    the chain == a library forward whose rows are replaced by W_i input_layernorm(h[anchor]) + b_i (the library's
+    own norm module, with non-unit gains in two of the three shapes); the tree rows do not change; and the
+    default (raw residual) differs from it."""
+    shape, weights, hfv = variant
+    k = 3
+    prompt = si.prompt(shape, length=12)
+    Wf = si.bf16_bits_to_f32(weights["pred_w"]).astype(np.float64)
+    bf = np.zeros((k, shape.d))
+    o = oracle.Oracle(shape, weights, max_ctx=64, kv_bf16=False, prenorm=True)
+    plain = fresh(shape, weights, max_ctx=64)
+    for orc in (o, plain):
+        orc.forward(prompt, si.chain_template(prompt.size), 0, 0)
+        orc.commit(np.arange(prompt.size))
+    tokens, parents = si.random_tokens(shape, 8, 9), si.tree_template(8)
+    l = layers if np.isscalar(layers) else list(layers)
+    out, ref_out = o.forward(tokens, parents, k, l, anchor=0), plain.forward(tokens, parents, k, l, anchor=0)
+    ids = list(prompt) + [int(tokens[0])] + [0] * k
+    ref = hf_logits_with_replaced_rows(hfv, ids, layers, prompt.size + 1, list(Wf), list(bf), prompt.size, prenorm=True)
+    assert np.abs(out["logits"][8:] - ref[prompt.size + 1:]).max() < 1e-5
+    assert np.array_equal(out["logits"][:8], ref_out["logits"][:8])
+    assert np.abs(out["logits"][8:] - ref_out["logits"][8:]).max() > 1e-3
