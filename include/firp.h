@@ -113,7 +113,8 @@ int firp_init_weights(firp_ctx *ctx, const firp_weights *w);
  * (greedy next token), n_accepted = 1, next_tree_tokens = the first draft tree on the
  * template `next_parents` (HOST, [T_next]), topb_*; logits (if given) holds 1+k rows:
  * the last prompt row, then the pseudo rows.  d_prompt is a DEVICE array [P].
- * k = 0 gives plain prefill (T_next must then be 1).
+ * k = 0 gives plain prefill (T_next must then be 1).  The prompt is processed 144 - k rows at a time
+ * (one pass over the weights per chunk), whatever max_rows is.
  */
 int firp_prefill(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int32_t P, int32_t k, int32_t l,
                  const int32_t *next_parents, int32_t T_next, const firp_step_out *out, void *stream);
@@ -179,6 +180,14 @@ int firp_step_chains(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const
  * positions are unchanged.  Applies to every later firp_prefill* / firp_step* call of the context.
  */
 int firp_set_pseudo_masked(firp_ctx *ctx, int32_t masked);
+
+/*
+ * What Eq. 3 reads (Section 3.3 writes W_i h^{t_i} + b_i and does not say whether h^{t_i} is taken before or
+ * after the layer's normalisation).  on == 0 (default): the raw residual stream entering layer t_i.  on != 0: the
+ * state the decoder layer itself reads, h~_i = W_i rmsnorm(h^{t_i}; g_attn[t_i]) + b_i.  Applies to every later
+ * firp_prefill* / firp_step* call of the context.
+ */
+int firp_set_pred_prenorm(firp_ctx *ctx, int32_t on);
 
 /*
  * Commit after a step: for each sequence move the cache rows of path[j] to slot n + j

@@ -46,7 +46,7 @@ EXPORTS = ("firp_create", "firp_destroy", "firp_last_error", "firp_workspace_byt
            "firp_bind_buffers", "firp_init_weights", "firp_prefill", "firp_step", "firp_kv_commit",
            "firp_context_len", "firp_set_context_len", "firp_last_launch_count", "firp_profile_enable",
            "firp_profile_read", "firp_kernel_class_name", "firp_topb_static", "firp_prefill_layers", "firp_step_layers", "firp_step_chains", "firp_set_pseudo_masked",
-           "firp_set_fused", "firp_set_wait_limit_us", "firp_selftest_wait")
+           "firp_set_fused", "firp_set_wait_limit_us", "firp_selftest_wait", "firp_set_pred_prenorm")
 
 
 def lib_path() -> str:
@@ -80,6 +80,7 @@ def load_library():
     lib.firp_step_chains.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp, ctypes.POINTER(StepOutC), vp]
     lib.firp_set_pseudo_masked.argtypes = [vp, i32]
     lib.firp_set_fused.argtypes = [vp, i32]
+    lib.firp_set_pred_prenorm.argtypes = [vp, i32]
     lib.firp_set_wait_limit_us.argtypes = [vp, ctypes.c_int64]
     lib.firp_selftest_wait.argtypes = [vp, vp]
     lib.firp_kv_commit.argtypes = [vp, i32, vp, vp, vp, vp]
@@ -195,6 +196,11 @@ def firp_step_chains(ctx, n_seq: int, seq_ids, d_tokens_ptr: int, tree_parents, 
 def firp_set_pseudo_masked(ctx, masked: bool):
     """Section 4.3 "Masked" ablation: pseudo rows do not see one another."""
     _check(ctx, load_library().firp_set_pseudo_masked(ctx, int(bool(masked))))
+
+
+def firp_set_pred_prenorm(ctx, on: bool):
+    """Eq. 3 on the anchor's state after the insertion layer's input RMSNorm (variant) instead of the raw residual."""
+    _check(ctx, load_library().firp_set_pred_prenorm(ctx, int(bool(on))))
 
 
 def firp_set_fused(ctx, on: bool):
@@ -355,6 +361,9 @@ class FirpEngine:
 
     def set_pseudo_masked(self, masked: bool):
         firp_set_pseudo_masked(self.ctx, masked)
+
+    def set_pred_prenorm(self, on: bool):
+        firp_set_pred_prenorm(self.ctx, on)
 
     def set_fused(self, on: bool):
         firp_set_fused(self.ctx, on)

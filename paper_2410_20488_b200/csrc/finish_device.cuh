@@ -171,10 +171,15 @@ __device__ __forceinline__ void pseudo_finish_item(const Partials &p, const Gemm
   Item it;
   if (!item_of(t, n_st, a.R, it)) return;
   const int n0 = it.st * 256 + it.i4;
+  // pre-norm variant (a.ss given): the operand was h * g; divide by the RMS of the source row of the residual stream
+  int src_row;
+  if (a.rw.chains) { const int s = it.m / a.rw.T; src_row = s * a.rw.Ms + (it.m - s * a.rw.T); }
+  else src_row = it.m * a.rw.Ms + a.rw.anchor;
+  const float rs = row_rms_scale(a, src_row);       // before any lane drops out: the warp adds together
   if (n0 >= a.N) return;
   float4 v0, v1;
   sum_partials(p, it.st, it.m, it.i4, v0, v1);
-  const float e[2][4] = {{v0.x, v0.y, v0.z, v0.w}, {v1.x, v1.y, v1.z, v1.w}};
+  const float e[2][4] = {{v0.x * rs, v0.y * rs, v0.z * rs, v0.w * rs}, {v1.x * rs, v1.y * rs, v1.z * rs, v1.w * rs}};
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
     const int n = n0 + 128 * t;                   // d is a multiple of 128: the 4 outputs belong to one map

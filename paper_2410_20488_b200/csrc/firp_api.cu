@@ -49,7 +49,8 @@ struct firp_ctx {
   std::string err;
   int launches = 0;
   bool bound = false, have_weights = false, stepped = false;
-  int Rmax = 0, S = 0;
+  int Rmax = 0, S = 0;                  // rows the workspace holds (a prefill chunk), path stride
+  int row_cap = 0;                      // rows one step may carry (max_rows of the configuration)
   bool use_pdl = true;                  // programmatic dependent launch
   bool use_fused = false;               // firp_set_fused: steps of at most 48 rows run their layers as one persistent kernel
   unsigned long long wait_ns = 0;       // bound of device-side waits (0: the kernels' default)
@@ -77,6 +78,7 @@ struct firp_ctx {
   std::vector<int32_t> last_parents, last_next_parents, last_seq_ids;
   int last_n_seq = 0, last_T = 0, last_k = 0;
   int pseudo_masked = 0;     // Section 4.3 "Masked": pseudo rows do not see one another
+  int pred_prenorm = 0;      // Eq. 3 reads the anchor through the insertion layer's input RMSNorm
 
   size_t kv_plane() const { return (size_t)cfg.max_ctx * cfg.n_kv_heads * cfg.head_dim; }
   size_t kv_layer() const { return 2 * kv_plane(); }
@@ -229,7 +231,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
   const bool fused = c->use_fused && fused_eligible(fshape, rw);
   if (fused) {      // all decoder layers (and the lm-head) as one persistent kernel
     FusedStep fs{};
-    fs.shape = fshape; fs.rw = rw; memcpy(fs.tl, ra.tl, sizeof(fs.tl)); fs.want_head = ra.want_head; fs.Rp = (int)Rp;
+    fs.shape = fshape; fs.rw = rw; memcpy(fs.tl, ra.tl, sizeof(fs.tl)); fs.want_head = ra.want_head; fs.prenorm = c->pred_prenorm != 0; fs.Rp = (int)Rp;
     fs.n_hi_max = ra.n_hi_max; fs.max_batch = cfg.max_batch; fs.weights_gen = c->weights_gen; fs.wait_ns = c->wait_ns;
     fs.wqkv = c->wqkv.data(); fs.wo = c->wo.data(); fs.wgu = c->wgu.data(); fs.wd = c->wd.data();
     fs.g_attn = c->g_attn.data(); fs.g_mlp = c->g_mlp.data();
@@ -279,13 +281,14 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     if (insert) {   // Eq. 3 on the raw (now complete) residual row of the root, then the norm of the new rows
       { FIRP_TIMED(KC_PSEUDO_PROJ);      // this layer's maps as one [ins d][d] GEMM on the source rows (the anchor of
                                          // each sequence, or every tree row when each node carries a chain)
-        launch_root_split(rw, c->h, d, c->xp, Rp * d, pdl, st); ++nl;
+        launch_root_split(rw, c->h, c->pred_prenorm ? (const bf16 *)c->g_attn[j] : nullptr, d, c->xp, Rp * d, pdl, st); ++nl;
         GemmArgs g{};
         g.X = c->xp; g.x_lo_off = Rp * d; g.plane_rows = (int)Rp; g.planes = 2; g.err = c->dev_status; g.wait_ns = c->wait_ns;
         g.W = (const bf16 *)c->w.pred_w + (size_t)alive * d * d; g.R = rw.n_seq * per_step; g.N = ins * d; g.K = d; g.rw = rw;
         g.rows_active = act;
         g.ws = c->gemm_ws; g.l2_ahead = 48;
         g.h_rows = c->h; g.pseudo0 = alive;      // map i of this GEMM is prediction step alive + i
+        if (c->pred_prenorm) { g.ss = c->ss; g.eps = cfg.rms_eps; }   // the finisher divides by the source row's RMS
         g.pred_b = c->w.pred_b ? (const bf16 *)c->w.pred_b + (size_t)alive * d : nullptr;
         Partials p = pending;
         FIRP_CUDA(c, launch_gemm_tc(EPI_PSEUDO, g, pdl, st, &p.sk)); ++nl;
@@ -407,7 +410,8 @@ int firp_create(const firp_model_cfg *cfg, firp_ctx **out) {
   if (rows > 144) return bad("max_batch * (max_tree + max_k) must be <= 144 rows");
   if (cfg->max_rows < 0 || cfg->max_rows > 144) return bad("max_rows must be 0..144");
   if (cfg->max_rows > rows) rows = cfg->max_rows;
-  c->Rmax = (int)align_up(rows, 16);
+  c->row_cap = (int)align_up(rows, 16);
+  c->Rmax = 144;          // the workspace always holds the largest row count, so that a prompt is prefilled 141 rows at a time
   c->S = cfg->max_depth + 1;
   c->n_hi.assign(cfg->max_batch, 0);
 
@@ -542,8 +546,8 @@ static int step_impl(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const
   if ((rc = check_seq_ids(ctx, n_seq, seq_ids, ids))) return rc;
   const int pseudo = chains ? T * k : k;       // pseudo rows per sequence
   const int Ms = T + pseudo;
-  if (Ms > kMaxTreeRows || n_seq * Ms > ctx->Rmax)
-    return fail(ctx, FIRP_ERR_CAPACITY, "%d sequences x %d rows exceed the row capacity %d (max_rows of the configuration)", n_seq, Ms, ctx->Rmax);
+  if (Ms > kMaxTreeRows || n_seq * Ms > ctx->row_cap)
+    return fail(ctx, FIRP_ERR_CAPACITY, "%d sequences x %d rows exceed the row capacity %d (max_rows of the configuration)", n_seq, Ms, ctx->row_cap);
   std::vector<int> depth;
   const int maxd = tree_depths(tree_parents, T, depth);
   if (maxd < 0) return fail(ctx, FIRP_ERR_BAD_TREE, "parents[0] must be -1 and 0 <= parents[v] < v");
@@ -610,7 +614,8 @@ int firp_prefill_layers(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int
   if ((rc = upload_i32(ctx, ctx->seq_ids, ids.data(), 1, ctx->last_seq_ids, st))) return rc;
   if ((rc = upload_i32(ctx, ctx->next_parents, next_parents, T_next, ctx->last_next_parents, st))) return rc;
   // chain template for the prompt rows
-  // the prompt runs in chunks of as many rows as one step may carry (fewer passes over the weights)
+  // the prompt runs in chunks of as many rows as the kernels take at once (144 less the pseudo rows of the last
+  // chunk): a 512-token prompt is four passes over the weights
   const int chunk = std::min(ctx->Rmax, kMaxTreeRows) - k;
   std::vector<int32_t> chain(chunk);
   for (int i = 0; i < chunk; ++i) chain[i] = i - 1;
@@ -647,6 +652,13 @@ int firp_prefill_layers(firp_ctx *ctx, int32_t seq, const int32_t *d_prompt, int
 int firp_set_pseudo_masked(firp_ctx *ctx, int32_t masked) {
   if (!ctx) return FIRP_ERR_BAD_ARG;
   ctx->pseudo_masked = masked ? 1 : 0;
+  return FIRP_OK;
+}
+
+int firp_set_pred_prenorm(firp_ctx *ctx, int32_t on) {
+  if (!ctx) return FIRP_ERR_BAD_ARG;
+  ctx->pred_prenorm = on ? 1 : 0;
+  ++ctx->weights_gen;      // cached launch plans depend on it
   return FIRP_OK;
 }
 

@@ -95,7 +95,9 @@ cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Parti
 // every node carries a chain: row s * T + v) as (hi, lo) bf16 planes; one chain: into row s of
 // xp; the GEMM (EPI_PSEUDO) multiplies; launch_gemm_finish(EPI_PSEUDO) sums the partial tiles, adds the bias and
 // stores the k new residual rows (GemmArgs: h_rows = residual stream, pred_b = bias or NULL, R = n_seq).
-void launch_root_split(const Rows &rw, const float *h, int d, bf16 *xp, size_t xp_lo_off, bool pdl, cudaStream_t st);
+// g (may be NULL): gain vector of the pre-norm variant: the planes then hold h * g and the finisher divides by the
+// source row's RMS (GemmArgs::ss of the EPI_PSEUDO finisher)
+void launch_root_split(const Rows &rw, const float *h, const bf16 *g, int d, bf16 *xp, size_t xp_lo_off, bool pdl, cudaStream_t st);
 
 // top-B of every row of logits by (value desc, id asc)
 // Two passes: per 2048-logit segment candidates (scratch cand_*: [R][topb_segments(V)][B]), then the row's top-B.
@@ -206,6 +208,7 @@ struct FusedStep {
   Rows rw;
   int tl[8];                 // insertion layer of each prediction step (non-decreasing)
   bool want_head;            // final norm + lm-head
+  bool prenorm;              // Eq. 3 reads the anchor through the insertion layer's input RMSNorm
   int Rp;                    // rows per activation plane
   int n_hi_max;              // upper bound of the longest committed context among the sequences
   int max_batch;             // of the configuration (sizes the attention scratch)

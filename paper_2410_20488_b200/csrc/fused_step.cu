@@ -69,7 +69,7 @@ struct GemmClass {
 };
 
 struct FusedOp {
-  uint8_t type, cls, planes, pad;   // cls: GEMM class (OP_GEMM / OP_FINISH)
+  uint8_t type, cls, planes, pad;   // cls: GEMM class (OP_GEMM / OP_FINISH); planes: OP_NORM output planes, OP_FINISH(pseudo): 1 = pre-norm variant
   int16_t layer;                    // decoder layer (cache plane of the finisher / attention), -1: none
   int16_t v0, nv;                   // OP_NORM: rows [v0, v0 + nv) of every sequence
   int16_t act;                      // rows alive in this layer
@@ -346,7 +346,7 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
         }
         case OP_ROOT_SPLIT: {
           const unsigned total = (unsigned)(P.rw.n_seq * (P.rw.chains ? P.rw.T : 1) * (P.d >> 2));
-          for (unsigned t = tbase; t < total; t += tstride) root_split_item(P.rw, P.h, P.d, P.xp, (size_t)P.Rp * P.d, t);
+          for (unsigned t = tbase; t < total; t += tstride) root_split_item(P.rw, P.h, (const bf16 *)op.ptr, P.d, P.xp, (size_t)P.Rp * P.d, t);
           break;
         }
         case OP_FINISH: {
@@ -367,6 +367,7 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
           } else {               // EPI_PSEUDO: one token row per source row of Eq. 3
             a.R = P.rw.n_seq * (P.rw.chains ? P.rw.T : 1);
             a.h_rows = P.h; a.pred_b = (const bf16 *)op.ptr; a.pseudo0 = op.aux;
+            if (op.planes) a.ss = P.ss;      // pre-norm variant: divide by the source row's RMS
           }
           const unsigned total = (unsigned)(n_st * a.R * 32);
           for (unsigned t = tbase; t < total; t += tstride) {
@@ -659,9 +660,9 @@ cudaError_t launch_fused_layers(FusedPlan *plan, const FusedStep &fs, bool pdl, 
         if (!class_fits(P.cls[cls], G)) return cudaErrorInvalidConfiguration;
         if (!encode_map(&maps[m_pred0 + n_pred], (const bf16 *)fs.pred_w + (size_t)alive * d * d, (uint64_t)ins * d, d, BM, 0))
           return cudaErrorInvalidValue;
-        add_op(OP_ROOT_SPLIT, 0, 0, j, 0, 0, act, 0, nullptr);
+        add_op(OP_ROOT_SPLIT, 0, 0, j, 0, 0, act, 0, fs.prenorm ? fs.g_attn[j] : nullptr);
         add_gemm(cls, m_pred0 + n_pred, j, act);
-        add_op(OP_FINISH, cls, 0, j, 0, 0, act, alive, fs.pred_b ? (const bf16 *)fs.pred_b + (size_t)alive * d : nullptr);
+        add_op(OP_FINISH, cls, fs.prenorm ? 1 : 0, j, 0, 0, act, alive, fs.pred_b ? (const bf16 *)fs.pred_b + (size_t)alive * d : nullptr);
         add_op(OP_NORM, 0, 3, j, carried, act - carried, act, -1, fs.g_attn[j]);
         ++n_pred;
         alive += ins;

@@ -5,7 +5,8 @@
 //                  row's RMS; ss[r][w] = sum of h[r][c]^2 over the 128 columns of warp w.  The division by
 //                  sqrt(mean(h^2) + eps) commutes with the GEMM that consumes x, so that GEMM's finisher applies it
 //                  to the fp32 sums (it adds the ss[r][*] in a fixed order).  No reduction beyond a warp, no barrier.
-//   root_split_item: the raw fp32 residual rows Eq. 3 reads, as (hi, lo) bf16 planes.
+//   root_split_item: the fp32 residual rows Eq. 3 reads (raw, or times a gain for the pre-norm variant), as (hi, lo)
+//                  bf16 planes.
 #pragma once
 #include "firp_kernels.cuh"
 
@@ -69,14 +70,21 @@ __device__ __forceinline__ void rmsnorm_item(const Rows &rw, int v0, int nv, flo
 }
 
 
-__device__ __forceinline__ void root_split_item(const Rows &rw, const float *h, int d, bf16 *xp, size_t xp_lo_off, unsigned t) {
+// g != NULL: the planes hold h * g (the pre-norm variant of Eq. 3; the division by the row's RMS is applied by
+// the finisher of the GEMM, as for every other normalised operand)
+__device__ __forceinline__ void root_split_item(const Rows &rw, const float *h, const bf16 *g, int d, bf16 *xp, size_t xp_lo_off, unsigned t) {
   const int nvec = d >> 2;
   const int per_seq = rw.chains ? rw.T : 1;                 // source rows per sequence
   if (t >= (unsigned)(rw.n_seq * per_seq * nvec)) return;
   const int m = (int)(t / (unsigned)nvec), idx = (int)(t % (unsigned)nvec);
   const int sq = m / per_seq, v = rw.chains ? m - sq * per_seq : rw.anchor;
   const int s = m;                                          // destination row in xp
-  const float4 a = __ldcg(reinterpret_cast<const float4 *>(h + (size_t)(sq * rw.Ms + v) * d) + idx);
+  float4 a = __ldcg(reinterpret_cast<const float4 *>(h + (size_t)(sq * rw.Ms + v) * d) + idx);
+  if (g != nullptr) {
+    const float2 ga = __bfloat1622float2(reinterpret_cast<const __nv_bfloat162 *>(g)[2 * idx]);
+    const float2 gb = __bfloat1622float2(reinterpret_cast<const __nv_bfloat162 *>(g)[2 * idx + 1]);
+    a.x *= ga.x; a.y *= ga.y; a.z *= gb.x; a.w *= gb.y;
+  }
   const __nv_bfloat162 o01 = __floats2bfloat162_rn(a.x, a.y), o23 = __floats2bfloat162_rn(a.z, a.w);
   const float2 f01 = __bfloat1622float2(o01), f23 = __bfloat1622float2(o23);
   const __nv_bfloat162 l01 = __floats2bfloat162_rn(a.x - f01.x, a.y - f01.y), l23 = __floats2bfloat162_rn(a.z - f23.x, a.w - f23.y);

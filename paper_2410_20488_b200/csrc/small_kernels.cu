@@ -133,14 +133,14 @@ cudaError_t launch_rmsnorm(const Rows &rw, int v0, int v1, float *h, const Parti
 // sequence, untouched by any norm, as (hi, lo) bf16 planes in row s of xp.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-root_split_kernel(Rows rw, const float *h, int d, bf16 *xp, size_t xp_lo_off, int pdl) {
+root_split_kernel(Rows rw, const float *h, const bf16 *g, int d, bf16 *xp, size_t xp_lo_off, int pdl) {
   if (pdl) { griddep_launch(); griddep_wait(); }
-  root_split_item(rw, h, d, xp, xp_lo_off, blockIdx.x * 256 + threadIdx.x);
+  root_split_item(rw, h, g, d, xp, xp_lo_off, blockIdx.x * 256 + threadIdx.x);
 }
 
-void launch_root_split(const Rows &rw, const float *h, int d, bf16 *xp, size_t xp_lo_off, bool pdl, cudaStream_t st) {
+void launch_root_split(const Rows &rw, const float *h, const bf16 *g, int d, bf16 *xp, size_t xp_lo_off, bool pdl, cudaStream_t st) {
   const int threads = rw.n_seq * (rw.chains ? rw.T : 1) * (d >> 2);
-  launch_k(root_split_kernel, dim3((threads + 255) / 256), dim3(256), 0, st, pdl, rw, h, d, xp, xp_lo_off, pdl ? 1 : 0);
+  launch_k(root_split_kernel, dim3((threads + 255) / 256), dim3(256), 0, st, pdl, rw, h, g, d, xp, xp_lo_off, pdl ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------

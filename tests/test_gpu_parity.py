@@ -18,14 +18,16 @@ def torch_cuda():
     return torch
 
 
-def make_pair(shape, weights, max_ctx, masked=False, fused=False, **kw):
+def make_pair(shape, weights, max_ctx, masked=False, fused=False, prenorm=False, **kw):
     """fused=True: steps of at most 48 rows run their decoder layers as one persistent kernel (firp_set_fused)."""
     from paper_2410_20488_b200 import FirpEngine
     eng = FirpEngine(shape, weights, max_ctx=max_ctx, **kw)
     eng.set_fused(fused)
-    orc = oracle.Oracle(shape, weights, max_ctx=max_ctx, n_seq=kw.get("max_batch", 1), masked=masked)
+    orc = oracle.Oracle(shape, weights, max_ctx=max_ctx, n_seq=kw.get("max_batch", 1), masked=masked, prenorm=prenorm)
     if masked:
         eng.set_pseudo_masked(True)
+    if prenorm:
+        eng.set_pred_prenorm(True)
     return eng, orc
 
 
@@ -231,6 +233,22 @@ def test_c1_masked_pseudo_rows(torch_cuda, c1, c1_weights, chains, fused):
     st = lockstep_run(eng, orc, c1, parents, si.prompt(c1, length=40), 4, k=3, l=1 if chains else [0, 1, 1], chains=chains)
     assert st.steps == 4
     eng.close()
+
+
+@pytest.mark.parametrize("fused", [False, True])
+def test_c1_eq3_on_the_normalised_state(torch_cuda, c1, fused):
+    """The variant of Eq. 3 that reads the anchor through the insertion layer's input RMSNorm
+    (firp_set_pred_prenorm), with non-unit gains and a bias: one chain with per-step layers, and a chain under
+    every node; greedy and forced."""
+    shape = si.scaled(c1, L=4, Hkv=2)
+    weights = si.all_weights(shape, gains=True)
+    weights["pred_b"] = si.normal_bf16(shape.seed, si.stream_id("pred_w", 9), shape.k * shape.d, 0.5).reshape(shape.k, shape.d)
+    parents = si.random_tree(6, 12, 3, 3)
+    for chains, layers in ((False, [0, 2, 3]), (True, [1, 1, 2]), (False, 2)):
+        eng, orc = make_pair(shape, weights, 256, prenorm=True, fused=fused, max_tree=16, max_k=3, max_depth=3, max_rows=12 * 4)
+        st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=37), 4, k=3, l=layers, chains=chains, forced_steps=(2,))
+        assert st.steps == 4
+        eng.close()
 
 
 def test_chains_need_the_row_capacity(torch_cuda, c1, c1_weights):
