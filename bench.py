@@ -358,6 +358,8 @@ def run_sweep(args, shape, weights, dev, rank):
     K, W = args.steps, max(args.warmup, 3)
     eng = FirpEngine(shape, weights, max_ctx=max(si.C4_CONTEXTS) + (K + W + 2) * 4 + 128 + 3 + 64, max_tree=128, max_k=3,
                      max_depth=3, device=str(dev))
+    if args.fused >= 0:
+        eng.set_fused(bool(args.fused))
     peaks = {}
     try:
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
@@ -392,7 +394,8 @@ def run_sweep(args, shape, weights, dev, rank):
             gbs = ab["total"] / (ms * 1e-3) / 1e9
             print(json.dumps(dict(workload=pt.name, T=T, k=pt.k, context=n_ctx, steps=K, ms_per_step=ms,
                                   tokens_per_s=(n_end - n_w) / (ms * K * 1e-3), bytes_per_step=ab["total"],
-                                  achieved_gbs=gbs, frac_of_measured_peak=gbs / peak_gbs, frac_of_8tbs=gbs / 8000.0)),
+                                  achieved_gbs=gbs, frac_of_measured_peak=gbs / peak_gbs, frac_of_8tbs=gbs / 8000.0,
+                                  layers_as="one persistent kernel where a step has at most 48 rows" if eng_fused(args) else "one kernel per operation")),
                   flush=True)
     eng.close()
 

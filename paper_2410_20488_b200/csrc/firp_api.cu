@@ -119,7 +119,7 @@ struct firp_ctx {
     dev_status = c.take<int>(1);
     grid_bar = c.take<unsigned>(1);
     attn_ws = c.take<float>(fused_attn_ws_floats(cfg.max_batch, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim));
-    d_maps = c.take<uint8_t>(fused_map_bytes(cfg.n_layers));
+    d_maps = c.take<uint8_t>(2 * fused_map_bytes(cfg.n_layers));   // one set for the step plan, one for the prefill plan
     return align_up(c.off, 256);
   }
 };
@@ -240,8 +240,10 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     fs.x = c->x; fs.xp = c->xp; fs.q = c->q; fs.o = c->o; fs.y = c->y; fs.kv = c->kv;
     fs.kv_seq = c->kv_seq(); fs.kv_layer = c->kv_layer(); fs.kv_plane = c->kv_plane();
     fs.rope = c->meta.rope; fs.pos = c->meta.pos; fs.seq_ids = c->seq_ids; fs.ctx_len = c->ctx_len; fs.mask = c->meta.mask;
-    fs.err = c->dev_status; fs.bar = c->grid_bar; fs.d_maps = c->d_maps;
-    FusedPlan *&plan = ra.prefill_last_row >= 0 ? c->plan_prefill : c->plan_step;
+    // each cached plan owns its tensor maps on the device: a prefill between two steps must not replace the step's
+    const bool for_prefill = ra.prefill_last_row >= 0;
+    fs.err = c->dev_status; fs.bar = c->grid_bar; fs.d_maps = c->d_maps + (for_prefill ? fused_map_bytes(cfg.n_layers) : 0);
+    FusedPlan *&plan = for_prefill ? c->plan_prefill : c->plan_step;
     if (!plan) plan = fused_plan_create();
     FIRP_TIMED(KC_FUSED_LAYERS);
     FIRP_CUDA(c, launch_fused_layers(plan, fs, pdl, st, &nl));

@@ -554,7 +554,7 @@ struct FusedPlan {
 
 FusedPlan *fused_plan_create() { return new FusedPlan(); }
 void fused_plan_destroy(FusedPlan *p) { delete p; }
-size_t fused_map_bytes(int n_layers) { return sizeof(CUtensorMap) * (size_t)(4 * n_layers + 1 + 8 + 4); }
+size_t fused_map_bytes(int n_layers) { return sizeof(CUtensorMap) * (size_t)(4 * n_layers + 1 + 8 + 4 + 1); }   // rounded up to 256 bytes
 size_t fused_attn_ws_floats(int max_batch, int H, int Hkv, int dh) {
   const int Gq = H / Hkv;
   const int groups = max_batch * Hkv * ((48 * Gq + kAttnQRows - 1) / kAttnQRows);

@@ -163,6 +163,18 @@ def test_fused_and_per_operation_paths_agree_and_repeat_bit_for_bit(torch_cuda, 
         assert np.abs(a - b).max() < 1e-4, np.abs(a - b).max()
 
 
+def test_fused_prefill_between_steps_keeps_the_steps_launch_plan_intact(torch_cuda, c1, c1_weights):
+    """Steps and prefill chunks of at most 48 rows both run as the persistent kernel, each with its own cached launch
+    plan and tensor maps on the device.  Prefill, step, prefill a prompt of another length, step again on one
+    engine, each time in lock-step with the oracle (a prefill that replaced the step plan's maps would show here)."""
+    parents = si.tree_template(c1.T)
+    eng, orc = make_pair(c1, c1_weights, 256, fused=True)
+    for length in (20, 33, 7, 45):
+        st = lockstep_run(eng, orc, c1, parents, si.prompt(c1, length=length), 3, forced_steps=(1,))
+        assert st.steps == 3
+    eng.close()
+
+
 def test_a_wait_that_runs_out_is_reported_and_the_context_goes_on(torch_cuda, c1, c1_weights):
     """The time-out path: with the wait limit set to 200 us, firp_selftest_wait enqueues a kernel that waits (with
     the routine the product kernels use) on a barrier nobody arrives on; the wait runs out, the kernel returns, the
