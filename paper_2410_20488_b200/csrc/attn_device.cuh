@@ -3,9 +3,8 @@
 //
 // Every new row attends to the whole committed prefix [0, n) and, among the new rows of its own sequence (cache
 // slots n .. n+rows-1), only to its ancestors and itself; the visibility bits come from the parent array (built
-// once per step).  A work item stages 64-position K and V tiles of its split in shared memory (cp.async; one K and
-// one V buffer, refilled out of phase: the next K tile loads while P V runs, the next V tile while the next Q K^T
-// runs), each warp owns 16 query rows (row x head-of-group for grouped-query attention), S = Q K^T and
+// once per step).  A work item stages 64-position K and V tiles of its split in shared memory (cp.async, double
+// buffered), each warp owns 16 query rows (row x head-of-group for grouped-query attention), S = Q K^T and
 // O += P V run on the tensor cores with an online softmax in fp32.  Queries and probabilities enter the tensor
 // cores as bf16 (hi, lo) pairs accumulated into the same fp32 accumulators, so the only bf16 rounding on this
 // path is the cache's own storage format.
@@ -46,16 +45,16 @@ template <int DH> __device__ __forceinline__ int tile_off(int r, int c) {
   return r * (DH * 2) + (((c & ~7) | ((c ^ r) & 7)) << 4);
 }
 
-// Shared memory of one work item: smem = [2 planes][kAttnQRows][DH] queries, [kAttnTile][DH] keys, [kAttnTile][DH] values
+// Shared memory of one work item: smem = [2 planes][kAttnQRows][DH] queries, [2][kAttnTile][DH] keys, [2][kAttnTile][DH] values
 // (attn_smem_bytes<DH>() bytes, 128-byte aligned); s_mask [kAttnQRows][kMaskWords]; s_row [kAttnQRows].
-template <int DH> __host__ __device__ constexpr int attn_smem_bytes() { return 2 * kAttnQRows * DH * 2 + 2 * kAttnTile * DH * 2; }
+template <int DH> __host__ __device__ constexpr int attn_smem_bytes() { return 2 * kAttnQRows * DH * 2 + 4 * kAttnTile * DH * 2; }
 
 struct AttnCtaSync { static __device__ __forceinline__ void sync() { __syncthreads(); } };
 
 // One work item = (sequence s, kv head, 64-row query block qb, kv split `split` of `nsplits`), computed by the
 // 128 threads tid = 0..127 (4 warps) that share `smem`.  Leaves the split's unnormalised result -- per query
 // row its running max (log2 units) m_out[i], its sum l_out[i] and o_out[i][DH] -- in the given arrays, which may
-// live in shared or in global memory.  o_out may alias the key and value tiles of `smem` (it is written after the last
+// live in shared or in global memory.  o_out may alias the key tiles of `smem` (it is written after the last
 // tile has been consumed).  Sync::sync() is a barrier over exactly those 128 threads.
 template <int DH, typename Sync>
 __device__ __forceinline__ void attn_split_item(const AttnArgs &a, uint8_t *smem, uint32_t (*s_mask)[kMaskWords], int *s_row,
@@ -65,8 +64,8 @@ __device__ __forceinline__ void attn_split_item(const AttnArgs &a, uint8_t *smem
   constexpr int TILE_BYTES = kAttnTile * DH * 2;
   uint8_t *sQ = smem;                               // [2 planes][kAttnQRows][DH]
   constexpr int Q_BYTES = kAttnQRows * DH * 2;
-  uint8_t *sK = sQ + 2 * Q_BYTES;                   // [kAttnTile][DH]
-  uint8_t *sV = sK + TILE_BYTES;                    // [kAttnTile][DH]
+  uint8_t *sK = sQ + 2 * Q_BYTES;                   // [2][kAttnTile][DH]
+  uint8_t *sV = sK + 2 * TILE_BYTES;                // [2][kAttnTile][DH]
   const int warp = tid >> 5, lane = tid & 31;
   const int G = a.H / a.Hkv;
   const int qrows_total = a.rows_active * G;
@@ -89,20 +88,17 @@ __device__ __forceinline__ void attn_split_item(const AttnArgs &a, uint8_t *smem
   const bf16 *kbase = a.kcache + (size_t)slot * a.seq_stride + (size_t)kvh * DH;
   const bf16 *vbase = kbase + a.kv_stride;
   const size_t pos_stride = (size_t)a.Hkv * DH;
-  auto load_tile = [&](uint8_t *dst, const bf16 *src_base, int t) {
+  auto load_kv = [&](int buf, int t) {
     const int p0 = t * kAttnTile;
     for (int ch = tid; ch < kAttnTile * CH; ch += kAttnThreads) {
       const int i = ch / CH, c = ch % CH;
       const bool valid = (p0 + i) < kv_len;
       const size_t off = (size_t)(p0 + i) * pos_stride + c * 8;
-      cp_async_16(attn_smem_u32(dst + tile_off<DH>(i, c)), valid ? src_base + off : src_base, valid);
+      cp_async_16(attn_smem_u32(sK + buf * TILE_BYTES + tile_off<DH>(i, c)), valid ? kbase + off : kbase, valid);
+      cp_async_16(attn_smem_u32(sV + buf * TILE_BYTES + tile_off<DH>(i, c)), valid ? vbase + off : vbase, valid);
     }
   };
-  // cp.async groups alternate K_t, V_t, K_t+1, V_t+1, ...: before Q K^T of tile t everything but the newest group
-  // (V_t) has to be complete, before P V everything but the newest group (K_t+1)
-  if (t0 < t1) load_tile(sK, kbase, t0);
-  cp_async_commit();                                // queries + K of the first tile
-  if (t0 < t1) load_tile(sV, vbase, t0);
+  if (t0 < t1) load_kv(0, t0);
   cp_async_commit();
   // query rows of this block: qr -> (tree row v = qr / G, head = kvh * G + qr % G), and their visibility words
   for (int i = tid; i < kAttnQRows; i += kAttnThreads) {
@@ -121,9 +117,12 @@ __device__ __forceinline__ void attn_split_item(const AttnArgs &a, uint8_t *smem
   for (int i = 0; i < DH / 8; ++i) { o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f; }
 
   for (int t = t0; t < t1; ++t) {
-    cp_async_wait<1>();                             // K_t (and the queries) have landed
+    const int buf = (t - t0) & 1;
+    if (t + 1 < t1) load_kv(buf ^ 1, t + 1);
+    cp_async_commit();
+    cp_async_wait<1>();
     Sync::sync();
-    const uint8_t *kt = sK, *vt = sV;
+    const uint8_t *kt = sK + buf * TILE_BYTES, *vt = sV + buf * TILE_BYTES;
     // S = Q K^T over the 64 positions of the tile
     float sc[kAttnTile / 8][4];
 #pragma unroll
@@ -147,9 +146,6 @@ __device__ __forceinline__ void attn_split_item(const AttnArgs &a, uint8_t *smem
         mma_bf16(sc[2 * p + 1], ql, b2, b3);
       }
     }
-    Sync::sync();                                   // every warp has read K_t: its buffer takes the next K tile
-    if (t + 1 < t1) load_tile(sK, kbase, t + 1);
-    cp_async_commit();
     // mask, scale, online softmax (rows g and g+8 of this warp's 16)
     const int p0 = t * kAttnTile;
     const bool need_mask = (p0 + kAttnTile > n);
@@ -215,8 +211,6 @@ __device__ __forceinline__ void attn_split_item(const AttnArgs &a, uint8_t *smem
       pl[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(e2 - f23.x, e3 - f23.y);
     }
     // O += P V
-    cp_async_wait<1>();                             // V_t has landed (K_t+1 may still be on its way)
-    Sync::sync();
 #pragma unroll
     for (int j = 0; j < kAttnTile / 16; ++j) {
 #pragma unroll
@@ -230,9 +224,7 @@ __device__ __forceinline__ void attn_split_item(const AttnArgs &a, uint8_t *smem
         mma_bf16(o_acc[2 * d2 + 1], pl[j], b2, b3);
       }
     }
-    Sync::sync();                                   // every warp has read V_t: its buffer takes the next V tile
-    if (t + 1 < t1) load_tile(sV, vbase, t + 1);
-    cp_async_commit();
+    Sync::sync();
   }
   cp_async_wait<0>();
 

@@ -43,9 +43,9 @@ constexpr int BM = 128, TM = 2, BK = kGemmBK;
 constexpr int W_TILE = BM * 128, W_STAGE = TM * W_TILE;   // one unit: 2 x 128 weight rows x 64 k = 32 KB
 constexpr int kFThreads = 352;                            // 11 warps: 3 single-thread roles + 8 worker warps
 constexpr int kWorkers = 256;
-constexpr int SW = 5;                                     // weight stages (160 KB in flight per SM)
-constexpr int SX = 3;                                     // activation stages
-constexpr int kRegion = 64 * 1024;                        // activation ring, reused by the attention phases
+constexpr int SW = 4;                                     // weight stages (128 KB in flight per SM; a fifth changed nothing)
+constexpr int SX = 4;                                     // activation stages
+constexpr int kRegion = 96 * 1024;                        // activation ring, reused by the attention phases
 constexpr int kSmallBytes = kAttnQRows * kMaskWords * 4 + kAttnQRows * 4;   // s_mask, s_row
 constexpr int kBarBytes = 256;
 constexpr int kFusedSmem = SW * W_STAGE + kRegion + kSmallBytes + kBarBytes;
