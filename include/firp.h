@@ -95,7 +95,8 @@ void firp_destroy(firp_ctx *ctx);
 const char *firp_last_error(const firp_ctx *ctx);
 
 /* Bytes of device memory the caller must provide: scratch workspace and bf16 KV cache
- * (layout [seq][layer][K|V][position][kv_head][head_dim]). */
+ * (layout [layer][K|V][row][kv_head][head_dim] with row = slot * max_ctx + position, or, with a page table
+ * (firp_set_kv_pages), row = page * 64 + position % 64). */
 size_t firp_workspace_bytes(const firp_ctx *ctx);
 size_t firp_kv_bytes(const firp_ctx *ctx);
 
@@ -180,6 +181,16 @@ int firp_step_chains(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const
  * positions are unchanged.  Applies to every later firp_prefill* / firp_step* call of the context.
  */
 int firp_set_pseudo_masked(firp_ctx *ctx, int32_t masked);
+
+/*
+ * Non-contiguous KV cache (the paper's loop, Section 3.4, only needs the accepted prefix to be addressable; how
+ * it is stored is the serving system's business).  page_table: HOST [max_batch][max_ctx / 64]; entry
+ * [slot][p] is the physical page (0 .. max_batch * max_ctx / 64 - 1, each used once) that holds positions
+ * 64 p .. 64 p + 63 of that slot; inside a (layer, K|V) plane of the cache a page is 64 consecutive rows.
+ * The table is checked and copied into the workspace (synchronises `stream`); NULL goes back to contiguous rows.
+ * max_ctx must be a multiple of 64.  Cache contents are not moved: set the table before the slot is prefilled.
+ */
+int firp_set_kv_pages(firp_ctx *ctx, const int32_t *page_table, void *stream);
 
 /*
  * What Eq. 3 reads (Section 3.3 writes W_i h^{t_i} + b_i and does not say whether h^{t_i} is taken before or

@@ -46,7 +46,7 @@ EXPORTS = ("firp_create", "firp_destroy", "firp_last_error", "firp_workspace_byt
            "firp_bind_buffers", "firp_init_weights", "firp_prefill", "firp_step", "firp_kv_commit",
            "firp_context_len", "firp_set_context_len", "firp_last_launch_count", "firp_profile_enable",
            "firp_profile_read", "firp_kernel_class_name", "firp_topb_static", "firp_prefill_layers", "firp_step_layers", "firp_step_chains", "firp_set_pseudo_masked",
-           "firp_set_fused", "firp_set_wait_limit_us", "firp_selftest_wait", "firp_set_pred_prenorm")
+           "firp_set_fused", "firp_set_wait_limit_us", "firp_selftest_wait", "firp_set_pred_prenorm", "firp_set_kv_pages")
 
 
 def lib_path() -> str:
@@ -80,6 +80,7 @@ def load_library():
     lib.firp_step_chains.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp, ctypes.POINTER(StepOutC), vp]
     lib.firp_set_pseudo_masked.argtypes = [vp, i32]
     lib.firp_set_fused.argtypes = [vp, i32]
+    lib.firp_set_kv_pages.argtypes = [vp, vp, vp]
     lib.firp_set_pred_prenorm.argtypes = [vp, i32]
     lib.firp_set_wait_limit_us.argtypes = [vp, ctypes.c_int64]
     lib.firp_selftest_wait.argtypes = [vp, vp]
@@ -203,6 +204,13 @@ def firp_set_pred_prenorm(ctx, on: bool):
     _check(ctx, load_library().firp_set_pred_prenorm(ctx, int(bool(on))))
 
 
+def firp_set_kv_pages(ctx, page_table, stream: int = 0):
+    """page_table: host int32 [max_batch][max_ctx / 64] (physical page of every logical page), or None for
+    contiguous rows."""
+    arr, ptr = _host_i32(page_table)
+    _check(ctx, load_library().firp_set_kv_pages(ctx, ptr, stream))
+
+
 def firp_set_fused(ctx, on: bool):
     """Run the layers of small steps as one persistent kernel (default) or one kernel per operation."""
     _check(ctx, load_library().firp_set_fused(ctx, int(bool(on))))
@@ -300,6 +308,7 @@ class FirpEngine:
                             vocab=s.V, rms_eps=s.eps, rope_theta=s.theta, max_batch=max_batch, max_ctx=max_ctx,
                             max_tree=max_tree, max_k=max_k, max_depth=max_depth, top_b=top_b, max_rows=max_rows)
         self.S, self.B = max_depth + 1, top_b
+        self.page_table = None
         self.ctx = firp_create(self.cfg)
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(firp_workspace_bytes(self.ctx), dtype=torch.uint8, device=self.device)
@@ -364,6 +373,11 @@ class FirpEngine:
 
     def set_pred_prenorm(self, on: bool):
         firp_set_pred_prenorm(self.ctx, on)
+
+    def set_kv_pages(self, page_table):
+        """Scatter the cache over pages of 64 positions (None: contiguous); remembered for the test harness."""
+        firp_set_kv_pages(self.ctx, page_table, self.stream)
+        self.page_table = None if page_table is None else np.ascontiguousarray(page_table, np.int32).reshape(self.cfg.max_batch, -1)
 
     def set_fused(self, on: bool):
         firp_set_fused(self.ctx, on)

@@ -85,15 +85,16 @@ __device__ __forceinline__ void attn_split_item(const AttnArgs &a, uint8_t *smem
   // balanced ranges; a remainder goes to the first splits, the last one owns the (slower) masked tiles
   const int t0 = (split * tiles_total + nsplits - 1) / nsplits, t1 = ((split + 1) * tiles_total + nsplits - 1) / nsplits;
 
-  const bf16 *kbase = a.kcache + (size_t)slot * a.seq_stride + (size_t)kvh * DH;
+  const bf16 *kbase = a.kcache + (size_t)kvh * DH;       // row 0 of the plane; a tile's rows follow from kv_row()
   const bf16 *vbase = kbase + a.kv_stride;
   const size_t pos_stride = (size_t)a.Hkv * DH;
   auto load_kv = [&](int buf, int t) {
     const int p0 = t * kAttnTile;
+    const size_t row0 = kv_row(a.pages, slot, p0, a.max_ctx);      // the tile lies inside one page
     for (int ch = tid; ch < kAttnTile * CH; ch += kAttnThreads) {
       const int i = ch / CH, c = ch % CH;
       const bool valid = (p0 + i) < kv_len;
-      const size_t off = (size_t)(p0 + i) * pos_stride + c * 8;
+      const size_t off = (row0 + i) * pos_stride + c * 8;
       cp_async_16(attn_smem_u32(sK + buf * TILE_BYTES + tile_off<DH>(i, c)), valid ? kbase + off : kbase, valid);
       cp_async_16(attn_smem_u32(sV + buf * TILE_BYTES + tile_off<DH>(i, c)), valid ? vbase + off : vbase, valid);
     }

@@ -114,7 +114,7 @@ __device__ __forceinline__ void qkv_finish_item(const Partials &p, const GemmArg
     const int slot = a.seq_ids[s];
     const int pos = a.pos[s * a.rw.Ms] + v;        // committed length (position of the root row) + row index
     if (pos < a.max_ctx) {
-      bf16 *dst = a.kcache + (size_t)slot * a.seq_stride + (is_v ? a.kv_stride : 0) + ((size_t)pos * a.Hkv + kvh) * a.dh + c;
+      bf16 *dst = a.kcache + (is_v ? a.kv_stride : 0) + (kv_row(a.pages, slot, pos, a.max_ctx) * a.Hkv + kvh) * a.dh + c;
       *reinterpret_cast<uint2 *>(dst) = round4(x1);
       *reinterpret_cast<uint2 *>(dst + half) = round4(x2);
     }

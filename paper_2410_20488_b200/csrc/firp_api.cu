@@ -60,6 +60,10 @@ struct firp_ctx {
   unsigned *grid_bar = nullptr;         // arrival counter of the fused kernel's grid barrier
   float *attn_ws = nullptr;             // partial results of its attention splits
   uint8_t *d_maps = nullptr;            // its tensor maps
+  int32_t *d_pages = nullptr;           // page table of the KV cache (device copy), [max_batch][pages_per_seq]
+  bool paged = false;
+  int pages_per_seq() const { return (cfg.max_ctx + kKvPage - 1) / kKvPage; }
+  KvPages pages() const { return KvPages{paged ? d_pages : nullptr, pages_per_seq()}; }
   // weights
   firp_weights w{};
   std::vector<const void *> wqkv, wo, wgu, wd, g_attn, g_mlp;
@@ -80,9 +84,10 @@ struct firp_ctx {
   int pseudo_masked = 0;     // Section 4.3 "Masked": pseudo rows do not see one another
   int pred_prenorm = 0;      // Eq. 3 reads the anchor through the insertion layer's input RMSNorm
 
-  size_t kv_plane() const { return (size_t)cfg.max_ctx * cfg.n_kv_heads * cfg.head_dim; }
+  // cache layout [layer][K|V][row][kv_head][head_dim]; row = slot * max_ctx + position, or through the page table
+  size_t kv_seq() const { return (size_t)cfg.max_ctx * cfg.n_kv_heads * cfg.head_dim; }      // elements per slot of a plane
+  size_t kv_plane() const { return (size_t)cfg.max_batch * kv_seq(); }                        // one K or V plane of a layer
   size_t kv_layer() const { return 2 * kv_plane(); }
-  size_t kv_seq() const { return (size_t)cfg.n_layers * kv_layer(); }
 
   size_t carve(void *base) {
     Carver c{reinterpret_cast<uint8_t *>(base), 0};
@@ -119,6 +124,7 @@ struct firp_ctx {
     dev_status = c.take<int>(1);
     grid_bar = c.take<unsigned>(1);
     attn_ws = c.take<float>(fused_attn_ws_floats(cfg.max_batch, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim));
+    d_pages = c.take<int32_t>((size_t)cfg.max_batch * pages_per_seq());
     d_maps = c.take<uint8_t>(2 * fused_map_bytes(cfg.n_layers));   // one set for the step plan, one for the prefill plan
     return align_up(c.off, 256);
   }
@@ -238,7 +244,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     fs.g_final = c->w.g_final; fs.lm_head = c->w.lm_head; fs.pred_w = c->w.pred_w; fs.pred_b = c->w.pred_b;
     fs.h = c->h; fs.ws = c->gemm_ws; fs.ss = c->ss; fs.logits = ra.logits_dst; fs.attn_ws = c->attn_ws;
     fs.x = c->x; fs.xp = c->xp; fs.q = c->q; fs.o = c->o; fs.y = c->y; fs.kv = c->kv;
-    fs.kv_seq = c->kv_seq(); fs.kv_layer = c->kv_layer(); fs.kv_plane = c->kv_plane();
+    fs.kv_seq = c->kv_seq(); fs.kv_layer = c->kv_layer(); fs.kv_plane = c->kv_plane(); fs.pages = c->pages();
     fs.rope = c->meta.rope; fs.pos = c->meta.pos; fs.seq_ids = c->seq_ids; fs.ctx_len = c->ctx_len; fs.mask = c->meta.mask;
     // each cached plan owns its tensor maps on the device: a prefill between two steps must not replace the step's
     const bool for_prefill = ra.prefill_last_row >= 0;
@@ -308,7 +314,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       set_next(g, 0, EPI_RESIDUAL, c->wo[j], d, nq);
       g.planes = 3;   // keys and values are rounded to bf16 for the cache: their inputs carry ~24 mantissa bits
       g.rope = c->meta.rope; g.seq_ids = c->seq_ids; g.ctx_len = c->ctx_len; g.pos = c->meta.pos;
-      g.q = c->q; g.q_lo_off = Rp * nq; g.kcache = kplane; g.seq_stride = c->kv_seq(); g.kv_stride = c->kv_plane(); g.max_ctx = cfg.max_ctx;
+      g.q = c->q; g.q_lo_off = Rp * nq; g.kcache = kplane; g.seq_stride = c->kv_seq(); g.kv_stride = c->kv_plane(); g.max_ctx = cfg.max_ctx; g.pages = c->pages();
       Partials p = pending;
       { FIRP_TIMED(KC_GEMM_QKV);
         FIRP_CUDA(c, launch_gemm_tc(EPI_QKV_ROPE, g, pdl, st, &p.sk)); ++nl; }
@@ -318,7 +324,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     {
       AttnArgs a{};
       a.rw = rw; a.rows_active = act; a.H = H; a.Hkv = Hkv; a.dh = dh;
-      a.q = c->q; a.q_lo_off = Rp * nq; a.kcache = kplane; a.seq_stride = c->kv_seq(); a.kv_stride = c->kv_plane(); a.max_ctx = cfg.max_ctx;
+      a.q = c->q; a.q_lo_off = Rp * nq; a.kcache = kplane; a.seq_stride = c->kv_seq(); a.kv_stride = c->kv_plane(); a.max_ctx = cfg.max_ctx; a.pages = c->pages();
       a.seq_ids = c->seq_ids; a.ctx_len = c->ctx_len; a.pos = c->meta.pos; a.mask = c->meta.mask;
       const int tiles = (ra.n_hi_max + act + kAttnTile - 1) / kAttnTile;
       const int G = H / Hkv, qblocks = (act * G + 63) / 64;
@@ -435,7 +441,7 @@ const char *firp_last_error(const firp_ctx *ctx) { return ctx ? ctx->err.c_str()
 size_t firp_workspace_bytes(const firp_ctx *ctx) { return ctx ? ctx->ws_bytes : 0; }
 
 size_t firp_kv_bytes(const firp_ctx *ctx) {
-  return ctx ? (size_t)ctx->cfg.max_batch * ctx->kv_seq() * sizeof(bf16) : 0;
+  return ctx ? (size_t)ctx->cfg.n_layers * ctx->kv_layer() * sizeof(bf16) : 0;
 }
 
 int firp_bind_buffers(firp_ctx *ctx, void *workspace, void *kv_cache, void *stream) {
@@ -664,6 +670,26 @@ int firp_set_pred_prenorm(firp_ctx *ctx, int32_t on) {
   return FIRP_OK;
 }
 
+int firp_set_kv_pages(firp_ctx *ctx, const int32_t *page_table, void *stream) {
+  if (!ctx) return FIRP_ERR_BAD_ARG;
+  if (!ctx->bound) return fail(ctx, FIRP_ERR_STATE, "firp_bind_buffers has not been called");
+  cudaStream_t st = (cudaStream_t)stream;
+  ++ctx->weights_gen;                      // cached launch plans carry the table pointer
+  if (!page_table) { ctx->paged = false; return FIRP_OK; }
+  const int pps = ctx->pages_per_seq(), total = ctx->cfg.max_batch * pps;
+  if (ctx->cfg.max_ctx % kKvPage) return fail(ctx, FIRP_ERR_BAD_ARG, "a paged cache needs max_ctx to be a multiple of %d", kKvPage);
+  std::vector<char> seen(total, 0);
+  for (int i = 0; i < total; ++i) {
+    const int32_t pg = page_table[i];
+    if (pg < 0 || pg >= total || seen[pg]) return fail(ctx, FIRP_ERR_BAD_ARG, "page table entry %d: page %d out of range or used twice", i, pg);
+    seen[pg] = 1;
+  }
+  FIRP_CUDA(ctx, cudaMemcpyAsync(ctx->d_pages, page_table, sizeof(int32_t) * total, cudaMemcpyHostToDevice, st));
+  FIRP_CUDA(ctx, cudaStreamSynchronize(st));
+  ctx->paged = true;
+  return FIRP_OK;
+}
+
 int firp_set_fused(firp_ctx *ctx, int32_t on) {
   if (!ctx) return FIRP_ERR_BAD_ARG;
   ctx->use_fused = on != 0;
@@ -696,6 +722,7 @@ int firp_kv_commit(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const i
   const int S = ctx->S;
   CommitArgs a{};
   a.kv = ctx->kv; a.seq_stride = ctx->kv_seq(); a.layer_stride = ctx->kv_layer(); a.kv_stride = ctx->kv_plane();
+  a.max_ctx = ctx->cfg.max_ctx; a.pages = ctx->pages();
   a.n_layers = ctx->cfg.n_layers; a.nkv = ctx->cfg.n_kv_heads * ctx->cfg.head_dim; a.seq_ids = ctx->seq_ids;
   a.S = S; a.ctx_len = ctx->ctx_len;
   ctx->launches = 0;

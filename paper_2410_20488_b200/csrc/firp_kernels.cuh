@@ -29,6 +29,16 @@ struct Rows {
   int masked;  // != 0: a pseudo row sees no other pseudo row (the "Masked" ablation of Section 4.3)
 };
 
+// Rows of the KV cache.  A (layer, K|V) plane holds max_batch * max_ctx rows of Hkv * dh elements.  Without a
+// page table position `pos` of slot `slot` is row slot * max_ctx + pos; with one (pages of kKvPage positions,
+// table[slot * pages_per_seq + pos / kKvPage] = physical page) it is row page * kKvPage + pos % kKvPage.
+constexpr int kKvPage = 64;               // = kAttnTile: an attention tile never straddles two pages
+struct KvPages { const int32_t *table; int pages_per_seq; };
+__device__ __forceinline__ size_t kv_row(const KvPages &pg, int slot, int pos, int max_ctx) {
+  if (pg.table == nullptr) return (size_t)slot * max_ctx + pos;
+  return (size_t)pg.table[slot * pg.pages_per_seq + pos / kKvPage] * kKvPage + (pos % kKvPage);
+}
+
 constexpr int kGemmMaxCtas = 192;         // scratch slots are provided for this many CTAs
 constexpr int kGemmSlots = 3;             // partial tiles (segments) per CTA
 
@@ -134,6 +144,7 @@ struct CommitArgs {
   const int32_t *path_len;  // [n_seq] device
   int S;
   int32_t *ctx_len;         // [max_batch] device
+  int max_ctx; KvPages pages;
 };
 void launch_commit(int n_seq, const CommitArgs &a, bool pdl, cudaStream_t st);
 void launch_advance_ctx(int n_seq, const int32_t *seq_ids, int32_t *ctx_len, int amount, bool pdl, cudaStream_t st);
@@ -166,7 +177,8 @@ struct GemmArgs {
   int H, Hkv, dh;
   const float2 *rope; const int32_t *seq_ids; const int32_t *ctx_len; const int32_t *pos;   // pos[R]: row positions
   bf16 *q; size_t q_lo_off;      // [R][H*dh] hi plane, lo plane
-  bf16 *kcache; size_t seq_stride, kv_stride; int max_ctx;  // kcache points at this layer's K plane of sequence slot 0
+  bf16 *kcache; size_t seq_stride, kv_stride; int max_ctx;  // kcache points at this layer's K plane (row 0)
+  KvPages pages;
   // EPI_SWIGLU: y[R][F], N = 2F
   bf16 *y; size_t y_lo_off; int F;
   // EPI_LOGITS: logits[R][N]
@@ -191,6 +203,7 @@ struct AttnArgs {
   const bf16 *q; size_t q_lo_off;   // [R][H*dh] rotated queries, hi and lo planes
   const bf16 *kcache;         // this layer's K plane of slot 0; V plane = kcache + kv_stride
   size_t seq_stride, kv_stride; int max_ctx;
+  KvPages pages;
   const int32_t *seq_ids, *ctx_len;
   const int32_t *pos;         // [R] absolute position of every row (row 0 of a sequence: its committed length)
   const uint32_t *mask;       // [R][kMaskWords]
@@ -221,6 +234,7 @@ struct FusedStep {
   float *h, *ws, *ss, *logits, *attn_ws;
   bf16 *x, *xp, *q, *o, *y, *kv;
   size_t kv_seq, kv_layer, kv_plane;
+  KvPages pages;
   const float2 *rope; const int32_t *pos, *seq_ids, *ctx_len; const uint32_t *mask;
   int *err; unsigned *bar;   // status word; arrival counter of the grid barrier (zero before the launch)
   void *d_maps;              // device room for the tensor maps: fused_map_bytes(L) bytes, 128-byte aligned

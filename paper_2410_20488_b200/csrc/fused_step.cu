@@ -84,6 +84,7 @@ struct FusedParams {
   float *h, *ws, *ss, *logits, *attn_ws;
   bf16 *x, *xp, *q, *o, *y, *kv;
   size_t kv_seq, kv_layer, kv_plane;
+  KvPages pages;
   const float2 *rope; const int32_t *pos, *seq_ids, *ctx_len; const uint32_t *mask;
   int *err; unsigned *bar; unsigned long long wait_ns;
   const CUtensorMap *maps;
@@ -359,7 +360,7 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
           if (c.epi == EPI_QKV_ROPE) {
             a.ss = P.ss; a.H = P.H; a.Hkv = P.Hkv; a.dh = P.dh; a.rope = P.rope; a.seq_ids = P.seq_ids; a.pos = P.pos;
             a.q = P.q; a.q_lo_off = (size_t)P.Rp * nq; a.kcache = P.kv + (size_t)op.layer * P.kv_layer;
-            a.seq_stride = P.kv_seq; a.kv_stride = P.kv_plane; a.max_ctx = P.max_ctx;
+            a.seq_stride = P.kv_seq; a.kv_stride = P.kv_plane; a.max_ctx = P.max_ctx; a.pages = P.pages;
           } else if (c.epi == EPI_SWIGLU) {
             a.ss = P.ss; a.y = P.y; a.y_lo_off = (size_t)P.Rp * P.F; a.F = P.F;
           } else if (c.epi == EPI_LOGITS) {
@@ -382,7 +383,7 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
           AttnArgs a{};
           a.rw = P.rw; a.rows_active = op.act; a.H = P.H; a.Hkv = P.Hkv; a.dh = P.dh;
           a.q = P.q; a.q_lo_off = (size_t)P.Rp * nq; a.kcache = P.kv + (size_t)op.layer * P.kv_layer;
-          a.seq_stride = P.kv_seq; a.kv_stride = P.kv_plane; a.max_ctx = P.max_ctx;
+          a.seq_stride = P.kv_seq; a.kv_stride = P.kv_plane; a.max_ctx = P.max_ctx; a.pages = P.pages;
           a.seq_ids = P.seq_ids; a.ctx_len = P.ctx_len; a.pos = P.pos; a.mask = P.mask; a.splits = P.splits;
           const int Gq = P.H / P.Hkv;
           const int qblocks = (op.act * Gq + kAttnQRows - 1) / kAttnQRows;
@@ -606,7 +607,7 @@ cudaError_t launch_fused_layers(FusedPlan *plan, const FusedStep &fs, bool pdl, 
     P = FusedParams{};
     P.rw = rw; P.d = d; P.H = H; P.Hkv = Hkv; P.dh = dh; P.F = F; P.V = sh.V; P.Rp = fs.Rp; P.max_ctx = sh.max_ctx; P.eps = sh.eps;
     P.h = fs.h; P.ws = fs.ws; P.ss = fs.ss; P.attn_ws = fs.attn_ws; P.x = fs.x; P.xp = fs.xp; P.q = fs.q; P.o = fs.o; P.y = fs.y;
-    P.kv = fs.kv; P.kv_seq = fs.kv_seq; P.kv_layer = fs.kv_layer; P.kv_plane = fs.kv_plane;
+    P.kv = fs.kv; P.kv_seq = fs.kv_seq; P.kv_layer = fs.kv_layer; P.kv_plane = fs.kv_plane; P.pages = fs.pages;
     P.rope = fs.rope; P.pos = fs.pos; P.seq_ids = fs.seq_ids; P.ctx_len = fs.ctx_len; P.mask = fs.mask;
     P.err = fs.err; P.bar = fs.bar; P.maps = reinterpret_cast<const CUtensorMap *>(fs.d_maps);
     // tensor maps: 4 per layer, lm-head, one per Eq. 3 GEMM, then the activations x, xp, o, y

@@ -322,17 +322,21 @@ __global__ void __launch_bounds__(128) commit_kernel(CommitArgs a, int pdl) {
   const int n = a.ctx_len[slot];
   const int len = min(a.path_len[s], kMaxPath);
   const int32_t *path = a.path + (size_t)s * a.S;
-  bf16 *base = a.kv + (size_t)slot * a.seq_stride + (size_t)(plane >> 1) * a.layer_stride +
-               (size_t)(plane & 1) * a.kv_stride + (size_t)n * a.nkv;
+  bf16 *base = a.kv + (size_t)(plane >> 1) * a.layer_stride + (size_t)(plane & 1) * a.kv_stride;
   const int nvec = a.nkv >> 3;
+  size_t src_row[kMaxPath], dst_row[kMaxPath];
+#pragma unroll
+  for (int j = 0; j < kMaxPath; ++j) {
+    if (j < len) { src_row[j] = kv_row(a.pages, slot, n + path[j], a.max_ctx); dst_row[j] = kv_row(a.pages, slot, n + j, a.max_ctx); }
+  }
   for (int c = threadIdx.x; c < nvec; c += blockDim.x) {
     uint4 tmp[kMaxPath];
 #pragma unroll
     for (int j = 0; j < kMaxPath; ++j)
-      if (j < len) tmp[j] = reinterpret_cast<const uint4 *>(base + (size_t)path[j] * a.nkv)[c];
+      if (j < len) tmp[j] = reinterpret_cast<const uint4 *>(base + src_row[j] * a.nkv)[c];
 #pragma unroll
     for (int j = 0; j < kMaxPath; ++j)
-      if (j < len && path[j] != j) reinterpret_cast<uint4 *>(base + (size_t)j * a.nkv)[c] = tmp[j];
+      if (j < len && path[j] != j) reinterpret_cast<uint4 *>(base + dst_row[j] * a.nkv)[c] = tmp[j];
   }
 }
 

@@ -144,13 +144,21 @@ def gpu_outputs(out, s, T, k):
                 next_tokens=out.next_tree_tokens[s].cpu().numpy())
 
 
+def cache_row(engine, seq, pos):
+    """Row of cache position `pos` of slot `seq` inside a (layer, K|V) plane: contiguous, or through the page table
+    the engine was given (64 positions per page)."""
+    table = getattr(engine, "page_table", None)
+    if table is None:
+        return seq * engine.cfg.max_ctx + pos
+    return int(table[seq, pos // 64]) * 64 + pos % 64
+
+
 def read_gpu_cache(engine, seq, layer, which, slot):
     import torch
     s = engine.shape
     cfg = engine.cfg
     kvt = engine.kv.view(torch.bfloat16)
-    plane = cfg.max_ctx * s.n_kv
-    off = ((seq * s.L + layer) * 2 + which) * plane + slot * s.n_kv
+    off = ((layer * 2 + which) * cfg.max_batch * cfg.max_ctx + cache_row(engine, seq, slot)) * s.n_kv
     return kvt[off: off + s.n_kv].float().cpu().numpy()
 
 
@@ -170,10 +178,19 @@ def write_gpu_cache(engine, seq, layer, which, slot0, rows_bits):
     import torch
     s, cfg = engine.shape, engine.cfg
     kvt = engine.kv.view(torch.int16)
-    plane = cfg.max_ctx * s.n_kv
-    off = ((seq * s.L + layer) * 2 + which) * plane + slot0 * s.n_kv
-    src = torch.from_numpy(np.ascontiguousarray(rows_bits, np.uint16).view(np.int16).reshape(-1))
-    kvt[off: off + src.numel()].copy_(src.to(engine.device))
+    src = torch.from_numpy(np.ascontiguousarray(rows_bits, np.uint16).view(np.int16)).to(engine.device)
+    count = src.shape[0]
+    plane0 = (layer * 2 + which) * cfg.max_batch * cfg.max_ctx
+    if getattr(engine, "page_table", None) is None:          # contiguous rows
+        off = (plane0 + seq * cfg.max_ctx + slot0) * s.n_kv
+        kvt[off: off + src.numel()].copy_(src.reshape(-1))
+    else:                                                     # scattered through the page table, page by page
+        pos = slot0
+        while pos < slot0 + count:
+            n = min(64 - pos % 64, slot0 + count - pos)
+            off = (plane0 + cache_row(engine, seq, pos)) * s.n_kv
+            kvt[off: off + n * s.n_kv].copy_(src[pos - slot0: pos - slot0 + n].reshape(-1))
+            pos += n
 
 
 def seed_prefix(engine, orc, shape, seq, n):

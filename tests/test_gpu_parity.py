@@ -263,6 +263,38 @@ def test_c1_eq3_on_the_normalised_state(torch_cuda, c1, fused):
         eng.close()
 
 
+@pytest.mark.parametrize("fused", [False, True])
+def test_c1_paged_cache(torch_cuda, c1, fused):
+    """The KV cache scattered over pages of 64 positions through a shuffled page table (firp_set_kv_pages): two
+    sequences stepped together, contexts that start just below a page boundary so that the tree rows of a step
+    straddle two pages and the forced-accept commits compact rows from one page into another; every step in
+    lock-step with the oracle (which knows nothing of pages), committed cache rows compared through the table."""
+    from lockstep import lockstep_run_batch, lockstep_steps_batch
+    from paper_2410_20488_b200 import FirpError, binding
+    shape = si.scaled(c1, Hkv=2)
+    weights = si.all_weights(shape, gains=True)
+    parents = si.tree_template(shape.T)
+    eng, orc = make_pair(shape, weights, 256, max_batch=2, fused=fused)
+    pages = 2 * 256 // 64
+    table = si.uniform_i32(5, si.stream_id("tokens", 77), pages, 0, 1 << 20).argsort().astype(np.int32).reshape(2, -1)
+    assert sorted(table.reshape(-1).tolist()) == list(range(pages)) and not np.array_equal(table.reshape(-1), np.arange(pages))
+    bad = table.copy(); bad[0, 0] = bad[1, 1]
+    with pytest.raises(FirpError) as e:
+        eng.set_kv_pages(bad)                                    # a page used twice is refused
+    assert e.value.code == binding.FIRP_ERR_BAD_ARG
+    eng.set_kv_pages(table)
+    prompts = [si.prompt(shape, seq=0, length=61), si.prompt(shape, seq=1, length=120)]
+    st = lockstep_run_batch(eng, orc, shape, parents, prompts, 6)
+    assert st.steps == 12
+    # single sequence on the same paged engine: forced-accept steps (real compaction) with the cache rows compared
+    st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=58), 5, forced=True, seq=1, check_cache_rows=True)
+    assert st.steps == 5
+    eng.set_kv_pages(None)                                       # back to contiguous rows
+    st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=58), 2, seq=0, check_cache_rows=True)
+    assert st.steps == 2
+    eng.close()
+
+
 def test_chains_need_the_row_capacity(torch_cuda, c1, c1_weights):
     import torch
     from paper_2410_20488_b200 import FirpError, binding
