@@ -217,6 +217,19 @@ int firp_kv_commit(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const i
                    const int32_t *path_len, void *stream);
 
 /*
+ * Precision of the activations that enter the five weight GEMMs (the paper runs its models in half precision,
+ * Section 4 "Setup", and says nothing about the arithmetic of a step).  Every GEMM multiplies bf16 by bf16 into
+ * fp32 on the tensor cores; an activation is split into 1, 2 or 3 bf16 planes (hi; hi + lo; hi + mid + lo =
+ * 8, 16, 24 mantissa bits) whose products are summed.  Default: 2 everywhere; the step then tracks an fp32
+ * reference to ~3e-3 in the logits over 32 layers (a third plane on the QKV projection changes nothing measurable
+ * and costs 3 % of the step).  1 is the plain bf16 GEMM; it halves the tensor-core work and the activation
+ * traffic, which matters for steps of more than ~80 rows, at the price of 0.07-0.09 logit error over 32 layers
+ * when used on the O, gate/up or down projection (0.01-0.02 on the QKV projection or the lm-head alone).  Applies to the kernel-per-operation
+ * mode; the persistent kernel keeps the defaults.
+ */
+int firp_set_activation_planes(firp_ctx *ctx, int32_t qkv, int32_t o, int32_t gate_up, int32_t down, int32_t lm_head);
+
+/*
  * How the decoder layers of a step are launched (Section 3.4 describes one forward pass per round; the
  * paper gives no kernel design).  on != 0: a step of at most 48 rows over all its sequences runs its
  * layers, Eq. 3 and the lm-head as ONE persistent kernel (6 launches per step instead of ~300) whose weight

@@ -83,6 +83,7 @@ struct firp_ctx {
   int last_n_seq = 0, last_T = 0, last_k = 0;
   int pseudo_masked = 0;     // Section 4.3 "Masked": pseudo rows do not see one another
   int pred_prenorm = 0;      // Eq. 3 reads the anchor through the insertion layer's input RMSNorm
+  int planes[5] = {2, 2, 2, 2, 2};   // bf16 planes of the activations per GEMM class: qkv, o, gate/up, down, lm-head
 
   // cache layout [layer][K|V][row][kv_head][head_dim]; row = slot * max_ctx + position, or through the page table
   size_t kv_seq() const { return (size_t)cfg.max_ctx * cfg.n_kv_heads * cfg.head_dim; }      // elements per slot of a plane
@@ -284,7 +285,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     const int carried = rw.T + alive * per_step;
     const int act = carried + ins * per_step;                  // rows alive in this layer
     { FIRP_TIMED(KC_RMSNORM);
-      FIRP_CUDA(c, launch_rmsnorm(rw, 0, carried, c->h, pending, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, 3, c->ss, pdl, st)); ++nl; }
+      FIRP_CUDA(c, launch_rmsnorm(rw, 0, carried, c->h, pending, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, c->planes[0] == 3 ? 3 : 2, c->ss, pdl, st)); ++nl; }
     pending.sk.U = 0;
     if (insert) {   // Eq. 3 on the raw (now complete) residual row of the root, then the norm of the new rows
       { FIRP_TIMED(KC_PSEUDO_PROJ);      // this layer's maps as one [ins d][d] GEMM on the source rows (the anchor of
@@ -303,7 +304,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
         p.ws_rows = (int)Rp;
         FIRP_CUDA(c, launch_gemm_finish(EPI_PSEUDO, p, g, pdl, st)); ++nl; }
       FIRP_TIMED(KC_RMSNORM);
-      FIRP_CUDA(c, launch_rmsnorm(rw, carried, act, c->h, none, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, 3, c->ss, pdl, st)); ++nl;
+      FIRP_CUDA(c, launch_rmsnorm(rw, carried, act, c->h, none, (const bf16 *)c->g_attn[j], d, c->x, Rp * d, c->planes[0] == 3 ? 3 : 2, c->ss, pdl, st)); ++nl;
       alive += ins;
     }
     bf16 *kplane = c->kv + (size_t)j * c->kv_layer();
@@ -312,7 +313,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       g.H = H; g.Hkv = Hkv; g.dh = dh;
       g.l2_ahead = ahead[0];
       set_next(g, 0, EPI_RESIDUAL, c->wo[j], d, nq);
-      g.planes = 3;   // keys and values are rounded to bf16 for the cache: their inputs carry ~24 mantissa bits
+      g.planes = c->planes[0];
       g.rope = c->meta.rope; g.seq_ids = c->seq_ids; g.ctx_len = c->ctx_len; g.pos = c->meta.pos;
       g.q = c->q; g.q_lo_off = Rp * nq; g.kcache = kplane; g.seq_stride = c->kv_seq(); g.kv_stride = c->kv_plane(); g.max_ctx = cfg.max_ctx; g.pages = c->pages();
       Partials p = pending;
@@ -335,6 +336,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     }
     {
       GemmArgs g = gemm_base(c->o, Rp * nq, c->wo[j], d, nq, act);
+      g.planes = c->planes[1];
       g.l2_ahead = ahead[1];
       set_next(g, 1, EPI_SWIGLU, c->wgu[j], 2 * F, d);
       FIRP_TIMED(KC_GEMM_O);
@@ -345,6 +347,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     pending.sk.U = 0;
     {
       GemmArgs g = gemm_base(c->x, Rp * d, c->wgu[j], 2 * F, d, act);
+      g.planes = c->planes[2];
       g.y = c->y; g.y_lo_off = Rp * F; g.F = F; g.l2_ahead = ahead[2];
       set_next(g, 2, EPI_RESIDUAL, c->wd[j], d, F);
       Partials p = pending;
@@ -355,6 +358,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
     }
     {
       GemmArgs g = gemm_base(c->y, Rp * F, c->wd[j], d, F, act);
+      g.planes = c->planes[3];
       g.l2_ahead = ahead[3];
       if (j + 1 < cfg.n_layers) set_next(g, 3, EPI_QKV_ROPE, c->wqkv[j + 1], (H + 2 * Hkv) * dh, d);
       else if (ra.want_head) set_next(g, 3, EPI_LOGITS, c->w.lm_head, cfg.vocab, d);
@@ -367,6 +371,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       { FIRP_TIMED(KC_RMSNORM);
         FIRP_CUDA(c, launch_rmsnorm(rw, 0, rw.Ms, c->h, pending, (const bf16 *)c->w.g_final, d, c->x, Rp * d, 2, c->ss, pdl, st)); ++nl; }
       GemmArgs g = gemm_base(c->x, Rp * d, c->w.lm_head, cfg.vocab, d, rw.Ms);
+      g.planes = c->planes[4];
       g.logits = ra.logits_dst; g.l2_ahead = ahead[4];
       Partials p = pending;
       { FIRP_TIMED(KC_GEMM_LM_HEAD);
@@ -687,6 +692,15 @@ int firp_set_kv_pages(firp_ctx *ctx, const int32_t *page_table, void *stream) {
   FIRP_CUDA(ctx, cudaMemcpyAsync(ctx->d_pages, page_table, sizeof(int32_t) * total, cudaMemcpyHostToDevice, st));
   FIRP_CUDA(ctx, cudaStreamSynchronize(st));
   ctx->paged = true;
+  return FIRP_OK;
+}
+
+int firp_set_activation_planes(firp_ctx *ctx, int32_t qkv, int32_t o, int32_t gate_up, int32_t down, int32_t lm_head) {
+  if (!ctx) return FIRP_ERR_BAD_ARG;
+  const int32_t p[5] = {qkv, o, gate_up, down, lm_head};
+  for (int i = 0; i < 5; ++i)
+    if (p[i] < 1 || p[i] > (i == 0 ? 3 : 2)) return fail(ctx, FIRP_ERR_BAD_ARG, "planes must be 1..2 (1..3 for the QKV projection)");
+  for (int i = 0; i < 5; ++i) ctx->planes[i] = p[i];
   return FIRP_OK;
 }
 

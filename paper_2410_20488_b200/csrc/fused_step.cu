@@ -582,7 +582,7 @@ bool fused_eligible(const FusedShape &sh, const Rows &rw) {
   const int G = fused_sm_count();
   if (G > kGemmMaxCtas) return false;
   const int nq = sh.H * sh.dh;
-  const GemmClass c[5] = {make_class(EPI_QKV_ROPE, (sh.H + 2 * sh.Hkv) * sh.dh, sh.d, 3, 0, sh.F, sh.H, sh.Hkv, sh.dh),
+  const GemmClass c[5] = {make_class(EPI_QKV_ROPE, (sh.H + 2 * sh.Hkv) * sh.dh, sh.d, 2, 0, sh.F, sh.H, sh.Hkv, sh.dh),
                           make_class(EPI_RESIDUAL, sh.d, nq, 2, 0, sh.F, sh.H, sh.Hkv, sh.dh),
                           make_class(EPI_SWIGLU, 2 * sh.F, sh.d, 2, 0, sh.F, sh.H, sh.Hkv, sh.dh),
                           make_class(EPI_RESIDUAL, sh.d, sh.F, 2, 0, sh.F, sh.H, sh.Hkv, sh.dh),
@@ -630,7 +630,7 @@ cudaError_t launch_fused_layers(FusedPlan *plan, const FusedStep &fs, bool pdl, 
     if (!ok) return cudaErrorInvalidValue;
     // GEMM classes
     enum { C_QKV = 0, C_O, C_GU, C_DOWN, C_LM, C_PSEUDO0 };
-    P.cls[C_QKV] = make_class(EPI_QKV_ROPE, (H + 2 * Hkv) * dh, d, 3, m_x + 0, F, H, Hkv, dh);
+    P.cls[C_QKV] = make_class(EPI_QKV_ROPE, (H + 2 * Hkv) * dh, d, 2, m_x + 0, F, H, Hkv, dh);
     P.cls[C_O] = make_class(EPI_RESIDUAL, d, nq, 2, m_x + 2, F, H, Hkv, dh);
     P.cls[C_GU] = make_class(EPI_SWIGLU, 2 * F, d, 2, m_x + 0, F, H, Hkv, dh);
     P.cls[C_DOWN] = make_class(EPI_RESIDUAL, d, F, 2, m_x + 3, F, H, Hkv, dh);
@@ -652,7 +652,7 @@ cudaError_t launch_fused_layers(FusedPlan *plan, const FusedStep &fs, bool pdl, 
       int ins = 0;
       while (alive + ins < rw.kc && fs.tl[alive + ins] == j) ++ins;
       const int carried = rw.T + alive * per_step, act = carried + ins * per_step;
-      add_op(OP_NORM, 0, 3, j, 0, carried, carried, pending, fs.g_attn[j]);
+      add_op(OP_NORM, 0, 2, j, 0, carried, carried, pending, fs.g_attn[j]);
       pending = -1;
       if (ins > 0) {       // Eq. 3 on the raw (now complete) residual rows, then the norm of the new rows
         if (n_pred >= 8 || P.n_cls >= kMaxClasses) return cudaErrorInvalidConfiguration;
@@ -664,7 +664,7 @@ cudaError_t launch_fused_layers(FusedPlan *plan, const FusedStep &fs, bool pdl, 
         add_op(OP_ROOT_SPLIT, 0, 0, j, 0, 0, act, 0, fs.prenorm ? fs.g_attn[j] : nullptr);
         add_gemm(cls, m_pred0 + n_pred, j, act);
         add_op(OP_FINISH, cls, fs.prenorm ? 1 : 0, j, 0, 0, act, alive, fs.pred_b ? (const bf16 *)fs.pred_b + (size_t)alive * d : nullptr);
-        add_op(OP_NORM, 0, 3, j, carried, act - carried, act, -1, fs.g_attn[j]);
+        add_op(OP_NORM, 0, 2, j, carried, act - carried, act, -1, fs.g_attn[j]);
         ++n_pred;
         alive += ins;
       }

@@ -424,6 +424,12 @@ cudaError_t launch_rows(const GemmArgs &a, const Sched &sc, cudaStream_t st) {
     if (a.R <= 80) return launch_np<80, 3>(a, sc, st);
     return launch_np<144, 3>(a, sc, st);
   }
+  if (a.planes == 1) {   // plain bf16 activations (the hi plane alone)
+    if (a.R <= 16) return launch_np<16, 1>(a, sc, st);
+    if (a.R <= 48) return launch_np<48, 1>(a, sc, st);
+    if (a.R <= 80) return launch_np<80, 1>(a, sc, st);
+    return launch_np<144, 1>(a, sc, st);
+  }
   if (a.R <= 16) return launch_np<16, 2>(a, sc, st);
   if (a.R <= 40) return launch_np<40, 2>(a, sc, st);
   if (a.R <= 48) return launch_np<48, 2>(a, sc, st);
