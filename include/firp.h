@@ -229,6 +229,10 @@ int firp_kv_commit(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const i
  */
 int firp_set_activation_planes(firp_ctx *ctx, int32_t qkv, int32_t o, int32_t gate_up, int32_t down, int32_t lm_head);
 
+/* The same for the attention's two contractions: planes of the rotated queries (Q K^T) and of the softmax
+ * probabilities (P V); keys and values are the cache's bf16.  Default 2 and 2. */
+int firp_set_attention_planes(firp_ctx *ctx, int32_t q_planes, int32_t p_planes);
+
 /*
  * How the decoder layers of a step are launched (Section 3.4 describes one forward pass per round; the
  * paper gives no kernel design).  on != 0: a step of at most 48 rows over all its sequences runs its

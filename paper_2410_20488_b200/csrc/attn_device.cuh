@@ -143,8 +143,10 @@ __device__ __forceinline__ void attn_split_item(const AttnArgs &a, uint8_t *smem
         ldmatrix_x4(b0, b1, b2, b3, attn_smem_u32(kt + tile_off<DH>(row, chunk)));
         mma_bf16(sc[2 * p], qh, b0, b1);
         mma_bf16(sc[2 * p + 1], qh, b2, b3);
-        mma_bf16(sc[2 * p], ql, b0, b1);
-        mma_bf16(sc[2 * p + 1], ql, b2, b3);
+        if (a.q_planes > 1) {
+          mma_bf16(sc[2 * p], ql, b0, b1);
+          mma_bf16(sc[2 * p + 1], ql, b2, b3);
+        }
       }
     }
     // mask, scale, online softmax (rows g and g+8 of this warp's 16)
@@ -221,8 +223,10 @@ __device__ __forceinline__ void attn_split_item(const AttnArgs &a, uint8_t *smem
         ldmatrix_x4_trans(b0, b1, b2, b3, attn_smem_u32(vt + tile_off<DH>(row, chunk)));
         mma_bf16(o_acc[2 * d2], pf[j], b0, b1);
         mma_bf16(o_acc[2 * d2 + 1], pf[j], b2, b3);
-        mma_bf16(o_acc[2 * d2], pl[j], b0, b1);
-        mma_bf16(o_acc[2 * d2 + 1], pl[j], b2, b3);
+        if (a.p_planes > 1) {
+          mma_bf16(o_acc[2 * d2], pl[j], b0, b1);
+          mma_bf16(o_acc[2 * d2 + 1], pl[j], b2, b3);
+        }
       }
     }
     Sync::sync();

@@ -83,7 +83,8 @@ struct firp_ctx {
   int last_n_seq = 0, last_T = 0, last_k = 0;
   int pseudo_masked = 0;     // Section 4.3 "Masked": pseudo rows do not see one another
   int pred_prenorm = 0;      // Eq. 3 reads the anchor through the insertion layer's input RMSNorm
-  int planes[5] = {2, 2, 2, 2, 2};   // bf16 planes of the activations per GEMM class: qkv, o, gate/up, down, lm-head
+  int planes[5] = {2, 2, 2, 2, 2};
+  int attn_planes[2] = {2, 2};       // of the queries and of the probabilities in the attention   // bf16 planes of the activations per GEMM class: qkv, o, gate/up, down, lm-head
 
   // cache layout [layer][K|V][row][kv_head][head_dim]; row = slot * max_ctx + position, or through the page table
   size_t kv_seq() const { return (size_t)cfg.max_ctx * cfg.n_kv_heads * cfg.head_dim; }      // elements per slot of a plane
@@ -327,6 +328,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       a.rw = rw; a.rows_active = act; a.H = H; a.Hkv = Hkv; a.dh = dh;
       a.q = c->q; a.q_lo_off = Rp * nq; a.kcache = kplane; a.seq_stride = c->kv_seq(); a.kv_stride = c->kv_plane(); a.max_ctx = cfg.max_ctx; a.pages = c->pages();
       a.seq_ids = c->seq_ids; a.ctx_len = c->ctx_len; a.pos = c->meta.pos; a.mask = c->meta.mask;
+      a.q_planes = c->attn_planes[0]; a.p_planes = c->attn_planes[1];
       const int tiles = (ra.n_hi_max + act + kAttnTile - 1) / kAttnTile;
       const int G = H / Hkv, qblocks = (act * G + 63) / 64;
       a.splits = attention_splits(rw.n_seq * Hkv * qblocks, tiles);
@@ -701,6 +703,12 @@ int firp_set_activation_planes(firp_ctx *ctx, int32_t qkv, int32_t o, int32_t ga
   for (int i = 0; i < 5; ++i)
     if (p[i] < 1 || p[i] > (i == 0 ? 3 : 2)) return fail(ctx, FIRP_ERR_BAD_ARG, "planes must be 1..2 (1..3 for the QKV projection)");
   for (int i = 0; i < 5; ++i) ctx->planes[i] = p[i];
+  return FIRP_OK;
+}
+
+int firp_set_attention_planes(firp_ctx *ctx, int32_t q_planes, int32_t p_planes) {
+  if (!ctx || q_planes < 1 || q_planes > 2 || p_planes < 1 || p_planes > 2) return FIRP_ERR_BAD_ARG;
+  ctx->attn_planes[0] = q_planes; ctx->attn_planes[1] = p_planes;
   return FIRP_OK;
 }
 

@@ -208,6 +208,7 @@ struct AttnArgs {
   const int32_t *pos;         // [R] absolute position of every row (row 0 of a sequence: its committed length)
   const uint32_t *mask;       // [R][kMaskWords]
   int splits;                 // kv splits (grid.x = cluster size): 1, 2, 4 or 8
+  int q_planes, p_planes;     // bf16 planes of the queries / of the probabilities that enter the tensor cores: 2 (hi, lo) or 1
   bf16 *o; size_t o_lo_off;   // [R][H*dh] hi plane, lo plane
 };
 // kv splits for `groups` = sequences x kv heads x query blocks and `kv_tiles` 64-position tiles

@@ -385,6 +385,7 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_layers_kernel(const __grid
           a.q = P.q; a.q_lo_off = (size_t)P.Rp * nq; a.kcache = P.kv + (size_t)op.layer * P.kv_layer;
           a.seq_stride = P.kv_seq; a.kv_stride = P.kv_plane; a.max_ctx = P.max_ctx; a.pages = P.pages;
           a.seq_ids = P.seq_ids; a.ctx_len = P.ctx_len; a.pos = P.pos; a.mask = P.mask; a.splits = P.splits;
+          a.q_planes = 2; a.p_planes = 2;
           const int Gq = P.H / P.Hkv;
           const int qblocks = (op.act * Gq + kAttnQRows - 1) / kAttnQRows;
           const int n_items = P.rw.n_seq * qblocks * P.Hkv * P.splits;
