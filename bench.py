@@ -124,7 +124,7 @@ def kernel_source_digest() -> str:
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2410_20488_b200", "csrc")
     for name in sorted(os.listdir(csrc)):
-        if name.endswith((".cu", ".cuh")):
+        if name.endswith((".cu", ".cuh")) and name != "firp_api.cu":       # device code only (firp_api.cu is host code)
             h.update(open(os.path.join(csrc, name), "rb").read())
     return h.hexdigest()[:16]
 
@@ -156,7 +156,7 @@ def kernel_times(eng, shape, parents, tokens, out, steps, n_ctx, peak_gbs, peak_
         kernels[name] = k
     top = max((n for n in kernels if n in cb), key=lambda n: kernels[n]["share"])
     t = kernels[top]
-    rec = ncu_traffic(shape.name)
+    rec = None if CHAINS else ncu_traffic(shape.name)      # the capture is of the 35-row step
     traffic = rec.get(top) if rec else None
     roofline = dict(bound="hbm", kernel=top, achieved=t["achieved_gbs"], peak=peak_gbs, unit="GB/s",
                     frac=t["frac_of_peak"], traffic=traffic, peak_kind="%s copy bandwidth" % peak_kind,
@@ -317,7 +317,8 @@ def run_forced(eng, shape, parents, tokens, outs, K, dev, step_fn):
     ms = ev0.elapsed_time(ev1)
     emitted = eng.context_len(0) - n0
     return dict(tokens_per_s=emitted / (ms * 1e-3), tokens_per_step=emitted / K, ms_per_step=ms / K, steps=K, depth=D,
-                note="device-resident; the timed region also holds the three small torch kernels per step that plant the chain")
+                note="device-resident; the timed region also holds the three small torch kernels per step that plant the chain; "
+                     "a near-tie that the T = 1 pass and the tree pass resolve differently desynchronises every later step")
 
 
 def load_weights(shape, local_rank: int, world: int):

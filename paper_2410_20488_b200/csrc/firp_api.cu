@@ -51,6 +51,7 @@ struct firp_ctx {
   bool bound = false, have_weights = false, stepped = false;
   int Rmax = 0, S = 0;                  // rows the workspace holds (a prefill chunk), path stride
   int row_cap = 0;                      // rows one step may carry (max_rows of the configuration)
+  int sm_count = 148;                   // of the device the buffers were bound on
   bool use_pdl = true;                  // programmatic dependent launch
   bool use_fused = false;               // firp_set_fused: steps of at most 48 rows run their layers as one persistent kernel
   unsigned long long wait_ns = 0;       // bound of device-side waits (0: the kernels' default)
@@ -333,8 +334,14 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       const int G = H / Hkv, qblocks = (act * G + 63) / 64;
       a.splits = attention_splits(rw.n_seq * Hkv * qblocks, tiles);
       a.o = c->o; a.o_lo_off = Rp * nq;
+      // Early (programmatic) launch of the attention pays only when the rotary finisher before it has at least one
+      // CTA per SM.  Measured at the 7B shape, ms per step with / without it: 35 rows 3.61 / 3.76 at 512 cached
+      // tokens and 5.25 / 5.44 at 8192; 67 and 131 rows likewise 0.1 ms better with it; but 19 rows 3.68 / 3.60 and
+      // 6.36 / 5.26, 1 row 3.52 / 3.43 and 6.27 / 5.11.
+      const int half_dh = dh / 2, qkv_st = (H + 2 * Hkv + 128 / half_dh - 1) / (128 / half_dh);
+      const bool attn_early = pdl && (qkv_st * rw.R * 32 + 255) / 256 >= c->sm_count;
       FIRP_TIMED(KC_ATTENTION);
-      FIRP_CUDA(c, launch_attention(a, pdl, st)); ++nl;
+      FIRP_CUDA(c, launch_attention(a, attn_early, st)); ++nl;
     }
     {
       GemmArgs g = gemm_base(c->o, Rp * nq, c->wo[j], d, nq, act);
@@ -467,6 +474,10 @@ int firp_bind_buffers(firp_ctx *ctx, void *workspace, void *kv_cache, void *stre
   ctx->last_parents.clear(); ctx->last_next_parents.clear(); ctx->last_seq_ids.clear();
   if (!gemm_tc_available())
     return fail(ctx, FIRP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+  {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ctx->sm_count = n;
+  }
   ctx->bound = true; ctx->stepped = false;
   ++ctx->weights_gen;
   return FIRP_OK;
