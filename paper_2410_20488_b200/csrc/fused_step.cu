@@ -10,15 +10,16 @@
 // (Measured on B200: reading through L2 is not faster than reading HBM for this access pattern, so prefetching
 // into L2 buys nothing; the ring is the only buffer that hides a dependency.)
 //
-// Per CTA, 7 warps:
-//   warp 0    weight producer: TMA (128-byte swizzle) into a ring of 32 KB stages; depends on nothing
-//   warp 6    activation producer: the (hi, lo[, third]) bf16 planes of the k block, after the phase's inputs are
-//             complete (signalled by the workers through a shared-memory barrier)
-//   warp 1    MMA issuer: tcgen05.mma kind::f16, accumulators in TMEM; roles swapped as in the stand-alone GEMM
-//             (weight rows = MMA M, token rows = MMA N, the planes side by side as one N)
-//   warps 2-5 workers: TMEM -> partial tiles (stream-K), then every non-GEMM phase: the elementwise passes are
-//             spread over all CTAs, the attention runs one (kv head, query block, kv split) item per CTA at a time
-//             in the shared memory the activation ring does not need meanwhile
+// Per CTA, 11 warps:
+//   warp 0     weight producer: TMA (128-byte swizzle) into a ring of 32 KB stages; depends on nothing
+//   warp 6     activation producer: the (hi, lo) bf16 planes of the k block, after the phase's inputs are complete
+//              (signalled by the workers through a shared-memory barrier)
+//   warp 1     MMA issuer: tcgen05.mma kind::f16, accumulators in TMEM; roles swapped as in the stand-alone GEMM
+//              (weight rows = MMA M, token rows = MMA N, the planes side by side as one N)
+//   warps 2-5, 7-10  workers: TMEM -> partial tiles (stream-K; one group of four warps per weight tile of the
+//              supertile), then every non-GEMM phase: the elementwise passes are spread over all CTAs, the attention
+//              runs one (kv head, query block, kv split) item per CTA at a time on warps 2-5, in the shared memory
+//              the activation ring does not need meanwhile
 // Phases are separated by a grid-wide barrier (an arrival counter in global memory; every wait is bounded and
 // reports through the status word).  Partial tiles are summed in ascending CTA order, the attention splits in
 // ascending split order: results are identical from run to run.
@@ -107,7 +108,7 @@ struct AttnGroupSync { static __device__ __forceinline__ void sync() { asm volat
 
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// Grid-wide barrier of the worker warps (128 threads per CTA).  Monotonic arrival counter; `epoch` counts the
+// Grid-wide barrier of the worker warps (256 threads per CTA).  Monotonic arrival counter; `epoch` counts the
 // barriers passed.  The wait is bounded: on expiry the status word is set and this thread stops waiting for good.
 __device__ __forceinline__ void grid_sync(unsigned *ctr, unsigned &epoch, int wtid, int *err, bool &dead,
                                           unsigned long long wait_ns, bool tma_reads_follow) {

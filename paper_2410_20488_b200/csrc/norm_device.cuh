@@ -59,7 +59,7 @@ __device__ __forceinline__ void rmsnorm_item(const Rows &rw, int v0, int nv, flo
   lo2.x = *reinterpret_cast<const uint32_t *>(&l01); lo2.y = *reinterpret_cast<const uint32_t *>(&l23);
   *reinterpret_cast<uint2 *>(x + (size_t)r * d + 4 * idx) = hi2;
   *reinterpret_cast<uint2 *>(x + x_lo_off + (size_t)r * d + 4 * idx) = lo2;
-  if (planes == 3) {   // third plane: what hi + mid still miss (the K/V projections need fp32-grade inputs)
+  if (planes == 3) {   // third plane on request: what hi + mid still miss (measured: it changes no logit)
     const float2 m01 = __bfloat1622float2(l01), m23 = __bfloat1622float2(l23);
     const __nv_bfloat162 t01 = __floats2bfloat162_rn(y0 - f01.x - m01.x, y1 - f01.y - m01.y);
     const __nv_bfloat162 t23 = __floats2bfloat162_rn(y2 - f23.x - m23.x, y3 - f23.y - m23.y);
