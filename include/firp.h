@@ -175,6 +175,20 @@ int firp_step_chains(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const
                      const firp_step_out *out, void *stream);
 
 /*
+ * The step of firp_step_layers with a tree of its own for every sequence (Section 3.4 builds the tree from
+ * each sequence's own candidates; sequences at different points of their generation need not share a shape).
+ *   tree_parents  HOST [n_seq][T]: row s holds the parents of sequence s's tree in its first tree_sizes[s] entries
+ *   tree_sizes    HOST [n_seq]: 1 <= tree_sizes[s] <= T nodes
+ * Every sequence still occupies T + k rows: rows tree_sizes[s] .. T-1 are padding (their tokens are ignored, they
+ * can neither be accepted nor take a candidate; what the outputs hold for them is unspecified), the pseudo rows
+ * stay at rows T .. T+k-1.  Each tree is validated like the template of firp_step; the next tree of a sequence is
+ * built on its own shape.  Needs k > 0 unless every size equals T.
+ */
+int firp_step_trees(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
+                    const int32_t *tree_parents, const int32_t *tree_sizes, int32_t T, int32_t k,
+                    const int32_t *layers, const firp_step_out *out, void *stream);
+
+/*
  * Visibility among the pseudo rows (Section 4.3, ablation).  masked = 0 (default, the "No masked"
  * setting the paper adopts): chain row i sees rows 1..i-1 of its chain.  masked != 0 ("Masked"): a
  * pseudo row sees no other pseudo row, only the prefix, its node with its ancestors, and itself;

@@ -47,7 +47,7 @@ EXPORTS = ("firp_create", "firp_destroy", "firp_last_error", "firp_workspace_byt
            "firp_context_len", "firp_set_context_len", "firp_last_launch_count", "firp_profile_enable",
            "firp_profile_read", "firp_kernel_class_name", "firp_topb_static", "firp_prefill_layers", "firp_step_layers", "firp_step_chains", "firp_set_pseudo_masked",
            "firp_set_fused", "firp_set_wait_limit_us", "firp_selftest_wait", "firp_set_pred_prenorm", "firp_set_kv_pages",
-           "firp_set_activation_planes", "firp_set_attention_planes")
+           "firp_set_activation_planes", "firp_set_attention_planes", "firp_step_trees")
 
 
 def lib_path() -> str:
@@ -79,6 +79,7 @@ def load_library():
     lib.firp_prefill_layers.argtypes = [vp, i32, vp, i32, i32, vp, vp, i32, ctypes.POINTER(StepOutC), vp]
     lib.firp_step_layers.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp, ctypes.POINTER(StepOutC), vp]
     lib.firp_step_chains.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp, ctypes.POINTER(StepOutC), vp]
+    lib.firp_step_trees.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, vp, ctypes.POINTER(StepOutC), vp]
     lib.firp_set_pseudo_masked.argtypes = [vp, i32]
     lib.firp_set_fused.argtypes = [vp, i32]
     lib.firp_set_attention_planes.argtypes = [vp, i32, i32]
@@ -195,6 +196,19 @@ def firp_step_chains(ctx, n_seq: int, seq_ids, d_tokens_ptr: int, tree_parents, 
         raise ValueError("need one insertion layer per prediction step")
     _check(ctx, load_library().firp_step_chains(ctx, n_seq, ids_ptr, d_tokens_ptr, par_ptr, T, k, lay_ptr,
                                                 ctypes.byref(out) if out is not None else None, stream))
+
+
+def firp_step_trees(ctx, n_seq: int, seq_ids, d_tokens_ptr: int, tree_parents, tree_sizes, T: int, k: int, layers,
+                    out: StepOutC, stream: int = 0):
+    """A tree per sequence: tree_parents host [n_seq][T], tree_sizes host [n_seq] (see firp.h)."""
+    ids, ids_ptr = _host_i32(seq_ids)
+    par, par_ptr = _host_i32(tree_parents)
+    siz, siz_ptr = _host_i32(tree_sizes)
+    lay, lay_ptr = _host_i32(layers)
+    if par is None or par.size != n_seq * T or siz is None or siz.size != n_seq:
+        raise ValueError("tree_parents must be [n_seq][T] and tree_sizes [n_seq]")
+    _check(ctx, load_library().firp_step_trees(ctx, n_seq, ids_ptr, d_tokens_ptr, par_ptr, siz_ptr, T, k, lay_ptr,
+                                               ctypes.byref(out) if out is not None else None, stream))
 
 
 def firp_set_pseudo_masked(ctx, masked: bool):
@@ -379,6 +393,14 @@ class FirpEngine:
         layers = [l] * k if np.isscalar(l) else l
         firp_step_chains(self.ctx, n_seq, seq_ids, d_tokens.data_ptr(), parents, len(parents), k, layers,
                          out.c if out is not None else None, self.stream)
+
+    def step_trees(self, d_tokens, tree_parents, tree_sizes, k, l, out: StepOut, seq_ids=None):
+        """A tree per sequence: tree_parents [n_seq][T] (host), tree_sizes [n_seq]; d_tokens [n_seq][T]."""
+        par = np.ascontiguousarray(tree_parents, np.int32)
+        n_seq, T = par.shape
+        layers = [l] * k if np.isscalar(l) else l
+        firp_step_trees(self.ctx, n_seq, seq_ids, d_tokens.data_ptr(), par, tree_sizes, T, k, layers,
+                        out.c if out is not None else None, self.stream)
 
     def set_pseudo_masked(self, masked: bool):
         firp_set_pseudo_masked(self.ctx, masked)

@@ -75,12 +75,12 @@ struct firp_ctx {
   bf16 *x = nullptr, *xp = nullptr, *q = nullptr, *o = nullptr, *y = nullptr;
   int32_t *ctx_len = nullptr, *seq_ids = nullptr, *parents = nullptr, *next_parents = nullptr, *chain = nullptr;
   int32_t *top_ids = nullptr, *path = nullptr, *n_acc = nullptr, *accepted = nullptr, *next_tokens = nullptr;
-  int32_t *exp_path = nullptr, *exp_len = nullptr;
+  int32_t *exp_path = nullptr, *exp_len = nullptr, *tree_sizes = nullptr;
   TreeMeta meta{};
   size_t ws_bytes = 0;
   // host mirrors
   std::vector<int32_t> n_hi;           // upper bound of each slot's committed length
-  std::vector<int32_t> last_parents, last_next_parents, last_seq_ids;
+  std::vector<int32_t> last_parents, last_next_parents, last_seq_ids, last_sizes;
   int last_n_seq = 0, last_T = 0, last_k = 0;
   int pseudo_masked = 0;     // Section 4.3 "Masked": pseudo rows do not see one another
   int pred_prenorm = 0;      // Eq. 3 reads the anchor through the insertion layer's input RMSNorm
@@ -124,6 +124,7 @@ struct firp_ctx {
     next_tokens = c.take<int32_t>((size_t)kMaxSeq * kMaxTreeRows);
     exp_path = c.take<int32_t>((size_t)kMaxSeq * S);
     exp_len = c.take<int32_t>(kMaxSeq);
+    tree_sizes = c.take<int32_t>(kMaxSeq);
     dev_status = c.take<int>(1);
     grid_bar = c.take<unsigned>(1);
     attn_ws = c.take<float>(fused_attn_ws_floats(cfg.max_batch, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim));
@@ -213,6 +214,8 @@ struct RunArgs {
   const firp_step_out *out;
   float *logits_dst;         // where the lm-head writes (workspace or caller buffer)
   int n_hi_max;              // upper bound of the longest committed context among the sequences
+  int parents_stride;        // 0: one tree template for all sequences; T: a tree per sequence
+  const int32_t *d_sizes;    // per-sequence tree sizes (device) or NULL
 };
 
 int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
@@ -231,7 +234,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
 
   const int mw_out = (rw.Ms + 31) / 32;
   { FIRP_TIMED(KC_TREE_PREP);
-    launch_tree_prep(rw, c->parents, c->seq_ids, c->ctx_len, dh, cfg.rope_theta, c->meta, out ? out->depth : nullptr,
+    launch_tree_prep(rw, c->parents, ra.parents_stride, c->seq_ids, c->ctx_len, dh, cfg.rope_theta, c->meta, out ? out->depth : nullptr,
                      out ? out->mask : nullptr, mw_out, c->grid_bar, pdl, st); ++nl; }
   { FIRP_TIMED(KC_EMBED);
     launch_embed(rw, ra.d_tokens, (const bf16 *)c->w.embed, d, cfg.vocab, c->h, pdl, st); ++nl; }
@@ -393,6 +396,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       nl += 2; }
     AcceptArgs a{};
     a.tokens = ra.d_tokens; a.parents = c->parents; a.next_parents = c->next_parents;
+    a.parents_stride = ra.parents_stride; a.sizes = ra.d_sizes;
     a.top_ids = c->top_ids; a.top_vals = c->top_vals; a.T_next = ra.T_next; a.B = cfg.top_b; a.S = c->S;
     a.prefill_last_row = ra.prefill_last_row;
     a.path = c->path; a.n_accepted = c->n_acc; a.accepted = c->accepted; a.next_tokens = c->next_tokens;
@@ -471,7 +475,7 @@ int firp_bind_buffers(firp_ctx *ctx, void *workspace, void *kv_cache, void *stre
   FIRP_CUDA(ctx, cudaMemcpyAsync(ctx->chain, chain.data(), sizeof(int32_t) * kMaxTreeRows, cudaMemcpyHostToDevice, st));
   FIRP_CUDA(ctx, cudaStreamSynchronize(st));
   std::fill(ctx->n_hi.begin(), ctx->n_hi.end(), 0);
-  ctx->last_parents.clear(); ctx->last_next_parents.clear(); ctx->last_seq_ids.clear();
+  ctx->last_parents.clear(); ctx->last_next_parents.clear(); ctx->last_seq_ids.clear(); ctx->last_sizes.clear();
   if (!gemm_tc_available())
     return fail(ctx, FIRP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
   {
@@ -542,24 +546,33 @@ int firp_step(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_
 
 // One chain of k pseudo rows under the root (chains = false) or under every tree node (chains = true).
 static int step_impl(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
-                     const int32_t *tree_parents, int32_t T, int32_t k, const int32_t *layers, bool chains,
-                     const firp_step_out *out, void *stream);
+                     const int32_t *tree_parents, const int32_t *tree_sizes, int32_t T, int32_t k, const int32_t *layers,
+                     bool chains, const firp_step_out *out, void *stream);
 
 int firp_step_layers(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
                      const int32_t *tree_parents, int32_t T, int32_t k, const int32_t *layers, const firp_step_out *out,
                      void *stream) {
-  return step_impl(ctx, n_seq, seq_ids, d_tree_tokens, tree_parents, T, k, layers, false, out, stream);
+  return step_impl(ctx, n_seq, seq_ids, d_tree_tokens, tree_parents, nullptr, T, k, layers, false, out, stream);
 }
 
 int firp_step_chains(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
                      const int32_t *tree_parents, int32_t T, int32_t k, const int32_t *layers, const firp_step_out *out,
                      void *stream) {
-  return step_impl(ctx, n_seq, seq_ids, d_tree_tokens, tree_parents, T, k, layers, true, out, stream);
+  return step_impl(ctx, n_seq, seq_ids, d_tree_tokens, tree_parents, nullptr, T, k, layers, true, out, stream);
 }
 
+int firp_step_trees(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
+                    const int32_t *tree_parents, const int32_t *tree_sizes, int32_t T, int32_t k, const int32_t *layers,
+                    const firp_step_out *out, void *stream) {
+  if (!tree_sizes) return ctx ? fail(ctx, FIRP_ERR_BAD_ARG, "NULL tree sizes") : (int)FIRP_ERR_BAD_ARG;
+  return step_impl(ctx, n_seq, seq_ids, d_tree_tokens, tree_parents, tree_sizes, T, k, layers, false, out, stream);
+}
+
+// tree_sizes == NULL: one template tree_parents[T] for all sequences.  Otherwise tree_parents is [n_seq][T] and
+// sequence s uses its first tree_sizes[s] entries; the remaining rows are padding, hung under the root.
 static int step_impl(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const int32_t *d_tree_tokens,
-                     const int32_t *tree_parents, int32_t T, int32_t k, const int32_t *layers, bool chains,
-                     const firp_step_out *out, void *stream) {
+                     const int32_t *tree_parents, const int32_t *tree_sizes, int32_t T, int32_t k, const int32_t *layers,
+                     bool chains, const firp_step_out *out, void *stream) {
   int rc = check_ready(ctx);
   if (rc) return rc;
   const firp_model_cfg &cfg = ctx->cfg;
@@ -574,12 +587,22 @@ static int step_impl(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const
   const int Ms = T + pseudo;
   if (Ms > kMaxTreeRows || n_seq * Ms > ctx->row_cap)
     return fail(ctx, FIRP_ERR_CAPACITY, "%d sequences x %d rows exceed the row capacity %d (max_rows of the configuration)", n_seq, Ms, ctx->row_cap);
-  std::vector<int> depth;
-  const int maxd = tree_depths(tree_parents, T, depth);
-  if (maxd < 0) return fail(ctx, FIRP_ERR_BAD_TREE, "parents[0] must be -1 and 0 <= parents[v] < v");
-  if (maxd > cfg.max_depth) return fail(ctx, FIRP_ERR_BAD_TREE, "tree depth %d exceeds max_depth", maxd);
-  if (k > 0 && maxd > k) return fail(ctx, FIRP_ERR_BAD_TREE, "tree depth %d exceeds k = %d", maxd, k);
-  if (k > 0 && max_sibling_rank(tree_parents, T) >= cfg.top_b) return fail(ctx, FIRP_ERR_BAD_TREE, "more siblings than top_b");
+  // validate every tree (the shared template, or each sequence's own) and lay the parents out for the device
+  const int n_trees = tree_sizes ? n_seq : 1;
+  std::vector<int32_t> dev_parents((size_t)n_trees * T);
+  for (int t = 0; t < n_trees; ++t) {
+    const int32_t *par = tree_parents + (size_t)t * T;
+    const int size = tree_sizes ? tree_sizes[t] : T;
+    if (size < 1 || size > T) return fail(ctx, FIRP_ERR_BAD_TREE, "tree size %d outside 1..T", size);
+    if (size < T && k == 0) return fail(ctx, FIRP_ERR_BAD_TREE, "trees of different sizes need k > 0");
+    std::vector<int> depth;
+    const int maxd = tree_depths(par, size, depth);
+    if (maxd < 0) return fail(ctx, FIRP_ERR_BAD_TREE, "parents[0] must be -1 and 0 <= parents[v] < v");
+    if (maxd > cfg.max_depth) return fail(ctx, FIRP_ERR_BAD_TREE, "tree depth %d exceeds max_depth", maxd);
+    if (k > 0 && maxd > k) return fail(ctx, FIRP_ERR_BAD_TREE, "tree depth %d exceeds k = %d", maxd, k);
+    if (k > 0 && max_sibling_rank(par, size) >= cfg.top_b) return fail(ctx, FIRP_ERR_BAD_TREE, "more siblings than top_b");
+    for (int v = 0; v < T; ++v) dev_parents[(size_t)t * T + v] = v < size ? par[v] : 0;   // padding rows: children of the root
+  }
   int n_hi_max = 0;
   for (int s = 0; s < n_seq; ++s) {
     if (ctx->n_hi[ids[s]] + Ms > cfg.max_ctx) {
@@ -594,16 +617,18 @@ static int step_impl(firp_ctx *ctx, int32_t n_seq, const int32_t *seq_ids, const
   }
   ctx->launches = 0;
   if ((rc = upload_i32(ctx, ctx->seq_ids, ids.data(), n_seq, ctx->last_seq_ids, st))) return rc;
-  if ((rc = upload_i32(ctx, ctx->parents, tree_parents, T, ctx->last_parents, st))) return rc;
+  if ((rc = upload_i32(ctx, ctx->parents, dev_parents.data(), n_trees * T, ctx->last_parents, st))) return rc;
   const int32_t one = -1;
   const int T_next = (k > 0) ? T : 1;
-  if ((rc = upload_i32(ctx, ctx->next_parents, k > 0 ? tree_parents : &one, T_next, ctx->last_next_parents, st))) return rc;
+  if ((rc = upload_i32(ctx, ctx->next_parents, k > 0 ? dev_parents.data() : &one, k > 0 ? n_trees * T : 1, ctx->last_next_parents, st))) return rc;
+  if (tree_sizes && (rc = upload_i32(ctx, ctx->tree_sizes, tree_sizes, n_seq, ctx->last_sizes, st))) return rc;
 
   RunArgs ra{};
   ra.rw = Rows{n_seq, T, pseudo, Ms, n_seq * Ms, 0, chains ? 1 : 0, k, ctx->pseudo_masked};
   for (int i = 0; i < k; ++i) ra.tl[i] = layers[i];
   ra.d_tokens = d_tree_tokens; ra.want_head = true; ra.prefill_last_row = -1; ra.T_next = T_next;
   ra.out = out; ra.logits_dst = (out && out->logits) ? out->logits : ctx->logits; ra.n_hi_max = n_hi_max;
+  ra.parents_stride = tree_sizes ? T : 0; ra.d_sizes = tree_sizes ? ctx->tree_sizes : nullptr;
   if ((rc = run_rows(ctx, ra, st))) return rc;
   ctx->stepped = true; ctx->last_n_seq = n_seq; ctx->last_T = T; ctx->last_k = k;
   return FIRP_OK;

@@ -73,8 +73,9 @@ struct TreeMeta {
   uint32_t *mask;      // [R][kMaskWords] bit u: row v attends to new row u of its sequence
   float2 *rope;        // [R][dh/2] (cos, sin) of pos * theta^(-2c/dh)
 };
+// d_parents: [T] shared by the sequences (parents_stride 0) or [n_seq][T] (parents_stride T).
 // zero_word (may be NULL): a device word the kernel clears (the arrival counter of the fused decoder kernel)
-void launch_tree_prep(const Rows &rw, const int32_t *d_parents, const int32_t *d_seq_ids, const int32_t *d_ctx_len,
+void launch_tree_prep(const Rows &rw, const int32_t *d_parents, int parents_stride, const int32_t *d_seq_ids, const int32_t *d_ctx_len,
                       int dh, float theta, TreeMeta meta, int32_t *out_depth, uint32_t *out_mask, int out_mask_words,
                       unsigned *zero_word, bool pdl, cudaStream_t st);
 
@@ -118,8 +119,10 @@ void launch_topb(const float *logits, int R, int V, int B, int32_t *cand_ids, fl
 
 struct AcceptArgs {
   const int32_t *tokens;        // [n_seq][T]
-  const int32_t *parents;       // [T]
-  const int32_t *next_parents;  // [T_next]
+  const int32_t *parents;       // [T], or [n_seq][T] with parents_stride = T
+  const int32_t *next_parents;  // [T_next], likewise
+  int parents_stride;           // 0: one template for every sequence
+  const int32_t *sizes;         // NULL, or [n_seq]: nodes of each sequence's own tree (the rest of its T rows is padding)
   const int32_t *top_ids;       // [R][B] (row r's candidates; [0] is the argmax)
   const float *top_vals;        // [R][B]
   int T_next, B, S;             // S = path stride

@@ -12,7 +12,7 @@ namespace firp {
 // depth, absolute position, ancestor-or-self bitmask, rotary table.
 // One CTA per sequence; the extended parent array lives in shared memory.
 // ---------------------------------------------------------------------------
-__global__ void tree_prep_kernel(Rows rw, const int32_t *parents, const int32_t *seq_ids,
+__global__ void tree_prep_kernel(Rows rw, const int32_t *parents, int parents_stride, const int32_t *seq_ids,
                                  const int32_t *ctx_len, int dh, float theta, TreeMeta meta,
                                  int32_t *out_depth, uint32_t *out_mask, int out_mask_words, unsigned *zero_word, int pdl) {
   __shared__ int32_t ext[kMaxTreeRows];
@@ -23,7 +23,7 @@ __global__ void tree_prep_kernel(Rows rw, const int32_t *parents, const int32_t 
   const int n = ctx_len[seq_ids[s]];
   for (int v = tid; v < rw.Ms; v += blockDim.x) {
     int p;
-    if (v < rw.T) p = parents[v];
+    if (v < rw.T) p = parents[s * parents_stride + v];     // stride 0: one template for every sequence
     else if (rw.chains) p = v - rw.T;   // step 1 of node u (row T + u) hangs off u, step i off step i-1 of the same node
     else p = (v == rw.T) ? rw.anchor : v - 1;
     ext[v] = p;
@@ -66,10 +66,10 @@ __global__ void tree_prep_kernel(Rows rw, const int32_t *parents, const int32_t 
   }
 }
 
-void launch_tree_prep(const Rows &rw, const int32_t *d_parents, const int32_t *d_seq_ids, const int32_t *d_ctx_len,
+void launch_tree_prep(const Rows &rw, const int32_t *d_parents, int parents_stride, const int32_t *d_seq_ids, const int32_t *d_ctx_len,
                       int dh, float theta, TreeMeta meta, int32_t *out_depth, uint32_t *out_mask, int out_mask_words,
                       unsigned *zero_word, bool pdl, cudaStream_t st) {
-  launch_k(tree_prep_kernel, dim3(rw.n_seq), dim3(256), 0, st, pdl, rw, d_parents, d_seq_ids, d_ctx_len, dh, theta, meta,
+  launch_k(tree_prep_kernel, dim3(rw.n_seq), dim3(256), 0, st, pdl, rw, d_parents, parents_stride, d_seq_ids, d_ctx_len, dh, theta, meta,
            out_depth, out_mask, out_mask_words, zero_word, pdl ? 1 : 0);
 }
 
@@ -240,6 +240,9 @@ __global__ void accept_kernel(Rows rw, AcceptArgs a, int pdl) {
   if (pdl) { griddep_launch(); griddep_wait(); }
   const int s = blockIdx.x, tid = threadIdx.x;
   const int32_t *tok = a.tokens + (size_t)s * rw.T;
+  // own tree of the sequence (rows beyond its size are padding and can neither be accepted nor take a candidate)
+  const int32_t *parents = a.parents + (size_t)s * a.parents_stride, *next_parents = a.next_parents + (size_t)s * a.parents_stride;
+  const int Ts = a.sizes ? min(a.sizes[s], rw.T) : rw.T, Tn = a.sizes ? min(a.sizes[s], a.T_next) : a.T_next;
   for (int v = tid; v < rw.T; v += blockDim.x) {
     const int32_t b = a.top_ids[(size_t)(s * rw.Ms + v) * a.B];
     s_best[v] = b;
@@ -255,8 +258,8 @@ __global__ void accept_kernel(Rows rw, AcceptArgs a, int pdl) {
     } else {
       while (na + 1 < a.S) {
         int next = -1;
-        for (int ch = cur + 1; ch < rw.T; ++ch)
-          if (a.parents[ch] == cur && tok[ch] == s_best[cur]) { next = ch; break; }
+        for (int ch = cur + 1; ch < Ts; ++ch)
+          if (parents[ch] == cur && tok[ch] == s_best[cur]) { next = ch; break; }
         if (next < 0) break;
         acc[na] = tok[next];
         path[++na] = next;
@@ -288,13 +291,13 @@ __global__ void accept_kernel(Rows rw, AcceptArgs a, int pdl) {
   }
   for (int v = tid; v < a.T_next; v += blockDim.x) {
     int32_t t;
-    if (v == 0) {
+    if (v == 0 || v >= Tn) {
       t = s_bonus;
     } else {
       int dep = 0;
-      for (int u = v; u > 0 && dep <= a.T_next; u = a.next_parents[u]) ++dep;
+      for (int u = v; u > 0 && dep <= a.T_next; u = next_parents[u]) ++dep;
       int rank = 0;
-      for (int u = 1; u < v; ++u) rank += (a.next_parents[u] == a.next_parents[v]);
+      for (int u = 1; u < v; ++u) rank += (next_parents[u] == next_parents[v]);
       dep = min(dep, max(steps, 1));
       rank = min(rank, a.B - 1);
       t = (steps > 0) ? a.top_ids[(row0 + (size_t)(dep - 1) * row_step) * a.B + rank] : s_bonus;

@@ -153,6 +153,20 @@ def cache_row(engine, seq, pos):
     return int(table[seq, pos // 64]) * 64 + pos % 64
 
 
+def own_tree_view(g, Ts, T, k):
+    """Outputs of a sequence whose own tree has Ts of the T tree rows (firp_step_trees): drop the padding rows
+    Ts..T-1 so that the rows are those of an oracle step on the Ts-node tree (tree rows, then the k pseudo rows)."""
+    keep = list(range(Ts)) + list(range(T, T + k))
+    dense = unpack_mask(g["mask"], T + k)[np.ix_(keep, keep)]
+    words = np.zeros((len(keep), (len(keep) + 31) // 32), np.uint32)
+    for u in range(len(keep)):
+        words[:, u >> 5] |= dense[:, u].astype(np.uint32) << np.uint32(u & 31)
+    out = dict(g)
+    out.update(depth=g["depth"][keep], mask=words, logits=g["logits"][keep], best=g["best"][:Ts],
+               next_tokens=g["next_tokens"][:Ts])
+    return out
+
+
 def read_gpu_cache(engine, seq, layer, which, slot):
     import torch
     s = engine.shape

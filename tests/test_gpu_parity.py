@@ -295,6 +295,48 @@ def test_c1_paged_cache(torch_cuda, c1, fused):
     eng.close()
 
 
+@pytest.mark.parametrize("fused", [False, True])
+def test_c1_a_tree_of_its_own_for_every_sequence(torch_cuda, c1, fused):
+    """firp_step_trees: three sequences stepped together, each with its own tree shape and size (8, 5 and 3 of the
+    T = 8 rows), its own context length; every sequence is compared with an oracle step on ITS tree (the padding
+    rows dropped), both sides commit the oracle's path and take the oracle's next tree on the sequence's own shape.
+    A token that would be accepted is planted in a padding row: it must not be."""
+    import torch
+    from lockstep import own_tree_view
+    shape = si.scaled(c1, Hkv=2)
+    weights = si.all_weights(shape, gains=True)
+    T, k, l = 8, 3, 1
+    trees = [si.tree_template(8), si.random_tree(8, 5, 3, 1), si.chain_template(3)]
+    sizes = np.array([len(t) for t in trees], np.int32)
+    parents = np.full((3, T), 7, np.int32)                    # whatever lies beyond a tree's size is ignored
+    for s_i, t in enumerate(trees):
+        parents[s_i, : len(t)] = t
+    eng, orc = make_pair(shape, weights, 256, max_batch=3, fused=fused)
+    tokens = np.zeros((3, T), np.int32)
+    for s_i, n in enumerate((40, 9, 77)):
+        pout = eng.new_out(1, 1, k, T_next=len(trees[s_i]))
+        eng.prefill(s_i, torch.from_numpy(si.prompt(shape, seq=s_i, length=n)).cuda(), k, l, trees[s_i], pout)
+        ref = orc.prefill(si.prompt(shape, seq=s_i, length=n), k, l, trees[s_i], seq=s_i)
+        tokens[s_i, : sizes[s_i]] = ref["next_tokens"]
+    out = eng.new_out(3, T, k)
+    st = Stats()
+    for step in range(5):
+        refs = [orc.step(tokens[s_i, : sizes[s_i]], trees[s_i], k, l, seq=s_i) for s_i in range(3)]
+        for s_i in (1, 2):                                    # the padding rows carry the token the root would accept
+            tokens[s_i, sizes[s_i]:] = refs[s_i]["best"][0]
+        eng.step_trees(torch.from_numpy(tokens).cuda(), parents, sizes, k, l, out, seq_ids=[0, 1, 2])
+        for s_i in range(3):
+            g = own_tree_view(gpu_outputs(out, s_i, T, k), int(sizes[s_i]), T, k)
+            compare_step(shape, trees[s_i], tokens[s_i, : sizes[s_i]], k, g, refs[s_i], st)
+        eng.commit(3, seq_ids=[0, 1, 2], path=[r["path"] for r in refs])
+        for s_i in range(3):
+            orc.commit(refs[s_i]["path"], seq=s_i)
+            assert eng.context_len(s_i) == orc.context_len(s_i)
+            tokens[s_i, : sizes[s_i]] = refs[s_i]["next_tokens"]
+    assert st.steps == 15
+    eng.close()
+
+
 def test_chains_need_the_row_capacity(torch_cuda, c1, c1_weights):
     import torch
     from paper_2410_20488_b200 import FirpError, binding
