@@ -248,6 +248,15 @@ int firp_set_activation_planes(firp_ctx *ctx, int32_t qkv, int32_t o, int32_t ga
 int firp_set_attention_planes(firp_ctx *ctx, int32_t q_planes, int32_t p_planes);
 
 /*
+ * Which kernel computes the tree attention (Section 3.4) in the kernel-per-operation mode when head_dim is 128:
+ * tensor_core != 0: tiles of 128 cached positions as the M dimension of tcgen05 MMAs (S^T = K Q^T,
+ * O^T = V^T P^T, accumulators in tensor memory, K/V tiles by TMA); 0 (default): the warp-level mma.sync kernel
+ * with 64-position tiles, which is also what head_dim 64 and the persistent kernel always use.  Both compute the
+ * same masked softmax with (hi, lo) bf16 planes of Q and P and fp32 accumulation; summation orders differ.
+ */
+int firp_set_attention_kernel(firp_ctx *ctx, int32_t tensor_core);
+
+/*
  * How the decoder layers of a step are launched (Section 3.4 describes one forward pass per round; the
  * paper gives no kernel design).  on != 0: a step of at most 48 rows over all its sequences runs its
  * layers, Eq. 3 and the lm-head as ONE persistent kernel (6 launches per step instead of ~300) whose weight

@@ -9,4 +9,4 @@ from .binding import (FirpError, FirpEngine, StepOut, firp_create, firp_destroy,
                       firp_step, firp_kv_commit, firp_context_len, firp_set_context_len,
                       firp_last_launch_count, firp_profile_enable, firp_profile_read,
                       firp_kernel_class_name, firp_topb_static, firp_prefill_layers, firp_step_layers, firp_step_chains, firp_step_trees, firp_set_pseudo_masked,
-                      firp_set_fused, firp_set_pred_prenorm, firp_set_kv_pages, firp_set_activation_planes, firp_set_attention_planes, firp_set_wait_limit_us, firp_selftest_wait, lib_path, load_library, ModelCfg, Weights, StepOutC)
+                      firp_set_fused, firp_set_pred_prenorm, firp_set_kv_pages, firp_set_activation_planes, firp_set_attention_planes, firp_set_attention_kernel, firp_set_wait_limit_us, firp_selftest_wait, lib_path, load_library, ModelCfg, Weights, StepOutC)

@@ -47,7 +47,7 @@ EXPORTS = ("firp_create", "firp_destroy", "firp_last_error", "firp_workspace_byt
            "firp_context_len", "firp_set_context_len", "firp_last_launch_count", "firp_profile_enable",
            "firp_profile_read", "firp_kernel_class_name", "firp_topb_static", "firp_prefill_layers", "firp_step_layers", "firp_step_chains", "firp_set_pseudo_masked",
            "firp_set_fused", "firp_set_wait_limit_us", "firp_selftest_wait", "firp_set_pred_prenorm", "firp_set_kv_pages",
-           "firp_set_activation_planes", "firp_set_attention_planes", "firp_step_trees")
+           "firp_set_activation_planes", "firp_set_attention_planes", "firp_set_attention_kernel", "firp_step_trees")
 
 
 def lib_path() -> str:
@@ -83,6 +83,7 @@ def load_library():
     lib.firp_set_pseudo_masked.argtypes = [vp, i32]
     lib.firp_set_fused.argtypes = [vp, i32]
     lib.firp_set_attention_planes.argtypes = [vp, i32, i32]
+    lib.firp_set_attention_kernel.argtypes = [vp, i32]
     lib.firp_set_activation_planes.argtypes = [vp, i32, i32, i32, i32, i32]
     lib.firp_set_kv_pages.argtypes = [vp, vp, vp]
     lib.firp_set_pred_prenorm.argtypes = [vp, i32]
@@ -235,6 +236,10 @@ def firp_set_activation_planes(ctx, qkv=3, o=2, gate_up=2, down=2, lm_head=2):
 
 def firp_set_attention_planes(ctx, q_planes=2, p_planes=2):
     _check(ctx, load_library().firp_set_attention_planes(ctx, q_planes, p_planes))
+
+
+def firp_set_attention_kernel(ctx, tensor_core=True):
+    _check(ctx, load_library().firp_set_attention_kernel(ctx, 1 if tensor_core else 0))
 
 
 def firp_set_fused(ctx, on: bool):
@@ -418,6 +423,9 @@ class FirpEngine:
 
     def set_attention_planes(self, q_planes=2, p_planes=2):
         firp_set_attention_planes(self.ctx, q_planes, p_planes)
+
+    def set_attention_kernel(self, tensor_core=True):
+        firp_set_attention_kernel(self.ctx, tensor_core)
 
     def set_fused(self, on: bool):
         firp_set_fused(self.ctx, on)

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfirp_b200.so")
-SOURCES = ["firp_api.cu", "small_kernels.cu", "gemm_tcgen05.cu", "finish_kernels.cu", "attn_tree.cu", "fused_step.cu",
+SOURCES = ["firp_api.cu", "small_kernels.cu", "gemm_tcgen05.cu", "finish_kernels.cu", "attn_tree.cu", "attn_tc.cu", "fused_step.cu",
            "topb_static.cu"]
 HEADERS = ["firp_kernels.cuh", "launch_util.cuh", "tc_device.cuh", "finish_device.cuh", "norm_device.cuh", "attn_device.cuh",
            os.path.join("..", "..", "include", "firp.h")]

@@ -85,6 +85,7 @@ struct firp_ctx {
   int pseudo_masked = 0;     // Section 4.3 "Masked": pseudo rows do not see one another
   int pred_prenorm = 0;      // Eq. 3 reads the anchor through the insertion layer's input RMSNorm
   int planes[5] = {2, 2, 2, 2, 2};
+  bool attn_tc = false;              // head dimension 128: the tcgen05 attention kernel instead of the mma.sync one
   int attn_planes[2] = {2, 2};       // of the queries and of the probabilities in the attention   // bf16 planes of the activations per GEMM class: qkv, o, gate/up, down, lm-head
 
   // cache layout [layer][K|V][row][kv_head][head_dim]; row = slot * max_ctx + position, or through the page table
@@ -336,7 +337,13 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       const int tiles = (ra.n_hi_max + act + kAttnTile - 1) / kAttnTile;
       const int G = H / Hkv, qblocks = (act * G + 63) / 64;
       a.splits = attention_splits(rw.n_seq * Hkv * qblocks, tiles);
-      a.o = c->o; a.o_lo_off = Rp * nq;
+      a.o = c->o; a.o_lo_off = Rp * nq; a.err = c->dev_status; a.wait_ns = c->wait_ns;
+      const bool tc = c->attn_tc && dh == 128;
+      if (tc) {
+        int qb_tc, qper_tc;
+        attention_tc_blocks(act * G, &qb_tc, &qper_tc);
+        a.splits = attention_tc_splits(rw.n_seq * Hkv * qb_tc, (ra.n_hi_max + act + kAttnTcTile - 1) / kAttnTcTile, c->sm_count);
+      }
       // Early (programmatic) launch of the attention pays only when the rotary finisher before it has at least one
       // CTA per SM.  Measured at the 7B shape, ms per step with / without it: 35 rows 3.61 / 3.76 at 512 cached
       // tokens and 5.25 / 5.44 at 8192; 67 and 131 rows likewise 0.1 ms better with it; but 19 rows 3.68 / 3.60 and
@@ -344,7 +351,7 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       const int half_dh = dh / 2, qkv_st = (H + 2 * Hkv + 128 / half_dh - 1) / (128 / half_dh);
       const bool attn_early = pdl && (qkv_st * rw.R * 32 + 255) / 256 >= c->sm_count;
       FIRP_TIMED(KC_ATTENTION);
-      FIRP_CUDA(c, launch_attention(a, attn_early, st)); ++nl;
+      FIRP_CUDA(c, tc ? launch_attention_tc(a, attn_early, st) : launch_attention(a, attn_early, st)); ++nl;
     }
     {
       GemmArgs g = gemm_base(c->o, Rp * nq, c->wo[j], d, nq, act);
@@ -745,6 +752,12 @@ int firp_set_activation_planes(firp_ctx *ctx, int32_t qkv, int32_t o, int32_t ga
 int firp_set_attention_planes(firp_ctx *ctx, int32_t q_planes, int32_t p_planes) {
   if (!ctx || q_planes < 1 || q_planes > 2 || p_planes < 1 || p_planes > 2) return FIRP_ERR_BAD_ARG;
   ctx->attn_planes[0] = q_planes; ctx->attn_planes[1] = p_planes;
+  return FIRP_OK;
+}
+
+int firp_set_attention_kernel(firp_ctx *ctx, int32_t tensor_core) {
+  if (!ctx) return FIRP_ERR_BAD_ARG;
+  ctx->attn_tc = tensor_core != 0;
   return FIRP_OK;
 }
 

@@ -213,10 +213,17 @@ struct AttnArgs {
   int splits;                 // kv splits (grid.x = cluster size): 1, 2, 4 or 8
   int q_planes, p_planes;     // bf16 planes of the queries / of the probabilities that enter the tensor cores: 2 (hi, lo) or 1
   bf16 *o; size_t o_lo_off;   // [R][H*dh] hi plane, lo plane
+  int *err; unsigned long long wait_ns;   // status word and bound of the device-side waits (tensor-core kernel; 0: default)
 };
 // kv splits for `groups` = sequences x kv heads x query blocks and `kv_tiles` 64-position tiles
 int attention_splits(int groups, int kv_tiles);
 cudaError_t launch_attention(const AttnArgs &a, bool pdl, cudaStream_t st);
+// The tcgen05 kernel (head dimension 128): 128-position tiles, query blocks of at most kAttnTcMaxCols columns
+// (query rows x heads of the group), a.splits from attention_tc_splits.
+constexpr int kAttnTcTile = 128, kAttnTcMaxCols = 80;
+void attention_tc_blocks(int qrows, int *qblocks, int *qper);
+int attention_tc_splits(int groups, int kv_tiles, int sm_count);
+cudaError_t launch_attention_tc(const AttnArgs &a, bool pdl, cudaStream_t st);
 
 // ---- the decoder layers of a step as one persistent kernel (fused_step.cu) ------------------------------
 struct FusedShape { int L, d, H, Hkv, dh, F, V, max_ctx; float eps; };

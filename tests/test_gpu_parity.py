@@ -337,6 +337,52 @@ def test_c1_a_tree_of_its_own_for_every_sequence(torch_cuda, c1, fused):
     eng.close()
 
 
+# ---- head dimension 128: the tcgen05 attention kernel (and the mma.sync one on the same cases) ----------------
+def dh128_shape(c1, H, Hkv):
+    return si.scaled(c1, d=256, H=H, Hkv=Hkv, dh=128, F=512)
+
+
+@pytest.mark.parametrize("tensor_core", [True, False])
+@pytest.mark.parametrize("case", range(6))
+def test_dh128_tree_sizes_and_contexts(torch_cuda, c1, case, tensor_core):
+    """Tree sizes that select every query-block width of the tensor-core kernel (16, 32, 48, 80 columns, and two
+    blocks at 131 rows), contexts that end just below, on and above a 128-position tile boundary (so that the new
+    rows straddle tiles and the last tile is ragged), one to several tiles per split; gains non-unit."""
+    T, k, n0, steps = ((1, 0, 5, 3), (8, 3, 126, 4), (24, 3, 128, 4), (40, 3, 250, 4), (64, 3, 383, 3), (128, 3, 700, 3))[case]
+    shape = dh128_shape(c1, 2, 2)
+    weights = si.all_weights(shape, gains=True)
+    parents = si.chain_template(1) if T == 1 else si.random_tree(31, T, max(k, 1), case)
+    eng, orc = make_pair(shape, weights, 1024, max_tree=128, max_k=3, max_depth=3)
+    eng.set_attention_kernel(tensor_core)
+    st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=n0), steps, k=k, l=1, forced_steps=(1,))
+    assert st.steps == steps
+    eng.close()
+
+
+@pytest.mark.parametrize("tensor_core", [True, False])
+@pytest.mark.parametrize("Hkv", [2, 1])
+def test_dh128_grouped_queries_batch_and_pages(torch_cuda, c1, Hkv, tensor_core):
+    """4 query heads on 2 or 1 key/value heads (35 x 2 = 70 query columns in one block; 35 x 4 = 140 in two), three
+    sequences of different context lengths in one step, then the same engine with the cache scattered over pages."""
+    from lockstep import lockstep_run_batch
+    shape = dh128_shape(c1, 4, Hkv)
+    weights = si.all_weights(shape, gains=True)
+    parents = si.tree_template(32)
+    eng, orc = make_pair(shape, weights, 512, max_batch=3, max_tree=32, max_k=3, max_depth=3)
+    eng.set_attention_kernel(tensor_core)
+    prompts = [si.prompt(shape, seq=0, length=300), si.prompt(shape, seq=1, length=7), si.prompt(shape, seq=2, length=129)]
+    st = lockstep_run_batch(eng, orc, shape, parents, prompts, 4)
+    assert st.steps == 12
+    pages = 3 * 512 // 64
+    table = si.uniform_i32(6, si.stream_id("tokens", 78), pages, 0, 1 << 20).argsort().astype(np.int32).reshape(3, -1)
+    eng.set_kv_pages(table)
+    st = lockstep_run_batch(eng, orc, shape, parents, [p[:n] for p, n in zip(prompts, (190, 60, 255))], 4)
+    assert st.steps == 12
+    st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=120), 4, forced=True, seq=2, check_cache_rows=True)
+    assert st.steps == 4
+    eng.close()
+
+
 def test_chains_need_the_row_capacity(torch_cuda, c1, c1_weights):
     import torch
     from paper_2410_20488_b200 import FirpError, binding
