@@ -48,8 +48,8 @@ def parse():
     ap.add_argument("--no-kernel-times", action="store_true", help="skip the per-kernel event-timed pass")
     ap.add_argument("--fused", type=int, default=-1, choices=[-1, 0, 1], help="1: the decoder layers of a step as one persistent "
                     "kernel, 0: one kernel per operation, -1: the library's default")
-    ap.add_argument("--attention", default="mma", choices=["tc", "mma"], help="tree attention at head_dim 128: the mma.sync kernel "
-                    "(the library's default) or the tcgen05 one")
+    ap.add_argument("--attention", default="auto", choices=["auto", "tc", "mma"], help="tree attention at head_dim 128: chosen per "
+                    "step (the library's default), the tcgen05 kernel or the mma.sync one")
     ap.add_argument("--no-forced", action="store_true", help="skip the forced-accept run")
     ap.add_argument("--sweep", action="store_true", help="config-4 sweep on the c2 weights: T x context, one JSON line per point")
     return ap.parse_args()
@@ -363,7 +363,7 @@ def run_sweep(args, shape, weights, dev, rank):
                      max_depth=3, device=str(dev))
     if args.fused >= 0:
         eng.set_fused(bool(args.fused))
-    eng.set_attention_kernel(args.attention == "tc")
+    eng.set_attention_kernel({"auto": None, "tc": True, "mma": False}[args.attention])
     peaks = {}
     try:
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
@@ -454,7 +454,7 @@ def main():
     eng = FirpEngine(shape, weights, max_ctx=max_ctx, max_batch=B, device=str(dev), max_rows=B * rows_per_seq if chains else 0)
     if args.fused >= 0:
         eng.set_fused(bool(args.fused))
-    eng.set_attention_kernel(args.attention == "tc")
+    eng.set_attention_kernel({"auto": None, "tc": True, "mma": False}[args.attention])
     step_fn = eng.step_chains if chains else eng.step
     T_next = shape.T if shape.k > 0 else 1
     outs = [eng.new_out(B, shape.T, shape.k, want_logits=False, chains=chains) for _ in range(2)]

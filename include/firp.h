@@ -248,11 +248,14 @@ int firp_set_activation_planes(firp_ctx *ctx, int32_t qkv, int32_t o, int32_t ga
 int firp_set_attention_planes(firp_ctx *ctx, int32_t q_planes, int32_t p_planes);
 
 /*
- * Which kernel computes the tree attention (Section 3.4) in the kernel-per-operation mode when head_dim is 128:
- * tensor_core != 0: tiles of 128 cached positions as the M dimension of tcgen05 MMAs (S^T = K Q^T,
- * O^T = V^T P^T, accumulators in tensor memory, K/V tiles by TMA); 0 (default): the warp-level mma.sync kernel
- * with 64-position tiles, which is also what head_dim 64 and the persistent kernel always use.  Both compute the
- * same masked softmax with (hi, lo) bf16 planes of Q and P and fp32 accumulation; summation orders differ.
+ * Which kernel computes the tree attention (Section 3.4) in the kernel-per-operation mode when head_dim is 128.
+ * tensor_core = 1: tiles of 128 cached positions as the M dimension of tcgen05 MMAs (S^T = K Q^T, O^T = V^T P^T,
+ * accumulators in tensor memory, K/V tiles by TMA, two warpgroups alternating over the tiles); 0: the warp-level
+ * mma.sync kernel with 64-position tiles, which is also what head_dim 64 and the persistent kernel always use;
+ * -1 (default): chosen per step -- the tensor-core kernel once the longest context of the step spans at least
+ * three of its tiles (four when the query columns, rows x heads per kv head, need more than one block of 48),
+ * the mma.sync kernel for shorter contexts, where its lower fixed cost wins.  Both compute the same masked softmax with (hi, lo) bf16 planes of Q
+ * and P and fp32 accumulation; summation orders differ.  Other values: FIRP_ERR_BAD_ARG.
  */
 int firp_set_attention_kernel(firp_ctx *ctx, int32_t tensor_core);
 

@@ -238,8 +238,9 @@ def firp_set_attention_planes(ctx, q_planes=2, p_planes=2):
     _check(ctx, load_library().firp_set_attention_planes(ctx, q_planes, p_planes))
 
 
-def firp_set_attention_kernel(ctx, tensor_core=True):
-    _check(ctx, load_library().firp_set_attention_kernel(ctx, 1 if tensor_core else 0))
+def firp_set_attention_kernel(ctx, tensor_core=None):
+    """True: the tcgen05 kernel, False: the mma.sync kernel, None: chosen per step (the default)."""
+    _check(ctx, load_library().firp_set_attention_kernel(ctx, -1 if tensor_core is None else (1 if tensor_core else 0)))
 
 
 def firp_set_fused(ctx, on: bool):
@@ -424,7 +425,7 @@ class FirpEngine:
     def set_attention_planes(self, q_planes=2, p_planes=2):
         firp_set_attention_planes(self.ctx, q_planes, p_planes)
 
-    def set_attention_kernel(self, tensor_core=True):
+    def set_attention_kernel(self, tensor_core=None):
         firp_set_attention_kernel(self.ctx, tensor_core)
 
     def set_fused(self, on: bool):

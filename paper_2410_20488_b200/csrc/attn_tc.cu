@@ -2,20 +2,22 @@
 // for the pseudo rows), head dimension 128.
 //
 // Roles are swapped as in the GEMMs: a tile of 128 cached positions is the MMA's M dimension, the query rows of
-// the block (tree rows x heads of the group, <= 80) its N dimension.
+// the block (tree rows x heads of the group, <= 48) its N dimension.
 //   S^T = K Q^T      K tile [128 pos][128 dh] K-major (TMA, 128-byte swizzle), Q [NQ][128] K-major (hi and lo
-//                    bf16 planes, both accumulated into the same fp32 columns)           -> TMEM columns [0, NQ)
-//   softmax          thread i owns position i of the tile (= TMEM lane i): scale, visibility, column maxima over
-//                    the 128 positions (warp reduction + shared memory), P = 2^(s - m) as bf16 (hi, lo) planes
-//                    written to shared memory as [NQ][128 pos] K-major
-//   O^T = V^T P^T    V tile [128 pos][128 dh] as the MN-major A operand (M = dh)         -> TMEM columns [NQ, 2NQ)
-//   l^T = 1 P^T      an all-ones A tile: every lane receives the column sums of P        -> TMEM columns [2NQ, 3NQ)
-// The running (max, sum, O) of the online softmax live in shared memory / registers: thread i keeps O^T[i][*]
-// (dh index i, all query columns), rescaled per column when the maximum moves.  K and V tiles are double
-// buffered.  Grid = (kv split, kv head, sequence x query block), the splits of one (kv head, query block) form a
-// cluster and merge their partial results through distributed shared memory exactly like the mma.sync kernel.
-// One CTA per SM (shared memory), so the 256 TMEM columns it allocates are never contended.  Every mbarrier wait
-// is bounded; a wait that runs out sets the status word and the kernel runs to its end.
+//                    bf16 planes, both accumulated into the same fp32 columns)           -> NQ TMEM columns
+//   softmax          thread i of a warpgroup owns position i of the tile (= TMEM lane i): scale, visibility,
+//                    column maxima and sums over the 128 positions (warp butterflies + shared memory), P = 2^(s - m)
+//                    as bf16 (hi, lo) planes written to shared memory as [NQ][128 pos] K-major
+//   O^T = V^T P^T    V tile [128 pos][128 dh] as the MN-major A operand (M = dh)         -> NQ TMEM columns
+// A CTA keeps two tiles of its kv range in flight (tile groups 0 and 1 take the tiles in turn), each with its own
+// K, V and P buffers, TMEM columns and running (max, sum, O^T), so that the tensor-core work of one overlaps the
+// softmax of the other; the query columns of a tile are shared by two warpgroups (halves), which makes four
+// softmax warpgroups: thread i of each keeps O^T[i][its columns] (dh index i) in registers.  One thread issues
+// every MMA, two more feed the K and the V buffers by TMA.  The two partial results are merged in shared memory; the
+// CTAs of one (kv head, query block) -- the kv splits -- form a cluster and merge theirs by pushing each column
+// to the CTA that finalises it.  One CTA per SM (shared memory), so the 512 TMEM columns it allocates are never
+// contended.  Every mbarrier wait is bounded; a wait that runs out sets the status word and the kernel runs to
+// its end.
 #include <cooperative_groups.h>
 
 #include <map>
@@ -33,22 +35,24 @@ namespace {
 
 constexpr int kTcDh = 128;                  // head dimension this kernel is written for
 constexpr int kTcTile = 128;                // cached positions per tile (MMA M)
-constexpr int kTcThreads = 128;
+constexpr int kTcWg = 128;                  // threads of a warpgroup
+constexpr int kTcSoft = 4 * kTcWg;          // softmax threads: 2 tile groups x 2 column halves
+constexpr int kTcThreads = kTcSoft + 96;    // + the MMA issuer's warp, the K and the V producer's
 constexpr int kTcSlab = kTcTile * 128;      // bytes of one [128 rows][64 elements] slab
 constexpr int kTcStage = 2 * kTcSlab;       // a K or V tile: two slabs (dh halves)
 constexpr int kTcTmemCols = 256;
 
 template <int NQ> struct TcLayout {
   static constexpr int Q_SLAB = NQ * 128;                 // [NQ rows][64 elements]
-  static constexpr int K_OFF = 0;                         // [2 stages][2 dh halves][128 pos][128 B]
-  static constexpr int V_OFF = K_OFF + 2 * kTcStage;      // [2 stages][2 dh halves][128 pos][128 B]
-  static constexpr int ONES_OFF = V_OFF + 2 * kTcStage;   // [128 rows][16 elements], unswizzled
-  static constexpr int Q_OFF = ONES_OFF + 4096;           // [2 planes][2 dh halves][NQ][128 B]
-  static constexpr int P_OFF = Q_OFF + 4 * Q_SLAB;        // [2 planes][2 pos halves][NQ][128 B]
-  static constexpr int BYTES = P_OFF + 4 * Q_SLAB;
-  static_assert(NQ % 16 == 0 && NQ >= 16 && 3 * NQ <= kTcTmemCols, "query columns per block");
-  static_assert((NQ + 8) * kTcDh * 4 <= 2 * kTcStage, "a partial O^T must fit the key stages");
-  static_assert(BYTES + 1024 + 4096 <= 227 * 1024, "shared memory budget (dynamic + alignment + static)");
+  static constexpr int K_OFF = 0;                         // [2 warpgroups][2 dh halves][128 pos][128 B]
+  static constexpr int V_OFF = K_OFF + 2 * kTcStage;      // [2 warpgroups][2 dh halves][128 pos][128 B]
+  static constexpr int Q_OFF = V_OFF + 2 * kTcStage;      // [2 planes][2 dh halves][NQ][128 B]
+  static constexpr int P_OFF = Q_OFF + 4 * Q_SLAB;        // [2 warpgroups][2 planes][2 pos halves][NQ][128 B]
+  static constexpr int BYTES = P_OFF + 8 * Q_SLAB;
+  static_assert(NQ % 16 == 0 && NQ >= 16 && NQ <= 48 && 4 * NQ <= kTcTmemCols, "query columns per block");
+  static_assert(NQ * kTcDh * 4 <= kTcStage, "a warpgroup's partial O^T must fit its key buffer");
+  static_assert((NQ + 8) * kTcDh * 4 <= 2 * kTcStage, "the partials a CTA receives must fit the value buffers");
+  static_assert(BYTES + 1024 + 6144 <= 227 * 1024, "shared memory budget (dynamic + alignment + static)");
 };
 
 // MN-major operand, 128-byte swizzle: 64 elements of M contiguous (128 bytes), the 8 rows of a K group 128 bytes
@@ -58,9 +62,61 @@ __device__ __forceinline__ uint64_t smem_desc_mn(uint32_t addr, uint32_t lbo_byt
          ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-// order-preserving map float <-> int (its own inverse)
-__device__ __forceinline__ int f2ord(float f) { int b = __float_as_int(f); return b ^ ((b >> 31) & 0x7fffffff); }
-__device__ __forceinline__ float ord2f(int b) { return __int_as_float(b ^ ((b >> 31) & 0x7fffffff)); }
+__device__ __forceinline__ void wg_sync(int w) { asm volatile("bar.sync %0, 128;" ::"r"(1 + w) : "memory"); }
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, float *r) {
+  uint32_t *u = reinterpret_cast<uint32_t *>(r);
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7])
+               : "r"(taddr) : "memory");
+}
+// N = 8, 16 or 24 consecutive columns of this warp's lanes (no wait)
+template <int N> __device__ __forceinline__ void tc_ld_cols(uint32_t taddr, float *r) {
+  static_assert(N == 8 || N == 16 || N == 24, "columns per warpgroup");
+  if (N >= 16) tc_ld16(taddr, r);
+  if (N == 8) tc_ld8(taddr, r);
+  if (N == 24) tc_ld8(taddr + 16, r + 16);
+}
+// Reduction (max or sum) over the 32 lanes of N = 8 or 16 columns at once: in each butterfly step a lane keeps
+// half of its columns and trades the other half with its partner, so N columns cost N + log2(32 / N) - 1 shuffles
+// instead of 5 N.  Destroys v; lane L returns the result of column L * N / 32 (N = 16: L >> 1, N = 8: L >> 2).
+template <int N, bool SUM> __device__ __forceinline__ float warp_col_reduce(float *v, int lane) {
+  static_assert(N == 8 || N == 16, "columns per butterfly");
+  int m = 16;
+#pragma unroll
+  for (int half = N / 2; half >= 1; half >>= 1, m >>= 1) {
+    const bool up = (lane & m) != 0;
+#pragma unroll
+    for (int c = 0; c < half; ++c) {
+      const float got = __shfl_xor_sync(0xffffffffu, up ? v[c] : v[c + half], m);
+      const float kept = up ? v[c + half] : v[c];
+      v[c] = SUM ? kept + got : fmaxf(kept, got);
+    }
+  }
+#pragma unroll
+  for (; m >= 1; m >>= 1) {
+    const float got = __shfl_xor_sync(0xffffffffu, v[0], m);
+    v[0] = SUM ? v[0] + got : fmaxf(v[0], got);
+  }
+  return v[0];
+}
+// The same for NH = 8, 16 or 24 columns (a block of 16, then one of 8); the results go to dst[column][slot].
+template <int NH, bool SUM> __device__ __forceinline__ void warp_cols_to_smem(const float *v, float (*dst)[4], int slot, int lane) {
+  if (NH >= 16) {
+    float t[16];
+#pragma unroll
+    for (int c = 0; c < 16; ++c) t[c] = v[c];
+    const float r = warp_col_reduce<16, SUM>(t, lane);
+    if ((lane & 1) == 0) dst[lane >> 1][slot] = r;
+  }
+  if (NH == 8 || NH == 24) {
+    constexpr int o = NH == 24 ? 16 : 0;
+    float t[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) t[c] = v[o + c];
+    const float r = warp_col_reduce<8, SUM>(t, lane);
+    if ((lane & 3) == 0) dst[o + (lane >> 2)][slot] = r;
+  }
+}
 
 #ifdef FIRP_ATTN_TRACE
 __device__ unsigned long long g_attn_trace[16];
@@ -75,34 +131,43 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     int qper, int pdl) {
   using LY = TcLayout<NQ>;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(16) int s_red[NQ][4];        // per column: the four warps' maxima of the tile (order-mapped)
-  __shared__ __align__(16) float s_m[NQ];           // running max (log2 units)
-  __shared__ __align__(16) float s_corr[NQ];        // 2^(old max - new max) of the current tile
-  __shared__ __align__(16) float s_l[NQ];           // running sum
+  __shared__ __align__(16) float s_red[2][NQ][4];   // per tile group and column: its four warps' maxima of the tile
+  __shared__ __align__(16) float s_lred[2][NQ][4];  // and their sums of P, added to the running sum one tile later
+  __shared__ __align__(16) float s_m[2][NQ];        // running max (log2 units)
+  __shared__ __align__(16) float s_corr[2][NQ];     // 2^(old max - new max) of the current tile; merge weights at the end
+  __shared__ __align__(16) float s_l[2][NQ];        // running sum
   __shared__ float s_pm[NQ + kAttnMaxSplits], s_pl[NQ + kAttnMaxSplits];   // (max, sum) received for the merge: [split][slot]
-  __shared__ __align__(8) uint64_t s_bar[6];        // K landed [2], V landed [2], S^T complete, O^T and l^T complete
+  __shared__ uint32_t s_oidx[NQ];                   // element offset of each column's output row
+  // mbarriers: K landed [2], V landed [2], S^T complete [2], P written [2], O^T complete [2], Q written
+  __shared__ __align__(8) uint64_t s_bar[11];
   __shared__ uint32_t s_tmem;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   TC_STAMP(0);
   uint8_t *base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t sb = smem_u32(base);
-  const uint32_t bar0 = smem_u32(s_bar), bar_s = bar0 + 32, bar_o = bar0 + 40;
+  const uint32_t bar0 = smem_u32(s_bar);
+  const uint32_t full_k = bar0, full_v = bar0 + 16, s_ready = bar0 + 32, p_ready = bar0 + 48, o_ready = bar0 + 64,
+                 q_ready = bar0 + 80;               // [w] of a pair: + 8 w
 
   if (tid == 0) {
     for (int i = 0; i < 6; ++i) mbar_init(bar0 + 8 * i, 1);
+    mbar_init(p_ready, 2 * kTcWg); mbar_init(p_ready + 8, 2 * kTcWg);
+    mbar_init(o_ready, 1); mbar_init(o_ready + 8, 1);
+    mbar_init(q_ready, kTcSoft);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  {  // the all-ones A tile: [128 rows][16 elements], unswizzled 8 x 16-byte core matrices (4 KB)
-    const uint4 ones = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
-    uint4 *o = reinterpret_cast<uint4 *>(base + LY::ONES_OFF);
-    o[tid] = ones; o[tid + kTcThreads] = ones;
-  }
-  for (int j = tid; j < NQ; j += kTcThreads) { s_m[j] = -INFINITY; s_l[j] = 0.f; }
-  if (warp == 0) {
+  for (int j = tid; j < 2 * NQ * 4; j += kTcThreads) (&s_lred[0][0][0])[j] = 0.f;
+  for (int j = tid; j < 2 * NQ; j += kTcThreads) { (&s_m[0][0])[j] = -INFINITY; (&s_l[0][0])[j] = 0.f; }
+  if (warp == 16) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(kTcTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  fence_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
   if (pdl) { griddep_launch(); griddep_wait(); }
   TC_STAMP(1);
 
@@ -117,295 +182,325 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int kv_len = min(n + a.rows_active, a.max_ctx);
   const int tiles_total = (kv_len + kTcTile - 1) / kTcTile;
   const int t0 = (split * tiles_total + nsplits - 1) / nsplits, t1 = ((split + 1) * tiles_total + nsplits - 1) / nsplits;
+  const int ntiles = t1 - t0;                       // tile t0 + i goes to warpgroup i & 1 as its (i >> 1)-th
   const unsigned long long wait_ns = a.wait_ns ? a.wait_ns : kDefaultWaitNs;
   bool dead = false;
+  constexpr int NH = NQ / 2;                        // columns per warpgroup
+  float o_acc[NH];                                  // softmax threads: O^T[dh index][own columns] of the tiles so far
+#pragma unroll
+  for (int j = 0; j < NH; ++j) o_acc[j] = 0.f;
 
-  uint64_t pol = 0;
-  auto load_tile = [&](int st, int t) {             // thread 0: K and V of tile t as 64-position x 64-element boxes
-    mbar_expect_tx(bar0 + 8 * st, kTcStage);
-    mbar_expect_tx(bar0 + 16 + 8 * st, kTcStage);
+  if (warp >= 17) {
+    // ---- producers (one lane each): warp 17 feeds the K buffers, warp 18 the V buffers.  A buffer is free again
+    // when the MMAs that read it have completed, which is what s_ready / o_ready of its warpgroup report.
+    if (lane == 0) {
+      const bool is_v = warp == 18;
+      const CUtensorMap *tm = is_v ? &tmV : &tmK;
+      const uint32_t full = is_v ? full_v : full_k, freed = is_v ? o_ready : s_ready;
+      const uint32_t dst0 = sb + (is_v ? LY::V_OFF : LY::K_OFF);
+      uint64_t pol;
+      asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+      for (int i = 0; i < ntiles; ++i) {
+        const int w = i & 1, q = i >> 1, t = t0 + i;
+        if (q > 0) mbar_wait(freed + 8 * w, (q - 1) & 1, a.err, dead, wait_ns);
+        mbar_expect_tx(full + 8 * w, kTcStage);
 #pragma unroll
-    for (int ph = 0; ph < 2; ++ph) {
-      const int p0 = t * kTcTile + ph * 64;
-      const int row = (int)kv_row(a.pages, slot, p0 < kv_len ? p0 : 0, a.max_ctx);   // a half beyond the context: any rows
+        for (int ph = 0; ph < 2; ++ph) {            // 64-position x 64-element boxes; a half lies inside one page
+          const int p0 = t * kTcTile + ph * 64;
+          const int row = (int)kv_row(a.pages, slot, p0 < kv_len ? p0 : 0, a.max_ctx);   // a half beyond the context: any rows
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const uint32_t off = (uint32_t)(st * kTcStage + h * kTcSlab + ph * 8192);
-        tma_load_2d(sb + LY::K_OFF + off, &tmK, kvh * kTcDh + h * 64, row, bar0 + 8 * st, pol);
-        tma_load_2d(sb + LY::V_OFF + off, &tmV, kvh * kTcDh + h * 64, row, bar0 + 16 + 8 * st, pol);
+          for (int h = 0; h < 2; ++h)
+            tma_load_2d(dst0 + (uint32_t)(w * kTcStage + h * kTcSlab + ph * 8192), tm, kvh * kTcDh + h * 64, row,
+                        full + 8 * w, pol);
+        }
       }
     }
-  };
-  if (tid == 0) {
-    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
-    if (t0 < t1) load_tile(0, t0);
-    if (t0 + 1 < t1) load_tile(1, t0 + 1);
-  }
-  // queries of this block: column j = query row q0 + j -> (tree row (q0 + j) / G, head kvh G + (q0 + j) % G)
-  {
-    constexpr int IT = NQ * 16 / kTcThreads;          // 16-byte chunks per thread and plane
-    uint4 qh[IT], ql[IT];
+  } else if (warp == 16) {
+    // ---- MMA issuer (one lane): S^T of tile i, then O^T of tile i - 1
+    if (lane == 0) {
+      const uint32_t idesc_k = instr_desc_m128(NQ), idesc_mn = idesc_k | (1u << 15);
+      // operand descriptors of warpgroup 0; another buffer, dh half or k step only moves the start address
+      const uint64_t kdesc0 = smem_desc(sb + LY::K_OFF), qdesc0 = smem_desc(sb + LY::Q_OFF);
+      const uint64_t vdesc0 = smem_desc_mn(sb + LY::V_OFF, kTcSlab), pdesc0 = smem_desc(sb + LY::P_OFF);
+      mbar_wait(q_ready, 0, a.err, dead, wait_ns);
+      for (int i = 0; i <= ntiles; ++i) {
+        if (i < ntiles) {
+          const int w = i & 1, q = i >> 1;
+          mbar_wait(full_k + 8 * w, q & 1, a.err, dead, wait_ns);
+          if (q > 0) mbar_wait(p_ready + 8 * w, (q - 1) & 1, a.err, dead, wait_ns);   // S^T of its previous tile has been read
+          tc_fence_after();
+          uint32_t acc = 0;
+          for (int pl = 0; pl < a.q_planes; ++pl)
 #pragma unroll
-    for (int it = 0; it < IT; ++it) {                 // all loads in flight before the first store
-      const int idx = it * kTcThreads + tid, j = idx >> 4, c = idx & 15, qr = q0 + j;
-      qh[it] = make_uint4(0u, 0u, 0u, 0u); ql[it] = qh[it];
-      if (j < ncols) {
-        const bf16 *src = a.q + ((size_t)(s * a.rw.Ms + qr / G) * a.H + kvh * G + qr % G) * kTcDh + c * 8;
-        qh[it] = *reinterpret_cast<const uint4 *>(src);
-        ql[it] = *reinterpret_cast<const uint4 *>(src + a.q_lo_off);
+            for (int kk = 0; kk < 8; ++kk) {
+              tc_mma(tmem + w * 2 * NQ, kdesc0 + (uint64_t)((w * kTcStage + (kk >> 2) * kTcSlab + (kk & 3) * 32) >> 4),
+                     qdesc0 + (uint64_t)((pl * 2 * LY::Q_SLAB + (kk >> 2) * LY::Q_SLAB + (kk & 3) * 32) >> 4), idesc_k, acc);
+              acc = 1;
+            }
+          tc_commit(s_ready + 8 * w);
+        }
+        if (i >= 1) {
+          const int w = (i - 1) & 1, q = (i - 1) >> 1;
+          mbar_wait(p_ready + 8 * w, q & 1, a.err, dead, wait_ns);
+          mbar_wait(full_v + 8 * w, q & 1, a.err, dead, wait_ns);
+          tc_fence_after();
+          uint32_t acc = 0;
+          for (int pl = 0; pl < a.p_planes; ++pl)
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint64_t bdesc = pdesc0 + (uint64_t)((w * 4 * LY::Q_SLAB + pl * 2 * LY::Q_SLAB + (ks >> 2) * LY::Q_SLAB + (ks & 3) * 32) >> 4);
+              tc_mma(tmem + w * 2 * NQ + NQ, vdesc0 + (uint64_t)((w * kTcStage + ks * 2048) >> 4), bdesc, idesc_mn, acc);
+              acc = 1;
+            }
+          tc_commit(o_ready + 8 * w);
+        }
       }
     }
+  } else {
+    // ---- the four softmax warpgroups: tile group g takes tiles g, g + 2, ...; half h of it owns the query columns
+    // [h NH, (h + 1) NH) of those tiles
+    const int wgi = warp >> 2, g = wgi >> 1, h = wgi & 1, wt = tid & (kTcWg - 1);
+    const int c_lo = h * NH;
+    const uint32_t tlane = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(g * 2 * NQ + c_lo);
+    {
+      // queries of this block (all softmax threads share the work): column j = query row q0 + j -> (tree row
+      // (q0 + j) / G, head kvh G + (q0 + j) % G)
+      constexpr int IT = (NQ * 16 + kTcSoft - 1) / kTcSoft;
+      uint4 qh[IT], ql[IT];
 #pragma unroll
-    for (int it = 0; it < IT; ++it) {
-      const int idx = it * kTcThreads + tid, j = idx >> 4, c = idx & 15;
-      const int off = (c >> 3) * LY::Q_SLAB + j * 128 + (((c & 7) ^ (j & 7)) << 4);
-      *reinterpret_cast<uint4 *>(base + LY::Q_OFF + off) = qh[it];
-      *reinterpret_cast<uint4 *>(base + LY::Q_OFF + 2 * LY::Q_SLAB + off) = ql[it];
+      for (int it = 0; it < IT; ++it) {               // all loads in flight before the first store
+        const int idx = it * kTcSoft + tid, j = idx >> 4, c = idx & 15, qr = q0 + j;
+        qh[it] = make_uint4(0u, 0u, 0u, 0u); ql[it] = qh[it];
+        if (j < ncols) {
+          const bf16 *src = a.q + ((size_t)(s * a.rw.Ms + qr / G) * a.H + kvh * G + qr % G) * kTcDh + c * 8;
+          qh[it] = *reinterpret_cast<const uint4 *>(src);
+          ql[it] = *reinterpret_cast<const uint4 *>(src + a.q_lo_off);
+        }
+      }
+#pragma unroll
+      for (int it = 0; it < IT; ++it) {
+        const int idx = it * kTcSoft + tid, j = idx >> 4, c = idx & 15;
+        if (j < NQ) {
+          const int off = (c >> 3) * LY::Q_SLAB + j * 128 + (((c & 7) ^ (j & 7)) << 4);
+          *reinterpret_cast<uint4 *>(base + LY::Q_OFF + off) = qh[it];
+          *reinterpret_cast<uint4 *>(base + LY::Q_OFF + 2 * LY::Q_SLAB + off) = ql[it];
+        }
+      }
+      TC_STAMP(15);
+      fence_async_smem();
+      mbar_arrive(q_ready);
+      if (tid < ncols) {
+        const int qr = q0 + tid;
+        s_oidx[tid] = (uint32_t)(((s * a.rw.Ms + qr / G) * a.H + kvh * G + qr % G) * kTcDh);
+      }
     }
-  }
-  fence_async_smem();
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  TC_STAMP(2);
-  const uint32_t tmem = s_tmem;
-  const uint32_t tlane = tmem + ((uint32_t)(warp * 32) << 16);
+    TC_STAMP(2);
+    const float scale_log2 = rsqrtf((float)kTcDh) * 1.4426950408889634f;
+    // where this thread's position pair goes in a P row: 64-position half, 16-byte chunk, element
+    const int p_half = wt >> 6, p_chunk = (wt & 63) >> 3, p_el2 = wt & 6, odd = wt & 1;
+    uint8_t *pbase = base + LY::P_OFF + g * 4 * LY::Q_SLAB;
 
-  const uint32_t idesc_k = instr_desc_m128(NQ), idesc_mn = idesc_k | (1u << 15);
-  const uint64_t ones_desc = (uint64_t)(((sb + LY::ONES_OFF) & 0x3FFFFu) >> 4) | ((uint64_t)(128 >> 4) << 16) |
-                             ((uint64_t)(256 >> 4) << 32) | ((uint64_t)1 << 46);
-  // operand descriptors of stage 0; another stage, dh half or k step only moves the start address (16-byte units)
-  const uint64_t kdesc0 = smem_desc(sb + LY::K_OFF), qdesc0 = smem_desc(sb + LY::Q_OFF);
-  const uint64_t vdesc0 = smem_desc_mn(sb + LY::V_OFF, kTcSlab), pdesc0 = smem_desc(sb + LY::P_OFF);
-  auto issue_s = [&](int st) {                      // thread 0: S^T = K Q^T
-    uint32_t acc = 0;
-    for (int pl = 0; pl < a.q_planes; ++pl)
+    for (int i = g; i < ntiles; i += 2) {
+      const int q = i >> 1, t = t0 + i;
+      const int p = t * kTcTile + wt;
+      const bool pvalid = p < kv_len;
+      // visibility of position p for this half's query columns (bit jj = column c_lo + jj): the committed prefix
+      // is visible to all, new row u = p - n to the rows whose mask has bit u
+      uint32_t vis = pvalid ? ~0u : 0u;
+      if (pvalid && p >= n) {
+        const int u = p - n, mw = u >> 5, b = u & 31;
+        vis = 0u;
 #pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {
-        tc_mma(tmem, kdesc0 + (uint64_t)((st * kTcStage + (kk >> 2) * kTcSlab + (kk & 3) * 32) >> 4),
-               qdesc0 + (uint64_t)((pl * 2 * LY::Q_SLAB + (kk >> 2) * LY::Q_SLAB + (kk & 3) * 32) >> 4), idesc_k, acc);
-        acc = 1;
+        for (int jj = 0; jj < NH; ++jj) {
+          const int qr = min(q0 + c_lo + jj, qrows_total - 1);
+          const uint32_t word = a.mask[(size_t)(s * a.rw.Ms + qr / G) * kMaskWords + mw];
+          vis |= ((word >> b) & 1u) << jj;
+        }
       }
-    tc_commit(bar_s);
-  };
-  auto issue_o = [&](int st) {                      // thread 0: O^T = V^T P^T and l^T = 1 P^T
-    uint32_t acc = 0;
-    for (int pl = 0; pl < a.p_planes; ++pl)
-#pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        const uint64_t bdesc = pdesc0 + (uint64_t)((pl * 2 * LY::Q_SLAB + (ks >> 2) * LY::Q_SLAB + (ks & 3) * 32) >> 4);
-        tc_mma(tmem + NQ, vdesc0 + (uint64_t)((st * kTcStage + ks * 2048) >> 4), bdesc, idesc_mn, acc);
-        tc_mma(tmem + 2 * NQ, ones_desc, bdesc, idesc_k, acc);
-        acc = 1;
-      }
-    tc_commit(bar_o);
-  };
-
-  float o_acc[NQ];
-#pragma unroll
-  for (int j = 0; j < NQ; ++j) o_acc[j] = 0.f;
-  const float scale_log2 = rsqrtf((float)kTcDh) * 1.4426950408889634f;
-  // where this thread's position goes in a P row: 64-position half, 16-byte chunk, element
-  const int p_half = tid >> 6, p_chunk = (tid & 63) >> 3, p_el2 = tid & 6, odd = tid & 1;
-
-  if (tid == 0 && t0 < t1) {
-    mbar_wait(bar0, 0, a.err, dead, wait_ns);
-    tc_fence_after();
-    issue_s(0);
-  }
-  for (int t = t0; t < t1; ++t) {
-    const int i = t - t0, st = i & 1;
-    const int p = t * kTcTile + tid;
-    const bool pvalid = p < kv_len;
-    // visibility of position p for every query column: the committed prefix is visible to all, new row u = p - n
-    // to the rows whose mask has bit u
-    uint32_t vis[(NQ + 31) / 32];
-#pragma unroll
-    for (int w = 0; w < (NQ + 31) / 32; ++w) vis[w] = pvalid ? ~0u : 0u;
-    if (pvalid && p >= n) {
-      const int u = p - n, w = u >> 5, b = u & 31;
-#pragma unroll
-      for (int w2 = 0; w2 < (NQ + 31) / 32; ++w2) vis[w2] = 0u;
-#pragma unroll
-      for (int j = 0; j < NQ; ++j) {
-        const int qr = min(q0 + j, qrows_total - 1);
-        const uint32_t word = a.mask[(size_t)(s * a.rw.Ms + qr / G) * kMaskWords + w];
-        vis[j >> 5] |= ((word >> b) & 1u) << (j & 31);
-      }
-    }
-    __syncwarp();
-    mbar_wait(bar_s, i & 1, a.err, dead, wait_ns);
-    tc_fence_after();
-    if (i == 0) TC_STAMP(3);
-    // pass 1: column maxima over the tile's positions
-#pragma unroll
-    for (int c0 = 0; c0 < NQ; c0 += 16) {
-      float r[16];
-      tc_ld16(tlane + c0, r);
-      tc_ld_wait();
-      int mine = 0;
-#pragma unroll
-      for (int jj = 0; jj < 16; ++jj) {
-        const int j = c0 + jj;
-        const float v = ((vis[j >> 5] >> (j & 31)) & 1u) ? r[jj] * scale_log2 : -INFINITY;
-        const int o = __reduce_max_sync(0xffffffffu, f2ord(v));
-        if (lane == jj) mine = o;
-      }
-      if (lane < 16) s_red[c0 + lane][warp] = mine;
-    }
-    __syncthreads();
-    if (i == 0) TC_STAMP(4);
-    if (tid < NQ) {
-      const int4 v = *reinterpret_cast<const int4 *>(s_red[tid]);
-      const float mt = ord2f(max(max(v.x, v.y), max(v.z, v.w)));
-      const float m_old = s_m[tid], m_new = fmaxf(m_old, mt);
-      s_corr[tid] = exp2f(m_old - (m_new == -INFINITY ? 0.f : m_new));
-      s_m[tid] = m_new;
-    }
-    __syncthreads();
-    if (i == 0) TC_STAMP(5);
-    // pass 2: P = 2^(s - m) as bf16 (hi, lo) into the B operand of the second contraction.  Lanes 2i and 2i + 1
-    // hold neighbouring positions: they swap one column of each column pair, so that every lane converts and
-    // stores two neighbouring positions of one column as one 32-bit word.
-#pragma unroll
-    for (int c0 = 0; c0 < NQ; c0 += 16) {
-      float r[16], ms[16];
-      tc_ld16(tlane + c0, r);
-#pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        const float4 m4 = *reinterpret_cast<const float4 *>(&s_m[c0 + 4 * q4]);
-        ms[4 * q4] = m4.x; ms[4 * q4 + 1] = m4.y; ms[4 * q4 + 2] = m4.z; ms[4 * q4 + 3] = m4.w;
-      }
-      tc_ld_wait();
-#pragma unroll
-      for (int jj = 0; jj < 16; ++jj) {
-        const int j = c0 + jj;
-        const float msafe = (ms[jj] == -INFINITY) ? 0.f : ms[jj];
-        r[jj] = ((vis[j >> 5] >> (j & 31)) & 1u) ? exp2f(r[jj] * scale_log2 - msafe) : 0.f;
-      }
-#pragma unroll
-      for (int jj = 0; jj < 16; jj += 2) {
-        const float got = __shfl_xor_sync(0xffffffffu, odd ? r[jj] : r[jj + 1], 1);
-        const float x = odd ? got : r[jj], y = odd ? r[jj + 1] : got;      // positions 2i, 2i + 1 of column jj + odd
-        const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
-        const float2 hf = __bfloat1622float2(h);
-        const __nv_bfloat162 l = __floats2bfloat162_rn(x - hf.x, y - hf.y);
-        const int j = c0 + jj + odd;
-        const int off = p_half * LY::Q_SLAB + j * 128 + ((p_chunk ^ (j & 7)) << 4) + p_el2 * 2;
-        *reinterpret_cast<__nv_bfloat162 *>(base + LY::P_OFF + off) = h;
-        *reinterpret_cast<__nv_bfloat162 *>(base + LY::P_OFF + 2 * LY::Q_SLAB + off) = l;
-      }
-    }
-    if (!pvalid) {       // a position beyond the context: its V row may hold anything, and 0 x NaN is NaN
-      mbar_wait(bar0 + 16 + 8 * st, (i >> 1) & 1, a.err, dead, wait_ns);
-      uint4 *v0 = reinterpret_cast<uint4 *>(base + LY::V_OFF + st * kTcStage + tid * 128);
-      uint4 *v1 = reinterpret_cast<uint4 *>(base + LY::V_OFF + st * kTcStage + kTcSlab + tid * 128);
-#pragma unroll
-      for (int c = 0; c < 8; ++c) { v0[c] = make_uint4(0u, 0u, 0u, 0u); v1[c] = make_uint4(0u, 0u, 0u, 0u); }
-    }
-    fence_async_smem();
-    tc_fence_before();
-    __syncthreads();
-    if (i == 0) TC_STAMP(6);
-    if (tid == 0) {
+      __syncwarp();
+      mbar_wait(s_ready + 8 * g, q & 1, a.err, dead, wait_ns);
       tc_fence_after();
-      mbar_wait(bar0 + 16 + 8 * st, (i >> 1) & 1, a.err, dead, wait_ns);
-      issue_o(st);
-      if (t + 1 < t1) {
-        mbar_wait(bar0 + 8 * (st ^ 1), ((i + 1) >> 1) & 1, a.err, dead, wait_ns);
-        issue_s(st ^ 1);
-      }
-    }
-    __syncwarp();
-    mbar_wait(bar_o, i & 1, a.err, dead, wait_ns);
-    tc_fence_after();
-    if (i == 0) TC_STAMP(7);
-    if (tid == 0 && t + 2 < t1) load_tile(st, t + 2);       // both tiles of this stage have been consumed
-    __syncwarp();
-    // O^T of the tile joins the running one; the column sums go to the columns' owners
-#pragma unroll
-    for (int c0 = 0; c0 < NQ; c0 += 16) {
-      float r[16];
-      tc_ld16(tlane + NQ + c0, r);
+      if (i == 0) TC_STAMP(3);
+      // pass 1: the tile's scores of this position (one wait for all TMEM loads), scaled and masked, and the
+      // column maxima over the tile's positions
+      float sv[NH];
+      tc_ld_cols<NH>(tlane, sv);
       tc_ld_wait();
 #pragma unroll
-      for (int jj = 0; jj < 16; ++jj) o_acc[c0 + jj] = o_acc[c0 + jj] * s_corr[c0 + jj] + r[jj];
-      if (warp == ((c0 >> 4) & 3)) {
-        float ls[16];
-        tc_ld16(tlane + 2 * NQ + c0, ls);
-        tc_ld_wait();
-        float pick = 0.f;
-#pragma unroll
-        for (int jj = 0; jj < 16; ++jj) if (lane == jj) pick = ls[jj];
-        if (lane < 16) s_l[c0 + lane] = s_l[c0 + lane] * s_corr[c0 + lane] + pick;
+      for (int j = 0; j < NH; ++j) sv[j] = ((vis >> j) & 1u) ? sv[j] * scale_log2 : -INFINITY;
+      warp_cols_to_smem<NH, false>(sv, &s_red[g][c_lo], warp & 3, lane);
+      wg_sync(wgi);
+      if (i == 0) TC_STAMP(4);
+      if (wt < NH) {
+        const int j = c_lo + wt;
+        const float4 v = *reinterpret_cast<const float4 *>(s_red[g][j]);
+        const float4 ps = *reinterpret_cast<const float4 *>(s_lred[g][j]);      // the previous tile's sums of P
+        const float mt = fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w));
+        const float m_old = s_m[g][j], m_new = fmaxf(m_old, mt);
+        const float cr = exp2f(m_old - (m_new == -INFINITY ? 0.f : m_new));
+        s_corr[g][j] = cr;
+        s_m[g][j] = m_new;
+        s_l[g][j] = (s_l[g][j] + ((ps.x + ps.y) + (ps.z + ps.w))) * cr;
       }
+      wg_sync(wgi);
+      if (i == 0) TC_STAMP(5);
+      // pass 2: P = 2^(s - m) as bf16 (hi, lo) into the B operand of the second contraction.  Lanes 2i and 2i + 1
+      // hold neighbouring positions: they swap one column of each column pair, so that every lane converts and
+      // stores two neighbouring positions of one column as one 32-bit word.
+#pragma unroll
+      for (int c0 = 0; c0 < NH; c0 += 8) {
+        float ms[8];
+#pragma unroll
+        for (int q4 = 0; q4 < 2; ++q4) {
+          const float4 m4 = *reinterpret_cast<const float4 *>(&s_m[g][c_lo + c0 + 4 * q4]);
+          ms[4 * q4] = m4.x; ms[4 * q4 + 1] = m4.y; ms[4 * q4 + 2] = m4.z; ms[4 * q4 + 3] = m4.w;
+        }
+        float *r = sv + c0;
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+          const float msafe = (ms[jj] == -INFINITY) ? 0.f : ms[jj];
+          r[jj] = exp2f(r[jj] - msafe);                                       // masked: 2^-inf = 0
+        }
+#pragma unroll
+        for (int jj = 0; jj < 8; jj += 2) {
+          const float got = __shfl_xor_sync(0xffffffffu, odd ? r[jj] : r[jj + 1], 1);
+          const float x = odd ? got : r[jj], y = odd ? r[jj + 1] : got;      // positions 2i, 2i + 1 of column jj + odd
+          const __nv_bfloat162 hh = __floats2bfloat162_rn(x, y);
+          const float2 hf = __bfloat1622float2(hh);
+          const __nv_bfloat162 ll = __floats2bfloat162_rn(x - hf.x, y - hf.y);
+          const int j = c_lo + c0 + jj + odd;
+          const int off = p_half * LY::Q_SLAB + j * 128 + ((p_chunk ^ (j & 7)) << 4) + p_el2 * 2;
+          *reinterpret_cast<__nv_bfloat162 *>(pbase + off) = hh;
+          *reinterpret_cast<__nv_bfloat162 *>(pbase + 2 * LY::Q_SLAB + off) = ll;
+        }
+      }
+      warp_cols_to_smem<NH, true>(sv, &s_lred[g][c_lo], warp & 3, lane);      // this warp's sums of P per column
+      if (!pvalid && h == 0) {   // a position beyond the context: its V row may hold anything, and 0 x NaN is NaN
+        mbar_wait(full_v + 8 * g, q & 1, a.err, dead, wait_ns);
+        uint4 *v0 = reinterpret_cast<uint4 *>(base + LY::V_OFF + g * kTcStage + wt * 128);
+        uint4 *v1 = reinterpret_cast<uint4 *>(base + LY::V_OFF + g * kTcStage + kTcSlab + wt * 128);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) { v0[c] = make_uint4(0u, 0u, 0u, 0u); v1[c] = make_uint4(0u, 0u, 0u, 0u); }
+      }
+      fence_async_smem();
+      tc_fence_before();
+      mbar_arrive(p_ready + 8 * g);
+      if (i == 0) TC_STAMP(6);
+      mbar_wait(o_ready + 8 * g, q & 1, a.err, dead, wait_ns);
+      tc_fence_after();
+      if (i == 0) TC_STAMP(7);
+      // O^T of the tile joins the running one
+      float *ov = sv;                                  // the scores are dead
+      tc_ld_cols<NH>(tlane + NQ, ov);
+      tc_ld_wait();
+#pragma unroll
+      for (int q4 = 0; q4 < NH / 4; ++q4) {
+        const float4 c4 = *reinterpret_cast<const float4 *>(&s_corr[g][c_lo + 4 * q4]);
+        o_acc[4 * q4] = o_acc[4 * q4] * c4.x + ov[4 * q4];
+        o_acc[4 * q4 + 1] = o_acc[4 * q4 + 1] * c4.y + ov[4 * q4 + 1];
+        o_acc[4 * q4 + 2] = o_acc[4 * q4 + 2] * c4.z + ov[4 * q4 + 2];
+        o_acc[4 * q4 + 3] = o_acc[4 * q4 + 3] * c4.w + ov[4 * q4 + 3];
+      }
+      tc_fence_before();
+      if (i == 0) TC_STAMP(8);
     }
-    if (i == 0) TC_STAMP(8);
   }
   TC_STAMP(9);
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) {
+  if (warp == 16) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTcTmemCols) : "memory");
   }
-  // merge: o = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.  Column j is finalised by CTA j % splits: once every
-  // CTA of the cluster has left its tile loop (its stages are free), each pushes its partial (m, l, O^T column)
-  // into the owner's shared memory with plain remote stores; after a second cluster barrier the owners merge
-  // what they received, in split order, from their own shared memory.
-  cg::cluster_group cluster = cg::this_cluster();
-  TC_STAMP(10);
-  cluster.sync();
-  TC_STAMP(11);
-  const int rank = (int)cluster.block_rank(), nsp = (int)cluster.num_blocks();
-  const int slots = (NQ + nsp - 1) / nsp;                       // columns an owner may receive from one split
-  float *sM = reinterpret_cast<float *>(base + LY::K_OFF);      // [splits][slots][128] floats (<= (NQ + 8) x 512 B)
-  {
-    int owner = 0, slot = 0;
+  // ---- the two tile groups' partials become the CTA's: group 1 hands its O^T columns over through its key buffer
+  // (all its tiles have been consumed), group 0 rescales both to the common maximum
+  float *sO1 = reinterpret_cast<float *>(base + LY::K_OFF + kTcStage);          // [NQ][128] floats
+  const int my_g = warp >> 3, my_lo = ((warp >> 2) & 1) * NH, my_t = tid & (kTcWg - 1);   // of a softmax thread
+  if (warp < 16 && my_g == 1) {
 #pragma unroll
-    for (int j = 0; j < NQ; ++j) {
-      if (j < ncols) cluster.map_shared_rank(sM, owner)[(size_t)(rank * slots + slot) * kTcDh + tid] = o_acc[j];
-      if (++owner == nsp) { owner = 0; ++slot; }
-    }
-    if (tid < ncols) {
-      const int ow = tid % nsp, sl = tid / nsp;
-      cluster.map_shared_rank(s_pm, ow)[rank * slots + sl] = s_m[tid];
-      cluster.map_shared_rank(s_pl, ow)[rank * slots + sl] = s_l[tid];
+    for (int j = 0; j < NH; ++j) sO1[(my_lo + j) * kTcDh + my_t] = o_acc[j];
+  }
+  if (tid < NQ) {
+    const float m0 = s_m[0][tid], m1 = s_m[1][tid], M = fmaxf(m0, m1), Ms = (M == -INFINITY) ? 0.f : M;
+    const float w0 = exp2f(m0 - Ms), w1 = exp2f(m1 - Ms);                       // a side without tiles: 2^-inf = 0
+    const float4 p0 = *reinterpret_cast<const float4 *>(s_lred[0][tid]), p1 = *reinterpret_cast<const float4 *>(s_lred[1][tid]);
+    const float l0 = s_l[0][tid] + ((p0.x + p0.y) + (p0.z + p0.w)), l1 = s_l[1][tid] + ((p1.x + p1.y) + (p1.z + p1.w));   // the last tiles' sums
+    s_corr[0][tid] = w0; s_corr[1][tid] = w1;
+    s_m[0][tid] = M;
+    s_l[0][tid] = l0 * w0 + l1 * w1;
+  }
+  __syncthreads();
+  const bool pusher = warp < 16 && my_g == 0;      // the two warpgroups that now hold the CTA's O^T
+  if (pusher) {
+#pragma unroll
+    for (int j = 0; j < NH; ++j)
+      o_acc[j] = o_acc[j] * s_corr[0][my_lo + j] + sO1[(my_lo + j) * kTcDh + my_t] * s_corr[1][my_lo + j];
+  }
+  TC_STAMP(10);
+  // ---- merge over the kv splits: o = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.  Column j is finalised by CTA
+  // j % splits: once every CTA of the cluster has left its tile loop (its buffers are free), each pushes its
+  // partial (m, l, O^T column) into the owner's shared memory with plain remote stores; after a second cluster
+  // barrier the owners merge what they received, in split order, from their own shared memory.  A lone CTA takes
+  // the same route through its own shared memory (the transpose makes the global stores 8 bytes wide).
+  const int nsp = nsplits;
+  cg::cluster_group cluster = cg::this_cluster();
+  if (nsp > 1) cluster.sync();
+  TC_STAMP(11);
+  const int rank = (nsp > 1) ? (int)cluster.block_rank() : 0;
+  const int slots = (NQ + nsp - 1) / nsp;                       // columns an owner may receive from one split
+  float *sM = reinterpret_cast<float *>(base + LY::V_OFF);      // [splits][slots][128] floats (<= (NQ + 8) x 512 B)
+  if (pusher) {
+    if (nsp > 1) {
+      int owner = my_lo % nsp, slot_j = my_lo / nsp;
+#pragma unroll
+      for (int j = 0; j < NH; ++j) {
+        if (my_lo + j < ncols) cluster.map_shared_rank(sM, owner)[(size_t)(rank * slots + slot_j) * kTcDh + my_t] = o_acc[j];
+        if (++owner == nsp) { owner = 0; ++slot_j; }
+      }
+      if (tid < ncols) {
+        const int ow = tid % nsp, sl = tid / nsp;
+        cluster.map_shared_rank(s_pm, ow)[rank * slots + sl] = s_m[0][tid];
+        cluster.map_shared_rank(s_pl, ow)[rank * slots + sl] = s_l[0][tid];
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < NH; ++j) sM[(my_lo + j) * kTcDh + my_t] = o_acc[j];
+      if (tid < NQ) { s_pm[tid] = s_m[0][tid]; s_pl[tid] = s_l[0][tid]; }
     }
   }
   TC_STAMP(12);
-  cluster.sync();
+  if (nsp > 1) cluster.sync(); else __syncthreads();
   TC_STAMP(13);
-  constexpr int TPR = kTcDh / 4, RP = kTcThreads / TPR;      // threads per column, columns per pass
-  const int c4 = (tid % TPR) * 4, sub = tid / TPR;
-  for (int slot = sub; rank + slot * nsp < ncols; slot += RP) {
-    const int j = rank + slot * nsp;
-    float M = -INFINITY;
-    for (int sp = 0; sp < nsp; ++sp) M = fmaxf(M, s_pm[sp * slots + slot]);
-    float L = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int sp = 0; sp < nsp; ++sp) {
-      const float pm = s_pm[sp * slots + slot];
-      if (pm != -INFINITY) {
-        const float w = exp2f(pm - M);
-        const float4 ov = *reinterpret_cast<const float4 *>(sM + (size_t)(sp * slots + slot) * kTcDh + c4);
-        L += w * s_pl[sp * slots + slot];
-        acc.x += w * ov.x; acc.y += w * ov.y; acc.z += w * ov.z; acc.w += w * ov.w;
+  constexpr int TPR = kTcDh / 4;                             // threads per column
+  if (tid < 2 * kTcWg) {
+    const int c4 = (tid % TPR) * 4, sub = tid / TPR;         // 8 columns per pass
+    for (int sl = sub; rank + sl * nsp < ncols; sl += 2 * kTcWg / TPR) {
+      const int j = rank + sl * nsp;
+      float M = -INFINITY;
+      for (int sp = 0; sp < nsp; ++sp) M = fmaxf(M, s_pm[sp * slots + sl]);
+      float L = 0.f;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int sp = 0; sp < nsp; ++sp) {
+        const float pm = s_pm[sp * slots + sl];
+        if (pm != -INFINITY) {
+          const float wgt = exp2f(pm - M);
+          const float4 ov = *reinterpret_cast<const float4 *>(sM + (size_t)(sp * slots + sl) * kTcDh + c4);
+          L += wgt * s_pl[sp * slots + sl];
+          acc.x += wgt * ov.x; acc.y += wgt * ov.y; acc.z += wgt * ov.z; acc.w += wgt * ov.w;
+        }
       }
+      const float inv = (L > 0.f) ? 1.f / L : 0.f;
+      const float val[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
+      const __nv_bfloat162 h01 = __floats2bfloat162_rn(val[0], val[1]), h23 = __floats2bfloat162_rn(val[2], val[3]);
+      const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
+      const __nv_bfloat162 l01 = __floats2bfloat162_rn(val[0] - f01.x, val[1] - f01.y);
+      const __nv_bfloat162 l23 = __floats2bfloat162_rn(val[2] - f23.x, val[3] - f23.y);
+      const size_t idx = (size_t)s_oidx[j] + c4;
+      *reinterpret_cast<uint2 *>(a.o + idx) =
+          make_uint2(*reinterpret_cast<const uint32_t *>(&h01), *reinterpret_cast<const uint32_t *>(&h23));
+      *reinterpret_cast<uint2 *>(a.o + a.o_lo_off + idx) =
+          make_uint2(*reinterpret_cast<const uint32_t *>(&l01), *reinterpret_cast<const uint32_t *>(&l23));
     }
-    const float inv = (L > 0.f) ? 1.f / L : 0.f;
-    const float val[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
-    const int qr = q0 + j;
-    const int r = s * a.rw.Ms + qr / G, head = kvh * G + qr % G;
-    const __nv_bfloat162 h01 = __floats2bfloat162_rn(val[0], val[1]), h23 = __floats2bfloat162_rn(val[2], val[3]);
-    const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
-    const __nv_bfloat162 l01 = __floats2bfloat162_rn(val[0] - f01.x, val[1] - f01.y);
-    const __nv_bfloat162 l23 = __floats2bfloat162_rn(val[2] - f23.x, val[3] - f23.y);
-    const size_t idx = ((size_t)r * a.H + head) * kTcDh + c4;
-    *reinterpret_cast<uint2 *>(a.o + idx) =
-        make_uint2(*reinterpret_cast<const uint32_t *>(&h01), *reinterpret_cast<const uint32_t *>(&h23));
-    *reinterpret_cast<uint2 *>(a.o + a.o_lo_off + idx) =
-        make_uint2(*reinterpret_cast<const uint32_t *>(&l01), *reinterpret_cast<const uint32_t *>(&l23));
   }
   TC_STAMP(14);
 }
@@ -489,12 +584,14 @@ void attention_tc_blocks(int qrows, int *qblocks, int *qper) {
 }
 
 int attention_tc_splits(int groups, int kv_tiles, int sm_count) {
-  // one CTA per SM: the fewest rounds of the longest split's tiles (+ ~2 tiles' worth of fixed cost per round)
+  // one CTA per SM, two tiles in flight per CTA (one per tile group): rounds x (the longest split's tiles per tile
+  // group at ~2.8 us each + the fixed cost of a CTA, + the cluster barriers when there is more than one split)
   int best = 1;
   float best_cost = 1e30f;
   for (int s = 1; s <= kAttnMaxSplits && s <= (kv_tiles > 0 ? kv_tiles : 1); ++s) {
     const int rounds = (s * groups + sm_count - 1) / sm_count;
-    const float cost = (float)rounds * ((float)((kv_tiles + s - 1) / s) + 2.f);
+    const int per = (kv_tiles + s - 1) / s;
+    const float cost = (float)rounds * (2.8f * (float)((per + 1) / 2) + 8.f + (s > 1 ? 1.5f : 0.f));
     if (cost < best_cost - 1e-6f) { best_cost = cost; best = s; }
   }
   return best;
@@ -510,8 +607,7 @@ cudaError_t launch_attention_tc(const AttnArgs &a, bool pdl, cudaStream_t st) {
   if (!kv_map(&tmK, a.kcache, rows, width) || !kv_map(&tmV, a.kcache + a.kv_stride, rows, width)) return cudaErrorInvalidValue;
   if (qper <= 16) return launch_nq<16>(tmK, tmV, a, qblocks, qper, pdl, st);
   if (qper <= 32) return launch_nq<32>(tmK, tmV, a, qblocks, qper, pdl, st);
-  if (qper <= 48) return launch_nq<48>(tmK, tmV, a, qblocks, qper, pdl, st);
-  return launch_nq<80>(tmK, tmV, a, qblocks, qper, pdl, st);
+  return launch_nq<48>(tmK, tmV, a, qblocks, qper, pdl, st);
 }
 
 }  // namespace firp

@@ -85,7 +85,7 @@ struct firp_ctx {
   int pseudo_masked = 0;     // Section 4.3 "Masked": pseudo rows do not see one another
   int pred_prenorm = 0;      // Eq. 3 reads the anchor through the insertion layer's input RMSNorm
   int planes[5] = {2, 2, 2, 2, 2};
-  bool attn_tc = false;              // head dimension 128: the tcgen05 attention kernel instead of the mma.sync one
+  int attn_tc = -1;                  // head dimension 128: 1 the tcgen05 attention kernel, 0 the mma.sync one, -1 by the step's shape
   int attn_planes[2] = {2, 2};       // of the queries and of the probabilities in the attention   // bf16 planes of the activations per GEMM class: qkv, o, gate/up, down, lm-head
 
   // cache layout [layer][K|V][row][kv_head][head_dim]; row = slot * max_ctx + position, or through the page table
@@ -338,18 +338,26 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       const int G = H / Hkv, qblocks = (act * G + 63) / 64;
       a.splits = attention_splits(rw.n_seq * Hkv * qblocks, tiles);
       a.o = c->o; a.o_lo_off = Rp * nq; a.err = c->dev_status; a.wait_ns = c->wait_ns;
-      const bool tc = c->attn_tc && dh == 128;
-      if (tc) {
+      bool tc = false;
+      if (dh == 128 && c->attn_tc != 0) {
         int qb_tc, qper_tc;
         attention_tc_blocks(act * G, &qb_tc, &qper_tc);
-        a.splits = attention_tc_splits(rw.n_seq * Hkv * qb_tc, (ra.n_hi_max + act + kAttnTcTile - 1) / kAttnTcTile, c->sm_count);
+        const int tiles_tc = (ra.n_hi_max + act + kAttnTcTile - 1) / kAttnTcTile;
+        // Left to itself the tensor-core kernel takes every step whose longest context spans at least three of its
+        // 128-position tiles (four when the query columns need more than one block): its fixed cost is higher, its
+        // tile loop faster.  Measured at the 7B shape, one sequence, ms per step mma.sync / tcgen05: 35 columns
+        // 3.53 / 3.58 at 128 cached tokens, 3.72 / 3.65 at 512, 5.23 / 4.48 at 8192; 1 column 3.25 / 3.26 at 128,
+        // 3.37 / 3.28 at 512, 5.04 / 4.06 at 8192; 131 columns (three blocks) 5.53 / 5.74 at 128, 5.80 / 5.80 at
+        // 256, 5.96 / 5.88 at 512, 10.35 / 9.68 at 8192.
+        tc = c->attn_tc > 0 || tiles_tc >= (qb_tc == 1 ? 3 : 4);
+        if (tc) a.splits = attention_tc_splits(rw.n_seq * Hkv * qb_tc, tiles_tc, c->sm_count);
       }
-      // Early (programmatic) launch of the attention pays only when the rotary finisher before it has at least one
-      // CTA per SM.  Measured at the 7B shape, ms per step with / without it: 35 rows 3.61 / 3.76 at 512 cached
-      // tokens and 5.25 / 5.44 at 8192; 67 and 131 rows likewise 0.1 ms better with it; but 19 rows 3.68 / 3.60 and
-      // 6.36 / 5.26, 1 row 3.52 / 3.43 and 6.27 / 5.11.
+      // Early (programmatic) launch of the attention pays only when the rotary finisher before it has well over one
+      // CTA per SM (5/4).  Measured at the 7B shape, ms per step with / without it: 35 rows 3.61 / 3.76 at 512 cached
+      // tokens and 5.25 / 5.44 at 8192; 67 and 131 rows likewise 0.1 ms better with it; but 27 rows (162 CTAs on 148
+      // SMs) 3.70 / 3.66 and 6.30 / 5.33, 19 rows 3.68 / 3.60 and 6.36 / 5.26, 1 row 3.52 / 3.43 and 6.27 / 5.11.
       const int half_dh = dh / 2, qkv_st = (H + 2 * Hkv + 128 / half_dh - 1) / (128 / half_dh);
-      const bool attn_early = pdl && (qkv_st * rw.R * 32 + 255) / 256 >= c->sm_count;
+      const bool attn_early = pdl && (qkv_st * rw.R * 32 + 255) / 256 >= c->sm_count * 5 / 4;
       FIRP_TIMED(KC_ATTENTION);
       FIRP_CUDA(c, tc ? launch_attention_tc(a, attn_early, st) : launch_attention(a, attn_early, st)); ++nl;
     }
@@ -756,8 +764,8 @@ int firp_set_attention_planes(firp_ctx *ctx, int32_t q_planes, int32_t p_planes)
 }
 
 int firp_set_attention_kernel(firp_ctx *ctx, int32_t tensor_core) {
-  if (!ctx) return FIRP_ERR_BAD_ARG;
-  ctx->attn_tc = tensor_core != 0;
+  if (!ctx || tensor_core < -1 || tensor_core > 1) return FIRP_ERR_BAD_ARG;
+  ctx->attn_tc = tensor_core;
   return FIRP_OK;
 }
 

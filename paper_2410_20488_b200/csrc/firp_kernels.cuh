@@ -220,7 +220,7 @@ int attention_splits(int groups, int kv_tiles);
 cudaError_t launch_attention(const AttnArgs &a, bool pdl, cudaStream_t st);
 // The tcgen05 kernel (head dimension 128): 128-position tiles, query blocks of at most kAttnTcMaxCols columns
 // (query rows x heads of the group), a.splits from attention_tc_splits.
-constexpr int kAttnTcTile = 128, kAttnTcMaxCols = 80;
+constexpr int kAttnTcTile = 128, kAttnTcMaxCols = 48;
 void attention_tc_blocks(int qrows, int *qblocks, int *qper);
 int attention_tc_splits(int groups, int kv_tiles, int sm_count);
 cudaError_t launch_attention_tc(const AttnArgs &a, bool pdl, cudaStream_t st);
