@@ -338,28 +338,30 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
       const int G = H / Hkv, qblocks = (act * G + 63) / 64;
       a.splits = attention_splits(rw.n_seq * Hkv * qblocks, tiles);
       a.o = c->o; a.o_lo_off = Rp * nq; a.err = c->dev_status; a.wait_ns = c->wait_ns;
+      // Early (programmatic) launch of the mma.sync attention pays only when the rotary finisher before it has well
+      // over one CTA per SM (5/4).  Measured at the 7B shape, ms per step with / without it: 35 rows 3.61 / 3.76 at
+      // 512 cached tokens and 5.25 / 5.44 at 8192; 67 and 131 rows likewise 0.1 ms better with it; but 27 rows (162
+      // CTAs on 148 SMs) 3.70 / 3.66 and 6.30 / 5.33, 19 rows 3.68 / 3.60 and 6.36 / 5.26, 1 row 3.52 / 3.43 and
+      // 6.27 / 5.11.  The tensor-core kernel (one CTA per SM, all of them resident and set up before the finisher
+      // ends) gains from it at every size: 1 row 3.27 / 3.14 at 512, 27 rows 3.60 / 3.49, 35 rows 3.69 / 3.60.
+      const int half_dh = dh / 2, qkv_st = (H + 2 * Hkv + 128 / half_dh - 1) / (128 / half_dh);
+      const bool attn_early = pdl && (qkv_st * rw.R * 32 + 255) / 256 >= c->sm_count * 5 / 4;
       bool tc = false;
       if (dh == 128 && c->attn_tc != 0) {
         int qb_tc, qper_tc;
         attention_tc_blocks(act * G, &qb_tc, &qper_tc);
         const int tiles_tc = (ra.n_hi_max + act + kAttnTcTile - 1) / kAttnTcTile;
-        // Left to itself the tensor-core kernel takes every step whose longest context spans at least three of its
-        // 128-position tiles (four when the query columns need more than one block): its fixed cost is higher, its
-        // tile loop faster.  Measured at the 7B shape, one sequence, ms per step mma.sync / tcgen05: 35 columns
-        // 3.53 / 3.58 at 128 cached tokens, 3.72 / 3.65 at 512, 5.23 / 4.48 at 8192; 1 column 3.25 / 3.26 at 128,
-        // 3.37 / 3.28 at 512, 5.04 / 4.06 at 8192; 131 columns (three blocks) 5.53 / 5.74 at 128, 5.80 / 5.80 at
-        // 256, 5.96 / 5.88 at 512, 10.35 / 9.68 at 8192.
-        tc = c->attn_tc > 0 || tiles_tc >= (qb_tc == 1 ? 3 : 4);
+        // Left to itself the tensor-core kernel takes every step the other kernel would not be launched early for,
+        // and otherwise those whose longest context spans at least three of its 128-position tiles (four when the
+        // query columns need more than one block): its fixed cost is higher, its tile loop faster.  Measured at the
+        // 7B shape, one sequence, ms per step mma.sync / tcgen05: 1 column 3.23 / 3.06 at 64 cached tokens, 3.37 /
+        // 3.28 at 512, 5.04 / 4.06 at 8192; 35 columns 3.57 / 3.61 at 64, 3.64 / 3.65 at 128, 3.72 / 3.65 at 512,
+        // 5.23 / 4.48 at 8192; 131 columns (three blocks) 5.96 / 5.91 at 64, 6.09 / 6.07 at 256, 10.35 / 9.68 at 8192.
+        tc = c->attn_tc > 0 || !attn_early || tiles_tc >= (qb_tc == 1 ? 3 : 4);
         if (tc) a.splits = attention_tc_splits(rw.n_seq * Hkv * qb_tc, tiles_tc, c->sm_count);
       }
-      // Early (programmatic) launch of the attention pays only when the rotary finisher before it has well over one
-      // CTA per SM (5/4).  Measured at the 7B shape, ms per step with / without it: 35 rows 3.61 / 3.76 at 512 cached
-      // tokens and 5.25 / 5.44 at 8192; 67 and 131 rows likewise 0.1 ms better with it; but 27 rows (162 CTAs on 148
-      // SMs) 3.70 / 3.66 and 6.30 / 5.33, 19 rows 3.68 / 3.60 and 6.36 / 5.26, 1 row 3.52 / 3.43 and 6.27 / 5.11.
-      const int half_dh = dh / 2, qkv_st = (H + 2 * Hkv + 128 / half_dh - 1) / (128 / half_dh);
-      const bool attn_early = pdl && (qkv_st * rw.R * 32 + 255) / 256 >= c->sm_count * 5 / 4;
       FIRP_TIMED(KC_ATTENTION);
-      FIRP_CUDA(c, tc ? launch_attention_tc(a, attn_early, st) : launch_attention(a, attn_early, st)); ++nl;
+      FIRP_CUDA(c, tc ? launch_attention_tc(a, pdl, st) : launch_attention(a, attn_early, st)); ++nl;
     }
     {
       GemmArgs g = gemm_base(c->o, Rp * nq, c->wo[j], d, nq, act);
