@@ -13,10 +13,10 @@
 // K, V and P buffers, TMEM columns and running (max, sum, O^T), so that the tensor-core work of one overlaps the
 // softmax of the other; the query columns of a tile are shared by two warpgroups (halves), which makes four
 // softmax warpgroups: thread i of each keeps O^T[i][its columns] (dh index i) in registers.  One thread issues
-// every MMA, two more feed the K and the V buffers by TMA.  The two partial results are merged in shared memory; the
-// CTAs of one (kv head, query block) -- the kv splits -- form a cluster and merge theirs by pushing each column
-// to the CTA that finalises it.  One CTA per SM (shared memory), so the 512 TMEM columns it allocates are never
-// contended.  Every mbarrier wait is bounded; a wait that runs out sets the status word and the kernel runs to
+// every MMA, two more feed the K and the V buffers by TMA.  The CTAs of one (kv head, query block) -- the kv
+// splits -- form a cluster; every partial result (split, tile group) is pushed, four columns at a time, to the
+// CTA that finalises those columns.  One CTA per SM (shared memory), so the 256 TMEM columns it allocates are
+// never contended.  Every mbarrier wait is bounded; a wait that runs out sets the status word and the kernel runs to
 // its end.
 #include <cooperative_groups.h>
 
@@ -50,8 +50,7 @@ template <int NQ> struct TcLayout {
   static constexpr int P_OFF = Q_OFF + 4 * Q_SLAB;        // [2 warpgroups][2 planes][2 pos halves][NQ][128 B]
   static constexpr int BYTES = P_OFF + 8 * Q_SLAB;
   static_assert(NQ % 16 == 0 && NQ >= 16 && NQ <= 48 && 4 * NQ <= kTcTmemCols, "query columns per block");
-  static_assert(NQ * kTcDh * 4 <= kTcStage, "a warpgroup's partial O^T must fit its key buffer");
-  static_assert((NQ + 8) * kTcDh * 4 <= 2 * kTcStage, "the partials a CTA receives must fit the value buffers");
+  static_assert(2 * (NQ + 4 * 8) * kTcDh * 4 <= 4 * kTcStage, "the partials a CTA receives must fit the K and V buffers");
   static_assert(BYTES + 1024 + 6144 <= 227 * 1024, "shared memory budget (dynamic + alignment + static)");
 };
 
@@ -136,7 +135,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   __shared__ __align__(16) float s_m[2][NQ];        // running max (log2 units)
   __shared__ __align__(16) float s_corr[2][NQ];     // 2^(old max - new max) of the current tile; merge weights at the end
   __shared__ __align__(16) float s_l[2][NQ];        // running sum
-  __shared__ float s_pm[NQ + kAttnMaxSplits], s_pl[NQ + kAttnMaxSplits];   // (max, sum) received for the merge: [split][slot]
+  __shared__ __align__(16) float s_pm[2 * (NQ + 4 * kAttnMaxSplits)], s_pl[2 * (NQ + 4 * kAttnMaxSplits)];   // (max, sum) received for the merge: [partial][slot][4 columns]
   __shared__ uint32_t s_oidx[NQ];                   // element offset of each column's output row
   // mbarriers: K landed [2], V landed [2], S^T complete [2], P written [2], O^T complete [2], Q written
   __shared__ __align__(8) uint64_t s_bar[11];
@@ -179,6 +178,22 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int ncols = min(qper, qrows_total - q0);
   const int slot = a.seq_ids[s];
   const int n = a.pos[s * a.rw.Ms];                 // position of the root row = committed length
+  // queries of this block (all softmax threads share the work): column j = query row q0 + j -> (tree row
+  // (q0 + j) / G, head kvh G + (q0 + j) % G).  Their loads go out before the context length above is first used.
+  constexpr int QIT = (NQ * 16 + kTcSoft - 1) / kTcSoft;
+  uint4 qh[QIT], ql[QIT];
+  if (warp < 16) {
+#pragma unroll
+    for (int it = 0; it < QIT; ++it) {
+      const int idx = it * kTcSoft + tid, j = idx >> 4, c = idx & 15, qr = q0 + j;
+      qh[it] = make_uint4(0u, 0u, 0u, 0u); ql[it] = qh[it];
+      if (j < ncols) {
+        const bf16 *src = a.q + ((size_t)(s * a.rw.Ms + qr / G) * a.H + kvh * G + qr % G) * kTcDh + c * 8;
+        qh[it] = *reinterpret_cast<const uint4 *>(src);
+        ql[it] = *reinterpret_cast<const uint4 *>(src + a.q_lo_off);
+      }
+    }
+  }
   const int kv_len = min(n + a.rows_active, a.max_ctx);
   const int tiles_total = (kv_len + kTcTile - 1) / kTcTile;
   const int t0 = (split * tiles_total + nsplits - 1) / nsplits, t1 = ((split + 1) * tiles_total + nsplits - 1) / nsplits;
@@ -263,22 +278,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const int c_lo = h * NH;
     const uint32_t tlane = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(g * 2 * NQ + c_lo);
     {
-      // queries of this block (all softmax threads share the work): column j = query row q0 + j -> (tree row
-      // (q0 + j) / G, head kvh G + (q0 + j) % G)
-      constexpr int IT = (NQ * 16 + kTcSoft - 1) / kTcSoft;
-      uint4 qh[IT], ql[IT];
 #pragma unroll
-      for (int it = 0; it < IT; ++it) {               // all loads in flight before the first store
-        const int idx = it * kTcSoft + tid, j = idx >> 4, c = idx & 15, qr = q0 + j;
-        qh[it] = make_uint4(0u, 0u, 0u, 0u); ql[it] = qh[it];
-        if (j < ncols) {
-          const bf16 *src = a.q + ((size_t)(s * a.rw.Ms + qr / G) * a.H + kvh * G + qr % G) * kTcDh + c * 8;
-          qh[it] = *reinterpret_cast<const uint4 *>(src);
-          ql[it] = *reinterpret_cast<const uint4 *>(src + a.q_lo_off);
-        }
-      }
-#pragma unroll
-      for (int it = 0; it < IT; ++it) {
+      for (int it = 0; it < QIT; ++it) {
         const int idx = it * kTcSoft + tid, j = idx >> 4, c = idx & 15;
         if (j < NQ) {
           const int off = (c >> 3) * LY::Q_SLAB + j * 128 + (((c & 7) ^ (j & 7)) << 4);
@@ -406,100 +407,87 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     }
   }
   TC_STAMP(9);
+  // ---- merge: o = sum_p 2^(m_p - M) O_p / sum_p 2^(m_p - M) l_p over the partials p = (kv split, tile group).
+  // Columns go in groups of four; group c is finalised by CTA c % splits.  Once every CTA of the cluster has left
+  // its tile loop (its buffers are free), every softmax thread pushes its columns of its tile group's partial into
+  // the owners' shared memory (16-byte remote stores: O^T[dh][4 columns]), the columns' (m, l) likewise; after a
+  // second cluster barrier the owners merge what they received, in partial order, from their own shared memory.
+  // A lone CTA takes the same route through its own shared memory.
+  const int nsp = nsplits;
+  const int my_g = warp >> 3, my_lo = ((warp >> 2) & 1) * NH, my_t = tid & (kTcWg - 1);   // of a softmax thread
+  if (warp < 16) {
+    wg_sync(warp >> 2);                              // the last tile's sums of P are in shared memory
+    if (my_t < NH) {
+      const int j = my_lo + my_t;
+      const float4 ps = *reinterpret_cast<const float4 *>(s_lred[my_g][j]);
+      s_l[my_g][j] += (ps.x + ps.y) + (ps.z + ps.w);
+    }
+  }
   tc_fence_before();
-  __syncthreads();
+  cg::cluster_group cluster = cg::this_cluster();
+  if (nsp > 1) cluster.sync(); else __syncthreads();
+  TC_STAMP(11);
   if (warp == 16) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTcTmemCols) : "memory");
   }
-  // ---- the two tile groups' partials become the CTA's: group 1 hands its O^T columns over through its key buffer
-  // (all its tiles have been consumed), group 0 rescales both to the common maximum
-  float *sO1 = reinterpret_cast<float *>(base + LY::K_OFF + kTcStage);          // [NQ][128] floats
-  const int my_g = warp >> 3, my_lo = ((warp >> 2) & 1) * NH, my_t = tid & (kTcWg - 1);   // of a softmax thread
-  if (warp < 16 && my_g == 1) {
-#pragma unroll
-    for (int j = 0; j < NH; ++j) sO1[(my_lo + j) * kTcDh + my_t] = o_acc[j];
-  }
-  if (tid < NQ) {
-    const float m0 = s_m[0][tid], m1 = s_m[1][tid], M = fmaxf(m0, m1), Ms = (M == -INFINITY) ? 0.f : M;
-    const float w0 = exp2f(m0 - Ms), w1 = exp2f(m1 - Ms);                       // a side without tiles: 2^-inf = 0
-    const float4 p0 = *reinterpret_cast<const float4 *>(s_lred[0][tid]), p1 = *reinterpret_cast<const float4 *>(s_lred[1][tid]);
-    const float l0 = s_l[0][tid] + ((p0.x + p0.y) + (p0.z + p0.w)), l1 = s_l[1][tid] + ((p1.x + p1.y) + (p1.z + p1.w));   // the last tiles' sums
-    s_corr[0][tid] = w0; s_corr[1][tid] = w1;
-    s_m[0][tid] = M;
-    s_l[0][tid] = l0 * w0 + l1 * w1;
-  }
-  __syncthreads();
-  const bool pusher = warp < 16 && my_g == 0;      // the two warpgroups that now hold the CTA's O^T
-  if (pusher) {
-#pragma unroll
-    for (int j = 0; j < NH; ++j)
-      o_acc[j] = o_acc[j] * s_corr[0][my_lo + j] + sO1[(my_lo + j) * kTcDh + my_t] * s_corr[1][my_lo + j];
-  }
-  TC_STAMP(10);
-  // ---- merge over the kv splits: o = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.  Column j is finalised by CTA
-  // j % splits: once every CTA of the cluster has left its tile loop (its buffers are free), each pushes its
-  // partial (m, l, O^T column) into the owner's shared memory with plain remote stores; after a second cluster
-  // barrier the owners merge what they received, in split order, from their own shared memory.  A lone CTA takes
-  // the same route through its own shared memory (the transpose makes the global stores 8 bytes wide).
-  const int nsp = nsplits;
-  cg::cluster_group cluster = cg::this_cluster();
-  if (nsp > 1) cluster.sync();
-  TC_STAMP(11);
   const int rank = (nsp > 1) ? (int)cluster.block_rank() : 0;
-  const int slots = (NQ + nsp - 1) / nsp;                       // columns an owner may receive from one split
-  float *sM = reinterpret_cast<float *>(base + LY::V_OFF);      // [splits][slots][128] floats (<= (NQ + 8) x 512 B)
-  if (pusher) {
-    if (nsp > 1) {
-      int owner = my_lo % nsp, slot_j = my_lo / nsp;
+  constexpr int NG = NQ / 4;                                    // column groups
+  const int slots = (NG + nsp - 1) / nsp;                       // groups an owner may receive from one partial
+  const int nparts = 2 * nsp, part = 2 * rank + my_g;
+  float4 *sM = reinterpret_cast<float4 *>(base + LY::K_OFF);    // [partials][slots][128 dh] x 4 columns, over the K and V buffers
+  if (warp < 16) {
+    int owner = (my_lo / 4) % nsp, slot_c = (my_lo / 4) / nsp;
 #pragma unroll
-      for (int j = 0; j < NH; ++j) {
-        if (my_lo + j < ncols) cluster.map_shared_rank(sM, owner)[(size_t)(rank * slots + slot_j) * kTcDh + my_t] = o_acc[j];
-        if (++owner == nsp) { owner = 0; ++slot_j; }
+    for (int c = 0; c < NH / 4; ++c) {
+      if (my_lo + 4 * c < ncols) {
+        float4 *dst = (nsp > 1) ? cluster.map_shared_rank(sM, owner) : sM;
+        dst[(size_t)(part * slots + slot_c) * kTcDh + my_t] = make_float4(o_acc[4 * c], o_acc[4 * c + 1], o_acc[4 * c + 2], o_acc[4 * c + 3]);
       }
-      if (tid < ncols) {
-        const int ow = tid % nsp, sl = tid / nsp;
-        cluster.map_shared_rank(s_pm, ow)[rank * slots + sl] = s_m[0][tid];
-        cluster.map_shared_rank(s_pl, ow)[rank * slots + sl] = s_l[0][tid];
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < NH; ++j) sM[(my_lo + j) * kTcDh + my_t] = o_acc[j];
-      if (tid < NQ) { s_pm[tid] = s_m[0][tid]; s_pl[tid] = s_l[0][tid]; }
+      if (++owner == nsp) { owner = 0; ++slot_c; }
+    }
+    if (my_t < NH && my_lo + my_t < ncols) {
+      const int j = my_lo + my_t, ow = (j >> 2) % nsp, sl = (j >> 2) / nsp;
+      float *dm = (nsp > 1) ? cluster.map_shared_rank(s_pm, ow) : s_pm;
+      float *dl = (nsp > 1) ? cluster.map_shared_rank(s_pl, ow) : s_pl;
+      dm[(part * slots + sl) * 4 + (j & 3)] = s_m[my_g][j];
+      dl[(part * slots + sl) * 4 + (j & 3)] = s_l[my_g][j];
     }
   }
   TC_STAMP(12);
   if (nsp > 1) cluster.sync(); else __syncthreads();
   TC_STAMP(13);
-  constexpr int TPR = kTcDh / 4;                             // threads per column
-  if (tid < 2 * kTcWg) {
-    const int c4 = (tid % TPR) * 4, sub = tid / TPR;         // 8 columns per pass
-    for (int sl = sub; rank + sl * nsp < ncols; sl += 2 * kTcWg / TPR) {
-      const int j = rank + sl * nsp;
-      float M = -INFINITY;
-      for (int sp = 0; sp < nsp; ++sp) M = fmaxf(M, s_pm[sp * slots + sl]);
-      float L = 0.f;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int sp = 0; sp < nsp; ++sp) {
-        const float pm = s_pm[sp * slots + sl];
-        if (pm != -INFINITY) {
-          const float wgt = exp2f(pm - M);
-          const float4 ov = *reinterpret_cast<const float4 *>(sM + (size_t)(sp * slots + sl) * kTcDh + c4);
-          L += wgt * s_pl[sp * slots + sl];
-          acc.x += wgt * ov.x; acc.y += wgt * ov.y; acc.z += wgt * ov.z; acc.w += wgt * ov.w;
+  // owners: warpgroup w takes the received groups w, w + 4, ...; thread t of it dh index t of the group's four columns
+  if (warp < 16) {
+    for (int sl = warp >> 2; rank + sl * nsp < NG && 4 * (rank + sl * nsp) < ncols; sl += 4) {
+      const int j0 = 4 * (rank + sl * nsp);
+      float4 M = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+      for (int sp = 0; sp < nparts; ++sp) {
+        const float4 pm = *reinterpret_cast<const float4 *>(&s_pm[(sp * slots + sl) * 4]);
+        M.x = fmaxf(M.x, pm.x); M.y = fmaxf(M.y, pm.y); M.z = fmaxf(M.z, pm.z); M.w = fmaxf(M.w, pm.w);
+      }
+      float4 L = make_float4(0.f, 0.f, 0.f, 0.f), acc = L;
+      for (int sp = 0; sp < nparts; ++sp) {
+        const float4 pm = *reinterpret_cast<const float4 *>(&s_pm[(sp * slots + sl) * 4]);
+        const float4 pl = *reinterpret_cast<const float4 *>(&s_pl[(sp * slots + sl) * 4]);
+        const float4 ov = sM[(size_t)(sp * slots + sl) * kTcDh + my_t];
+        // a partial without tiles, or a column all of whose positions were masked in it: weight 0
+        const float wx = (pm.x == -INFINITY) ? 0.f : exp2f(pm.x - M.x), wy = (pm.y == -INFINITY) ? 0.f : exp2f(pm.y - M.y);
+        const float wz = (pm.z == -INFINITY) ? 0.f : exp2f(pm.z - M.z), ww = (pm.w == -INFINITY) ? 0.f : exp2f(pm.w - M.w);
+        L.x += wx * pl.x; L.y += wy * pl.y; L.z += wz * pl.z; L.w += ww * pl.w;
+        acc.x += wx * ov.x; acc.y += wy * ov.y; acc.z += wz * ov.z; acc.w += ww * ov.w;
+      }
+      const float val[4] = {acc.x * ((L.x > 0.f) ? 1.f / L.x : 0.f), acc.y * ((L.y > 0.f) ? 1.f / L.y : 0.f),
+                            acc.z * ((L.z > 0.f) ? 1.f / L.z : 0.f), acc.w * ((L.w > 0.f) ? 1.f / L.w : 0.f)};
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        if (j0 + c < ncols) {
+          const bf16 hv = __float2bfloat16_rn(val[c]);
+          const size_t idx = (size_t)s_oidx[j0 + c] + my_t;
+          a.o[idx] = hv;
+          a.o[a.o_lo_off + idx] = __float2bfloat16_rn(val[c] - __bfloat162float(hv));
         }
       }
-      const float inv = (L > 0.f) ? 1.f / L : 0.f;
-      const float val[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
-      const __nv_bfloat162 h01 = __floats2bfloat162_rn(val[0], val[1]), h23 = __floats2bfloat162_rn(val[2], val[3]);
-      const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
-      const __nv_bfloat162 l01 = __floats2bfloat162_rn(val[0] - f01.x, val[1] - f01.y);
-      const __nv_bfloat162 l23 = __floats2bfloat162_rn(val[2] - f23.x, val[3] - f23.y);
-      const size_t idx = (size_t)s_oidx[j] + c4;
-      *reinterpret_cast<uint2 *>(a.o + idx) =
-          make_uint2(*reinterpret_cast<const uint32_t *>(&h01), *reinterpret_cast<const uint32_t *>(&h23));
-      *reinterpret_cast<uint2 *>(a.o + a.o_lo_off + idx) =
-          make_uint2(*reinterpret_cast<const uint32_t *>(&l01), *reinterpret_cast<const uint32_t *>(&l23));
     }
   }
   TC_STAMP(14);

@@ -369,6 +369,8 @@ def test_dh128_grouped_queries_batch_and_pages(torch_cuda, c1, Hkv, tensor_core)
     weights = si.all_weights(shape, gains=True)
     parents = si.tree_template(32)
     eng, orc = make_pair(shape, weights, 512, max_batch=3, max_tree=32, max_k=3, max_depth=3)
+    from paper_2410_20488_b200 import binding
+    assert binding.load_library().firp_set_attention_kernel(eng.ctx, 2) == binding.FIRP_ERR_BAD_ARG
     eng.set_attention_kernel(tensor_core)
     prompts = [si.prompt(shape, seq=0, length=300), si.prompt(shape, seq=1, length=7), si.prompt(shape, seq=2, length=129)]
     st = lockstep_run_batch(eng, orc, shape, parents, prompts, 4)
