@@ -359,6 +359,21 @@ def test_dh128_tree_sizes_and_contexts(torch_cuda, c1, case, tensor_core):
     eng.close()
 
 
+@pytest.mark.parametrize("tensor_core", [True, False, None])
+def test_dh128_slot_rows_off_the_tile_grid(torch_cuda, c1, tensor_core):
+    """A cache of 300 positions per sequence (no multiple of a 64- or 128-position tile) and the second slot: its rows
+    start in the middle of a tile of the plane, the last tile of the context reaches into rows that are not its own,
+    and the context ends 20 positions below the capacity.  None: the library chooses the kernel."""
+    shape = dh128_shape(c1, 2, 2)
+    weights = si.all_weights(shape, gains=True)
+    parents = si.random_tree(33, 24, 3, 5)
+    eng, orc = make_pair(shape, weights, 300, max_batch=2, max_tree=24, max_k=3, max_depth=3)
+    eng.set_attention_kernel(tensor_core)
+    st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, seq=1, length=241), 3, k=3, l=1, forced_steps=(1,), seq=1)
+    assert st.steps == 3 and eng.context_len(1) <= 300 - 27
+    eng.close()
+
+
 @pytest.mark.parametrize("tensor_core", [True, False])
 @pytest.mark.parametrize("Hkv", [2, 1])
 def test_dh128_grouped_queries_batch_and_pages(torch_cuda, c1, Hkv, tensor_core):
