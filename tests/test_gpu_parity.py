@@ -343,16 +343,18 @@ def dh128_shape(c1, H, Hkv):
 
 
 @pytest.mark.parametrize("tensor_core", [True, False])
-@pytest.mark.parametrize("case", range(6))
+@pytest.mark.parametrize("case", range(7))
 def test_dh128_tree_sizes_and_contexts(torch_cuda, c1, case, tensor_core):
     """Tree sizes that select every query-block width of the tensor-core kernel (16, 32, 48, 80 columns, and two
     blocks at 131 rows), contexts that end just below, on and above a 128-position tile boundary (so that the new
-    rows straddle tiles and the last tile is ragged), one to several tiles per split; gains non-unit."""
-    T, k, n0, steps = ((1, 0, 5, 3), (8, 3, 126, 4), (24, 3, 128, 4), (40, 3, 250, 4), (64, 3, 383, 3), (128, 3, 700, 3))[case]
+    rows straddle tiles and the last tile is ragged), one to several tiles per split, and a context long enough for
+    the largest cluster (8 splits of two tiles); gains non-unit."""
+    T, k, n0, steps = ((1, 0, 5, 3), (8, 3, 126, 4), (24, 3, 128, 4), (40, 3, 250, 4), (64, 3, 383, 3), (128, 3, 700, 3),
+                       (8, 3, 1990, 3))[case]
     shape = dh128_shape(c1, 2, 2)
     weights = si.all_weights(shape, gains=True)
     parents = si.chain_template(1) if T == 1 else si.random_tree(31, T, max(k, 1), case)
-    eng, orc = make_pair(shape, weights, 1024, max_tree=128, max_k=3, max_depth=3)
+    eng, orc = make_pair(shape, weights, max(1024, n0 + 256), max_tree=128, max_k=3, max_depth=3)
     eng.set_attention_kernel(tensor_core)
     st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=n0), steps, k=k, l=1, forced_steps=(1,))
     assert st.steps == steps
