@@ -229,7 +229,7 @@ def firp_set_kv_pages(ctx, page_table, stream: int = 0):
     _check(ctx, load_library().firp_set_kv_pages(ctx, ptr, stream))
 
 
-def firp_set_activation_planes(ctx, qkv=3, o=2, gate_up=2, down=2, lm_head=2):
+def firp_set_activation_planes(ctx, qkv=2, o=2, gate_up=2, down=2, lm_head=2):
     """bf16 planes of the activations per GEMM class (1 = plain bf16; see firp.h)."""
     _check(ctx, load_library().firp_set_activation_planes(ctx, qkv, o, gate_up, down, lm_head))
 
@@ -419,7 +419,7 @@ class FirpEngine:
         firp_set_kv_pages(self.ctx, page_table, self.stream)
         self.page_table = None if page_table is None else np.ascontiguousarray(page_table, np.int32).reshape(self.cfg.max_batch, -1)
 
-    def set_activation_planes(self, qkv=3, o=2, gate_up=2, down=2, lm_head=2):
+    def set_activation_planes(self, qkv=2, o=2, gate_up=2, down=2, lm_head=2):
         firp_set_activation_planes(self.ctx, qkv, o, gate_up, down, lm_head)
 
     def set_attention_planes(self, q_planes=2, p_planes=2):

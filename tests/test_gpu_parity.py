@@ -361,6 +361,34 @@ def test_dh128_tree_sizes_and_contexts(torch_cuda, c1, case, tensor_core):
     eng.close()
 
 
+@pytest.mark.parametrize("tensor_core", [True, False])
+def test_dh128_plane_counts(torch_cuda, c1, tensor_core):
+    """firp_set_attention_planes / firp_set_activation_planes: plain bf16 operands (one plane) run through both
+    attention kernels and every GEMM class, stay inside the bound on this two-layer shape, and deviate more from the
+    oracle than the default (hi, lo) planes do; counts outside 1..2 (1..3 for the QKV projection) are refused."""
+    from paper_2410_20488_b200 import FirpError, binding
+    shape = dh128_shape(c1, 2, 2)
+    weights = si.all_weights(shape, gains=True)
+    parents = si.random_tree(35, 24, 3, 2)
+    dev = {}
+    for planes in (2, 1):
+        eng, orc = make_pair(shape, weights, 512, max_tree=24, max_k=3, max_depth=3)
+        eng.set_attention_kernel(tensor_core)
+        eng.set_attention_planes(planes, planes)
+        eng.set_activation_planes(planes, planes, planes, planes, planes)
+        st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=300), 3, k=3, l=1, check_cache_rows=planes == 2)
+        dev[planes] = st.max_abs
+        for bad in ((0, 2), (2, 3)):
+            with pytest.raises(FirpError) as e:
+                eng.set_attention_planes(*bad)
+            assert e.value.code == binding.FIRP_ERR_BAD_ARG
+        with pytest.raises(FirpError) as e:
+            eng.set_activation_planes(4, 2, 2, 2, 2)
+        assert e.value.code == binding.FIRP_ERR_BAD_ARG
+        eng.close()
+    assert dev[1] > 2 * dev[2], dev
+
+
 @pytest.mark.parametrize("tensor_core", [True, False, None])
 def test_dh128_slot_rows_off_the_tile_grid(torch_cuda, c1, tensor_core):
     """A cache of 300 positions per sequence (no multiple of a 64- or 128-position tile) and the second slot: its rows
