@@ -252,9 +252,10 @@ int firp_set_attention_planes(firp_ctx *ctx, int32_t q_planes, int32_t p_planes)
  * tensor_core = 1: tiles of 128 cached positions as the M dimension of tcgen05 MMAs (S^T = K Q^T, O^T = V^T P^T,
  * accumulators in tensor memory, K/V tiles by TMA, two warpgroups alternating over the tiles); 0: the warp-level
  * mma.sync kernel with 64-position tiles, which is also what head_dim 64 and the persistent kernel always use;
- * -1 (default): chosen per step -- the mma.sync kernel only for steps of about 29 rows or more (7B shape) whose
- * longest context spans fewer than three of the tensor-core kernel's tiles (four when the query columns, rows x
- * heads per kv head, need more than one block of 48), where its lower fixed cost wins.  Both compute the same masked softmax with (hi, lo) bf16 planes of Q
+ * -1 (default): chosen per step -- the mma.sync kernel only for steps of more than 16 query columns (rows x heads
+ * per kv head) and about 29 rows or more (7B shape) whose longest context spans fewer than three of the
+ * tensor-core kernel's tiles (four when the columns need more than one block of 48, eight when several sequences
+ * are stepped together), where its lower fixed cost wins.  Both compute the same masked softmax with (hi, lo) bf16 planes of Q
  * and P and fp32 accumulation; summation orders differ.  Other values: FIRP_ERR_BAD_ARG.
  */
 int firp_set_attention_kernel(firp_ctx *ctx, int32_t tensor_core);

@@ -351,13 +351,17 @@ int run_rows(firp_ctx *c, const RunArgs &ra, cudaStream_t st) {
         int qb_tc, qper_tc;
         attention_tc_blocks(act * G, &qb_tc, &qper_tc);
         const int tiles_tc = (ra.n_hi_max + act + kAttnTcTile - 1) / kAttnTcTile;
-        // Left to itself the tensor-core kernel takes every step the other kernel would not be launched early for,
-        // and otherwise those whose longest context spans at least three of its 128-position tiles (four when the
-        // query columns need more than one block): its fixed cost is higher, its tile loop faster.  Measured at the
-        // 7B shape, one sequence, ms per step mma.sync / tcgen05: 1 column 3.23 / 3.06 at 64 cached tokens, 3.37 /
+        // Left to itself the tensor-core kernel takes every step the other kernel would not be launched early for
+        // and every step of at most 16 query columns; otherwise those whose longest context spans at least three of
+        // its 128-position tiles (four when the query columns need more than one block, eight when several
+        // sequences are stepped together): its fixed cost is higher, its tile loop faster.  Measured at the 7B
+        // shape, ms per step mma.sync / tcgen05, one sequence: 1 column 3.23 / 3.06 at 64 cached tokens, 3.37 /
         // 3.28 at 512, 5.04 / 4.06 at 8192; 35 columns 3.57 / 3.61 at 64, 3.64 / 3.65 at 128, 3.72 / 3.65 at 512,
-        // 5.23 / 4.48 at 8192; 131 columns (three blocks) 5.96 / 5.91 at 64, 6.09 / 6.07 at 256, 10.35 / 9.68 at 8192.
-        tc = c->attn_tc > 0 || !attn_early || tiles_tc >= (qb_tc == 1 ? 3 : 4);
+        // 5.23 / 4.48 at 8192; 131 columns (three blocks) 5.96 / 5.91 at 64, 6.09 / 6.07 at 256, 10.35 / 9.68 at
+        // 8192; 4 sequences x 35 columns 5.77 / 5.88 at 256, 6.78 / 6.36 at 1024, 9.13 / 7.75 at 4096; 16 sequences
+        // x 9 columns 6.77 / 6.56 at 256, 19.41 / 12.13 at 4096.
+        const int min_tiles = qper_tc <= 16 ? 1 : (rw.n_seq > 1 ? 8 : (qb_tc == 1 ? 3 : 4));
+        tc = c->attn_tc > 0 || !attn_early || tiles_tc >= min_tiles;
         if (tc) a.splits = attention_tc_splits(rw.n_seq * Hkv * qb_tc, tiles_tc, c->sm_count);
       }
       FIRP_TIMED(KC_ATTENTION);
