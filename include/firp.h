@@ -77,7 +77,8 @@ typedef struct {
 /* Caller-owned DEVICE output buffers of one step; S = max_depth + 1, B = top_b.
  * Any pointer may be NULL (that result is then kept internal or not produced). */
 typedef struct {
-  int32_t *accepted_tokens;   /* [n_seq][S]  tokens emitted: accepted drafts, then the bonus token */
+  int32_t *accepted_tokens;   /* [n_seq][S]  tokens emitted: accepted drafts, then the bonus token; only the first
+                                 n_accepted entries of a row are written */
   int32_t *n_accepted;        /* [n_seq]     a + 1 */
   int32_t *path;              /* [n_seq][S]  accepted row indices, path[0] = 0: the KV compaction indices */
   int32_t *next_tree_tokens;  /* [n_seq][T_next] tokens of the next draft tree on the template */

@@ -361,6 +361,41 @@ def test_dh128_tree_sizes_and_contexts(torch_cuda, c1, case, tensor_core):
     eng.close()
 
 
+def test_dh128_free_running_decode_repeats_bit_for_bit(torch_cuda, c1):
+    """400 free-running steps (device-side commits) on the tensor-core attention, twice from the same state: the
+    context grows across tile boundaries and split counts, and every accepted token and every next tree must
+    repeat exactly (the kernel's barriers, buffers and merge order leave nothing to timing)."""
+    import hashlib
+    import torch
+    from paper_2410_20488_b200 import FirpEngine
+    shape = dh128_shape(c1, 4, 2)
+    weights = si.all_weights(shape, gains=True)
+    T, k = 16, 3
+    parents = si.random_tree(37, T, 3, 3)
+    eng = FirpEngine(shape, weights, max_ctx=2048, max_tree=T, max_k=k, max_depth=3)
+    eng.set_attention_kernel(True)
+    out = eng.new_out(1, T, k, want_logits=False)
+    digests = []
+    for rep in range(2):
+        eng.set_context_len(0, 90)
+        cur = torch.from_numpy(si.random_tokens(shape, T, 3)).cuda().reshape(1, T)
+        seen = []
+        for _ in range(400):
+            eng.step(cur, parents, k, 1, out)
+            eng.commit(1)
+            seen.append(out.n_accepted.clone())          # accepted_tokens holds n_accepted valid entries: compared through
+            seen.append(out.best.clone())                # the verification argmax of every row and the next tree instead
+            cur = out.next_tree_tokens.clone()
+            seen.append(cur)
+        torch.cuda.synchronize()
+        h = hashlib.sha256()
+        for t in seen:
+            h.update(t.cpu().numpy().tobytes())
+        digests.append((h.hexdigest(), eng.context_len(0)))
+    assert digests[0] == digests[1] and digests[0][1] >= 490
+    eng.close()
+
+
 @pytest.mark.parametrize("tensor_core", [True, False])
 def test_dh128_plane_counts(torch_cuda, c1, tensor_core):
     """firp_set_attention_planes / firp_set_activation_planes: plain bf16 operands (one plane) run through both
