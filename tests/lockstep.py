@@ -297,8 +297,8 @@ def lockstep_steps(engine, orc, shape, parents, tokens, steps, forced=False, k=N
     T = len(parents)
     tp = oracle.tree_prep_chains(parents, k) if chains else oracle.tree_prep(parents, k, 0)
     tp_tree = oracle.tree_prep(parents, 0, 0)
-    D = int(tp_tree["depth"].max())
     chain = principal_chain(parents, tp_tree["depth"])
+    D = len(chain) - 1        # forced steps plant the greedy continuation on the principal chain (which may end above the deepest node)
     dev = engine.device
     stats = Stats()
     tokens = np.array(tokens, np.int32)

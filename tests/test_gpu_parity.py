@@ -361,6 +361,50 @@ def test_dh128_tree_sizes_and_contexts(torch_cuda, c1, case, tensor_core):
     eng.close()
 
 
+@pytest.mark.parametrize("seed", [1, 2])
+def test_dh128_random_shapes_in_lockstep(torch_cuda, c1, seed):
+    """Twelve seeded random cases per seed at head dimension 128: heads per kv head 1 / 2 / 4 / 8, tree sizes 1..64
+    (every query-block width, one to three blocks), one to three sequences of unrelated context lengths (1..700,
+    i.e. any number of tiles and a ragged last one), contiguous or paged cache, the tensor-core kernel forced or the
+    library's own choice; three steps each (one forced-accept for single sequences) against the oracle."""
+    from lockstep import lockstep_run_batch
+    rng = np.random.default_rng(seed)
+    done = 0
+    while done < 12:
+        H, Hkv = [(2, 2), (4, 2), (4, 1), (8, 1), (4, 4)][rng.integers(5)]
+        T = int(rng.choice([1, 2, 5, 8, 13, 16, 17, 24, 29, 33, 40, 47, 64]))
+        k = 0 if T == 1 else (3 if T > 40 else int(rng.integers(2 if T > 9 else 1, 4)))
+        n_seq = int(rng.choice([1, 1, 2, 3]))
+        if n_seq * (T + k) > 144:
+            n_seq = 1
+        lengths = [int(rng.integers(1, 700)) for _ in range(n_seq)]
+        tensor_core = [True, None][rng.integers(2)]
+        paged = bool(rng.integers(2)) and n_seq > 1
+        shape = si.scaled(dh128_shape(c1, H, Hkv), seed=int(rng.integers(1000)))
+        try:
+            parents = si.chain_template(1) if T == 1 else si.random_tree(int(rng.integers(1000)), T, max(k, 1), done)
+        except ValueError:
+            continue                                           # no such tree under that depth
+        weights = si.all_weights(shape, gains=True)
+        eng, orc = make_pair(shape, weights, 1024, max_batch=n_seq, max_tree=T, max_k=max(k, 1), max_depth=3)
+        eng.set_attention_kernel(tensor_core)
+        if paged:
+            eng.set_kv_pages(rng.permutation(n_seq * 1024 // 64).astype(np.int32).reshape(n_seq, -1))
+        case = "H=%d Hkv=%d T=%d k=%d lengths=%s tensor_core=%s paged=%s" % (H, Hkv, T, k, lengths, tensor_core, paged)
+        try:
+            if n_seq == 1:
+                st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=lengths[0]), 3, k=k,
+                                  l=int(rng.integers(0, 2)), forced_steps=(1,))
+            else:
+                st = lockstep_run_batch(eng, orc, shape, parents,
+                                        [si.prompt(shape, seq=s_i, length=lengths[s_i]) for s_i in range(n_seq)], 3, k=k, l=1)
+        except AssertionError as e:
+            raise AssertionError("%s: %s" % (case, e))
+        assert st.steps == 3 * n_seq, case
+        eng.close()
+        done += 1
+
+
 def test_dh128_free_running_decode_repeats_bit_for_bit(torch_cuda, c1):
     """400 free-running steps (device-side commits) on the tensor-core attention, twice from the same state: the
     context grows across tile boundaries and split counts, and every accepted token and every next tree must
