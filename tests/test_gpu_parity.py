@@ -361,6 +361,36 @@ def test_dh128_tree_sizes_and_contexts(torch_cuda, c1, case, tensor_core):
     eng.close()
 
 
+@pytest.mark.parametrize("tensor_core", [True, False])
+@pytest.mark.parametrize("case", range(3))
+def test_dh128_chains_layers_and_masked_rows(torch_cuda, c1, case, tensor_core):
+    """The variants of the step at head dimension 128, on both attention kernels: a chain of pseudo rows under every
+    node (firp_step_chains: 36 x 4 = 144 rows, three query blocks, per-step insertion layers), one insertion layer
+    per prediction step (firp_step_layers), and the "Masked" ablation (pseudo rows do not see each other); four
+    layers deep, contexts that put the new rows across a tile boundary, greedy and forced."""
+    shape = si.scaled(dh128_shape(c1, 4, 2), L=4, l=1)
+    weights = si.all_weights(shape, gains=True)
+    for forced in (False, True):
+        if case == 0:
+            T, k, layers = 36, 3, [1, 2, 2]
+            parents = si.random_tree(9, T, k, 3)
+            eng, orc = make_pair(shape, weights, 512, max_tree=64, max_k=3, max_depth=3, max_rows=T * (1 + k))
+            eng.set_attention_kernel(tensor_core)
+            st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=131), 3, forced=forced, k=k, l=layers, chains=True)
+        elif case == 1:
+            parents = si.random_tree(5, 19, 3, 6)
+            eng, orc = make_pair(shape, weights, 512, max_tree=32, max_k=3, max_depth=3)
+            eng.set_attention_kernel(tensor_core)
+            st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=250), 3, forced=forced, k=3, l=[0, 1, 3])
+        else:
+            parents = si.tree_template(32)
+            eng, orc = make_pair(shape, weights, 512, masked=True, max_tree=32, max_k=3, max_depth=3)
+            eng.set_attention_kernel(tensor_core)
+            st = lockstep_run(eng, orc, shape, parents, si.prompt(shape, length=120), 3, forced=forced, k=3, l=1)
+        assert st.steps == 3
+        eng.close()
+
+
 @pytest.mark.parametrize("seed", [1, 2])
 def test_dh128_random_shapes_in_lockstep(torch_cuda, c1, seed):
     """Twelve seeded random cases per seed at head dimension 128: heads per kv head 1 / 2 / 4 / 8, tree sizes 1..64
