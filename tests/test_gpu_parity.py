@@ -295,15 +295,16 @@ def test_c1_paged_cache(torch_cuda, c1, fused):
     eng.close()
 
 
+@pytest.mark.parametrize("head_dim", [64, 128])
 @pytest.mark.parametrize("fused", [False, True])
-def test_c1_a_tree_of_its_own_for_every_sequence(torch_cuda, c1, fused):
+def test_c1_a_tree_of_its_own_for_every_sequence(torch_cuda, c1, fused, head_dim):
     """firp_step_trees: three sequences stepped together, each with its own tree shape and size (8, 5 and 3 of the
     T = 8 rows), its own context length; every sequence is compared with an oracle step on ITS tree (the padding
     rows dropped), both sides commit the oracle's path and take the oracle's next tree on the sequence's own shape.
     A token that would be accepted is planted in a padding row: it must not be."""
     import torch
     from lockstep import own_tree_view
-    shape = si.scaled(c1, Hkv=2)
+    shape = si.scaled(c1, Hkv=2) if head_dim == 64 else dh128_shape(c1, 4, 2)      # 128: the tensor-core attention
     weights = si.all_weights(shape, gains=True)
     T, k, l = 8, 3, 1
     trees = [si.tree_template(8), si.random_tree(8, 5, 3, 1), si.chain_template(3)]
